@@ -1,0 +1,195 @@
+/* libsop -- C-ABI boundary of the B200 (sm_100a) implementation of the Scaled Outer Product
+ * per-layer candidate sweep.
+ *
+ * One linear layer at a time: W is M x K bf16 (row-major, K contiguous, leading dimension ldw),
+ * calibration activations X are T x K fp32, blocks are g = 16 consecutive elements along K
+ * (paper Section "Block Scaling": Y = X W^T, scales shared along the contracted dimension K).
+ *
+ * Conventions for every entry point
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; pointers without the suffix
+ *     are HOST pointers read before the call returns.  The library never frees caller memory and
+ *     allocates nothing that outlives a call; scratch comes from a caller-provided device
+ *     workspace whose size the matching *_workspace() query reports.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     Outputs are valid after the stream has been synchronised.
+ *   - Return value: SOP_OK (0) or a negative SOP_ERR_* code; nothing throws, aborts or traps.
+ *     Argument errors are detected on the host before anything is launched.
+ *   - Required: K % 16 == 0, M, K, T >= 1, ldw >= K, ldx >= K, M*K < 2^31 blocks*16, finite inputs.
+ */
+#ifndef SOP_H_
+#define SOP_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SOP_G 16               /* block size along K */
+#define SOP_MAX_ATOMS 16       /* candidates per call, negations and FP formats included */
+#define SOP_MAX_ENTRIES 32     /* table entries per LUT atom (n <= 5) */
+#define SOP_K_AUTO (-1000)     /* k_mode: choose the F_layer shift on the device */
+#define SOP_K_FROM_RESULT (-1001) /* k_mode of sop_dd4_lloyd: take the shift from a previous search */
+#define SOP_FMTA_FROM_RESULT (-1) /* fmta_index of sop_dd4_lloyd: best single LUT candidate of a previous search */
+
+enum {
+  SOP_OK = 0,
+  SOP_ERR_NULL = -1,       /* a required pointer is NULL */
+  SOP_ERR_SHAPE = -2,      /* M, K, T <= 0, K % 16 != 0, ld < K, g != 16, size beyond the supported range */
+  SOP_ERR_FORMAT = -3,     /* bad scale format, or a sign / selector bit requested that the word does not have */
+  SOP_ERR_ALPHABET = -4,   /* bad atom: n_entries, unsorted or non-finite table, tmax <= 0, too many atoms */
+  SOP_ERR_WORKSPACE = -5,  /* workspace NULL, misaligned (256 B) or too small */
+  SOP_ERR_CUDA = -6,       /* a CUDA runtime call failed; see sop_last_cuda_error() */
+  SOP_ERR_RANGE = -7       /* k shift outside [-64, 64], pool_rank outside [1, N_b], iters outside [0, 64] */
+};
+
+enum { SOP_KIND_LUT = 0, SOP_KIND_FP_E2M3 = 1, SOP_KIND_FP_E4M3 = 2 };
+
+/* Scale word magnitude format ExMy with optional sign (Section "Scale Format and Metabit
+ * Allocation", SwExMy).  bias is 2^(x-1)-1 in every format the paper names.  Rounding is to
+ * nearest even with gradual underflow; all exponent codes are finite unless top_exp_reserved;
+ * overflow saturates; a positive scale never rounds to zero. */
+typedef struct {
+  int sign_bits;         /* w: 1 if the deployed word has a sign bit (enables the 4-way signed table) */
+  int exp_bits;          /* x in [1, 8] */
+  int man_bits;          /* y in [0, 10] */
+  int bias;
+  int top_exp_reserved;  /* 1: the all-ones exponent code is not used (needed for E8M7) */
+} sop_scale_fmt;
+
+/* One candidate codebook ("atom", Section "Per-Layer Pair Search").
+ * LUT kind: lut[0..n_entries) ascending (repeats allowed), n_entries <= 2^n_bits <= 32.
+ * negated = 1 makes the candidate -(lut): it is evaluated by running the table on -u, so that
+ * code_{-a}(-w) == code_a(w) exactly, ties included.
+ * FP kinds (E2M3: 6-bit, largest 7.5; E4M3: 8-bit OCP, largest 448) ignore lut.
+ * scope = 16: per-block scale in the layer's scale format, s = max|w_block| / tmax
+ * ("LUT-scale coupling": the scale is taken against max(LUT)).
+ * scope = 0: one power-of-two scale per layer, 2^ceil(log2(max|W| / tmax)) (the "^0" suffix). */
+typedef struct {
+  int n_bits;
+  int kind;
+  int negated;
+  int scope;
+  float tmax;
+  int n_entries;
+  float lut[SOP_MAX_ENTRIES];
+} sop_atom;
+
+/* Per-layer statistics of one candidate or one candidate pair. */
+typedef struct {
+  double acos;       /* mean over blocks of the selected c-weighted block cosine (Section "ACos") */
+  double mse;        /* sum over blocks of the selected squared error / (M K) */
+  long long n_sel1;  /* blocks whose selector bit is 1 (second codebook); -1 marks an undefined entry */
+  long long n_neg;   /* signed table only: blocks whose scale sign is negative */
+} sop_pair_stat;
+
+/* Device-resident result block of sop_pair_search (read it back with cudaMemcpy). */
+typedef struct {
+  int k[SOP_MAX_ATOMS];  /* F_layer shift used for each candidate (0 for scope-0 candidates) */
+  int best_a, best_b;    /* best two-codebook pair a < b by ACos, ties to the smallest (a, b); -1 if none */
+  int best_single;       /* best single LUT candidate by ACos, ties to the lowest index; -1 if none */
+  int best_sa, best_sb;  /* best pair of the signed table; -1 if none */
+  float layer_absmax;    /* max |W| */
+  int reserved[2];
+} sop_search_result;
+
+const char* sop_strerror(int code);
+/* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
+const char* sop_last_cuda_error(void);
+int sop_version(void);
+
+/* ---- channel norms:  c_k = sqrt((1/T) sum_t X[t,k]^2)   (Section "Channel Norms") ----------
+ * X_dev: T x K fp32, row stride ldx.  c_dev: K fp32.  Accumulation in FP64; order: chunks of 64
+ * rows, sequential fused multiply-add inside a chunk, chunk partials added in chunk order, so the
+ * result is bit-reproducible.  Workspace: ceil(T/64) * K doubles. */
+int sop_channel_norms_workspace(long long T, long long K, size_t* bytes);
+int sop_channel_norms(const float* X_dev, long long T, long long K, long long ldx, float* c_dev,
+                      void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---- the candidate sweep (Sections "Block Scaling", "ACos", "Per-Layer Pair Search" step 4,
+ *      "Per-layer scale shift") ----------------------------------------------------------------
+ * For every block and every candidate: scale = Q_fmt(absmax / tmax * 2^k) * 2^-k, codes = nearest
+ * table entry (or nearest-even FP grid value) of w * (1 / scale), c-weighted block cosine and
+ * squared error in fp32 with a fixed summation order; then per layer, in FP64:
+ *   pair_table_dev [n_atoms x n_atoms]: [a][a] = candidate a alone; [a][b], a < b, both LUT atoms of
+ *     equal n_bits = two-codebook quantisation with per-block selector [cos_b > cos_a];
+ *     other entries are marked n_sel1 = -1.
+ *   signed_table_dev [n_atoms x n_atoms] (may be NULL; filled only when fmt->sign_bits = 1): for
+ *     base atoms i <= j, each immediately followed in `atoms` by its own negation, the per-block
+ *     best of {i, -i, j, -j}, ties resolved in that order.
+ *   result_dev: shifts, best pair, best single.
+ *   block_cos_dev / block_sse_dev (may be NULL): [n_atoms x N_b] per-block values, N_b = M*K/16,
+ *     block index = m * (K/16) + j.
+ * k_mode: SOP_K_AUTO runs the F_layer search per distinct tmax (maximise the number of blocks whose
+ *   shifted scale exponent lies in the format's normal range, k in [-64, 64], ties to the smallest
+ *   |k| then to k > 0); any other value in [-64, 64] is used as the shift for every candidate.
+ * dd_lut_dev (may be NULL): device table of SOP_MAX_ENTRIES floats that replaces, at kernel time,
+ *   the lut of every atom whose index bit is set in dd_mask (a codebook produced by sop_dd4_lloyd
+ *   can be swept without a host round trip). */
+int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes);
+int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+                    const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
+                    const float* dd_lut_dev, unsigned dd_mask,
+                    sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
+                    sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
+                    void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Measurement aid (no counterpart in the paper): with profiling enabled, sop_pair_search records a
+ * CUDA event on `stream` directly before and after its sweep kernel; sop_profile_last_sweep_ms
+ * waits for the second event and returns that one launch's duration in milliseconds
+ * (SOP_ERR_RANGE if no sweep has run since profiling was enabled).  Not thread-safe. */
+int sop_profile_enable(int on);
+int sop_profile_last_sweep_ms(float* ms);
+
+/* ---- DD-n: per-layer data-derived codebook by Lloyd iteration (pair-search steps 2-3) -------
+ * Pool = blocks whose cosine under the primary codebook FMTa is <= the pool_rank-th smallest of
+ * the layer (ties all in).  Each iteration assigns every pool element u = w / scale (scale against
+ * tmax = 1) to its nearest entry, accumulates per entry sum(omega) and sum(omega u) with
+ * omega = c / max(c) in int64 fixed point (2^-24 units, |omega u| clamped to 256), replaces each
+ * non-empty entry by its centroid snapped to bf16, and re-sorts.
+ *   fmta_index: index into `atoms` of FMTa (its table is the initial codebook), or
+ *     SOP_FMTA_FROM_RESULT to use search_dev->best_single.
+ *   block_cos_dev: [n_atoms x N_b] as written by sop_pair_search (row fmta is read).
+ *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
+ *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
+ *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
+ *   pool_count_dev: one long long, number of blocks in the pool. */
+int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
+int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+                  const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
+                  const float* block_cos_dev, long long pool_rank, const sop_atom* atoms, int n_atoms,
+                  int fmta_index, int iters, float* out_lut_dev, double* distortion_dev,
+                  long long* pool_count_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---- materialise: codes + scale words for the chosen codebook(s) (Section "Overview" item 4:
+ *      2n bytes of codes per block; Section "Scale Format": bit placement) ---------------------
+ * Candidates per block in priority order a, (-a if use_sign), b, (-b if use_sign); the largest
+ * block cosine wins, ties keep the earlier.  selector = winner is b or -b; sign = winner is a
+ * negated variant.
+ *   atoms / n_atoms / dd_lut_dev / dd_mask: the alphabet, as for sop_pair_search.
+ *   index_a, index_b: indices into `atoms`; index_b = SOP_NO_ATOM packs a single codebook;
+ *     index_a = SOP_PAIR_FROM_RESULT takes the pair from search_dev (best_sa/best_sb when use_sign,
+ *     else best_a/best_b) so that the whole layer pipeline runs without a host round trip.
+ *   k_mode: a shift in [-64, 64] used for both atoms, or SOP_K_FROM_RESULT (search_dev->k[index]).
+ *   codes_dev: N_b * 2n bytes; block payload = one little-endian 16n-bit integer, element r in bits
+ *     [r n, r n + n).  LUT atoms: table index (for a negated table: the index found on -u);
+ *     FP atoms: the format's bit pattern sign|E|M.
+ *   words_dev: ceil(N_b * container_bits / 8) bytes, rounded up to a multiple of 4 (the stream is
+ *     written with 32-bit operations; the pointer must be 4-byte aligned), little-endian bit stream
+ *     of b-bit words in block order (b = 12: two words per three bytes; b in {8, 12, 16}).  Word layout:
+ *     word_sign_bits = 1: sign at bit b-1, selector at bit 0, magnitude E:M above the
+ *     m = b-1-x-y metabits; word_sign_bits = 0: selector at bit b-1 (if m >= 1), magnitude above
+ *     the remaining m-1 metabits.  Unused metabits are zero.
+ *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten. */
+#define SOP_NO_ATOM (-2)
+#define SOP_PAIR_FROM_RESULT (-1)
+int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+             const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
+             unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
+             int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
+             unsigned char* words_dev, long long* counts_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOP_H_ */

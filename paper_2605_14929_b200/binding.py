@@ -1,0 +1,220 @@
+"""ctypes binding of ``libsop.so``: the same entry points as ``include/sop.h``, with torch tensors
+supplying device memory and streams.  Argument marshalling only -- every step of the sweep runs in
+the library's CUDA kernels.  There is no CPU fallback: a missing library is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+K_AUTO = -1000
+K_FROM_RESULT = -1001
+FMTA_FROM_RESULT = -1
+PAIR_FROM_RESULT = -1
+NO_ATOM = -2
+MAX_ATOMS = 16
+MAX_ENTRIES = 32
+
+
+class SopError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().sop_strerror(code).decode()
+        if code == -6:
+            msg += ": " + lib().sop_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+class ScaleFmt(C.Structure):
+    _fields_ = [("sign_bits", C.c_int), ("exp_bits", C.c_int), ("man_bits", C.c_int), ("bias", C.c_int),
+                ("top_exp_reserved", C.c_int)]
+
+
+class AtomStruct(C.Structure):
+    _fields_ = [("n_bits", C.c_int), ("kind", C.c_int), ("negated", C.c_int), ("scope", C.c_int),
+                ("tmax", C.c_float), ("n_entries", C.c_int), ("lut", C.c_float * MAX_ENTRIES)]
+
+
+class PairStat(C.Structure):
+    _fields_ = [("acos", C.c_double), ("mse", C.c_double), ("n_sel1", C.c_longlong), ("n_neg", C.c_longlong)]
+
+
+class SearchResult(C.Structure):
+    _fields_ = [("k", C.c_int * MAX_ATOMS), ("best_a", C.c_int), ("best_b", C.c_int), ("best_single", C.c_int),
+                ("best_sa", C.c_int), ("best_sb", C.c_int), ("layer_absmax", C.c_float), ("reserved", C.c_int * 2)]
+
+
+PAIR_DTYPE = np.dtype([("acos", "f8"), ("mse", "f8"), ("n_sel1", "i8"), ("n_neg", "i8")])
+RESULT_BYTES = C.sizeof(SearchResult)
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """The loaded C-ABI library.  Built in-tree by ``build.py``; never silently replaced."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_build.LIB):
+            raise ImportError(f"{_build.LIB} is missing: run `python -m paper_2605_14929_b200.build` "
+                              "(nvcc, sm_100a).  There is no CPU fallback.")
+        _lib = C.CDLL(_build.LIB)
+        _lib.sop_strerror.restype = C.c_char_p
+        _lib.sop_last_cuda_error.restype = C.c_char_p
+    return _lib
+
+
+def exported_symbols():
+    return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
+            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd", "sop_pack",
+            "sop_profile_enable", "sop_profile_last_sweep_ms"]
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise SopError(rc, where)
+
+
+def make_fmt(f) -> ScaleFmt:
+    return ScaleFmt(f.sign_bits, f.exp_bits, f.man_bits, f.bias, f.top_exp_reserved)
+
+
+def make_atoms(atoms: Sequence) -> C.Array:
+    arr = (AtomStruct * max(1, len(atoms)))()
+    for i, a in enumerate(atoms):
+        s = arr[i]
+        s.n_bits, s.kind, s.negated, s.scope, s.tmax = a.n_bits, a.kind, a.negated, a.scope, a.tmax
+        s.n_entries = 0 if a.lut is None else len(a.lut)
+        if a.lut is not None:
+            for j, v in enumerate(a.lut):
+                s.lut[j] = float(v)
+    return arr
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _ll(v) -> C.c_longlong:
+    return C.c_longlong(int(v))
+
+
+# ------------------------------------------------------------------ workspace queries
+def channel_norms_workspace(T: int, K: int) -> int:
+    n = C.c_size_t()
+    _check(lib().sop_channel_norms_workspace(_ll(T), _ll(K), C.byref(n)), "sop_channel_norms_workspace")
+    return n.value
+
+
+def pair_search_workspace(M: int, K: int, n_atoms: int) -> int:
+    n = C.c_size_t()
+    _check(lib().sop_pair_search_workspace(_ll(M), _ll(K), n_atoms, C.byref(n)), "sop_pair_search_workspace")
+    return n.value
+
+
+def dd4_lloyd_workspace(M: int, K: int) -> int:
+    n = C.c_size_t()
+    _check(lib().sop_dd4_lloyd_workspace(_ll(M), _ll(K), C.byref(n)), "sop_dd4_lloyd_workspace")
+    return n.value
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """A 256-byte aligned device buffer (torch's caching allocator aligns to 512 bytes)."""
+    return torch.empty(max(256, nbytes), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------ entry points
+def sop_channel_norms(X: torch.Tensor, c_out: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    assert X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    assert c_out.is_cuda and c_out.dtype == torch.float32 and c_out.is_contiguous()
+    T, K = X.shape
+    _check(lib().sop_channel_norms(_ptr(X), _ll(T), _ll(K), _ll(X.stride(0)), _ptr(c_out), _ptr(workspace),
+                                   C.c_size_t(workspace.numel()), _stream(stream)), "sop_channel_norms")
+
+
+def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair_table: torch.Tensor,
+                    signed_table: Optional[torch.Tensor], result: torch.Tensor, workspace: torch.Tensor,
+                    k_mode: int = K_AUTO, dd_lut: Optional[torch.Tensor] = None, dd_mask: int = 0,
+                    block_cos: Optional[torch.Tensor] = None, block_sse: Optional[torch.Tensor] = None,
+                    stream=None, g: int = 16) -> None:
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    M, K = W.shape
+    _check(lib().sop_pair_search(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
+                                 make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), _ptr(pair_table),
+                                 _ptr(signed_table), _ptr(result), _ptr(block_cos), _ptr(block_sse), _ptr(workspace),
+                                 C.c_size_t(workspace.numel()), _stream(stream)), "sop_pair_search")
+
+
+def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_cos: torch.Tensor, pool_rank: int,
+                  iters: int, out_lut: torch.Tensor, distortion: torch.Tensor, pool_count: torch.Tensor,
+                  workspace: torch.Tensor, k_mode: int = K_FROM_RESULT, search_result: Optional[torch.Tensor] = None,
+                  fmta_index: int = FMTA_FROM_RESULT, stream=None, g: int = 16) -> None:
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    M, K = W.shape
+    _check(lib().sop_dd4_lloyd(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
+                               _ptr(search_result), _ptr(block_cos), _ll(pool_rank), make_atoms(atoms), len(atoms),
+                               fmta_index, iters, _ptr(out_lut), _ptr(distortion), _ptr(pool_count), _ptr(workspace),
+                               C.c_size_t(workspace.numel()), _stream(stream)), "sop_dd4_lloyd")
+
+
+def sop_pack(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes: torch.Tensor, words: torch.Tensor,
+             index_a: int = PAIR_FROM_RESULT, index_b: int = PAIR_FROM_RESULT, k_mode: int = K_FROM_RESULT,
+             search_result: Optional[torch.Tensor] = None, use_sign: int = 0, container_bits: int = 8,
+             word_sign_bits: int = 0, counts: Optional[torch.Tensor] = None, dd_lut: Optional[torch.Tensor] = None,
+             dd_mask: int = 0, stream=None, g: int = 16) -> None:
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    M, K = W.shape
+    _check(lib().sop_pack(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)),
+                          make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), index_a, index_b, k_mode,
+                          _ptr(search_result), use_sign, container_bits, word_sign_bits, _ptr(codes), _ptr(words),
+                          _ptr(counts), _stream(stream)), "sop_pack")
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib().sop_profile_enable(1 if on else 0), "sop_profile_enable")
+
+
+def profile_last_sweep_ms() -> float:
+    ms = C.c_float()
+    _check(lib().sop_profile_last_sweep_ms(C.byref(ms)), "sop_profile_last_sweep_ms")
+    return ms.value
+
+
+# ------------------------------------------------------------------ result readers (device -> host)
+def read_pair_table(t: torch.Tensor, n_atoms: int) -> np.ndarray:
+    return t.cpu().numpy().view(PAIR_DTYPE).reshape(n_atoms, n_atoms)
+
+
+def read_result(t: torch.Tensor) -> dict:
+    raw = t.cpu().numpy().tobytes()
+    r = SearchResult.from_buffer_copy(raw)
+    return dict(k=np.array(r.k[:], dtype=np.int32), best=np.array([r.best_a, r.best_b, r.best_single, r.best_sa, r.best_sb],
+                                                               dtype=np.int32), layer_absmax=r.layer_absmax)
+
+
+def new_pair_table(n_atoms: int, device) -> torch.Tensor:
+    return torch.zeros(n_atoms * n_atoms * PAIR_DTYPE.itemsize, dtype=torch.uint8, device=device)
+
+
+def new_result(device) -> torch.Tensor:
+    return torch.zeros(RESULT_BYTES, dtype=torch.uint8, device=device)
+
+
+def words_nbytes(n_blocks: int, container_bits: int) -> int:
+    """Bytes to allocate for the scale-word stream (whole 32-bit words)."""
+    return ((n_blocks * container_bits + 7) // 8 + 3) // 4 * 4

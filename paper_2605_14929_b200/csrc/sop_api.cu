@@ -1,0 +1,165 @@
+// Host-side argument validation, error text and the channel-norm kernels of libsop.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "sop_device.cuh"
+
+namespace sop {
+
+static thread_local char g_cuda_error[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
+}
+
+int validate_fmt(const sop_scale_fmt* f, FmtDev* out) {
+  if (!f) return SOP_ERR_NULL;
+  if (f->exp_bits < 1 || f->exp_bits > 8 || f->man_bits < 0 || f->man_bits > 10) return SOP_ERR_FORMAT;
+  if (f->sign_bits < 0 || f->sign_bits > 1 || f->top_exp_reserved < 0 || f->top_exp_reserved > 1) return SOP_ERR_FORMAT;
+  if (f->bias < 0 || f->bias > 127) return SOP_ERR_FORMAT;
+  const int top = (1 << f->exp_bits) - 1 - f->top_exp_reserved;
+  if (top < 1) return SOP_ERR_FORMAT;
+  out->y = f->man_bits;
+  out->bias = f->bias;
+  out->emin = 1 - f->bias;
+  out->emax = top - f->bias;
+  if (out->emax > 127) return SOP_ERR_FORMAT;  // largest scale must stay finite in fp32
+  out->code_max = (top << f->man_bits) | ((1 << f->man_bits) - 1);
+  out->sign_bits = f->sign_bits;
+  return SOP_OK;
+}
+
+int validate_atoms(const sop_atom* atoms, int n_atoms, unsigned dd_mask, const float* dd_lut, AtomsDev* out) {
+  if (!atoms) return SOP_ERR_NULL;
+  if (n_atoms < 1 || n_atoms > SOP_MAX_ATOMS) return SOP_ERR_ALPHABET;
+  if (dd_mask && !dd_lut) return SOP_ERR_NULL;
+  if (n_atoms < 32 && (dd_mask >> n_atoms)) return SOP_ERR_ALPHABET;
+  memset(out, 0, sizeof(*out));
+  out->n_atoms = n_atoms;
+  out->dd_mask = dd_mask;
+  out->dd_lut = dd_lut;
+  for (int i = 0; i < n_atoms; ++i) {
+    const sop_atom& a = atoms[i];
+    if (!(a.tmax > 0.0f) || !isfinite(a.tmax)) return SOP_ERR_ALPHABET;
+    if (a.scope != 0 && a.scope != SOP_G) return SOP_ERR_ALPHABET;
+    if (a.negated != 0 && a.negated != 1) return SOP_ERR_ALPHABET;
+    if (a.kind == SOP_KIND_LUT) {
+      if (a.scope != SOP_G) return SOP_ERR_ALPHABET;
+      if (a.n_bits < 1 || a.n_bits > 5) return SOP_ERR_ALPHABET;
+      if (a.n_entries < 2 || a.n_entries > (1 << a.n_bits)) return SOP_ERR_ALPHABET;
+      if (!((dd_mask >> i) & 1u)) {
+        for (int j = 0; j < a.n_entries; ++j) {
+          if (!isfinite(a.lut[j])) return SOP_ERR_ALPHABET;
+          if (j && a.lut[j] < a.lut[j - 1]) return SOP_ERR_ALPHABET;
+        }
+      }
+    } else if (a.kind == SOP_KIND_FP_E2M3) {
+      if (a.n_bits != 6 || a.negated) return SOP_ERR_ALPHABET;
+    } else if (a.kind == SOP_KIND_FP_E4M3) {
+      if (a.n_bits != 8 || a.negated) return SOP_ERR_ALPHABET;
+    } else {
+      return SOP_ERR_ALPHABET;
+    }
+    if (((dd_mask >> i) & 1u) && a.kind != SOP_KIND_LUT) return SOP_ERR_ALPHABET;
+    out->atoms[i] = a;
+  }
+  return SOP_OK;
+}
+
+int validate_layer(const void* W, long long M, long long K, long long ldw, const float* c, int g) {
+  if (!W || !c) return SOP_ERR_NULL;
+  if (g != SOP_G) return SOP_ERR_SHAPE;
+  if (M < 1 || K < 1 || (K % SOP_G) != 0 || ldw < K || (ldw % 8) != 0) return SOP_ERR_SHAPE;
+  if (((uintptr_t)W & 15u) != 0) return SOP_ERR_SHAPE;
+  if (M > (1ll << 31) / (K / SOP_G)) return SOP_ERR_SHAPE;  // block count must fit 31 bits
+  return SOP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Channel norms.  Two kernels: per-(chunk, column) FP64 partial sums over 64 rows in row order,
+// then per column the partials added in chunk order, divided by T, square-rooted, rounded to fp32.
+// HBM-bound: X is read exactly once with fully coalesced 128-byte rows per warp.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) norms_partial_kernel(const float* __restrict__ X, long long T, long long K,
+                                                            long long ldx, double* __restrict__ part) {
+  const long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long chunk = blockIdx.y;
+  if (k >= K) return;
+  const long long t0 = chunk * 64, t1 = min(T, t0 + 64);
+  const float* p = X + t0 * ldx + k;
+  double acc = 0.0;
+  long long t = t0;
+  for (; t + 8 <= t1; t += 8) {
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldg(p + (long long)i * ldx);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc = __fma_rn((double)v[i], (double)v[i], acc);
+    p += 8 * ldx;
+  }
+  for (; t < t1; ++t) {
+    const double x = (double)__ldg(p);
+    acc = __fma_rn(x, x, acc);
+    p += ldx;
+  }
+  part[chunk * K + k] = acc;
+}
+
+__global__ void __launch_bounds__(256) norms_final_kernel(const double* __restrict__ part, long long n_chunks, long long K,
+                                                          long long T, float* __restrict__ c) {
+  const long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= K) return;
+  double total = 0.0;
+  for (long long ch = 0; ch < n_chunks; ++ch) total = __dadd_rn(total, part[ch * K + k]);
+  c[k] = __double2float_rn(__dsqrt_rn(__ddiv_rn(total, (double)T)));
+}
+
+}  // namespace sop
+
+extern "C" {
+
+const char* sop_strerror(int code) {
+  switch (code) {
+    case SOP_OK: return "ok";
+    case SOP_ERR_NULL: return "a required pointer is NULL";
+    case SOP_ERR_SHAPE: return "bad shape: need M, K, T >= 1, K % 16 == 0, ld >= K (ldw % 8 == 0, W 16-byte aligned), g == 16";
+    case SOP_ERR_FORMAT: return "bad scale format or scale-word container";
+    case SOP_ERR_ALPHABET: return "bad alphabet: atom count, kind, n_bits, n_entries, tmax or unsorted table";
+    case SOP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SOP_ERR_CUDA: return "CUDA runtime error (see sop_last_cuda_error)";
+    case SOP_ERR_RANGE: return "argument out of range (k shift, pool_rank, iters or index)";
+    default: return "unknown error code";
+  }
+}
+
+const char* sop_last_cuda_error(void) { return sop::g_cuda_error; }
+
+int sop_version(void) { return 100; }
+
+int sop_channel_norms_workspace(long long T, long long K, size_t* bytes) {
+  if (!bytes) return SOP_ERR_NULL;
+  if (T < 1 || K < 1) return SOP_ERR_SHAPE;
+  *bytes = (size_t)((T + 63) / 64) * (size_t)K * sizeof(double);
+  return SOP_OK;
+}
+
+int sop_channel_norms(const float* X_dev, long long T, long long K, long long ldx, float* c_dev,
+                      void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (!X_dev || !c_dev) return SOP_ERR_NULL;
+  if (T < 1 || K < 1 || ldx < K) return SOP_ERR_SHAPE;
+  size_t need = 0;
+  sop_channel_norms_workspace(T, K, &need);
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < need) return SOP_ERR_WORKSPACE;
+  const long long n_chunks = (T + 63) / 64;
+  if (n_chunks > 65535) return SOP_ERR_SHAPE;
+  cudaStream_t st = (cudaStream_t)stream;
+  dim3 grid((unsigned)((K + 255) / 256), (unsigned)n_chunks);
+  sop::norms_partial_kernel<<<grid, 256, 0, st>>>(X_dev, T, K, ldx, (double*)workspace_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+  sop::norms_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>((const double*)workspace_dev, n_chunks, K, T, c_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+  return SOP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,236 @@
+// sop_pack: materialise the chosen codebook(s): per block re-evaluate the (up to four) candidates
+// with the same arithmetic as the sweep, keep the best, and emit 2n bytes of codes plus one b-bit
+// scale word (sign, exponent, mantissa, selector).  HBM-bound: reads W once, writes ~n/8 + b/128
+// bytes per element.
+#include <string.h>
+
+#include "sop_device.cuh"
+
+namespace sop {
+
+constexpr int PTB = 256;
+
+struct PackArgs {
+  const uint16_t* W;
+  const float* c;
+  long long M, K, ldw, nbk, NB;
+  int index_a, index_b, k_mode, use_sign;
+  int container_bits, word_sign_bits, meta_bits;
+  unsigned char* codes;
+  unsigned* words;       // zeroed before the kernel; filled with atomicOr
+  unsigned long long* counts;
+};
+
+struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
+
+// scalar evaluation of one candidate on one block; same operation order as the sweep kernel
+__device__ void eval_block_scalar(const float* w, const float* c, const float* tau, const float* lutv, const PackCand& cd,
+                                  const FmtDev& F, float pot, float& cos_out, uint32_t& scode, int* codes) {
+  float amax = 0.0f;
+  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(w[i]));
+  float s_hat;
+  scode = 0;
+  if (cd.scope == 0) {
+    s_hat = amax > 0.0f ? pot : 0.0f;
+  } else {
+    const float sigma = cd.tmax == 1.0f ? amax : __fdiv_rn(amax, cd.tmax);
+    const QScale qs = scale_quantize(sigma, cd.k, F);
+    s_hat = qs.s_hat;
+    scode = qs.code;
+  }
+  const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+  float qn[4], qd[4], qw[4];
+  for (int h = 0; h < 4; ++h) {
+    float an = 0.0f, ad = 0.0f, aw = 0.0f;
+    for (int r = 0; r < 4; ++r) {
+      const int i = 4 * h + r;
+      const float u = __fmul_rn(w[i], rcp);
+      float q;
+      if (cd.kind == SOP_KIND_LUT) {
+        const int code = count_below(tau, cd.neg ? -u : u);
+        codes[i] = code;
+        q = cd.neg ? -lutv[code] : lutv[code];
+      } else if (cd.kind == SOP_KIND_FP_E2M3) {
+        q = fp_quantize<SOP_KIND_FP_E2M3>(u);
+        codes[i] = (int)fp_code<SOP_KIND_FP_E2M3>(q);
+      } else {
+        q = fp_quantize<SOP_KIND_FP_E4M3>(u);
+        codes[i] = (int)fp_code<SOP_KIND_FP_E4M3>(q);
+      }
+      const float cw = __fmul_rn(c[i], w[i]);
+      const float cq = __fmul_rn(c[i], q);
+      aw = __fmaf_rn(cw, w[i], aw);
+      ad = __fmaf_rn(cw, q, ad);
+      an = __fmaf_rn(cq, q, an);
+    }
+    qn[h] = an; qd[h] = ad; qw[h] = aw;
+  }
+  cos_out = block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd));
+}
+
+__global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
+  __shared__ float lutv[2][32], tau[2][32];
+  __shared__ PackCand base[2];
+  __shared__ int s_nb, s_nbits;
+  __shared__ float s_pot[2];
+  __shared__ unsigned s_cnt[2];
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    int ia = a.index_a, ib = a.index_b;
+    if (ia == SOP_PAIR_FROM_RESULT) {
+      ia = a.use_sign ? res->best_sa : res->best_a;
+      ib = a.use_sign ? res->best_sb : res->best_b;
+    }
+    ia = max(0, min(A.n_atoms - 1, ia));
+    int nb = 1;
+    if (ib != SOP_NO_ATOM) { ib = max(0, min(A.n_atoms - 1, ib)); nb = 2; }
+    s_nb = nb;
+    s_nbits = A.atoms[ia].n_bits;
+    const float wmax = res ? res->layer_absmax : 0.0f;
+    for (int t = 0; t < nb; ++t) {
+      const int idx = t ? ib : ia;
+      const sop_atom& at = A.atoms[idx];
+      base[t].table = t; base[t].kind = at.kind; base[t].neg = at.negated; base[t].scope = at.scope; base[t].tmax = at.tmax;
+      base[t].k = a.k_mode == SOP_K_FROM_RESULT ? res->k[idx] : a.k_mode;
+      s_pot[t] = at.scope == 0 ? layer_pot_scale(wmax, at.tmax) : 0.0f;
+      const bool dd = (A.dd_mask >> idx) & 1u;
+      const int ne = at.kind == SOP_KIND_LUT ? at.n_entries : 2;
+      for (int j = 0; j < 32; ++j) lutv[t][j] = at.kind == SOP_KIND_LUT ? (dd ? A.dd_lut[min(j, ne - 1)] : at.lut[min(j, ne - 1)]) : 0.0f;
+      build_thresholds(lutv[t], ne, tau[t]);
+    }
+    s_cnt[0] = s_cnt[1] = 0;
+  }
+  __syncthreads();
+  const int nb = s_nb, n = s_nbits, b = a.container_bits;
+  unsigned my_sel = 0, my_neg = 0;
+  for (long long blk = (long long)blockIdx.x * PTB + tid; blk < a.NB; blk += (long long)gridDim.x * PTB) {
+    const long long m = blk / a.nbk, j = blk - m * a.nbk;
+    const uint4* p = reinterpret_cast<const uint4*>(a.W + m * a.ldw + j * SOP_G);
+    const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+    const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    float w[16], c[16];
+    for (int i = 0; i < 8; ++i) { w[2 * i] = bf16lo(wb[i]); w[2 * i + 1] = bf16hi(wb[i]); }
+    for (int i = 0; i < 16; ++i) c[i] = __ldg(a.c + j * SOP_G + i);
+    float best_cos = 0.0f;
+    uint32_t best_scode = 0;
+    int best_codes[16], pick = -1;
+    for (int t = 0; t < nb; ++t)
+      for (int sg = 0; sg < (a.use_sign ? 2 : 1); ++sg) {
+        PackCand cd = base[t];
+        if (sg) cd.neg = 1 - cd.neg;
+        float cs;
+        uint32_t sc;
+        int codes[16];
+        eval_block_scalar(w, c, tau[t], lutv[t], cd, F, s_pot[t], cs, sc, codes);
+        if (pick < 0 || cs > best_cos) {
+          best_cos = cs; best_scode = sc; pick = 2 * t + sg;
+          for (int i = 0; i < 16; ++i) best_codes[i] = codes[i];
+        }
+      }
+    const unsigned sel = pick >> 1, sgn = pick & 1;
+    my_sel += sel; my_neg += sgn;
+    // codes: 16 n-bit fields, little-endian, 2n bytes = n 16-bit stores
+    unsigned long long lo = 0, hi = 0;   // 128-bit accumulator
+    for (int i = 0; i < 16; ++i) {
+      const int pos = i * n;
+      const unsigned long long v = (unsigned long long)best_codes[i];
+      if (pos < 64) {
+        lo |= v << pos;
+        if (pos + n > 64) hi |= v >> (64 - pos);
+      } else {
+        hi |= v << (pos - 64);
+      }
+    }
+    unsigned short* dst = reinterpret_cast<unsigned short*>(a.codes + blk * 2 * n);
+    for (int i = 0; i < n; ++i) dst[i] = (unsigned short)((i < 4 ? lo >> (16 * i) : hi >> (16 * (i - 4))) & 0xFFFFu);
+    // scale word
+    unsigned word;
+    if (a.word_sign_bits) word = (sgn << (b - 1)) | (best_scode << a.meta_bits) | (a.meta_bits >= 1 ? sel : 0u);
+    else if (a.meta_bits >= 1) word = (sel << (b - 1)) | (best_scode << (a.meta_bits - 1));
+    else word = best_scode;
+    const long long bit = blk * b;
+    const long long wi = bit >> 5;
+    const int sh = (int)(bit & 31);
+    if (word) {
+      atomicOr(&a.words[wi], word << sh);
+      if (sh + b > 32) atomicOr(&a.words[wi + 1], word >> (32 - sh));
+    }
+  }
+  if (a.counts) {
+    atomicAdd(&s_cnt[0], my_sel);
+    atomicAdd(&s_cnt[1], my_neg);
+    __syncthreads();
+    if (tid < 2 && s_cnt[tid]) atomicAdd(&a.counts[tid], (unsigned long long)s_cnt[tid]);
+  }
+}
+
+int num_sms();
+
+}  // namespace sop
+
+extern "C" {
+
+int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+             const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
+             unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
+             int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
+             unsigned char* words_dev, long long* counts_dev, void* stream) {
+  using namespace sop;
+  int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
+  if (rc) return rc;
+  if (!codes_dev || !words_dev) return SOP_ERR_NULL;
+  FmtDev F;
+  if ((rc = validate_fmt(fmt, &F))) return rc;
+  AtomsDev A;
+  if ((rc = validate_atoms(atoms, n_atoms, dd_mask, dd_lut_dev, &A))) return rc;
+  if (use_sign != 0 && use_sign != 1) return SOP_ERR_FORMAT;
+  if (word_sign_bits != 0 && word_sign_bits != 1) return SOP_ERR_FORMAT;
+  if (container_bits != 8 && container_bits != 12 && container_bits != 16) return SOP_ERR_FORMAT;
+  const int meta = container_bits - word_sign_bits - fmt->exp_bits - fmt->man_bits;
+  if (meta < 0 || (use_sign && !word_sign_bits)) return SOP_ERR_FORMAT;
+  const bool from_result = index_a == SOP_PAIR_FROM_RESULT;
+  if (from_result) {
+    if (!search_dev) return SOP_ERR_NULL;
+    if (index_b == SOP_NO_ATOM) return SOP_ERR_RANGE;
+  } else {
+    if (index_a < 0 || index_a >= n_atoms) return SOP_ERR_RANGE;
+    if (index_b != SOP_NO_ATOM && (index_b < 0 || index_b >= n_atoms)) return SOP_ERR_RANGE;
+    if (index_b != SOP_NO_ATOM && (atoms[index_a].n_bits != atoms[index_b].n_bits || atoms[index_a].kind != SOP_KIND_LUT ||
+                                   atoms[index_b].kind != SOP_KIND_LUT)) return SOP_ERR_ALPHABET;
+    if (use_sign && atoms[index_a].kind != SOP_KIND_LUT) return SOP_ERR_ALPHABET;
+  }
+  const bool pair = index_b != SOP_NO_ATOM;
+  if (pair && meta < 1) return SOP_ERR_FORMAT;     // the selector needs a metabit
+  if (k_mode == SOP_K_FROM_RESULT) { if (!search_dev) return SOP_ERR_NULL; }
+  else if (k_mode < -64 || k_mode > 64) return SOP_ERR_RANGE;
+  bool need_wmax = false;
+  for (int i = 0; i < n_atoms; ++i) need_wmax |= atoms[i].scope == 0;
+  if (need_wmax && !search_dev) return SOP_ERR_NULL;  // the layer power-of-two scale comes from a previous search
+  if (((uintptr_t)codes_dev & 1u) || ((uintptr_t)words_dev & 3u)) return SOP_ERR_SHAPE;
+  // every atom that can be picked must share n_bits with the first LUT atom when the pair comes from the device
+  int n_bits = from_result ? 0 : atoms[index_a].n_bits;
+  if (from_result) {
+    for (int i = 0; i < n_atoms; ++i)
+      if (atoms[i].kind == SOP_KIND_LUT) { if (!n_bits) n_bits = atoms[i].n_bits; else if (atoms[i].n_bits != n_bits) return SOP_ERR_ALPHABET; }
+    if (!n_bits) return SOP_ERR_ALPHABET;
+  }
+
+  PackArgs a;
+  a.W = (const uint16_t*)W_dev; a.c = c_dev; a.M = M; a.K = K; a.ldw = ldw; a.nbk = K / SOP_G; a.NB = M * a.nbk;
+  a.index_a = index_a; a.index_b = index_b; a.k_mode = k_mode; a.use_sign = use_sign;
+  a.container_bits = container_bits; a.word_sign_bits = word_sign_bits; a.meta_bits = meta;
+  a.codes = codes_dev; a.words = (unsigned*)words_dev; a.counts = (unsigned long long*)counts_dev;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t word_bytes = (size_t)((a.NB * container_bits + 7) / 8);
+  // the word stream is written with 32-bit atomicOr: the caller's buffer must hold whole 32-bit words
+  SOP_CUDA_TRY(cudaMemsetAsync(words_dev, 0, (word_bytes + 3) & ~(size_t)3, st));
+  if (counts_dev) SOP_CUDA_TRY(cudaMemsetAsync(counts_dev, 0, 2 * sizeof(long long), st));
+  long long grid = (a.NB + PTB - 1) / PTB;
+  const int sms = num_sms();
+  if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+  pack_kernel<<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+  return SOP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,759 @@
+// sop_pair_search: the per-layer candidate sweep.
+//
+//   prepass_kernel   reads W once: per-block absmax -> exponent histogram of sigma = absmax / tmax
+//                    for every scale class that needs an F_layer search, and max|W|.        (HBM-bound)
+//   kselect_kernel   one CTA: the F_layer shift k* per class from the histogram, the layer
+//                    power-of-two scale for "^0" candidates.
+//   sweep_kernel     persistent, one thread per 16-element block: phase 1 evaluates every candidate
+//                    in registers (cell-table lookup of the reconstruction value, packed f32x2
+//                    fused multiply-adds for the block metric, fixed quad-tree order); phase 2
+//                    reduces the per-block (cos, sse) of the CTA's tile into per-pair sums, one
+//                    pair per thread, FP64 accumulators.                                    (ALU-bound)
+//   finalize_kernel  one CTA: adds the per-CTA partials in CTA order (deterministic), writes the
+//                    tables and picks the best pair / best single.
+#include <math.h>
+#include <string.h>
+
+#include "sop_device.cuh"
+
+namespace sop {
+
+constexpr int TB = 512;             // threads per CTA of the sweep kernel
+constexpr int MAX_SLOTS = 192;      // pair slots per call: 16 singles + 120 pairs + 36 signed < 192
+constexpr int MAX_GRID = 1024;
+constexpr float MAGIC = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+
+struct CandDev { unsigned char cls, kind, neg, table; };
+struct ClassDev {
+  float tmax;
+  float invh2;       // cells per unit of u2 = 2u (power of two)
+  int scope, kind;   // kind of the quantiser: LUT, E2M3, E4M3
+  int c_half;        // table rows = 2 * c_half + 1
+  int auto_k;        // 1: k* from the histogram
+  int n_cand;
+  unsigned char cand[SOP_MAX_ATOMS];
+};
+struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (i0 == i1: single); 1: signed (i0, i0+1, i1, i1+1)
+
+struct Plan {
+  int n_atoms, n_classes, n_tables, n_slots, n_pair_slots;
+  int k_mode, rows, a_pad;
+  CandDev cand[SOP_MAX_ATOMS];
+  ClassDev cls[SOP_MAX_CLASSES];
+  unsigned char table_atom[SOP_MAX_TABLES];   // atom whose lut fills the table
+  unsigned char table_cls[SOP_MAX_TABLES];
+  SlotDev slots[MAX_SLOTS];
+};
+
+struct WsHeader {
+  unsigned wmax_bits;
+  int cls_k[SOP_MAX_CLASSES];
+  float cls_pot[SOP_MAX_CLASSES];
+  int pad[7];
+};
+struct Partial { double gap, sse; long long n1, nneg; };
+
+static size_t ws_hist_off() { return 256; }
+static size_t ws_part_off() { return 256 + sizeof(unsigned) * SOP_MAX_CLASSES * SOP_HIST_BINS; }
+static size_t ws_total() { return ((ws_part_off() + sizeof(Partial) * (size_t)MAX_GRID * MAX_SLOTS) + 255) & ~(size_t)255; }
+
+struct LayerArgs {
+  const uint16_t* W;
+  const float* c;
+  long long M, K, ldw;
+  long long nbk;      // K / 16
+  long long NB;       // M * nbk
+};
+
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void load_block_bits(const uint16_t* p, uint32_t (&v)[8]) {
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint4 b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+__device__ __forceinline__ float absmax_bits(const uint32_t (&v)[8]) {
+  // bf16 magnitudes order like their bit patterns
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    m = max(m, v[i] & 0x7FFFu);
+    m = max(m, (v[i] >> 16) & 0x7FFFu);
+  }
+  return __uint_as_float(m << 16);
+}
+
+__global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, unsigned* __restrict__ hist, WsHeader* __restrict__ hdr) {
+  __shared__ unsigned sh[SOP_MAX_CLASSES * SOP_HIST_BINS];
+  for (int i = threadIdx.x; i < P.n_classes * SOP_HIST_BINS; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  uint32_t wmax = 0;
+  for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < L.NB; b += (long long)gridDim.x * blockDim.x) {
+    const long long m = b / L.nbk, j = b - m * L.nbk;
+    uint32_t v[8];
+    load_block_bits(L.W + m * L.ldw + j * SOP_G, v);
+    const float a = absmax_bits(v);
+    wmax = max(wmax, __float_as_uint(a));
+    if (a > 0.0f) {
+      for (int cl = 0; cl < P.n_classes; ++cl) {
+        if (!P.cls[cl].auto_k) continue;
+        const float sigma = P.cls[cl].tmax == 1.0f ? a : __fdiv_rn(a, P.cls[cl].tmax);
+        if (sigma > 0.0f) atomicAdd(&sh[cl * SOP_HIST_BINS + ilogb_pos(sigma) + SOP_HIST_OFF], 1u);
+      }
+    }
+  }
+  for (int o = 16; o; o >>= 1) wmax = max(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+  if ((threadIdx.x & 31) == 0) atomicMax(&hdr->wmax_bits, wmax);
+  __syncthreads();
+  for (int i = threadIdx.x; i < P.n_classes * SOP_HIST_BINS; i += blockDim.x)
+    if (sh[i]) atomicAdd(&hist[i], sh[i]);
+}
+
+__global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const unsigned* __restrict__ hist, WsHeader* __restrict__ hdr,
+                                                      sop_search_result* __restrict__ res) {
+  __shared__ unsigned long long cnt[129];
+  const float wmax = __uint_as_float(hdr->wmax_bits);
+  for (int cl = 0; cl < P.n_classes; ++cl) {
+    int kstar = P.k_mode == SOP_K_AUTO ? 0 : P.k_mode;
+    if (P.cls[cl].scope == 0) kstar = 0;
+    if (P.cls[cl].auto_k) {
+      if (threadIdx.x < 129) {
+        const int k = (int)threadIdx.x - 64;
+        unsigned long long c = 0;
+        for (int e = -SOP_HIST_OFF; e < SOP_HIST_BINS - SOP_HIST_OFF; ++e)
+          if (e + k >= F.emin && e + k <= F.emax) c += hist[cl * SOP_HIST_BINS + e + SOP_HIST_OFF];
+        cnt[threadIdx.x] = c;
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        // largest count; ties to the smallest |k|, then to k > 0
+        unsigned long long best = cnt[64];
+        kstar = 0;
+        for (int mag = 1; mag <= 64; ++mag) {
+          if (cnt[64 + mag] > best) { best = cnt[64 + mag]; kstar = mag; }
+          if (cnt[64 - mag] > best) { best = cnt[64 - mag]; kstar = -mag; }
+        }
+      }
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      hdr->cls_k[cl] = kstar;
+      hdr->cls_pot[cl] = P.cls[cl].scope == 0 ? layer_pot_scale(wmax, P.cls[cl].tmax) : 0.0f;
+      for (int i = 0; i < P.cls[cl].n_cand; ++i) res->k[P.cls[cl].cand[i]] = kstar;
+    }
+  }
+  if (threadIdx.x == 0) {
+    for (int i = P.n_atoms; i < SOP_MAX_ATOMS; ++i) res->k[i] = 0;
+    res->layer_absmax = wmax;
+    res->reserved[0] = res->reserved[1] = 0;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Phase-1 evaluators.  Element layout inside a thread: index idx = 2 * i + p holds, as a float2,
+// element i of quads 2p (x) and 2p + 1 (y): the two lanes of a packed f32x2 operation are two
+// independent sequential chains, which is exactly the quad-tree summation order.
+// ---------------------------------------------------------------------------------------------
+struct BlockRegs {
+  float2 w[8], c[8], cw[8], u2[8];
+  int r32[16];      // cell row * 32 (word offset into a lane-replicated table), per element
+};
+
+__device__ __forceinline__ float fold(const float2 a, const float2 b) {
+  return __fadd_rn(__fadd_rn(a.x, a.y), __fadd_rn(b.x, b.y));
+}
+
+struct Metric { float nq, dot, sse; };
+
+template <bool NEG>
+__device__ __forceinline__ Metric eval_lut_cells(const uint32_t* __restrict__ tbl_lane, int mirror, const BlockRegs& B, float s_hat) {
+  float2 nq[2], dot[2], sse[2];
+  nq[0] = nq[1] = dot[0] = dot[1] = sse[0] = sse[1] = make_float2(0.0f, 0.0f);
+  const float sg = NEG ? s_hat : -s_hat;
+  const float2 ns = make_float2(sg, sg);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      const int idx = 2 * i + p;
+      const uint32_t wa = tbl_lane[NEG ? mirror - B.r32[2 * idx] : B.r32[2 * idx]];
+      const uint32_t wb = tbl_lane[NEG ? mirror - B.r32[2 * idx + 1] : B.r32[2 * idx + 1]];
+      const float la = bf16lo(wa), ha = bf16hi(wa), lb = bf16lo(wb), hb = bf16hi(wb);
+      const float sa = __fadd_rn(la, ha), sb = __fadd_rn(lb, hb);
+      float2 q;
+      q.x = (NEG ? (-B.u2[idx].x > sa) : (B.u2[idx].x > sa)) ? ha : la;
+      q.y = (NEG ? (-B.u2[idx].y > sb) : (B.u2[idx].y > sb)) ? hb : lb;
+      const float2 cq = __fmul2_rn(B.c[idx], q);
+      nq[p] = __ffma2_rn(cq, q, nq[p]);
+      dot[p] = __ffma2_rn(B.cw[idx], q, dot[p]);
+      const float2 e = __ffma2_rn(ns, q, B.w[idx]);
+      sse[p] = __ffma2_rn(e, e, sse[p]);
+    }
+  }
+  Metric m;
+  m.nq = fold(nq[0], nq[1]);
+  const float d = fold(dot[0], dot[1]);
+  m.dot = NEG ? -d : d;
+  m.sse = fold(sse[0], sse[1]);
+  return m;
+}
+
+// mode 0: table through binary search over the thresholds (any table); mode 1 / 2: E2M3 / E4M3 grid
+template <int MODE, bool NEG>
+__device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, const float* __restrict__ lutv, const BlockRegs& B, float s_hat) {
+  float2 nq[2], dot[2], sse[2];
+  nq[0] = nq[1] = dot[0] = dot[1] = sse[0] = sse[1] = make_float2(0.0f, 0.0f);
+  const float sg = NEG ? s_hat : -s_hat;
+  const float2 ns = make_float2(sg, sg);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      const int idx = 2 * i + p;
+      const float ux = __fmul_rn(B.u2[idx].x, 0.5f), uy = __fmul_rn(B.u2[idx].y, 0.5f);
+      float2 q;
+      if (MODE == 0) {
+        q.x = lutv[count_below(tau, NEG ? -ux : ux)];
+        q.y = lutv[count_below(tau, NEG ? -uy : uy)];
+      } else {
+        q.x = fp_quantize<MODE>(ux);
+        q.y = fp_quantize<MODE>(uy);
+      }
+      const float2 cq = __fmul2_rn(B.c[idx], q);
+      nq[p] = __ffma2_rn(cq, q, nq[p]);
+      dot[p] = __ffma2_rn(B.cw[idx], q, dot[p]);
+      const float2 e = __ffma2_rn(ns, q, B.w[idx]);
+      sse[p] = __ffma2_rn(e, e, sse[p]);
+    }
+  }
+  Metric m;
+  m.nq = fold(nq[0], nq[1]);
+  const float d = fold(dot[0], dot[1]);
+  m.dot = NEG ? -d : d;
+  m.sse = fold(sse[0], sse[1]);
+  return m;
+}
+
+// Build the shared-memory tables of one CTA: table values and thresholds, then the lane-replicated
+// cell tables.  A cell row r (k = r - c_half) covers the u2 values that round to k:
+// u2 * invh2 in [k - 1/2, k + 1/2]; row 0 and the last row extend to -inf / +inf.  A row is usable
+// when at most one distinct threshold falls inside its closed interval and lo + hi is exact in
+// fp32 (then "u2 > lo + hi" is the exact nearest-entry decision); otherwise the whole table is
+// marked slow and its candidates take the binary-search path.
+__device__ void build_tables(const Plan& P, const AtomsDev& A, uint32_t* cell, float* tau, float* lutv, int* fast) {
+  const int tid = threadIdx.x;
+  for (int i = tid; i < P.n_tables * 32; i += blockDim.x) {
+    const int t = i >> 5, j = i & 31;
+    const int a = P.table_atom[t];
+    const int ne = A.atoms[a].n_entries;
+    const int jj = min(j, ne - 1);
+    lutv[i] = ((A.dd_mask >> a) & 1u) ? A.dd_lut[jj] : A.atoms[a].lut[jj];
+  }
+  if (tid < SOP_MAX_TABLES) fast[tid] = 1;
+  __syncthreads();
+  if (tid < P.n_tables) build_thresholds(lutv + tid * 32, A.atoms[P.table_atom[tid]].n_entries, tau + tid * 32);
+  __syncthreads();
+  const int rows = P.rows;
+  for (int i = tid; i < P.n_tables * rows; i += blockDim.x) {
+    const int t = i / rows, r = i - t * rows;
+    const ClassDev& C = P.cls[P.table_cls[t]];
+    const int ne = A.atoms[P.table_atom[t]].n_entries;
+    const int nrow = 2 * C.c_half + 1;
+    uint32_t word = 0;
+    if (r < nrow) {
+      const float hh = __fdiv_rn(0.5f, C.invh2);                    // cell width in u (a power of two)
+      const float kf = (float)(r - C.c_half);
+      const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, hh);
+      const float hi_edge = r == nrow - 1 ? INFINITY : __fmul_rn(kf + 0.5f, hh);
+      const float* tt = tau + t * 32;
+      const float* lv = lutv + t * 32;
+      int nbelow = 0, ninside = 0, ndistinct = 0;
+      float prev = 0.0f;
+      for (int j = 0; j < ne - 1; ++j) {
+        const float x = tt[j];
+        if (x < lo_edge) ++nbelow;
+        else if (x <= hi_edge) {
+          if (ninside == 0 || x != prev) ++ndistinct;
+          prev = x;
+          ++ninside;
+        }
+      }
+      const float lo = lv[nbelow], hi = lv[min(nbelow + ninside, ne - 1)];
+      const uint32_t lb = __float_as_uint(lo), hb = __float_as_uint(hi);
+      bool ok = ndistinct <= 1 && (lb & 0xFFFFu) == 0 && (hb & 0xFFFFu) == 0;
+      if (ok && ninside) ok = (double)__fadd_rn(lo, hi) == (double)lo + (double)hi;
+      if (!ok) atomicAnd(&fast[t], 0);
+      word = (hb & 0xFFFF0000u) | (lb >> 16);
+    }
+    uint32_t* dst = cell + (size_t)i * 32;
+    for (int l = 0; l < 32; ++l) dst[l] = word;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, const WsHeader* __restrict__ hdr,
+                                                      Partial* __restrict__ partials, float* __restrict__ block_cos,
+                                                      float* __restrict__ block_sse) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  uint32_t* cell = reinterpret_cast<uint32_t*>(smem);
+  float* tau = reinterpret_cast<float*>(cell + (size_t)P.n_tables * P.rows * 32);
+  float* lutv = tau + SOP_MAX_TABLES * 32;
+  int* fast = reinterpret_cast<int*>(lutv + SOP_MAX_TABLES * 32);
+  int* cls_k = fast + SOP_MAX_TABLES;
+  float* cls_pot = reinterpret_cast<float*>(cls_k + SOP_MAX_CLASSES);
+  float2* cs = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [TB][a_pad] (cos, sse)
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  build_tables(P, A, cell, tau, lutv, fast);
+  if (tid < SOP_MAX_CLASSES) { cls_k[tid] = hdr->cls_k[tid]; cls_pot[tid] = hdr->cls_pot[tid]; }
+  __syncthreads();
+
+  // thread -> fixed column block j, rows m = r0, r0 + R, ...
+  const long long GT = (long long)gridDim.x * TB;
+  const long long R = GT / L.nbk;                 // rows in flight (host guarantees R >= 1)
+  const long long gt = (long long)blockIdx.x * TB + tid;
+  const bool lane_on = gt < R * L.nbk;
+  const long long j = lane_on ? gt % L.nbk : 0;
+  const long long r0 = gt / L.nbk;
+  const long long n_iter = (L.M + R - 1) / R;
+
+  BlockRegs B;
+  {
+    const float4* cp = reinterpret_cast<const float4*>(L.c + j * SOP_G);
+    float cc[16];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 v = __ldg(cp + q);
+      cc[4 * q] = v.x; cc[4 * q + 1] = v.y; cc[4 * q + 2] = v.z; cc[4 * q + 3] = v.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int p = 0; p < 2; ++p) B.c[2 * i + p] = make_float2(cc[8 * p + i], cc[8 * p + 4 + i]);
+  }
+
+  // phase-2 role of this thread
+  const int n_slots = P.n_slots;
+  const int n_groups = TB / n_slots;
+  const int slot = tid % n_slots, grp = tid / n_slots;
+  const bool red_on = grp < n_groups;
+  const SlotDev sd = P.slots[slot];
+  double acc_gap = 0.0, acc_sse = 0.0;
+  int acc_n1 = 0, acc_nneg = 0;
+  const int a_pad = P.a_pad;
+
+  uint32_t wb[8];
+  if (lane_on && r0 < L.M) load_block_bits(L.W + r0 * L.ldw + j * SOP_G, wb);
+
+  for (long long it = 0; it < n_iter; ++it) {
+    const long long m = r0 + it * R;
+    const bool on = lane_on && m < L.M;
+    // number of valid threads of this CTA in this iteration (they form a prefix)
+    long long nv = min(L.M - it * R, R) * L.nbk - (long long)blockIdx.x * TB;
+    nv = max(0ll, min((long long)TB, nv));
+    if (on) {
+      // ---- unpack, block statistics ----
+      float wf[16];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { wf[2 * q] = bf16lo(wb[q]); wf[2 * q + 1] = bf16hi(wb[q]); }
+      const float amax = absmax_bits(wb);
+      const long long mn = m + R;
+      if (mn < L.M) load_block_bits(L.W + mn * L.ldw + j * SOP_G, wb);   // prefetch the next row's block
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int p = 0; p < 2; ++p) B.w[2 * i + p] = make_float2(wf[8 * p + i], wf[8 * p + 4 + i]);
+      float2 nw2[2];
+      nw2[0] = nw2[1] = make_float2(0.0f, 0.0f);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          B.cw[2 * i + p] = __fmul2_rn(B.c[2 * i + p], B.w[2 * i + p]);
+          nw2[p] = __ffma2_rn(B.cw[2 * i + p], B.w[2 * i + p], nw2[p]);
+        }
+      const float nw = fold(nw2[0], nw2[1]);
+      const long long blk = m * L.nbk + j;
+      float2* my = cs + (size_t)tid * a_pad;
+
+      for (int cl = 0; cl < P.n_classes; ++cl) {
+        const ClassDev& C = P.cls[cl];
+        float s_hat;
+        if (C.scope == 0) {
+          s_hat = amax > 0.0f ? cls_pot[cl] : 0.0f;
+        } else {
+          const float sigma = C.tmax == 1.0f ? amax : __fdiv_rn(amax, C.tmax);
+          s_hat = scale_quantize(sigma, cls_k[cl], F).s_hat;
+        }
+        const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+        const float2 r2 = make_float2(rcp, rcp);
+        const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
+#pragma unroll
+        for (int idx = 0; idx < 8; ++idx) {
+          const float2 u = __fmul2_rn(B.w[idx], r2);
+          B.u2[idx] = __fadd2_rn(u, u);
+          if (C.kind == SOP_KIND_LUT) {
+            const float tx = fminf(fmaxf(__fmaf_rn(B.u2[idx].x, C.invh2, toff), tlo), thi);
+            const float ty = fminf(fmaxf(__fmaf_rn(B.u2[idx].y, C.invh2, toff), tlo), thi);
+            B.r32[2 * idx] = (int)(__float_as_uint(tx) - __float_as_uint(MAGIC)) * 32;
+            B.r32[2 * idx + 1] = (int)(__float_as_uint(ty) - __float_as_uint(MAGIC)) * 32;
+          }
+        }
+        const int mirror = 2 * C.c_half * 32;
+        for (int ci = 0; ci < C.n_cand; ++ci) {
+          const int a = C.cand[ci];
+          const CandDev cd = P.cand[a];
+          Metric mt;
+          if (cd.kind == SOP_KIND_LUT) {
+            const int t = cd.table;
+            if (fast[t]) {
+              const uint32_t* tl = cell + (size_t)t * P.rows * 32 + lane;
+              mt = cd.neg ? eval_lut_cells<true>(tl, mirror, B, s_hat) : eval_lut_cells<false>(tl, mirror, B, s_hat);
+            } else {
+              mt = cd.neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
+                          : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
+            }
+          } else if (cd.kind == SOP_KIND_FP_E2M3) {
+            mt = eval_generic<SOP_KIND_FP_E2M3, false>(nullptr, nullptr, B, s_hat);
+          } else {
+            mt = eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat);
+          }
+          const float cosv = block_cosine(nw, mt.nq, mt.dot);
+          my[a] = make_float2(cosv, mt.sse);
+          if (block_cos) block_cos[(size_t)a * L.NB + blk] = cosv;
+          if (block_sse) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+        }
+      }
+    }
+    __syncthreads();
+    // ---- phase 2: one pair slot per thread, blocks grp, grp + n_groups, ... of the tile ----
+    if (red_on) {
+      const int nvi = (int)nv;
+      float cg = 0.0f, ce = 0.0f;
+      int cnt = 0;
+      for (int b = grp; b < nvi; b += n_groups) {
+        const float2* row = cs + (size_t)b * a_pad;
+        float2 sel = row[sd.i0];
+        if (sd.type == 0) {
+          const float2 v = row[sd.i1];
+          const bool mu = v.x > sel.x;
+          if (mu) sel = v;
+          acc_n1 += mu ? 1 : 0;
+        } else {
+          int pick = 0;
+          float2 v = row[sd.i0 + 1];
+          if (v.x > sel.x) { sel = v; pick = 1; }
+          if (sd.i1 != sd.i0) {
+            v = row[sd.i1];
+            if (v.x > sel.x) { sel = v; pick = 2; }
+            v = row[sd.i1 + 1];
+            if (v.x > sel.x) { sel = v; pick = 3; }
+          }
+          acc_n1 += pick >> 1;
+          acc_nneg += pick & 1;
+        }
+        cg = __fadd_rn(cg, __fsub_rn(1.0f, sel.x));
+        ce = __fadd_rn(ce, sel.y);
+        if (++cnt == 8) {
+          acc_gap += (double)cg; acc_sse += (double)ce;
+          cg = ce = 0.0f; cnt = 0;
+        }
+      }
+      acc_gap += (double)cg; acc_sse += (double)ce;
+    }
+    __syncthreads();
+  }
+
+  // ---- per-CTA partials: groups added in group order by the group-0 thread of each slot ----
+  Partial* sc = reinterpret_cast<Partial*>(cs);
+  if (red_on) { Partial p; p.gap = acc_gap; p.sse = acc_sse; p.n1 = acc_n1; p.nneg = acc_nneg; sc[grp * n_slots + slot] = p; }
+  __syncthreads();
+  if (tid < n_slots) {
+    Partial t = sc[tid];
+    for (int g = 1; g < n_groups; ++g) {
+      const Partial q = sc[g * n_slots + tid];
+      t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
+    }
+    partials[(size_t)blockIdx.x * MAX_SLOTS + tid] = t;
+  }
+}
+
+__global__ void __launch_bounds__(MAX_SLOTS) finalize_kernel(LayerArgs L, Plan P, FmtDev F, int grid, const Partial* __restrict__ partials,
+                                                             sop_pair_stat* __restrict__ pair_table, sop_pair_stat* __restrict__ signed_table,
+                                                             sop_search_result* __restrict__ res) {
+  const int A = P.n_atoms, tid = threadIdx.x;
+  for (int i = tid; i < A * A; i += blockDim.x) {
+    sop_pair_stat u; u.acos = 0.0; u.mse = 0.0; u.n_sel1 = -1; u.n_neg = -1;
+    pair_table[i] = u;
+    if (signed_table) signed_table[i] = u;
+  }
+  __syncthreads();
+  if (tid < P.n_slots) {
+    Partial t = partials[tid];
+    for (int g = 1; g < grid; ++g) {
+      const Partial q = partials[(size_t)g * MAX_SLOTS + tid];
+      t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
+    }
+    sop_pair_stat s;
+    s.acos = ((double)L.NB - t.gap) / (double)L.NB;
+    s.mse = t.sse / ((double)L.M * (double)L.K);
+    s.n_sel1 = t.n1;
+    const SlotDev sd = P.slots[tid];
+    if (sd.type == 0) { s.n_neg = 0; pair_table[sd.i0 * A + sd.i1] = s; }
+    else if (signed_table) { s.n_neg = t.nneg; signed_table[sd.i0 * A + sd.i1] = s; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int ba = -1, bb = -1, bs = -1, bsa = -1, bsb = -1;
+    double vp = -2.0, vs = -2.0, vsp = -2.0;
+    for (int a = 0; a < A; ++a) {
+      if (P.cand[a].kind == SOP_KIND_LUT && pair_table[a * A + a].acos > vs) { vs = pair_table[a * A + a].acos; bs = a; }
+      for (int b = a + 1; b < A; ++b) {
+        const sop_pair_stat p = pair_table[a * A + b];
+        if (p.n_sel1 >= 0 && p.acos > vp) { vp = p.acos; ba = a; bb = b; }
+        if (signed_table) {
+          const sop_pair_stat q = signed_table[a * A + b];
+          if (q.n_sel1 >= 0 && q.acos > vsp) { vsp = q.acos; bsa = a; bsb = b; }
+        }
+      }
+    }
+    res->best_a = ba; res->best_b = bb; res->best_single = bs; res->best_sa = bsa; res->best_sb = bsb;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host: plan construction
+// ---------------------------------------------------------------------------------------------
+static bool same_table(const sop_atom& a, const sop_atom& b) {
+  return a.n_entries == b.n_entries && memcmp(a.lut, b.lut, sizeof(float) * a.n_entries) == 0;
+}
+
+// smallest gap between distinct decision thresholds of a host-known table (in u)
+static double min_threshold_gap(const sop_atom& a) {
+  double prev = 0, best = 1e30;
+  bool have = false;
+  for (int j = 0; j + 1 < a.n_entries; ++j) {
+    if (a.lut[j] == a.lut[j + 1]) continue;
+    const double t = 0.5 * ((double)a.lut[j] + (double)a.lut[j + 1]);
+    if (have && t > prev) best = fmin(best, t - prev);
+    prev = t;
+    have = true;
+  }
+  return best;
+}
+
+int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
+  memset(P, 0, sizeof(*P));
+  const int n = A.n_atoms;
+  P->n_atoms = n;
+  P->k_mode = k_mode;
+  // classes
+  for (int i = 0; i < n; ++i) {
+    const sop_atom& a = A.atoms[i];
+    int cl = -1;
+    for (int c = 0; c < P->n_classes; ++c)
+      if (P->cls[c].scope == a.scope && P->cls[c].tmax == a.tmax && P->cls[c].kind == a.kind) cl = c;
+    if (cl < 0) {
+      if (P->n_classes == SOP_MAX_CLASSES) return SOP_ERR_ALPHABET;
+      cl = P->n_classes++;
+      P->cls[cl].scope = a.scope; P->cls[cl].tmax = a.tmax; P->cls[cl].kind = a.kind;
+      P->cls[cl].auto_k = (k_mode == SOP_K_AUTO && a.scope != 0) ? 1 : 0;
+      P->cls[cl].invh2 = 1.0f; P->cls[cl].c_half = 0;
+    }
+    ClassDev& C = P->cls[cl];
+    C.cand[C.n_cand++] = (unsigned char)i;
+    P->cand[i].cls = (unsigned char)cl;
+    P->cand[i].kind = (unsigned char)a.kind;
+    P->cand[i].neg = (unsigned char)a.negated;
+    P->cand[i].table = 0;
+    if (a.kind != SOP_KIND_LUT) continue;
+    const bool dd = (A.dd_mask >> i) & 1u;
+    int t = -1;
+    for (int q = 0; q < P->n_tables; ++q) {
+      const int o = P->table_atom[q];
+      const bool odd = (A.dd_mask >> o) & 1u;
+      if (P->table_cls[q] != cl || odd != dd) continue;
+      if (dd ? (A.atoms[o].n_entries == a.n_entries) : same_table(A.atoms[o], a)) t = q;
+    }
+    if (t < 0) {
+      if (P->n_tables == SOP_MAX_TABLES) return SOP_ERR_ALPHABET;
+      t = P->n_tables++;
+      P->table_atom[t] = (unsigned char)i;
+      P->table_cls[t] = (unsigned char)cl;
+    }
+    P->cand[i].table = (unsigned char)t;
+  }
+  // cell geometry per LUT class: cell width (in u) below the smallest threshold gap, a power of two
+  int rows = 1;
+  for (int c = 0; c < P->n_classes; ++c) {
+    ClassDev& C = P->cls[c];
+    if (C.kind != SOP_KIND_LUT) continue;
+    double gap = 1e30;
+    bool any_dd = false;
+    for (int q = 0; q < P->n_tables; ++q) {
+      if (P->table_cls[q] != c) continue;
+      const int o = P->table_atom[q];
+      if ((A.dd_mask >> o) & 1u) { any_dd = true; continue; }
+      gap = fmin(gap, min_threshold_gap(A.atoms[o]));
+    }
+    if (gap > C.tmax) gap = C.tmax / 8.0;
+    if (any_dd) gap = fmin(gap, C.tmax / 48.0);           // a data-derived table: assume a finer grid
+    int e = (int)floor(log2(gap * 0.999));
+    double h = ldexp(1.0, e);
+    const double reach = 1.25 * C.tmax;                    // scale rounding can push |u| a little above tmax
+    while (2 * (int)ceil(reach / h) + 1 > 257) h *= 2.0;   // bound the table size
+    C.c_half = (int)ceil(reach / h);
+    C.invh2 = (float)(0.5 / h);
+    rows = rows > 2 * C.c_half + 1 ? rows : 2 * C.c_half + 1;
+  }
+  P->rows = rows;
+  P->a_pad = n | 1;
+  // slots: pair-type first (singles as (a, a)), then signed
+  int ns = 0;
+  for (int a = 0; a < n; ++a) { P->slots[ns].type = 0; P->slots[ns].i0 = P->slots[ns].i1 = (unsigned char)a; ++ns; }
+  for (int a = 0; a < n; ++a)
+    for (int b = a + 1; b < n; ++b) {
+      if (A.atoms[a].kind != SOP_KIND_LUT || A.atoms[b].kind != SOP_KIND_LUT || A.atoms[a].n_bits != A.atoms[b].n_bits) continue;
+      P->slots[ns].type = 0; P->slots[ns].i0 = (unsigned char)a; P->slots[ns].i1 = (unsigned char)b; ++ns;
+    }
+  P->n_pair_slots = ns;
+  if (F.sign_bits) {
+    bool base[SOP_MAX_ATOMS];
+    for (int i = 0; i < n; ++i) {
+      base[i] = false;
+      if (i + 1 >= n) continue;
+      const sop_atom &a = A.atoms[i], &b = A.atoms[i + 1];
+      if (a.kind != SOP_KIND_LUT || b.kind != SOP_KIND_LUT || a.negated || !b.negated || a.tmax != b.tmax) continue;
+      const bool da = (A.dd_mask >> i) & 1u, db = (A.dd_mask >> (i + 1)) & 1u;
+      base[i] = (da && db && a.n_entries == b.n_entries) || (!da && !db && same_table(a, b));
+    }
+    for (int i = 0; i < n; ++i)
+      for (int j = i; j < n; ++j) {
+        if (!base[i] || !base[j] || A.atoms[i].n_bits != A.atoms[j].n_bits) continue;
+        P->slots[ns].type = 1; P->slots[ns].i0 = (unsigned char)i; P->slots[ns].i1 = (unsigned char)j; ++ns;
+      }
+  }
+  if (ns > MAX_SLOTS) return SOP_ERR_ALPHABET;
+  P->n_slots = ns;
+  return SOP_OK;
+}
+
+size_t sweep_smem_bytes(const Plan& P) {
+  size_t b = (size_t)P.n_tables * P.rows * 32 * 4;
+  b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
+  size_t tile = (size_t)TB * P.a_pad * sizeof(float2);
+  const size_t red = sizeof(Partial) * (size_t)TB;
+  b += tile > red ? tile : red;
+  return (b + 15) & ~(size_t)15;
+}
+
+// optional timing of the sweep kernel alone (CUDA events on the launching stream)
+static bool g_profile = false;
+static cudaEvent_t g_ev0 = nullptr, g_ev1 = nullptr;
+static bool g_ev_valid = false;
+
+static int g_num_sms = 0;
+int num_sms() {
+  if (!g_num_sms) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    g_num_sms = n;
+  }
+  return g_num_sms;
+}
+
+}  // namespace sop
+
+extern "C" {
+
+int sop_profile_enable(int on) {
+  sop::g_profile = on != 0;
+  sop::g_ev_valid = false;
+  return SOP_OK;
+}
+
+int sop_profile_last_sweep_ms(float* ms) {
+  if (!ms) return SOP_ERR_NULL;
+  if (!sop::g_ev_valid) return SOP_ERR_RANGE;
+  SOP_CUDA_TRY(cudaEventSynchronize(sop::g_ev1));
+  SOP_CUDA_TRY(cudaEventElapsedTime(ms, sop::g_ev0, sop::g_ev1));
+  return SOP_OK;
+}
+
+int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes) {
+  if (!bytes) return SOP_ERR_NULL;
+  if (M < 1 || K < 1 || (K % SOP_G) != 0) return SOP_ERR_SHAPE;
+  if (n_atoms < 1 || n_atoms > SOP_MAX_ATOMS) return SOP_ERR_ALPHABET;
+  *bytes = sop::ws_total();
+  return SOP_OK;
+}
+
+int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+                    const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
+                    const float* dd_lut_dev, unsigned dd_mask,
+                    sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
+                    sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
+                    void* workspace_dev, size_t workspace_bytes, void* stream) {
+  using namespace sop;
+  int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
+  if (rc) return rc;
+  if (!pair_table_dev || !result_dev) return SOP_ERR_NULL;
+  FmtDev F;
+  if ((rc = validate_fmt(fmt, &F))) return rc;
+  AtomsDev A;
+  if ((rc = validate_atoms(atoms, n_atoms, dd_mask, dd_lut_dev, &A))) return rc;
+  if (k_mode != SOP_K_AUTO && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < ws_total()) return SOP_ERR_WORKSPACE;
+  Plan P;
+  if ((rc = build_plan(A, F, k_mode, &P))) return rc;
+
+  LayerArgs L;
+  L.W = (const uint16_t*)W_dev; L.c = c_dev; L.M = M; L.K = K; L.ldw = ldw; L.nbk = K / SOP_G; L.NB = M * L.nbk;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned char* ws = (unsigned char*)workspace_dev;
+  WsHeader* hdr = (WsHeader*)ws;
+  unsigned* hist = (unsigned*)(ws + ws_hist_off());
+  Partial* partials = (Partial*)(ws + ws_part_off());
+
+  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
+  bool need_prepass = false;
+  for (int c = 0; c < P.n_classes; ++c) need_prepass |= P.cls[c].auto_k || P.cls[c].scope == 0;
+  const int sms = num_sms();
+  {
+    // max|W| is part of the result block, so the prepass always runs; it is a single read of W
+    (void)need_prepass;
+    long long want = (L.NB + 255) / 256;
+    const int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
+    prepass_kernel<<<grid, 256, 0, st>>>(L, P, hist, hdr);
+    SOP_CUDA_TRY(cudaGetLastError());
+  }
+  kselect_kernel<<<1, 160, 0, st>>>(P, F, hist, hdr, result_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+
+  const size_t smem = sweep_smem_bytes(P);
+  if (smem > 227 * 1024) return SOP_ERR_ALPHABET;
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    smem_set = 227 * 1024;
+  }
+  // persistent grid: one CTA per SM, fewer when the layer is small; at least enough threads for one row
+  long long grid = (L.NB + TB - 1) / TB;
+  if (grid > sms) grid = sms;
+  const long long min_grid = (L.nbk + TB - 1) / TB;
+  if (grid < min_grid) grid = min_grid;
+  if (grid > MAX_GRID) return SOP_ERR_SHAPE;
+  if (g_profile) {
+    if (!g_ev0) { SOP_CUDA_TRY(cudaEventCreate(&g_ev0)); SOP_CUDA_TRY(cudaEventCreate(&g_ev1)); }
+    SOP_CUDA_TRY(cudaEventRecord(g_ev0, st));
+  }
+  sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+  if (g_profile) { SOP_CUDA_TRY(cudaEventRecord(g_ev1, st)); g_ev_valid = true; }
+  finalize_kernel<<<1, MAX_SLOTS, 0, st>>>(L, P, F, (int)grid, partials, pair_table_dev, signed_table_dev, result_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
+  return SOP_OK;
+}
+
+}  // extern "C"

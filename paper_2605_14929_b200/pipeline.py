@@ -1,0 +1,120 @@
+"""The per-layer hot path as a sequence of C-ABI calls on one stream, with no host round trip
+in between: channel norms -> sweep of the ROM alphabet (finds FMTa and its per-block cosines) ->
+DD-n Lloyd refinement -> sweep of the full alphabet (ROM atoms, DD-n, negations, FP singles) ->
+pack of the chosen pair.  This module only allocates buffers and orders the calls.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs as I
+
+
+def scale_word_container(fmt, need_sign: bool, need_selector: bool) -> int:
+    """Smallest container b in {8, 12, 16} holding sign + exponent + mantissa + selector."""
+    need = fmt.exp_bits + fmt.man_bits + (1 if need_sign else 0) + (1 if need_selector else 0)
+    for b in (8, 12, 16):
+        if b >= need:
+            return b
+    raise ValueError("scale word does not fit 16 bits")
+
+
+@dataclasses.dataclass
+class SweepOutputs:
+    c: torch.Tensor
+    pair_table: np.ndarray
+    signed_table: np.ndarray
+    result: dict
+    rom_result: dict
+    dd_lut: np.ndarray
+    distortion: np.ndarray
+    pool_count: int
+    codes: torch.Tensor
+    words: torch.Tensor
+    counts: np.ndarray
+    atoms: List[I.Atom]
+
+
+class LayerSweep:
+    """Buffers and call order for one layer shape.  ``rom`` are base ROM atom names; every ROM atom
+    is followed by its negation; ``fp`` are FP singles; ``lloyd_iters`` = 0 disables the DD atom."""
+
+    def __init__(self, M: int, K: int, T: int, fmt: I.ScaleFormat, rom: Sequence[str], fp: Sequence[str] = (),
+                 lloyd_iters: int = 8, pool_percent: float = 50.0, device="cuda", want_blocks: bool = False):
+        self.M, self.K, self.T, self.fmt = M, K, T, fmt
+        self.dev = torch.device(device)
+        self.iters = lloyd_iters
+        self.rom_atoms = I.alphabet(rom, with_negations=True)
+        n_bits = self.rom_atoms[0].n_bits
+        self.full_atoms = list(self.rom_atoms)
+        self.dd_mask = 0
+        if lloyd_iters > 0:
+            dd = I.Atom(f"DD{n_bits}", n_bits, I.KIND_LUT, 0, I.SCOPE_BLOCK, 1.0, np.zeros(1 << n_bits, np.float32))
+            self.dd_mask = (1 << len(self.full_atoms)) | (1 << (len(self.full_atoms) + 1))
+            self.full_atoms += [dd, dd.negation()]
+        self.full_atoms += [I.fp_atom(f) for f in fp]
+        self.NB = M * (K // 16)
+        self.pool_rank = int(math.ceil(self.NB * (100.0 - pool_percent) / 100.0))
+        self.pool_rank = max(1, min(self.NB, self.pool_rank))
+        nR, nF = len(self.rom_atoms), len(self.full_atoms)
+        d = self.dev
+        self.c = torch.empty(K, dtype=torch.float32, device=d)
+        self.ws_norm = B.alloc_workspace(B.channel_norms_workspace(T, K), d)
+        self.ws_search = B.alloc_workspace(B.pair_search_workspace(M, K, nF), d)
+        self.ws_lloyd = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), d)
+        self.rom_table = B.new_pair_table(nR, d)
+        self.rom_result = B.new_result(d)
+        self.block_cos = torch.empty((nR, self.NB), dtype=torch.float32, device=d)
+        self.dd_lut = torch.zeros(B.MAX_ENTRIES, dtype=torch.float32, device=d)
+        self.distortion = torch.zeros(max(1, lloyd_iters + 1), dtype=torch.float64, device=d)
+        self.pool_count = torch.zeros(1, dtype=torch.int64, device=d)
+        self.pair_table = B.new_pair_table(nF, d)
+        self.signed_table = B.new_pair_table(nF, d)
+        self.result = B.new_result(d)
+        self.use_sign = 1 if fmt.sign_bits else 0
+        self.container = scale_word_container(fmt, bool(self.use_sign), True)
+        self.codes = torch.empty(self.NB * 2 * n_bits, dtype=torch.uint8, device=d)
+        self.words = torch.empty(B.words_nbytes(self.NB, self.container), dtype=torch.uint8, device=d)
+        self.counts = torch.zeros(2, dtype=torch.int64, device=d)
+        self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d) if want_blocks else None
+        self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d) if want_blocks else None
+        self.kernel_launches_per_step = 0
+
+    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None) -> None:
+        """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32."""
+        n = 0
+        B.sop_channel_norms(X, self.c, self.ws_norm, stream)
+        n += 2
+        if self.iters > 0:
+            B.sop_pair_search(W, self.c, self.fmt, self.rom_atoms, self.rom_table, None, self.rom_result, self.ws_search,
+                              block_cos=self.block_cos, stream=stream)
+            n += 4
+            B.sop_dd4_lloyd(W, self.c, self.fmt, self.rom_atoms, self.block_cos, self.pool_rank, self.iters, self.dd_lut,
+                            self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
+            n += 4 + 2 * (self.iters + 1)
+        B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
+                          self.ws_search, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
+                          block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
+        n += 4
+        B.sop_pack(W, self.c, self.fmt, self.full_atoms, self.codes, self.words, search_result=self.result,
+                   use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
+                   counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask, stream=stream)
+        n += 1
+        self.kernel_launches_per_step = n
+
+    def outputs(self) -> SweepOutputs:
+        torch.cuda.synchronize(self.dev)
+        nF, nR = len(self.full_atoms), len(self.rom_atoms)
+        return SweepOutputs(
+            c=self.c.cpu(), pair_table=B.read_pair_table(self.pair_table, nF),
+            signed_table=B.read_pair_table(self.signed_table, nF), result=B.read_result(self.result),
+            rom_result=B.read_result(self.rom_result) if self.iters > 0 else {},
+            dd_lut=self.dd_lut.cpu().numpy(), distortion=self.distortion.cpu().numpy(),
+            pool_count=int(self.pool_count.item()), codes=self.codes.cpu(), words=self.words.cpu(),
+            counts=self.counts.cpu().numpy(), atoms=self.full_atoms)

@@ -1,0 +1,112 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and rejects bad arguments on the host before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2605_14929_b200 import binding as B
+from paper_2605_14929_b200 import build as libbuild
+from paper_2605_14929_b200 import inputs as I
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    libbuild.build()
+    return B.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "sop.h")).read()
+    declared = set(re.findall(r"\b(sop_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(B.exported_symbols())
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.sop_version() >= 100
+
+
+def test_struct_layouts_match_header():
+    assert C.sizeof(B.AtomStruct) == 6 * 4 + 32 * 4
+    assert C.sizeof(B.PairStat) == 32 and B.PAIR_DTYPE.itemsize == 32
+    assert C.sizeof(B.SearchResult) == 16 * 4 + 5 * 4 + 4 + 8
+    assert C.sizeof(B.ScaleFmt) == 20
+
+
+def test_error_text(lib):
+    for code in range(0, -8, -1):
+        assert len(lib.sop_strerror(code)) > 1
+    assert b"unknown" in lib.sop_strerror(-99)
+
+
+FAKE = C.c_void_p(0x10000)     # never dereferenced: every call below fails validation first
+
+
+def _search(lib, M=4, K=64, ldw=64, g=16, fmt=None, atoms=None, n=None, k=B.K_AUTO, W=FAKE, ws=FAKE, wsb=1 << 30,
+            dd=None, mask=0):
+    fmt = fmt or I.scale_format("UE4M4")
+    atoms = atoms if atoms is not None else I.alphabet(["NF4"])
+    n = len(atoms) if n is None else n
+    return lib.sop_pair_search(W, C.c_longlong(M), C.c_longlong(K), C.c_longlong(ldw), FAKE, g, C.byref(B.make_fmt(fmt)), k,
+                               B.make_atoms(atoms), n, dd, C.c_uint(mask), FAKE, None, FAKE, None, None, ws,
+                               C.c_size_t(wsb), None)
+
+
+def test_pair_search_rejects_bad_arguments(lib):
+    assert _search(lib, W=None) == -1
+    assert _search(lib, K=60, ldw=60) == -2            # K % 16
+    assert _search(lib, M=0) == -2
+    assert _search(lib, ldw=32) == -2                  # ld < K
+    assert _search(lib, g=32) == -2
+    assert _search(lib, W=C.c_void_p(0x10004)) == -2   # W not 16-byte aligned
+    bad = I.ScaleFormat("bad", 0, 9, 3, 7)
+    assert _search(lib, fmt=bad) == -3
+    assert _search(lib, fmt=I.ScaleFormat("bad", 0, 8, 7, 127, 0)) == -3   # largest scale not finite in fp32
+    assert _search(lib, n=0) == -4 and _search(lib, n=17) == -4
+    a = I.rom_atom("NF4")
+    a.lut = a.lut[::-1].copy()
+    assert _search(lib, atoms=[a]) == -4               # unsorted table
+    a = I.rom_atom("NF4")
+    a.tmax = 0.0
+    assert _search(lib, atoms=[a]) == -4
+    a = I.fp_atom("E2M3")
+    a.n_bits = 5
+    assert _search(lib, atoms=[a]) == -4
+    assert _search(lib, k=65) == -7
+    assert _search(lib, ws=None) == -5 and _search(lib, wsb=16) == -5
+    assert _search(lib, ws=C.c_void_p(0x10010)) == -5  # workspace not 256-byte aligned
+    assert _search(lib, mask=1) == -1                  # dd_mask without a device table
+    assert _search(lib, mask=4, dd=FAKE) == -4         # mask bit beyond the alphabet
+
+
+def test_other_entry_points_reject_bad_arguments(lib):
+    ll = C.c_longlong
+    n = C.c_size_t()
+    assert lib.sop_channel_norms_workspace(ll(0), ll(8), C.byref(n)) == -2
+    assert lib.sop_channel_norms_workspace(ll(130), ll(8), C.byref(n)) == 0 and n.value == 3 * 8 * 8
+    assert lib.sop_channel_norms(None, ll(4), ll(8), ll(8), FAKE, FAKE, C.c_size_t(1 << 20), None) == -1
+    assert lib.sop_channel_norms(FAKE, ll(4), ll(8), ll(4), FAKE, FAKE, C.c_size_t(1 << 20), None) == -2
+    assert lib.sop_channel_norms(FAKE, ll(4), ll(8), ll(8), FAKE, FAKE, C.c_size_t(8), None) == -5
+    fmt = C.byref(B.make_fmt(I.scale_format("UE4M4")))
+    atoms = I.alphabet(["NF4", "SH4"])
+    arr = B.make_atoms(atoms)
+
+    def lloyd(rank=1, iters=8, k=0, fmta=0, res=None):
+        return lib.sop_dd4_lloyd(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, k, res, FAKE, ll(rank), arr, len(atoms), fmta,
+                                 iters, FAKE, FAKE, FAKE, FAKE, C.c_size_t(1 << 20), None)
+    assert lloyd(rank=0) == -7 and lloyd(rank=17) == -7 and lloyd(iters=65) == -7 and lloyd(k=99) == -7
+    assert lloyd(fmta=9) == -7
+    assert lloyd(k=B.K_FROM_RESULT) == -1 and lloyd(fmta=B.FMTA_FROM_RESULT) == -1
+
+    def pack(ia=0, ib=2, k=0, sign=0, b=12, wsb=0, res=None, f=fmt):
+        return lib.sop_pack(FAKE, ll(4), ll(64), ll(64), FAKE, 16, f, arr, len(atoms), None, C.c_uint(0), ia, ib, k, res,
+                            sign, b, wsb, FAKE, FAKE, None, None)
+    assert pack(b=8) == -3                  # UE4M4 in 8 bits has no metabit for the selector
+    assert pack(b=10) == -3
+    assert pack(sign=1, wsb=0) == -3        # sign requested, word has no sign bit
+    assert pack(ia=5) == -7 and pack(ib=7) == -7
+    assert pack(ia=B.PAIR_FROM_RESULT) == -1
+    assert pack(k=B.K_FROM_RESULT) == -1
