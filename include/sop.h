@@ -171,8 +171,8 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
  *     index_a = SOP_PAIR_FROM_RESULT takes the pair from search_dev (best_sa/best_sb when use_sign,
  *     else best_a/best_b) so that the whole layer pipeline runs without a host round trip.
  *   k_mode: a shift in [-64, 64] used for both atoms, or SOP_K_FROM_RESULT (search_dev->k[index]).
- *   codes_dev: N_b * 2n bytes; block payload = one little-endian 16n-bit integer, element r in bits
- *     [r n, r n + n).  LUT atoms: table index (for a negated table: the index found on -u);
+ *   codes_dev: N_b * 2n bytes, 16-byte aligned; block payload = one little-endian 16n-bit integer,
+ *     element r in bits [r n, r n + n).  LUT atoms: table index (for a negated table: the index found on -u);
  *     FP atoms: the format's bit pattern sign|E|M.
  *   words_dev: ceil(N_b * container_bits / 8) bytes, rounded up to a multiple of 4 (the stream is
  *     written with 32-bit operations; the pointer must be 4-byte aligned), little-endian bit stream

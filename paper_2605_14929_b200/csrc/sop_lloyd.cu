@@ -2,13 +2,19 @@
 // that the primary codebook reconstructs worst.
 //
 //   select_kernel<PASS>   three-pass radix select (11 + 11 + 10 bits) of the pool_rank-th smallest
-//                         block cosine; each pass re-derives the prefix from the previous histogram.
+//                         block cosine; each pass re-derives the prefix from the previous histograms
+//                         with a CTA-wide scan.
 //   lloyd_setup_kernel    threshold tau and pool count from the last histogram, max(c), the shift k,
-//                         the initial table (FMTa, reversed and negated if FMTa is a negated atom).
+//                         the initial table (FMTa, reversed and negated if FMTa is a negated atom),
+//                         and the per-channel weight tables omega = c / max(c) and fix(omega).
+//   pool_list_kernel      compacts the indices of the pool blocks (cos <= tau) into a dense list, so
+//                         that every lane of the iteration kernel has work.
 //   lloyd_iter_kernel     one thread per pool block: u = w / scale, nearest entry by binary search
-//                         over exact thresholds, per-entry int64 fixed-point sums (exactly
-//                         associative, so atomics reproduce a sequential sum bit for bit), FP64 distortion.
-//   lloyd_update_kernel   centroids -> bf16 -> sort; clears the accumulators.
+//                         over exact thresholds, per-entry int64 fixed-point sums kept in
+//                         thread-private shared-memory slots (no atomics in the element loop; the sums
+//                         are exactly associative, so any order reproduces a sequential sum bit for
+//                         bit), FP64 distortion.  The CTA that finishes last turns the sums into
+//                         centroids, snaps them to bf16, sorts, and clears the accumulators.
 #include <math.h>
 #include <string.h>
 
@@ -17,6 +23,7 @@
 namespace sop {
 
 constexpr int LTB = 256;
+constexpr int SETUP_TB = 1024;
 
 struct LloydWs {
   // radix select state
@@ -31,6 +38,8 @@ struct LloydWs {
   int k;
   int fmta;
   int n_entries;
+  unsigned done;         // CTAs of the running iteration that have added their sums
+  unsigned list_count;   // blocks appended to the pool list
   int pad;
   long long pool_count;
 };
@@ -38,11 +47,21 @@ struct LloydWs {
 struct LloydArgs {
   const uint16_t* W;
   const float* c;
-  const float* cosrow_base;   // [n_atoms x NB] or [NB]
+  const float* cosrow_base;   // [n_atoms x NB]
   long long M, K, ldw, nbk, NB;
   long long pool_rank;
   int k_mode, fmta_index, n_atoms;
+  float* omega;               // workspace: K floats, c / max(c)
+  unsigned* omega_fix;        // workspace: K words, round(omega * 2^24)
+  unsigned* pool_idx;         // workspace: NB words, indices of the pool blocks
 };
+
+static size_t lloyd_off_omega() { return (sizeof(LloydWs) + 255) & ~(size_t)255; }
+static size_t lloyd_off_fix(long long K) { return lloyd_off_omega() + (((size_t)K * 4 + 255) & ~(size_t)255); }
+static size_t lloyd_off_idx(long long K) { return lloyd_off_fix(K) + (((size_t)K * 4 + 255) & ~(size_t)255); }
+static size_t lloyd_ws_bytes(long long M, long long K) {
+  return lloyd_off_idx(K) + ((((size_t)M * (size_t)(K / SOP_G)) * 4 + 255) & ~(size_t)255);
+}
 
 __device__ __forceinline__ unsigned cos_key(float x) {
   const unsigned b = __float_as_uint(__fadd_rn(x, 0.0f));   // -0 -> +0
@@ -54,32 +73,57 @@ __device__ __forceinline__ int resolve_fmta(const LloydArgs& a, const sop_search
   return max(0, min(a.n_atoms - 1, f));
 }
 
-// After pass p the selected element lies in bin sel[p] of hist[p]; rank is the rank inside that bin.
-// Recomputed by every CTA from the histograms (a 2048-entry scan): cheaper than one more launch.
-__device__ void derive_prefix(const LloydWs* ws, long long pool_rank, int passes, unsigned* prefix, long long* rank_out,
-                              long long* below_out, unsigned* last_count) {
-  __shared__ long long s_rank, s_below;
-  __shared__ unsigned s_prefix, s_cnt;
-  if (threadIdx.x == 0) {
-    long long rank = pool_rank, below = 0;
-    unsigned pre = 0, cnt = 0;
-    for (int p = 0; p < passes; ++p) {
-      const int nb = p < 2 ? 2048 : 1024;
-      long long run = 0;
-      int b = 0;
-      for (; b < nb; ++b) {
-        const unsigned h = ws->hist[p][b];
-        if (run + h >= rank) { cnt = h; break; }
-        run += h;
-      }
-      rank -= run;
-      below += run;
-      pre = (pre << (p < 2 ? 11 : 10)) | (unsigned)b;
+// CTA-wide (a multiple of 32 threads, at most 1024): the bin of `hist` (nb <= 2048 bins) holding the
+// element of 1-based rank `rank`; *before = elements in lower bins, *count = elements in that bin.
+__device__ void find_bin(const unsigned* __restrict__ hist, int nb, long long rank, int* bin, long long* before, unsigned* count) {
+  __shared__ long long s_warp[32];
+  __shared__ int s_bin;
+  __shared__ long long s_before;
+  __shared__ unsigned s_cnt;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  const int per = (nb + nt - 1) / nt;
+  const int b0 = tid * per;
+  long long local = 0;
+  for (int i = 0; i < per; ++i)
+    if (b0 + i < nb) local += hist[b0 + i];
+  long long incl = local;
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  long long base = 0;
+  for (int w = 0; w < warp; ++w) base += s_warp[w];
+  const long long excl = base + incl - local;
+  if (local > 0 && excl < rank && rank <= excl + local) {
+    long long run = excl;
+    for (int i = 0; i < per; ++i) {
+      const unsigned h = hist[b0 + i];
+      if (run + h >= rank) { s_bin = b0 + i; s_before = run; s_cnt = h; break; }
+      run += h;
     }
-    s_rank = rank; s_below = below; s_prefix = pre; s_cnt = cnt;
   }
   __syncthreads();
-  *prefix = s_prefix; *rank_out = s_rank; *below_out = s_below; *last_count = s_cnt;
+  *bin = s_bin; *before = s_before; *count = s_cnt;
+  __syncthreads();
+}
+
+// After pass p the selected element lies in one bin of hist[p]; the key prefix, the rank inside
+// that bin and the number of elements below it follow from the histograms of the passes so far.
+__device__ void derive_prefix(const LloydWs* ws, long long pool_rank, int passes, unsigned* prefix, long long* rank_out,
+                              long long* below_out, unsigned* last_count) {
+  long long rank = pool_rank, below = 0;
+  unsigned pre = 0, cnt = 0;
+  for (int p = 0; p < passes; ++p) {
+    int bin;
+    long long before;
+    find_bin(ws->hist[p], p < 2 ? 2048 : 1024, rank, &bin, &before, &cnt);
+    rank -= before;
+    below += before;
+    pre = (pre << (p < 2 ? 11 : 10)) | (unsigned)bin;
+  }
+  *prefix = pre; *rank_out = rank; *below_out = below; *last_count = cnt;
 }
 
 template <int PASS>
@@ -90,7 +134,7 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
   long long rank, below;
   if (PASS > 0) derive_prefix(ws, a.pool_rank, PASS, &prefix, &rank, &below, &cnt);
   __syncthreads();
-  const float* row = a.cosrow_base + (a.n_atoms > 0 ? (size_t)resolve_fmta(a, res) * a.NB : 0);
+  const float* row = a.cosrow_base + (size_t)resolve_fmta(a, res) * a.NB;
   for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += (long long)gridDim.x * LTB) {
     const unsigned key = cos_key(__ldg(row + i));
     if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
@@ -102,19 +146,29 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
     if (sh[i]) atomicAdd(&ws->hist[PASS][i], sh[i]);
 }
 
-__global__ void __launch_bounds__(LTB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
-                                                          LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
+__global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
+                                                               LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
   unsigned prefix, cnt;
   long long rank, below;
   derive_prefix(ws, a.pool_rank, 3, &prefix, &rank, &below, &cnt);
-  __shared__ float red[LTB];
+  __shared__ float red[SETUP_TB / 32];
+  __shared__ float s_cmax;
   float mx = 0.0f;
-  for (long long i = threadIdx.x; i < a.K; i += LTB) mx = fmaxf(mx, __ldg(a.c + i));
-  red[threadIdx.x] = mx;
+  for (long long i = threadIdx.x; i < a.K; i += SETUP_TB) mx = fmaxf(mx, __ldg(a.c + i));
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
   __syncthreads();
-  for (int s = LTB / 2; s; s >>= 1) {
-    if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
-    __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = red[0];
+    for (int w = 1; w < SETUP_TB / 32; ++w) t = fmaxf(t, red[w]);
+    s_cmax = t;
+  }
+  __syncthreads();
+  const float cmax = s_cmax;
+  for (long long i = threadIdx.x; i < a.K; i += SETUP_TB) {
+    const float om = cmax > 0.0f ? __fdiv_rn(__ldg(a.c + i), cmax) : 0.0f;
+    a.omega[i] = om;
+    a.omega_fix[i] = (unsigned)__float2ll_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]: at most 2^24
   }
   if (threadIdx.x == 0) {
     const unsigned key = prefix;   // full 32-bit key after three passes
@@ -122,7 +176,7 @@ __global__ void __launch_bounds__(LTB) lloyd_setup_kernel(LloydArgs a, AtomsDev 
     ws->tau = __uint_as_float(b);
     ws->pool_count = below + cnt;
     *pool_count_out = below + cnt;
-    ws->cmax = red[0];
+    ws->cmax = cmax;
     const int f = resolve_fmta(a, res);
     ws->fmta = f;
     ws->k = a.k_mode == SOP_K_FROM_RESULT ? res->k[f] : a.k_mode;
@@ -141,115 +195,155 @@ __global__ void __launch_bounds__(LTB) lloyd_setup_kernel(LloydArgs a, AtomsDev 
     }
     for (int j = 0; j < SOP_MAX_ENTRIES; ++j) { ws->accN[j] = 0; ws->accS[j] = 0; }
     ws->accD = 0.0;
+    ws->done = 0;
+    ws->list_count = 0;
   }
 }
 
-__global__ void __launch_bounds__(LTB) lloyd_iter_kernel(LloydArgs a, FmtDev F, const sop_search_result* __restrict__ res,
-                                                         LloydWs* __restrict__ ws, int accumulate_sums) {
+// Dense list of the pool blocks.  The order of the list depends on the scheduling of the warps;
+// nothing downstream depends on it (integer sums, and an FP64 sum compared with a tolerance).
+__global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __restrict__ ws) {
+  const float tau = ws->tau;
+  const float* row = a.cosrow_base + (size_t)ws->fmta * a.NB;
+  const int lane = threadIdx.x & 31;
+  const long long stride = (long long)gridDim.x * LTB;
+  const long long n_round = (a.NB + stride - 1) / stride;
+  long long i = (long long)blockIdx.x * LTB + threadIdx.x;
+  for (long long r = 0; r < n_round; ++r, i += stride) {
+    const bool in = i < a.NB && __ldg(row + i) <= tau;
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, in);
+    if (!bal) continue;
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(&ws->list_count, (unsigned)__popc(bal));
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    if (in) a.pool_idx[base + __popc(bal & ((1u << lane) - 1u))] = (unsigned)i;
+  }
+}
+
+// replace non-empty entries by their centroids snapped to bf16 (ties to even), sort ascending
+__device__ void lloyd_update(LloydWs* ws, double* __restrict__ distortion, int it, int last, float* __restrict__ out_lut) {
+  volatile LloydWs* v = ws;
+  distortion[it] = v->accD;
+  const int ne = v->n_entries;
+  if (!last) {
+    float t[SOP_MAX_ENTRIES];
+    for (int j = 0; j < ne; ++j) {
+      t[j] = v->lut[j];
+      const unsigned long long n = v->accN[j];
+      if (n) {
+        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn(v->accS[j]), __ull2double_rn(n)));
+        uint32_t b = __float_as_uint(cen);
+        b += 0x7FFFu + ((b >> 16) & 1u);
+        b &= 0xFFFF0000u;                      // nearest bf16, ties to even
+        t[j] = __uint_as_float(b);
+      }
+    }
+    for (int i = 1; i < ne; ++i) {             // insertion sort, ascending
+      const float x = t[i];
+      int p = i - 1;
+      while (p >= 0 && t[p] > x) { t[p + 1] = t[p]; --p; }
+      t[p + 1] = x;
+    }
+    for (int j = 0; j < ne; ++j) v->lut[j] = t[j];
+  } else {
+    for (int j = 0; j < SOP_MAX_ENTRIES; ++j) out_lut[j] = j < ne ? v->lut[j] : 0.0f;
+  }
+  for (int j = 0; j < SOP_MAX_ENTRIES; ++j) { v->accN[j] = 0; v->accS[j] = 0; }
+  v->accD = 0.0;
+  v->done = 0;
+}
+
+__global__ void __launch_bounds__(LTB) lloyd_iter_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                         int it, int last, float* __restrict__ out_lut) {
+  extern __shared__ __align__(16) unsigned char lsm[];
+  ulonglong2* acc = reinterpret_cast<ulonglong2*>(lsm);    // [n_entries][blockDim.x]: (sum fix(omega), sum fix(omega u))
   __shared__ float lutv[32], tau[32];
-  __shared__ unsigned long long sN[LTB / 32][SOP_MAX_ENTRIES];
-  __shared__ unsigned long long sS[LTB / 32][SOP_MAX_ENTRIES];
   __shared__ double sD[LTB / 32];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  __shared__ int s_is_last;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, BD = blockDim.x;
   const int ne = ws->n_entries;
   if (tid < 32) lutv[tid] = ws->lut[min(tid, ne - 1)];
-  for (int i = tid; i < (LTB / 32) * SOP_MAX_ENTRIES; i += LTB) { (&sN[0][0])[i] = 0; (&sS[0][0])[i] = 0; }
+  if (!last)
+    for (int i = tid; i < ne * BD; i += BD) acc[i] = make_ulonglong2(0ull, 0ull);
   __syncthreads();
   if (tid == 0) build_thresholds(lutv, ne, tau);
   __syncthreads();
-  const float cos_tau = ws->tau, cmax = ws->cmax;
   const int k = ws->k;
-  const float* row = a.cosrow_base + (a.n_atoms > 0 ? (size_t)ws->fmta * a.NB : 0);
+  const unsigned count = ws->list_count;
+  const unsigned nbk = (unsigned)a.nbk;
+  ulonglong2* mine = acc + tid;
 
-  const long long GT = (long long)gridDim.x * LTB;
-  const long long R = GT / a.nbk;
-  const long long gt = (long long)blockIdx.x * LTB + tid;
-  const bool lane_on = gt < R * a.nbk;
-  const long long j = lane_on ? gt % a.nbk : 0;
-  const long long r0 = gt / a.nbk;
-  float om[16];
-  long long fixw[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const float cv = __ldg(a.c + j * SOP_G + i);
-    om[i] = cmax > 0.0f ? __fdiv_rn(cv, cmax) : 0.0f;
-    fixw[i] = __float2ll_rn(__fmul_rn(om[i], 16777216.0f));
-  }
   double D = 0.0;
-  if (lane_on) {
-    for (long long m = r0; m < a.M; m += R) {
-      const long long blk = m * a.nbk + j;
-      if (!(__ldg(row + blk) <= cos_tau)) continue;
-      const uint4* p = reinterpret_cast<const uint4*>(a.W + m * a.ldw + j * SOP_G);
-      const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
-      const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-      uint32_t mb = 0;
+  for (unsigned i = blockIdx.x * BD + tid; i < count; i += gridDim.x * BD) {
+    const unsigned blk = a.pool_idx[i];
+    const unsigned m = blk / nbk, j = blk - m * nbk;
+    const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
+    const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+    const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    float om[16];
+    unsigned fx[16];
+    {
+      const float4* op = reinterpret_cast<const float4*>(a.omega + (size_t)j * SOP_G);
+      const uint4* fp = reinterpret_cast<const uint4*>(a.omega_fix + (size_t)j * SOP_G);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
-      const float amax = __uint_as_float(mb << 16);
-      const float s_hat = scale_quantize(amax, k, F).s_hat;    // a DD table declares tmax = 1
-      const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+      for (int q = 0; q < 4; ++q) {
+        const float4 o = __ldg(op + q);
+        const uint4 f = __ldg(fp + q);
+        om[4 * q] = o.x; om[4 * q + 1] = o.y; om[4 * q + 2] = o.z; om[4 * q + 3] = o.w;
+        fx[4 * q] = f.x; fx[4 * q + 1] = f.y; fx[4 * q + 2] = f.z; fx[4 * q + 3] = f.w;
+      }
+    }
+    uint32_t mb = 0;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const float w = (i & 1) ? bf16hi(wb[i >> 1]) : bf16lo(wb[i >> 1]);
-        const float u = __fmul_rn(w, rcp);
-        const int code = count_below(tau, u);
-        const double d = (double)u - (double)lutv[code];
-        D += ((double)om[i] * d) * d;
-        if (accumulate_sums) {
-          const float ou = fminf(fmaxf(__fmul_rn(om[i], u), -256.0f), 256.0f);
-          atomicAdd(&sN[warp][code], (unsigned long long)fixw[i]);
-          atomicAdd(&sS[warp][code], (unsigned long long)__float2ll_rn(__fmul_rn(ou, 16777216.0f)));
-        }
+    for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
+    const float amax = __uint_as_float(mb << 16);
+    const float s_hat = scale_quantize(amax, k, F).s_hat;    // a DD table declares tmax = 1
+    const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const float w = (e & 1) ? bf16hi(wb[e >> 1]) : bf16lo(wb[e >> 1]);
+      const float u = __fmul_rn(w, rcp);
+      const int code = count_below(tau, u);
+      const double d = (double)u - (double)lutv[code];
+      D += ((double)om[e] * d) * d;
+      if (!last) {
+        const float ou = fminf(fmaxf(__fmul_rn(om[e], u), -256.0f), 256.0f);
+        ulonglong2 t = mine[code * BD];
+        t.x += (unsigned long long)fx[e];
+        t.y += (unsigned long long)__float2ll_rn(__fmul_rn(ou, 16777216.0f));
+        mine[code * BD] = t;
       }
     }
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
   if (lane == 0) sD[warp] = D;
   __syncthreads();
-  if (tid < ne && accumulate_sums) {
-    unsigned long long n = 0, s = 0;
-    for (int w = 0; w < LTB / 32; ++w) { n += sN[w][tid]; s += sS[w][tid]; }
-    if (n) atomicAdd(&ws->accN[tid], n);
-    if (s) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[tid]), s);
+  const int n_warps = BD >> 5;
+  if (!last) {
+    for (int j = warp; j < ne; j += n_warps) {
+      unsigned long long n = 0, s = 0;
+      for (int q = lane; q < BD; q += 32) { const ulonglong2 t = acc[j * BD + q]; n += t.x; s += t.y; }
+      for (int o = 16; o; o >>= 1) { n += __shfl_xor_sync(0xFFFFFFFFu, n, o); s += __shfl_xor_sync(0xFFFFFFFFu, s, o); }
+      if (lane == 0) {
+        if (n) atomicAdd(&ws->accN[j], n);
+        if (s) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[j]), s);
+      }
+    }
   }
   if (tid == 0) {
     double t = 0.0;
-    for (int w = 0; w < LTB / 32; ++w) t += sD[w];
+    for (int w = 0; w < n_warps; ++w) t += sD[w];
     if (t != 0.0) atomicAdd(&ws->accD, t);
   }
-}
-
-__global__ void lloyd_update_kernel(LloydWs* __restrict__ ws, double* __restrict__ distortion, int it, int last,
-                                    float* __restrict__ out_lut) {
-  if (threadIdx.x != 0) return;
-  distortion[it] = ws->accD;
-  const int ne = ws->n_entries;
-  if (!last) {
-    float v[SOP_MAX_ENTRIES];
-    for (int j = 0; j < ne; ++j) {
-      v[j] = ws->lut[j];
-      const unsigned long long n = ws->accN[j];
-      if (n) {
-        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn(ws->accS[j]), __ull2double_rn(n)));
-        uint32_t b = __float_as_uint(cen);
-        b += 0x7FFFu + ((b >> 16) & 1u);
-        b &= 0xFFFF0000u;                      // nearest bf16, ties to even
-        v[j] = __uint_as_float(b);
-      }
-    }
-    for (int i = 1; i < ne; ++i) {             // insertion sort, ascending
-      const float x = v[i];
-      int p = i - 1;
-      while (p >= 0 && v[p] > x) { v[p + 1] = v[p]; --p; }
-      v[p + 1] = x;
-    }
-    for (int j = 0; j < ne; ++j) ws->lut[j] = v[j];
-  } else {
-    for (int j = 0; j < SOP_MAX_ENTRIES; ++j) out_lut[j] = j < ne ? ws->lut[j] : 0.0f;
+  // the CTA that arrives last owns the update; no CTA waits for another
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_is_last = atomicAdd(&ws->done, 1u) == gridDim.x - 1 ? 1 : 0;
+  __syncthreads();
+  if (s_is_last && tid == 0) {
+    __threadfence();
+    lloyd_update(ws, distortion, it, last, out_lut);
   }
-  for (int j = 0; j < SOP_MAX_ENTRIES; ++j) { ws->accN[j] = 0; ws->accS[j] = 0; }
-  ws->accD = 0.0;
 }
 
 int num_sms();
@@ -261,7 +355,8 @@ extern "C" {
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
   if (M < 1 || K < 1 || (K % SOP_G) != 0) return SOP_ERR_SHAPE;
-  *bytes = (sizeof(sop::LloydWs) + 255) & ~(size_t)255;
+  if (M > (1ll << 31) / (K / SOP_G)) return SOP_ERR_SHAPE;
+  *bytes = sop::lloyd_ws_bytes(M, K);
   return SOP_OK;
 }
 
@@ -289,10 +384,14 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   sop_dd4_lloyd_workspace(M, K, &need);
   if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < need) return SOP_ERR_WORKSPACE;
 
+  unsigned char* wsb = (unsigned char*)workspace_dev;
   LloydArgs a;
   a.W = (const uint16_t*)W_dev; a.c = c_dev; a.cosrow_base = block_cos_dev;
   a.M = M; a.K = K; a.ldw = ldw; a.nbk = K / SOP_G; a.NB = NB; a.pool_rank = pool_rank;
   a.k_mode = k_mode; a.fmta_index = fmta_index; a.n_atoms = n_atoms;
+  a.omega = (float*)(wsb + lloyd_off_omega());
+  a.omega_fix = (unsigned*)(wsb + lloyd_off_fix(K));
+  a.pool_idx = (unsigned*)(wsb + lloyd_off_idx(K));
   LloydWs* ws = (LloydWs*)workspace_dev;
   cudaStream_t st = (cudaStream_t)stream;
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(LloydWs), st));
@@ -304,16 +403,29 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   select_kernel<1><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
   select_kernel<2><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
   SOP_CUDA_TRY(cudaGetLastError());
-  lloyd_setup_kernel<<<1, LTB, 0, st>>>(a, A, search_dev, ws, pool_count_dev);
+  lloyd_setup_kernel<<<1, SETUP_TB, 0, st>>>(a, A, search_dev, ws, pool_count_dev);
   SOP_CUDA_TRY(cudaGetLastError());
-  long long grid = (NB + LTB - 1) / LTB;
-  if (grid > (long long)sms * 4) grid = (long long)sms * 4;
-  const long long min_grid = (a.nbk + LTB - 1) / LTB;
-  if (grid < min_grid) grid = min_grid;
+  pool_list_kernel<<<(int)sg, LTB, 0, st>>>(a, ws);
+  SOP_CUDA_TRY(cudaGetLastError());
+
+  // iteration kernel: the per-thread accumulator slots bound the threads per SM (16 bytes x entries x threads)
+  int max_entries = 2;
+  for (int i = 0; i < n_atoms; ++i)
+    if (atoms[i].kind == SOP_KIND_LUT && atoms[i].n_entries > max_entries) max_entries = atoms[i].n_entries;
+  const int bd = max_entries <= 16 ? 256 : 128;
+  const size_t smem = (size_t)max_entries * bd * sizeof(ulonglong2);
+  static size_t smem_set = 0;
+  if (smem > 48 * 1024 && smem > smem_set) {
+    SOP_CUDA_TRY(cudaFuncSetAttribute(lloyd_iter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+    smem_set = 128 * 1024;
+  }
+  const int per_sm = (int)((200 * 1024) / (smem + 2048));
+  long long grid = (NB + bd - 1) / bd;
+  if (grid > (long long)sms * per_sm) grid = (long long)sms * per_sm;
+  if (grid < 1) grid = 1;
   for (int it = 0; it <= iters; ++it) {
     const int last = it == iters;
-    lloyd_iter_kernel<<<(int)grid, LTB, 0, st>>>(a, F, search_dev, ws, last ? 0 : 1);
-    lloyd_update_kernel<<<1, 32, 0, st>>>(ws, distortion_dev, it, last, out_lut_dev);
+    lloyd_iter_kernel<<<(int)grid, bd, smem, st>>>(a, F, ws, distortion_dev, it, last, out_lut_dev);
   }
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;

@@ -23,40 +23,33 @@ struct PackArgs {
 
 struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
 
-// scalar evaluation of one candidate on one block; same operation order as the sweep kernel
-__device__ void eval_block_scalar(const float* w, const float* c, const float* tau, const float* lutv, const PackCand& cd,
-                                  const FmtDev& F, float pot, float& cos_out, uint32_t& scode, int* codes) {
-  float amax = 0.0f;
-  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(w[i]));
-  float s_hat;
-  scode = 0;
-  if (cd.scope == 0) {
-    s_hat = amax > 0.0f ? pot : 0.0f;
-  } else {
-    const float sigma = cd.tmax == 1.0f ? amax : __fdiv_rn(amax, cd.tmax);
-    const QScale qs = scale_quantize(sigma, cd.k, F);
-    s_hat = qs.s_hat;
-    scode = qs.code;
-  }
-  const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+// One candidate on one block, everything in registers; same operation order as the sweep kernel.
+// The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
+__device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
+                                                const float* __restrict__ lutv, int kind, int neg, float rcp,
+                                                float& cos_out, uint32_t (&code4)[4]) {
   float qn[4], qd[4], qw[4];
+#pragma unroll
   for (int h = 0; h < 4; ++h) {
     float an = 0.0f, ad = 0.0f, aw = 0.0f;
+    uint32_t packed = 0;
+#pragma unroll
     for (int r = 0; r < 4; ++r) {
       const int i = 4 * h + r;
       const float u = __fmul_rn(w[i], rcp);
       float q;
-      if (cd.kind == SOP_KIND_LUT) {
-        const int code = count_below(tau, cd.neg ? -u : u);
-        codes[i] = code;
-        q = cd.neg ? -lutv[code] : lutv[code];
-      } else if (cd.kind == SOP_KIND_FP_E2M3) {
+      uint32_t code;
+      if (kind == SOP_KIND_LUT) {
+        code = (uint32_t)count_below(tau, neg ? -u : u);
+        q = neg ? -lutv[code] : lutv[code];
+      } else if (kind == SOP_KIND_FP_E2M3) {
         q = fp_quantize<SOP_KIND_FP_E2M3>(u);
-        codes[i] = (int)fp_code<SOP_KIND_FP_E2M3>(q);
+        code = fp_code<SOP_KIND_FP_E2M3>(q);
       } else {
         q = fp_quantize<SOP_KIND_FP_E4M3>(u);
-        codes[i] = (int)fp_code<SOP_KIND_FP_E4M3>(q);
+        code = fp_code<SOP_KIND_FP_E4M3>(q);
       }
+      packed |= code << (8 * r);
       const float cw = __fmul_rn(c[i], w[i]);
       const float cq = __fmul_rn(c[i], q);
       aw = __fmaf_rn(cw, w[i], aw);
@@ -64,6 +57,7 @@ __device__ void eval_block_scalar(const float* w, const float* c, const float* t
       an = __fmaf_rn(cq, q, an);
     }
     qn[h] = an; qd[h] = ad; qw[h] = aw;
+    code4[h] = packed;
   }
   cos_out = block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd));
 }
@@ -102,6 +96,7 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
   }
   __syncthreads();
   const int nb = s_nb, n = s_nbits, b = a.container_bits;
+  const int n_sign = a.use_sign ? 2 : 1;
   unsigned my_sel = 0, my_neg = 0;
   for (long long blk = (long long)blockIdx.x * PTB + tid; blk < a.NB; blk += (long long)gridDim.x * PTB) {
     const long long m = blk / a.nbk, j = blk - m * a.nbk;
@@ -109,31 +104,55 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
     const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     float w[16], c[16];
+#pragma unroll
     for (int i = 0; i < 8; ++i) { w[2 * i] = bf16lo(wb[i]); w[2 * i + 1] = bf16hi(wb[i]); }
-    for (int i = 0; i < 16; ++i) c[i] = __ldg(a.c + j * SOP_G + i);
+    {
+      const float4* cp = reinterpret_cast<const float4*>(a.c + j * SOP_G);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = __ldg(cp + q);
+        c[4 * q] = v.x; c[4 * q + 1] = v.y; c[4 * q + 2] = v.z; c[4 * q + 3] = v.w;
+      }
+    }
+    uint32_t mb = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
+    const float amax = __uint_as_float(mb << 16);
     float best_cos = 0.0f;
-    uint32_t best_scode = 0;
-    int best_codes[16], pick = -1;
-    for (int t = 0; t < nb; ++t)
-      for (int sg = 0; sg < (a.use_sign ? 2 : 1); ++sg) {
-        PackCand cd = base[t];
-        if (sg) cd.neg = 1 - cd.neg;
+    uint32_t best_scode = 0, best4[4] = {0u, 0u, 0u, 0u};
+    int pick = -1;
+    for (int t = 0; t < nb; ++t) {
+      const PackCand cd = base[t];
+      float s_hat;
+      uint32_t sc = 0;
+      if (cd.scope == 0) {
+        s_hat = amax > 0.0f ? s_pot[t] : 0.0f;
+      } else {
+        const float sigma = cd.tmax == 1.0f ? amax : __fdiv_rn(amax, cd.tmax);
+        const QScale qs = scale_quantize(sigma, cd.k, F);
+        s_hat = qs.s_hat;
+        sc = qs.code;
+      }
+      const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+      for (int sg = 0; sg < n_sign; ++sg) {
         float cs;
-        uint32_t sc;
-        int codes[16];
-        eval_block_scalar(w, c, tau[t], lutv[t], cd, F, s_pot[t], cs, sc, codes);
+        uint32_t c4[4];
+        eval_block_regs(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, cs, c4);
         if (pick < 0 || cs > best_cos) {
           best_cos = cs; best_scode = sc; pick = 2 * t + sg;
-          for (int i = 0; i < 16; ++i) best_codes[i] = codes[i];
+#pragma unroll
+          for (int h = 0; h < 4; ++h) best4[h] = c4[h];
         }
       }
+    }
     const unsigned sel = pick >> 1, sgn = pick & 1;
     my_sel += sel; my_neg += sgn;
-    // codes: 16 n-bit fields, little-endian, 2n bytes = n 16-bit stores
+    // codes: 16 n-bit fields, little-endian, 2n bytes
     unsigned long long lo = 0, hi = 0;   // 128-bit accumulator
+#pragma unroll
     for (int i = 0; i < 16; ++i) {
       const int pos = i * n;
-      const unsigned long long v = (unsigned long long)best_codes[i];
+      const unsigned long long v = (unsigned long long)((best4[i >> 2] >> (8 * (i & 3))) & 0xFFu);
       if (pos < 64) {
         lo |= v << pos;
         if (pos + n > 64) hi |= v >> (64 - pos);
@@ -142,7 +161,13 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
       }
     }
     unsigned short* dst = reinterpret_cast<unsigned short*>(a.codes + blk * 2 * n);
-    for (int i = 0; i < n; ++i) dst[i] = (unsigned short)((i < 4 ? lo >> (16 * i) : hi >> (16 * (i - 4))) & 0xFFFFu);
+    if (n == 4) {
+      *reinterpret_cast<uint2*>(dst) = make_uint2((unsigned)lo, (unsigned)(lo >> 32));
+    } else if (n == 8) {
+      *reinterpret_cast<uint4*>(dst) = make_uint4((unsigned)lo, (unsigned)(lo >> 32), (unsigned)hi, (unsigned)(hi >> 32));
+    } else {
+      for (int i = 0; i < n; ++i) dst[i] = (unsigned short)((i < 4 ? lo >> (16 * i) : hi >> (16 * (i - 4))) & 0xFFFFu);
+    }
     // scale word
     unsigned word;
     if (a.word_sign_bits) word = (sgn << (b - 1)) | (best_scode << a.meta_bits) | (a.meta_bits >= 1 ? sel : 0u);
@@ -206,7 +231,7 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   bool need_wmax = false;
   for (int i = 0; i < n_atoms; ++i) need_wmax |= atoms[i].scope == 0;
   if (need_wmax && !search_dev) return SOP_ERR_NULL;  // the layer power-of-two scale comes from a previous search
-  if (((uintptr_t)codes_dev & 1u) || ((uintptr_t)words_dev & 3u)) return SOP_ERR_SHAPE;
+  if (((uintptr_t)codes_dev & 15u) || ((uintptr_t)words_dev & 3u)) return SOP_ERR_SHAPE;
   // every atom that can be picked must share n_bits with the first LUT atom when the pair comes from the device
   int n_bits = from_result ? 0 : atoms[index_a].n_bits;
   if (from_result) {

@@ -113,16 +113,19 @@ __global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, unsig
 __global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const unsigned* __restrict__ hist, WsHeader* __restrict__ hdr,
                                                       sop_search_result* __restrict__ res) {
   __shared__ unsigned long long cnt[129];
+  __shared__ unsigned sh_hist[SOP_HIST_BINS];
   const float wmax = __uint_as_float(hdr->wmax_bits);
   for (int cl = 0; cl < P.n_classes; ++cl) {
     int kstar = P.k_mode == SOP_K_AUTO ? 0 : P.k_mode;
     if (P.cls[cl].scope == 0) kstar = 0;
     if (P.cls[cl].auto_k) {
+      for (int i = threadIdx.x; i < SOP_HIST_BINS; i += blockDim.x) sh_hist[i] = hist[cl * SOP_HIST_BINS + i];
+      __syncthreads();
       if (threadIdx.x < 129) {
         const int k = (int)threadIdx.x - 64;
         unsigned long long c = 0;
         for (int e = -SOP_HIST_OFF; e < SOP_HIST_BINS - SOP_HIST_OFF; ++e)
-          if (e + k >= F.emin && e + k <= F.emax) c += hist[cl * SOP_HIST_BINS + e + SOP_HIST_OFF];
+          if (e + k >= F.emin && e + k <= F.emax) c += sh_hist[e + SOP_HIST_OFF];
         cnt[threadIdx.x] = c;
       }
       __syncthreads();
@@ -479,41 +482,59 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   }
 }
 
-__global__ void __launch_bounds__(MAX_SLOTS) finalize_kernel(LayerArgs L, Plan P, FmtDev F, int grid, const Partial* __restrict__ partials,
-                                                             sop_pair_stat* __restrict__ pair_table, sop_pair_stat* __restrict__ signed_table,
-                                                             sop_search_result* __restrict__ res) {
-  const int A = P.n_atoms, tid = threadIdx.x;
+constexpr int FIN_TB = 1024;
+
+// One warp per slot: lane l adds the partials of CTAs l, l + 32, ... in that order, then the lanes
+// are combined by a fixed butterfly: the result depends only on the grid size, not on scheduling.
+// The tables are staged in shared memory so that the final scan for the best pair reads no global memory.
+__global__ void __launch_bounds__(FIN_TB) finalize_kernel(LayerArgs L, Plan P, FmtDev F, int grid, const Partial* __restrict__ partials,
+                                                          sop_pair_stat* __restrict__ pair_table, sop_pair_stat* __restrict__ signed_table,
+                                                          sop_search_result* __restrict__ res) {
+  __shared__ sop_pair_stat s_pair[SOP_MAX_ATOMS * SOP_MAX_ATOMS], s_sig[SOP_MAX_ATOMS * SOP_MAX_ATOMS];
+  const int A = P.n_atoms, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < A * A; i += blockDim.x) {
     sop_pair_stat u; u.acos = 0.0; u.mse = 0.0; u.n_sel1 = -1; u.n_neg = -1;
-    pair_table[i] = u;
-    if (signed_table) signed_table[i] = u;
+    s_pair[i] = u;
+    s_sig[i] = u;
   }
   __syncthreads();
-  if (tid < P.n_slots) {
-    Partial t = partials[tid];
-    for (int g = 1; g < grid; ++g) {
-      const Partial q = partials[(size_t)g * MAX_SLOTS + tid];
+  for (int slot = warp; slot < P.n_slots; slot += FIN_TB / 32) {
+    Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
+    for (int g = lane; g < grid; g += 32) {
+      const Partial q = partials[(size_t)g * MAX_SLOTS + slot];
       t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
     }
-    sop_pair_stat s;
-    s.acos = ((double)L.NB - t.gap) / (double)L.NB;
-    s.mse = t.sse / ((double)L.M * (double)L.K);
-    s.n_sel1 = t.n1;
-    const SlotDev sd = P.slots[tid];
-    if (sd.type == 0) { s.n_neg = 0; pair_table[sd.i0 * A + sd.i1] = s; }
-    else if (signed_table) { s.n_neg = t.nneg; signed_table[sd.i0 * A + sd.i1] = s; }
+    for (int o = 16; o; o >>= 1) {
+      t.gap += __shfl_xor_sync(0xFFFFFFFFu, t.gap, o);
+      t.sse += __shfl_xor_sync(0xFFFFFFFFu, t.sse, o);
+      t.n1 += __shfl_xor_sync(0xFFFFFFFFu, t.n1, o);
+      t.nneg += __shfl_xor_sync(0xFFFFFFFFu, t.nneg, o);
+    }
+    if (lane == 0) {
+      sop_pair_stat st;
+      st.acos = ((double)L.NB - t.gap) / (double)L.NB;
+      st.mse = t.sse / ((double)L.M * (double)L.K);
+      st.n_sel1 = t.n1;
+      const SlotDev sd = P.slots[slot];
+      if (sd.type == 0) { st.n_neg = 0; s_pair[sd.i0 * A + sd.i1] = st; }
+      else { st.n_neg = t.nneg; s_sig[sd.i0 * A + sd.i1] = st; }
+    }
   }
   __syncthreads();
+  for (int i = tid; i < A * A; i += blockDim.x) {
+    pair_table[i] = s_pair[i];
+    if (signed_table) signed_table[i] = s_sig[i];
+  }
   if (tid == 0) {
     int ba = -1, bb = -1, bs = -1, bsa = -1, bsb = -1;
     double vp = -2.0, vs = -2.0, vsp = -2.0;
     for (int a = 0; a < A; ++a) {
-      if (P.cand[a].kind == SOP_KIND_LUT && pair_table[a * A + a].acos > vs) { vs = pair_table[a * A + a].acos; bs = a; }
+      if (P.cand[a].kind == SOP_KIND_LUT && s_pair[a * A + a].acos > vs) { vs = s_pair[a * A + a].acos; bs = a; }
       for (int b = a + 1; b < A; ++b) {
-        const sop_pair_stat p = pair_table[a * A + b];
+        const sop_pair_stat p = s_pair[a * A + b];
         if (p.n_sel1 >= 0 && p.acos > vp) { vp = p.acos; ba = a; bb = b; }
         if (signed_table) {
-          const sop_pair_stat q = signed_table[a * A + b];
+          const sop_pair_stat q = s_sig[a * A + b];
           if (q.n_sel1 >= 0 && q.acos > vsp) { vsp = q.acos; bsa = a; bsb = b; }
         }
       }
@@ -751,7 +772,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   if (g_profile) { SOP_CUDA_TRY(cudaEventRecord(g_ev1, st)); g_ev_valid = true; }
-  finalize_kernel<<<1, MAX_SLOTS, 0, st>>>(L, P, F, (int)grid, partials, pair_table_dev, signed_table_dev, result_dev);
+  finalize_kernel<<<1, FIN_TB, 0, st>>>(L, P, F, (int)grid, partials, pair_table_dev, signed_table_dev, result_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }
