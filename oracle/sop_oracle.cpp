@@ -231,8 +231,10 @@ BlockEval eval_block(const float* w, const float* c, const Atom& a, const ScaleF
     cq[i] = c[i] * r.q[i];
     err[i] = std::fmaf(-r.s_hat, r.q[i], w[i]);
   }
+  // <a, b>_c = sum_i c_i a_i b_i; association (paper silent): <w, w> as (c w) w, <q, q> as (c q) q,
+  // <w, q> as (c q) w
   const float nw = quad_tree_dot(cw, w);
-  const float dot = quad_tree_dot(cw, r.q);
+  const float dot = quad_tree_dot(cq, w);
   const float nq = quad_tree_dot(cq, r.q);
   r.sse = quad_tree_dot(err, err);
   // zero norms (paper silent): both zero -> 1, exactly one zero -> 0

@@ -53,7 +53,7 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
       const float cw = __fmul_rn(c[i], w[i]);
       const float cq = __fmul_rn(c[i], q);
       aw = __fmaf_rn(cw, w[i], aw);
-      ad = __fmaf_rn(cw, q, ad);
+      ad = __fmaf_rn(cq, w[i], ad);
       an = __fmaf_rn(cq, q, an);
     }
     qn[h] = an; qd[h] = ad; qw[h] = aw;

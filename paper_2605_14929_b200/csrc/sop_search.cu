@@ -26,7 +26,7 @@ constexpr float MAGIC = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an inte
 struct CandDev { unsigned char cls, kind, neg, table; };
 struct ClassDev {
   float tmax;
-  float invh2;       // cells per unit of u2 = 2u (power of two)
+  float invh;        // cells per unit of u (a power of two)
   int scope, kind;   // kind of the quantiser: LUT, E2M3, E4M3
   int c_half;        // table rows = 2 * c_half + 1
   int auto_k;        // 1: k* from the histogram
@@ -38,6 +38,7 @@ struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (
 struct Plan {
   int n_atoms, n_classes, n_tables, n_slots, n_pair_slots;
   int k_mode, rows, a_pad;
+  int red_t1, red_g0, red_g1;   // phase-2 thread split of a half CTA: [0, t1) pair slots in g0 groups, [t1, 256) signed slots in g1 groups
   CandDev cand[SOP_MAX_ATOMS];
   ClassDev cls[SOP_MAX_CLASSES];
   unsigned char table_atom[SOP_MAX_TABLES];   // atom whose lut fills the table
@@ -159,8 +160,8 @@ __global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const un
 // independent sequential chains, which is exactly the quad-tree summation order.
 // ---------------------------------------------------------------------------------------------
 struct BlockRegs {
-  float2 w[8], c[8], cw[8], u2[8];
-  int r32[16];      // cell row * 32 (word offset into a lane-replicated table), per element
+  float2 w[8], c[8], u[8];
+  int off[16];      // byte offset of the element's cell entry inside a table: row * 128 + (lane & 15) * 8
 };
 
 __device__ __forceinline__ float fold(const float2 a, const float2 b) {
@@ -169,8 +170,11 @@ __device__ __forceinline__ float fold(const float2 a, const float2 b) {
 
 struct Metric { float nq, dot, sse; };
 
+// One cell entry is {threshold, hi bf16 : lo bf16}: the reconstruction value is hi when u lies
+// strictly above the threshold, else lo.  A negated candidate runs the base table on -u (mirrored
+// row) and flips the sign of the dot product and of the scale in the error term.
 template <bool NEG>
-__device__ __forceinline__ Metric eval_lut_cells(const uint32_t* __restrict__ tbl_lane, int mirror, const BlockRegs& B, float s_hat) {
+__device__ __forceinline__ Metric eval_lut_cells(const unsigned char* __restrict__ tp, int moff, const BlockRegs& B, float s_hat) {
   float2 nq[2], dot[2], sse[2];
   nq[0] = nq[1] = dot[0] = dot[1] = sse[0] = sse[1] = make_float2(0.0f, 0.0f);
   const float sg = NEG ? s_hat : -s_hat;
@@ -180,16 +184,16 @@ __device__ __forceinline__ Metric eval_lut_cells(const uint32_t* __restrict__ tb
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
       const int idx = 2 * i + p;
-      const uint32_t wa = tbl_lane[NEG ? mirror - B.r32[2 * idx] : B.r32[2 * idx]];
-      const uint32_t wb = tbl_lane[NEG ? mirror - B.r32[2 * idx + 1] : B.r32[2 * idx + 1]];
-      const float la = bf16lo(wa), ha = bf16hi(wa), lb = bf16lo(wb), hb = bf16hi(wb);
-      const float sa = __fadd_rn(la, ha), sb = __fadd_rn(lb, hb);
+      const uint2 ea = *reinterpret_cast<const uint2*>(tp + (NEG ? moff - B.off[2 * idx] : B.off[2 * idx]));
+      const uint2 eb = *reinterpret_cast<const uint2*>(tp + (NEG ? moff - B.off[2 * idx + 1] : B.off[2 * idx + 1]));
+      const bool pa = NEG ? (-B.u[idx].x > __uint_as_float(ea.x)) : (B.u[idx].x > __uint_as_float(ea.x));
+      const bool pb = NEG ? (-B.u[idx].y > __uint_as_float(eb.x)) : (B.u[idx].y > __uint_as_float(eb.x));
       float2 q;
-      q.x = (NEG ? (-B.u2[idx].x > sa) : (B.u2[idx].x > sa)) ? ha : la;
-      q.y = (NEG ? (-B.u2[idx].y > sb) : (B.u2[idx].y > sb)) ? hb : lb;
+      q.x = __uint_as_float(__byte_perm(ea.y, 0u, pa ? 0x3244u : 0x1044u));
+      q.y = __uint_as_float(__byte_perm(eb.y, 0u, pb ? 0x3244u : 0x1044u));
       const float2 cq = __fmul2_rn(B.c[idx], q);
       nq[p] = __ffma2_rn(cq, q, nq[p]);
-      dot[p] = __ffma2_rn(B.cw[idx], q, dot[p]);
+      dot[p] = __ffma2_rn(cq, B.w[idx], dot[p]);
       const float2 e = __ffma2_rn(ns, q, B.w[idx]);
       sse[p] = __ffma2_rn(e, e, sse[p]);
     }
@@ -214,7 +218,7 @@ __device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, co
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
       const int idx = 2 * i + p;
-      const float ux = __fmul_rn(B.u2[idx].x, 0.5f), uy = __fmul_rn(B.u2[idx].y, 0.5f);
+      const float ux = B.u[idx].x, uy = B.u[idx].y;
       float2 q;
       if (MODE == 0) {
         q.x = lutv[count_below(tau, NEG ? -ux : ux)];
@@ -225,7 +229,7 @@ __device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, co
       }
       const float2 cq = __fmul2_rn(B.c[idx], q);
       nq[p] = __ffma2_rn(cq, q, nq[p]);
-      dot[p] = __ffma2_rn(B.cw[idx], q, dot[p]);
+      dot[p] = __ffma2_rn(cq, B.w[idx], dot[p]);
       const float2 e = __ffma2_rn(ns, q, B.w[idx]);
       sse[p] = __ffma2_rn(e, e, sse[p]);
     }
@@ -238,13 +242,14 @@ __device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, co
   return m;
 }
 
-// Build the shared-memory tables of one CTA: table values and thresholds, then the lane-replicated
-// cell tables.  A cell row r (k = r - c_half) covers the u2 values that round to k:
-// u2 * invh2 in [k - 1/2, k + 1/2]; row 0 and the last row extend to -inf / +inf.  A row is usable
-// when at most one distinct threshold falls inside its closed interval and lo + hi is exact in
-// fp32 (then "u2 > lo + hi" is the exact nearest-entry decision); otherwise the whole table is
-// marked slow and its candidates take the binary-search path.
-__device__ void build_tables(const Plan& P, const AtomsDev& A, uint32_t* cell, float* tau, float* lutv, int* fast) {
+// Build the shared-memory tables of one CTA: table values and thresholds, then the cell tables.
+// A cell row r (k = r - c_half) covers the u values that round to k: u * invh in [k - 1/2, k + 1/2];
+// row 0 and the last row extend to -inf / +inf.  A row is usable when at most one distinct threshold
+// falls inside its closed interval and both neighbouring table values are bf16 numbers (they are
+// stored as one 32-bit pair); otherwise the whole table is marked slow and its candidates take the
+// binary-search path.  Every row is stored 16 times (128 bytes): lanes l and l + 16 read copy l & 15,
+// so a 64-bit load of any 32 rows by a warp is free of bank conflicts.
+__device__ void build_tables(const Plan& P, const AtomsDev& A, uint2* cell, float* tau, float* lutv, int* fast) {
   const int tid = threadIdx.x;
   for (int i = tid; i < P.n_tables * 32; i += blockDim.x) {
     const int t = i >> 5, j = i & 31;
@@ -263,9 +268,9 @@ __device__ void build_tables(const Plan& P, const AtomsDev& A, uint32_t* cell, f
     const ClassDev& C = P.cls[P.table_cls[t]];
     const int ne = A.atoms[P.table_atom[t]].n_entries;
     const int nrow = 2 * C.c_half + 1;
-    uint32_t word = 0;
+    uint2 entry = make_uint2(0x7F800000u, 0u);
     if (r < nrow) {
-      const float hh = __fdiv_rn(0.5f, C.invh2);                    // cell width in u (a power of two)
+      const float hh = __fdiv_rn(1.0f, C.invh);                     // cell width in u (a power of two)
       const float kf = (float)(r - C.c_half);
       const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, hh);
       const float hi_edge = r == nrow - 1 ? INFINITY : __fmul_rn(kf + 0.5f, hh);
@@ -284,33 +289,42 @@ __device__ void build_tables(const Plan& P, const AtomsDev& A, uint32_t* cell, f
       }
       const float lo = lv[nbelow], hi = lv[min(nbelow + ninside, ne - 1)];
       const uint32_t lb = __float_as_uint(lo), hb = __float_as_uint(hi);
-      bool ok = ndistinct <= 1 && (lb & 0xFFFFu) == 0 && (hb & 0xFFFFu) == 0;
-      if (ok && ninside) ok = (double)__fadd_rn(lo, hi) == (double)lo + (double)hi;
+      const bool ok = ndistinct <= 1 && (lb & 0xFFFFu) == 0 && (hb & 0xFFFFu) == 0;
       if (!ok) atomicAnd(&fast[t], 0);
-      word = (hb & 0xFFFF0000u) | (lb >> 16);
+      entry.x = ninside ? __float_as_uint(prev) : 0x7F800000u;
+      entry.y = (hb & 0xFFFF0000u) | (lb >> 16);
     }
-    uint32_t* dst = cell + (size_t)i * 32;
-    for (int l = 0; l < 32; ++l) dst[l] = word;
+    uint2* dst = cell + (size_t)i * 16;
+    for (int l = 0; l < 16; ++l) dst[l] = entry;
   }
   __syncthreads();
 }
 
+__device__ __forceinline__ void half_barrier(int half) {
+  asm volatile("bar.sync %0, %1;" ::"r"(half + 1), "n"(TB / 2) : "memory");
+}
+
+// The CTA works as two halves of 256 threads with a barrier each, so that one half reduces its tile
+// (phase 2) while the other still evaluates candidates (phase 1).
 __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, const WsHeader* __restrict__ hdr,
                                                       Partial* __restrict__ partials, float* __restrict__ block_cos,
                                                       float* __restrict__ block_sse) {
   extern __shared__ __align__(16) unsigned char smem[];
-  uint32_t* cell = reinterpret_cast<uint32_t*>(smem);
-  float* tau = reinterpret_cast<float*>(cell + (size_t)P.n_tables * P.rows * 32);
+  uint2* cell = reinterpret_cast<uint2*>(smem);
+  float* tau = reinterpret_cast<float*>(cell + (size_t)P.n_tables * P.rows * 16);
   float* lutv = tau + SOP_MAX_TABLES * 32;
   int* fast = reinterpret_cast<int*>(lutv + SOP_MAX_TABLES * 32);
   int* cls_k = fast + SOP_MAX_TABLES;
   float* cls_pot = reinterpret_cast<float*>(cls_k + SOP_MAX_CLASSES);
-  float2* cs = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [TB][a_pad] (cos, sse)
+  float2* cs_all = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [2][TB / 2][a_pad] (cos, sse)
 
-  const int tid = threadIdx.x, lane = tid & 31;
+  constexpr int HB = TB / 2;
+  const int tid = threadIdx.x, lane = tid & 31, half = tid / HB, htid = tid - half * HB;
   build_tables(P, A, cell, tau, lutv, fast);
   if (tid < SOP_MAX_CLASSES) { cls_k[tid] = hdr->cls_k[tid]; cls_pot[tid] = hdr->cls_pot[tid]; }
   __syncthreads();
+  const int a_pad = P.a_pad;
+  float2* cs = cs_all + (size_t)half * HB * a_pad;
 
   // thread -> fixed column block j, rows m = r0, r0 + R, ...
   const long long GT = (long long)gridDim.x * TB;
@@ -336,15 +350,21 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       for (int p = 0; p < 2; ++p) B.c[2 * i + p] = make_float2(cc[8 * p + i], cc[8 * p + 4 + i]);
   }
 
-  // phase-2 role of this thread
-  const int n_slots = P.n_slots;
-  const int n_groups = TB / n_slots;
-  const int slot = tid % n_slots, grp = tid / n_slots;
-  const bool red_on = grp < n_groups;
+  // phase-2 role of this thread inside its half: warps are homogeneous (two-way slots in threads
+  // [0, t1), four-way signed slots in [t1, 256)), so the two loop bodies never diverge inside a warp
+  const int n_slots = P.n_slots, n0 = P.n_pair_slots, n1 = n_slots - n0;
+  const bool four_way = htid >= P.red_t1;
+  const int rt = four_way ? htid - P.red_t1 : htid;
+  const int rn = four_way ? n1 : n0;
+  const int n_groups = four_way ? P.red_g1 : P.red_g0;
+  const int grp = rn ? rt / rn : 0;
+  const int slot = rn ? (four_way ? n0 : 0) + rt % rn : 0;
+  const bool red_on = rn > 0 && grp < n_groups;
   const SlotDev sd = P.slots[slot];
   double acc_gap = 0.0, acc_sse = 0.0;
   int acc_n1 = 0, acc_nneg = 0;
-  const int a_pad = P.a_pad;
+  const int copy_off = (lane & 15) * 8;
+  const unsigned char* cell_bytes = reinterpret_cast<const unsigned char*>(cell);
 
   uint32_t wb[8];
   if (lane_on && r0 < L.M) load_block_bits(L.W + r0 * L.ldw + j * SOP_G, wb);
@@ -352,9 +372,9 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   for (long long it = 0; it < n_iter; ++it) {
     const long long m = r0 + it * R;
     const bool on = lane_on && m < L.M;
-    // number of valid threads of this CTA in this iteration (they form a prefix)
-    long long nv = min(L.M - it * R, R) * L.nbk - (long long)blockIdx.x * TB;
-    nv = max(0ll, min((long long)TB, nv));
+    // number of valid threads of this half in this iteration (the valid threads of a CTA form a prefix)
+    long long nv = min(L.M - it * R, R) * L.nbk - (long long)blockIdx.x * TB - (long long)half * HB;
+    nv = max(0ll, min((long long)HB, nv));
     if (on) {
       // ---- unpack, block statistics ----
       float wf[16];
@@ -373,12 +393,12 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-          B.cw[2 * i + p] = __fmul2_rn(B.c[2 * i + p], B.w[2 * i + p]);
-          nw2[p] = __ffma2_rn(B.cw[2 * i + p], B.w[2 * i + p], nw2[p]);
+          const float2 cw = __fmul2_rn(B.c[2 * i + p], B.w[2 * i + p]);
+          nw2[p] = __ffma2_rn(cw, B.w[2 * i + p], nw2[p]);
         }
       const float nw = fold(nw2[0], nw2[1]);
       const long long blk = m * L.nbk + j;
-      float2* my = cs + (size_t)tid * a_pad;
+      float2* my = cs + (size_t)htid * a_pad;
 
       for (int cl = 0; cl < P.n_classes; ++cl) {
         const ClassDev& C = P.cls[cl];
@@ -391,19 +411,20 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         }
         const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
         const float2 r2 = make_float2(rcp, rcp);
-        const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
 #pragma unroll
-        for (int idx = 0; idx < 8; ++idx) {
-          const float2 u = __fmul2_rn(B.w[idx], r2);
-          B.u2[idx] = __fadd2_rn(u, u);
-          if (C.kind == SOP_KIND_LUT) {
-            const float tx = fminf(fmaxf(__fmaf_rn(B.u2[idx].x, C.invh2, toff), tlo), thi);
-            const float ty = fminf(fmaxf(__fmaf_rn(B.u2[idx].y, C.invh2, toff), tlo), thi);
-            B.r32[2 * idx] = (int)(__float_as_uint(tx) - __float_as_uint(MAGIC)) * 32;
-            B.r32[2 * idx + 1] = (int)(__float_as_uint(ty) - __float_as_uint(MAGIC)) * 32;
+        for (int idx = 0; idx < 8; ++idx) B.u[idx] = __fmul2_rn(B.w[idx], r2);
+        if (C.kind == SOP_KIND_LUT) {
+          const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
+          const float invh = C.invh;
+#pragma unroll
+          for (int idx = 0; idx < 8; ++idx) {
+            const float tx = fminf(fmaxf(__fmaf_rn(B.u[idx].x, invh, toff), tlo), thi);
+            const float ty = fminf(fmaxf(__fmaf_rn(B.u[idx].y, invh, toff), tlo), thi);
+            B.off[2 * idx] = (int)(__float_as_uint(tx) - __float_as_uint(MAGIC)) * 128 + copy_off;
+            B.off[2 * idx + 1] = (int)(__float_as_uint(ty) - __float_as_uint(MAGIC)) * 128 + copy_off;
           }
         }
-        const int mirror = 2 * C.c_half * 32;
+        const int moff = 2 * C.c_half * 128 + 2 * copy_off;
         for (int ci = 0; ci < C.n_cand; ++ci) {
           const int a = C.cand[ci];
           const CandDev cd = P.cand[a];
@@ -411,8 +432,8 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
           if (cd.kind == SOP_KIND_LUT) {
             const int t = cd.table;
             if (fast[t]) {
-              const uint32_t* tl = cell + (size_t)t * P.rows * 32 + lane;
-              mt = cd.neg ? eval_lut_cells<true>(tl, mirror, B, s_hat) : eval_lut_cells<false>(tl, mirror, B, s_hat);
+              const unsigned char* tp = cell_bytes + (size_t)t * P.rows * 128;
+              mt = cd.neg ? eval_lut_cells<true>(tp, moff, B, s_hat) : eval_lut_cells<false>(tp, moff, B, s_hat);
             } else {
               mt = cd.neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
                           : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
@@ -429,55 +450,85 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         }
       }
     }
-    __syncthreads();
-    // ---- phase 2: one pair slot per thread, blocks grp, grp + n_groups, ... of the tile ----
+    half_barrier(half);
+    // ---- phase 2: one slot per thread, blocks grp, grp + n_groups, ... of the half's tile; fp32 sums of
+    //      eight gaps 1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
     if (red_on) {
       const int nvi = (int)nv;
-      float cg = 0.0f, ce = 0.0f;
-      int cnt = 0;
-      for (int b = grp; b < nvi; b += n_groups) {
-        const float2* row = cs + (size_t)b * a_pad;
-        float2 sel = row[sd.i0];
-        if (sd.type == 0) {
-          const float2 v = row[sd.i1];
-          const bool mu = v.x > sel.x;
-          if (mu) sel = v;
-          acc_n1 += mu ? 1 : 0;
-        } else {
-          int pick = 0;
-          float2 v = row[sd.i0 + 1];
-          if (v.x > sel.x) { sel = v; pick = 1; }
-          if (sd.i1 != sd.i0) {
-            v = row[sd.i1];
-            if (v.x > sel.x) { sel = v; pick = 2; }
-            v = row[sd.i1 + 1];
-            if (v.x > sel.x) { sel = v; pick = 3; }
+      const float2* base = cs;
+      const int step = n_groups * a_pad;
+      if (!four_way) {
+        const int i0 = sd.i0, i1 = sd.i1;
+        int b = grp;
+        const float2* row = base + (size_t)b * a_pad;
+        for (; b + 7 * n_groups < nvi; b += 8 * n_groups, row += 8 * step) {
+          float cg = 0.0f, ce = 0.0f;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float2 va = row[k * step + i0], vb = row[k * step + i1];
+            const bool mu = vb.x > va.x;
+            const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
+            acc_n1 += mu ? 1 : 0;
+            cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
+            ce = __fadd_rn(ce, se_);
           }
+          acc_gap += (double)cg; acc_sse += (double)ce;
+        }
+        float cg = 0.0f, ce = 0.0f;
+        for (; b < nvi; b += n_groups, row += step) {
+          const float2 va = row[i0], vb = row[i1];
+          const bool mu = vb.x > va.x;
+          const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
+          acc_n1 += mu ? 1 : 0;
+          cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
+          ce = __fadd_rn(ce, se_);
+        }
+        acc_gap += (double)cg; acc_sse += (double)ce;
+      } else {
+        // candidates i0, i0 + 1, i1, i1 + 1 in priority order (i1 == i0: the second pair repeats the first and never wins)
+        const int i0 = sd.i0, i1 = sd.i1;
+        int b = grp;
+        const float2* row = base + (size_t)b * a_pad;
+        float cg = 0.0f, ce = 0.0f;
+        int cnt = 0;
+        for (; b < nvi; b += n_groups, row += step) {
+          const float2 v0 = row[i0], v1 = row[i0 + 1], v2 = row[i1], v3 = row[i1 + 1];
+          const bool p1 = v1.x > v0.x;
+          float sc_ = p1 ? v1.x : v0.x, se_ = p1 ? v1.y : v0.y;
+          int pick = p1 ? 1 : 0;
+          const bool p2 = v2.x > sc_;
+          sc_ = p2 ? v2.x : sc_; se_ = p2 ? v2.y : se_; pick = p2 ? 2 : pick;
+          const bool p3 = v3.x > sc_;
+          sc_ = p3 ? v3.x : sc_; se_ = p3 ? v3.y : se_; pick = p3 ? 3 : pick;
           acc_n1 += pick >> 1;
           acc_nneg += pick & 1;
+          cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
+          ce = __fadd_rn(ce, se_);
+          if (++cnt == 8) {
+            acc_gap += (double)cg; acc_sse += (double)ce;
+            cg = ce = 0.0f; cnt = 0;
+          }
         }
-        cg = __fadd_rn(cg, __fsub_rn(1.0f, sel.x));
-        ce = __fadd_rn(ce, sel.y);
-        if (++cnt == 8) {
-          acc_gap += (double)cg; acc_sse += (double)ce;
-          cg = ce = 0.0f; cnt = 0;
-        }
+        acc_gap += (double)cg; acc_sse += (double)ce;
       }
-      acc_gap += (double)cg; acc_sse += (double)ce;
     }
-    __syncthreads();
+    half_barrier(half);
   }
 
-  // ---- per-CTA partials: groups added in group order by the group-0 thread of each slot ----
-  Partial* sc = reinterpret_cast<Partial*>(cs);
-  if (red_on) { Partial p; p.gap = acc_gap; p.sse = acc_sse; p.n1 = acc_n1; p.nneg = acc_nneg; sc[grp * n_slots + slot] = p; }
+  // ---- per-CTA partials: every phase-2 thread parks its sums; one thread per slot adds them in a fixed order ----
+  __syncthreads();
+  Partial* sc = reinterpret_cast<Partial*>(cs_all);
+  { Partial p; p.gap = acc_gap; p.sse = acc_sse; p.n1 = acc_n1; p.nneg = acc_nneg; sc[tid] = p; }
   __syncthreads();
   if (tid < n_slots) {
-    Partial t = sc[tid];
-    for (int g = 1; g < n_groups; ++g) {
-      const Partial q = sc[g * n_slots + tid];
-      t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
-    }
+    const bool fw = tid >= n0;
+    const int first = fw ? P.red_t1 + (tid - n0) : tid, stride = fw ? n1 : n0, ng = fw ? P.red_g1 : P.red_g0;
+    Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
+    for (int h = 0; h < 2; ++h)
+      for (int g = 0; g < ng; ++g) {
+        const Partial q = sc[h * HB + first + g * stride];
+        t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
+      }
     partials[(size_t)blockIdx.x * MAX_SLOTS + tid] = t;
   }
 }
@@ -580,7 +631,7 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
       cl = P->n_classes++;
       P->cls[cl].scope = a.scope; P->cls[cl].tmax = a.tmax; P->cls[cl].kind = a.kind;
       P->cls[cl].auto_k = (k_mode == SOP_K_AUTO && a.scope != 0) ? 1 : 0;
-      P->cls[cl].invh2 = 1.0f; P->cls[cl].c_half = 0;
+      P->cls[cl].invh = 1.0f; P->cls[cl].c_half = 0;
     }
     ClassDev& C = P->cls[cl];
     C.cand[C.n_cand++] = (unsigned char)i;
@@ -625,7 +676,7 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
     const double reach = 1.25 * C.tmax;                    // scale rounding can push |u| a little above tmax
     while (2 * (int)ceil(reach / h) + 1 > 257) h *= 2.0;   // bound the table size
     C.c_half = (int)ceil(reach / h);
-    C.invh2 = (float)(0.5 / h);
+    C.invh = (float)(1.0 / h);
     rows = rows > 2 * C.c_half + 1 ? rows : 2 * C.c_half + 1;
   }
   P->rows = rows;
@@ -657,11 +708,27 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
   }
   if (ns > MAX_SLOTS) return SOP_ERR_ALPHABET;
   P->n_slots = ns;
+  {
+    // split the 256 threads of a half CTA between two-way and four-way slots in proportion to their work
+    // (a four-way step costs about twice a two-way step), on a warp boundary
+    const int half_threads = TB / 2, n0 = P->n_pair_slots, n1 = ns - n0;
+    int t1 = 0;
+    if (n1 > 0) {
+      t1 = (int)lround((double)half_threads * (2.0 * n1) / (2.0 * n1 + n0) / 32.0) * 32;
+      const int need1 = (n1 + 31) / 32 * 32;
+      if (t1 < need1) t1 = need1;
+      while (half_threads - t1 < n0 && t1 > need1) t1 -= 32;
+      if (half_threads - t1 < n0) return SOP_ERR_ALPHABET;
+    }
+    P->red_t1 = half_threads - t1;
+    P->red_g0 = n0 ? P->red_t1 / n0 : 0;
+    P->red_g1 = n1 ? t1 / n1 : 0;
+  }
   return SOP_OK;
 }
 
 size_t sweep_smem_bytes(const Plan& P) {
-  size_t b = (size_t)P.n_tables * P.rows * 32 * 4;
+  size_t b = (size_t)P.n_tables * P.rows * 16 * 8;
   b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
   size_t tile = (size_t)TB * P.a_pad * sizeof(float2);
   const size_t red = sizeof(Partial) * (size_t)TB;
