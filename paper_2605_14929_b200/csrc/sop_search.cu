@@ -316,15 +316,15 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   int* fast = reinterpret_cast<int*>(lutv + SOP_MAX_TABLES * 32);
   int* cls_k = fast + SOP_MAX_TABLES;
   float* cls_pot = reinterpret_cast<float*>(cls_k + SOP_MAX_CLASSES);
-  float2* cs_all = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [2][TB / 2][a_pad] (cos, sse)
+  float2* cs_all = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [2][n_atoms][HBP] (cos, sse), candidate-major
 
   constexpr int HB = TB / 2;
   const int tid = threadIdx.x, lane = tid & 31, half = tid / HB, htid = tid - half * HB;
   build_tables(P, A, cell, tau, lutv, fast);
   if (tid < SOP_MAX_CLASSES) { cls_k[tid] = hdr->cls_k[tid]; cls_pot[tid] = hdr->cls_pot[tid]; }
   __syncthreads();
-  const int a_pad = P.a_pad;
-  float2* cs = cs_all + (size_t)half * HB * a_pad;
+  constexpr int HBP = HB + 1;   // row pitch: candidates land in different banks
+  float2* cs = cs_all + (size_t)half * P.n_atoms * HBP;
 
   // thread -> fixed column block j, rows m = r0, r0 + R, ...
   const long long GT = (long long)gridDim.x * TB;
@@ -366,8 +366,13 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   const int copy_off = (lane & 15) * 8;
   const unsigned char* cell_bytes = reinterpret_cast<const unsigned char*>(cell);
 
+  // Warp-uniform control flow: every thread evaluates a block in every iteration (a thread without
+  // work re-evaluates a valid block whose results nothing reads), so the class / candidate loops
+  // below are uniform branches.
+  const unsigned fast_mask = __ballot_sync(0xFFFFFFFFu, fast[lane & (SOP_MAX_TABLES - 1)] != 0);
+  const uint16_t* wcol = L.W + j * SOP_G;
   uint32_t wb[8];
-  if (lane_on && r0 < L.M) load_block_bits(L.W + r0 * L.ldw + j * SOP_G, wb);
+  load_block_bits(wcol + min(r0, L.M - 1) * L.ldw, wb);
 
   for (long long it = 0; it < n_iter; ++it) {
     const long long m = r0 + it * R;
@@ -375,14 +380,13 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
     // number of valid threads of this half in this iteration (the valid threads of a CTA form a prefix)
     long long nv = min(L.M - it * R, R) * L.nbk - (long long)blockIdx.x * TB - (long long)half * HB;
     nv = max(0ll, min((long long)HB, nv));
-    if (on) {
+    {
       // ---- unpack, block statistics ----
       float wf[16];
 #pragma unroll
       for (int q = 0; q < 8; ++q) { wf[2 * q] = bf16lo(wb[q]); wf[2 * q + 1] = bf16hi(wb[q]); }
       const float amax = absmax_bits(wb);
-      const long long mn = m + R;
-      if (mn < L.M) load_block_bits(L.W + mn * L.ldw + j * SOP_G, wb);   // prefetch the next row's block
+      load_block_bits(wcol + min(m + R, L.M - 1) * L.ldw, wb);   // prefetch the next row's block
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -398,7 +402,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         }
       const float nw = fold(nw2[0], nw2[1]);
       const long long blk = m * L.nbk + j;
-      float2* my = cs + (size_t)htid * a_pad;
+      float2* my = cs + htid;
 
       for (int cl = 0; cl < P.n_classes; ++cl) {
         const ClassDev& C = P.cls[cl];
@@ -431,7 +435,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
           Metric mt;
           if (cd.kind == SOP_KIND_LUT) {
             const int t = cd.table;
-            if (fast[t]) {
+            if ((fast_mask >> t) & 1u) {
               const unsigned char* tp = cell_bytes + (size_t)t * P.rows * 128;
               mt = cd.neg ? eval_lut_cells<true>(tp, moff, B, s_hat) : eval_lut_cells<false>(tp, moff, B, s_hat);
             } else {
@@ -444,9 +448,9 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
             mt = eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat);
           }
           const float cosv = block_cosine(nw, mt.nq, mt.dot);
-          my[a] = make_float2(cosv, mt.sse);
-          if (block_cos) block_cos[(size_t)a * L.NB + blk] = cosv;
-          if (block_sse) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+          my[a * HBP] = make_float2(cosv, mt.sse);
+          if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
+          if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
         }
       }
     }
@@ -455,17 +459,17 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
     //      eight gaps 1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
     if (red_on) {
       const int nvi = (int)nv;
-      const float2* base = cs;
-      const int step = n_groups * a_pad;
+      const int len = (nvi + n_groups - 1) / n_groups;     // group g takes blocks [g len, (g + 1) len) of the tile
+      const int lo = grp * len, hi = min(nvi, lo + len);
       if (!four_way) {
-        const int i0 = sd.i0, i1 = sd.i1;
-        int b = grp;
-        const float2* row = base + (size_t)b * a_pad;
-        for (; b + 7 * n_groups < nvi; b += 8 * n_groups, row += 8 * step) {
+        const float2* pa = cs + sd.i0 * HBP + lo;
+        const float2* pb = cs + sd.i1 * HBP + lo;
+        int b = lo;
+        for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
           float cg = 0.0f, ce = 0.0f;
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const float2 va = row[k * step + i0], vb = row[k * step + i1];
+            const float2 va = pa[k], vb = pb[k];
             const bool mu = vb.x > va.x;
             const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
             acc_n1 += mu ? 1 : 0;
@@ -475,8 +479,8 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
           acc_gap += (double)cg; acc_sse += (double)ce;
         }
         float cg = 0.0f, ce = 0.0f;
-        for (; b < nvi; b += n_groups, row += step) {
-          const float2 va = row[i0], vb = row[i1];
+        for (; b < hi; ++b, ++pa, ++pb) {
+          const float2 va = pa[0], vb = pb[0];
           const bool mu = vb.x > va.x;
           const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
           acc_n1 += mu ? 1 : 0;
@@ -486,13 +490,31 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         acc_gap += (double)cg; acc_sse += (double)ce;
       } else {
         // candidates i0, i0 + 1, i1, i1 + 1 in priority order (i1 == i0: the second pair repeats the first and never wins)
-        const int i0 = sd.i0, i1 = sd.i1;
-        int b = grp;
-        const float2* row = base + (size_t)b * a_pad;
+        const float2* pa = cs + sd.i0 * HBP + lo;
+        const float2* pb = cs + sd.i1 * HBP + lo;
+        int b = lo;
+        for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
+          float cg = 0.0f, ce = 0.0f;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float2 v0 = pa[k], v1 = pa[HBP + k], v2 = pb[k], v3 = pb[HBP + k];
+            const bool p1 = v1.x > v0.x;
+            float sc_ = p1 ? v1.x : v0.x, se_ = p1 ? v1.y : v0.y;
+            int pick = p1 ? 1 : 0;
+            const bool p2 = v2.x > sc_;
+            sc_ = p2 ? v2.x : sc_; se_ = p2 ? v2.y : se_; pick = p2 ? 2 : pick;
+            const bool p3 = v3.x > sc_;
+            sc_ = p3 ? v3.x : sc_; se_ = p3 ? v3.y : se_; pick = p3 ? 3 : pick;
+            acc_n1 += pick >> 1;
+            acc_nneg += pick & 1;
+            cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
+            ce = __fadd_rn(ce, se_);
+          }
+          acc_gap += (double)cg; acc_sse += (double)ce;
+        }
         float cg = 0.0f, ce = 0.0f;
-        int cnt = 0;
-        for (; b < nvi; b += n_groups, row += step) {
-          const float2 v0 = row[i0], v1 = row[i0 + 1], v2 = row[i1], v3 = row[i1 + 1];
+        for (; b < hi; ++b, ++pa, ++pb) {
+          const float2 v0 = pa[0], v1 = pa[HBP], v2 = pb[0], v3 = pb[HBP];
           const bool p1 = v1.x > v0.x;
           float sc_ = p1 ? v1.x : v0.x, se_ = p1 ? v1.y : v0.y;
           int pick = p1 ? 1 : 0;
@@ -504,10 +526,6 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
           acc_nneg += pick & 1;
           cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
           ce = __fadd_rn(ce, se_);
-          if (++cnt == 8) {
-            acc_gap += (double)cg; acc_sse += (double)ce;
-            cg = ce = 0.0f; cnt = 0;
-          }
         }
         acc_gap += (double)cg; acc_sse += (double)ce;
       }
@@ -730,7 +748,7 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
 size_t sweep_smem_bytes(const Plan& P) {
   size_t b = (size_t)P.n_tables * P.rows * 16 * 8;
   b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
-  size_t tile = (size_t)TB * P.a_pad * sizeof(float2);
+  size_t tile = (size_t)2 * P.n_atoms * (TB / 2 + 1) * sizeof(float2);
   const size_t red = sizeof(Partial) * (size_t)TB;
   b += tile > red ? tile : red;
   return (b + 15) & ~(size_t)15;
