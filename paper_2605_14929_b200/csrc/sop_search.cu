@@ -43,6 +43,9 @@ struct Plan {
   ClassDev cls[SOP_MAX_CLASSES];
   unsigned char table_atom[SOP_MAX_TABLES];   // atom whose lut fills the table
   unsigned char table_cls[SOP_MAX_TABLES];
+  unsigned char table_pos[SOP_MAX_TABLES];    // candidate that uses the table as it is (255: none)
+  unsigned char table_neg[SOP_MAX_TABLES];    // candidate that uses the negated table (255: none)
+  unsigned char cls_tables[SOP_MAX_CLASSES];  // bit t: table t belongs to the class
   SlotDev slots[MAX_SLOTS];
 };
 
@@ -161,7 +164,7 @@ __global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const un
 // ---------------------------------------------------------------------------------------------
 struct BlockRegs {
   float2 w[8], c[8], u[8];
-  int off[16];      // byte offset of the element's cell entry inside a table: row * 128 + (lane & 15) * 8
+  unsigned off[16]; // byte offset of the element's cell row: row * (n_tables * 128) + (lane & 15) * 8; table t adds t * 128
 };
 
 __device__ __forceinline__ float fold(const float2 a, const float2 b) {
@@ -174,7 +177,7 @@ struct Metric { float nq, dot, sse; };
 // strictly above the threshold, else lo.  A negated candidate runs the base table on -u (mirrored
 // row) and flips the sign of the dot product and of the scale in the error term.
 template <bool NEG>
-__device__ __forceinline__ Metric eval_lut_cells(const unsigned char* __restrict__ tp, int moff, const BlockRegs& B, float s_hat) {
+__device__ __forceinline__ Metric eval_lut_cells(const unsigned char* __restrict__ tp, unsigned moff, const BlockRegs& B, float s_hat) {
   float2 nq[2], dot[2], sse[2];
   nq[0] = nq[1] = dot[0] = dot[1] = sse[0] = sse[1] = make_float2(0.0f, 0.0f);
   const float sg = NEG ? s_hat : -s_hat;
@@ -248,7 +251,9 @@ __device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, co
 // falls inside its closed interval and both neighbouring table values are bf16 numbers (they are
 // stored as one 32-bit pair); otherwise the whole table is marked slow and its candidates take the
 // binary-search path.  Every row is stored 16 times (128 bytes): lanes l and l + 16 read copy l & 15,
-// so a 64-bit load of any 32 rows by a warp is free of bank conflicts.
+// so a 64-bit load of any 32 rows by a warp is free of bank conflicts.  The tables are interleaved
+// row by row ([row][table][copy]): a thread keeps one offset per element and the table is an
+// immediate displacement of the load.
 __device__ void build_tables(const Plan& P, const AtomsDev& A, uint2* cell, float* tau, float* lutv, int* fast) {
   const int tid = threadIdx.x;
   for (int i = tid; i < P.n_tables * 32; i += blockDim.x) {
@@ -294,7 +299,7 @@ __device__ void build_tables(const Plan& P, const AtomsDev& A, uint2* cell, floa
       entry.x = ninside ? __float_as_uint(prev) : 0x7F800000u;
       entry.y = (hb & 0xFFFF0000u) | (lb >> 16);
     }
-    uint2* dst = cell + (size_t)i * 16;
+    uint2* dst = cell + ((size_t)r * P.n_tables + t) * 16;
     for (int l = 0; l < 16; ++l) dst[l] = entry;
   }
   __syncthreads();
@@ -417,40 +422,74 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         const float2 r2 = make_float2(rcp, rcp);
 #pragma unroll
         for (int idx = 0; idx < 8; ++idx) B.u[idx] = __fmul2_rn(B.w[idx], r2);
+        unsigned moff = 0;
         if (C.kind == SOP_KIND_LUT) {
           const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
           const float invh = C.invh;
+          const unsigned pitch = (unsigned)P.n_tables * 128u;
+          const unsigned cbias = (unsigned)copy_off - __float_as_uint(MAGIC) * pitch;   // modulo 2^32
 #pragma unroll
           for (int idx = 0; idx < 8; ++idx) {
             const float tx = fminf(fmaxf(__fmaf_rn(B.u[idx].x, invh, toff), tlo), thi);
             const float ty = fminf(fmaxf(__fmaf_rn(B.u[idx].y, invh, toff), tlo), thi);
-            B.off[2 * idx] = (int)(__float_as_uint(tx) - __float_as_uint(MAGIC)) * 128 + copy_off;
-            B.off[2 * idx + 1] = (int)(__float_as_uint(ty) - __float_as_uint(MAGIC)) * 128 + copy_off;
+            B.off[2 * idx] = __float_as_uint(tx) * pitch + cbias;
+            B.off[2 * idx + 1] = __float_as_uint(ty) * pitch + cbias;
           }
-        }
-        const int moff = 2 * C.c_half * 128 + 2 * copy_off;
-        for (int ci = 0; ci < C.n_cand; ++ci) {
-          const int a = C.cand[ci];
-          const CandDev cd = P.cand[a];
-          Metric mt;
-          if (cd.kind == SOP_KIND_LUT) {
-            const int t = cd.table;
-            if ((fast_mask >> t) & 1u) {
-              const unsigned char* tp = cell_bytes + (size_t)t * P.rows * 128;
-              mt = cd.neg ? eval_lut_cells<true>(tp, moff, B, s_hat) : eval_lut_cells<false>(tp, moff, B, s_hat);
-            } else {
-              mt = cd.neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
-                          : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
+          moff = 2u * (unsigned)C.c_half * pitch + 2u * (unsigned)copy_off;
+          // tables of this class with a usable cell grid: the table slot is a compile-time displacement
+#pragma unroll
+          for (int T = 0; T < SOP_MAX_TABLES; ++T) {
+            if (T < P.n_tables && P.table_cls[T] == cl && ((fast_mask >> T) & 1u)) {
+              const unsigned char* tp = cell_bytes + T * 128;
+              const int ap = P.table_pos[T], an = P.table_neg[T];
+              if (ap != 255) {
+                const Metric mt = eval_lut_cells<false>(tp, moff, B, s_hat);
+                const float cosv = block_cosine(nw, mt.nq, mt.dot);
+                my[ap * HBP] = make_float2(cosv, mt.sse);
+                if (block_cos && on) block_cos[(size_t)ap * L.NB + blk] = cosv;
+                if (block_sse && on) block_sse[(size_t)ap * L.NB + blk] = mt.sse;
+              }
+              if (an != 255) {
+                const Metric mt = eval_lut_cells<true>(tp, moff, B, s_hat);
+                const float cosv = block_cosine(nw, mt.nq, mt.dot);
+                my[an * HBP] = make_float2(cosv, mt.sse);
+                if (block_cos && on) block_cos[(size_t)an * L.NB + blk] = cosv;
+                if (block_sse && on) block_sse[(size_t)an * L.NB + blk] = mt.sse;
+              }
             }
-          } else if (cd.kind == SOP_KIND_FP_E2M3) {
-            mt = eval_generic<SOP_KIND_FP_E2M3, false>(nullptr, nullptr, B, s_hat);
-          } else {
-            mt = eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat);
           }
-          const float cosv = block_cosine(nw, mt.nq, mt.dot);
-          my[a * HBP] = make_float2(cosv, mt.sse);
-          if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
-          if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+          // tables without a usable cell grid: binary search over the thresholds
+          if (P.cls_tables[cl] & ~fast_mask) {
+            for (int ci = 0; ci < C.n_cand; ++ci) {
+              const int a = C.cand[ci];
+              const int t = P.cand[a].table;
+              if ((fast_mask >> t) & 1u) continue;
+              const Metric mt = P.cand[a].neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
+                                              : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
+              const float cosv = block_cosine(nw, mt.nq, mt.dot);
+              my[a * HBP] = make_float2(cosv, mt.sse);
+              if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
+              if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+            }
+          }
+        } else if (C.kind == SOP_KIND_FP_E2M3) {
+          for (int ci = 0; ci < C.n_cand; ++ci) {
+            const int a = C.cand[ci];
+            const Metric mt = eval_generic<SOP_KIND_FP_E2M3, false>(nullptr, nullptr, B, s_hat);
+            const float cosv = block_cosine(nw, mt.nq, mt.dot);
+            my[a * HBP] = make_float2(cosv, mt.sse);
+            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
+            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+          }
+        } else {
+          for (int ci = 0; ci < C.n_cand; ++ci) {
+            const int a = C.cand[ci];
+            const Metric mt = eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat);
+            const float cosv = block_cosine(nw, mt.nq, mt.dot);
+            my[a * HBP] = make_float2(cosv, mt.sse);
+            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
+            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+          }
         }
       }
     }
@@ -664,6 +703,7 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
       const int o = P->table_atom[q];
       const bool odd = (A.dd_mask >> o) & 1u;
       if (P->table_cls[q] != cl || odd != dd) continue;
+      if ((a.negated ? P->table_neg[q] : P->table_pos[q]) != 255) continue;   // one candidate per table and sign
       if (dd ? (A.atoms[o].n_entries == a.n_entries) : same_table(A.atoms[o], a)) t = q;
     }
     if (t < 0) {
@@ -671,7 +711,10 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
       t = P->n_tables++;
       P->table_atom[t] = (unsigned char)i;
       P->table_cls[t] = (unsigned char)cl;
+      P->table_pos[t] = P->table_neg[t] = 255;
     }
+    (a.negated ? P->table_neg[t] : P->table_pos[t]) = (unsigned char)i;
+    P->cls_tables[cl] |= (unsigned char)(1u << t);
     P->cand[i].table = (unsigned char)t;
   }
   // cell geometry per LUT class: cell width (in u) below the smallest threshold gap, a power of two
