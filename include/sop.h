@@ -31,6 +31,8 @@ extern "C" {
 #define SOP_K_AUTO (-1000)     /* k_mode: choose the F_layer shift on the device */
 #define SOP_K_FROM_RESULT (-1001) /* k_mode of sop_dd4_lloyd: take the shift from a previous search */
 #define SOP_FMTA_FROM_RESULT (-1) /* fmta_index of sop_dd4_lloyd: best single LUT candidate of a previous search */
+#define SOP_ALL_ATOMS 0xFFFFFFFFu /* eval_mask of sop_pair_search: evaluate every candidate */
+#define SOP_SEARCH_SINGLES_ONLY 1 /* flags of sop_pair_search: reduce single candidates only, no pair / signed entries */
 
 enum {
   SOP_OK = 0,
@@ -125,11 +127,20 @@ int sop_channel_norms(const float* X_dev, long long T, long long K, long long ld
  *   |k| then to k > 0); any other value in [-64, 64] is used as the shift for every candidate.
  * dd_lut_dev (may be NULL): device table of SOP_MAX_ENTRIES floats that replaces, at kernel time,
  *   the lut of every atom whose index bit is set in dd_mask (a codebook produced by sop_dd4_lloyd
- *   can be swept without a host round trip). */
+ *   can be swept without a host round trip).
+ * eval_mask / load_mask: the sweep in two calls ("only the new columns").  Candidates in eval_mask
+ *   (SOP_ALL_ATOMS: all) are evaluated; candidates in load_mask are not evaluated again: their
+ *   per-block cosine and error are read from block_cos_dev / block_sse_dev as an earlier call on
+ *   the same layer, alphabet, format and shift wrote them (both arrays are then required).  A
+ *   candidate in neither mask is absent: every table entry that involves it is marked undefined and
+ *   its shift is reported as 0.  The masks must be disjoint and not both empty.  At most 8 distinct
+ *   tables may be evaluated per call (an atom and its negation share one).
+ * flags: SOP_SEARCH_SINGLES_ONLY fills only the diagonal (and best_single): enough to choose the
+ *   primary codebook FMTa before the Lloyd refinement. */
 int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes);
 int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                     const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
-                    const float* dd_lut_dev, unsigned dd_mask,
+                    const float* dd_lut_dev, unsigned dd_mask, unsigned eval_mask, unsigned load_mask, int flags,
                     sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
                     sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream);

@@ -30,14 +30,17 @@ struct ClassDev {
   int scope, kind;   // kind of the quantiser: LUT, E2M3, E4M3
   int c_half;        // table rows = 2 * c_half + 1
   int auto_k;        // 1: k* from the histogram
-  int n_cand;
+  int n_cand;                            // candidates evaluated in this call
   unsigned char cand[SOP_MAX_ATOMS];
+  int n_mem;                             // candidates present in this call (evaluated or loaded)
+  unsigned char mem[SOP_MAX_ATOMS];
 };
 struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (i0 == i1: single); 1: signed (i0, i0+1, i1, i1+1)
 
 struct Plan {
   int n_atoms, n_classes, n_tables, n_slots, n_pair_slots;
   int k_mode, rows, a_pad;
+  unsigned eval_mask, load_mask;   // candidates evaluated here / read from the per-block arrays of an earlier call
   int red_t1, red_g0, red_g1;   // phase-2 thread split of a half CTA: [0, t1) pair slots in g0 groups, [t1, 256) signed slots in g1 groups
   CandDev cand[SOP_MAX_ATOMS];
   ClassDev cls[SOP_MAX_CLASSES];
@@ -147,11 +150,12 @@ __global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const un
     if (threadIdx.x == 0) {
       hdr->cls_k[cl] = kstar;
       hdr->cls_pot[cl] = P.cls[cl].scope == 0 ? layer_pot_scale(wmax, P.cls[cl].tmax) : 0.0f;
-      for (int i = 0; i < P.cls[cl].n_cand; ++i) res->k[P.cls[cl].cand[i]] = kstar;
+      for (int i = 0; i < P.cls[cl].n_mem; ++i) res->k[P.cls[cl].mem[i]] = kstar;
     }
   }
   if (threadIdx.x == 0) {
-    for (int i = P.n_atoms; i < SOP_MAX_ATOMS; ++i) res->k[i] = 0;
+    for (int i = 0; i < SOP_MAX_ATOMS; ++i)
+      if (i >= P.n_atoms || !(((P.eval_mask | P.load_mask) >> i) & 1u)) res->k[i] = 0;
     res->layer_absmax = wmax;
     res->reserved[0] = res->reserved[1] = 0;
   }
@@ -409,8 +413,20 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       const long long blk = m * L.nbk + j;
       float2* my = cs + htid;
 
+      // candidates evaluated by an earlier call: their per-block values go from the arrays straight into
+      // the staging buffer (asynchronous 4-byte copies, no registers held) while this call's candidates
+      // are evaluated; the copies are awaited before the half's barrier
+      if (on) {
+        for (unsigned lm = P.load_mask; lm; lm &= lm - 1u) {
+          const int a = __ffs((int)lm) - 1;
+          const unsigned dst = (unsigned)__cvta_generic_to_shared(my + a * HBP);
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(block_cos + (size_t)a * L.NB + blk) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + 4u), "l"(block_sse + (size_t)a * L.NB + blk) : "memory");
+        }
+      }
       for (int cl = 0; cl < P.n_classes; ++cl) {
         const ClassDev& C = P.cls[cl];
+        if (C.n_cand == 0) continue;
         float s_hat;
         if (C.scope == 0) {
           s_hat = amax > 0.0f ? cls_pot[cl] : 0.0f;
@@ -493,6 +509,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         }
       }
     }
+    if (P.load_mask) asm volatile("cp.async.wait_all;" ::: "memory");
     half_barrier(half);
     // ---- phase 2: one slot per thread, blocks grp, grp + n_groups, ... of the half's tile; fp32 sums of
     //      eight gaps 1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
@@ -637,7 +654,7 @@ __global__ void __launch_bounds__(FIN_TB) finalize_kernel(LayerArgs L, Plan P, F
     int ba = -1, bb = -1, bs = -1, bsa = -1, bsb = -1;
     double vp = -2.0, vs = -2.0, vsp = -2.0;
     for (int a = 0; a < A; ++a) {
-      if (P.cand[a].kind == SOP_KIND_LUT && s_pair[a * A + a].acos > vs) { vs = s_pair[a * A + a].acos; bs = a; }
+      if (P.cand[a].kind == SOP_KIND_LUT && s_pair[a * A + a].n_sel1 >= 0 && s_pair[a * A + a].acos > vs) { vs = s_pair[a * A + a].acos; bs = a; }
       for (int b = a + 1; b < A; ++b) {
         const sop_pair_stat p = s_pair[a * A + b];
         if (p.n_sel1 >= 0 && p.acos > vp) { vp = p.acos; ba = a; bb = b; }
@@ -672,14 +689,20 @@ static double min_threshold_gap(const sop_atom& a) {
   return best;
 }
 
-int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
+int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mask, unsigned load_mask, int singles_only, Plan* P) {
   memset(P, 0, sizeof(*P));
   const int n = A.n_atoms;
   P->n_atoms = n;
   P->k_mode = k_mode;
+  P->eval_mask = eval_mask;
+  P->load_mask = load_mask;
+  const unsigned present = eval_mask | load_mask;
   // classes
   for (int i = 0; i < n; ++i) {
     const sop_atom& a = A.atoms[i];
+    P->cand[i].kind = (unsigned char)a.kind;
+    P->cand[i].neg = (unsigned char)a.negated;
+    if (!((present >> i) & 1u)) continue;
     int cl = -1;
     for (int c = 0; c < P->n_classes; ++c)
       if (P->cls[c].scope == a.scope && P->cls[c].tmax == a.tmax && P->cls[c].kind == a.kind) cl = c;
@@ -691,11 +714,11 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
       P->cls[cl].invh = 1.0f; P->cls[cl].c_half = 0;
     }
     ClassDev& C = P->cls[cl];
-    C.cand[C.n_cand++] = (unsigned char)i;
+    C.mem[C.n_mem++] = (unsigned char)i;
     P->cand[i].cls = (unsigned char)cl;
-    P->cand[i].kind = (unsigned char)a.kind;
-    P->cand[i].neg = (unsigned char)a.negated;
     P->cand[i].table = 0;
+    if (!((eval_mask >> i) & 1u)) continue;
+    C.cand[C.n_cand++] = (unsigned char)i;
     if (a.kind != SOP_KIND_LUT) continue;
     const bool dd = (A.dd_mask >> i) & 1u;
     int t = -1;
@@ -744,18 +767,23 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, Plan* P) {
   P->a_pad = n | 1;
   // slots: pair-type first (singles as (a, a)), then signed
   int ns = 0;
-  for (int a = 0; a < n; ++a) { P->slots[ns].type = 0; P->slots[ns].i0 = P->slots[ns].i1 = (unsigned char)a; ++ns; }
-  for (int a = 0; a < n; ++a)
+  auto has = [present](int i) { return ((present >> i) & 1u) != 0; };
+  for (int a = 0; a < n; ++a) {
+    if (!has(a)) continue;
+    P->slots[ns].type = 0; P->slots[ns].i0 = P->slots[ns].i1 = (unsigned char)a; ++ns;
+  }
+  for (int a = 0; a < n && !singles_only; ++a)
     for (int b = a + 1; b < n; ++b) {
+      if (!has(a) || !has(b)) continue;
       if (A.atoms[a].kind != SOP_KIND_LUT || A.atoms[b].kind != SOP_KIND_LUT || A.atoms[a].n_bits != A.atoms[b].n_bits) continue;
       P->slots[ns].type = 0; P->slots[ns].i0 = (unsigned char)a; P->slots[ns].i1 = (unsigned char)b; ++ns;
     }
   P->n_pair_slots = ns;
-  if (F.sign_bits) {
+  if (F.sign_bits && !singles_only) {
     bool base[SOP_MAX_ATOMS];
     for (int i = 0; i < n; ++i) {
       base[i] = false;
-      if (i + 1 >= n) continue;
+      if (i + 1 >= n || !has(i) || !has(i + 1)) continue;
       const sop_atom &a = A.atoms[i], &b = A.atoms[i + 1];
       if (a.kind != SOP_KIND_LUT || b.kind != SOP_KIND_LUT || a.negated || !b.negated || a.tmax != b.tmax) continue;
       const bool da = (A.dd_mask >> i) & 1u, db = (A.dd_mask >> (i + 1)) & 1u;
@@ -840,7 +868,7 @@ int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* byt
 
 int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                     const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
-                    const float* dd_lut_dev, unsigned dd_mask,
+                    const float* dd_lut_dev, unsigned dd_mask, unsigned eval_mask, unsigned load_mask, int flags,
                     sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
                     sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream) {
@@ -854,8 +882,13 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if ((rc = validate_atoms(atoms, n_atoms, dd_mask, dd_lut_dev, &A))) return rc;
   if (k_mode != SOP_K_AUTO && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
   if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < ws_total()) return SOP_ERR_WORKSPACE;
+  const unsigned all = n_atoms >= 32 ? 0xFFFFFFFFu : ((1u << n_atoms) - 1u);
+  eval_mask &= all;
+  if ((load_mask & ~all) || (load_mask & eval_mask) || !(eval_mask | load_mask)) return SOP_ERR_ALPHABET;
+  if (load_mask && (!block_cos_dev || !block_sse_dev)) return SOP_ERR_NULL;
+  if (flags & ~SOP_SEARCH_SINGLES_ONLY) return SOP_ERR_RANGE;
   Plan P;
-  if ((rc = build_plan(A, F, k_mode, &P))) return rc;
+  if ((rc = build_plan(A, F, k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, &P))) return rc;
 
   LayerArgs L;
   L.W = (const uint16_t*)W_dev; L.c = c_dev; L.M = M; L.K = K; L.ldw = ldw; L.nbk = K / SOP_G; L.NB = M * L.nbk;

@@ -1,7 +1,9 @@
 """The per-layer hot path as a sequence of C-ABI calls on one stream, with no host round trip
-in between: channel norms -> sweep of the ROM alphabet (finds FMTa and its per-block cosines) ->
-DD-n Lloyd refinement -> sweep of the full alphabet (ROM atoms, DD-n, negations, FP singles) ->
-pack of the chosen pair.  This module only allocates buffers and orders the calls.
+in between: channel norms -> sweep of every fixed candidate (ROM atoms, negations, FP singles;
+single-candidate reduction only: it finds FMTa and leaves every candidate's per-block cosine and
+error in device arrays) -> DD-n Lloyd refinement -> sweep of the two new columns (DD-n and its
+negation) with the fixed candidates' per-block values loaded, reducing every pair -> pack of the
+chosen pair.  This module only allocates buffers and orders the calls.
 """
 from __future__ import annotations
 
@@ -68,9 +70,9 @@ class LayerSweep:
         self.ws_norm = B.alloc_workspace(B.channel_norms_workspace(T, K), d)
         self.ws_search = B.alloc_workspace(B.pair_search_workspace(M, K, nF), d)
         self.ws_lloyd = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), d)
-        self.rom_table = B.new_pair_table(nR, d)
+        self.rom_table = B.new_pair_table(nF, d)
         self.rom_result = B.new_result(d)
-        self.block_cos = torch.empty((nR, self.NB), dtype=torch.float32, device=d)
+        self.fixed_mask = ((1 << nF) - 1) & ~self.dd_mask
         self.dd_lut = torch.zeros(B.MAX_ENTRIES, dtype=torch.float32, device=d)
         self.distortion = torch.zeros(max(1, lloyd_iters + 1), dtype=torch.float64, device=d)
         self.pool_count = torch.zeros(1, dtype=torch.int64, device=d)
@@ -82,8 +84,8 @@ class LayerSweep:
         self.codes = torch.empty(self.NB * 2 * n_bits, dtype=torch.uint8, device=d)
         self.words = torch.empty(B.words_nbytes(self.NB, self.container), dtype=torch.uint8, device=d)
         self.counts = torch.zeros(2, dtype=torch.int64, device=d)
-        self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d) if want_blocks else None
-        self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d) if want_blocks else None
+        self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
+        self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
         self.kernel_launches_per_step = 0
 
     def run(self, W: torch.Tensor, X: torch.Tensor, stream=None) -> None:
@@ -92,15 +94,19 @@ class LayerSweep:
         B.sop_channel_norms(X, self.c, self.ws_norm, stream)
         n += 2
         if self.iters > 0:
-            B.sop_pair_search(W, self.c, self.fmt, self.rom_atoms, self.rom_table, None, self.rom_result, self.ws_search,
-                              block_cos=self.block_cos, stream=stream)
+            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.rom_table, None, self.rom_result, self.ws_search,
+                              block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
+                              singles_only=True, stream=stream)
             n += 4
-            B.sop_dd4_lloyd(W, self.c, self.fmt, self.rom_atoms, self.block_cos, self.pool_rank, self.iters, self.dd_lut,
+            B.sop_dd4_lloyd(W, self.c, self.fmt, self.full_atoms, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
             n += 5 + (self.iters + 1)
-        B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
-                          self.ws_search, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
-                          block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
+            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
+                              self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
+                              block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask, stream=stream)
+        else:
+            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
+                              self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
         n += 4
         B.sop_pack(W, self.c, self.fmt, self.full_atoms, self.codes, self.words, search_result=self.result,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,

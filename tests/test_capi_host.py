@@ -46,12 +46,13 @@ FAKE = C.c_void_p(0x10000)     # never dereferenced: every call below fails vali
 
 
 def _search(lib, M=4, K=64, ldw=64, g=16, fmt=None, atoms=None, n=None, k=B.K_AUTO, W=FAKE, ws=FAKE, wsb=1 << 30,
-            dd=None, mask=0):
+            dd=None, mask=0, emask=0xFFFFFFFF, lmask=0, flags=0, bc=None):
     fmt = fmt or I.scale_format("UE4M4")
     atoms = atoms if atoms is not None else I.alphabet(["NF4"])
     n = len(atoms) if n is None else n
     return lib.sop_pair_search(W, C.c_longlong(M), C.c_longlong(K), C.c_longlong(ldw), FAKE, g, C.byref(B.make_fmt(fmt)), k,
-                               B.make_atoms(atoms), n, dd, C.c_uint(mask), FAKE, None, FAKE, None, None, ws,
+                               B.make_atoms(atoms), n, dd, C.c_uint(mask), C.c_uint(emask), C.c_uint(lmask), flags, FAKE, None, FAKE, bc,
+                               bc, ws,
                                C.c_size_t(wsb), None)
 
 
@@ -80,6 +81,12 @@ def test_pair_search_rejects_bad_arguments(lib):
     assert _search(lib, ws=C.c_void_p(0x10010)) == -5  # workspace not 256-byte aligned
     assert _search(lib, mask=1) == -1                  # dd_mask without a device table
     assert _search(lib, mask=4, dd=FAKE) == -4         # mask bit beyond the alphabet
+    assert _search(lib, emask=0) == -4                 # nothing evaluated and nothing loaded
+    assert _search(lib, emask=1, lmask=1, bc=FAKE) == -4   # a candidate both evaluated and loaded
+    assert _search(lib, emask=0, lmask=4, bc=FAKE) == -4   # load bit beyond the alphabet
+    atoms2 = I.alphabet(["NF4"])
+    assert _search(lib, atoms=atoms2, emask=1, lmask=2) == -1   # loading needs the per-block arrays
+    assert _search(lib, flags=2) == -7
 
 
 def test_other_entry_points_reject_bad_arguments(lib):

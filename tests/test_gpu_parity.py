@@ -38,7 +38,7 @@ def gpu_norms(B, X):
     return c
 
 
-def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0):
+def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0, two_calls_split=None):
     M, K = W.shape
     A = len(atoms)
     NB = M * K // 16
@@ -47,11 +47,26 @@ def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0):
     bc = torch.full((A, NB), -7.0, dtype=torch.float32, device=dev())
     bs = torch.full((A, NB), -7.0, dtype=torch.float32, device=dev())
     ws = B.alloc_workspace(B.pair_search_workspace(M, K, A), dev())
-    B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=B.K_AUTO if k_mode is None else k_mode,
-                      dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc, block_sse=bs)
+    km = B.K_AUTO if k_mode is None else k_mode
+    if two_calls_split is None:
+        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
+                          block_sse=bs)
+    else:
+        # first the candidates in the mask (single-candidate reduction only), then the rest with the first ones loaded
+        first = two_calls_split
+        rest = ((1 << A) - 1) & ~first
+        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
+                          block_sse=bs, eval_mask=first, singles_only=True)
+        torch.cuda.synchronize()
+        first_pass = dict(pair=B.read_pair_table(pt, A).copy(), **B.read_result(res))
+        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
+                          block_sse=bs, eval_mask=rest, load_mask=first)
     torch.cuda.synchronize()
-    return dict(pair=B.read_pair_table(pt, A), signed=B.read_pair_table(st, A), block_cos=bc.cpu().numpy(),
-                block_sse=bs.cpu().numpy(), res_t=res, Wd=Wd, cd=cd, bc_t=bc, **B.read_result(res))
+    out = dict(pair=B.read_pair_table(pt, A), signed=B.read_pair_table(st, A), block_cos=bc.cpu().numpy(),
+               block_sse=bs.cpu().numpy(), res_t=res, Wd=Wd, cd=cd, bc_t=bc, **B.read_result(res))
+    if two_calls_split is not None:
+        out["first_pass"] = first_pass
+    return out
 
 
 def assert_tables(got, want, A):
@@ -156,6 +171,38 @@ def test_tables_that_need_the_binary_search_path(B):
     a2 = I.Atom("dup", 4, I.KIND_LUT, 0, 16, 1.0, np.sort(dup))
     a3 = I.Atom("two", 4, I.KIND_LUT, 0, 16, 1.0, np.array([-0.5, 0.75], np.float32))
     check_search(B, L, "E5M6", [a1, a1.negation(), a2, a2.negation(), a3, I.rom_atom("E2M2")])
+
+
+@pytest.mark.parametrize("fmt_name", ["UE4M4", "E5M6"])
+def test_sweep_in_two_calls_equals_one_call(B, fmt_name):
+    # "only the new columns": candidates evaluated by an earlier call are loaded, not evaluated again
+    L = I.outlier_channel_layer(5, 200, 1024, 64)
+    fmt = I.scale_format(fmt_name)
+    atoms = I.alphabet(["NF4", "SH4", "BOF4"], fp=["E2M3", "E4M3^0"])
+    c = oracle.channel_norms(L.X.numpy())
+    want = oracle.pair_search(L.W, c, fmt, atoms, want_blocks=True)
+    first = 0b10110011     # NF4, -NF4, BOF4, -BOF4, E4M3^0 first; SH4, -SH4, E2M3 in the second call
+    got = gpu_search(B, L.W, c, fmt, atoms, two_calls_split=first)
+    assert np.array_equal(got["block_cos"].view(np.uint32), want["block_cos"].view(np.uint32))
+    assert np.array_equal(got["block_sse"].view(np.uint32), want["block_sse"].view(np.uint32))
+    assert_tables(got, want, len(atoms))
+    one = gpu_search(B, L.W, c, fmt, atoms)
+    for name in ("pair", "signed"):
+        assert np.array_equal(got[name]["n_sel1"], one[name]["n_sel1"])
+    # the first call: diagonal entries of its candidates only, shifts of absent candidates reported as 0
+    fp = got["first_pass"]
+    A = len(atoms)
+    for a in range(A):
+        for b in range(A):
+            defined = a == b and (first >> a) & 1
+            assert (fp["pair"]["n_sel1"][a, b] >= 0) == bool(defined)
+            if defined:
+                assert np.isclose(fp["pair"]["acos"][a, a], want["pair"]["acos"][a, a], rtol=REL, atol=0)
+    present = np.array([(first >> a) & 1 for a in range(A)], dtype=bool)
+    assert np.array_equal(fp["k"][:A][present], want["k"][present]) and not fp["k"][:A][~present].any()
+    lut_first = [a for a in range(A) if present[a] and atoms[a].kind == I.KIND_LUT]
+    assert fp["best"][2] == max(lut_first, key=lambda a: (want["pair"]["acos"][a, a], -a))
+    assert fp["best"][0] == -1 and fp["best"][3] == -1
 
 
 def test_negation_symmetry_on_gpu(B):
@@ -270,7 +317,7 @@ def test_pipeline_matches_oracle(B, fmt_name, rom, fp, iters, shape):
     assert np.array_equal(got.dd_lut[:ne].view(np.uint32), want["dd_lut"].view(np.uint32))
     assert got.pool_count == want["pool_count"]
     assert np.allclose(got.distortion, want["distortion"], rtol=REL, atol=0)
-    assert np.array_equal(got.rom_result["best"][:3], want["rom"]["best"][:3])   # the ROM pass fills no signed table
+    assert got.rom_result["best"][2] == want["rom"]["best"][2]   # the first pass reduces single candidates only: FMTa
     A = len(want["atoms"])
     full = dict(pair=got.pair_table, signed=got.signed_table, k=got.result["k"], best=got.result["best"])
     assert_tables(full, want["full"], A)
