@@ -191,14 +191,20 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
  *     word_sign_bits = 1: sign at bit b-1, selector at bit 0, magnitude E:M above the
  *     m = b-1-x-y metabits; word_sign_bits = 0: selector at bit b-1 (if m >= 1), magnitude above
  *     the remaining m-1 metabits.  Unused metabits are zero.
- *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten. */
+ *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten.
+ *   block_cos_dev (may be NULL): [n_atoms x N_b] per-block cosines written by sop_pair_search for the
+ *     same layer, alphabet, format and shift.  When every candidate of the choice has a row there
+ *     (with use_sign, the negated variant of an atom is the atom of the alphabet with the same table
+ *     and the opposite `negated`; from a search result it is the next atom), the winner of each block
+ *     is read off these cosines and only the winner is encoded: the output is identical, the cost
+ *     drops to one encode per block.  Otherwise the candidates are evaluated here. */
 #define SOP_NO_ATOM (-2)
 #define SOP_PAIR_FROM_RESULT (-1)
 int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
              const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
              unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
              int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
-             unsigned char* words_dev, long long* counts_dev, void* stream);
+             unsigned char* words_dev, long long* counts_dev, const float* block_cos_dev, void* stream);
 
 #ifdef __cplusplus
 }

@@ -180,13 +180,13 @@ def sop_pack(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes: torc
              index_a: int = PAIR_FROM_RESULT, index_b: int = PAIR_FROM_RESULT, k_mode: int = K_FROM_RESULT,
              search_result: Optional[torch.Tensor] = None, use_sign: int = 0, container_bits: int = 8,
              word_sign_bits: int = 0, counts: Optional[torch.Tensor] = None, dd_lut: Optional[torch.Tensor] = None,
-             dd_mask: int = 0, stream=None, g: int = 16) -> None:
+             dd_mask: int = 0, stream=None, g: int = 16, block_cos: Optional[torch.Tensor] = None) -> None:
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_pack(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)),
                           make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), index_a, index_b, k_mode,
                           _ptr(search_result), use_sign, container_bits, word_sign_bits, _ptr(codes), _ptr(words),
-                          _ptr(counts), _stream(stream)), "sop_pack")
+                          _ptr(counts), _ptr(block_cos), _stream(stream)), "sop_pack")
 
 
 def profile_enable(on: bool) -> None:

@@ -19,12 +19,15 @@ struct PackArgs {
   unsigned char* codes;
   unsigned* words;       // zeroed before the kernel; filled with atomicOr
   unsigned long long* counts;
+  const float* block_cos;   // optional [n_atoms x NB]: per-block cosines of an earlier sweep
+  int cos_neg_a, cos_neg_b; // rows of the negated variants of index_a / index_b (-1: unknown, evaluate instead)
 };
 
 struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
 // The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
+template <bool WANT_COS>
 __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int kind, int neg, float rcp,
                                                 float& cos_out, uint32_t (&code4)[4]) {
@@ -50,16 +53,18 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
         code = fp_code<SOP_KIND_FP_E4M3>(q);
       }
       packed |= code << (8 * r);
-      const float cw = __fmul_rn(c[i], w[i]);
-      const float cq = __fmul_rn(c[i], q);
-      aw = __fmaf_rn(cw, w[i], aw);
-      ad = __fmaf_rn(cq, w[i], ad);
-      an = __fmaf_rn(cq, q, an);
+      if (WANT_COS) {
+        const float cw = __fmul_rn(c[i], w[i]);
+        const float cq = __fmul_rn(c[i], q);
+        aw = __fmaf_rn(cw, w[i], aw);
+        ad = __fmaf_rn(cq, w[i], ad);
+        an = __fmaf_rn(cq, q, an);
+      }
     }
     qn[h] = an; qd[h] = ad; qw[h] = aw;
     code4[h] = packed;
   }
-  cos_out = block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd));
+  cos_out = WANT_COS ? block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd)) : 0.0f;
 }
 
 __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
@@ -68,9 +73,11 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
   __shared__ int s_nb, s_nbits;
   __shared__ float s_pot[2];
   __shared__ unsigned s_cnt[2];
+  __shared__ int s_row[4];   // rows of block_cos for the candidates a, -a, b, -b (-1: none)
   const int tid = threadIdx.x;
   if (tid == 0) {
     int ia = a.index_a, ib = a.index_b;
+    const bool from_result = ia == SOP_PAIR_FROM_RESULT;
     if (ia == SOP_PAIR_FROM_RESULT) {
       ia = a.use_sign ? res->best_sa : res->best_a;
       ib = a.use_sign ? res->best_sb : res->best_b;
@@ -92,10 +99,18 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
       for (int j = 0; j < 32; ++j) lutv[t][j] = at.kind == SOP_KIND_LUT ? (dd ? A.dd_lut[min(j, ne - 1)] : at.lut[min(j, ne - 1)]) : 0.0f;
       build_thresholds(lutv[t], ne, tau[t]);
     }
+    // from a search result with signs, a and b are base atoms and each is followed by its negation
+    s_row[0] = ia;
+    s_row[1] = from_result ? ia + 1 : a.cos_neg_a;
+    s_row[2] = nb == 2 ? ib : -1;
+    s_row[3] = nb == 2 ? (from_result ? ib + 1 : a.cos_neg_b) : -1;
     s_cnt[0] = s_cnt[1] = 0;
   }
   __syncthreads();
   const int nb = s_nb, n = s_nbits, b = a.container_bits;
+  bool use_cos = a.block_cos != nullptr;
+  for (int t = 0; t < nb; ++t)
+    for (int sg = 0; sg < (a.use_sign ? 2 : 1); ++sg) use_cos = use_cos && s_row[2 * t + sg] >= 0;
   const int n_sign = a.use_sign ? 2 : 1;
   unsigned my_sel = 0, my_neg = 0;
   for (long long blk = (long long)blockIdx.x * PTB + tid; blk < a.NB; blk += (long long)gridDim.x * PTB) {
@@ -121,27 +136,50 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     float best_cos = 0.0f;
     uint32_t best_scode = 0, best4[4] = {0u, 0u, 0u, 0u};
     int pick = -1;
-    for (int t = 0; t < nb; ++t) {
+    if (use_cos) {
+      // the winner follows from the cosines of the sweep (same arithmetic, bit for bit): only it is encoded
+      for (int t = 0; t < nb; ++t)
+        for (int sg = 0; sg < n_sign; ++sg) {
+          const float cs = __ldg(a.block_cos + (size_t)s_row[2 * t + sg] * a.NB + blk);
+          if (pick < 0 || cs > best_cos) { best_cos = cs; pick = 2 * t + sg; }
+        }
+      const int t = pick >> 1, sg = pick & 1;
       const PackCand cd = base[t];
       float s_hat;
-      uint32_t sc = 0;
       if (cd.scope == 0) {
         s_hat = amax > 0.0f ? s_pot[t] : 0.0f;
       } else {
         const float sigma = cd.tmax == 1.0f ? amax : __fdiv_rn(amax, cd.tmax);
         const QScale qs = scale_quantize(sigma, cd.k, F);
         s_hat = qs.s_hat;
-        sc = qs.code;
+        best_scode = qs.code;
       }
       const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
-      for (int sg = 0; sg < n_sign; ++sg) {
-        float cs;
-        uint32_t c4[4];
-        eval_block_regs(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, cs, c4);
-        if (pick < 0 || cs > best_cos) {
-          best_cos = cs; best_scode = sc; pick = 2 * t + sg;
+      float unused;
+      eval_block_regs<false>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, unused, best4);
+    } else {
+      for (int t = 0; t < nb; ++t) {
+        const PackCand cd = base[t];
+        float s_hat;
+        uint32_t sc = 0;
+        if (cd.scope == 0) {
+          s_hat = amax > 0.0f ? s_pot[t] : 0.0f;
+        } else {
+          const float sigma = cd.tmax == 1.0f ? amax : __fdiv_rn(amax, cd.tmax);
+          const QScale qs = scale_quantize(sigma, cd.k, F);
+          s_hat = qs.s_hat;
+          sc = qs.code;
+        }
+        const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+        for (int sg = 0; sg < n_sign; ++sg) {
+          float cs;
+          uint32_t c4[4];
+          eval_block_regs<true>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, cs, c4);
+          if (pick < 0 || cs > best_cos) {
+            best_cos = cs; best_scode = sc; pick = 2 * t + sg;
 #pragma unroll
-          for (int h = 0; h < 4; ++h) best4[h] = c4[h];
+            for (int h = 0; h < 4; ++h) best4[h] = c4[h];
+          }
         }
       }
     }
@@ -199,7 +237,7 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
              const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
              unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
              int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
-             unsigned char* words_dev, long long* counts_dev, void* stream) {
+             unsigned char* words_dev, long long* counts_dev, const float* block_cos_dev, void* stream) {
   using namespace sop;
   int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
   if (rc) return rc;
@@ -245,6 +283,21 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   a.index_a = index_a; a.index_b = index_b; a.k_mode = k_mode; a.use_sign = use_sign;
   a.container_bits = container_bits; a.word_sign_bits = word_sign_bits; a.meta_bits = meta;
   a.codes = codes_dev; a.words = (unsigned*)words_dev; a.counts = (unsigned long long*)counts_dev;
+  a.block_cos = block_cos_dev;
+  a.cos_neg_a = a.cos_neg_b = -1;
+  if (block_cos_dev && use_sign && !from_result) {
+    // row of the negated variant of an explicitly given atom: same table and scale reference, opposite sign
+    auto find_neg = [&](int i) {
+      for (int j = 0; j < n_atoms; ++j)
+        if (j != i && atoms[j].kind == atoms[i].kind && atoms[j].negated != atoms[i].negated && atoms[j].tmax == atoms[i].tmax &&
+            atoms[j].n_entries == atoms[i].n_entries && ((dd_mask >> j) & 1u) == ((dd_mask >> i) & 1u) &&
+            (((dd_mask >> i) & 1u) || memcmp(atoms[j].lut, atoms[i].lut, sizeof(float) * atoms[i].n_entries) == 0))
+          return j;
+      return -1;
+    };
+    a.cos_neg_a = find_neg(index_a);
+    if (index_b != SOP_NO_ATOM) a.cos_neg_b = find_neg(index_b);
+  }
   cudaStream_t st = (cudaStream_t)stream;
   const size_t word_bytes = (size_t)((a.NB * container_bits + 7) / 8);
   // the word stream is written with 32-bit atomicOr: the caller's buffer must hold whole 32-bit words

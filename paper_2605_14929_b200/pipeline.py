@@ -110,7 +110,8 @@ class LayerSweep:
         n += 4
         B.sop_pack(W, self.c, self.fmt, self.full_atoms, self.codes, self.words, search_result=self.result,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
-                   counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask, stream=stream)
+                   counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
+                   block_cos=self.full_cos, stream=stream)
         n += 1
         self.kernel_launches_per_step = n
 

@@ -110,7 +110,7 @@ def test_other_entry_points_reject_bad_arguments(lib):
 
     def pack(ia=0, ib=2, k=0, sign=0, b=12, wsb=0, res=None, f=fmt):
         return lib.sop_pack(FAKE, ll(4), ll(64), ll(64), FAKE, 16, f, arr, len(atoms), None, C.c_uint(0), ia, ib, k, res,
-                            sign, b, wsb, FAKE, FAKE, None, None)
+                            sign, b, wsb, FAKE, FAKE, None, None, None)
     assert pack(b=8) == -3                  # UE4M4 in 8 bits has no metabit for the selector
     assert pack(b=10) == -3
     assert pack(sign=1, wsb=0) == -3        # sign requested, word has no sign bit

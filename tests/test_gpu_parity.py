@@ -250,7 +250,7 @@ def test_lloyd_matches_oracle(B, fmt_name, names, iters):
 
 
 # ------------------------------------------------------------------ pack
-def gpu_pack(B, W, c, fmt, atoms, ia, ib, k, use_sign, b, wsign):
+def gpu_pack(B, W, c, fmt, atoms, ia, ib, k, use_sign, b, wsign, block_cos=None):
     M, K = W.shape
     NB = M * K // 16
     n = atoms[ia].n_bits
@@ -258,7 +258,7 @@ def gpu_pack(B, W, c, fmt, atoms, ia, ib, k, use_sign, b, wsign):
     words = torch.full((B.words_nbytes(NB, b),), 0xAB, dtype=torch.uint8, device=dev())
     counts = torch.zeros(2, dtype=torch.int64, device=dev())
     B.sop_pack(W.to(dev()), torch.as_tensor(c).to(dev()), fmt, atoms, codes, words, index_a=ia, index_b=ib, k_mode=k,
-               use_sign=use_sign, container_bits=b, word_sign_bits=wsign, counts=counts)
+               use_sign=use_sign, container_bits=b, word_sign_bits=wsign, counts=counts, block_cos=block_cos)
     torch.cuda.synchronize()
     return codes.cpu().numpy().reshape(NB, 2 * n), words.cpu().numpy(), counts.cpu().numpy()
 
@@ -279,6 +279,11 @@ def test_pack_matches_oracle(B, fmt_name, ia, ib, sign, b, wsign):
     assert np.array_equal(codes, want["codes"])
     assert np.array_equal(words[:want["words"].size], want["words"])
     assert (int(counts[0]), int(counts[1])) == (want["n_sel1"], want["n_neg"])
+    # the same choice read off the per-block cosines of a sweep: identical bytes
+    bc = gpu_search(B, L.W, c, fmt, atoms, k_mode=1)["bc_t"]
+    codes2, words2, counts2 = gpu_pack(B, L.W, c, fmt, atoms, ia, B.NO_ATOM if ib is None else ib, 1, sign, b, wsign,
+                                       block_cos=bc)
+    assert np.array_equal(codes2, codes) and np.array_equal(words2, words) and np.array_equal(counts2, counts)
 
 
 def test_pack_five_bit_pair(B):
