@@ -67,7 +67,10 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
   cos_out = WANT_COS ? block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd)) : 0.0f;
 }
 
-__global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
+// USE_COS: the winner of each block is read off the per-block cosines of a sweep and only it is encoded
+// (no channel norms needed); otherwise every candidate of the choice is evaluated here.
+template <bool USE_COS>
+__global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
   __shared__ float lutv[2][32], tau[2][32];
   __shared__ PackCand base[2];
   __shared__ int s_nb, s_nbits;
@@ -108,9 +111,7 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
   }
   __syncthreads();
   const int nb = s_nb, n = s_nbits, b = a.container_bits;
-  bool use_cos = a.block_cos != nullptr;
-  for (int t = 0; t < nb; ++t)
-    for (int sg = 0; sg < (a.use_sign ? 2 : 1); ++sg) use_cos = use_cos && s_row[2 * t + sg] >= 0;
+
   const int n_sign = a.use_sign ? 2 : 1;
   unsigned my_sel = 0, my_neg = 0;
   for (long long blk = (long long)blockIdx.x * PTB + tid; blk < a.NB; blk += (long long)gridDim.x * PTB) {
@@ -121,7 +122,10 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     float w[16], c[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) { w[2 * i] = bf16lo(wb[i]); w[2 * i + 1] = bf16hi(wb[i]); }
-    {
+    if (USE_COS) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) c[i] = 0.0f;
+    } else {
       const float4* cp = reinterpret_cast<const float4*>(a.c + j * SOP_G);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -136,7 +140,7 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     float best_cos = 0.0f;
     uint32_t best_scode = 0, best4[4] = {0u, 0u, 0u, 0u};
     int pick = -1;
-    if (use_cos) {
+    if (USE_COS) {
       // the winner follows from the cosines of the sweep (same arithmetic, bit for bit): only it is encoded
       for (int t = 0; t < nb; ++t)
         for (int sg = 0; sg < n_sign; ++sg) {
@@ -187,6 +191,15 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     my_sel += sel; my_neg += sgn;
     // codes: 16 n-bit fields, little-endian, 2n bytes
     unsigned long long lo = 0, hi = 0;   // 128-bit accumulator
+    if (n == 4) {
+      uint32_t h16[4];
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const uint32_t y = (best4[h] | (best4[h] >> 4)) & 0x00FF00FFu;   // bytes 0 and 2 hold two codes each
+        h16[h] = (y | (y >> 8)) & 0xFFFFu;
+      }
+      lo = (unsigned long long)(h16[0] | (h16[1] << 16)) | ((unsigned long long)(h16[2] | (h16[3] << 16)) << 32);
+    } else
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const int pos = i * n;
@@ -214,7 +227,11 @@ __global__ void __launch_bounds__(PTB) pack_kernel(PackArgs a, AtomsDev A, FmtDe
     const long long bit = blk * b;
     const long long wi = bit >> 5;
     const int sh = (int)(bit & 31);
-    if (word) {
+    if (b == 16) {
+      reinterpret_cast<unsigned short*>(a.words)[blk] = (unsigned short)word;
+    } else if (b == 8) {
+      reinterpret_cast<unsigned char*>(a.words)[blk] = (unsigned char)word;
+    } else if (word) {
       atomicOr(&a.words[wi], word << sh);
       if (sh + b > 32) atomicOr(&a.words[wi + 1], word >> (32 - sh));
     }
@@ -300,13 +317,18 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   }
   cudaStream_t st = (cudaStream_t)stream;
   const size_t word_bytes = (size_t)((a.NB * container_bits + 7) / 8);
-  // the word stream is written with 32-bit atomicOr: the caller's buffer must hold whole 32-bit words
-  SOP_CUDA_TRY(cudaMemsetAsync(words_dev, 0, (word_bytes + 3) & ~(size_t)3, st));
+  // 12-bit words are merged into the stream with 32-bit atomicOr (the caller's buffer holds whole 32-bit
+  // words and starts from zero); 8- and 16-bit words are stored directly, only the padding is cleared
+  const size_t padded = (word_bytes + 3) & ~(size_t)3;
+  if (container_bits == 12) SOP_CUDA_TRY(cudaMemsetAsync(words_dev, 0, padded, st));
+  else SOP_CUDA_TRY(cudaMemsetAsync(words_dev + padded - 4, 0, 4, st));
   if (counts_dev) SOP_CUDA_TRY(cudaMemsetAsync(counts_dev, 0, 2 * sizeof(long long), st));
   long long grid = (a.NB + PTB - 1) / PTB;
   const int sms = num_sms();
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
-  pack_kernel<<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
+  const bool negs_known = !use_sign || from_result || (a.cos_neg_a >= 0 && (!pair || a.cos_neg_b >= 0));
+  if (block_cos_dev && negs_known) pack_kernel<true><<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
+  else pack_kernel<false><<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }
