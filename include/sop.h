@@ -164,7 +164,9 @@ int sop_profile_last_sweep_ms(float* ms);
  *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
  *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
  *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
- *   pool_count_dev: one long long, number of blocks in the pool. */
+ *   pool_count_dev: one long long, number of blocks in the pool.
+ * Workspace: 8 bytes per weight element (u and omega of every pool element are kept across the
+ *   iterations), 4 bytes per block (the pool list) and 4 bytes per channel, plus a fixed header. */
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,

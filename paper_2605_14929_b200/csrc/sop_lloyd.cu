@@ -6,15 +6,19 @@
 //                         with a CTA-wide scan.
 //   lloyd_setup_kernel    threshold tau and pool count from the last histogram, max(c), the shift k,
 //                         the initial table (FMTa, reversed and negated if FMTa is a negated atom),
-//                         and the per-channel weight tables omega = c / max(c) and fix(omega).
+//                         and the per-channel weight table omega = c / max(c).
 //   pool_list_kernel      compacts the indices of the pool blocks (cos <= tau) into a dense list, so
 //                         that every lane of the iteration kernel has work.
-//   lloyd_iter_kernel     one thread per pool block: u = w / scale, nearest entry by binary search
-//                         over exact thresholds, per-entry int64 fixed-point sums kept in
-//                         thread-private shared-memory slots (no atomics in the element loop; the sums
-//                         are exactly associative, so any order reproduces a sequential sum bit for
-//                         bit), FP64 distortion.  The CTA that finishes last turns the sums into
-//                         centroids, snaps them to bf16, sorts, and clears the accumulators.
+//   pool_cache_kernel     the pool elements never change between iterations, only the table does:
+//                         (u, omega) of every pool element is computed once (u = w / scale) and kept
+//                         in one array.
+//   lloyd_stream_kernel   one iteration = one coalesced stream over that array: the cell of u on a
+//                         uniform grid gives the (at most two) candidate entries and the exact
+//                         threshold between them; per-entry int64 fixed-point sums are kept in
+//                         thread-private shared-memory slots (no atomics in the element loop; the
+//                         sums are exactly associative, so any order reproduces a sequential sum bit
+//                         for bit), distortion in FP64.  The CTA that finishes last turns the sums
+//                         into centroids, snaps them to bf16, sorts, and clears the accumulators.
 #include <math.h>
 #include <string.h>
 
@@ -24,6 +28,10 @@ namespace sop {
 
 constexpr int LTB = 256;
 constexpr int SETUP_TB = 1024;
+constexpr int SORT_CHALF = 320;                 // lookup grid on u: cell width 2^-8, rows cover |u| <= 1.25,
+constexpr int SORT_ROWS = 2 * SORT_CHALF + 1;   // the first and last row take everything beyond
+constexpr float SORT_INVH = 256.0f;
+constexpr float SORT_MAGIC = 12582912.0f;       // 1.5 * 2^23
 
 struct LloydWs {
   // radix select state
@@ -52,15 +60,15 @@ struct LloydArgs {
   long long pool_rank;
   int k_mode, fmta_index, n_atoms;
   float* omega;               // workspace: K floats, c / max(c)
-  unsigned* omega_fix;        // workspace: K words, round(omega * 2^24)
   unsigned* pool_idx;         // workspace: NB words, indices of the pool blocks
+  uint2* cache;               // workspace: 16 NB pairs (u, omega) as bit patterns, in pool-list order
 };
 
 static size_t lloyd_off_omega() { return (sizeof(LloydWs) + 255) & ~(size_t)255; }
-static size_t lloyd_off_fix(long long K) { return lloyd_off_omega() + (((size_t)K * 4 + 255) & ~(size_t)255); }
-static size_t lloyd_off_idx(long long K) { return lloyd_off_fix(K) + (((size_t)K * 4 + 255) & ~(size_t)255); }
+static size_t lloyd_off_idx(long long K) { return lloyd_off_omega() + (((size_t)K * 4 + 255) & ~(size_t)255); }
+static size_t lloyd_off_cache(long long M, long long K) { return lloyd_off_idx(K) + ((((size_t)M * (size_t)(K / SOP_G)) * 4 + 255) & ~(size_t)255); }
 static size_t lloyd_ws_bytes(long long M, long long K) {
-  return lloyd_off_idx(K) + ((((size_t)M * (size_t)(K / SOP_G)) * 4 + 255) & ~(size_t)255);
+  return lloyd_off_cache(M, K) + (size_t)M * (size_t)K * sizeof(uint2);
 }
 
 __device__ __forceinline__ unsigned cos_key(float x) {
@@ -168,7 +176,6 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   for (long long i = threadIdx.x; i < a.K; i += SETUP_TB) {
     const float om = cmax > 0.0f ? __fdiv_rn(__ldg(a.c + i), cmax) : 0.0f;
     a.omega[i] = om;
-    a.omega_fix[i] = (unsigned)__float2ll_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]: at most 2^24
   }
   if (threadIdx.x == 0) {
     const unsigned key = prefix;   // full 32-bit key after three passes
@@ -261,89 +268,138 @@ __device__ void lloyd_update(LloydWs* ws, double* __restrict__ distortion, int i
   v->done = 0;
 }
 
-__global__ void __launch_bounds__(LTB) lloyd_iter_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                         int it, int last, float* __restrict__ out_lut) {
+__device__ __forceinline__ int sort_cell(float u) {
+  const float t = fminf(fmaxf(__fmaf_rn(u, SORT_INVH, SORT_MAGIC + (float)SORT_CHALF), SORT_MAGIC), SORT_MAGIC + (float)(2 * SORT_CHALF));
+  return (int)(__float_as_uint(t) - __float_as_uint(SORT_MAGIC));
+}
+
+// u of the 16 elements of pool block `blk`
+__device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F, int k, unsigned blk, float (&u)[16], unsigned& j_out) {
+  const unsigned nbk = (unsigned)a.nbk;
+  const unsigned m = blk / nbk, j = blk - m * nbk;
+  j_out = j;
+  const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
+  const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+  const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+  uint32_t mb = 0;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
+  const float amax = __uint_as_float(mb << 16);
+  const float s_hat = scale_quantize(amax, k, F).s_hat;    // a DD table declares tmax = 1
+  const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+#pragma unroll
+  for (int e = 0; e < 16; ++e) u[e] = __fmul_rn((e & 1) ? bf16hi(wb[e >> 1]) : bf16lo(wb[e >> 1]), rcp);
+}
+
+__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, const LloydWs* __restrict__ ws) {
+  const unsigned count = ws->list_count;
+  const int k = ws->k;
+  for (unsigned i = blockIdx.x * LTB + threadIdx.x; i < count; i += gridDim.x * LTB) {
+    float u[16];
+    unsigned j;
+    pool_block_u(a, F, k, a.pool_idx[i], u, j);
+    const float4* op = reinterpret_cast<const float4*>(a.omega + (size_t)j * SOP_G);
+    uint4* dst = reinterpret_cast<uint4*>(a.cache + (size_t)i * 16);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float4 o = __ldg(op + q);
+      dst[2 * q] = make_uint4(__float_as_uint(u[4 * q]), __float_as_uint(o.x), __float_as_uint(u[4 * q + 1]), __float_as_uint(o.y));
+      dst[2 * q + 1] = make_uint4(__float_as_uint(u[4 * q + 2]), __float_as_uint(o.z), __float_as_uint(u[4 * q + 3]), __float_as_uint(o.w));
+    }
+  }
+}
+
+struct CellEntry { float thr; unsigned codes; };   // codes: lo | hi << 8; 0xFFFF: more than one threshold in the cell
+
+__device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exact scaling, one rounding to an integer
+  const float s = __fmul_rn(v, 16777216.0f);
+  return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
+}
+
+__global__ void __launch_bounds__(LTB) lloyd_stream_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                           int it, int last, float* __restrict__ out_lut) {
   extern __shared__ __align__(16) unsigned char lsm[];
-  ulonglong2* acc = reinterpret_cast<ulonglong2*>(lsm);    // [n_entries][blockDim.x]: (sum fix(omega), sum fix(omega u))
+  ulonglong2* acc = reinterpret_cast<ulonglong2*>(lsm);    // [n_entries][LTB]: (sum fix(omega), sum fix(omega u))
   __shared__ float lutv[32], tau[32];
+  __shared__ CellEntry cellt[SORT_ROWS];
   __shared__ double sD[LTB / 32];
   __shared__ int s_is_last;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, BD = blockDim.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int ne = ws->n_entries;
   if (tid < 32) lutv[tid] = ws->lut[min(tid, ne - 1)];
   if (!last)
-    for (int i = tid; i < ne * BD; i += BD) acc[i] = make_ulonglong2(0ull, 0ull);
+    for (int i = tid; i < ne * LTB; i += LTB) acc[i] = make_ulonglong2(0ull, 0ull);
   __syncthreads();
   if (tid == 0) build_thresholds(lutv, ne, tau);
   __syncthreads();
-  const int k = ws->k;
-  const unsigned count = ws->list_count;
-  const unsigned nbk = (unsigned)a.nbk;
-  ulonglong2* mine = acc + tid;
+  // cell r covers u * 256 in [k - 1/2, k + 1/2], k = r - 320 (first / last row: everything beyond)
+  for (int r = tid; r < SORT_ROWS; r += LTB) {
+    const float kf = (float)(r - SORT_CHALF);
+    const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, 1.0f / SORT_INVH);
+    const float hi_edge = r == SORT_ROWS - 1 ? INFINITY : __fmul_rn(kf + 0.5f, 1.0f / SORT_INVH);
+    int nbelow = 0, ninside = 0, ndistinct = 0;
+    float prev = 0.0f;
+    for (int j = 0; j < ne - 1; ++j) {
+      const float x = tau[j];
+      if (x < lo_edge) ++nbelow;
+      else if (x <= hi_edge) {
+        if (ninside == 0 || x != prev) ++ndistinct;
+        prev = x;
+        ++ninside;
+      }
+    }
+    CellEntry e;
+    e.thr = ninside ? prev : INFINITY;
+    e.codes = ndistinct <= 1 ? ((unsigned)nbelow | ((unsigned)min(nbelow + ninside, ne - 1) << 8)) : 0xFFFFu;
+    cellt[r] = e;
+  }
+  __syncthreads();
 
+  const unsigned total4 = ws->list_count * 4u;                 // the cache as groups of four elements (two 16-byte loads)
+  ulonglong2* mine = acc + tid;
   double D = 0.0;
-  for (unsigned i = blockIdx.x * BD + tid; i < count; i += gridDim.x * BD) {
-    const unsigned blk = a.pool_idx[i];
-    const unsigned m = blk / nbk, j = blk - m * nbk;
-    const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
-    const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
-    const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    float om[16];
-    unsigned fx[16];
-    {
-      const float4* op = reinterpret_cast<const float4*>(a.omega + (size_t)j * SOP_G);
-      const uint4* fp = reinterpret_cast<const uint4*>(a.omega_fix + (size_t)j * SOP_G);
+  const uint4* src = reinterpret_cast<const uint4*>(a.cache);
+  for (unsigned g = blockIdx.x * LTB + tid; g < total4; g += gridDim.x * LTB) {
+    const uint4 p0 = __ldg(src + 2 * (size_t)g), p1 = __ldg(src + 2 * (size_t)g + 1);
+    const float uu[4] = {__uint_as_float(p0.x), __uint_as_float(p0.z), __uint_as_float(p1.x), __uint_as_float(p1.z)};
+    const float oo[4] = {__uint_as_float(p0.y), __uint_as_float(p0.w), __uint_as_float(p1.y), __uint_as_float(p1.w)};
+    float dq = 0.0f;   // four positive fp32 terms, then FP64
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float4 o = __ldg(op + q);
-        const uint4 f = __ldg(fp + q);
-        om[4 * q] = o.x; om[4 * q + 1] = o.y; om[4 * q + 2] = o.z; om[4 * q + 3] = o.w;
-        fx[4 * q] = f.x; fx[4 * q + 1] = f.y; fx[4 * q + 2] = f.z; fx[4 * q + 3] = f.w;
-      }
-    }
-    uint32_t mb = 0;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
-    const float amax = __uint_as_float(mb << 16);
-    const float s_hat = scale_quantize(amax, k, F).s_hat;    // a DD table declares tmax = 1
-    const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
-    float dq[4] = {0.0f, 0.0f, 0.0f, 0.0f};   // the block's 16 distortion terms in fp32, four partial sums (all terms
-                                              // positive: relative error below 6e-7 in the worst case), then FP64
-#pragma unroll
-    for (int e = 0; e < 16; ++e) {
-      const float w = (e & 1) ? bf16hi(wb[e >> 1]) : bf16lo(wb[e >> 1]);
-      const float u = __fmul_rn(w, rcp);
-      const int code = count_below(tau, u);
+    for (int e4 = 0; e4 < 4; ++e4) {
+      const float u = uu[e4], om = oo[e4];
+      const CellEntry e = cellt[sort_cell(u)];
+      int code;
+      if (e.codes == 0xFFFFu) code = count_below(tau, u);
+      else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
       const float d = __fsub_rn(u, lutv[code]);
-      dq[e & 3] = __fmaf_rn(__fmul_rn(om[e], d), d, dq[e & 3]);
+      dq = __fmaf_rn(__fmul_rn(om, d), d, dq);
       if (!last) {
-        const float ou = fminf(fmaxf(__fmul_rn(om[e], u), -256.0f), 256.0f);
-        ulonglong2 t = mine[code * BD];
-        t.x += (unsigned long long)fx[e];
-        t.y += (unsigned long long)__float2ll_rn(__fmul_rn(ou, 16777216.0f));
-        mine[code * BD] = t;
+        const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
+        ulonglong2 t = mine[code * LTB];
+        t.x += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
+        t.y += (unsigned long long)fix24(ou);
+        mine[code * LTB] = t;
       }
     }
-    D += (double)__fadd_rn(__fadd_rn(dq[0], dq[1]), __fadd_rn(dq[2], dq[3]));
+    D += (double)dq;
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
   if (lane == 0) sD[warp] = D;
   __syncthreads();
-  const int n_warps = BD >> 5;
   if (!last) {
-    for (int j = warp; j < ne; j += n_warps) {
-      unsigned long long n = 0, s = 0;
-      for (int q = lane; q < BD; q += 32) { const ulonglong2 t = acc[j * BD + q]; n += t.x; s += t.y; }
-      for (int o = 16; o; o >>= 1) { n += __shfl_xor_sync(0xFFFFFFFFu, n, o); s += __shfl_xor_sync(0xFFFFFFFFu, s, o); }
+    for (int j = warp; j < ne; j += LTB / 32) {
+      unsigned long long n = 0, sv = 0;
+      for (int q = lane; q < LTB; q += 32) { const ulonglong2 t = acc[j * LTB + q]; n += t.x; sv += t.y; }
+      for (int o = 16; o; o >>= 1) { n += __shfl_xor_sync(0xFFFFFFFFu, n, o); sv += __shfl_xor_sync(0xFFFFFFFFu, sv, o); }
       if (lane == 0) {
         if (n) atomicAdd(&ws->accN[j], n);
-        if (s) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[j]), s);
+        if (sv) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[j]), sv);
       }
     }
   }
   if (tid == 0) {
     double t = 0.0;
-    for (int w = 0; w < n_warps; ++w) t += sD[w];
+    for (int w = 0; w < LTB / 32; ++w) t += sD[w];
     if (t != 0.0) atomicAdd(&ws->accD, t);
   }
   // the CTA that arrives last owns the update; no CTA waits for another
@@ -401,8 +457,8 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   a.M = M; a.K = K; a.ldw = ldw; a.nbk = K / SOP_G; a.NB = NB; a.pool_rank = pool_rank;
   a.k_mode = k_mode; a.fmta_index = fmta_index; a.n_atoms = n_atoms;
   a.omega = (float*)(wsb + lloyd_off_omega());
-  a.omega_fix = (unsigned*)(wsb + lloyd_off_fix(K));
   a.pool_idx = (unsigned*)(wsb + lloyd_off_idx(K));
+  a.cache = (uint2*)(wsb + lloyd_off_cache(M, K));
   LloydWs* ws = (LloydWs*)workspace_dev;
   cudaStream_t st = (cudaStream_t)stream;
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(LloydWs), st));
@@ -419,24 +475,29 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   pool_list_kernel<<<(int)sg, LTB, 0, st>>>(a, ws);
   SOP_CUDA_TRY(cudaGetLastError());
 
-  // iteration kernel: the per-thread accumulator slots bound the threads per SM (16 bytes x entries x threads)
+  // (u, omega) of every pool element, once
+  {
+    long long cg = (NB + LTB - 1) / LTB;      // one pool block per thread: the kernel is bound by memory latency
+    if (cg > (long long)sms * 16) cg = (long long)sms * 16;
+    pool_cache_kernel<<<(int)cg, LTB, 0, st>>>(a, F, ws);
+  }
+  SOP_CUDA_TRY(cudaGetLastError());
   int max_entries = 2;
   for (int i = 0; i < n_atoms; ++i)
     if (atoms[i].kind == SOP_KIND_LUT && atoms[i].n_entries > max_entries) max_entries = atoms[i].n_entries;
-  const int bd = max_entries <= 16 ? 256 : 128;
-  const size_t smem = (size_t)max_entries * bd * sizeof(ulonglong2);
+  const size_t smem = (size_t)max_entries * LTB * sizeof(ulonglong2);   // 64 KB for 16 entries, 128 KB for 32
   static size_t smem_set = 0;
-  if (smem > 48 * 1024 && smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(lloyd_iter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+  if (smem > 40 * 1024 && smem > smem_set) {
+    SOP_CUDA_TRY(cudaFuncSetAttribute(lloyd_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
     smem_set = 128 * 1024;
   }
-  const int per_sm = (int)((200 * 1024) / (smem + 2048));
-  long long grid = (NB + bd - 1) / bd;
+  const int per_sm = (int)((220 * 1024) / (smem + 8 * 1024));
+  long long grid = (NB * 4 + LTB - 1) / LTB;
   if (grid > (long long)sms * per_sm) grid = (long long)sms * per_sm;
   if (grid < 1) grid = 1;
   for (int it = 0; it <= iters; ++it) {
     const int last = it == iters;
-    lloyd_iter_kernel<<<(int)grid, bd, smem, st>>>(a, F, ws, distortion_dev, it, last, out_lut_dev);
+    lloyd_stream_kernel<<<(int)grid, LTB, smem, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
   }
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;

@@ -100,7 +100,7 @@ class LayerSweep:
             n += 4
             B.sop_dd4_lloyd(W, self.c, self.fmt, self.full_atoms, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
-            n += 5 + (self.iters + 1)
+            n += 6 + (self.iters + 1)
             B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
                               block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask, stream=stream)
