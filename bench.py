@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the SOP per-layer candidate sweep on B200.
 
-One step = one pass of the whole hot path over one synthetic layer: channel norms, sweep of the
-ROM alphabet, DD4 Lloyd refinement, sweep of the full alphabet (all pairs), pack of the chosen pair.
+One step = one pass of the whole hot path over one synthetic layer: channel norms, sweep of every fixed
+candidate (single-candidate reduction: finds FMTa), DD4 Lloyd refinement, sweep of the two DD4 columns
+with the fixed candidates' per-block values loaded (all pairs), pack of the chosen pair.
 Workload at every N: the attention-projection configuration (W 4096 x 4096 bf16 with 1 % outlier
 channels, X 512 x 4096, E5M6 scale, NF4/SH4/BOF4/Split87/DD4 and negations plus E2M3/E4M3 singles).
 With N > 1 every rank sweeps its own layer (layers are independent: no data-path collective).
@@ -35,11 +36,17 @@ WORKLOAD = dict(workload="config2: attention projection 4096x4096 bf16, 1% outli
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 
 
-def ops_per_element(n_lut: int, n_bits: int, n_fp: int, n_pairs: int, n_cand: int) -> float:
-    """Algorithmic thread-level operations per weight element of one sweep: 6 shared, 2n + 5 per LUT
-    candidate (n-step search + reconstruct + 4 fused multiply-adds), 12 per FP candidate, and per
-    block 2 per pair plus 6 per candidate (sqrt, divide, products)."""
-    return 6 + n_lut * (2 * n_bits + 5) + n_fp * 12 + (2 * n_pairs + 6 * n_cand) / 16.0
+def sweep_ops_per_element(n_lut: int, n_bits: int, n_fp: int, n_loaded: int, n_slots2: int, n_slots4: int) -> float:
+    """Algorithmic thread-level operations per weight element of one sweep launch: 6 shared (unpack,
+    absmax, c w, norm, u), 2n + 5 per evaluated LUT candidate (n-step search + reconstruct + 4 fused
+    multiply-adds), 12 per evaluated FP candidate, and per block: 6 per evaluated candidate (sqrt,
+    divide, products), 2 per loaded candidate, 2 per two-way table entry and 6 per four-way entry."""
+    n_eval = n_lut + n_fp
+    return 6 + n_lut * (2 * n_bits + 5) + n_fp * 12 + (6 * n_eval + 2 * n_loaded + 2 * n_slots2 + 6 * n_slots4) / 16.0
+
+
+LLOYD_BYTES_PER_POOL_ELEMENT = 8.0     # one (u, omega) pair read per pool element and iteration
+LLOYD_OPS_PER_POOL_ELEMENT = 20.0      # cell index 4, entry select 3, distortion 3, fixed-point sums 10
 
 
 class ClockSampler:
@@ -172,11 +179,16 @@ def run_gpu(args) -> None:
         sampler.start()
         time.sleep(0.3)
     barrier()
-    evs, sweep_ms = [], []
+    evs, kern = [], dict(sweep1=[], sweep2=[], lloyd=[], pack=[], norms=[])
     t_wall = time.perf_counter()
     for _ in range(args.steps):
         evs.append(one_step())
-        sweep_ms.append(B.profile_last_sweep_ms())       # waits for this step's full-alphabet sweep kernel
+        # the library's own events around its main kernels, on the launching stream (waits for this step)
+        kern["sweep2"].append(B.profile_ms(B.PROFILE_SWEEP, 0))
+        kern["sweep1"].append(B.profile_ms(B.PROFILE_SWEEP, 1))
+        kern["lloyd"].append(B.profile_ms(B.PROFILE_LLOYD, 0))
+        kern["pack"].append(B.profile_ms(B.PROFILE_PACK, 0))
+        kern["norms"].append(B.profile_ms(B.PROFILE_NORMS, 0))
     barrier()
     t_wall = time.perf_counter() - t_wall
     step_ms = [a.elapsed_time(b) for a, b in evs]
@@ -215,10 +227,14 @@ def run_gpu(args) -> None:
     e2e_ms = e0.elapsed_time(e1) / args.steps
 
     ms = sum(step_ms) / len(step_ms)
-    t = torch.tensor([ms, e2e_ms, sum(sweep_ms) / len(sweep_ms)], dtype=torch.float64, device=dev)
+    kavg = {k: sum(v) / len(v) for k, v in kern.items()}
+    knames = sorted(kavg)
+    t = torch.tensor([ms, e2e_ms] + [kavg[k] for k in knames], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, sw_ms = (float(x) for x in t.cpu())
+    vals = [float(x) for x in t.cpu()]
+    ms, e2e_ms = vals[0], vals[1]
+    kavg = dict(zip(knames, vals[2:]))
     E = M * K
     if rank == 0:
         peaks = {}
@@ -227,14 +243,42 @@ def run_gpu(args) -> None:
         except OSError:
             pass
         full = sw.full_atoms
+        nb = full[0].n_bits
         n_lut = sum(a.kind == I.KIND_LUT for a in full)
         n_fp = len(full) - n_lut
-        n_pairs = n_lut * (n_lut + 1) // 2 + n_fp + (len(WORKLOAD["rom"]) + 1) * (len(WORKLOAD["rom"]) + 2) // 2 * fmt.sign_bits
-        ops = ops_per_element(n_lut, full[0].n_bits, n_fp, n_pairs, len(full)) * E
+        n_dd = bin(sw.dd_mask).count("1")
+        n_base = (n_lut // 2) if fmt.sign_bits else 0
+        slots2 = len(full) + n_lut * (n_lut - 1) // 2
+        slots4 = n_base * (n_base + 1) // 2
+        ops1 = sweep_ops_per_element(n_lut - n_dd, nb, n_fp, 0, len(full) - n_dd, 0)      # fixed candidates, singles only
+        ops2 = sweep_ops_per_element(n_dd, nb, 0, len(full) - n_dd, slots2, slots4)       # DD columns, every pair
         sm_max = peaks.get("sm_max_mhz", 1965.0)
         alu_peak = SM_COUNT * SCHEDULERS * LANES * sm_max * 1e6 / 1e12          # T thread-instructions/s
-        achieved = ops / (sw_ms * 1e-3) / 1e12
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
+        of = "measured" if peaks else "fallback"
+        # sweep kernel: two launches per step; achieved = algorithmic ops of both / time of both
+        sweep_t = (kavg["sweep1"] + kavg["sweep2"]) * 1e-3
+        sweep_ach = (ops1 + ops2) * E / sweep_t / 1e12
+        sweep_roof = dict(kernel="sweep_kernel", launches_per_step=2, bound="alu", achieved=sweep_ach, peak=alu_peak,
+                          unit="T thread-instr/s", frac=sweep_ach / alu_peak, traffic=None,
+                          peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz (clocks.max.sm, {of})",
+                          ops_per_element=dict(fixed_candidates_singles=ops1, dd_columns_all_pairs=ops2),
+                          avg_launch_ms=sweep_t * 1e3 / 2,
+                          hbm=dict(achieved=2 * 2.0 * E / sweep_t / 1e9, peak=hbm_peak, unit="GB/s",
+                                   frac=2 * 2.0 * E / sweep_t / 1e9 / hbm_peak, of=of,
+                                   note="W read once per launch; the kernel is far from the HBM roofline"))
+        # Lloyd iteration kernel: iters + 1 launches per step, each streams 8 bytes per pool element
+        pool_elems = sw.pool_rank * 16
+        n_it = sw.iters + 1
+        lloyd_t = kavg["lloyd"] * 1e-3
+        lloyd_ach = LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e9
+        lloyd_roof = dict(kernel="lloyd_stream_kernel", launches_per_step=n_it, bound="hbm", achieved=lloyd_ach, peak=hbm_peak,
+                          unit="GB/s", frac=lloyd_ach / hbm_peak, traffic=None, of=of, avg_launch_ms=lloyd_t * 1e3 / n_it,
+                          bytes_per_launch=LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems,
+                          alu=dict(achieved=LLOYD_OPS_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e12, peak=alu_peak,
+                                   unit="T thread-instr/s",
+                                   frac=LLOYD_OPS_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e12 / alu_peak))
+        dominant, other = (sweep_roof, lloyd_roof) if sweep_t >= lloyd_t else (lloyd_roof, sweep_roof)
         cpu_rows = 1024
         cpu_val, cpu_dt = cpu_oracle_time(cpu_rows)
         line = dict(
@@ -242,14 +286,10 @@ def run_gpu(args) -> None:
             warmup=max(3, args.warmup), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
             dtype="f32", data="synthetic", config=dict(WORKLOAD, l2="flushed between timed steps (256 MB write)",
                                                        parallelism=f"layer-parallel x{world}, no collective"),
-            sweep_kernel=dict(ms=sw_ms, value=E / (sw_ms * 1e-3) / 1e9, unit=UNIT,
-                              note="full-alphabet sweep kernel alone, CUDA events around the launch"),
-            roofline=dict(bound="alu", achieved=achieved, peak=alu_peak, unit="T thread-instr/s", frac=achieved / alu_peak,
-                          traffic=None, peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz "
-                                                    "(clocks.max.sm of measured peaks file)" if peaks else "fallback clocks",
-                          ops_per_element=ops / E,
-                          hbm=dict(achieved=4.0 * E / (sw_ms * 1e-3) / 1e9, peak=hbm_peak, unit="GB/s",
-                                   frac=4.0 * E / (sw_ms * 1e-3) / 1e9 / hbm_peak, of="measured" if peaks else "fallback")),
+            kernels_ms=dict(kavg, note="per step, CUDA events recorded by the library around its main kernels; "
+                                       "sweep1 = fixed candidates (singles), sweep2 = DD columns (all pairs), "
+                                       "lloyd = all iteration launches"),
+            roofline=dominant, roofline_other=other,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
                               sample=f"first {cpu_rows} of {M} rows, whole pipeline, {cpu_dt:.1f} s"),
             e2e=dict(value=world * E / (e2e_ms * 1e-3) / 1e9, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,

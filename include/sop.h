@@ -145,12 +145,20 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
                     sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream);
 
-/* Measurement aid (no counterpart in the paper): with profiling enabled, sop_pair_search records a
- * CUDA event on `stream` directly before and after its sweep kernel; sop_profile_last_sweep_ms
- * waits for the second event and returns that one launch's duration in milliseconds
- * (SOP_ERR_RANGE if no sweep has run since profiling was enabled).  Not thread-safe. */
+/* Measurement aid (no counterpart in the paper): with profiling enabled, an entry point records a
+ * CUDA event on `stream` directly before the first and after the last launch of its main kernel:
+ *   SOP_PROFILE_SWEEP   the sweep kernel of sop_pair_search (one launch)
+ *   SOP_PROFILE_LLOYD   the iteration kernel of sop_dd4_lloyd (iters + 1 launches)
+ *   SOP_PROFILE_PACK    the kernel of sop_pack
+ *   SOP_PROFILE_NORMS   both kernels of sop_channel_norms
+ * sop_profile_ms waits for the second event of a call of that kind (back = 0: the last call, 1: the one
+ * before, ... up to 7) and returns the time between its two events in milliseconds (SOP_ERR_RANGE if
+ * no such call has run since profiling was enabled).  Not thread-safe. */
+enum { SOP_PROFILE_SWEEP = 0, SOP_PROFILE_LLOYD = 1, SOP_PROFILE_PACK = 2, SOP_PROFILE_NORMS = 3, SOP_PROFILE_KINDS = 4 };
 int sop_profile_enable(int on);
-int sop_profile_last_sweep_ms(float* ms);
+int sop_profile_ms(int which, int back, float* ms);
+int sop_profile_last_ms(int which, float* ms);    /* = sop_profile_ms(which, 0, ms) */
+int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE_SWEEP, ms) */
 
 /* ---- DD-n: per-layer data-derived codebook by Lloyd iteration (pair-search steps 2-3) -------
  * Pool = blocks whose cosine under the primary codebook FMTa is <= the pool_rank-th smallest of

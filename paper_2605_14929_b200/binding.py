@@ -78,7 +78,7 @@ def lib():
 def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
             "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd", "sop_pack",
-            "sop_profile_enable", "sop_profile_last_sweep_ms"]
+            "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
 
 
 def _check(rc: int, where: str):
@@ -193,10 +193,22 @@ def profile_enable(on: bool) -> None:
     _check(lib().sop_profile_enable(1 if on else 0), "sop_profile_enable")
 
 
-def profile_last_sweep_ms() -> float:
+PROFILE_SWEEP, PROFILE_LLOYD, PROFILE_PACK, PROFILE_NORMS = 0, 1, 2, 3
+
+
+def profile_ms(which: int, back: int = 0) -> float:
+    """Milliseconds of the main kernel(s) of the ``back``-th last call of that kind (waits for it)."""
     ms = C.c_float()
-    _check(lib().sop_profile_last_sweep_ms(C.byref(ms)), "sop_profile_last_sweep_ms")
+    _check(lib().sop_profile_ms(which, back, C.byref(ms)), "sop_profile_ms")
     return ms.value
+
+
+def profile_last_ms(which: int) -> float:
+    return profile_ms(which, 0)
+
+
+def profile_last_sweep_ms() -> float:
+    return profile_last_ms(PROFILE_SWEEP)
 
 
 # ------------------------------------------------------------------ result readers (device -> host)

@@ -13,6 +13,25 @@ void set_cuda_error(cudaError_t e, const char* where) {
   snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e), where);
 }
 
+constexpr int PROFILE_RING = 8;            // the last eight calls of every kind stay readable
+static bool g_profile = false;
+static cudaEvent_t g_ev[SOP_PROFILE_KINDS][PROFILE_RING][2];
+static bool g_ev_made = false;
+static long long g_ev_count[SOP_PROFILE_KINDS];
+
+int profile_mark(int which, int edge, cudaStream_t st) {
+  if (!g_profile) return SOP_OK;
+  if (!g_ev_made) {
+    for (int i = 0; i < SOP_PROFILE_KINDS; ++i)
+      for (int r = 0; r < PROFILE_RING; ++r)
+        for (int e = 0; e < 2; ++e) SOP_CUDA_TRY(cudaEventCreate(&g_ev[i][r][e]));
+    g_ev_made = true;
+  }
+  SOP_CUDA_TRY(cudaEventRecord(g_ev[which][g_ev_count[which] % PROFILE_RING][edge], st));
+  if (edge == 1) ++g_ev_count[which];
+  return SOP_OK;
+}
+
 int validate_fmt(const sop_scale_fmt* f, FmtDev* out) {
   if (!f) return SOP_ERR_NULL;
   if (f->exp_bits < 1 || f->exp_bits > 8 || f->man_bits < 0 || f->man_bits > 10) return SOP_ERR_FORMAT;
@@ -135,7 +154,25 @@ const char* sop_strerror(int code) {
 
 const char* sop_last_cuda_error(void) { return sop::g_cuda_error; }
 
-int sop_version(void) { return 100; }
+int sop_version(void) { return 101; }
+
+int sop_profile_enable(int on) {
+  sop::g_profile = on != 0;
+  for (int i = 0; i < SOP_PROFILE_KINDS; ++i) sop::g_ev_count[i] = 0;
+  return SOP_OK;
+}
+
+int sop_profile_ms(int which, int back, float* ms) {
+  if (!ms) return SOP_ERR_NULL;
+  if (which < 0 || which >= SOP_PROFILE_KINDS || back < 0 || back >= sop::PROFILE_RING || back >= sop::g_ev_count[which]) return SOP_ERR_RANGE;
+  cudaEvent_t* ev = sop::g_ev[which][(sop::g_ev_count[which] - 1 - back) % sop::PROFILE_RING];
+  SOP_CUDA_TRY(cudaEventSynchronize(ev[1]));
+  SOP_CUDA_TRY(cudaEventElapsedTime(ms, ev[0], ev[1]));
+  return SOP_OK;
+}
+
+int sop_profile_last_ms(int which, float* ms) { return sop_profile_ms(which, 0, ms); }
+int sop_profile_last_sweep_ms(float* ms) { return sop_profile_ms(SOP_PROFILE_SWEEP, 0, ms); }
 
 int sop_channel_norms_workspace(long long T, long long K, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
@@ -155,10 +192,13 @@ int sop_channel_norms(const float* X_dev, long long T, long long K, long long ld
   if (n_chunks > 65535) return SOP_ERR_SHAPE;
   cudaStream_t st = (cudaStream_t)stream;
   dim3 grid((unsigned)((K + 255) / 256), (unsigned)n_chunks);
+  int rc;
+  if ((rc = sop::profile_mark(SOP_PROFILE_NORMS, 0, st))) return rc;
   sop::norms_partial_kernel<<<grid, 256, 0, st>>>(X_dev, T, K, ldx, (double*)workspace_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   sop::norms_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>((const double*)workspace_dev, n_chunks, K, T, c_dev);
   SOP_CUDA_TRY(cudaGetLastError());
+  if ((rc = sop::profile_mark(SOP_PROFILE_NORMS, 1, st))) return rc;
   return SOP_OK;
 }
 

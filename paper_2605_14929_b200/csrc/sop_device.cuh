@@ -26,6 +26,10 @@ void set_cuda_error(cudaError_t e, const char* where);
     }                                                      \
   } while (0)
 
+// Optional timing of one kernel family of a call (CUDA events on the launching stream): edge 0 before
+// the first launch, edge 1 after the last.  No-op unless profiling is enabled.
+int profile_mark(int which, int edge, cudaStream_t st);
+
 // ---- kernel parameter blocks ---------------------------------------------------------------
 struct FmtDev {
   int y;                // mantissa bits

@@ -495,10 +495,12 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   long long grid = (NB * 4 + LTB - 1) / LTB;
   if (grid > (long long)sms * per_sm) grid = (long long)sms * per_sm;
   if (grid < 1) grid = 1;
+  if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
   for (int it = 0; it <= iters; ++it) {
     const int last = it == iters;
     lloyd_stream_kernel<<<(int)grid, LTB, smem, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
   }
+  if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }

@@ -326,9 +326,11 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   long long grid = (a.NB + PTB - 1) / PTB;
   const int sms = num_sms();
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+  if ((rc = profile_mark(SOP_PROFILE_PACK, 0, st))) return rc;
   const bool negs_known = !use_sign || from_result || (a.cos_neg_a >= 0 && (!pair || a.cos_neg_b >= 0));
   if (block_cos_dev && negs_known) pack_kernel<true><<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
   else pack_kernel<false><<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
+  if ((rc = profile_mark(SOP_PROFILE_PACK, 1, st))) return rc;
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }

@@ -825,11 +825,6 @@ size_t sweep_smem_bytes(const Plan& P) {
   return (b + 15) & ~(size_t)15;
 }
 
-// optional timing of the sweep kernel alone (CUDA events on the launching stream)
-static bool g_profile = false;
-static cudaEvent_t g_ev0 = nullptr, g_ev1 = nullptr;
-static bool g_ev_valid = false;
-
 static int g_num_sms = 0;
 int num_sms() {
   if (!g_num_sms) {
@@ -843,20 +838,6 @@ int num_sms() {
 }  // namespace sop
 
 extern "C" {
-
-int sop_profile_enable(int on) {
-  sop::g_profile = on != 0;
-  sop::g_ev_valid = false;
-  return SOP_OK;
-}
-
-int sop_profile_last_sweep_ms(float* ms) {
-  if (!ms) return SOP_ERR_NULL;
-  if (!sop::g_ev_valid) return SOP_ERR_RANGE;
-  SOP_CUDA_TRY(cudaEventSynchronize(sop::g_ev1));
-  SOP_CUDA_TRY(cudaEventElapsedTime(ms, sop::g_ev0, sop::g_ev1));
-  return SOP_OK;
-}
 
 int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
@@ -926,13 +907,10 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   const long long min_grid = (L.nbk + TB - 1) / TB;
   if (grid < min_grid) grid = min_grid;
   if (grid > MAX_GRID) return SOP_ERR_SHAPE;
-  if (g_profile) {
-    if (!g_ev0) { SOP_CUDA_TRY(cudaEventCreate(&g_ev0)); SOP_CUDA_TRY(cudaEventCreate(&g_ev1)); }
-    SOP_CUDA_TRY(cudaEventRecord(g_ev0, st));
-  }
+  if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
   sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev);
   SOP_CUDA_TRY(cudaGetLastError());
-  if (g_profile) { SOP_CUDA_TRY(cudaEventRecord(g_ev1, st)); g_ev_valid = true; }
+  if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
   finalize_kernel<<<1, FIN_TB, 0, st>>>(L, P, F, (int)grid, partials, pair_table_dev, signed_table_dev, result_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
