@@ -18,6 +18,28 @@ from . import binding as B
 from . import inputs as I
 
 
+def layers_for_rank(n_layers: int, rank: int, world: int) -> List[int]:
+    """Layer-parallel sharding: layers are independent units of the sweep, layer l goes to rank
+    l mod world; no data-path collective is involved."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("need 0 <= rank < world")
+    return list(range(rank, n_layers, world))
+
+
+def job_throughput(units_per_rank: float, local_seconds: float, group=None) -> float:
+    """Whole-job throughput of a layer-parallel run: the units all ranks processed divided by the
+    slowest rank's time (sum and max over the process group; a single process when no group is up)."""
+    import torch.distributed as dist
+    t = torch.tensor([units_per_rank, local_seconds], dtype=torch.float64)
+    if dist.is_available() and dist.is_initialized():
+        dev = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend(group) == "nccl" else torch.device("cpu")
+        units, secs = t[:1].to(dev), t[1:].to(dev)
+        dist.all_reduce(units, op=dist.ReduceOp.SUM, group=group)
+        dist.all_reduce(secs, op=dist.ReduceOp.MAX, group=group)
+        return float(units.item() / secs.item())
+    return float(t[0] / t[1])
+
+
 def scale_word_container(fmt, need_sign: bool, need_selector: bool) -> int:
     """Smallest container b in {8, 12, 16} holding sign + exponent + mantissa + selector."""
     need = fmt.exp_bits + fmt.man_bits + (1 if need_sign else 0) + (1 if need_selector else 0)
