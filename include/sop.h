@@ -42,7 +42,8 @@ enum {
   SOP_ERR_ALPHABET = -4,   /* bad atom: n_entries, unsorted or non-finite table, tmax <= 0, too many atoms */
   SOP_ERR_WORKSPACE = -5,  /* workspace NULL, misaligned (256 B) or too small */
   SOP_ERR_CUDA = -6,       /* a CUDA runtime call failed; see sop_last_cuda_error() */
-  SOP_ERR_RANGE = -7       /* k shift outside [-64, 64], pool_rank outside [1, N_b], iters outside [0, 64] */
+  SOP_ERR_RANGE = -7,      /* k shift outside [-64, 64], pool_rank outside [1, N_b], iters outside [0, 64] */
+  SOP_ERR_TOO_LARGE = -8   /* sop_channel_norms_static: ceil(T/64) * K exceeds the built-in scratch */
 };
 
 enum { SOP_KIND_LUT = 0, SOP_KIND_FP_E2M3 = 1, SOP_KIND_FP_E4M3 = 2 };
@@ -107,6 +108,27 @@ int sop_version(void);
 int sop_channel_norms_workspace(long long T, long long K, size_t* bytes);
 int sop_channel_norms(const float* X_dev, long long T, long long K, long long ldx, float* c_dev,
                       void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---- channel norms for callers that cannot allocate (the paper has no counterpart: this is a
+ *      packaging variant of sop_channel_norms, same arithmetic, same result bit for bit) ---------
+ * Who needs it: a caller that may not, or cannot, obtain device memory for the workspace -- a
+ * serving process that handed all device memory to its own arena at start-up and treats any later
+ * cudaMalloc as a fault, a latency-critical loop that must avoid the device-wide synchronisation
+ * that cudaMalloc / cudaFree imply, or a plug-in that is handed only the tensors and owns no
+ * allocator.  This entry point takes no workspace and calls no allocation routine: its scratch is
+ * a fixed array of SOP_NORMS_STATIC_DOUBLES doubles (4 MiB) that is part of the library image on
+ * every GPU that loads the library, for the life of the process.
+ *   Limit: ceil(T / 64) * K <= SOP_NORMS_STATIC_DOUBLES, else SOP_ERR_TOO_LARGE (for example
+ *   T = 2048 tokens at K = 14336, or T = 1024 at K = 28672, fit; T = 4096 at K = 14336 does not).
+ *   First call on a device: looks up the array's device address (one cudaGetSymbolAddress with that
+ *   device current) and remembers it; make that first call outside any stream capture.
+ *   Sharing: every call on a device uses the same array and finds the previous call's partials in
+ *   it.  Nothing needs clearing (each call overwrites every partial it reads), but two calls whose
+ *   kernels can overlap on the GPU -- different streams, no ordering between them -- would
+ *   overwrite each other's partials: order such calls (one stream, or events).
+ * X_dev, T, K, ldx, c_dev, stream: as for sop_channel_norms. */
+#define SOP_NORMS_STATIC_DOUBLES (1 << 19)
+int sop_channel_norms_static(const float* X_dev, long long T, long long K, long long ldx, float* c_dev, void* stream);
 
 /* ---- the candidate sweep (Sections "Block Scaling", "ACos", "Per-Layer Pair Search" step 4,
  *      "Per-layer scale shift") ----------------------------------------------------------------

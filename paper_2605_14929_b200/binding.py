@@ -77,6 +77,7 @@ def lib():
 
 def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
+            "sop_channel_norms_static",
             "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd", "sop_pack",
             "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
 
@@ -147,6 +148,20 @@ def sop_channel_norms(X: torch.Tensor, c_out: torch.Tensor, workspace: torch.Ten
     T, K = X.shape
     _check(lib().sop_channel_norms(_ptr(X), _ll(T), _ll(K), _ll(X.stride(0)), _ptr(c_out), _ptr(workspace),
                                    C.c_size_t(workspace.numel()), _stream(stream)), "sop_channel_norms")
+
+
+NORMS_STATIC_DOUBLES = 1 << 19
+
+
+def sop_channel_norms_static(X: torch.Tensor, c_out: torch.Tensor, stream=None) -> None:
+    """Channel norms with the library's built-in scratch instead of a caller workspace: for callers
+    that must not allocate device memory.  Needs ceil(T / 64) * K <= NORMS_STATIC_DOUBLES; calls on
+    one device share the scratch and must not overlap on the GPU."""
+    assert X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    assert c_out.is_cuda and c_out.dtype == torch.float32 and c_out.is_contiguous()
+    T, K = X.shape
+    _check(lib().sop_channel_norms_static(_ptr(X), _ll(T), _ll(K), _ll(X.stride(0)), _ptr(c_out), _stream(stream)),
+           "sop_channel_norms_static")
 
 
 def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair_table: torch.Tensor,

@@ -148,6 +148,7 @@ const char* sop_strerror(int code) {
     case SOP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case SOP_ERR_CUDA: return "CUDA runtime error (see sop_last_cuda_error)";
     case SOP_ERR_RANGE: return "argument out of range (k shift, pool_rank, iters or index)";
+    case SOP_ERR_TOO_LARGE: return "problem larger than the built-in scratch of the no-allocation entry point";
     default: return "unknown error code";
   }
 }
@@ -199,6 +200,56 @@ int sop_channel_norms(const float* X_dev, long long T, long long K, long long ld
   sop::norms_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>((const double*)workspace_dev, n_chunks, K, T, c_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   if ((rc = sop::profile_mark(SOP_PROFILE_NORMS, 1, st))) return rc;
+  return SOP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Channel norms without a caller workspace.  The chunk partials live in a fixed array inside the
+// library image: SOP_NORMS_STATIC_DOUBLES doubles (4 MiB) on every GPU that loads the library, held
+// until the process exits.  Host code cannot use the array's name as a pointer (on the host it is
+// only a handle for the symbol), so its device address is looked up once per device with
+// cudaGetSymbolAddress while that device is current, and that address is what the kernels get.
+// ---------------------------------------------------------------------------------------------
+namespace sop {
+static __device__ __align__(256) double g_norms_scratch[SOP_NORMS_STATIC_DOUBLES];
+
+constexpr int MAX_DEVICES = 64;
+static double* g_norms_scratch_addr[MAX_DEVICES];   // device address of g_norms_scratch, per device ordinal
+static bool g_norms_scratch_known[MAX_DEVICES];
+
+// Address of the scratch array on the current device (looked up on the first call per device).
+static int norms_scratch_address(double** out) {
+  int dev = -1;
+  SOP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return SOP_ERR_RANGE;
+  if (!g_norms_scratch_known[dev]) {
+    void* p = nullptr;
+    SOP_CUDA_TRY(cudaGetSymbolAddress(&p, g_norms_scratch));
+    g_norms_scratch_addr[dev] = static_cast<double*>(p);
+    g_norms_scratch_known[dev] = true;
+  }
+  *out = g_norms_scratch_addr[dev];
+  return SOP_OK;
+}
+}  // namespace sop
+
+int sop_channel_norms_static(const float* X_dev, long long T, long long K, long long ldx, float* c_dev, void* stream) {
+  if (!X_dev || !c_dev) return SOP_ERR_NULL;
+  if (T < 1 || K < 1 || ldx < K) return SOP_ERR_SHAPE;
+  const long long n_chunks = (T + 63) / 64;
+  if (n_chunks > 65535) return SOP_ERR_SHAPE;
+  if (n_chunks > SOP_NORMS_STATIC_DOUBLES / K) return SOP_ERR_TOO_LARGE;   // n_chunks * K doubles must fit the array
+  double* scratch = nullptr;
+  int rc = sop::norms_scratch_address(&scratch);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  // every partial that the second kernel reads is written by the first one in this call: nothing has
+  // to be cleared, whatever an earlier call left in the array
+  dim3 grid((unsigned)((K + 255) / 256), (unsigned)n_chunks);
+  sop::norms_partial_kernel<<<grid, 256, 0, st>>>(X_dev, T, K, ldx, scratch);
+  SOP_CUDA_TRY(cudaGetLastError());
+  sop::norms_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(scratch, n_chunks, K, T, c_dev);
+  SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }
 
