@@ -359,8 +359,16 @@ __global__ void __launch_bounds__(LTB) lloyd_stream_kernel(LloydArgs a, LloydWs*
   ulonglong2* mine = acc + tid;
   double D = 0.0;
   const uint4* src = reinterpret_cast<const uint4*>(a.cache);
-  for (unsigned g = blockIdx.x * LTB + tid; g < total4; g += gridDim.x * LTB) {
-    const uint4 p0 = __ldg(src + 2 * (size_t)g), p1 = __ldg(src + 2 * (size_t)g + 1);
+  const unsigned gstride = gridDim.x * LTB;
+  unsigned g = blockIdx.x * LTB + tid;
+  uint4 n0 = make_uint4(0u, 0u, 0u, 0u), n1 = n0;
+  if (g < total4) { n0 = __ldg(src + 2 * (size_t)g); n1 = __ldg(src + 2 * (size_t)g + 1); }
+  for (; g < total4; g += gstride) {
+    const uint4 p0 = n0, p1 = n1;
+    if (g + gstride < total4) {        // the next group's loads are in flight while this one is processed
+      n0 = __ldg(src + 2 * (size_t)(g + gstride));
+      n1 = __ldg(src + 2 * (size_t)(g + gstride) + 1);
+    }
     const float uu[4] = {__uint_as_float(p0.x), __uint_as_float(p0.z), __uint_as_float(p1.x), __uint_as_float(p1.z)};
     const float oo[4] = {__uint_as_float(p0.y), __uint_as_float(p0.w), __uint_as_float(p1.y), __uint_as_float(p1.w)};
     float dq = 0.0f;   // four positive fp32 terms, then FP64
