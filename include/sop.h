@@ -29,7 +29,7 @@ extern "C" {
 #define SOP_MAX_ATOMS 16       /* candidates per call, negations and FP formats included */
 #define SOP_MAX_ENTRIES 32     /* table entries per LUT atom (n <= 5) */
 #define SOP_K_AUTO (-1000)     /* k_mode: choose the F_layer shift on the device */
-#define SOP_K_FROM_RESULT (-1001) /* k_mode of sop_dd4_lloyd: take the shift from a previous search */
+#define SOP_K_FROM_RESULT (-1001) /* k_mode: take the shift(s) from the result block of a previous search */
 #define SOP_FMTA_FROM_RESULT (-1) /* fmta_index of sop_dd4_lloyd: best single LUT candidate of a previous search */
 #define SOP_ALL_ATOMS 0xFFFFFFFFu /* eval_mask of sop_pair_search: evaluate every candidate */
 #define SOP_SEARCH_SINGLES_ONLY 1 /* flags of sop_pair_search: reduce single candidates only, no pair / signed entries */
@@ -146,7 +146,8 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *     block index = m * (K/16) + j.
  * k_mode: SOP_K_AUTO runs the F_layer search per distinct tmax (maximise the number of blocks whose
  *   shifted scale exponent lies in the format's normal range, k in [-64, 64], ties to the smallest
- *   |k| then to k > 0); any other value in [-64, 64] is used as the shift for every candidate.
+ *   |k| then to k > 0); SOP_K_FROM_RESULT: see prev_result_dev; any other value in [-64, 64] is used as
+ *   the shift for every candidate.
  * dd_lut_dev (may be NULL): device table of SOP_MAX_ENTRIES floats that replaces, at kernel time,
  *   the lut of every atom whose index bit is set in dd_mask (a codebook produced by sop_dd4_lloyd
  *   can be swept without a host round trip).
@@ -158,11 +159,16 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *   its shift is reported as 0.  The masks must be disjoint and not both empty.  At most 8 distinct
  *   tables may be evaluated per call (an atom and its negation share one).
  * flags: SOP_SEARCH_SINGLES_ONLY fills only the diagonal (and best_single): enough to choose the
- *   primary codebook FMTa before the Lloyd refinement. */
+ *   primary codebook FMTa before the Lloyd refinement.
+ * prev_result_dev (may be NULL): with k_mode = SOP_K_FROM_RESULT, the result block of the earlier call on
+ *   this layer (not result_dev itself).  The shift of every scale class and max|W| are taken from it
+ *   instead of reading W once more; every per-block-scaled class of this call must then contain a
+ *   candidate of load_mask (SOP_ERR_RANGE otherwise). */
 int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes);
 int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                     const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
                     const float* dd_lut_dev, unsigned dd_mask, unsigned eval_mask, unsigned load_mask, int flags,
+                    const sop_search_result* prev_result_dev,
                     sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
                     sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream);

@@ -169,12 +169,13 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
                     k_mode: int = K_AUTO, dd_lut: Optional[torch.Tensor] = None, dd_mask: int = 0,
                     block_cos: Optional[torch.Tensor] = None, block_sse: Optional[torch.Tensor] = None,
                     stream=None, g: int = 16, eval_mask: int = ALL_ATOMS, load_mask: int = 0,
-                    singles_only: bool = False) -> None:
+                    singles_only: bool = False, prev_result: Optional[torch.Tensor] = None) -> None:
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_pair_search(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
                                  make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), C.c_uint(eval_mask),
-                                 C.c_uint(load_mask), SEARCH_SINGLES_ONLY if singles_only else 0, _ptr(pair_table),
+                                 C.c_uint(load_mask), SEARCH_SINGLES_ONLY if singles_only else 0, _ptr(prev_result),
+                                 _ptr(pair_table),
                                  _ptr(signed_table), _ptr(result), _ptr(block_cos), _ptr(block_sse), _ptr(workspace),
                                  C.c_size_t(workspace.numel()), _stream(stream)), "sop_pair_search")
 

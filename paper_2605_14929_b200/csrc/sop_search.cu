@@ -1,16 +1,16 @@
 // sop_pair_search: the per-layer candidate sweep.
 //
 //   prepass_kernel   reads W once: per-block absmax -> exponent histogram of sigma = absmax / tmax
-//                    for every scale class that needs an F_layer search, and max|W|.        (HBM-bound)
-//   kselect_kernel   one CTA: the F_layer shift k* per class from the histogram, the layer
-//                    power-of-two scale for "^0" candidates.
+//                    for every scale class that needs an F_layer search, and max|W|   (HBM-bound);
+//                    the CTA that finishes last derives the F_layer shift k* per class from the
+//                    histogram and the layer power-of-two scale for "^0" candidates.
 //   sweep_kernel     persistent, one thread per 16-element block: phase 1 evaluates every candidate
 //                    in registers (cell-table lookup of the reconstruction value, packed f32x2
 //                    fused multiply-adds for the block metric, fixed quad-tree order); phase 2
 //                    reduces the per-block (cos, sse) of the CTA's tile into per-pair sums, one
 //                    pair per thread, FP64 accumulators.                                    (ALU-bound)
-//   finalize_kernel  one CTA: adds the per-CTA partials in CTA order (deterministic), writes the
-//                    tables and picks the best pair / best single.
+//                    The CTA that finishes last adds the per-CTA partials in a fixed order
+//                    (deterministic), writes the tables and picks the best pair / best single.
 #include <math.h>
 #include <string.h>
 
@@ -34,6 +34,7 @@ struct ClassDev {
   unsigned char cand[SOP_MAX_ATOMS];
   int n_mem;                             // candidates present in this call (evaluated or loaded)
   unsigned char mem[SOP_MAX_ATOMS];
+  int k_src;                             // candidate whose shift an earlier result holds (k from result), or -1
 };
 struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (i0 == i1: single); 1: signed (i0, i0+1, i1, i1+1)
 
@@ -41,6 +42,7 @@ struct Plan {
   int n_atoms, n_classes, n_tables, n_slots, n_pair_slots;
   int k_mode, rows, a_pad;
   unsigned eval_mask, load_mask;   // candidates evaluated here / read from the per-block arrays of an earlier call
+  int k_from_result;               // 1: shifts and max|W| come from the result block of an earlier call, no prepass
   int red_t1, red_g0, red_g1;   // phase-2 thread split of a half CTA: [0, t1) pair slots in g0 groups, [t1, 256) signed slots in g1 groups
   CandDev cand[SOP_MAX_ATOMS];
   ClassDev cls[SOP_MAX_CLASSES];
@@ -56,7 +58,8 @@ struct WsHeader {
   unsigned wmax_bits;
   int cls_k[SOP_MAX_CLASSES];
   float cls_pot[SOP_MAX_CLASSES];
-  int pad[7];
+  unsigned done_prepass, done_sweep;   // CTAs that have finished (the last one does the serial tail)
+  int pad[5];
 };
 struct Partial { double gap, sse; long long n1, nneg; };
 
@@ -91,7 +94,9 @@ __device__ __forceinline__ float absmax_bits(const uint32_t (&v)[8]) {
   return __uint_as_float(m << 16);
 }
 
-__global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, unsigned* __restrict__ hist, WsHeader* __restrict__ hdr) {
+__device__ void kselect_body(const Plan& P, const FmtDev& F, const unsigned* hist, WsHeader* hdr);
+
+__global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, FmtDev F, unsigned* __restrict__ hist, WsHeader* __restrict__ hdr) {
   __shared__ unsigned sh[SOP_MAX_CLASSES * SOP_HIST_BINS];
   for (int i = threadIdx.x; i < P.n_classes * SOP_HIST_BINS; i += blockDim.x) sh[i] = 0;
   __syncthreads();
@@ -115,18 +120,29 @@ __global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, unsig
   __syncthreads();
   for (int i = threadIdx.x; i < P.n_classes * SOP_HIST_BINS; i += blockDim.x)
     if (sh[i]) atomicAdd(&hist[i], sh[i]);
+  // the CTA that arrives last turns the histogram into shifts; nobody waits for anybody
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&hdr->done_prepass, 1u) == gridDim.x - 1 ? 1 : 0;
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    kselect_body(P, F, hist, hdr);
+  }
 }
 
-__global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const unsigned* __restrict__ hist, WsHeader* __restrict__ hdr,
-                                                      sop_search_result* __restrict__ res) {
+// One CTA of at least 160 threads.  Reads the global histogram and max|W| through the L2 (they were
+// written by other CTAs' atomics).
+__device__ void kselect_body(const Plan& P, const FmtDev& F, const unsigned* hist, WsHeader* hdr) {
   __shared__ unsigned long long cnt[129];
   __shared__ unsigned sh_hist[SOP_HIST_BINS];
-  const float wmax = __uint_as_float(hdr->wmax_bits);
+  const float wmax = __uint_as_float(__ldcg(&hdr->wmax_bits));
   for (int cl = 0; cl < P.n_classes; ++cl) {
     int kstar = P.k_mode == SOP_K_AUTO ? 0 : P.k_mode;
     if (P.cls[cl].scope == 0) kstar = 0;
     if (P.cls[cl].auto_k) {
-      for (int i = threadIdx.x; i < SOP_HIST_BINS; i += blockDim.x) sh_hist[i] = hist[cl * SOP_HIST_BINS + i];
+      for (int i = threadIdx.x; i < SOP_HIST_BINS; i += blockDim.x) sh_hist[i] = __ldcg(&hist[cl * SOP_HIST_BINS + i]);
       __syncthreads();
       if (threadIdx.x < 129) {
         const int k = (int)threadIdx.x - 64;
@@ -150,14 +166,7 @@ __global__ void __launch_bounds__(160) kselect_kernel(Plan P, FmtDev F, const un
     if (threadIdx.x == 0) {
       hdr->cls_k[cl] = kstar;
       hdr->cls_pot[cl] = P.cls[cl].scope == 0 ? layer_pot_scale(wmax, P.cls[cl].tmax) : 0.0f;
-      for (int i = 0; i < P.cls[cl].n_mem; ++i) res->k[P.cls[cl].mem[i]] = kstar;
     }
-  }
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < SOP_MAX_ATOMS; ++i)
-      if (i >= P.n_atoms || !(((P.eval_mask | P.load_mask) >> i) & 1u)) res->k[i] = 0;
-    res->layer_absmax = wmax;
-    res->reserved[0] = res->reserved[1] = 0;
   }
 }
 
@@ -315,9 +324,15 @@ __device__ __forceinline__ void half_barrier(int half) {
 
 // The CTA works as two halves of 256 threads with a barrier each, so that one half reduces its tile
 // (phase 2) while the other still evaluates candidates (phase 1).
-__global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, const WsHeader* __restrict__ hdr,
+__device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const Partial* partials, sop_pair_stat* s_pair, sop_pair_stat* s_sig,
+                              Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
+                              const int* cls_k, float wmax);
+
+__global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, WsHeader* __restrict__ hdr,
                                                       Partial* __restrict__ partials, float* __restrict__ block_cos,
-                                                      float* __restrict__ block_sse) {
+                                                      float* __restrict__ block_sse, sop_pair_stat* __restrict__ pair_table,
+                                                      sop_pair_stat* __restrict__ signed_table, sop_search_result* __restrict__ res,
+                                                      const sop_search_result* __restrict__ prev) {
   extern __shared__ __align__(16) unsigned char smem[];
   uint2* cell = reinterpret_cast<uint2*>(smem);
   float* tau = reinterpret_cast<float*>(cell + (size_t)P.n_tables * P.rows * 16);
@@ -330,7 +345,17 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   constexpr int HB = TB / 2;
   const int tid = threadIdx.x, lane = tid & 31, half = tid / HB, htid = tid - half * HB;
   build_tables(P, A, cell, tau, lutv, fast);
-  if (tid < SOP_MAX_CLASSES) { cls_k[tid] = hdr->cls_k[tid]; cls_pot[tid] = hdr->cls_pot[tid]; }
+  const float layer_wmax = P.k_from_result ? prev->layer_absmax : __uint_as_float(hdr->wmax_bits);
+  if (tid < SOP_MAX_CLASSES) {
+    if (P.k_from_result) {
+      const bool live = tid < P.n_classes;
+      cls_k[tid] = live && P.cls[tid].k_src >= 0 ? prev->k[P.cls[tid].k_src] : 0;
+      cls_pot[tid] = live && P.cls[tid].scope == 0 ? layer_pot_scale(layer_wmax, P.cls[tid].tmax) : 0.0f;
+    } else {
+      cls_k[tid] = hdr->cls_k[tid];
+      cls_pot[tid] = hdr->cls_pot[tid];
+    }
+  }
   __syncthreads();
   constexpr int HBP = HB + 1;   // row pitch: candidates land in different banks
   float2* cs = cs_all + (size_t)half * P.n_atoms * HBP;
@@ -605,66 +630,113 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       }
     partials[(size_t)blockIdx.x * MAX_SLOTS + tid] = t;
   }
+  // the CTA that arrives last adds everybody's partials and writes the tables; nobody waits for anybody
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&hdr->done_sweep, 1u) == gridDim.x - 1 ? 1 : 0;
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    sop_pair_stat* s_pair = reinterpret_cast<sop_pair_stat*>(cs_all);
+    sop_pair_stat* s_sig = s_pair + SOP_MAX_ATOMS * SOP_MAX_ATOMS;
+    finalize_body(L, P, (int)gridDim.x, partials, s_pair, s_sig, reinterpret_cast<Partial*>(s_sig + SOP_MAX_ATOMS * SOP_MAX_ATOMS), pair_table,
+                  signed_table, res, cls_k, layer_wmax);
+  }
 }
 
-constexpr int FIN_TB = 1024;
+// Block-wide argmax of (value, index) with ties to the smaller index; index -1 = nothing.  `red` holds
+// blockDim.x / 32 entries.  Every thread returns the winner's index.
+__device__ int block_argmax(double v, int idx, double* red_v, int* red_i) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int o = 16; o; o >>= 1) {
+    const double ov = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const int oi = __shfl_xor_sync(0xFFFFFFFFu, idx, o);
+    if (oi >= 0 && (idx < 0 || ov > v || (ov == v && oi < idx))) { v = ov; idx = oi; }
+  }
+  __syncthreads();
+  if (lane == 0) { red_v[warp] = v; red_i[warp] = idx; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < n_warps; ++w) {
+      const double ov = red_v[w];
+      const int oi = red_i[w];
+      if (oi >= 0 && (idx < 0 || ov > v || (ov == v && oi < idx))) { v = ov; idx = oi; }
+    }
+    red_i[0] = idx;
+  }
+  __syncthreads();
+  return red_i[0];
+}
 
-// One warp per slot: lane l adds the partials of CTAs l, l + 32, ... in that order, then the lanes
-// are combined by a fixed butterfly: the result depends only on the grid size, not on scheduling.
-// The tables are staged in shared memory so that the final scan for the best pair reads no global memory.
-__global__ void __launch_bounds__(FIN_TB) finalize_kernel(LayerArgs L, Plan P, FmtDev F, int grid, const Partial* __restrict__ partials,
-                                                          sop_pair_stat* __restrict__ pair_table, sop_pair_stat* __restrict__ signed_table,
-                                                          sop_search_result* __restrict__ res) {
-  __shared__ sop_pair_stat s_pair[SOP_MAX_ATOMS * SOP_MAX_ATOMS], s_sig[SOP_MAX_ATOMS * SOP_MAX_ATOMS];
-  const int A = P.n_atoms, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// Run by one whole CTA of TB threads.  Thread (slot, chunk) adds the partials of CTAs chunk, chunk + C,
+// ... in that order (C = TB / n_slots chunks, loads coalesced over the slots), the chunks are then added
+// in chunk order: the result depends only on the grid size, not on scheduling.  s_pair / s_sig
+// (n_atoms^2 entries each) and s_red (TB entries) are shared-memory staging.
+__device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const Partial* partials, sop_pair_stat* s_pair, sop_pair_stat* s_sig,
+                              Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
+                              const int* cls_k, float wmax) {
+  __shared__ double red_v[TB / 32];
+  __shared__ int red_i[TB / 32];
+  const int A = P.n_atoms, tid = threadIdx.x, n_slots = P.n_slots;
   for (int i = tid; i < A * A; i += blockDim.x) {
     sop_pair_stat u; u.acos = 0.0; u.mse = 0.0; u.n_sel1 = -1; u.n_neg = -1;
     s_pair[i] = u;
     s_sig[i] = u;
   }
-  __syncthreads();
-  for (int slot = warp; slot < P.n_slots; slot += FIN_TB / 32) {
+  const int n_chunks = (int)blockDim.x / n_slots;
+  const int slot = tid % n_slots, chunk = tid / n_slots;
+  if (chunk < n_chunks) {
     Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
-    for (int g = lane; g < grid; g += 32) {
-      const Partial q = partials[(size_t)g * MAX_SLOTS + slot];
+    for (int g = chunk; g < grid; g += n_chunks) {
+      const double2* q = reinterpret_cast<const double2*>(partials + (size_t)g * MAX_SLOTS + slot);
+      const double2 a = __ldcg(q);
+      const longlong2 b = __ldcg(reinterpret_cast<const longlong2*>(q + 1));
+      t.gap += a.x; t.sse += a.y; t.n1 += b.x; t.nneg += b.y;
+    }
+    s_red[tid] = t;
+  }
+  __syncthreads();
+  if (tid < n_slots) {
+    Partial t = s_red[tid];
+    for (int c = 1; c < n_chunks; ++c) {
+      const Partial q = s_red[c * n_slots + tid];
       t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
     }
-    for (int o = 16; o; o >>= 1) {
-      t.gap += __shfl_xor_sync(0xFFFFFFFFu, t.gap, o);
-      t.sse += __shfl_xor_sync(0xFFFFFFFFu, t.sse, o);
-      t.n1 += __shfl_xor_sync(0xFFFFFFFFu, t.n1, o);
-      t.nneg += __shfl_xor_sync(0xFFFFFFFFu, t.nneg, o);
-    }
-    if (lane == 0) {
-      sop_pair_stat st;
-      st.acos = ((double)L.NB - t.gap) / (double)L.NB;
-      st.mse = t.sse / ((double)L.M * (double)L.K);
-      st.n_sel1 = t.n1;
-      const SlotDev sd = P.slots[slot];
-      if (sd.type == 0) { st.n_neg = 0; s_pair[sd.i0 * A + sd.i1] = st; }
-      else { st.n_neg = t.nneg; s_sig[sd.i0 * A + sd.i1] = st; }
-    }
+    sop_pair_stat st;
+    st.acos = ((double)L.NB - t.gap) / (double)L.NB;
+    st.mse = t.sse / ((double)L.M * (double)L.K);
+    st.n_sel1 = t.n1;
+    const SlotDev sd = P.slots[tid];
+    if (sd.type == 0) { st.n_neg = 0; s_pair[sd.i0 * A + sd.i1] = st; }
+    else { st.n_neg = t.nneg; s_sig[sd.i0 * A + sd.i1] = st; }
   }
   __syncthreads();
   for (int i = tid; i < A * A; i += blockDim.x) {
     pair_table[i] = s_pair[i];
     if (signed_table) signed_table[i] = s_sig[i];
   }
+  if (tid < SOP_MAX_ATOMS) {
+    const bool present = tid < A && (((P.eval_mask | P.load_mask) >> tid) & 1u);
+    res->k[tid] = present ? cls_k[P.cand[tid].cls] : 0;
+  }
+  // best two-codebook pair, best single LUT candidate, best signed pair: largest ACos, ties to the smallest (a, b)
+  const int a = tid / A, b = tid - a * A;
+  const bool in = tid < A * A;
+  int ip = -1, is = -1, isg = -1;
+  double vp = 0.0, vs = 0.0, vsg = 0.0;
+  if (in && b > a && s_pair[tid].n_sel1 >= 0) { ip = tid; vp = s_pair[tid].acos; }
+  if (in && b == a && P.cand[a].kind == SOP_KIND_LUT && s_pair[tid].n_sel1 >= 0) { is = tid; vs = s_pair[tid].acos; }
+  if (in && b > a && signed_table && s_sig[tid].n_sel1 >= 0) { isg = tid; vsg = s_sig[tid].acos; }
+  ip = block_argmax(vp, ip, red_v, red_i);
+  is = block_argmax(vs, is, red_v, red_i);
+  isg = block_argmax(vsg, isg, red_v, red_i);
   if (tid == 0) {
-    int ba = -1, bb = -1, bs = -1, bsa = -1, bsb = -1;
-    double vp = -2.0, vs = -2.0, vsp = -2.0;
-    for (int a = 0; a < A; ++a) {
-      if (P.cand[a].kind == SOP_KIND_LUT && s_pair[a * A + a].n_sel1 >= 0 && s_pair[a * A + a].acos > vs) { vs = s_pair[a * A + a].acos; bs = a; }
-      for (int b = a + 1; b < A; ++b) {
-        const sop_pair_stat p = s_pair[a * A + b];
-        if (p.n_sel1 >= 0 && p.acos > vp) { vp = p.acos; ba = a; bb = b; }
-        if (signed_table) {
-          const sop_pair_stat q = s_sig[a * A + b];
-          if (q.n_sel1 >= 0 && q.acos > vsp) { vsp = q.acos; bsa = a; bsb = b; }
-        }
-      }
-    }
-    res->best_a = ba; res->best_b = bb; res->best_single = bs; res->best_sa = bsa; res->best_sb = bsb;
+    res->layer_absmax = wmax;
+    res->reserved[0] = res->reserved[1] = 0;
+    res->best_a = ip >= 0 ? ip / A : -1; res->best_b = ip >= 0 ? ip % A : -1;
+    res->best_single = is >= 0 ? is / A : -1;
+    res->best_sa = isg >= 0 ? isg / A : -1; res->best_sb = isg >= 0 ? isg % A : -1;
   }
 }
 
@@ -820,7 +892,8 @@ size_t sweep_smem_bytes(const Plan& P) {
   size_t b = (size_t)P.n_tables * P.rows * 16 * 8;
   b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
   size_t tile = (size_t)2 * P.n_atoms * (TB / 2 + 1) * sizeof(float2);
-  const size_t red = sizeof(Partial) * (size_t)TB;
+  // the closing reduction of the last CTA: two staged tables and one partial per thread
+  const size_t red = sizeof(Partial) * (size_t)TB + 2 * sizeof(sop_pair_stat) * SOP_MAX_ATOMS * SOP_MAX_ATOMS;
   b += tile > red ? tile : red;
   return (b + 15) & ~(size_t)15;
 }
@@ -850,6 +923,7 @@ int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* byt
 int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                     const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
                     const float* dd_lut_dev, unsigned dd_mask, unsigned eval_mask, unsigned load_mask, int flags,
+                    const sop_search_result* prev_result_dev,
                     sop_pair_stat* pair_table_dev, sop_pair_stat* signed_table_dev,
                     sop_search_result* result_dev, float* block_cos_dev, float* block_sse_dev,
                     void* workspace_dev, size_t workspace_bytes, void* stream) {
@@ -861,7 +935,9 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if ((rc = validate_fmt(fmt, &F))) return rc;
   AtomsDev A;
   if ((rc = validate_atoms(atoms, n_atoms, dd_mask, dd_lut_dev, &A))) return rc;
-  if (k_mode != SOP_K_AUTO && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
+  const bool k_from_result = k_mode == SOP_K_FROM_RESULT;
+  if (k_mode != SOP_K_AUTO && !k_from_result && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
+  if (k_from_result && (!prev_result_dev || prev_result_dev == result_dev)) return SOP_ERR_NULL;
   if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < ws_total()) return SOP_ERR_WORKSPACE;
   const unsigned all = n_atoms >= 32 ? 0xFFFFFFFFu : ((1u << n_atoms) - 1u);
   eval_mask &= all;
@@ -869,7 +945,15 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if (load_mask && (!block_cos_dev || !block_sse_dev)) return SOP_ERR_NULL;
   if (flags & ~SOP_SEARCH_SINGLES_ONLY) return SOP_ERR_RANGE;
   Plan P;
-  if ((rc = build_plan(A, F, k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, &P))) return rc;
+  if ((rc = build_plan(A, F, k_from_result ? 0 : k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, &P))) return rc;
+  P.k_from_result = k_from_result ? 1 : 0;
+  for (int c = 0; c < P.n_classes; ++c) {
+    // the shift of a class is read from a candidate of that class that the earlier call had
+    P.cls[c].k_src = -1;
+    for (int i = 0; i < P.cls[c].n_mem; ++i)
+      if ((load_mask >> P.cls[c].mem[i]) & 1u) { P.cls[c].k_src = P.cls[c].mem[i]; break; }
+    if (k_from_result && P.cls[c].scope != 0 && P.cls[c].k_src < 0) return SOP_ERR_RANGE;
+  }
 
   LayerArgs L;
   L.W = (const uint16_t*)W_dev; L.c = c_dev; L.M = M; L.K = K; L.ldw = ldw; L.nbk = K / SOP_G; L.NB = M * L.nbk;
@@ -880,26 +964,22 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   Partial* partials = (Partial*)(ws + ws_part_off());
 
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
-  bool need_prepass = false;
-  for (int c = 0; c < P.n_classes; ++c) need_prepass |= P.cls[c].auto_k || P.cls[c].scope == 0;
   const int sms = num_sms();
-  {
-    // max|W| is part of the result block, so the prepass always runs; it is a single read of W
-    (void)need_prepass;
+  if (!k_from_result) {
+    // one read of W: block scales' exponent histogram, max|W|, then the shifts (last CTA)
     long long want = (L.NB + 255) / 256;
     const int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
-    prepass_kernel<<<grid, 256, 0, st>>>(L, P, hist, hdr);
+    prepass_kernel<<<grid, 256, 0, st>>>(L, P, F, hist, hdr);
     SOP_CUDA_TRY(cudaGetLastError());
   }
-  kselect_kernel<<<1, 160, 0, st>>>(P, F, hist, hdr, result_dev);
-  SOP_CUDA_TRY(cudaGetLastError());
 
   const size_t smem = sweep_smem_bytes(P);
-  if (smem > 227 * 1024) return SOP_ERR_ALPHABET;
+  constexpr size_t SMEM_MAX = 226 * 1024;   // 227 KB per CTA minus the kernel's few static bytes
+  if (smem > SMEM_MAX) return SOP_ERR_ALPHABET;
   static size_t smem_set = 0;
   if (smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    smem_set = 227 * 1024;
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+    smem_set = SMEM_MAX;
   }
   // persistent grid: one CTA per SM, fewer when the layer is small; at least enough threads for one row
   long long grid = (L.NB + TB - 1) / TB;
@@ -908,11 +988,10 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if (grid < min_grid) grid = min_grid;
   if (grid > MAX_GRID) return SOP_ERR_SHAPE;
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
-  sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev);
+  sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev, signed_table_dev,
+                                            result_dev, prev_result_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
-  finalize_kernel<<<1, FIN_TB, 0, st>>>(L, P, F, (int)grid, partials, pair_table_dev, signed_table_dev, result_dev);
-  SOP_CUDA_TRY(cudaGetLastError());
   return SOP_OK;
 }
 

@@ -101,7 +101,9 @@ class LayerSweep:
         self.pair_table = B.new_pair_table(nF, d)
         self.signed_table = B.new_pair_table(nF, d)
         self.result = B.new_result(d)
-        self.use_sign = 1 if fmt.sign_bits else 0
+        # the packed word carries sign + selector when both fit 16 bits; a 16-bit signed format (E8M7) has no
+        # metabit left, so its pair is packed without the sign (the selector takes the sign's bit)
+        self.use_sign = 1 if fmt.sign_bits and fmt.exp_bits + fmt.man_bits + 2 <= 16 else 0
         self.container = scale_word_container(fmt, bool(self.use_sign), True)
         self.codes = torch.empty(self.NB * 2 * n_bits, dtype=torch.uint8, device=d)
         self.words = torch.empty(B.words_nbytes(self.NB, self.container), dtype=torch.uint8, device=d)
@@ -119,17 +121,19 @@ class LayerSweep:
             B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.rom_table, None, self.rom_result, self.ws_search,
                               block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
                               singles_only=True, stream=stream)
-            n += 4
+            n += 2
             B.sop_dd4_lloyd(W, self.c, self.fmt, self.full_atoms, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
             n += 6 + (self.iters + 1)
             B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
-                              block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask, stream=stream)
+                              block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask,
+                              k_mode=B.K_FROM_RESULT, prev_result=self.rom_result, stream=stream)
         else:
             B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
                               self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
-        n += 4
+            n += 1
+        n += 1
         B.sop_pack(W, self.c, self.fmt, self.full_atoms, self.codes, self.words, search_result=self.result,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
                    counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,

@@ -33,7 +33,7 @@ def run(layer, fmt, rom, fp=(), lloyd_iters=8, pool_percent=50.0, want_blocks=Fa
     full += [I.fp_atom(f) for f in fp]
     r2 = oracle.pair_search(layer.W, c, fmt, full, want_blocks=want_blocks)
     out.update(full=r2, atoms=full)
-    sign = 1 if fmt.sign_bits else 0
+    sign = 1 if fmt.sign_bits and fmt.exp_bits + fmt.man_bits + 2 <= 16 else 0
     ia, ib = (int(r2["best"][3]), int(r2["best"][4])) if sign else (int(r2["best"][0]), int(r2["best"][1]))
     b = container_bits(fmt, bool(sign), True)
     pk = oracle.pack(layer.W, c, fmt, full[ia], int(r2["k"][ia]), full[ib], int(r2["k"][ib]), use_sign=sign,

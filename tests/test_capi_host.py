@@ -46,12 +46,12 @@ FAKE = C.c_void_p(0x10000)     # never dereferenced: every call below fails vali
 
 
 def _search(lib, M=4, K=64, ldw=64, g=16, fmt=None, atoms=None, n=None, k=B.K_AUTO, W=FAKE, ws=FAKE, wsb=1 << 30,
-            dd=None, mask=0, emask=0xFFFFFFFF, lmask=0, flags=0, bc=None):
+            dd=None, mask=0, emask=0xFFFFFFFF, lmask=0, flags=0, bc=None, prev=None):
     fmt = fmt or I.scale_format("UE4M4")
     atoms = atoms if atoms is not None else I.alphabet(["NF4"])
     n = len(atoms) if n is None else n
     return lib.sop_pair_search(W, C.c_longlong(M), C.c_longlong(K), C.c_longlong(ldw), FAKE, g, C.byref(B.make_fmt(fmt)), k,
-                               B.make_atoms(atoms), n, dd, C.c_uint(mask), C.c_uint(emask), C.c_uint(lmask), flags, FAKE, None, FAKE, bc,
+                               B.make_atoms(atoms), n, dd, C.c_uint(mask), C.c_uint(emask), C.c_uint(lmask), flags, prev, FAKE, None, FAKE, bc,
                                bc, ws,
                                C.c_size_t(wsb), None)
 
@@ -87,6 +87,8 @@ def test_pair_search_rejects_bad_arguments(lib):
     atoms2 = I.alphabet(["NF4"])
     assert _search(lib, atoms=atoms2, emask=1, lmask=2) == -1   # loading needs the per-block arrays
     assert _search(lib, flags=2) == -7
+    assert _search(lib, k=B.K_FROM_RESULT) == -1       # shifts from an earlier result need that result
+    assert _search(lib, k=B.K_FROM_RESULT, prev=C.c_void_p(0x20000)) == -7   # ... and a loaded candidate in every class
 
 
 def test_other_entry_points_reject_bad_arguments(lib):

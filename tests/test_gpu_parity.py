@@ -55,12 +55,14 @@ def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0, two_cal
         # first the candidates in the mask (single-candidate reduction only), then the rest with the first ones loaded
         first = two_calls_split
         rest = ((1 << A) - 1) & ~first
-        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
+        res1 = B.new_result(dev())
+        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res1, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
                           block_sse=bs, eval_mask=first, singles_only=True)
         torch.cuda.synchronize()
-        first_pass = dict(pair=B.read_pair_table(pt, A).copy(), **B.read_result(res))
-        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
-                          block_sse=bs, eval_mask=rest, load_mask=first)
+        first_pass = dict(pair=B.read_pair_table(pt, A).copy(), **B.read_result(res1))
+        # the second call takes the shifts and max|W| from the first call's result instead of reading W again
+        B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=B.K_FROM_RESULT, prev_result=res1, dd_lut=dd_lut,
+                          dd_mask=dd_mask, block_cos=bc, block_sse=bs, eval_mask=rest, load_mask=first)
     torch.cuda.synchronize()
     out = dict(pair=B.read_pair_table(pt, A), signed=B.read_pair_table(st, A), block_cos=bc.cpu().numpy(),
                block_sse=bs.cpu().numpy(), res_t=res, Wd=Wd, cd=cd, bc_t=bc, **B.read_result(res))
@@ -181,7 +183,7 @@ def test_sweep_in_two_calls_equals_one_call(B, fmt_name):
     atoms = I.alphabet(["NF4", "SH4", "BOF4"], fp=["E2M3", "E4M3^0"])
     c = oracle.channel_norms(L.X.numpy())
     want = oracle.pair_search(L.W, c, fmt, atoms, want_blocks=True)
-    first = 0b10110011     # NF4, -NF4, BOF4, -BOF4, E4M3^0 first; SH4, -SH4, E2M3 in the second call
+    first = 0b01110011     # NF4, -NF4, BOF4, -BOF4, E2M3 first; SH4, -SH4, E4M3^0 in the second call
     got = gpu_search(B, L.W, c, fmt, atoms, two_calls_split=first)
     assert np.array_equal(got["block_cos"].view(np.uint32), want["block_cos"].view(np.uint32))
     assert np.array_equal(got["block_sse"].view(np.uint32), want["block_sse"].view(np.uint32))
