@@ -88,10 +88,16 @@ def _check(rc: int, where: str):
 
 
 def make_fmt(f) -> ScaleFmt:
+    """A ``ScaleFmt`` struct from a descriptor (a struct is passed through: marshal once, call often)."""
+    if isinstance(f, ScaleFmt):
+        return f
     return ScaleFmt(f.sign_bits, f.exp_bits, f.man_bits, f.bias, f.top_exp_reserved)
 
 
-def make_atoms(atoms: Sequence) -> C.Array:
+def make_atoms(atoms) -> C.Array:
+    """An array of ``AtomStruct`` from a list of descriptors (an array is passed through)."""
+    if isinstance(atoms, C.Array):
+        return atoms
     arr = (AtomStruct * max(1, len(atoms)))()
     for i, a in enumerate(atoms):
         s = arr[i]

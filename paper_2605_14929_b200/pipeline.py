@@ -83,6 +83,9 @@ class LayerSweep:
             self.dd_mask = (1 << len(self.full_atoms)) | (1 << (len(self.full_atoms) + 1))
             self.full_atoms += [dd, dd.negation()]
         self.full_atoms += [I.fp_atom(f) for f in fp]
+        # marshalled once: the calls of run() then cost no Python loops
+        self.atoms_c = B.make_atoms(self.full_atoms)
+        self.fmt_c = B.make_fmt(fmt)
         self.NB = M * (K // 16)
         self.pool_rank = int(math.ceil(self.NB * (100.0 - pool_percent) / 100.0))
         self.pool_rank = max(1, min(self.NB, self.pool_rank))
@@ -118,23 +121,23 @@ class LayerSweep:
         B.sop_channel_norms(X, self.c, self.ws_norm, stream)
         n += 2
         if self.iters > 0:
-            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.rom_table, None, self.rom_result, self.ws_search,
+            B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.rom_table, None, self.rom_result, self.ws_search,
                               block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
                               singles_only=True, stream=stream)
             n += 2
-            B.sop_dd4_lloyd(W, self.c, self.fmt, self.full_atoms, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
+            B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
             n += 6 + (self.iters + 1)
-            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
+            B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
                               block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask,
                               k_mode=B.K_FROM_RESULT, prev_result=self.rom_result, stream=stream)
         else:
-            B.sop_pair_search(W, self.c, self.fmt, self.full_atoms, self.pair_table, self.signed_table, self.result,
+            B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
             n += 1
         n += 1
-        B.sop_pack(W, self.c, self.fmt, self.full_atoms, self.codes, self.words, search_result=self.result,
+        B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, search_result=self.result,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
                    counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
                    block_cos=self.full_cos, stream=stream)
