@@ -11,14 +11,19 @@
 //                         that every lane of the iteration kernel has work.
 //   pool_cache_kernel     the pool elements never change between iterations, only the table does:
 //                         (u, omega) of every pool element is computed once (u = w / scale) and kept
-//                         in one array.
-//   lloyd_stream_kernel   one iteration = one coalesced stream over that array: the cell of u on a
-//                         uniform grid gives the (at most two) candidate entries and the exact
-//                         threshold between them; per-entry int64 fixed-point sums are kept in
-//                         thread-private shared-memory slots (no atomics in the element loop; the
-//                         sums are exactly associative, so any order reproduces a sequential sum bit
-//                         for bit), distortion in FP64.  The CTA that finishes last turns the sums
-//                         into centroids, snaps them to bf16, sorts, and clears the accumulators.
+//                         in one array, in tiles of 4096 elements that are counting-sorted by the
+//                         cell of u on a uniform grid (in shared memory) and stored so that thread t of
+//                         a CTA reads the 16 consecutive sorted elements 16 t .. 16 t + 15 with
+//                         coalesced loads.
+//   lloyd_stream_kernel   one iteration = one coalesced stream over that array: the cell of u gives
+//                         the (at most two) candidate entries and the exact threshold between them.
+//                         A thread's elements come in ascending cells, so its entry rarely changes:
+//                         the int64 fixed-point sums of the current entry stay in registers and are
+//                         parked in a thread-private shared-memory slot when the entry changes (no
+//                         atomics; the sums are exactly associative, so any order reproduces a
+//                         sequential sum bit for bit); distortion in FP64.  The CTA that finishes
+//                         last turns the sums into centroids, snaps them to bf16, sorts, and clears
+//                         the accumulators.
 #include <math.h>
 #include <string.h>
 
@@ -32,6 +37,8 @@ constexpr int SORT_CHALF = 320;                 // lookup grid on u: cell width 
 constexpr int SORT_ROWS = 2 * SORT_CHALF + 1;   // the first and last row take everything beyond
 constexpr float SORT_INVH = 256.0f;
 constexpr float SORT_MAGIC = 12582912.0f;       // 1.5 * 2^23
+
+struct CellEntry { float thr; unsigned codes; };   // codes: lo | hi << 8; 0xFFFF: more than one threshold in the cell
 
 struct LloydWs {
   // radix select state
@@ -50,6 +57,9 @@ struct LloydWs {
   unsigned list_count;   // blocks appended to the pool list
   int pad;
   long long pool_count;
+  // lookup tables of the current codebook, rebuilt by whoever changes it (set-up, then each update)
+  float tau_tab[SOP_MAX_ENTRIES];
+  CellEntry cellt[SORT_ROWS];
 };
 
 struct LloydArgs {
@@ -61,14 +71,16 @@ struct LloydArgs {
   int k_mode, fmta_index, n_atoms;
   float* omega;               // workspace: K floats, c / max(c)
   unsigned* pool_idx;         // workspace: NB words, indices of the pool blocks
-  uint2* cache;               // workspace: 16 NB pairs (u, omega) as bit patterns, in pool-list order
+  uint2* cache;               // workspace: pairs (u, omega) as bit patterns, tiles of TILE_ELEMS sorted by cell
 };
 
 static size_t lloyd_off_omega() { return (sizeof(LloydWs) + 255) & ~(size_t)255; }
 static size_t lloyd_off_idx(long long K) { return lloyd_off_omega() + (((size_t)K * 4 + 255) & ~(size_t)255); }
 static size_t lloyd_off_cache(long long M, long long K) { return lloyd_off_idx(K) + ((((size_t)M * (size_t)(K / SOP_G)) * 4 + 255) & ~(size_t)255); }
+constexpr int TILE_ELEMS = LTB * SOP_G;   // pool elements per cache tile: one block per thread of a CTA
 static size_t lloyd_ws_bytes(long long M, long long K) {
-  return lloyd_off_cache(M, K) + (size_t)M * (size_t)K * sizeof(uint2);
+  const size_t nb = (size_t)M * (size_t)(K / SOP_G);
+  return lloyd_off_cache(M, K) + ((nb + LTB - 1) / LTB) * TILE_ELEMS * sizeof(uint2);   // whole tiles
 }
 
 __device__ __forceinline__ unsigned cos_key(float x) {
@@ -154,6 +166,35 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
     if (sh[i]) atomicAdd(&ws->hist[PASS][i], sh[i]);
 }
 
+// Whole CTA.  s_lut holds the current table padded to 32 entries.  Exact decision thresholds, then the
+// cell table: cell r covers u * 256 in [k - 1/2, k + 1/2], k = r - 320 (first / last row: everything
+// beyond); its entry holds the one threshold inside (if any) and the two candidate entries.
+__device__ void lloyd_prepare_tables(LloydWs* ws, const float* s_lut, float* s_tau, int ne) {
+  if (threadIdx.x == 0) build_thresholds(s_lut, ne, s_tau);
+  __syncthreads();
+  if (threadIdx.x < SOP_MAX_ENTRIES) ws->tau_tab[threadIdx.x] = s_tau[threadIdx.x];
+  for (int r = threadIdx.x; r < SORT_ROWS; r += blockDim.x) {
+    const float kf = (float)(r - SORT_CHALF);
+    const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, 1.0f / SORT_INVH);
+    const float hi_edge = r == SORT_ROWS - 1 ? INFINITY : __fmul_rn(kf + 0.5f, 1.0f / SORT_INVH);
+    int nbelow = 0, ninside = 0, ndistinct = 0;
+    float prev = 0.0f;
+    for (int j = 0; j < ne - 1; ++j) {
+      const float x = s_tau[j];
+      if (x < lo_edge) ++nbelow;
+      else if (x <= hi_edge) {
+        if (ninside == 0 || x != prev) ++ndistinct;
+        prev = x;
+        ++ninside;
+      }
+    }
+    CellEntry e;
+    e.thr = ninside ? prev : INFINITY;
+    e.codes = ndistinct <= 1 ? ((unsigned)nbelow | ((unsigned)min(nbelow + ninside, ne - 1) << 8)) : 0xFFFFu;
+    ws->cellt[r] = e;
+  }
+}
+
 __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
                                                                LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
   unsigned prefix, cnt;
@@ -205,6 +246,12 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
     ws->done = 0;
     ws->list_count = 0;
   }
+  __shared__ float s_lut[SOP_MAX_ENTRIES], s_tau[SOP_MAX_ENTRIES];
+  __syncthreads();
+  const int ne = *(volatile int*)&ws->n_entries;
+  if (threadIdx.x < SOP_MAX_ENTRIES) s_lut[threadIdx.x] = ((volatile float*)ws->lut)[min((int)threadIdx.x, ne - 1)];
+  __syncthreads();
+  lloyd_prepare_tables(ws, s_lut, s_tau, ne);
 }
 
 // Dense list of the pool blocks.  One counter update per CTA and round: the warps' counts are scanned
@@ -291,25 +338,75 @@ __device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F
   for (int e = 0; e < 16; ++e) u[e] = __fmul_rn((e & 1) ? bf16hi(wb[e >> 1]) : bf16lo(wb[e >> 1]), rcp);
 }
 
+// One tile = the 256 pool blocks (4096 elements) of one CTA pass.  The tile is counting-sorted by
+// cell in shared memory; sorted position p is stored at (p % 16) * 256 + p / 16, so that thread t of
+// the iteration kernel reads positions 16 t .. 16 t + 15 as loads number 0 .. 15 at index i * 256 + t.
+// A tile that the pool does not fill is padded with (u, omega) = (0, 0): such elements add nothing.
 __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, const LloydWs* __restrict__ ws) {
+  __shared__ unsigned hist[SORT_ROWS + 3];
+  __shared__ unsigned warp_tot[LTB / 32];
+  __shared__ uint2 stage[TILE_ELEMS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned count = ws->list_count;
+  const unsigned n_tiles = (count + LTB - 1) / LTB;
   const int k = ws->k;
-  for (unsigned i = blockIdx.x * LTB + threadIdx.x; i < count; i += gridDim.x * LTB) {
-    float u[16];
-    unsigned j;
-    pool_block_u(a, F, k, a.pool_idx[i], u, j);
-    const float4* op = reinterpret_cast<const float4*>(a.omega + (size_t)j * SOP_G);
-    uint4* dst = reinterpret_cast<uint4*>(a.cache + (size_t)i * 16);
+  for (unsigned tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    for (int i = tid; i < SORT_ROWS + 3; i += LTB) hist[i] = 0;
+    __syncthreads();
+    const unsigned i = tile * LTB + tid;
+    float u[16], om[16];
+    if (i < count) {
+      unsigned j;
+      pool_block_u(a, F, k, a.pool_idx[i], u, j);
+      const float4* op = reinterpret_cast<const float4*>(a.omega + (size_t)j * SOP_G);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float4 o = __ldg(op + q);
-      dst[2 * q] = make_uint4(__float_as_uint(u[4 * q]), __float_as_uint(o.x), __float_as_uint(u[4 * q + 1]), __float_as_uint(o.y));
-      dst[2 * q + 1] = make_uint4(__float_as_uint(u[4 * q + 2]), __float_as_uint(o.z), __float_as_uint(u[4 * q + 3]), __float_as_uint(o.w));
+      for (int q = 0; q < 4; ++q) {
+        const float4 o = __ldg(op + q);
+        om[4 * q] = o.x; om[4 * q + 1] = o.y; om[4 * q + 2] = o.z; om[4 * q + 3] = o.w;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) { u[e] = 0.0f; om[e] = 0.0f; }
     }
+    unsigned where[16];   // cell << 16 | arrival number inside the cell
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const unsigned c = (unsigned)sort_cell(u[e]);
+      where[e] = (c << 16) | atomicAdd(&hist[c], 1u);
+    }
+    __syncthreads();
+    // exclusive scan of the 641 counts: three bins per thread
+    {
+      const int b0 = 3 * tid;
+      unsigned c0 = 0, c1 = 0, c2 = 0;
+      if (b0 < SORT_ROWS) { c0 = hist[b0]; c1 = hist[b0 + 1]; c2 = hist[b0 + 2]; }
+      const unsigned local = c0 + c1 + c2;
+      unsigned incl = local;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (lane == 31) warp_tot[warp] = incl;
+      __syncthreads();
+      unsigned base = 0;
+      for (int w = 0; w < warp; ++w) base += warp_tot[w];
+      const unsigned excl = base + incl - local;
+      if (b0 < SORT_ROWS) { hist[b0] = excl; hist[b0 + 1] = excl + c0; hist[b0 + 2] = excl + c0 + c1; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const unsigned p = hist[where[e] >> 16] + (where[e] & 0xFFFFu);
+      stage[(p & 15u) * LTB + (p >> 4)] = make_uint2(__float_as_uint(u[e]), __float_as_uint(om[e]));
+    }
+    __syncthreads();
+    uint4* dst = reinterpret_cast<uint4*>(a.cache + (size_t)tile * TILE_ELEMS);
+    const uint4* src = reinterpret_cast<const uint4*>(stage);
+#pragma unroll
+    for (int q = 0; q < TILE_ELEMS / 2 / LTB; ++q) dst[q * LTB + tid] = src[q * LTB + tid];
+    __syncthreads();
   }
 }
-
-struct CellEntry { float thr; unsigned codes; };   // codes: lo | hi << 8; 0xFFFF: more than one threshold in the cell
 
 __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exact scaling, one rounding to an integer
   const float s = __fmul_rn(v, 16777216.0f);
@@ -326,70 +423,56 @@ __global__ void __launch_bounds__(LTB) lloyd_stream_kernel(LloydArgs a, LloydWs*
   __shared__ int s_is_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int ne = ws->n_entries;
-  if (tid < 32) lutv[tid] = ws->lut[min(tid, ne - 1)];
+  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; }
+  for (int r = tid; r < SORT_ROWS; r += LTB) cellt[r] = ws->cellt[r];
   if (!last)
     for (int i = tid; i < ne * LTB; i += LTB) acc[i] = make_ulonglong2(0ull, 0ull);
   __syncthreads();
-  if (tid == 0) build_thresholds(lutv, ne, tau);
-  __syncthreads();
-  // cell r covers u * 256 in [k - 1/2, k + 1/2], k = r - 320 (first / last row: everything beyond)
-  for (int r = tid; r < SORT_ROWS; r += LTB) {
-    const float kf = (float)(r - SORT_CHALF);
-    const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, 1.0f / SORT_INVH);
-    const float hi_edge = r == SORT_ROWS - 1 ? INFINITY : __fmul_rn(kf + 0.5f, 1.0f / SORT_INVH);
-    int nbelow = 0, ninside = 0, ndistinct = 0;
-    float prev = 0.0f;
-    for (int j = 0; j < ne - 1; ++j) {
-      const float x = tau[j];
-      if (x < lo_edge) ++nbelow;
-      else if (x <= hi_edge) {
-        if (ninside == 0 || x != prev) ++ndistinct;
-        prev = x;
-        ++ninside;
-      }
-    }
-    CellEntry e;
-    e.thr = ninside ? prev : INFINITY;
-    e.codes = ndistinct <= 1 ? ((unsigned)nbelow | ((unsigned)min(nbelow + ninside, ne - 1) << 8)) : 0xFFFFu;
-    cellt[r] = e;
-  }
-  __syncthreads();
 
-  const unsigned total4 = ws->list_count * 4u;                 // the cache as groups of four elements (two 16-byte loads)
+  const unsigned n_tiles = (ws->list_count + LTB - 1) / LTB;
   ulonglong2* mine = acc + tid;
   double D = 0.0;
-  const uint4* src = reinterpret_cast<const uint4*>(a.cache);
-  const unsigned gstride = gridDim.x * LTB;
-  unsigned g = blockIdx.x * LTB + tid;
-  uint4 n0 = make_uint4(0u, 0u, 0u, 0u), n1 = n0;
-  if (g < total4) { n0 = __ldg(src + 2 * (size_t)g); n1 = __ldg(src + 2 * (size_t)g + 1); }
-  for (; g < total4; g += gstride) {
-    const uint4 p0 = n0, p1 = n1;
-    if (g + gstride < total4) {        // the next group's loads are in flight while this one is processed
-      n0 = __ldg(src + 2 * (size_t)(g + gstride));
-      n1 = __ldg(src + 2 * (size_t)(g + gstride) + 1);
-    }
-    const float uu[4] = {__uint_as_float(p0.x), __uint_as_float(p0.z), __uint_as_float(p1.x), __uint_as_float(p1.z)};
-    const float oo[4] = {__uint_as_float(p0.y), __uint_as_float(p0.w), __uint_as_float(p1.y), __uint_as_float(p1.w)};
-    float dq = 0.0f;   // four positive fp32 terms, then FP64
+  int cur = 0;                         // the entry whose sums are in registers
+  float cur_q = lutv[0];
+  unsigned long long n = 0, sacc = 0;
+  for (unsigned tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint2* src = a.cache + (size_t)tile * TILE_ELEMS + tid;
+    uint2 v[16];
 #pragma unroll
-    for (int e4 = 0; e4 < 4; ++e4) {
-      const float u = uu[e4], om = oo[e4];
-      const CellEntry e = cellt[sort_cell(u)];
-      int code;
-      if (e.codes == 0xFFFFu) code = count_below(tau, u);
-      else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
-      const float d = __fsub_rn(u, lutv[code]);
-      dq = __fmaf_rn(__fmul_rn(om, d), d, dq);
-      if (!last) {
-        const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
-        ulonglong2 t = mine[code * LTB];
-        t.x += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
-        t.y += (unsigned long long)fix24(ou);
-        mine[code * LTB] = t;
+    for (int i = 0; i < 16; ++i) v[i] = __ldg(src + i * LTB);
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      float dq = 0.0f;   // four positive fp32 terms, then FP64
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const float u = __uint_as_float(v[4 * h + r].x), om = __uint_as_float(v[4 * h + r].y);
+        const CellEntry e = cellt[sort_cell(u)];
+        int code;
+        if (e.codes == 0xFFFFu) code = count_below(tau, u);
+        else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
+        if (code != cur) {
+          if (!last) {
+            ulonglong2 t = mine[cur * LTB];
+            t.x += n; t.y += sacc;
+            mine[cur * LTB] = t;
+          }
+          cur = code; cur_q = lutv[code]; n = 0; sacc = 0;
+        }
+        const float d = __fsub_rn(u, cur_q);
+        dq = __fmaf_rn(__fmul_rn(om, d), d, dq);
+        if (!last) {
+          const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
+          n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
+          sacc += (unsigned long long)fix24(ou);
+        }
       }
+      D += (double)dq;
     }
-    D += (double)dq;
+  }
+  if (!last) {
+    ulonglong2 t = mine[cur * LTB];
+    t.x += n; t.y += sacc;
+    mine[cur * LTB] = t;
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
   if (lane == 0) sD[warp] = D;
@@ -415,9 +498,17 @@ __global__ void __launch_bounds__(LTB) lloyd_stream_kernel(LloydArgs a, LloydWs*
   __syncthreads();
   if (tid == 0) s_is_last = atomicAdd(&ws->done, 1u) == gridDim.x - 1 ? 1 : 0;
   __syncthreads();
-  if (s_is_last && tid == 0) {
-    __threadfence();
-    lloyd_update(ws, distortion, it, last, out_lut);
+  if (s_is_last) {
+    if (tid == 0) {
+      __threadfence();
+      lloyd_update(ws, distortion, it, last, out_lut);
+    }
+    __syncthreads();
+    if (!last) {                      // the next iteration's lookup tables
+      if (tid < 32) lutv[tid] = ((volatile float*)ws->lut)[min(tid, ne - 1)];
+      __syncthreads();
+      lloyd_prepare_tables(ws, lutv, tau, ne);
+    }
   }
 }
 
@@ -485,8 +576,8 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
 
   // (u, omega) of every pool element, once
   {
-    long long cg = (NB + LTB - 1) / LTB;      // one pool block per thread: the kernel is bound by memory latency
-    if (cg > (long long)sms * 16) cg = (long long)sms * 16;
+    long long cg = (NB + LTB - 1) / LTB;      // one tile per CTA pass
+    if (cg > (long long)sms * 6) cg = (long long)sms * 6;
     pool_cache_kernel<<<(int)cg, LTB, 0, st>>>(a, F, ws);
   }
   SOP_CUDA_TRY(cudaGetLastError());
@@ -500,7 +591,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     smem_set = 128 * 1024;
   }
   const int per_sm = (int)((220 * 1024) / (smem + 8 * 1024));
-  long long grid = (NB * 4 + LTB - 1) / LTB;
+  long long grid = (NB + LTB - 1) / LTB;               // at most one CTA per cache tile
   if (grid > (long long)sms * per_sm) grid = (long long)sms * per_sm;
   if (grid < 1) grid = 1;
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
