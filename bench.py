@@ -47,6 +47,9 @@ def sweep_ops_per_element(n_lut: int, n_bits: int, n_fp: int, n_loaded: int, n_s
 
 LLOYD_BYTES_PER_POOL_ELEMENT = 8.0     # one (u, omega) pair read per pool element and iteration
 LLOYD_OPS_PER_POOL_ELEMENT = 20.0      # cell index 4, entry select 3, distortion 3, fixed-point sums 10
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of these kernels on this
+# workload (cold cache; see the summaries under profiles/); average over the launches of one step
+NCU_TRAFFIC_BYTES = dict(sweep_kernel=(33.7e6 + 27.1e6 + 117.6e6 + 9.6e6) / 2, lloyd_stream_kernel=(8 * 68.0e6 + 67.7e6) / 9)
 
 
 class ClockSampler:
@@ -262,7 +265,8 @@ def run_gpu(args) -> None:
         sweep_t = (kavg["sweep1"] + kavg["sweep2"]) * 1e-3
         sweep_ach = (ops1 + ops2) * E / sweep_t / 1e12
         sweep_roof = dict(kernel="sweep_kernel", launches_per_step=2, bound="alu", achieved=sweep_ach, peak=alu_peak,
-                          unit="T thread-instr/s", frac=sweep_ach / alu_peak, traffic=None,
+                          unit="T thread-instr/s", frac=sweep_ach / alu_peak,
+                          traffic=NCU_TRAFFIC_BYTES["sweep_kernel"] if (M, K) == (4096, 4096) else None,
                           peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz (clocks.max.sm, {of})",
                           ops_per_element=dict(fixed_candidates_singles=ops1, dd_columns_all_pairs=ops2),
                           avg_launch_ms=sweep_t * 1e3 / 2,
@@ -275,7 +279,8 @@ def run_gpu(args) -> None:
         lloyd_t = kavg["lloyd"] * 1e-3
         lloyd_ach = LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e9
         lloyd_roof = dict(kernel="lloyd_stream_kernel", launches_per_step=n_it, bound="hbm", achieved=lloyd_ach, peak=hbm_peak,
-                          unit="GB/s", frac=lloyd_ach / hbm_peak, traffic=None, of=of, avg_launch_ms=lloyd_t * 1e3 / n_it,
+                          unit="GB/s", frac=lloyd_ach / hbm_peak,
+                          traffic=NCU_TRAFFIC_BYTES["lloyd_stream_kernel"] if (M, K) == (4096, 4096) else None, of=of, avg_launch_ms=lloyd_t * 1e3 / n_it,
                           bytes_per_launch=LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems,
                           alu=dict(achieved=LLOYD_OPS_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e12, peak=alu_peak,
                                    unit="T thread-instr/s",
