@@ -11,19 +11,21 @@
 //                         that every lane of the iteration kernel has work.
 //   pool_cache_kernel     the pool elements never change between iterations, only the table does:
 //                         (u, omega) of every pool element is computed once (u = w / scale) and kept
-//                         in one array, in tiles of 4096 elements that are counting-sorted by the
-//                         cell of u on a uniform grid (in shared memory) and stored so that thread t of
-//                         a CTA reads the 16 consecutive sorted elements 16 t .. 16 t + 15 with
-//                         coalesced loads.
-//   lloyd_stream_kernel   one iteration = one coalesced stream over that array: the cell of u gives
-//                         the (at most two) candidate entries and the exact threshold between them.
-//                         A thread's elements come in ascending cells, so its entry rarely changes:
-//                         the int64 fixed-point sums of the current entry stay in registers and are
-//                         parked in a thread-private shared-memory slot when the entry changes (no
-//                         atomics; the sums are exactly associative, so any order reproduces a
-//                         sequential sum bit for bit); distortion in FP64.  The CTA that finishes
-//                         last turns the sums into centroids, snaps them to bf16, sorts, and clears
-//                         the accumulators.
+//                         in tiles of 4096 elements, each counting-sorted by the cell of u on a
+//                         uniform grid (641 cells of width 2^-8); the start of every cell inside
+//                         every tile is kept too, and per cell, over the whole pool, the int64
+//                         fixed-point sums of omega and omega u and the FP64 moments
+//                         sum omega, sum omega u, sum omega u^2.
+//   lloyd_split_kernel    one iteration.  A cell that holds no decision threshold of the current
+//                         table lies inside one entry's interval: its elements are accounted for
+//                         by the cell's sums and moments, without touching them.  Only the cells
+//                         that hold a threshold (at most one per threshold) are walked element by
+//                         element, exactly: one warp per tile, one lane per such cell.  Per-entry
+//                         sums are int64 fixed point (exactly associative: the table is the same
+//                         bit for bit as a sequential sum over all elements gives), distortion
+//                         FP64.  The CTA that finishes last adds the untouched cells, turns the
+//                         sums into centroids, snaps them to bf16, sorts, prepares the next
+//                         iteration's tables and clears the accumulators.
 #include <math.h>
 #include <string.h>
 
@@ -60,6 +62,12 @@ struct LloydWs {
   // lookup tables of the current codebook, rebuilt by whoever changes it (set-up, then each update)
   float tau_tab[SOP_MAX_ENTRIES];
   CellEntry cellt[SORT_ROWS];
+  unsigned n_split;                        // cells that hold a threshold of the current table (walked element by element)
+  unsigned short split_cells[SORT_ROWS];
+  // per cell, over the whole pool (filled once by pool_cache_kernel)
+  unsigned long long cellN[SORT_ROWS];     // sum fix(omega)
+  long long cellS[SORT_ROWS];              // sum fix(omega u)
+  double cellA[3][SORT_ROWS];              // sum omega, sum omega u, sum omega u^2
 };
 
 struct LloydArgs {
@@ -72,15 +80,20 @@ struct LloydArgs {
   float* omega;               // workspace: K floats, c / max(c)
   unsigned* pool_idx;         // workspace: NB words, indices of the pool blocks
   uint2* cache;               // workspace: pairs (u, omega) as bit patterns, tiles of TILE_ELEMS sorted by cell
+  unsigned short* tile_start; // workspace: [tiles][SORT_ROWS + 1] first sorted position of every cell in every tile
 };
 
 static size_t lloyd_off_omega() { return (sizeof(LloydWs) + 255) & ~(size_t)255; }
 static size_t lloyd_off_idx(long long K) { return lloyd_off_omega() + (((size_t)K * 4 + 255) & ~(size_t)255); }
 static size_t lloyd_off_cache(long long M, long long K) { return lloyd_off_idx(K) + ((((size_t)M * (size_t)(K / SOP_G)) * 4 + 255) & ~(size_t)255); }
 constexpr int TILE_ELEMS = LTB * SOP_G;   // pool elements per cache tile: one block per thread of a CTA
-static size_t lloyd_ws_bytes(long long M, long long K) {
+static size_t lloyd_off_tiles(long long M, long long K) {
   const size_t nb = (size_t)M * (size_t)(K / SOP_G);
   return lloyd_off_cache(M, K) + ((nb + LTB - 1) / LTB) * TILE_ELEMS * sizeof(uint2);   // whole tiles
+}
+static size_t lloyd_ws_bytes(long long M, long long K) {
+  const size_t nb = (size_t)M * (size_t)(K / SOP_G);
+  return lloyd_off_tiles(M, K) + ((((nb + LTB - 1) / LTB) * (SORT_ROWS + 1) * sizeof(unsigned short) + 255) & ~(size_t)255);
 }
 
 __device__ __forceinline__ unsigned cos_key(float x) {
@@ -170,7 +183,7 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
 // cell table: cell r covers u * 256 in [k - 1/2, k + 1/2], k = r - 320 (first / last row: everything
 // beyond); its entry holds the one threshold inside (if any) and the two candidate entries.
 __device__ void lloyd_prepare_tables(LloydWs* ws, const float* s_lut, float* s_tau, int ne) {
-  if (threadIdx.x == 0) build_thresholds(s_lut, ne, s_tau);
+  if (threadIdx.x == 0) { build_thresholds(s_lut, ne, s_tau); atomicExch(&ws->n_split, 0u); }
   __syncthreads();
   if (threadIdx.x < SOP_MAX_ENTRIES) ws->tau_tab[threadIdx.x] = s_tau[threadIdx.x];
   for (int r = threadIdx.x; r < SORT_ROWS; r += blockDim.x) {
@@ -192,6 +205,7 @@ __device__ void lloyd_prepare_tables(LloydWs* ws, const float* s_lut, float* s_t
     e.thr = ninside ? prev : INFINITY;
     e.codes = ndistinct <= 1 ? ((unsigned)nbelow | ((unsigned)min(nbelow + ninside, ne - 1) << 8)) : 0xFFFFu;
     ws->cellt[r] = e;
+    if (ninside > 0) ws->split_cells[atomicAdd(&ws->n_split, 1u)] = (unsigned short)r;   // order irrelevant
   }
 }
 
@@ -246,6 +260,9 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
     ws->done = 0;
     ws->list_count = 0;
   }
+  for (int r = threadIdx.x; r < SORT_ROWS; r += SETUP_TB) {
+    ws->cellN[r] = 0; ws->cellS[r] = 0; ws->cellA[0][r] = 0.0; ws->cellA[1][r] = 0.0; ws->cellA[2][r] = 0.0;
+  }
   __shared__ float s_lut[SOP_MAX_ENTRIES], s_tau[SOP_MAX_ENTRIES];
   __syncthreads();
   const int ne = *(volatile int*)&ws->n_entries;
@@ -282,38 +299,6 @@ __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __
   }
 }
 
-// replace non-empty entries by their centroids snapped to bf16 (ties to even), sort ascending
-__device__ void lloyd_update(LloydWs* ws, double* __restrict__ distortion, int it, int last, float* __restrict__ out_lut) {
-  volatile LloydWs* v = ws;
-  distortion[it] = v->accD;
-  const int ne = v->n_entries;
-  if (!last) {
-    float t[SOP_MAX_ENTRIES];
-    for (int j = 0; j < ne; ++j) {
-      t[j] = v->lut[j];
-      const unsigned long long n = v->accN[j];
-      if (n) {
-        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn(v->accS[j]), __ull2double_rn(n)));
-        uint32_t b = __float_as_uint(cen);
-        b += 0x7FFFu + ((b >> 16) & 1u);
-        b &= 0xFFFF0000u;                      // nearest bf16, ties to even
-        t[j] = __uint_as_float(b);
-      }
-    }
-    for (int i = 1; i < ne; ++i) {             // insertion sort, ascending
-      const float x = t[i];
-      int p = i - 1;
-      while (p >= 0 && t[p] > x) { t[p + 1] = t[p]; --p; }
-      t[p + 1] = x;
-    }
-    for (int j = 0; j < ne; ++j) v->lut[j] = t[j];
-  } else {
-    for (int j = 0; j < SOP_MAX_ENTRIES; ++j) out_lut[j] = j < ne ? v->lut[j] : 0.0f;
-  }
-  for (int j = 0; j < SOP_MAX_ENTRIES; ++j) { v->accN[j] = 0; v->accS[j] = 0; }
-  v->accD = 0.0;
-  v->done = 0;
-}
 
 __device__ __forceinline__ int sort_cell(float u) {
   const float t = fminf(fmaxf(__fmaf_rn(u, SORT_INVH, SORT_MAGIC + (float)SORT_CHALF), SORT_MAGIC), SORT_MAGIC + (float)(2 * SORT_CHALF));
@@ -342,11 +327,19 @@ __device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F
 // cell in shared memory; sorted position p is stored at (p % 16) * 256 + p / 16, so that thread t of
 // the iteration kernel reads positions 16 t .. 16 t + 15 as loads number 0 .. 15 at index i * 256 + t.
 // A tile that the pool does not fill is padded with (u, omega) = (0, 0): such elements add nothing.
-__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, const LloydWs* __restrict__ ws) {
+__device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exact scaling, one rounding to an integer
+  const float s = __fmul_rn(v, 16777216.0f);
+  return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
+}
+
+__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws) {
   __shared__ unsigned hist[SORT_ROWS + 3];
   __shared__ unsigned warp_tot[LTB / 32];
-  __shared__ uint2 stage[TILE_ELEMS];
+  extern __shared__ __align__(16) uint2 stage[];                  // TILE_ELEMS pairs (dynamic: the kernel needs 60 KB in all)
+  __shared__ unsigned long long cN[SORT_ROWS], cS[SORT_ROWS];     // this CTA's share of the per-cell sums
+  __shared__ double cA[3][SORT_ROWS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int r = tid; r < SORT_ROWS; r += LTB) { cN[r] = 0; cS[r] = 0; cA[0][r] = 0.0; cA[1][r] = 0.0; cA[2][r] = 0.0; }
   const unsigned count = ws->list_count;
   const unsigned n_tiles = (count + LTB - 1) / LTB;
   const int k = ws->k;
@@ -404,108 +397,207 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
     const uint4* src = reinterpret_cast<const uint4*>(stage);
 #pragma unroll
     for (int q = 0; q < TILE_ELEMS / 2 / LTB; ++q) dst[q * LTB + tid] = src[q * LTB + tid];
+    unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
+    for (int r = tid; r <= SORT_ROWS; r += LTB) ts[r] = (unsigned short)hist[r];      // hist[SORT_ROWS] = 4096: the end of the last cell
+    // per-cell sums: thread t owns the sorted positions 16 t .. 16 t + 15 (ascending cells), keeps the
+    // current cell's sums in registers and adds them to the CTA's arrays when the cell changes
+    {
+      int cur = -1;
+      unsigned long long n = 0, sv = 0;
+      double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+#pragma unroll 4
+      for (int i2 = 0; i2 < 16; ++i2) {
+        const uint2 v = stage[i2 * LTB + tid];
+        const float u = __uint_as_float(v.x), om = __uint_as_float(v.y);
+        const int c = sort_cell(u);
+        if (c != cur) {
+          if (cur >= 0) { atomicAdd(&cN[cur], n); atomicAdd(&cS[cur], sv); atomicAdd(&cA[0][cur], a0); atomicAdd(&cA[1][cur], a1); atomicAdd(&cA[2][cur], a2); }
+          cur = c; n = 0; sv = 0; a0 = a1 = a2 = 0.0;
+        }
+        const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
+        n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
+        sv += (unsigned long long)fix24(ou);
+        const double dou = (double)om * (double)u;
+        a0 += (double)om; a1 += dou; a2 += dou * (double)u;
+      }
+      atomicAdd(&cN[cur], n); atomicAdd(&cS[cur], sv); atomicAdd(&cA[0][cur], a0); atomicAdd(&cA[1][cur], a1); atomicAdd(&cA[2][cur], a2);
+    }
     __syncthreads();
   }
+  for (int r = tid; r < SORT_ROWS; r += LTB) {
+    if (cN[r]) atomicAdd(&ws->cellN[r], cN[r]);
+    if (cS[r]) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellS[r]), cS[r]);
+    if (cA[0][r] != 0.0) { atomicAdd(&ws->cellA[0][r], cA[0][r]); atomicAdd(&ws->cellA[1][r], cA[1][r]); atomicAdd(&ws->cellA[2][r], cA[2][r]); }
+  }
 }
 
-__device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exact scaling, one rounding to an integer
-  const float s = __fmul_rn(v, 16777216.0f);
-  return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
-}
+// One warp per tile.  The elements of the tile that lie in cells holding a threshold (sorted positions
+// [start[c], start[c + 1]) for every such cell c) are dealt to the 32 lanes round robin, four loads
+// in flight per lane: entry lo or hi by the exact threshold.  Sums go to the CTA's per-entry
+// accumulators with shared-memory atomics (a few hundred elements per tile).
+constexpr int MAX_SPLIT = 64;   // cells with a threshold handled per pass (a table has at most 31 thresholds)
 
-__global__ void __launch_bounds__(LTB) lloyd_stream_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                           int it, int last, float* __restrict__ out_lut) {
-  extern __shared__ __align__(16) unsigned char lsm[];
-  ulonglong2* acc = reinterpret_cast<ulonglong2*>(lsm);    // [n_entries][LTB]: (sum fix(omega), sum fix(omega u))
+__global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                          int it, int last, float* __restrict__ out_lut) {
   __shared__ float lutv[32], tau[32];
-  __shared__ CellEntry cellt[SORT_ROWS];
-  __shared__ double sD[LTB / 32];
+  __shared__ unsigned long long sN[SOP_MAX_ENTRIES], sS[SOP_MAX_ENTRIES];
+  __shared__ double sD;
   __shared__ int s_is_last;
+  __shared__ CellEntry s_entry[MAX_SPLIT];
+  __shared__ unsigned short s_cell[MAX_SPLIT];
+  __shared__ unsigned short s_off[LTB / 32][MAX_SPLIT + 1];   // per warp: first item of every split cell in the tile
+  __shared__ unsigned short s_p0[LTB / 32][MAX_SPLIT];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int ne = ws->n_entries;
-  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; }
-  for (int r = tid; r < SORT_ROWS; r += LTB) cellt[r] = ws->cellt[r];
-  if (!last)
-    for (int i = tid; i < ne * LTB; i += LTB) acc[i] = make_ulonglong2(0ull, 0ull);
-  __syncthreads();
-
+  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; sN[tid] = 0; sS[tid] = 0; }
+  if (tid == 0) sD = 0.0;
   const unsigned n_tiles = (ws->list_count + LTB - 1) / LTB;
-  ulonglong2* mine = acc + tid;
+  const unsigned n_split_all = ws->n_split;
   double D = 0.0;
-  int cur = 0;                         // the entry whose sums are in registers
-  float cur_q = lutv[0];
-  unsigned long long n = 0, sacc = 0;
-  for (unsigned tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    const uint2* src = a.cache + (size_t)tile * TILE_ELEMS + tid;
-    uint2 v[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __ldg(src + i * LTB);
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      float dq = 0.0f;   // four positive fp32 terms, then FP64
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const float u = __uint_as_float(v[4 * h + r].x), om = __uint_as_float(v[4 * h + r].y);
-        const CellEntry e = cellt[sort_cell(u)];
-        int code;
-        if (e.codes == 0xFFFFu) code = count_below(tau, u);
-        else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
-        if (code != cur) {
-          if (!last) {
-            ulonglong2 t = mine[cur * LTB];
-            t.x += n; t.y += sacc;
-            mine[cur * LTB] = t;
-          }
-          cur = code; cur_q = lutv[code]; n = 0; sacc = 0;
-        }
-        const float d = __fsub_rn(u, cur_q);
-        dq = __fmaf_rn(__fmul_rn(om, d), d, dq);
-        if (!last) {
-          const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
-          n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
-          sacc += (unsigned long long)fix24(ou);
-        }
+  __syncthreads();
+  {
+    // every cell without a threshold through its sums and moments, one thread of the grid per cell:
+    // sum omega (u - q)^2 = A2 - 2 q A1 + q^2 A0 for the cell's entry value q
+    for (int r = blockIdx.x * LTB + tid; r < SORT_ROWS; r += gridDim.x * LTB) {
+      const CellEntry e = ws->cellt[r];
+      const unsigned long long cn = ws->cellN[r];
+      const long long cs = ws->cellS[r];
+      const double a0 = ws->cellA[0][r], a1 = ws->cellA[1][r], a2 = ws->cellA[2][r];
+      if (e.codes != 0xFFFFu && e.thr == INFINITY && (cn || a0 != 0.0)) {
+        const int j = (int)(e.codes & 0xFFu);
+        if (!last) { atomicAdd(&sN[j], cn); atomicAdd(&sS[j], (unsigned long long)cs); }
+        const double q = (double)lutv[j];
+        D += a2 - 2.0 * q * a1 + q * q * a0;
       }
-      D += (double)dq;
     }
   }
-  if (!last) {
-    ulonglong2 t = mine[cur * LTB];
-    t.x += n; t.y += sacc;
-    mine[cur * LTB] = t;
+  for (unsigned sbase = 0; sbase < n_split_all; sbase += MAX_SPLIT) {
+    const int n_split = (int)min((unsigned)MAX_SPLIT, n_split_all - sbase);
+    __syncthreads();
+    if (tid < n_split) { const int c = ws->split_cells[sbase + tid]; s_cell[tid] = (unsigned short)c; s_entry[tid] = ws->cellt[c]; }
+    __syncthreads();
+    for (unsigned tile = blockIdx.x * (LTB / 32) + warp; tile < n_tiles; tile += gridDim.x * (LTB / 32)) {
+      const unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
+      const uint2* src = a.cache + (size_t)tile * TILE_ELEMS;
+      // segment lengths -> exclusive offsets (two cells per lane)
+      unsigned len0 = 0, len1 = 0, q0 = 0, q1 = 0;
+      if (lane < n_split) { const int c = s_cell[lane]; q0 = ts[c]; len0 = ts[c + 1] - q0; }
+      if (lane + 32 < n_split) { const int c = s_cell[lane + 32]; q1 = ts[c]; len1 = ts[c + 1] - q1; }
+      unsigned inc0 = len0, inc1 = len1;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned v0 = __shfl_up_sync(0xFFFFFFFFu, inc0, o), v1 = __shfl_up_sync(0xFFFFFFFFu, inc1, o);
+        if (lane >= o) { inc0 += v0; inc1 += v1; }
+      }
+      const unsigned tot0 = __shfl_sync(0xFFFFFFFFu, inc0, 31), total = tot0 + __shfl_sync(0xFFFFFFFFu, inc1, 31);
+      __syncwarp();
+      s_off[warp][lane] = (unsigned short)(inc0 - len0); s_p0[warp][lane] = (unsigned short)q0;
+      s_off[warp][lane + 32] = (unsigned short)(tot0 + inc1 - len1); s_p0[warp][lane + 32] = (unsigned short)q1;
+      if (lane == 0) s_off[warp][MAX_SPLIT] = (unsigned short)total;
+      __syncwarp();
+      // every lane takes a contiguous share of the items: its entry changes a few times at most, so the
+      // sums of the current entry stay in registers and reach the CTA's accumulators on a change
+      const unsigned share = (total + 31u) / 32u;
+      const unsigned i_lo = min(total, lane * share), i_hi = min(total, i_lo + share);
+      int cur = -1;
+      unsigned long long n = 0, sv = 0;
+      for (unsigned base = i_lo; base < i_hi; base += 4) {
+        uint2 v[4];
+        int cell_l[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const unsigned item = base + k;
+          cell_l[k] = -1;
+          v[k] = make_uint2(0u, 0u);
+          if (item < i_hi) {
+            int l = 0;                       // the split cell whose item range holds `item`: binary search over <= 64 offsets
+#pragma unroll
+            for (int step = 32; step >= 1; step >>= 1)
+              if (l + step < n_split && s_off[warp][l + step] <= item) l += step;
+            cell_l[k] = l;
+            const unsigned pp = s_p0[warp][l] + (item - s_off[warp][l]);
+            v[k] = __ldg(src + (pp & 15u) * LTB + (pp >> 4));
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (cell_l[k] < 0) continue;
+          const CellEntry e = s_entry[cell_l[k]];
+          const float u = __uint_as_float(v[k].x), om = __uint_as_float(v[k].y);
+          int code;
+          if (e.codes == 0xFFFFu) code = count_below(tau, u);   // several thresholds in one cell: the general search
+          else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
+          const float d = __fsub_rn(u, lutv[code]);
+          D += (double)__fmul_rn(__fmul_rn(om, d), d);
+          if (!last) {
+            if (code != cur) {
+              if (cur >= 0) { atomicAdd(&sN[cur], n); atomicAdd(&sS[cur], sv); }
+              cur = code; n = 0; sv = 0;
+            }
+            const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
+            n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
+            sv += (unsigned long long)fix24(ou);
+          }
+        }
+      }
+      if (cur >= 0) { atomicAdd(&sN[cur], n); atomicAdd(&sS[cur], sv); }
+    }
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
-  if (lane == 0) sD[warp] = D;
+  if (lane == 0 && D != 0.0) atomicAdd(&sD, D);
   __syncthreads();
-  if (!last) {
-    for (int j = warp; j < ne; j += LTB / 32) {
-      unsigned long long n = 0, sv = 0;
-      for (int q = lane; q < LTB; q += 32) { const ulonglong2 t = acc[j * LTB + q]; n += t.x; sv += t.y; }
-      for (int o = 16; o; o >>= 1) { n += __shfl_xor_sync(0xFFFFFFFFu, n, o); sv += __shfl_xor_sync(0xFFFFFFFFu, sv, o); }
-      if (lane == 0) {
-        if (n) atomicAdd(&ws->accN[j], n);
-        if (sv) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[j]), sv);
-      }
-    }
+  if (tid < ne && !last) {
+    if (sN[tid]) atomicAdd(&ws->accN[tid], sN[tid]);
+    if (sS[tid]) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[tid]), sS[tid]);
   }
-  if (tid == 0) {
-    double t = 0.0;
-    for (int w = 0; w < LTB / 32; ++w) t += sD[w];
-    if (t != 0.0) atomicAdd(&ws->accD, t);
-  }
+  if (tid == 0 && sD != 0.0) atomicAdd(&ws->accD, sD);
   // the CTA that arrives last owns the update; no CTA waits for another
   __threadfence();
   __syncthreads();
   if (tid == 0) s_is_last = atomicAdd(&ws->done, 1u) == gridDim.x - 1 ? 1 : 0;
   __syncthreads();
   if (s_is_last) {
-    if (tid == 0) {
-      __threadfence();
-      lloyd_update(ws, distortion, it, last, out_lut);
+    __threadfence();
+    // totals so far (cells with a threshold), then every other cell through its sums and moments:
+    // sum omega (u - q)^2 = A2 - 2 q A1 + q^2 A0 for the cell's entry value q
+    // every CTA has added its share (cells with a threshold element by element, the others by their sums)
+    if (tid < 32) { sN[tid] = __ldcg(&ws->accN[tid]); sS[tid] = (unsigned long long)__ldcg(&ws->accS[tid]); }
+    if (tid == 0) sD = __ldcg(&ws->accD);
+    __syncthreads();
+    // centroids: one thread per entry; thread 0 sorts and publishes
+    if (!last && tid < ne) {
+      float t = lutv[tid];
+      const unsigned long long n = sN[tid];
+      if (n) {
+        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn((long long)sS[tid]), __ull2double_rn(n)));
+        uint32_t b = __float_as_uint(cen);
+        b += 0x7FFFu + ((b >> 16) & 1u);
+        b &= 0xFFFF0000u;                      // nearest bf16, ties to even
+        t = __uint_as_float(b);
+      }
+      tau[tid] = t;                            // tau is free here: the new, unsorted table
     }
     __syncthreads();
+    if (tid == 0) {
+      distortion[it] = sD;
+      if (!last) {
+        for (int i = 1; i < ne; ++i) {         // insertion sort, ascending
+          const float x = tau[i];
+          int p = i - 1;
+          while (p >= 0 && tau[p] > x) { tau[p + 1] = tau[p]; --p; }
+          tau[p + 1] = x;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < SOP_MAX_ENTRIES) {
+      if (!last) { if (tid < ne) ws->lut[tid] = tau[tid]; }
+      else out_lut[tid] = tid < ne ? lutv[tid] : 0.0f;
+      ws->accN[tid] = 0; ws->accS[tid] = 0;
+    }
+    if (tid == 0) { ws->accD = 0.0; ws->done = 0; }
+    __syncthreads();
     if (!last) {                      // the next iteration's lookup tables
-      if (tid < 32) lutv[tid] = ((volatile float*)ws->lut)[min(tid, ne - 1)];
+      if (tid < 32) lutv[tid] = tau[min(tid, ne - 1)];
       __syncthreads();
       lloyd_prepare_tables(ws, lutv, tau, ne);
     }
@@ -558,6 +650,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   a.omega = (float*)(wsb + lloyd_off_omega());
   a.pool_idx = (unsigned*)(wsb + lloyd_off_idx(K));
   a.cache = (uint2*)(wsb + lloyd_off_cache(M, K));
+  a.tile_start = (unsigned short*)(wsb + lloyd_off_tiles(M, K));
   LloydWs* ws = (LloydWs*)workspace_dev;
   cudaStream_t st = (cudaStream_t)stream;
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(LloydWs), st));
@@ -574,30 +667,26 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   pool_list_kernel<<<(int)sg, LTB, 0, st>>>(a, ws);
   SOP_CUDA_TRY(cudaGetLastError());
 
-  // (u, omega) of every pool element, once
+  // (u, omega) of every pool element, once: sorted tiles, cell starts, per-cell sums and moments
   {
     long long cg = (NB + LTB - 1) / LTB;      // one tile per CTA pass
-    if (cg > (long long)sms * 6) cg = (long long)sms * 6;
-    pool_cache_kernel<<<(int)cg, LTB, 0, st>>>(a, F, ws);
+    if (cg > (long long)sms * 3) cg = (long long)sms * 3;
+    const size_t stage_bytes = (size_t)TILE_ELEMS * sizeof(uint2);
+    static bool attr_set = false;
+    if (!attr_set) {
+      SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
+      attr_set = true;
+    }
+    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws);
+    SOP_CUDA_TRY(cudaGetLastError());
   }
-  SOP_CUDA_TRY(cudaGetLastError());
-  int max_entries = 2;
-  for (int i = 0; i < n_atoms; ++i)
-    if (atoms[i].kind == SOP_KIND_LUT && atoms[i].n_entries > max_entries) max_entries = atoms[i].n_entries;
-  const size_t smem = (size_t)max_entries * LTB * sizeof(ulonglong2);   // 64 KB for 16 entries, 128 KB for 32
-  static size_t smem_set = 0;
-  if (smem > 40 * 1024 && smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(lloyd_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-    smem_set = 128 * 1024;
-  }
-  const int per_sm = (int)((220 * 1024) / (smem + 8 * 1024));
-  long long grid = (NB + LTB - 1) / LTB;               // at most one CTA per cache tile
-  if (grid > (long long)sms * per_sm) grid = (long long)sms * per_sm;
+  long long grid = ((NB + LTB - 1) / LTB + LTB / 32 - 1) / (LTB / 32);   // one warp per cache tile
+  if (grid > (long long)sms * 8) grid = (long long)sms * 8;
   if (grid < 1) grid = 1;
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
   for (int it = 0; it <= iters; ++it) {
     const int last = it == iters;
-    lloyd_stream_kernel<<<(int)grid, LTB, smem, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
+    lloyd_split_kernel<<<(int)grid, LTB, 0, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
   }
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;
   SOP_CUDA_TRY(cudaGetLastError());
