@@ -437,10 +437,25 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
 // accumulators with shared-memory atomics (a few hundred elements per tile).
 constexpr int MAX_SPLIT = 64;   // cells with a threshold handled per pass (a table has at most 31 thresholds)
 
+// A CTA walks at most 2^17 elements per launch (8 warps, a few tiles each), every element adds at most
+// 2^24 to n and 2^32 in magnitude to sv, and there is at most one flush per element.  With 12-bit low
+// limbs every limb sum stays below 2^31: n = 12 bits + the rest, sv = 12 + 12 bits + the signed rest.
+__device__ __forceinline__ void flush_limbs(unsigned* n0, unsigned* n1, unsigned* s0, unsigned* s1, int* s2, int code,
+                                            unsigned long long n, unsigned long long sv) {
+  atomicAdd(&n0[code], (unsigned)(n & 0xFFFull));
+  atomicAdd(&n1[code], (unsigned)(n >> 12));
+  atomicAdd(&s0[code], (unsigned)(sv & 0xFFFull));
+  atomicAdd(&s1[code], (unsigned)((sv >> 12) & 0xFFFull));
+  atomicAdd(&s2[code], (int)((long long)sv >> 24));
+}
+
 __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
                                                           int it, int last, float* __restrict__ out_lut) {
   __shared__ float lutv[32], tau[32];
   __shared__ unsigned long long sN[SOP_MAX_ENTRIES], sS[SOP_MAX_ENTRIES];
+  // flushes of the element walk: native 32-bit atomics on limbs, combined into sN / sS afterwards
+  __shared__ unsigned lN[2][SOP_MAX_ENTRIES], lS0[SOP_MAX_ENTRIES], lS1[SOP_MAX_ENTRIES];
+  __shared__ int lS2[SOP_MAX_ENTRIES];
   __shared__ double sD;
   __shared__ int s_is_last;
   __shared__ CellEntry s_entry[MAX_SPLIT];
@@ -449,7 +464,7 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
   __shared__ unsigned short s_p0[LTB / 32][MAX_SPLIT];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int ne = ws->n_entries;
-  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; sN[tid] = 0; sS[tid] = 0; }
+  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; sN[tid] = 0; sS[tid] = 0; lN[0][tid] = lN[1][tid] = lS0[tid] = lS1[tid] = 0; lS2[tid] = 0; }
   if (tid == 0) sD = 0.0;
   const unsigned n_tiles = (ws->list_count + LTB - 1) / LTB;
   const unsigned n_split_all = ws->n_split;
@@ -530,7 +545,7 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
           D += (double)__fmul_rn(__fmul_rn(om, d), d);
           if (!last) {
             if (code != cur) {
-              if (cur >= 0) { atomicAdd(&sN[cur], n); atomicAdd(&sS[cur], sv); }
+              if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
               cur = code; n = 0; sv = 0;
             }
             const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
@@ -539,13 +554,15 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
           }
         }
       }
-      if (cur >= 0) { atomicAdd(&sN[cur], n); atomicAdd(&sS[cur], sv); }
+      if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
     }
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
   if (lane == 0 && D != 0.0) atomicAdd(&sD, D);
   __syncthreads();
   if (tid < ne && !last) {
+    sN[tid] += (unsigned long long)lN[0][tid] + ((unsigned long long)lN[1][tid] << 12);
+    sS[tid] += (unsigned long long)lS0[tid] + ((unsigned long long)lS1[tid] << 12) + ((unsigned long long)(long long)lS2[tid] << 24);
     if (sN[tid]) atomicAdd(&ws->accN[tid], sN[tid]);
     if (sS[tid]) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->accS[tid]), sS[tid]);
   }
@@ -682,6 +699,11 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   }
   long long grid = ((NB + LTB - 1) / LTB + LTB / 32 - 1) / (LTB / 32);   // one warp per cache tile
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+  {
+    // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
+    const long long tiles = (NB + LTB - 1) / LTB, need = (tiles + 4 * (LTB / 32) - 1) / (4 * (LTB / 32));
+    if (grid < need) grid = need;
+  }
   if (grid < 1) grid = 1;
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
   for (int it = 0; it <= iters; ++it) {
