@@ -43,7 +43,8 @@ struct Plan {
   int k_mode, rows, a_pad;
   unsigned eval_mask, load_mask;   // candidates evaluated here / read from the per-block arrays of an earlier call
   int k_from_result;               // 1: shifts and max|W| come from the result block of an earlier call, no prepass
-  int red_t1, red_g0, red_g1;   // phase-2 thread split of a half CTA: [0, t1) pair slots in g0 groups, [t1, 256) signed slots in g1 groups
+  int n_bases;                               // base atoms (each followed by its negation) of the signed table
+  unsigned char base_atom[SOP_MAX_ATOMS];    // signed-best column n_atoms + b holds the better of base_atom[b] and its negation
   CandDev cand[SOP_MAX_ATOMS];
   ClassDev cls[SOP_MAX_CLASSES];
   unsigned char table_atom[SOP_MAX_TABLES];   // atom whose lut fills the table
@@ -358,7 +359,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   }
   __syncthreads();
   constexpr int HBP = HB + 1;   // row pitch: candidates land in different banks
-  float2* cs = cs_all + (size_t)half * P.n_atoms * HBP;
+  float2* cs = cs_all + (size_t)half * (P.n_atoms + P.n_bases) * HBP;
 
   // thread -> fixed column block j, rows m = r0, r0 + R, ...
   const long long GT = (long long)gridDim.x * TB;
@@ -384,17 +385,13 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       for (int p = 0; p < 2; ++p) B.c[2 * i + p] = make_float2(cc[8 * p + i], cc[8 * p + 4 + i]);
   }
 
-  // phase-2 role of this thread inside its half: warps are homogeneous (two-way slots in threads
-  // [0, t1), four-way signed slots in [t1, 256)), so the two loop bodies never diverge inside a warp
-  const int n_slots = P.n_slots, n0 = P.n_pair_slots, n1 = n_slots - n0;
-  const bool four_way = htid >= P.red_t1;
-  const int rt = four_way ? htid - P.red_t1 : htid;
-  const int rn = four_way ? n1 : n0;
-  const int n_groups = four_way ? P.red_g1 : P.red_g0;
-  const int grp = rn ? rt / rn : 0;
-  const int slot = rn ? (four_way ? n0 : 0) + rt % rn : 0;
-  const bool red_on = rn > 0 && grp < n_groups;
+  // phase-2 role of this thread inside its half: slot = table entry, group = range of the tile's blocks
+  const int n_slots = P.n_slots;
+  const int n_groups = HB / n_slots;
+  const int grp = htid / n_slots, slot = htid - grp * n_slots;
+  const bool red_on = grp < n_groups;
   const SlotDev sd = P.slots[slot];
+  float2* my = cs + htid;                      // this thread's block in the staging buffer: my[a * HBP]
   double acc_gap = 0.0, acc_sse = 0.0;
   int acc_n1 = 0, acc_nneg = 0;
   const int copy_off = (lane & 15) * 8;
@@ -436,7 +433,6 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
         }
       const float nw = fold(nw2[0], nw2[1]);
       const long long blk = m * L.nbk + j;
-      float2* my = cs + htid;
 
       // candidates evaluated by an earlier call: their per-block values go from the arrays straight into
       // the staging buffer (asynchronous 4-byte copies, no registers held) while this call's candidates
@@ -536,80 +532,53 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
     }
     if (P.load_mask) asm volatile("cp.async.wait_all;" ::: "memory");
     half_barrier(half);
-    // ---- phase 2: one slot per thread, blocks grp, grp + n_groups, ... of the half's tile; fp32 sums of
-    //      eight gaps 1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
+    // ---- signed bests: for every base atom the better of the atom and its negation (ties to the atom), as
+    //      one more column of the staging buffer; the sign of the stored error marks a negated winner.  The
+    //      four-way entry (i, -i, j, -j) is then the two-way entry of the columns of i and j, with the same
+    //      tie order ----
+    if (P.n_bases) {
+      for (int bi = 0; bi < P.n_bases; ++bi) {
+        const int a = P.base_atom[bi];
+        const float2 vp = my[a * HBP], vn = my[(a + 1) * HBP];
+        const bool neg = vn.x > vp.x;
+        my[(P.n_atoms + bi) * HBP] = make_float2(neg ? vn.x : vp.x, neg ? -vn.y : vp.y);
+      }
+      half_barrier(half);
+    }
+    // ---- phase 2: one slot per thread, a contiguous range of the half's tile; fp32 sums of eight gaps
+    //      1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
     if (red_on) {
       const int nvi = (int)nv;
       const int len = (nvi + n_groups - 1) / n_groups;     // group g takes blocks [g len, (g + 1) len) of the tile
       const int lo = grp * len, hi = min(nvi, lo + len);
-      if (!four_way) {
-        const float2* pa = cs + sd.i0 * HBP + lo;
-        const float2* pb = cs + sd.i1 * HBP + lo;
-        int b = lo;
-        for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
-          float cg = 0.0f, ce = 0.0f;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float2 va = pa[k], vb = pb[k];
-            const bool mu = vb.x > va.x;
-            const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
-            acc_n1 += mu ? 1 : 0;
-            cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-            ce = __fadd_rn(ce, se_);
-          }
-          acc_gap += (double)cg; acc_sse += (double)ce;
-        }
+      const float2* pa = cs + sd.i0 * HBP + lo;
+      const float2* pb = cs + sd.i1 * HBP + lo;
+      int b = lo;
+      for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
         float cg = 0.0f, ce = 0.0f;
-        for (; b < hi; ++b, ++pa, ++pb) {
-          const float2 va = pa[0], vb = pb[0];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float2 va = pa[k], vb = pb[k];
           const bool mu = vb.x > va.x;
           const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
           acc_n1 += mu ? 1 : 0;
+          acc_nneg += (int)(__float_as_uint(se_) >> 31);       // a negated winner of a signed column (error stored negative)
           cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-          ce = __fadd_rn(ce, se_);
-        }
-        acc_gap += (double)cg; acc_sse += (double)ce;
-      } else {
-        // candidates i0, i0 + 1, i1, i1 + 1 in priority order (i1 == i0: the second pair repeats the first and never wins)
-        const float2* pa = cs + sd.i0 * HBP + lo;
-        const float2* pb = cs + sd.i1 * HBP + lo;
-        int b = lo;
-        for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
-          float cg = 0.0f, ce = 0.0f;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float2 v0 = pa[k], v1 = pa[HBP + k], v2 = pb[k], v3 = pb[HBP + k];
-            const bool p1 = v1.x > v0.x;
-            float sc_ = p1 ? v1.x : v0.x, se_ = p1 ? v1.y : v0.y;
-            int pick = p1 ? 1 : 0;
-            const bool p2 = v2.x > sc_;
-            sc_ = p2 ? v2.x : sc_; se_ = p2 ? v2.y : se_; pick = p2 ? 2 : pick;
-            const bool p3 = v3.x > sc_;
-            sc_ = p3 ? v3.x : sc_; se_ = p3 ? v3.y : se_; pick = p3 ? 3 : pick;
-            acc_n1 += pick >> 1;
-            acc_nneg += pick & 1;
-            cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-            ce = __fadd_rn(ce, se_);
-          }
-          acc_gap += (double)cg; acc_sse += (double)ce;
-        }
-        float cg = 0.0f, ce = 0.0f;
-        for (; b < hi; ++b, ++pa, ++pb) {
-          const float2 v0 = pa[0], v1 = pa[HBP], v2 = pb[0], v3 = pb[HBP];
-          const bool p1 = v1.x > v0.x;
-          float sc_ = p1 ? v1.x : v0.x, se_ = p1 ? v1.y : v0.y;
-          int pick = p1 ? 1 : 0;
-          const bool p2 = v2.x > sc_;
-          sc_ = p2 ? v2.x : sc_; se_ = p2 ? v2.y : se_; pick = p2 ? 2 : pick;
-          const bool p3 = v3.x > sc_;
-          sc_ = p3 ? v3.x : sc_; se_ = p3 ? v3.y : se_; pick = p3 ? 3 : pick;
-          acc_n1 += pick >> 1;
-          acc_nneg += pick & 1;
-          cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-          ce = __fadd_rn(ce, se_);
+          ce = __fadd_rn(ce, fabsf(se_));
         }
         acc_gap += (double)cg; acc_sse += (double)ce;
       }
+      float cg = 0.0f, ce = 0.0f;
+      for (; b < hi; ++b, ++pa, ++pb) {
+        const float2 va = pa[0], vb = pb[0];
+        const bool mu = vb.x > va.x;
+        const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
+        acc_n1 += mu ? 1 : 0;
+        acc_nneg += (int)(__float_as_uint(se_) >> 31);
+        cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
+        ce = __fadd_rn(ce, fabsf(se_));
+      }
+      acc_gap += (double)cg; acc_sse += (double)ce;
     }
     half_barrier(half);
   }
@@ -620,12 +589,10 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   { Partial p; p.gap = acc_gap; p.sse = acc_sse; p.n1 = acc_n1; p.nneg = acc_nneg; sc[tid] = p; }
   __syncthreads();
   if (tid < n_slots) {
-    const bool fw = tid >= n0;
-    const int first = fw ? P.red_t1 + (tid - n0) : tid, stride = fw ? n1 : n0, ng = fw ? P.red_g1 : P.red_g0;
     Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
     for (int h = 0; h < 2; ++h)
-      for (int g = 0; g < ng; ++g) {
-        const Partial q = sc[h * HB + first + g * stride];
+      for (int g = 0; g < n_groups; ++g) {
+        const Partial q = sc[h * HB + g * n_slots + tid];
         t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
       }
     partials[(size_t)blockIdx.x * MAX_SLOTS + tid] = t;
@@ -709,7 +676,7 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
     st.n_sel1 = t.n1;
     const SlotDev sd = P.slots[tid];
     if (sd.type == 0) { st.n_neg = 0; s_pair[sd.i0 * A + sd.i1] = st; }
-    else { st.n_neg = t.nneg; s_sig[sd.i0 * A + sd.i1] = st; }
+    else { st.n_neg = t.nneg; s_sig[P.base_atom[sd.i0 - A] * A + P.base_atom[sd.i1 - A]] = st; }
   }
   __syncthreads();
   for (int i = tid; i < A * A; i += blockDim.x) {
@@ -861,37 +828,27 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mas
       const bool da = (A.dd_mask >> i) & 1u, db = (A.dd_mask >> (i + 1)) & 1u;
       base[i] = (da && db && a.n_entries == b.n_entries) || (!da && !db && same_table(a, b));
     }
+    int col[SOP_MAX_ATOMS];
+    for (int i = 0; i < n; ++i) {
+      col[i] = -1;
+      if (base[i]) { col[i] = n + P->n_bases; P->base_atom[P->n_bases++] = (unsigned char)i; }
+    }
     for (int i = 0; i < n; ++i)
       for (int j = i; j < n; ++j) {
         if (!base[i] || !base[j] || A.atoms[i].n_bits != A.atoms[j].n_bits) continue;
-        P->slots[ns].type = 1; P->slots[ns].i0 = (unsigned char)i; P->slots[ns].i1 = (unsigned char)j; ++ns;
+        P->slots[ns].type = 1; P->slots[ns].i0 = (unsigned char)col[i]; P->slots[ns].i1 = (unsigned char)col[j]; ++ns;
       }
   }
   if (ns > MAX_SLOTS) return SOP_ERR_ALPHABET;
   P->n_slots = ns;
-  {
-    // split the 256 threads of a half CTA between two-way and four-way slots in proportion to their work
-    // (a four-way step costs about twice a two-way step), on a warp boundary
-    const int half_threads = TB / 2, n0 = P->n_pair_slots, n1 = ns - n0;
-    int t1 = 0;
-    if (n1 > 0) {
-      t1 = (int)lround((double)half_threads * (2.0 * n1) / (2.0 * n1 + n0) / 32.0) * 32;
-      const int need1 = (n1 + 31) / 32 * 32;
-      if (t1 < need1) t1 = need1;
-      while (half_threads - t1 < n0 && t1 > need1) t1 -= 32;
-      if (half_threads - t1 < n0) return SOP_ERR_ALPHABET;
-    }
-    P->red_t1 = half_threads - t1;
-    P->red_g0 = n0 ? P->red_t1 / n0 : 0;
-    P->red_g1 = n1 ? t1 / n1 : 0;
-  }
+  if (ns > TB / 2) return SOP_ERR_ALPHABET;
   return SOP_OK;
 }
 
 size_t sweep_smem_bytes(const Plan& P) {
   size_t b = (size_t)P.n_tables * P.rows * 16 * 8;
   b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
-  size_t tile = (size_t)2 * P.n_atoms * (TB / 2 + 1) * sizeof(float2);
+  size_t tile = (size_t)2 * (P.n_atoms + P.n_bases) * (TB / 2 + 1) * sizeof(float2);
   // the closing reduction of the last CTA: two staged tables and one partial per thread
   const size_t red = sizeof(Partial) * (size_t)TB + 2 * sizeof(sop_pair_stat) * SOP_MAX_ATOMS * SOP_MAX_ATOMS;
   b += tile > red ? tile : red;
