@@ -45,11 +45,9 @@ def sweep_ops_per_element(n_lut: int, n_bits: int, n_fp: int, n_loaded: int, n_s
     return 6 + n_lut * (2 * n_bits + 5) + n_fp * 12 + (6 * n_eval + 2 * n_loaded + 2 * n_slots2 + 6 * n_slots4) / 16.0
 
 
-LLOYD_BYTES_PER_POOL_ELEMENT = 8.0     # one (u, omega) pair read per pool element and iteration
-LLOYD_OPS_PER_POOL_ELEMENT = 20.0      # cell index 4, entry select 3, distortion 3, fixed-point sums 10
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of these kernels on this
-# workload (cold cache; see the summaries under profiles/); average over the launches of one step
-NCU_TRAFFIC_BYTES = dict(sweep_kernel=(33.7e6 + 27.1e6 + 117.6e6 + 9.6e6) / 2, lloyd_stream_kernel=(8 * 68.0e6 + 67.7e6) / 9)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of the sweep kernel on this
+# workload (cold cache; see the summary under profiles/); average over the two launches of one step
+NCU_TRAFFIC_BYTES = dict(sweep_kernel=None)
 
 
 class ClockSampler:
@@ -273,19 +271,9 @@ def run_gpu(args) -> None:
                           hbm=dict(achieved=2 * 2.0 * E / sweep_t / 1e9, peak=hbm_peak, unit="GB/s",
                                    frac=2 * 2.0 * E / sweep_t / 1e9 / hbm_peak, of=of,
                                    note="W read once per launch; the kernel is far from the HBM roofline"))
-        # Lloyd iteration kernel: iters + 1 launches per step, each streams 8 bytes per pool element
-        pool_elems = sw.pool_rank * 16
-        n_it = sw.iters + 1
-        lloyd_t = kavg["lloyd"] * 1e-3
-        lloyd_ach = LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e9
-        lloyd_roof = dict(kernel="lloyd_stream_kernel", launches_per_step=n_it, bound="hbm", achieved=lloyd_ach, peak=hbm_peak,
-                          unit="GB/s", frac=lloyd_ach / hbm_peak,
-                          traffic=NCU_TRAFFIC_BYTES["lloyd_stream_kernel"] if (M, K) == (4096, 4096) else None, of=of, avg_launch_ms=lloyd_t * 1e3 / n_it,
-                          bytes_per_launch=LLOYD_BYTES_PER_POOL_ELEMENT * pool_elems,
-                          alu=dict(achieved=LLOYD_OPS_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e12, peak=alu_peak,
-                                   unit="T thread-instr/s",
-                                   frac=LLOYD_OPS_PER_POOL_ELEMENT * pool_elems * n_it / lloyd_t / 1e12 / alu_peak))
-        dominant, other = (sweep_roof, lloyd_roof) if sweep_t >= lloyd_t else (lloyd_roof, sweep_roof)
+        # the Lloyd iterations walk only the pool elements in cells that hold a decision threshold (a few per
+        # cent of the pool), so their launches are bound by launch and dependency latency, not by a roofline
+        dominant = sweep_roof
         cpu_rows = 1024
         cpu_val, cpu_dt = cpu_oracle_time(cpu_rows)
         line = dict(
@@ -296,7 +284,7 @@ def run_gpu(args) -> None:
             kernels_ms=dict(kavg, note="per step, CUDA events recorded by the library around its main kernels; "
                                        "sweep1 = fixed candidates (singles), sweep2 = DD columns (all pairs), "
                                        "lloyd = all iteration launches"),
-            roofline=dominant, roofline_other=other,
+            roofline=dominant,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
                               sample=f"first {cpu_rows} of {M} rows, whole pipeline, {cpu_dt:.1f} s"),
             e2e=dict(value=world * E / (e2e_ms * 1e-3) / 1e9, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,

@@ -27,9 +27,9 @@ struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
 // The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
-template <bool WANT_COS>
-__device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
-                                                const float* __restrict__ lutv, int kind, int neg, float rcp,
+template <bool WANT_COS, int KIND>
+__device__ __forceinline__ void eval_block_kind(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
+                                                const float* __restrict__ lutv, int neg, float rcp,
                                                 float& cos_out, uint32_t (&code4)[4]) {
   float qn[4], qd[4], qw[4];
 #pragma unroll
@@ -42,10 +42,10 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
       const float u = __fmul_rn(w[i], rcp);
       float q;
       uint32_t code;
-      if (kind == SOP_KIND_LUT) {
+      if (KIND == SOP_KIND_LUT) {
         code = (uint32_t)count_below(tau, neg ? -u : u);
         q = neg ? -lutv[code] : lutv[code];
-      } else if (kind == SOP_KIND_FP_E2M3) {
+      } else if (KIND == SOP_KIND_FP_E2M3) {
         q = fp_quantize<SOP_KIND_FP_E2M3>(u);
         code = fp_code<SOP_KIND_FP_E2M3>(q);
       } else {
@@ -65,6 +65,17 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
     code4[h] = packed;
   }
   cos_out = WANT_COS ? block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd)) : 0.0f;
+}
+
+// the quantiser kind is decided once per block, outside the element loops: a kind test inside them lets
+// the compiler hoist the FP-grid arithmetic into the table path
+template <bool WANT_COS>
+__device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
+                                                const float* __restrict__ lutv, int kind, int neg, float rcp,
+                                                float& cos_out, uint32_t (&code4)[4]) {
+  if (kind == SOP_KIND_LUT) eval_block_kind<WANT_COS, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, cos_out, code4);
+  else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<WANT_COS, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, cos_out, code4);
+  else eval_block_kind<WANT_COS, SOP_KIND_FP_E4M3>(w, c, tau, lutv, neg, rcp, cos_out, code4);
 }
 
 // USE_COS: the winner of each block is read off the per-block cosines of a sweep and only it is encoded

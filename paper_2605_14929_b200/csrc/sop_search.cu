@@ -133,38 +133,63 @@ __global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, FmtDe
   }
 }
 
-// One CTA of at least 160 threads.  Reads the global histogram and max|W| through the L2 (they were
-// written by other CTAs' atomics).
+// One CTA of 256 threads.  Reads the global histogram and max|W| through the L2 (they were written by
+// other CTAs' atomics).  Per class: prefix sums of the 320 bins, the count of every shift k in
+// [-64, 64] as a difference of two prefix values, then the largest count with ties to the smallest |k|
+// and then to k > 0 (preference order 0, +1, -1, +2, -2, ...).
 __device__ void kselect_body(const Plan& P, const FmtDev& F, const unsigned* hist, WsHeader* hdr) {
-  __shared__ unsigned long long cnt[129];
-  __shared__ unsigned sh_hist[SOP_HIST_BINS];
+  __shared__ unsigned long long pre[SOP_HIST_BINS + 1];
+  __shared__ unsigned long long red_c[8];
+  __shared__ int red_o[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float wmax = __uint_as_float(__ldcg(&hdr->wmax_bits));
   for (int cl = 0; cl < P.n_classes; ++cl) {
     int kstar = P.k_mode == SOP_K_AUTO ? 0 : P.k_mode;
     if (P.cls[cl].scope == 0) kstar = 0;
     if (P.cls[cl].auto_k) {
-      for (int i = threadIdx.x; i < SOP_HIST_BINS; i += blockDim.x) sh_hist[i] = __ldcg(&hist[cl * SOP_HIST_BINS + i]);
-      __syncthreads();
-      if (threadIdx.x < 129) {
-        const int k = (int)threadIdx.x - 64;
-        unsigned long long c = 0;
-        for (int e = -SOP_HIST_OFF; e < SOP_HIST_BINS - SOP_HIST_OFF; ++e)
-          if (e + k >= F.emin && e + k <= F.emax) c += sh_hist[e + SOP_HIST_OFF];
-        cnt[threadIdx.x] = c;
+      // inclusive prefix of the bins: two bins per thread (320 <= 512), warp scan, warp totals
+      unsigned long long v0 = 0, v1 = 0;
+      if (2 * tid < SOP_HIST_BINS) v0 = __ldcg(&hist[cl * SOP_HIST_BINS + 2 * tid]);
+      if (2 * tid + 1 < SOP_HIST_BINS) v1 = __ldcg(&hist[cl * SOP_HIST_BINS + 2 * tid + 1]);
+      unsigned long long incl = v0 + v1;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        // largest count; ties to the smallest |k|, then to k > 0
-        unsigned long long best = cnt[64];
-        kstar = 0;
-        for (int mag = 1; mag <= 64; ++mag) {
-          if (cnt[64 + mag] > best) { best = cnt[64 + mag]; kstar = mag; }
-          if (cnt[64 - mag] > best) { best = cnt[64 - mag]; kstar = -mag; }
-        }
+      if (lane == 31) red_c[warp] = incl;
+      __syncthreads();
+      unsigned long long base = 0;
+      for (int w = 0; w < warp; ++w) base += red_c[w];
+      if (tid == 0) pre[0] = 0;
+      if (2 * tid < SOP_HIST_BINS) pre[2 * tid + 1] = base + incl - v1;
+      if (2 * tid + 1 < SOP_HIST_BINS) pre[2 * tid + 2] = base + incl;
+      __syncthreads();
+      // shift k = tid - 64 keeps the exponents e with emin <= e + k <= emax; bin of e is e + SOP_HIST_OFF
+      unsigned long long c = 0;
+      int order = 1 << 30;
+      if (tid < 129) {
+        const int k = tid - 64;
+        const int lo = max(F.emin - k + SOP_HIST_OFF, 0), hi = min(F.emax - k + SOP_HIST_OFF, SOP_HIST_BINS - 1);
+        c = hi >= lo ? pre[hi + 1] - pre[lo] : 0ull;
+        order = k == 0 ? 0 : (k > 0 ? 2 * k - 1 : -2 * k);
+      }
+      for (int o = 16; o; o >>= 1) {
+        const unsigned long long oc = __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        const int oo = __shfl_xor_sync(0xFFFFFFFFu, order, o);
+        if (oc > c || (oc == c && oo < order)) { c = oc; order = oo; }
+      }
+      __syncthreads();
+      if (lane == 0) { red_c[warp] = c; red_o[warp] = order; }
+      __syncthreads();
+      if (tid == 0) {
+        for (int w = 1; w < 8; ++w)
+          if (red_c[w] > c || (red_c[w] == c && red_o[w] < order)) { c = red_c[w]; order = red_o[w]; }
+        kstar = order == 0 ? 0 : ((order & 1) ? (order + 1) / 2 : -(order / 2));
       }
       __syncthreads();
     }
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
       hdr->cls_k[cl] = kstar;
       hdr->cls_pot[cl] = P.cls[cl].scope == 0 ? layer_pot_scale(wmax, P.cls[cl].tmax) : 0.0f;
     }
