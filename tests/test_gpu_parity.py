@@ -251,6 +251,30 @@ def test_lloyd_matches_oracle(B, fmt_name, names, iters):
             assert np.allclose(got[1], want[1], rtol=REL, atol=0)
 
 
+def test_lloyd_with_entries_closer_than_the_lookup_grid(B):
+    # an initial table with several entries inside one cell of the iteration's lookup grid (width 2^-8):
+    # those cells take the general search; zero rows and a zero column block are in the pool as well
+    L = I.outlier_channel_layer(21, 160, 512, 64)
+    W = L.W.clone()
+    W[5] = 0
+    W[:, 64:80] = 0
+    L = I.Layer(W, L.X)
+    fmt = I.scale_format("UE4M4")
+    dense = np.sort(np.concatenate([np.linspace(-1, 1, 11), [0.001, 0.0011, 0.00111, 0.0028, 0.3]])).astype(np.float32)
+    dense = I.snap_bf16(dense)
+    atoms = [I.Atom("dense", 4, I.KIND_LUT, 0, 16, 1.0, np.sort(dense)), I.rom_atom("NF4")]
+    c = oracle.channel_norms(L.X.numpy())
+    r = oracle.pair_search(L.W, c, fmt, atoms, want_blocks=True)
+    NB = r["block_cos"].shape[1]
+    bc = torch.from_numpy(r["block_cos"]).to(dev())
+    for rank in (NB, NB // 3):
+        want = oracle.dd_lloyd(L.W, c, fmt, int(r["k"][0]), r["block_cos"][0], rank, atoms[0].lut, 6)
+        got = gpu_lloyd(B, L.W, c, fmt, atoms, bc, rank, 6, int(r["k"][0]), 0)
+        assert np.array_equal(got[0][:16].view(np.uint32), want[0].view(np.uint32))
+        assert got[2] == want[2]
+        assert np.allclose(got[1], want[1], rtol=REL, atol=0)
+
+
 # ------------------------------------------------------------------ pack
 def gpu_pack(B, W, c, fmt, atoms, ia, ib, k, use_sign, b, wsign, block_cos=None):
     M, K = W.shape
