@@ -42,6 +42,17 @@ constexpr float SORT_MAGIC = 12582912.0f;       // 1.5 * 2^23
 
 struct CellEntry { float thr; unsigned codes; };   // codes: lo | hi << 8; 0xFFFF: more than one threshold in the cell
 
+// Everything an iteration reads about the current table, contiguous so that a CTA fetches it with one
+// load per thread: the table (padded with its last entry), the exact decision thresholds (+inf padded)
+// and the lookup cell of every threshold (ascending, like the thresholds).
+struct IterDesc {
+  int n_entries;
+  int pad[3];
+  float lut[SOP_MAX_ENTRIES];
+  float tau[SOP_MAX_ENTRIES];
+  int thr_cell[SOP_MAX_ENTRIES];
+};
+
 struct LloydWs {
   // radix select state
   unsigned hist[3][2048];
@@ -49,21 +60,16 @@ struct LloydWs {
   unsigned long long accN[SOP_MAX_ENTRIES];
   long long accS[SOP_MAX_ENTRIES];
   double accD;
-  float lut[SOP_MAX_ENTRIES];
   float tau;         // pool threshold on the block cosine
   float cmax;
   int k;
   int fmta;
-  int n_entries;
   unsigned done;         // CTAs of the running iteration that have added their sums
   unsigned list_count;   // blocks appended to the pool list
   int pad;
   long long pool_count;
-  // lookup tables of the current codebook, rebuilt by whoever changes it (set-up, then each update)
-  float tau_tab[SOP_MAX_ENTRIES];
-  CellEntry cellt[SORT_ROWS];
-  unsigned n_split;                        // cells that hold a threshold of the current table (walked element by element)
-  unsigned short split_cells[SORT_ROWS];
+  // the current codebook, rewritten by whoever changes it (set-up, then each update)
+  IterDesc desc;
   // per cell, over the whole pool (filled once by pool_cache_kernel)
   unsigned long long cellN[SORT_ROWS];     // sum fix(omega)
   long long cellS[SORT_ROWS];              // sum fix(omega u)
@@ -179,34 +185,27 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
     if (sh[i]) atomicAdd(&ws->hist[PASS][i], sh[i]);
 }
 
-// Whole CTA.  s_lut holds the current table padded to 32 entries.  Exact decision thresholds, then the
-// cell table: cell r covers u * 256 in [k - 1/2, k + 1/2], k = r - 320 (first / last row: everything
-// beyond); its entry holds the one threshold inside (if any) and the two candidate entries.
-__device__ void lloyd_prepare_tables(LloydWs* ws, const float* s_lut, float* s_tau, int ne) {
-  if (threadIdx.x == 0) { build_thresholds(s_lut, ne, s_tau); atomicExch(&ws->n_split, 0u); }
-  __syncthreads();
-  if (threadIdx.x < SOP_MAX_ENTRIES) ws->tau_tab[threadIdx.x] = s_tau[threadIdx.x];
-  for (int r = threadIdx.x; r < SORT_ROWS; r += blockDim.x) {
-    const float kf = (float)(r - SORT_CHALF);
-    const float lo_edge = r == 0 ? -INFINITY : __fmul_rn(kf - 0.5f, 1.0f / SORT_INVH);
-    const float hi_edge = r == SORT_ROWS - 1 ? INFINITY : __fmul_rn(kf + 0.5f, 1.0f / SORT_INVH);
-    int nbelow = 0, ninside = 0, ndistinct = 0;
-    float prev = 0.0f;
-    for (int j = 0; j < ne - 1; ++j) {
-      const float x = s_tau[j];
-      if (x < lo_edge) ++nbelow;
-      else if (x <= hi_edge) {
-        if (ninside == 0 || x != prev) ++ndistinct;
-        prev = x;
-        ++ninside;
-      }
-    }
-    CellEntry e;
-    e.thr = ninside ? prev : INFINITY;
-    e.codes = ndistinct <= 1 ? ((unsigned)nbelow | ((unsigned)min(nbelow + ninside, ne - 1) << 8)) : 0xFFFFu;
-    ws->cellt[r] = e;
-    if (ninside > 0) ws->split_cells[atomicAdd(&ws->n_split, 1u)] = (unsigned short)r;   // order irrelevant
-  }
+__device__ __forceinline__ int sort_cell(float u) {
+  const float t = fminf(fmaxf(__fmaf_rn(u, SORT_INVH, SORT_MAGIC + (float)SORT_CHALF), SORT_MAGIC), SORT_MAGIC + (float)(2 * SORT_CHALF));
+  return (int)(__float_as_uint(t) - __float_as_uint(SORT_MAGIC));
+}
+
+// Threads 0..31 of a CTA; s_lut holds the sorted table padded to 32 entries with its last value.
+// Thread j writes entry j, its decision threshold (the same rule as build_thresholds: the largest
+// fp32 <= the midpoint, a repeated entry takes the threshold above it, +inf from n_entries - 1 on)
+// and the lookup cell of that threshold.  sort_cell is monotone, so an element in a lower cell than a
+// threshold's is below the threshold and one in a higher cell is above it: only the elements of the
+// cells listed here need the comparison itself.
+__device__ void lloyd_publish_desc(LloydWs* ws, const float* s_lut, int ne) {
+  const int j = threadIdx.x;
+  if (j >= SOP_MAX_ENTRIES) return;
+  int jj = j;
+  while (jj < ne - 1 && s_lut[jj] == s_lut[jj + 1]) ++jj;
+  const float t = jj < ne - 1 ? __double2float_rd(0.5 * ((double)s_lut[jj] + (double)s_lut[jj + 1])) : __int_as_float(0x7F800000);
+  ws->desc.lut[j] = s_lut[j];
+  ws->desc.tau[j] = t;
+  ws->desc.thr_cell[j] = j < ne - 1 ? sort_cell(t) : SORT_ROWS;
+  if (j == 0) ws->desc.n_entries = ne;
 }
 
 __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
@@ -216,6 +215,8 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   derive_prefix(ws, a.pool_rank, 3, &prefix, &rank, &below, &cnt);
   __shared__ float red[SETUP_TB / 32];
   __shared__ float s_cmax;
+  __shared__ float s_lut[SOP_MAX_ENTRIES];
+  __shared__ int s_ne;
   float mx = 0.0f;
   for (long long i = threadIdx.x; i < a.K; i += SETUP_TB) mx = fmaxf(mx, __ldg(a.c + i));
   for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
@@ -244,16 +245,13 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
     ws->k = a.k_mode == SOP_K_FROM_RESULT ? res->k[f] : a.k_mode;
     const sop_atom& at = A.atoms[f];
     const int ne = at.n_entries;
-    ws->n_entries = ne;
+    s_ne = ne;
     const bool dd = (A.dd_mask >> f) & 1u;
     for (int j = 0; j < SOP_MAX_ENTRIES; ++j) {
-      float v = 0.0f;
-      if (j < ne) {
-        const int src = at.negated ? ne - 1 - j : j;
-        v = dd ? A.dd_lut[src] : at.lut[src];
-        if (at.negated) v = -v;
-      }
-      ws->lut[j] = v;
+      const int src = at.negated ? ne - 1 - min(j, ne - 1) : min(j, ne - 1);   // padded with the last entry
+      float v = dd ? A.dd_lut[src] : at.lut[src];
+      if (at.negated) v = -v;
+      s_lut[j] = v;
     }
     for (int j = 0; j < SOP_MAX_ENTRIES; ++j) { ws->accN[j] = 0; ws->accS[j] = 0; }
     ws->accD = 0.0;
@@ -263,12 +261,8 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   for (int r = threadIdx.x; r < SORT_ROWS; r += SETUP_TB) {
     ws->cellN[r] = 0; ws->cellS[r] = 0; ws->cellA[0][r] = 0.0; ws->cellA[1][r] = 0.0; ws->cellA[2][r] = 0.0;
   }
-  __shared__ float s_lut[SOP_MAX_ENTRIES], s_tau[SOP_MAX_ENTRIES];
   __syncthreads();
-  const int ne = *(volatile int*)&ws->n_entries;
-  if (threadIdx.x < SOP_MAX_ENTRIES) s_lut[threadIdx.x] = ((volatile float*)ws->lut)[min((int)threadIdx.x, ne - 1)];
-  __syncthreads();
-  lloyd_prepare_tables(ws, s_lut, s_tau, ne);
+  lloyd_publish_desc(ws, s_lut, s_ne);
 }
 
 // Dense list of the pool blocks.  One counter update per CTA and round: the warps' counts are scanned
@@ -299,11 +293,6 @@ __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __
   }
 }
 
-
-__device__ __forceinline__ int sort_cell(float u) {
-  const float t = fminf(fmaxf(__fmaf_rn(u, SORT_INVH, SORT_MAGIC + (float)SORT_CHALF), SORT_MAGIC), SORT_MAGIC + (float)(2 * SORT_CHALF));
-  return (int)(__float_as_uint(t) - __float_as_uint(SORT_MAGIC));
-}
 
 // u of the 16 elements of pool block `blk`
 __device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F, int k, unsigned blk, float (&u)[16], unsigned& j_out) {
@@ -432,10 +421,10 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
 }
 
 // One warp per tile.  The elements of the tile that lie in cells holding a threshold (sorted positions
-// [start[c], start[c + 1]) for every such cell c) are dealt to the 32 lanes round robin, four loads
-// in flight per lane: entry lo or hi by the exact threshold.  Sums go to the CTA's per-entry
+// [start[c], start[c + 1]) for every such cell c) are dealt to the 32 lanes in contiguous shares, four
+// loads in flight per lane: entry lo or hi by the exact threshold.  Sums go to the CTA's per-entry
 // accumulators with shared-memory atomics (a few hundred elements per tile).
-constexpr int MAX_SPLIT = 64;   // cells with a threshold handled per pass (a table has at most 31 thresholds)
+constexpr int MAX_SPLIT = 32;   // a table has at most 31 thresholds, so at most 31 cells hold one
 
 // A CTA walks at most 2^17 elements per launch (8 warps, a few tiles each), every element adds at most
 // 2^24 to n and 2^32 in magnitude to sv, and there is at most one flush per element.  With 12-bit low
@@ -451,111 +440,135 @@ __device__ __forceinline__ void flush_limbs(unsigned* n0, unsigned* n1, unsigned
 
 __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
                                                           int it, int last, float* __restrict__ out_lut) {
-  __shared__ float lutv[32], tau[32];
+  __shared__ __align__(16) IterDesc d;
   __shared__ unsigned long long sN[SOP_MAX_ENTRIES], sS[SOP_MAX_ENTRIES];
   // flushes of the element walk: native 32-bit atomics on limbs, combined into sN / sS afterwards
   __shared__ unsigned lN[2][SOP_MAX_ENTRIES], lS0[SOP_MAX_ENTRIES], lS1[SOP_MAX_ENTRIES];
   __shared__ int lS2[SOP_MAX_ENTRIES];
   __shared__ double sD;
   __shared__ int s_is_last;
+  __shared__ unsigned s_list_count;
   __shared__ CellEntry s_entry[MAX_SPLIT];
   __shared__ unsigned short s_cell[MAX_SPLIT];
   __shared__ unsigned short s_off[LTB / 32][MAX_SPLIT + 1];   // per warp: first item of every split cell in the tile
   __shared__ unsigned short s_p0[LTB / 32][MAX_SPLIT];
+  __shared__ float s_new[SOP_MAX_ENTRIES];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int ne = ws->n_entries;
-  if (tid < 32) { lutv[tid] = ws->lut[min(tid, ne - 1)]; tau[tid] = ws->tau_tab[tid]; sN[tid] = 0; sS[tid] = 0; lN[0][tid] = lN[1][tid] = lS0[tid] = lS1[tid] = 0; lS2[tid] = 0; }
-  if (tid == 0) sD = 0.0;
-  const unsigned n_tiles = (ws->list_count + LTB - 1) / LTB;
-  const unsigned n_split_all = ws->n_split;
-  double D = 0.0;
-  __syncthreads();
   {
-    // every cell without a threshold through its sums and moments, one thread of the grid per cell:
-    // sum omega (u - q)^2 = A2 - 2 q A1 + q^2 A0 for the cell's entry value q
-    for (int r = blockIdx.x * LTB + tid; r < SORT_ROWS; r += gridDim.x * LTB) {
-      const CellEntry e = ws->cellt[r];
+    constexpr int DW = (int)(sizeof(IterDesc) / sizeof(unsigned));
+    static_assert(DW <= LTB, "one descriptor word per thread");
+    if (tid < DW) reinterpret_cast<unsigned*>(&d)[tid] = reinterpret_cast<const unsigned*>(&ws->desc)[tid];
+    if (tid == LTB - 1) s_list_count = ws->list_count;
+    if (tid < 32) { sN[tid] = 0; sS[tid] = 0; lN[0][tid] = lN[1][tid] = lS0[tid] = lS1[tid] = 0; lS2[tid] = 0; }
+    if (tid == 0) sD = 0.0;
+  }
+  __syncthreads();
+  const int ne = d.n_entries;
+  const unsigned n_tiles = (s_list_count + LTB - 1) / LTB;
+  const float* lutv = d.lut;
+  const float* tau = d.tau;
+  // the cells that hold thresholds: thresholds ascend, so those of one cell are neighbours.  Every warp
+  // derives the same list and writes the same values.
+  int n_split;
+  {
+    const bool on = lane < ne - 1;
+    const int c = d.thr_cell[lane];
+    const int cp = __shfl_up_sync(0xFFFFFFFFu, c, 1), cn = __shfl_down_sync(0xFFFFFFFFu, c, 1);
+    const bool first = on && (lane == 0 || cp != c);
+    const bool single = lane == ne - 2 || cn != c;
+    const unsigned fm = __ballot_sync(0xFFFFFFFFu, first);
+    n_split = __popc(fm);
+    if (first) {
+      const int idx = __popc(fm & ((1u << lane) - 1u));
+      CellEntry e;
+      e.thr = tau[lane];
+      e.codes = single ? ((unsigned)lane | ((unsigned)(lane + 1) << 8)) : 0xFFFFu;
+      s_cell[idx] = (unsigned short)c;
+      s_entry[idx] = e;
+    }
+    __syncwarp();
+  }
+  double D = 0.0;
+  {
+    // every cell without a threshold through its sums and moments, spread over the grid (a thread takes
+    // one cell): its entry is the number of thresholds in lower cells, and
+    // sum omega (u - q)^2 = A2 - 2 q A1 + q^2 A0 for the entry's value q
+    for (int r = (int)blockIdx.x + (int)gridDim.x * (LTB - 1 - tid); r < SORT_ROWS; r += (int)gridDim.x * LTB) {
       const unsigned long long cn = ws->cellN[r];
       const long long cs = ws->cellS[r];
       const double a0 = ws->cellA[0][r], a1 = ws->cellA[1][r], a2 = ws->cellA[2][r];
-      if (e.codes != 0xFFFFu && e.thr == INFINITY && (cn || a0 != 0.0)) {
-        const int j = (int)(e.codes & 0xFFu);
+      int j = 0;
+      bool split = false;
+      for (int k = 0; k < ne - 1; ++k) { const int c = d.thr_cell[k]; j += c < r ? 1 : 0; split |= c == r; }
+      if (!split && (cn || a0 != 0.0)) {
         if (!last) { atomicAdd(&sN[j], cn); atomicAdd(&sS[j], (unsigned long long)cs); }
         const double q = (double)lutv[j];
         D += a2 - 2.0 * q * a1 + q * q * a0;
       }
     }
   }
-  for (unsigned sbase = 0; sbase < n_split_all; sbase += MAX_SPLIT) {
-    const int n_split = (int)min((unsigned)MAX_SPLIT, n_split_all - sbase);
-    __syncthreads();
-    if (tid < n_split) { const int c = ws->split_cells[sbase + tid]; s_cell[tid] = (unsigned short)c; s_entry[tid] = ws->cellt[c]; }
-    __syncthreads();
-    for (unsigned tile = blockIdx.x * (LTB / 32) + warp; tile < n_tiles; tile += gridDim.x * (LTB / 32)) {
-      const unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
-      const uint2* src = a.cache + (size_t)tile * TILE_ELEMS;
-      // segment lengths -> exclusive offsets (two cells per lane)
-      unsigned len0 = 0, len1 = 0, q0 = 0, q1 = 0;
-      if (lane < n_split) { const int c = s_cell[lane]; q0 = ts[c]; len0 = ts[c + 1] - q0; }
-      if (lane + 32 < n_split) { const int c = s_cell[lane + 32]; q1 = ts[c]; len1 = ts[c + 1] - q1; }
-      unsigned inc0 = len0, inc1 = len1;
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned v0 = __shfl_up_sync(0xFFFFFFFFu, inc0, o), v1 = __shfl_up_sync(0xFFFFFFFFu, inc1, o);
-        if (lane >= o) { inc0 += v0; inc1 += v1; }
-      }
-      const unsigned tot0 = __shfl_sync(0xFFFFFFFFu, inc0, 31), total = tot0 + __shfl_sync(0xFFFFFFFFu, inc1, 31);
-      __syncwarp();
-      s_off[warp][lane] = (unsigned short)(inc0 - len0); s_p0[warp][lane] = (unsigned short)q0;
-      s_off[warp][lane + 32] = (unsigned short)(tot0 + inc1 - len1); s_p0[warp][lane + 32] = (unsigned short)q1;
-      if (lane == 0) s_off[warp][MAX_SPLIT] = (unsigned short)total;
-      __syncwarp();
-      // every lane takes a contiguous share of the items: its entry changes a few times at most, so the
-      // sums of the current entry stay in registers and reach the CTA's accumulators on a change
-      const unsigned share = (total + 31u) / 32u;
-      const unsigned i_lo = min(total, lane * share), i_hi = min(total, i_lo + share);
-      int cur = -1;
-      unsigned long long n = 0, sv = 0;
-      for (unsigned base = i_lo; base < i_hi; base += 4) {
-        uint2 v[4];
-        int cell_l[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const unsigned item = base + k;
-          cell_l[k] = -1;
-          v[k] = make_uint2(0u, 0u);
-          if (item < i_hi) {
-            int l = 0;                       // the split cell whose item range holds `item`: binary search over <= 64 offsets
-#pragma unroll
-            for (int step = 32; step >= 1; step >>= 1)
-              if (l + step < n_split && s_off[warp][l + step] <= item) l += step;
-            cell_l[k] = l;
-            const unsigned pp = s_p0[warp][l] + (item - s_off[warp][l]);
-            v[k] = __ldg(src + (pp & 15u) * LTB + (pp >> 4));
-          }
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (cell_l[k] < 0) continue;
-          const CellEntry e = s_entry[cell_l[k]];
-          const float u = __uint_as_float(v[k].x), om = __uint_as_float(v[k].y);
-          int code;
-          if (e.codes == 0xFFFFu) code = count_below(tau, u);   // several thresholds in one cell: the general search
-          else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
-          const float d = __fsub_rn(u, lutv[code]);
-          D += (double)__fmul_rn(__fmul_rn(om, d), d);
-          if (!last) {
-            if (code != cur) {
-              if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
-              cur = code; n = 0; sv = 0;
-            }
-            const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
-            n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
-            sv += (unsigned long long)fix24(ou);
-          }
-        }
-      }
-      if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
+  for (unsigned tile = blockIdx.x * (LTB / 32) + warp; tile < n_tiles; tile += gridDim.x * (LTB / 32)) {
+    const unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
+    const uint2* src = a.cache + (size_t)tile * TILE_ELEMS;
+    // segment lengths -> exclusive offsets (one cell per lane)
+    unsigned len0 = 0, q0 = 0;
+    if (lane < n_split) { const int c = s_cell[lane]; q0 = ts[c]; len0 = ts[c + 1] - q0; }
+    unsigned inc0 = len0;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned v0 = __shfl_up_sync(0xFFFFFFFFu, inc0, o);
+      if (lane >= o) inc0 += v0;
     }
+    const unsigned total = __shfl_sync(0xFFFFFFFFu, inc0, 31);
+    __syncwarp();
+    s_off[warp][lane] = (unsigned short)(inc0 - len0); s_p0[warp][lane] = (unsigned short)q0;
+    if (lane == 0) s_off[warp][MAX_SPLIT] = (unsigned short)total;
+    __syncwarp();
+    // every lane takes a contiguous share of the items: its entry changes a few times at most, so the
+    // sums of the current entry stay in registers and reach the CTA's accumulators on a change
+    const unsigned share = (total + 31u) / 32u;
+    const unsigned i_lo = min(total, lane * share), i_hi = min(total, i_lo + share);
+    int cur = -1;
+    unsigned long long n = 0, sv = 0;
+    for (unsigned base = i_lo; base < i_hi; base += 4) {
+      uint2 v[4];
+      int cell_l[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned item = base + k;
+        cell_l[k] = -1;
+        v[k] = make_uint2(0u, 0u);
+        if (item < i_hi) {
+          int l = 0;                       // the split cell whose item range holds `item`: binary search over <= 32 offsets
+#pragma unroll
+          for (int step = 16; step >= 1; step >>= 1)
+            if (l + step < n_split && s_off[warp][l + step] <= item) l += step;
+          cell_l[k] = l;
+          const unsigned pp = s_p0[warp][l] + (item - s_off[warp][l]);
+          v[k] = __ldg(src + (pp & 15u) * LTB + (pp >> 4));
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (cell_l[k] < 0) continue;
+        const CellEntry e = s_entry[cell_l[k]];
+        const float u = __uint_as_float(v[k].x), om = __uint_as_float(v[k].y);
+        int code;
+        if (e.codes == 0xFFFFu) code = count_below(tau, u);   // several thresholds in one cell: the general search
+        else code = (int)((u > e.thr ? e.codes >> 8 : e.codes) & 0xFFu);
+        const float dd = __fsub_rn(u, lutv[code]);
+        D += (double)__fmul_rn(__fmul_rn(om, dd), dd);
+        if (!last) {
+          if (code != cur) {
+            if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
+            cur = code; n = 0; sv = 0;
+          }
+          const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
+          n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
+          sv += (unsigned long long)fix24(ou);
+        }
+      }
+    }
+    if (cur >= 0) flush_limbs(lN[0], lN[1], lS0, lS1, lS2, cur, n, sv);
   }
   for (int o = 16; o; o >>= 1) D += __shfl_xor_sync(0xFFFFFFFFu, D, o);
   if (lane == 0 && D != 0.0) atomicAdd(&sD, D);
@@ -572,51 +585,41 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
   __syncthreads();
   if (tid == 0) s_is_last = atomicAdd(&ws->done, 1u) == gridDim.x - 1 ? 1 : 0;
   __syncthreads();
-  if (s_is_last) {
+  if (s_is_last && tid < 32) {
+    // one warp: every CTA has added its share (cells with a threshold element by element, the others by
+    // their sums).  Centroids one lane per entry, a rank sort, and the next iteration's descriptor.
     __threadfence();
-    // totals so far (cells with a threshold), then every other cell through its sums and moments:
-    // sum omega (u - q)^2 = A2 - 2 q A1 + q^2 A0 for the cell's entry value q
-    // every CTA has added its share (cells with a threshold element by element, the others by their sums)
-    if (tid < 32) { sN[tid] = __ldcg(&ws->accN[tid]); sS[tid] = (unsigned long long)__ldcg(&ws->accS[tid]); }
-    if (tid == 0) sD = __ldcg(&ws->accD);
-    __syncthreads();
-    // centroids: one thread per entry; thread 0 sorts and publishes
-    if (!last && tid < ne) {
-      float t = lutv[tid];
-      const unsigned long long n = sN[tid];
-      if (n) {
-        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn((long long)sS[tid]), __ull2double_rn(n)));
+    const unsigned long long n = __ldcg(&ws->accN[tid]);
+    const long long sv = __ldcg(&ws->accS[tid]);
+    if (tid == 0) distortion[it] = __ldcg(&ws->accD);
+    ws->accN[tid] = 0; ws->accS[tid] = 0;
+    if (tid == 0) { ws->accD = 0.0; ws->done = 0; }
+    if (last) {
+      out_lut[tid] = tid < ne ? lutv[tid] : 0.0f;
+    } else {
+      float t = lutv[tid];                       // lanes from n_entries on hold the last entry's value
+      if (tid < ne && n) {
+        const float cen = __double2float_rn(__ddiv_rn(__ll2double_rn(sv), __ull2double_rn(n)));
         uint32_t b = __float_as_uint(cen);
         b += 0x7FFFu + ((b >> 16) & 1u);
-        b &= 0xFFFF0000u;                      // nearest bf16, ties to even
+        b &= 0xFFFF0000u;                        // nearest bf16, ties to even
         t = __uint_as_float(b);
       }
-      tau[tid] = t;                            // tau is free here: the new, unsorted table
-    }
-    __syncthreads();
-    if (tid == 0) {
-      distortion[it] = sD;
-      if (!last) {
-        for (int i = 1; i < ne; ++i) {         // insertion sort, ascending
-          const float x = tau[i];
-          int p = i - 1;
-          while (p >= 0 && tau[p] > x) { tau[p + 1] = tau[p]; --p; }
-          tau[p + 1] = x;
-        }
+      // ascending order: the rank of an entry is the number of entries before it (ties by index)
+      int rank = 0;
+      for (int k = 0; k < 32; ++k) {
+        const float o = __shfl_sync(0xFFFFFFFFu, t, k);
+        rank += (k < ne && (o < t || (o == t && k < tid))) ? 1 : 0;
       }
-    }
-    __syncthreads();
-    if (tid < SOP_MAX_ENTRIES) {
-      if (!last) { if (tid < ne) ws->lut[tid] = tau[tid]; }
-      else out_lut[tid] = tid < ne ? lutv[tid] : 0.0f;
-      ws->accN[tid] = 0; ws->accS[tid] = 0;
-    }
-    if (tid == 0) { ws->accD = 0.0; ws->done = 0; }
-    __syncthreads();
-    if (!last) {                      // the next iteration's lookup tables
-      if (tid < 32) lutv[tid] = tau[min(tid, ne - 1)];
-      __syncthreads();
-      lloyd_prepare_tables(ws, lutv, tau, ne);
+      if (tid < ne) s_new[rank] = t;
+      __syncwarp();
+      if (tid >= ne) s_new[tid] = 0.0f;
+      __syncwarp();
+      const float top = s_new[ne - 1];
+      __syncwarp();
+      if (tid >= ne) s_new[tid] = top;           // padded with the last entry
+      __syncwarp();
+      lloyd_publish_desc(ws, s_new, ne);
     }
   }
 }
