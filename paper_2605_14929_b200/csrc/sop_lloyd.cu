@@ -321,14 +321,59 @@ __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exa
   return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
 }
 
+constexpr int CELL_LIMBS = 14;
+constexpr unsigned CELL_SPILL_TILES = 128;
+constexpr double MOMENT_UNIT = 1099511627776.0;   // 2^40
+
+__device__ __forceinline__ void add_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell, long long v) {
+  atomicAdd(&cL[first][cell], (unsigned)(v & 0xFFFFll));
+  atomicAdd(&cL[first + 1][cell], (unsigned)((v >> 16) & 0xFFFFll));
+  atomicAdd(&cL[first + 2][cell], (unsigned)(int)(v >> 32));
+}
+
+// One run of elements of one cell (at most 16): fix(omega) sums below 2^28, fix(omega u) sums below 2^37
+// in magnitude, moments below 2^6 in magnitude (so below 2^46 in units of 2^-40).
+__device__ __forceinline__ void flush_cell(unsigned (*cL)[SORT_ROWS], int cell, unsigned long long n, unsigned long long sv,
+                                           double a0, double a1, double a2) {
+  atomicAdd(&cL[0][cell], (unsigned)(n & 0xFFFFull));
+  atomicAdd(&cL[1][cell], (unsigned)(n >> 16));
+  add_limbs3(cL, 2, cell, (long long)sv);
+  add_limbs3(cL, 5, cell, __double2ll_rn(a0 * MOMENT_UNIT));
+  add_limbs3(cL, 8, cell, __double2ll_rn(a1 * MOMENT_UNIT));
+  add_limbs3(cL, 11, cell, __double2ll_rn(a2 * MOMENT_UNIT));
+}
+
+__device__ __forceinline__ long long join_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell) {
+  return (long long)cL[first][cell] + ((long long)cL[first + 1][cell] << 16) + ((long long)(int)cL[first + 2][cell] << 32);
+}
+
+// Whole CTA, after a barrier: the CTA's limbs are added to the per-cell sums of the pool and cleared.
+__device__ void spill_cells(unsigned (*cL)[SORT_ROWS], LloydWs* ws) {
+  for (int r = threadIdx.x; r < SORT_ROWS; r += blockDim.x) {
+    const unsigned long long n = (unsigned long long)cL[0][r] + ((unsigned long long)cL[1][r] << 16);
+    const long long sv = join_limbs3(cL, 2, r);
+    const long long m0 = join_limbs3(cL, 5, r), m1 = join_limbs3(cL, 8, r), m2 = join_limbs3(cL, 11, r);
+    if (n) atomicAdd(&ws->cellN[r], n);
+    if (sv) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellS[r]), (unsigned long long)sv);
+    if (m0) atomicAdd(&ws->cellA[0][r], (double)m0 * (1.0 / MOMENT_UNIT));
+    if (m1) atomicAdd(&ws->cellA[1][r], (double)m1 * (1.0 / MOMENT_UNIT));
+    if (m2) atomicAdd(&ws->cellA[2][r], (double)m2 * (1.0 / MOMENT_UNIT));
+#pragma unroll
+    for (int l = 0; l < CELL_LIMBS; ++l) cL[l][r] = 0;
+  }
+}
+
 __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws) {
   __shared__ unsigned hist[SORT_ROWS + 3];
   __shared__ unsigned warp_tot[LTB / 32];
   extern __shared__ __align__(16) uint2 stage[];                  // TILE_ELEMS pairs (dynamic: the kernel needs 60 KB in all)
-  __shared__ unsigned long long cN[SORT_ROWS], cS[SORT_ROWS];     // this CTA's share of the per-cell sums
-  __shared__ double cA[3][SORT_ROWS];
+  // this CTA's share of the per-cell sums, as 32-bit limbs that native shared-memory atomics add:
+  // [0..1] sum fix(omega), [2..4] sum fix(omega u), [5..7], [8..10], [11..13] the three moments in units
+  // of 2^-40.  Low limbs hold 16 bits, the top limb the signed rest.
+  __shared__ unsigned cL[CELL_LIMBS][SORT_ROWS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int r = tid; r < SORT_ROWS; r += LTB) { cN[r] = 0; cS[r] = 0; cA[0][r] = 0.0; cA[1][r] = 0.0; cA[2][r] = 0.0; }
+  for (int i = tid; i < CELL_LIMBS * SORT_ROWS; i += LTB) (&cL[0][0])[i] = 0;
+  unsigned tiles_since_spill = 0;
   const unsigned count = ws->list_count;
   const unsigned n_tiles = (count + LTB - 1) / LTB;
   const int k = ws->k;
@@ -389,7 +434,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
     unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
     for (int r = tid; r <= SORT_ROWS; r += LTB) ts[r] = (unsigned short)hist[r];      // hist[SORT_ROWS] = 4096: the end of the last cell
     // per-cell sums: thread t owns the sorted positions 16 t .. 16 t + 15 (ascending cells), keeps the
-    // current cell's sums in registers and adds them to the CTA's arrays when the cell changes
+    // current cell's sums in registers and adds them to the CTA's limbs when the cell changes
     {
       int cur = -1;
       unsigned long long n = 0, sv = 0;
@@ -400,7 +445,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
         const float u = __uint_as_float(v.x), om = __uint_as_float(v.y);
         const int c = sort_cell(u);
         if (c != cur) {
-          if (cur >= 0) { atomicAdd(&cN[cur], n); atomicAdd(&cS[cur], sv); atomicAdd(&cA[0][cur], a0); atomicAdd(&cA[1][cur], a1); atomicAdd(&cA[2][cur], a2); }
+          if (cur >= 0) flush_cell(cL, cur, n, sv, a0, a1, a2);
           cur = c; n = 0; sv = 0; a0 = a1 = a2 = 0.0;
         }
         const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
@@ -409,15 +454,18 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
         const double dou = (double)om * (double)u;
         a0 += (double)om; a1 += dou; a2 += dou * (double)u;
       }
-      atomicAdd(&cN[cur], n); atomicAdd(&cS[cur], sv); atomicAdd(&cA[0][cur], a0); atomicAdd(&cA[1][cur], a1); atomicAdd(&cA[2][cur], a2);
+      flush_cell(cL, cur, n, sv, a0, a1, a2);
     }
     __syncthreads();
+    // a cell takes at most 258 flushes per tile and a low limb 2^16 - 1 per flush: the limbs go to the
+    // global sums before they can wrap
+    if (++tiles_since_spill == CELL_SPILL_TILES) {
+      spill_cells(cL, ws);
+      tiles_since_spill = 0;
+      __syncthreads();
+    }
   }
-  for (int r = tid; r < SORT_ROWS; r += LTB) {
-    if (cN[r]) atomicAdd(&ws->cellN[r], cN[r]);
-    if (cS[r]) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellS[r]), cS[r]);
-    if (cA[0][r] != 0.0) { atomicAdd(&ws->cellA[0][r], cA[0][r]); atomicAdd(&ws->cellA[1][r], cA[1][r]); atomicAdd(&ws->cellA[2][r], cA[2][r]); }
-  }
+  if (tiles_since_spill) spill_cells(cL, ws);
 }
 
 // One warp per tile.  The elements of the tile that lie in cells holding a threshold (sorted positions
