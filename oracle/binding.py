@@ -142,8 +142,9 @@ def eval_block(w, c, atom, fmt, k: int, pot_scale: float = 0.0):
     return dict(cos=cs.value, sse=se.value, s_hat=sh.value, E=E.value, M=M.value, codes=codes, q=q)
 
 
-def pair_search(W, c, fmt, atoms, k_mode: int = K_AUTO, want_blocks: bool = False):
-    """Returns dict(pair, signed, k, best, block_cos, block_sse)."""
+def pair_search(W, c, fmt, atoms, k_mode: int = K_AUTO, want_blocks: bool = False, select_metric: int = 0):
+    """Returns dict(pair, signed, k, best, block_cos, block_sse).  select_metric: 0 = the block cosine decides
+    the per-block reassignment, 1 = the block squared error does (design axis ii)."""
     w16 = _w16(W)
     M, K = w16.shape
     c = np.ascontiguousarray(np.asarray(c, dtype=np.float32))
@@ -155,15 +156,18 @@ def pair_search(W, c, fmt, atoms, k_mode: int = K_AUTO, want_blocks: bool = Fals
     best = np.zeros(5, dtype=np.int32)
     bc = np.zeros((A, NB), dtype=np.float32) if want_blocks else None
     bs = np.zeros((A, NB), dtype=np.float32) if want_blocks else None
-    lib().osop_pair_search(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
-                           C.byref(_fmt(fmt)), k_mode, _atoms(atoms), A, _p(pair, _PairStat), _p(sgn, _PairStat),
+    lib().osop_pair_search_axes(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
+                           C.byref(_fmt(fmt)), k_mode, _atoms(atoms), A, int(select_metric), _p(pair, _PairStat), _p(sgn, _PairStat),
                            _p(k_out, C.c_int), _p(best, C.c_int),
                            _p(bc, C.c_float) if want_blocks else None, _p(bs, C.c_float) if want_blocks else None)
     return dict(pair=pair, signed=sgn, k=k_out, best=best, block_cos=bc, block_sse=bs)
 
 
-def dd_lloyd(W, c, fmt, k: int, block_cos, pool_rank: int, init_lut, iters: int):
-    """Returns (lut, distortion[iters + 1], pool_count)."""
+def dd_lloyd(W, c, fmt, k: int, block_cos, pool_rank: int, init_lut, iters: int, pool_by_error: bool = False,
+             pool_threshold: float = 0.0, uniform_weights: bool = False):
+    """Returns (lut, distortion[iters + 1], pool_count).  block_cos holds the per-block metric that ranks the
+    blocks: cosines, or squared errors with pool_by_error (axis i); pool_rank = 0 takes pool_threshold instead of
+    a rank (axis iv); uniform_weights sets every Lloyd weight to 1 (axis iii)."""
     w16 = _w16(W)
     M, K = w16.shape
     c = np.ascontiguousarray(np.asarray(c, dtype=np.float32))
@@ -172,14 +176,15 @@ def dd_lloyd(W, c, fmt, k: int, block_cos, pool_rank: int, init_lut, iters: int)
     out = np.zeros(len(init), dtype=np.float32)
     dist = np.zeros(iters + 1, dtype=np.float64)
     cnt = C.c_longlong()
-    lib().osop_dd_lloyd(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
-                        C.byref(_fmt(fmt)), k, _p(bc, C.c_float), C.c_longlong(pool_rank), _p(init, C.c_float),
-                        len(init), iters, _p(out, C.c_float), _p(dist, C.c_double), C.byref(cnt))
+    lib().osop_dd_lloyd_axes(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
+                             C.byref(_fmt(fmt)), k, _p(bc, C.c_float), int(bool(pool_by_error)), C.c_longlong(pool_rank),
+                             C.c_float(pool_threshold), int(bool(uniform_weights)), _p(init, C.c_float),
+                             len(init), iters, _p(out, C.c_float), _p(dist, C.c_double), C.byref(cnt))
     return out, dist, cnt.value
 
 
 def pack(W, c, fmt, a, k_a: int, b=None, k_b: int = 0, use_sign: int = 0, container_bits: int = 8,
-         word_sign_bits: int = 0):
+         word_sign_bits: int = 0, select_metric: int = 0):
     """Returns dict(rc, codes [N_b, 2n] uint8, words uint8 stream, n_sel1, n_neg)."""
     w16 = _w16(W)
     M, K = w16.shape
@@ -188,8 +193,8 @@ def pack(W, c, fmt, a, k_a: int, b=None, k_b: int = 0, use_sign: int = 0, contai
     codes = np.zeros((NB, 2 * a.n_bits), dtype=np.uint8)
     words = np.zeros((NB * container_bits + 7) // 8, dtype=np.uint8)
     n1, nn = C.c_longlong(), C.c_longlong()
-    rc = lib().osop_pack(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
+    rc = lib().osop_pack_axes(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
                          C.byref(_fmt(fmt)), C.byref(_atom(a)), k_a, C.byref(_atom(b)) if b is not None else None, k_b,
-                         use_sign, container_bits, word_sign_bits, _p(codes, C.c_ubyte), _p(words, C.c_ubyte),
+                         use_sign, container_bits, word_sign_bits, int(select_metric), _p(codes, C.c_ubyte), _p(words, C.c_ubyte),
                          C.byref(n1), C.byref(nn))
     return dict(rc=rc, codes=codes, words=words, n_sel1=n1.value, n_neg=nn.value)

@@ -20,6 +20,8 @@
 //   sign-negated atoms as separate candidates ......... Section "Per-Layer Pair Search"
 //   data-derived DD-n by Lloyd updates + snap ......... Section "Per-Layer Pair Search" (steps 2-3, PO2 description)
 //   payload: 2n bytes of codes per g = 16 block ....... Section "Overview", item 4
+//   design axes (i)-(iv): partition metric, reassignment metric, Lloyd weighting, pool definition
+//                                                       paragraph "Pair-search design axes"
 //
 // Where the paper is silent the reading taken is stated at the function that needs it.
 //
@@ -346,9 +348,13 @@ static void layer_prepass(const uint16_t* W, long long M, long long K, long long
 //   best[5] = {best_a, best_b (a < b by ACos, ties to the smallest (a, b)), best single LUT candidate,
 //              best signed pair i, j}; -1 where undefined.
 //   block_cos / block_sse (optional) [n_atoms x N_b].
-void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
-                      int k_mode, const Atom* atoms, int n_atoms, PairStat* pair_table, PairStat* signed_table,
-                      int* k_out, int* best, float* block_cos, float* block_sse) {
+//   select_metric (design axis ii, the metric of the per-block finishing reassignment): 0 = block
+//     cosine (the larger wins), 1 = block squared error (the smaller wins); ties keep the earlier
+//     candidate either way.  The reported ACos / mse / counts are those of the resulting assignment;
+//     the best pair is ranked by ACos in both cases.
+void osop_pair_search_axes(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
+                           int k_mode, const Atom* atoms, int n_atoms, int select_metric, PairStat* pair_table,
+                           PairStat* signed_table, int* k_out, int* best, float* block_cos, float* block_sse) {
   const long long nbk = K / G, NB = M * nbk;
   std::vector<float> pot(n_atoms);
   layer_prepass(W, M, K, ldw, *f, k_mode, atoms, n_atoms, k_out, pot.data());
@@ -376,7 +382,7 @@ void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw
         if (atoms[a].kind != KIND_LUT) continue;
         for (int a2 = a + 1; a2 < A; ++a2) {
           if (atoms[a2].kind != KIND_LUT || atoms[a2].n_bits != atoms[a].n_bits) continue;
-          const bool mu = cs[a2] > cs[a];
+          const bool mu = select_metric ? er[a2] < er[a] : cs[a2] > cs[a];
           S[a * A + a2] += (double)(mu ? cs[a2] : cs[a]);
           E[a * A + a2] += (double)(mu ? er[a2] : er[a]);
           N1[a * A + a2] += mu ? 1 : 0;
@@ -390,7 +396,7 @@ void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw
             const int cand[4] = {i, i + 1, j2, j2 + 1};
             int pick = 0;
             for (int t = 1; t < (j2 == i ? 2 : 4); ++t)
-              if (cs[cand[t]] > cs[cand[pick]]) pick = t;
+              if (select_metric ? er[cand[t]] < er[cand[pick]] : cs[cand[t]] > cs[cand[pick]]) pick = t;
             SS[i * A + j2] += (double)cs[cand[pick]];
             ES[i * A + j2] += (double)er[cand[pick]];
             NS1[i * A + j2] += pick >= 2 ? 1 : 0;
@@ -421,6 +427,12 @@ void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw
   }
 }
 
+void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
+                      int k_mode, const Atom* atoms, int n_atoms, PairStat* pair_table, PairStat* signed_table,
+                      int* k_out, int* best, float* block_cos, float* block_sse) {
+  osop_pair_search_axes(W, M, K, ldw, c, f, k_mode, atoms, n_atoms, 0, pair_table, signed_table, k_out, best, block_cos, block_sse);
+}
+
 // Data-derived DD-n codebook: Lloyd iteration on the pool of blocks that the primary codebook
 // reconstructs worst (pair-search steps 2-3).
 //   pool      = blocks whose cosine under the primary codebook is <= the pool_rank-th smallest
@@ -432,17 +444,33 @@ void osop_pair_search(const uint16_t* W, long long M, long long K, long long ldw
 //               an empty code keeps its entry; every centroid is snapped to bf16; entries re-sorted.
 //   distortion[i] = sum omega (u - q)^2 (FP64) under the table used in iteration i; distortion[iters]
 //               under the final table.
-void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f, int k,
-                   const float* block_cos, long long pool_rank, const float* init_lut, int n_entries, int iters,
-                   float* out_lut, double* distortion, long long* pool_count) {
+// Design axes (paragraph "Pair-search design axes"):
+//   (i)   pool_by_error = 0: block_metric holds block cosines, the worst blocks are the smallest;
+//         pool_by_error = 1: block_metric holds block squared errors (unweighted), the worst are the largest.
+//   (iii) uniform_weights = 1: omega = 1 for every channel instead of c / max c.
+//   (iv)  pool_rank >= 1: the pool is every block at least as bad as the pool_rank-th worst (the p %
+//         rule and top-k are both a rank); pool_rank = 0: the pool is every block at least as bad as
+//         the given pool_threshold on the metric (quantile threshold fixed by the caller).
+void osop_dd_lloyd_axes(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f, int k,
+                        const float* block_metric, int pool_by_error, long long pool_rank, float pool_threshold,
+                        int uniform_weights, const float* init_lut, int n_entries, int iters,
+                        float* out_lut, double* distortion, long long* pool_count) {
   const long long nbk = K / G, NB = M * nbk;
-  std::vector<float> sorted(block_cos, block_cos + NB);
-  std::nth_element(sorted.begin(), sorted.begin() + (pool_rank - 1), sorted.end());
-  const float tau = sorted[pool_rank - 1];
+  const float* block_cos = block_metric;
+  float tau = pool_threshold;
+  if (pool_rank >= 1) {
+    std::vector<float> sorted(block_metric, block_metric + NB);
+    if (pool_by_error) {
+      std::nth_element(sorted.begin(), sorted.begin() + (pool_rank - 1), sorted.end(), [](float x, float y) { return x > y; });
+    } else {
+      std::nth_element(sorted.begin(), sorted.begin() + (pool_rank - 1), sorted.end());
+    }
+    tau = sorted[pool_rank - 1];
+  }
   float cmax = 0.0f;
   for (long long i = 0; i < K; ++i) cmax = std::max(cmax, c[i]);
   std::vector<float> omega(K);
-  for (long long i = 0; i < K; ++i) omega[i] = cmax > 0.0f ? c[i] / cmax : 0.0f;
+  for (long long i = 0; i < K; ++i) omega[i] = uniform_weights ? 1.0f : (cmax > 0.0f ? c[i] / cmax : 0.0f);
   std::vector<float> lut(init_lut, init_lut + n_entries);
   long long cnt = 0;
   for (int it = 0; it <= iters; ++it) {
@@ -451,7 +479,8 @@ void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, c
     cnt = 0;
     for (long long m = 0; m < M; ++m)
       for (long long j = 0; j < nbk; ++j) {
-        if (!(block_cos[m * nbk + j] <= tau)) continue;
+        const float metric = block_cos[m * nbk + j];
+        if (!(pool_by_error ? metric >= tau : metric <= tau)) continue;
         ++cnt;
         float w[G], absmax = 0.0f;
         load_block(W, ldw, m, j, w);
@@ -480,6 +509,12 @@ void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, c
   *pool_count = cnt;
 }
 
+void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f, int k,
+                   const float* block_cos, long long pool_rank, const float* init_lut, int n_entries, int iters,
+                   float* out_lut, double* distortion, long long* pool_count) {
+  osop_dd_lloyd_axes(W, M, K, ldw, c, f, k, block_cos, 0, pool_rank, 0.0f, 0, init_lut, n_entries, iters, out_lut, distortion, pool_count);
+}
+
 // Materialise: codes and scale words for the chosen codebook(s).
 //   candidates per block, in priority order: a, (-a if use_sign), b, (-b if use_sign); the one with the
 //   largest block cosine wins, ties keep the earlier.  selector = winner is b or -b; sign = winner is a
@@ -489,9 +524,10 @@ void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, c
 //   index found on -u); for FP atoms it is the format's bit pattern.
 //   words: b-bit scale words, block index ascending, as one little-endian bit stream
 //   (b = 12: two words per three bytes).  Returns 0, or -1 when a needed sign/selector bit does not exist.
-int osop_pack(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
-              const Atom* a, int k_a, const Atom* b, int k_b, int use_sign, int container_bits, int word_sign_bits,
-              unsigned char* codes, unsigned char* words, long long* n_sel1, long long* n_neg) {
+//   select_metric: 0 = the largest block cosine wins, 1 = the smallest block squared error wins (design axis ii).
+int osop_pack_axes(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
+                   const Atom* a, int k_a, const Atom* b, int k_b, int use_sign, int container_bits, int word_sign_bits,
+                   int select_metric, unsigned char* codes, unsigned char* words, long long* n_sel1, long long* n_neg) {
   const long long nbk = K / G, NB = M * nbk;
   const int n = a->n_bits;
   const int x = f->exp_bits, y = f->man_bits;
@@ -515,7 +551,7 @@ int osop_pack(const uint16_t* W, long long M, long long K, long long ldw, const 
           Atom cand = base;
           if (sg) cand.negated = 1 - cand.negated;
           const BlockEval r = eval_block(w, c + j * G, cand, *f, which ? k_b : k_a, layer_pot_scale(wmax, cand.tmax));
-          if (pick < 0 || r.cos > bestr.cos) { bestr = r; pick = which * 2 + sg; }
+          if (pick < 0 || (select_metric ? r.sse < bestr.sse : r.cos > bestr.cos)) { bestr = r; pick = which * 2 + sg; }
         }
       }
       const uint32_t sel = pick >= 2, sgn = pick & 1;
@@ -535,6 +571,12 @@ int osop_pack(const uint16_t* W, long long M, long long K, long long ldw, const 
         }
     }
   return 0;
+}
+
+int osop_pack(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
+              const Atom* a, int k_a, const Atom* b, int k_b, int use_sign, int container_bits, int word_sign_bits,
+              unsigned char* codes, unsigned char* words, long long* n_sel1, long long* n_neg) {
+  return osop_pack_axes(W, M, K, ldw, c, f, a, k_a, b, k_b, use_sign, container_bits, word_sign_bits, 0, codes, words, n_sel1, n_neg);
 }
 
 }  // extern "C"
