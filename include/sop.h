@@ -33,6 +33,7 @@ extern "C" {
 #define SOP_FMTA_FROM_RESULT (-1) /* fmta_index of sop_dd4_lloyd: best single LUT candidate of a previous search */
 #define SOP_ALL_ATOMS 0xFFFFFFFFu /* eval_mask of sop_pair_search: evaluate every candidate */
 #define SOP_SEARCH_SINGLES_ONLY 1 /* flags of sop_pair_search: reduce single candidates only, no pair / signed entries */
+#define SOP_SEARCH_SELECT_MSE 2   /* flags of sop_pair_search: the per-block reassignment takes the smaller block error */
 
 enum {
   SOP_OK = 0,
@@ -159,7 +160,10 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *   its shift is reported as 0.  The masks must be disjoint and not both empty.  At most 8 distinct
  *   tables may be evaluated per call (an atom and its negation share one).
  * flags: SOP_SEARCH_SINGLES_ONLY fills only the diagonal (and best_single): enough to choose the
- *   primary codebook FMTa before the Lloyd refinement.
+ *   primary codebook FMTa before the Lloyd refinement.  SOP_SEARCH_SELECT_MSE (paragraph "Pair-search
+ *   design axes", axis ii): in every two-way and signed entry the block goes to the candidate with the
+ *   smaller block squared error instead of the larger block cosine (ties keep the earlier candidate);
+ *   acos, mse and the counts are those of that assignment, the best pair is still ranked by acos.
  * prev_result_dev (may be NULL): with k_mode = SOP_K_FROM_RESULT, the result block of the earlier call on
  *   this layer (not result_dev itself).  The shift of every scale class and max|W| are taken from it
  *   instead of reading W once more; every per-block-scaled class of this call must then contain a
@@ -189,24 +193,37 @@ int sop_profile_last_ms(int which, float* ms);    /* = sop_profile_ms(which, 0, 
 int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE_SWEEP, ms) */
 
 /* ---- DD-n: per-layer data-derived codebook by Lloyd iteration (pair-search steps 2-3) -------
- * Pool = blocks whose cosine under the primary codebook FMTa is <= the pool_rank-th smallest of
- * the layer (ties all in).  Each iteration assigns every pool element u = w / scale (scale against
- * tmax = 1) to its nearest entry, accumulates per entry sum(omega) and sum(omega u) with
- * omega = c / max(c) in int64 fixed point (2^-24 units, |omega u| clamped to 256), replaces each
- * non-empty entry by its centroid snapped to bf16, and re-sorts.
+ * Pool = blocks at least as bad under the primary codebook FMTa as the pool_rank-th worst of the
+ * layer (ties all in).  By default "bad" is a small block cosine.  Each iteration assigns every pool
+ * element u = w / scale (scale against tmax = 1) to its nearest entry, accumulates per entry
+ * sum(omega) and sum(omega u) with omega = c / max(c) in int64 fixed point (2^-24 units, |omega u|
+ * clamped to 256), replaces each non-empty entry by its centroid snapped to bf16, and re-sorts.
  *   fmta_index: index into `atoms` of FMTa (its table is the initial codebook), or
  *     SOP_FMTA_FROM_RESULT to use search_dev->best_single.
- *   block_cos_dev: [n_atoms x N_b] as written by sop_pair_search (row fmta is read).
+ *   block_metric_dev: [n_atoms x N_b] as written by sop_pair_search (row fmta is read): the block
+ *     cosines, or with SOP_LLOYD_POOL_BY_ERROR the block squared errors.
+ *   pool_rank in [1, N_b].  The p % rule of the paper is the rank ceil(N_b (100 - p) / 100); a top-k
+ *     pool is the rank k.
+ *   flags (paragraph "Pair-search design axes"):
+ *     SOP_LLOYD_POOL_BY_ERROR    axis (i): rank the blocks by their squared error (the largest are the worst);
+ *     SOP_LLOYD_UNIFORM_WEIGHTS  axis (iii): omega = 1 for every channel;
+ *     SOP_LLOYD_POOL_THRESHOLD   axis (iv): the pool is every block whose metric is at least as bad as
+ *       pool_threshold (cosine <= threshold, or error >= threshold); pool_rank is ignored.  An empty pool
+ *       leaves the table as it is.
  *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
  *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
  *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
  *   pool_count_dev: one long long, number of blocks in the pool.
  * Workspace: 8 bytes per weight element (u and omega of every pool element are kept across the
  *   iterations), 4 bytes per block (the pool list) and 4 bytes per channel, plus a fixed header. */
+#define SOP_LLOYD_POOL_BY_ERROR 1
+#define SOP_LLOYD_UNIFORM_WEIGHTS 2
+#define SOP_LLOYD_POOL_THRESHOLD 4
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
-                  const float* block_cos_dev, long long pool_rank, const sop_atom* atoms, int n_atoms,
+                  const float* block_metric_dev, long long pool_rank, float pool_threshold, int flags,
+                  const sop_atom* atoms, int n_atoms,
                   int fmta_index, int iters, float* out_lut_dev, double* distortion_dev,
                   long long* pool_count_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
@@ -230,19 +247,22 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
  *     m = b-1-x-y metabits; word_sign_bits = 0: selector at bit b-1 (if m >= 1), magnitude above
  *     the remaining m-1 metabits.  Unused metabits are zero.
  *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten.
- *   block_cos_dev (may be NULL): [n_atoms x N_b] per-block cosines written by sop_pair_search for the
- *     same layer, alphabet, format and shift.  When every candidate of the choice has a row there
- *     (with use_sign, the negated variant of an atom is the atom of the alphabet with the same table
- *     and the opposite `negated`; from a search result it is the next atom), the winner of each block
- *     is read off these cosines and only the winner is encoded: the output is identical, the cost
- *     drops to one encode per block.  Otherwise the candidates are evaluated here. */
+ *   flags: SOP_PACK_SELECT_MSE (paragraph "Pair-search design axes", axis ii): the smallest block squared
+ *     error wins instead of the largest block cosine, ties keep the earlier candidate.
+ *   block_metric_dev (may be NULL): [n_atoms x N_b] per-block cosines (with SOP_PACK_SELECT_MSE: per-block
+ *     errors) written by sop_pair_search for the same layer, alphabet, format and shift.  When every
+ *     candidate of the choice has a row there (with use_sign, the negated variant of an atom is the atom
+ *     of the alphabet with the same table and the opposite `negated`; from a search result it is the next
+ *     atom), the winner of each block is read off these values and only the winner is encoded: the output
+ *     is identical, the cost drops to one encode per block.  Otherwise the candidates are evaluated here. */
 #define SOP_NO_ATOM (-2)
 #define SOP_PAIR_FROM_RESULT (-1)
+#define SOP_PACK_SELECT_MSE 1
 int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
              const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
              unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
              int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
-             unsigned char* words_dev, long long* counts_dev, const float* block_cos_dev, void* stream);
+             unsigned char* words_dev, long long* counts_dev, const float* block_metric_dev, int flags, void* stream);
 
 #ifdef __cplusplus
 }

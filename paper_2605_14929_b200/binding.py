@@ -21,6 +21,9 @@ NO_ATOM = -2
 MAX_ATOMS = 16
 ALL_ATOMS = 0xFFFFFFFF
 SEARCH_SINGLES_ONLY = 1
+SEARCH_SELECT_MSE = 2
+LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD = 1, 2, 4
+PACK_SELECT_MSE = 1
 MAX_ENTRIES = 32
 
 
@@ -175,12 +178,14 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
                     k_mode: int = K_AUTO, dd_lut: Optional[torch.Tensor] = None, dd_mask: int = 0,
                     block_cos: Optional[torch.Tensor] = None, block_sse: Optional[torch.Tensor] = None,
                     stream=None, g: int = 16, eval_mask: int = ALL_ATOMS, load_mask: int = 0,
-                    singles_only: bool = False, prev_result: Optional[torch.Tensor] = None) -> None:
+                    singles_only: bool = False, prev_result: Optional[torch.Tensor] = None,
+                    select_mse: bool = False) -> None:
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_pair_search(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
                                  make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), C.c_uint(eval_mask),
-                                 C.c_uint(load_mask), SEARCH_SINGLES_ONLY if singles_only else 0, _ptr(prev_result),
+                                 C.c_uint(load_mask),
+                                 (SEARCH_SINGLES_ONLY if singles_only else 0) | (SEARCH_SELECT_MSE if select_mse else 0), _ptr(prev_result),
                                  _ptr(pair_table),
                                  _ptr(signed_table), _ptr(result), _ptr(block_cos), _ptr(block_sse), _ptr(workspace),
                                  C.c_size_t(workspace.numel()), _stream(stream)), "sop_pair_search")
@@ -189,11 +194,18 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
 def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_cos: torch.Tensor, pool_rank: int,
                   iters: int, out_lut: torch.Tensor, distortion: torch.Tensor, pool_count: torch.Tensor,
                   workspace: torch.Tensor, k_mode: int = K_FROM_RESULT, search_result: Optional[torch.Tensor] = None,
-                  fmta_index: int = FMTA_FROM_RESULT, stream=None, g: int = 16) -> None:
+                  fmta_index: int = FMTA_FROM_RESULT, stream=None, g: int = 16, pool_by_error: bool = False,
+                  uniform_weights: bool = False, pool_threshold: Optional[float] = None) -> None:
+    """``block_cos`` is the per-block metric that ranks the blocks: cosines, or errors with ``pool_by_error``.
+    A ``pool_threshold`` replaces the rank."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_dd4_lloyd(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
-                               _ptr(search_result), _ptr(block_cos), _ll(pool_rank), make_atoms(atoms), len(atoms),
+                               _ptr(search_result), _ptr(block_cos), _ll(pool_rank),
+                               C.c_float(0.0 if pool_threshold is None else pool_threshold),
+                               (LLOYD_POOL_BY_ERROR if pool_by_error else 0) | (LLOYD_UNIFORM_WEIGHTS if uniform_weights else 0)
+                               | (LLOYD_POOL_THRESHOLD if pool_threshold is not None else 0),
+                               make_atoms(atoms), len(atoms),
                                fmta_index, iters, _ptr(out_lut), _ptr(distortion), _ptr(pool_count), _ptr(workspace),
                                C.c_size_t(workspace.numel()), _stream(stream)), "sop_dd4_lloyd")
 
@@ -202,13 +214,15 @@ def sop_pack(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes: torc
              index_a: int = PAIR_FROM_RESULT, index_b: int = PAIR_FROM_RESULT, k_mode: int = K_FROM_RESULT,
              search_result: Optional[torch.Tensor] = None, use_sign: int = 0, container_bits: int = 8,
              word_sign_bits: int = 0, counts: Optional[torch.Tensor] = None, dd_lut: Optional[torch.Tensor] = None,
-             dd_mask: int = 0, stream=None, g: int = 16, block_cos: Optional[torch.Tensor] = None) -> None:
+             dd_mask: int = 0, stream=None, g: int = 16, block_cos: Optional[torch.Tensor] = None,
+             select_mse: bool = False) -> None:
+    """``block_cos``: per-block cosines of a sweep, or with ``select_mse`` its per-block errors."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_pack(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)),
                           make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), index_a, index_b, k_mode,
                           _ptr(search_result), use_sign, container_bits, word_sign_bits, _ptr(codes), _ptr(words),
-                          _ptr(counts), _ptr(block_cos), _stream(stream)), "sop_pack")
+                          _ptr(counts), _ptr(block_cos), PACK_SELECT_MSE if select_mse else 0, _stream(stream)), "sop_pack")
 
 
 def profile_enable(on: bool) -> None:

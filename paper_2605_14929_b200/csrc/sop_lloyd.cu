@@ -60,14 +60,13 @@ struct LloydWs {
   unsigned long long accN[SOP_MAX_ENTRIES];
   long long accS[SOP_MAX_ENTRIES];
   double accD;
-  float tau;         // pool threshold on the block cosine
+  unsigned tau_key;  // pool threshold as a ranking key: the pool is every block whose key is not above it
   float cmax;
   int k;
   int fmta;
   unsigned done;         // CTAs of the running iteration that have added their sums
   unsigned list_count;   // blocks appended to the pool list
   int pad;
-  long long pool_count;
   // the current codebook, rewritten by whoever changes it (set-up, then each update)
   IterDesc desc;
   // per cell, over the whole pool (filled once by pool_cache_kernel)
@@ -83,6 +82,8 @@ struct LloydArgs {
   long long M, K, ldw, nbk, NB;
   long long pool_rank;
   int k_mode, fmta_index, n_atoms;
+  int flags;                  // SOP_LLOYD_*
+  float pool_threshold;       // with SOP_LLOYD_POOL_THRESHOLD
   float* omega;               // workspace: K floats, c / max(c)
   unsigned* pool_idx;         // workspace: NB words, indices of the pool blocks
   uint2* cache;               // workspace: pairs (u, omega) as bit patterns, tiles of TILE_ELEMS sorted by cell
@@ -105,6 +106,12 @@ static size_t lloyd_ws_bytes(long long M, long long K) {
 __device__ __forceinline__ unsigned cos_key(float x) {
   const unsigned b = __float_as_uint(__fadd_rn(x, 0.0f));   // -0 -> +0
   return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+// Ranking key of a block: ascending key = worst block first.  By cosine the worst is the smallest value,
+// by error (SOP_LLOYD_POOL_BY_ERROR) the largest.
+__device__ __forceinline__ unsigned pool_key(float x, int flags) {
+  const unsigned k = cos_key(x);
+  return (flags & SOP_LLOYD_POOL_BY_ERROR) ? ~k : k;
 }
 
 __device__ __forceinline__ int resolve_fmta(const LloydArgs& a, const sop_search_result* res) {
@@ -175,7 +182,7 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
   __syncthreads();
   const float* row = a.cosrow_base + (size_t)resolve_fmta(a, res) * a.NB;
   for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += (long long)gridDim.x * LTB) {
-    const unsigned key = cos_key(__ldg(row + i));
+    const unsigned key = pool_key(__ldg(row + i), a.flags);
     if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
     else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&sh[(key >> 10) & 2047u], 1u); }
     else { if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u); }
@@ -209,10 +216,11 @@ __device__ void lloyd_publish_desc(LloydWs* ws, const float* s_lut, int ne) {
 }
 
 __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
-                                                               LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
-  unsigned prefix, cnt;
-  long long rank, below;
-  derive_prefix(ws, a.pool_rank, 3, &prefix, &rank, &below, &cnt);
+                                                               LloydWs* __restrict__ ws) {
+  unsigned prefix = 0, cnt = 0;
+  long long rank = 0, below = 0;
+  if (a.flags & SOP_LLOYD_POOL_THRESHOLD) prefix = pool_key(a.pool_threshold, a.flags);   // the caller fixes the threshold
+  else derive_prefix(ws, a.pool_rank, 3, &prefix, &rank, &below, &cnt);
   __shared__ float red[SETUP_TB / 32];
   __shared__ float s_cmax;
   __shared__ float s_lut[SOP_MAX_ENTRIES];
@@ -230,15 +238,11 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   __syncthreads();
   const float cmax = s_cmax;
   for (long long i = threadIdx.x; i < a.K; i += SETUP_TB) {
-    const float om = cmax > 0.0f ? __fdiv_rn(__ldg(a.c + i), cmax) : 0.0f;
+    const float om = (a.flags & SOP_LLOYD_UNIFORM_WEIGHTS) ? 1.0f : (cmax > 0.0f ? __fdiv_rn(__ldg(a.c + i), cmax) : 0.0f);
     a.omega[i] = om;
   }
   if (threadIdx.x == 0) {
-    const unsigned key = prefix;   // full 32-bit key after three passes
-    const unsigned b = key ^ ((key >> 31) ? 0x80000000u : 0xFFFFFFFFu);
-    ws->tau = __uint_as_float(b);
-    ws->pool_count = below + cnt;
-    *pool_count_out = below + cnt;
+    ws->tau_key = prefix;          // full 32-bit key after three passes (or the key of the given threshold)
     ws->cmax = cmax;
     const int f = resolve_fmta(a, res);
     ws->fmta = f;
@@ -271,14 +275,14 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
 __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __restrict__ ws) {
   __shared__ unsigned s_cnt[LTB / 32];
   __shared__ unsigned s_base;
-  const float tau = ws->tau;
+  const unsigned tau_key = ws->tau_key;
   const float* row = a.cosrow_base + (size_t)ws->fmta * a.NB;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long stride = (long long)gridDim.x * LTB;
   const long long n_round = (a.NB + stride - 1) / stride;
   long long i = (long long)blockIdx.x * LTB + threadIdx.x;
   for (long long r = 0; r < n_round; ++r, i += stride) {
-    const bool in = i < a.NB && __ldg(row + i) <= tau;
+    const bool in = i < a.NB && pool_key(__ldg(row + i), a.flags) <= tau_key;
     const unsigned bal = __ballot_sync(0xFFFFFFFFu, in);
     if (lane == 0) s_cnt[warp] = (unsigned)__popc(bal);
     __syncthreads();
@@ -363,7 +367,7 @@ __device__ void spill_cells(unsigned (*cL)[SORT_ROWS], LloydWs* ws) {
   }
 }
 
-__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws) {
+__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
   __shared__ unsigned hist[SORT_ROWS + 3];
   __shared__ unsigned warp_tot[LTB / 32];
   extern __shared__ __align__(16) uint2 stage[];                  // TILE_ELEMS pairs (dynamic: the kernel needs 60 KB in all)
@@ -377,6 +381,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
   const unsigned count = ws->list_count;
   const unsigned n_tiles = (count + LTB - 1) / LTB;
   const int k = ws->k;
+  if (blockIdx.x == 0 && tid == 0) *pool_count_out = (long long)count;   // the list is complete: its length is the pool size
   for (unsigned tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     for (int i = tid; i < SORT_ROWS + 3; i += LTB) hist[i] = 0;
     __syncthreads();
@@ -688,19 +693,23 @@ int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes) {
 
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
-                  const float* block_cos_dev, long long pool_rank, const sop_atom* atoms, int n_atoms,
+                  const float* block_metric_dev, long long pool_rank, float pool_threshold, int flags,
+                  const sop_atom* atoms, int n_atoms,
                   int fmta_index, int iters, float* out_lut_dev, double* distortion_dev,
                   long long* pool_count_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
   using namespace sop;
   int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
   if (rc) return rc;
-  if (!block_cos_dev || !out_lut_dev || !distortion_dev || !pool_count_dev) return SOP_ERR_NULL;
+  if (!block_metric_dev || !out_lut_dev || !distortion_dev || !pool_count_dev) return SOP_ERR_NULL;
+  if (flags & ~(SOP_LLOYD_POOL_BY_ERROR | SOP_LLOYD_UNIFORM_WEIGHTS | SOP_LLOYD_POOL_THRESHOLD)) return SOP_ERR_RANGE;
+  const bool by_threshold = (flags & SOP_LLOYD_POOL_THRESHOLD) != 0;
+  if (by_threshold && !(pool_threshold == pool_threshold)) return SOP_ERR_RANGE;   // NaN orders nothing
   FmtDev F;
   if ((rc = validate_fmt(fmt, &F))) return rc;
   AtomsDev A;
   if ((rc = validate_atoms(atoms, n_atoms, 0u, nullptr, &A))) return rc;
   const long long NB = M * (K / SOP_G);
-  if (pool_rank < 1 || pool_rank > NB || iters < 0 || iters > 64) return SOP_ERR_RANGE;
+  if ((!by_threshold && (pool_rank < 1 || pool_rank > NB)) || iters < 0 || iters > 64) return SOP_ERR_RANGE;
   if (k_mode != SOP_K_FROM_RESULT && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
   if ((k_mode == SOP_K_FROM_RESULT || fmta_index == SOP_FMTA_FROM_RESULT) && !search_dev) return SOP_ERR_NULL;
   if (fmta_index != SOP_FMTA_FROM_RESULT && (fmta_index < 0 || fmta_index >= n_atoms)) return SOP_ERR_RANGE;
@@ -712,9 +721,10 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
 
   unsigned char* wsb = (unsigned char*)workspace_dev;
   LloydArgs a;
-  a.W = (const uint16_t*)W_dev; a.c = c_dev; a.cosrow_base = block_cos_dev;
+  a.W = (const uint16_t*)W_dev; a.c = c_dev; a.cosrow_base = block_metric_dev;
   a.M = M; a.K = K; a.ldw = ldw; a.nbk = K / SOP_G; a.NB = NB; a.pool_rank = pool_rank;
   a.k_mode = k_mode; a.fmta_index = fmta_index; a.n_atoms = n_atoms;
+  a.flags = flags; a.pool_threshold = pool_threshold;
   a.omega = (float*)(wsb + lloyd_off_omega());
   a.pool_idx = (unsigned*)(wsb + lloyd_off_idx(K));
   a.cache = (uint2*)(wsb + lloyd_off_cache(M, K));
@@ -726,11 +736,13 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   long long sg = (NB + LTB * 8 - 1) / (LTB * 8);
   if (sg > sms * 4) sg = sms * 4;
   if (sg < 1) sg = 1;
-  select_kernel<0><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
-  select_kernel<1><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
-  select_kernel<2><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
-  SOP_CUDA_TRY(cudaGetLastError());
-  lloyd_setup_kernel<<<1, SETUP_TB, 0, st>>>(a, A, search_dev, ws, pool_count_dev);
+  if (!by_threshold) {     // radix select of the pool_rank-th worst block (three passes over the ranking keys)
+    select_kernel<0><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
+    select_kernel<1><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
+    select_kernel<2><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
+    SOP_CUDA_TRY(cudaGetLastError());
+  }
+  lloyd_setup_kernel<<<1, SETUP_TB, 0, st>>>(a, A, search_dev, ws);
   SOP_CUDA_TRY(cudaGetLastError());
   pool_list_kernel<<<(int)sg, LTB, 0, st>>>(a, ws);
   SOP_CUDA_TRY(cudaGetLastError());
@@ -745,7 +757,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
       SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
       attr_set = true;
     }
-    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws);
+    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev);
     SOP_CUDA_TRY(cudaGetLastError());
   }
   long long grid = ((NB + LTB - 1) / LTB + LTB / 32 - 1) / (LTB / 32);   // one warp per cache tile

@@ -19,7 +19,8 @@ struct PackArgs {
   unsigned char* codes;
   unsigned* words;       // zeroed before the kernel; filled with atomicOr
   unsigned long long* counts;
-  const float* block_cos;   // optional [n_atoms x NB]: per-block cosines of an earlier sweep
+  const float* block_cos;   // optional [n_atoms x NB]: per-block cosines (or errors, with select_err) of an earlier sweep
+  int select_err;           // 1: the smallest block error wins instead of the largest block cosine
   int cos_neg_a, cos_neg_b; // rows of the negated variants of index_a / index_b (-1: unknown, evaluate instead)
 };
 
@@ -27,9 +28,10 @@ struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
 // The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
-template <bool WANT_COS, int KIND>
+// METRIC: 0 = codes only, 1 = also the block cosine, 2 = also the block squared error (in cos_out).
+template <int METRIC, int KIND>
 __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
-                                                const float* __restrict__ lutv, int neg, float rcp,
+                                                const float* __restrict__ lutv, int neg, float rcp, float s_hat,
                                                 float& cos_out, uint32_t (&code4)[4]) {
   float qn[4], qd[4], qw[4];
 #pragma unroll
@@ -53,29 +55,32 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
         code = fp_code<SOP_KIND_FP_E4M3>(q);
       }
       packed |= code << (8 * r);
-      if (WANT_COS) {
+      if (METRIC == 1) {
         const float cw = __fmul_rn(c[i], w[i]);
         const float cq = __fmul_rn(c[i], q);
         aw = __fmaf_rn(cw, w[i], aw);
         ad = __fmaf_rn(cq, w[i], ad);
         an = __fmaf_rn(cq, q, an);
+      } else if (METRIC == 2) {
+        const float e = __fmaf_rn(-s_hat, q, w[i]);     // w - s q with one rounding, as the sweep forms it
+        an = __fmaf_rn(e, e, an);
       }
     }
     qn[h] = an; qd[h] = ad; qw[h] = aw;
     code4[h] = packed;
   }
-  cos_out = WANT_COS ? block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd)) : 0.0f;
+  cos_out = METRIC == 1 ? block_cosine(quad_tree(qw), quad_tree(qn), quad_tree(qd)) : (METRIC == 2 ? quad_tree(qn) : 0.0f);
 }
 
 // the quantiser kind is decided once per block, outside the element loops: a kind test inside them lets
 // the compiler hoist the FP-grid arithmetic into the table path
-template <bool WANT_COS>
+template <int METRIC>
 __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
-                                                const float* __restrict__ lutv, int kind, int neg, float rcp,
+                                                const float* __restrict__ lutv, int kind, int neg, float rcp, float s_hat,
                                                 float& cos_out, uint32_t (&code4)[4]) {
-  if (kind == SOP_KIND_LUT) eval_block_kind<WANT_COS, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, cos_out, code4);
-  else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<WANT_COS, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, cos_out, code4);
-  else eval_block_kind<WANT_COS, SOP_KIND_FP_E4M3>(w, c, tau, lutv, neg, rcp, cos_out, code4);
+  if (kind == SOP_KIND_LUT) eval_block_kind<METRIC, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+  else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<METRIC, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+  else eval_block_kind<METRIC, SOP_KIND_FP_E4M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
 }
 
 // USE_COS: the winner of each block is read off the per-block cosines of a sweep and only it is encoded
@@ -156,7 +161,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
       for (int t = 0; t < nb; ++t)
         for (int sg = 0; sg < n_sign; ++sg) {
           const float cs = __ldg(a.block_cos + (size_t)s_row[2 * t + sg] * a.NB + blk);
-          if (pick < 0 || cs > best_cos) { best_cos = cs; pick = 2 * t + sg; }
+          if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) { best_cos = cs; pick = 2 * t + sg; }
         }
       const int t = pick >> 1, sg = pick & 1;
       const PackCand cd = base[t];
@@ -171,7 +176,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
       }
       const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
       float unused;
-      eval_block_regs<false>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, unused, best4);
+      eval_block_regs<0>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, unused, best4);
     } else {
       for (int t = 0; t < nb; ++t) {
         const PackCand cd = base[t];
@@ -189,8 +194,9 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
         for (int sg = 0; sg < n_sign; ++sg) {
           float cs;
           uint32_t c4[4];
-          eval_block_regs<true>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, cs, c4);
-          if (pick < 0 || cs > best_cos) {
+          if (a.select_err) eval_block_regs<2>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4);
+          else eval_block_regs<1>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4);
+          if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) {
             best_cos = cs; best_scode = sc; pick = 2 * t + sg;
 #pragma unroll
             for (int h = 0; h < 4; ++h) best4[h] = c4[h];
@@ -265,8 +271,10 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
              const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev,
              unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
              int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
-             unsigned char* words_dev, long long* counts_dev, const float* block_cos_dev, void* stream) {
+             unsigned char* words_dev, long long* counts_dev, const float* block_metric_dev, int flags, void* stream) {
   using namespace sop;
+  const float* block_cos_dev = block_metric_dev;
+  if (flags & ~SOP_PACK_SELECT_MSE) return SOP_ERR_RANGE;
   int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
   if (rc) return rc;
   if (!codes_dev || !words_dev) return SOP_ERR_NULL;
@@ -312,6 +320,7 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   a.container_bits = container_bits; a.word_sign_bits = word_sign_bits; a.meta_bits = meta;
   a.codes = codes_dev; a.words = (unsigned*)words_dev; a.counts = (unsigned long long*)counts_dev;
   a.block_cos = block_cos_dev;
+  a.select_err = (flags & SOP_PACK_SELECT_MSE) ? 1 : 0;
   a.cos_neg_a = a.cos_neg_b = -1;
   if (block_cos_dev && use_sign && !from_result) {
     // row of the negated variant of an explicitly given atom: same table and scale reference, opposite sign

@@ -354,6 +354,9 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
                               Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
                               const int* cls_k, float wmax);
 
+// SEL_ERR: the per-block reassignment takes the smaller block error instead of the larger block cosine
+// (paragraph "Pair-search design axes", axis ii); ties keep the earlier candidate either way.
+template <bool SEL_ERR>
 __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, WsHeader* __restrict__ hdr,
                                                       Partial* __restrict__ partials, float* __restrict__ block_cos,
                                                       float* __restrict__ block_sse, sop_pair_stat* __restrict__ pair_table,
@@ -565,7 +568,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       for (int bi = 0; bi < P.n_bases; ++bi) {
         const int a = P.base_atom[bi];
         const float2 vp = my[a * HBP], vn = my[(a + 1) * HBP];
-        const bool neg = vn.x > vp.x;
+        const bool neg = SEL_ERR ? vn.y < vp.y : vn.x > vp.x;
         my[(P.n_atoms + bi) * HBP] = make_float2(neg ? vn.x : vp.x, neg ? -vn.y : vp.y);
       }
       half_barrier(half);
@@ -584,7 +587,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const float2 va = pa[k], vb = pb[k];
-          const bool mu = vb.x > va.x;
+          const bool mu = SEL_ERR ? fabsf(vb.y) < fabsf(va.y) : vb.x > va.x;
           const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
           acc_n1 += mu ? 1 : 0;
           acc_nneg += (int)(__float_as_uint(se_) >> 31);       // a negated winner of a signed column (error stored negative)
@@ -596,7 +599,7 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
       float cg = 0.0f, ce = 0.0f;
       for (; b < hi; ++b, ++pa, ++pb) {
         const float2 va = pa[0], vb = pb[0];
-        const bool mu = vb.x > va.x;
+        const bool mu = SEL_ERR ? fabsf(vb.y) < fabsf(va.y) : vb.x > va.x;
         const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
         acc_n1 += mu ? 1 : 0;
         acc_nneg += (int)(__float_as_uint(se_) >> 31);
@@ -925,7 +928,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   eval_mask &= all;
   if ((load_mask & ~all) || (load_mask & eval_mask) || !(eval_mask | load_mask)) return SOP_ERR_ALPHABET;
   if (load_mask && (!block_cos_dev || !block_sse_dev)) return SOP_ERR_NULL;
-  if (flags & ~SOP_SEARCH_SINGLES_ONLY) return SOP_ERR_RANGE;
+  if (flags & ~(SOP_SEARCH_SINGLES_ONLY | SOP_SEARCH_SELECT_MSE)) return SOP_ERR_RANGE;
   Plan P;
   if ((rc = build_plan(A, F, k_from_result ? 0 : k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, &P))) return rc;
   P.k_from_result = k_from_result ? 1 : 0;
@@ -960,7 +963,8 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if (smem > SMEM_MAX) return SOP_ERR_ALPHABET;
   static size_t smem_set = 0;
   if (smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
     smem_set = SMEM_MAX;
   }
   // persistent grid: one CTA per SM, fewer when the layer is small; at least enough threads for one row
@@ -970,8 +974,12 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if (grid < min_grid) grid = min_grid;
   if (grid > MAX_GRID) return SOP_ERR_SHAPE;
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
-  sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev, signed_table_dev,
-                                            result_dev, prev_result_dev);
+  if (flags & SOP_SEARCH_SELECT_MSE)
+    sweep_kernel<true><<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev,
+                                                    signed_table_dev, result_dev, prev_result_dev);
+  else
+    sweep_kernel<false><<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev,
+                                                     signed_table_dev, result_dev, prev_result_dev);
   SOP_CUDA_TRY(cudaGetLastError());
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
   return SOP_OK;

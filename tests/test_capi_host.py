@@ -86,7 +86,7 @@ def test_pair_search_rejects_bad_arguments(lib):
     assert _search(lib, emask=0, lmask=4, bc=FAKE) == -4   # load bit beyond the alphabet
     atoms2 = I.alphabet(["NF4"])
     assert _search(lib, atoms=atoms2, emask=1, lmask=2) == -1   # loading needs the per-block arrays
-    assert _search(lib, flags=2) == -7
+    assert _search(lib, flags=4) == -7
     assert _search(lib, k=B.K_FROM_RESULT) == -1       # shifts from an earlier result need that result
     assert _search(lib, k=B.K_FROM_RESULT, prev=C.c_void_p(0x20000)) == -7   # ... and a loaded candidate in every class
 
@@ -103,16 +103,20 @@ def test_other_entry_points_reject_bad_arguments(lib):
     atoms = I.alphabet(["NF4", "SH4"])
     arr = B.make_atoms(atoms)
 
-    def lloyd(rank=1, iters=8, k=0, fmta=0, res=None):
-        return lib.sop_dd4_lloyd(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, k, res, FAKE, ll(rank), arr, len(atoms), fmta,
-                                 iters, FAKE, FAKE, FAKE, FAKE, C.c_size_t(1 << 20), None)
+    def lloyd(rank=1, iters=8, k=0, fmta=0, res=None, flags=0, thr=0.0):
+        return lib.sop_dd4_lloyd(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, k, res, FAKE, ll(rank), C.c_float(thr), flags, arr,
+                                 len(atoms), fmta, iters, FAKE, FAKE, FAKE, FAKE, C.c_size_t(1 << 20), None)
     assert lloyd(rank=0) == -7 and lloyd(rank=17) == -7 and lloyd(iters=65) == -7 and lloyd(k=99) == -7
+    assert lloyd(flags=8) == -7                                           # unknown flag
+    assert lloyd(flags=B.LLOYD_POOL_THRESHOLD, thr=float("nan")) == -7    # a NaN threshold orders nothing
+    assert lloyd(rank=0, flags=B.LLOYD_POOL_THRESHOLD, iters=65) == -7    # the rank is ignored, the rest is still checked
     assert lloyd(fmta=9) == -7
     assert lloyd(k=B.K_FROM_RESULT) == -1 and lloyd(fmta=B.FMTA_FROM_RESULT) == -1
 
-    def pack(ia=0, ib=2, k=0, sign=0, b=12, wsb=0, res=None, f=fmt):
+    def pack(ia=0, ib=2, k=0, sign=0, b=12, wsb=0, res=None, f=fmt, flags=0):
         return lib.sop_pack(FAKE, ll(4), ll(64), ll(64), FAKE, 16, f, arr, len(atoms), None, C.c_uint(0), ia, ib, k, res,
-                            sign, b, wsb, FAKE, FAKE, None, None, None)
+                            sign, b, wsb, FAKE, FAKE, None, None, flags, None)
+    assert pack(flags=2) == -7
     assert pack(b=8) == -3                  # UE4M4 in 8 bits has no metabit for the selector
     assert pack(b=10) == -3
     assert pack(sign=1, wsb=0) == -3        # sign requested, word has no sign bit
