@@ -20,7 +20,8 @@ class _Fmt(C.Structure):
 
 class _Atom(C.Structure):
     _fields_ = [("n_bits", C.c_int), ("kind", C.c_int), ("negated", C.c_int), ("scope", C.c_int),
-                ("tmax", C.c_float), ("n_entries", C.c_int), ("lut", C.c_float * 32)]
+                ("tmax", C.c_float), ("n_entries", C.c_int), ("lut", C.c_float * 32),
+                ("grid_exp_bits", C.c_int), ("grid_man_bits", C.c_int), ("grid_bias", C.c_int), ("grid_neg_max", C.c_float)]
 
 
 class _PairStat(C.Structure):
@@ -42,6 +43,8 @@ def lib():
         _lib.osop_fp_quantize.restype = C.c_float
         _lib.osop_fp_grid_value.restype = C.c_double
         _lib.osop_layer_pot_scale.restype = C.c_float
+        _lib.osop_grid_quantize.restype = C.c_float
+        _lib.osop_grid_value.restype = C.c_double
     return _lib
 
 
@@ -57,6 +60,9 @@ def _atom(a) -> _Atom:
         s.n_entries = len(a.lut)
         for i, v in enumerate(a.lut):
             s.lut[i] = float(v)
+    g = getattr(a, "grid", None)
+    if g is not None:
+        s.grid_exp_bits, s.grid_man_bits, s.grid_bias, s.grid_neg_max = g
     return s
 
 
@@ -124,6 +130,17 @@ def fp_quantize(kind: int, u: float):
 
 def fp_grid_value(kind: int, code: int) -> float:
     return lib().osop_fp_grid_value(kind, code)
+
+
+def grid_quantize(atom, u: float):
+    """(value, code) of u on the parametric element grid of ``atom`` (kind 3)."""
+    code = C.c_int()
+    q = lib().osop_grid_quantize(C.byref(_atom(atom)), C.c_float(u), C.byref(code))
+    return q, code.value
+
+
+def grid_value(atom, j: int) -> float:
+    return lib().osop_grid_value(C.byref(_atom(atom)), j)
 
 
 def layer_pot_scale(wmax: float, tmax: float) -> float:

@@ -20,6 +20,8 @@
 //   sign-negated atoms as separate candidates ......... Section "Per-Layer Pair Search"
 //   data-derived DD-n by Lloyd updates + snap ......... Section "Per-Layer Pair Search" (steps 2-3, PO2 description)
 //   payload: 2n bytes of codes per g = 16 block ....... Section "Overview", item 4
+//   element grids by parameters (FP8/10/12 class, HIF7/HIF8) ... Section "Promotion Profiles";
+//                                                       paragraph "HIF7/HIF8 hardware rationale"
 //   design axes (i)-(iv): partition metric, reassignment metric, Lloyd weighting, pool definition
 //                                                       paragraph "Pair-search design axes"
 //
@@ -41,10 +43,14 @@ namespace {
 
 constexpr int G = 16;  // block size along K (the paper's default g = 16)
 
-enum { KIND_LUT = 0, KIND_FP_E2M3 = 1, KIND_FP_E4M3 = 2 };
+enum { KIND_LUT = 0, KIND_FP_E2M3 = 1, KIND_FP_E4M3 = 2, KIND_FP_GRID = 3 };
 
 struct ScaleFmt { int sign_bits, exp_bits, man_bits, bias, top_exp_reserved; };
-struct Atom { int n_bits, kind, negated, scope; float tmax; int n_entries; float lut[32]; };
+struct Atom {
+  int n_bits, kind, negated, scope; float tmax; int n_entries; float lut[32];
+  // KIND_FP_GRID only: a floating-point element grid given by its parameters (see grid_value)
+  int grid_exp_bits, grid_man_bits, grid_bias; float grid_neg_max;
+};
 struct PairStat { double acos, mse; long long n_sel1, n_neg; };
 
 inline float bf16_to_float(uint16_t h) {
@@ -188,6 +194,35 @@ float fp_quantize(int kind, float u, int* code_out) {
   return neg ? -q : q;
 }
 
+// A floating-point element grid by its parameters (promotion-profile formats: FP8 / FP10 / FP12 class
+// grids, Section "Promotion Profiles"; HIF7 / HIF8, paragraph "HIF7/HIF8 hardware rationale").
+// Magnitude number j = E * 2^y + M has the value (M / 2^y) 2^(1 - bias) for E = 0 and
+// (1 + M / 2^y) 2^(E - bias) otherwise: gradual underflow, then binades of 2^y steps.  The grid is the
+// magnitudes up to tmax on the positive side and up to neg_max (>= tmax) on the negative side: a
+// two's-complement coefficient reaches one step further below zero (HIF7: +120 / -128).  Rounding is to
+// the nearest grid value, ties to the even magnitude number, saturating.  The code is sign | j with the
+// sign above x + y bits (x = 0: a grid without a sign|E|M code; the sign then sits at bit n_bits - 1).
+double grid_value(const Atom& a, int j) {
+  const int y = a.grid_man_bits, E = j >> y, M = j & ((1 << y) - 1);
+  return E == 0 ? std::ldexp((double)M, 1 - a.grid_bias - y) : std::ldexp((double)((1 << y) + M), E - a.grid_bias - y);
+}
+
+float grid_quantize(const Atom& a, float u, int* code_out) {
+  const bool neg = std::signbit(u);
+  const double limit = neg ? (double)a.grid_neg_max : (double)a.tmax;
+  const double au = std::fabs((double)u);
+  int best = 0;
+  for (int j = 1; grid_value(a, j) <= limit; ++j) {
+    const double lo = grid_value(a, best), hi = grid_value(a, j);
+    if (2.0 * au > lo + hi) best = j;
+    else if (2.0 * au == lo + hi && (j & 1) == 0) best = j;   // tie: even magnitude number
+  }
+  const int sign_pos = a.grid_exp_bits > 0 ? a.grid_exp_bits + a.grid_man_bits : a.n_bits - 1;
+  if (code_out) *code_out = best | (neg ? 1 << sign_pos : 0);
+  const float q = (float)grid_value(a, best);
+  return neg ? -q : q;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Per-block evaluation of one candidate.
 // Order of the 16-term fp32 sums (paper silent): four quads of 4 consecutive elements, inside a
@@ -226,6 +261,8 @@ BlockEval eval_block(const float* w, const float* c, const Atom& a, const ScaleF
       const float uu = a.negated ? -u : u;
       r.code[i] = encode_lut(a.lut, a.n_entries, uu);
       r.q[i] = a.negated ? -a.lut[r.code[i]] : a.lut[r.code[i]];
+    } else if (a.kind == KIND_FP_GRID) {
+      r.q[i] = grid_quantize(a, u, &r.code[i]);
     } else {
       r.q[i] = fp_quantize(a.kind, u, &r.code[i]);
     }
@@ -301,6 +338,8 @@ int osop_encode_lut(const float* lut, int n, float u) { return encode_lut(lut, n
 float osop_fp_quantize(int kind, float u, int* code) { return fp_quantize(kind, u, code); }
 double osop_fp_grid_value(int kind, int code) { return fp_grid_value(kind, code); }
 float osop_layer_pot_scale(float wmax, float tmax) { return layer_pot_scale(wmax, tmax); }
+float osop_grid_quantize(const Atom* a, float u, int* code) { return grid_quantize(*a, u, code); }
+double osop_grid_value(const Atom* a, int j) { return grid_value(*a, j); }
 
 // one block under one candidate: cos, sse, s_hat, E, M, codes[16], q[16]
 void osop_eval_block(const float* w, const float* c, const Atom* a, const ScaleFmt* f, int k, float pot_scale,

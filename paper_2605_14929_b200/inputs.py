@@ -32,6 +32,7 @@ import torch
 KIND_LUT = 0
 KIND_FP_E2M3 = 1
 KIND_FP_E4M3 = 2
+KIND_FP_GRID = 3      # an element grid given by parameters: (exp_bits, man_bits, bias, largest negative magnitude)
 
 SCOPE_BLOCK = 16
 SCOPE_LAYER_POT = 0
@@ -95,6 +96,7 @@ class Atom:
     scope: int = SCOPE_BLOCK
     tmax: float = 1.0
     lut: Optional[np.ndarray] = None
+    grid: Optional[tuple] = None      # KIND_FP_GRID: (exp_bits, man_bits, bias, neg_max); exp_bits 0 = no sign|E|M code
 
     def negation(self) -> "Atom":
         assert self.kind == KIND_LUT
@@ -219,7 +221,43 @@ def fp_atom(name: str) -> Atom:
         return Atom(name, 8, KIND_FP_E4M3, 0, SCOPE_BLOCK, 448.0)
     if name == "E4M3^0":
         return Atom(name, 8, KIND_FP_E4M3, 0, SCOPE_LAYER_POT, 448.0)
+    if name in GRID_FORMATS or (name.endswith("^0") and name[:-2] in GRID_FORMATS):
+        return grid_atom(name)
     raise KeyError(name)
+
+
+def ieee_like_grid(x: int, y: int) -> tuple:
+    """(bias, largest value) of an ExMy element grid with bias 2^(x-1)-1 (at least 1) and the all-ones
+    exponent code left out: the convention under which the paper's E2M5 tops out at 3.94."""
+    bias = max(1, (1 << (x - 1)) - 1)
+    top = (1 << x) - 2
+    return bias, float((2.0 - 2.0 ** -y) * 2.0 ** (top - bias))
+
+
+# promotion-profile element grids beyond E2M3 / E4M3: name -> (n_bits, exp_bits, man_bits, bias, tmax, neg_max).
+# HIF7 / HIF8 are 5-bit two's-complement coefficients times 2^s (s up to 3 / 4): magnitudes 0..15 and then
+# 8..15 times 2^s, with -16 * 2^s reaching one step further on the negative side.
+def _grid_table():
+    t = {}
+    for nm, x, y in (("E3M4", 3, 4), ("E2M5", 2, 5), ("E5M2", 5, 2), ("E3M6", 3, 6), ("E4M5", 4, 5), ("E3M8", 3, 8),
+                     ("E4M7", 4, 7), ("E5M6e", 5, 6)):
+        bias, top = ieee_like_grid(x, y)
+        t[nm] = (1 + x + y, x, y, bias, top, top)
+    t["HIF7"] = (7, 0, 3, -2, 120.0, 128.0)
+    t["HIF8"] = (8, 0, 3, -2, 240.0, 256.0)
+    return t
+
+
+GRID_FORMATS = _grid_table()
+
+
+def grid_atom(name: str) -> Atom:
+    scope = SCOPE_BLOCK
+    base = name
+    if name.endswith("^0"):
+        scope, base = SCOPE_LAYER_POT, name[:-2]
+    n, x, y, bias, tmax, neg_max = GRID_FORMATS[base]
+    return Atom(name, n, KIND_FP_GRID, 0, scope, tmax, None, (x, y, bias, neg_max))
 
 
 def alphabet(names: Sequence[str], with_negations: bool = True, fp: Sequence[str] = ()) -> List[Atom]:
