@@ -47,7 +47,7 @@ enum {
   SOP_ERR_TOO_LARGE = -8   /* sop_channel_norms_static: ceil(T/64) * K exceeds the built-in scratch */
 };
 
-enum { SOP_KIND_LUT = 0, SOP_KIND_FP_E2M3 = 1, SOP_KIND_FP_E4M3 = 2 };
+enum { SOP_KIND_LUT = 0, SOP_KIND_FP_E2M3 = 1, SOP_KIND_FP_E4M3 = 2, SOP_KIND_FP_GRID = 3 };
 
 /* Scale word magnitude format ExMy with optional sign (Section "Scale Format and Metabit
  * Allocation", SwExMy).  bias is 2^(x-1)-1 in every format the paper names.  Rounding is to
@@ -66,6 +66,14 @@ typedef struct {
  * negated = 1 makes the candidate -(lut): it is evaluated by running the table on -u, so that
  * code_{-a}(-w) == code_a(w) exactly, ties included.
  * FP kinds (E2M3: 6-bit, largest 7.5; E4M3: 8-bit OCP, largest 448) ignore lut.
+ * SOP_KIND_FP_GRID: a floating-point element grid given by parameters (Section "Promotion Profiles":
+ *   FP8 / FP10 / FP12-class promotion formats; paragraph "HIF7/HIF8 hardware rationale").  Magnitude
+ *   number j = E * 2^y + M (y = grid_man_bits) has the value (M / 2^y) 2^(1 - grid_bias) for E = 0 and
+ *   (1 + M / 2^y) 2^(E - grid_bias) otherwise.  The grid is the magnitudes up to tmax on the positive
+ *   side and up to grid_neg_max >= tmax on the negative side (both must be grid values); rounding is to
+ *   nearest, ties to the even magnitude number, saturating.  HIF7 is y = 3, bias = -2, tmax = 120,
+ *   grid_neg_max = 128.  grid_exp_bits = x > 0 gives the element code sign | E | M with the sign above
+ *   x + y bits; x = 0 marks a grid without such a code (it can be swept but not packed).  lut is ignored.
  * scope = 16: per-block scale in the layer's scale format, s = max|w_block| / tmax
  * ("LUT-scale coupling": the scale is taken against max(LUT)).
  * scope = 0: one power-of-two scale per layer, 2^ceil(log2(max|W| / tmax)) (the "^0" suffix). */
@@ -77,6 +85,10 @@ typedef struct {
   float tmax;
   int n_entries;
   float lut[SOP_MAX_ENTRIES];
+  int grid_exp_bits;     /* SOP_KIND_FP_GRID only (zero otherwise): x in [0, 8] */
+  int grid_man_bits;     /* y in [0, 10] */
+  int grid_bias;         /* the smallest normal magnitude is 2^(1 - grid_bias) */
+  float grid_neg_max;    /* largest magnitude on the negative side, >= tmax */
 } sop_atom;
 
 /* Per-layer statistics of one candidate or one candidate pair. */

@@ -43,7 +43,8 @@ class ScaleFmt(C.Structure):
 
 class AtomStruct(C.Structure):
     _fields_ = [("n_bits", C.c_int), ("kind", C.c_int), ("negated", C.c_int), ("scope", C.c_int),
-                ("tmax", C.c_float), ("n_entries", C.c_int), ("lut", C.c_float * MAX_ENTRIES)]
+                ("tmax", C.c_float), ("n_entries", C.c_int), ("lut", C.c_float * MAX_ENTRIES),
+                ("grid_exp_bits", C.c_int), ("grid_man_bits", C.c_int), ("grid_bias", C.c_int), ("grid_neg_max", C.c_float)]
 
 
 class PairStat(C.Structure):
@@ -109,6 +110,9 @@ def make_atoms(atoms) -> C.Array:
         if a.lut is not None:
             for j, v in enumerate(a.lut):
                 s.lut[j] = float(v)
+        g = getattr(a, "grid", None)
+        if g is not None:
+            s.grid_exp_bits, s.grid_man_bits, s.grid_bias, s.grid_neg_max = g
     return arr
 
 

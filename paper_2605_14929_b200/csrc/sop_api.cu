@@ -77,6 +77,21 @@ int validate_atoms(const sop_atom* atoms, int n_atoms, unsigned dd_mask, const f
       if (a.n_bits != 6 || a.negated) return SOP_ERR_ALPHABET;
     } else if (a.kind == SOP_KIND_FP_E4M3) {
       if (a.n_bits != 8 || a.negated) return SOP_ERR_ALPHABET;
+    } else if (a.kind == SOP_KIND_FP_GRID) {
+      if (a.negated || a.n_bits < 2 || a.n_bits > 16) return SOP_ERR_ALPHABET;
+      if (a.grid_exp_bits < 0 || a.grid_exp_bits > 8 || a.grid_man_bits < 0 || a.grid_man_bits > 10) return SOP_ERR_ALPHABET;
+      if (a.grid_bias < -100 || a.grid_bias > 100) return SOP_ERR_ALPHABET;
+      if (a.grid_exp_bits && 1 + a.grid_exp_bits + a.grid_man_bits > a.n_bits) return SOP_ERR_ALPHABET;
+      if (!isfinite(a.grid_neg_max) || a.grid_neg_max < a.tmax) return SOP_ERR_ALPHABET;
+      // both ends must be values of the grid: a whole number of steps of their binade (or of the subnormal step)
+      const float ends[2] = {a.tmax, a.grid_neg_max};
+      for (int e = 0; e < 2; ++e) {
+        int ex = 0;
+        frexp((double)ends[e], &ex);                       // ends[e] = f * 2^ex, f in [1/2, 1)
+        const int binade = ex - 1 > 1 - a.grid_bias ? ex - 1 : 1 - a.grid_bias;
+        const double steps = ldexp((double)ends[e], a.grid_man_bits - binade);
+        if (steps != floor(steps)) return SOP_ERR_ALPHABET;
+      }
     } else {
       return SOP_ERR_ALPHABET;
     }
@@ -155,7 +170,7 @@ const char* sop_strerror(int code) {
 
 const char* sop_last_cuda_error(void) { return sop::g_cuda_error; }
 
-int sop_version(void) { return 101; }
+int sop_version(void) { return 102; }
 
 int sop_profile_enable(int on) {
   sop::g_profile = on != 0;

@@ -138,6 +138,29 @@ __device__ __forceinline__ float fp_quantize(float u) {
   return __uint_as_float(__float_as_uint(q) | (__float_as_uint(u) & 0x80000000u));
 }
 
+// Element grid given by parameters (SOP_KIND_FP_GRID): min_eb = biased fp32 exponent of the smallest normal
+// magnitude (127 + 1 - bias), sh = 23 - man_bits, saturation at vpos above zero and at vneg below.
+struct GridDev { int min_eb, sh; float vpos, vneg; };
+
+__device__ __forceinline__ float grid_quantize(float u, const GridDev g) {
+  const float au = fminf(fabsf(u), u < 0.0f ? g.vneg : g.vpos);
+  const int eb = (int)(__float_as_uint(au) >> 23);
+  const float magic = __uint_as_float((uint32_t)(max(eb, g.min_eb) + g.sh) << 23);
+  const float q = __fsub_rn(__fadd_rn(au, magic), magic);     // nearest multiple of the binade's step, ties to even
+  return __uint_as_float(__float_as_uint(q) | (__float_as_uint(u) & 0x80000000u));
+}
+
+// magnitude number E * 2^y + M of a value already on such a grid, the sign at bit sign_pos
+__device__ __forceinline__ uint32_t grid_code(float q, const GridDev g, int sign_pos) {
+  const uint32_t b = __float_as_uint(q);
+  const int y = 23 - g.sh;
+  const int eb = (int)((b >> 23) & 255u);
+  uint32_t mag;
+  if (eb < g.min_eb) mag = (uint32_t)__float2int_rn(__fmul_rn(fabsf(q), __uint_as_float((uint32_t)(127 + 127 - g.min_eb + y) << 23)));
+  else mag = ((uint32_t)(eb - g.min_eb + 1) << y) | ((b >> g.sh) & ((1u << y) - 1u));
+  return ((b >> 31) << sign_pos) | mag;
+}
+
 // bit pattern sign|E|M of a value already on the grid
 template <int KIND>
 __device__ __forceinline__ uint32_t fp_code(float q) {

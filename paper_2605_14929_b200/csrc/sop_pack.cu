@@ -24,7 +24,7 @@ struct PackArgs {
   int cos_neg_a, cos_neg_b; // rows of the negated variants of index_a / index_b (-1: unknown, evaluate instead)
 };
 
-struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
+struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; GridDev grid; int sign_pos; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
 // The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
@@ -32,7 +32,7 @@ struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; };
 template <int METRIC, int KIND>
 __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int neg, float rcp, float s_hat,
-                                                float& cos_out, uint32_t (&code4)[4]) {
+                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid = GridDev(), int sign_pos = 0) {
   float qn[4], qd[4], qw[4];
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
@@ -50,6 +50,9 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
       } else if (KIND == SOP_KIND_FP_E2M3) {
         q = fp_quantize<SOP_KIND_FP_E2M3>(u);
         code = fp_code<SOP_KIND_FP_E2M3>(q);
+      } else if (KIND == SOP_KIND_FP_GRID) {
+        q = grid_quantize(u, grid);
+        code = grid_code(q, grid, sign_pos);      // at most 8 bits: the host refuses wider grids here
       } else {
         q = fp_quantize<SOP_KIND_FP_E4M3>(u);
         code = fp_code<SOP_KIND_FP_E4M3>(q);
@@ -77,8 +80,9 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
 template <int METRIC>
 __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int kind, int neg, float rcp, float s_hat,
-                                                float& cos_out, uint32_t (&code4)[4]) {
+                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid, int sign_pos) {
   if (kind == SOP_KIND_LUT) eval_block_kind<METRIC, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+  else if (kind == SOP_KIND_FP_GRID) eval_block_kind<METRIC, SOP_KIND_FP_GRID>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4, grid, sign_pos);
   else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<METRIC, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
   else eval_block_kind<METRIC, SOP_KIND_FP_E4M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
 }
@@ -86,7 +90,7 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
 // USE_COS: the winner of each block is read off the per-block cosines of a sweep and only it is encoded
 // (no channel norms needed); otherwise every candidate of the choice is evaluated here.
 template <bool USE_COS>
-__global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
+__global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
   __shared__ float lutv[2][32], tau[2][32];
   __shared__ PackCand base[2];
   __shared__ int s_nb, s_nbits;
@@ -112,6 +116,9 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
       const sop_atom& at = A.atoms[idx];
       base[t].table = t; base[t].kind = at.kind; base[t].neg = at.negated; base[t].scope = at.scope; base[t].tmax = at.tmax;
       base[t].k = a.k_mode == SOP_K_FROM_RESULT ? res->k[idx] : a.k_mode;
+      base[t].grid.min_eb = 128 - at.grid_bias; base[t].grid.sh = 23 - at.grid_man_bits;
+      base[t].grid.vpos = at.tmax; base[t].grid.vneg = at.grid_neg_max;
+      base[t].sign_pos = at.grid_exp_bits + at.grid_man_bits;
       s_pot[t] = at.scope == 0 ? layer_pot_scale(wmax, at.tmax) : 0.0f;
       const bool dd = (A.dd_mask >> idx) & 1u;
       const int ne = at.kind == SOP_KIND_LUT ? at.n_entries : 2;
@@ -176,7 +183,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
       }
       const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
       float unused;
-      eval_block_regs<0>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, unused, best4);
+      eval_block_regs<0>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, unused, best4, cd.grid, cd.sign_pos);
     } else {
       for (int t = 0; t < nb; ++t) {
         const PackCand cd = base[t];
@@ -194,8 +201,8 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 2) pack_kernel(PackArgs a, 
         for (int sg = 0; sg < n_sign; ++sg) {
           float cs;
           uint32_t c4[4];
-          if (a.select_err) eval_block_regs<2>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4);
-          else eval_block_regs<1>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4);
+          if (a.select_err) eval_block_regs<2>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos);
+          else eval_block_regs<1>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos);
           if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) {
             best_cos = cs; best_scode = sc; pick = 2 * t + sg;
 #pragma unroll
@@ -300,6 +307,9 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   }
   const bool pair = index_b != SOP_NO_ATOM;
   if (pair && meta < 1) return SOP_ERR_FORMAT;     // the selector needs a metabit
+  // a parametric grid is packed as sign | E | M in at most 8 bits; wider grids and grids without such a code are swept only
+  if (!from_result && atoms[index_a].kind == SOP_KIND_FP_GRID &&
+      (atoms[index_a].grid_exp_bits < 1 || atoms[index_a].n_bits > 8)) return SOP_ERR_ALPHABET;
   if (k_mode == SOP_K_FROM_RESULT) { if (!search_dev) return SOP_ERR_NULL; }
   else if (k_mode < -64 || k_mode > 64) return SOP_ERR_RANGE;
   bool need_wmax = false;

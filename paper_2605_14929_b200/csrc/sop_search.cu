@@ -35,6 +35,7 @@ struct ClassDev {
   int n_mem;                             // candidates present in this call (evaluated or loaded)
   unsigned char mem[SOP_MAX_ATOMS];
   int k_src;                             // candidate whose shift an earlier result holds (k from result), or -1
+  GridDev grid;                          // kind SOP_KIND_FP_GRID: the grid's parameters
 };
 struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (i0 == i1: single); 1: signed (i0, i0+1, i1, i1+1)
 
@@ -248,9 +249,11 @@ __device__ __forceinline__ Metric eval_lut_cells(const unsigned char* __restrict
   return m;
 }
 
-// mode 0: table through binary search over the thresholds (any table); mode 1 / 2: E2M3 / E4M3 grid
+// mode 0: table through binary search over the thresholds (any table); mode 1 / 2: E2M3 / E4M3 grid;
+// mode 3: grid given by parameters
 template <int MODE, bool NEG>
-__device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, const float* __restrict__ lutv, const BlockRegs& B, float s_hat) {
+__device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, const float* __restrict__ lutv, const BlockRegs& B, float s_hat,
+                                               const GridDev grid = GridDev()) {
   float2 nq[2], dot[2], sse[2];
   nq[0] = nq[1] = dot[0] = dot[1] = sse[0] = sse[1] = make_float2(0.0f, 0.0f);
   const float sg = NEG ? s_hat : -s_hat;
@@ -262,9 +265,12 @@ __device__ __forceinline__ Metric eval_generic(const float* __restrict__ tau, co
       const int idx = 2 * i + p;
       const float ux = B.u[idx].x, uy = B.u[idx].y;
       float2 q;
-      if (MODE == 0) {
+      if constexpr (MODE == 0) {
         q.x = lutv[count_below(tau, NEG ? -ux : ux)];
         q.y = lutv[count_below(tau, NEG ? -uy : uy)];
+      } else if constexpr (MODE == SOP_KIND_FP_GRID) {
+        q.x = grid_quantize(ux, grid);
+        q.y = grid_quantize(uy, grid);
       } else {
         q.x = fp_quantize<MODE>(ux);
         q.y = fp_quantize<MODE>(uy);
@@ -546,6 +552,15 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
             if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
             if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
           }
+        } else if (C.kind == SOP_KIND_FP_GRID) {
+          for (int ci = 0; ci < C.n_cand; ++ci) {
+            const int a = C.cand[ci];
+            const Metric mt = eval_generic<SOP_KIND_FP_GRID, false>(nullptr, nullptr, B, s_hat, C.grid);
+            const float cosv = block_cosine(nw, mt.nq, mt.dot);
+            my[a * HBP] = make_float2(cosv, mt.sse);
+            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
+            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
+          }
         } else {
           for (int ci = 0; ci < C.n_cand; ++ci) {
             const int a = C.cand[ci];
@@ -772,13 +787,17 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mas
     if (!((present >> i) & 1u)) continue;
     int cl = -1;
     for (int c = 0; c < P->n_classes; ++c)
-      if (P->cls[c].scope == a.scope && P->cls[c].tmax == a.tmax && P->cls[c].kind == a.kind) cl = c;
+      if (P->cls[c].scope == a.scope && P->cls[c].tmax == a.tmax && P->cls[c].kind == a.kind &&
+          (a.kind != SOP_KIND_FP_GRID || (P->cls[c].grid.min_eb == 128 - a.grid_bias && P->cls[c].grid.sh == 23 - a.grid_man_bits &&
+                                          P->cls[c].grid.vneg == a.grid_neg_max))) cl = c;
     if (cl < 0) {
       if (P->n_classes == SOP_MAX_CLASSES) return SOP_ERR_ALPHABET;
       cl = P->n_classes++;
       P->cls[cl].scope = a.scope; P->cls[cl].tmax = a.tmax; P->cls[cl].kind = a.kind;
       P->cls[cl].auto_k = (k_mode == SOP_K_AUTO && a.scope != 0) ? 1 : 0;
       P->cls[cl].invh = 1.0f; P->cls[cl].c_half = 0;
+      P->cls[cl].grid.min_eb = 128 - a.grid_bias; P->cls[cl].grid.sh = 23 - a.grid_man_bits;
+      P->cls[cl].grid.vpos = a.tmax; P->cls[cl].grid.vneg = a.grid_neg_max;
     }
     ClassDev& C = P->cls[cl];
     C.mem[C.n_mem++] = (unsigned char)i;

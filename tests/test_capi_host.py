@@ -1,6 +1,7 @@
 """Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
 header declares, and rejects bad arguments on the host before anything is launched."""
 import ctypes as C
+import dataclasses
 import os
 import re
 
@@ -30,7 +31,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_layouts_match_header():
-    assert C.sizeof(B.AtomStruct) == 6 * 4 + 32 * 4
+    assert C.sizeof(B.AtomStruct) == 6 * 4 + 32 * 4 + 4 * 4
     assert C.sizeof(B.PairStat) == 32 and B.PAIR_DTYPE.itemsize == 32
     assert C.sizeof(B.SearchResult) == 16 * 4 + 5 * 4 + 4 + 8
     assert C.sizeof(B.ScaleFmt) == 20
@@ -123,3 +124,27 @@ def test_other_entry_points_reject_bad_arguments(lib):
     assert pack(ia=5) == -7 and pack(ib=7) == -7
     assert pack(ia=B.PAIR_FROM_RESULT) == -1
     assert pack(k=B.K_FROM_RESULT) == -1
+
+
+def test_grid_arguments_are_checked_on_the_host(lib):
+    FAKE = C.c_void_p(0x1000)
+    ll = C.c_longlong
+    fmt = C.byref(B.make_fmt(I.scale_format("UE4M4")))
+
+    def search(atom):
+        arr = B.make_atoms([atom])
+        return lib.sop_pair_search(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, 0, arr, 1, None, C.c_uint(0), C.c_uint(1), C.c_uint(0), 0,
+                                   None, FAKE, None, FAKE, None, None, None, C.c_size_t(0), None)
+
+    good = I.fp_atom("HIF7")
+    assert search(dataclasses.replace(good, tmax=121.0)) == -4                       # 121 is not a value of the grid
+    assert search(dataclasses.replace(good, grid=(0, 3, -2, 100.0))) == -4           # negative end below the positive one
+    assert search(dataclasses.replace(good, grid=(0, 11, -2, 128.0))) == -4          # too many mantissa bits
+    assert search(dataclasses.replace(good, negated=1)) == -4
+    assert search(good) == -5                                                          # passes the atom checks, stops at the workspace
+    # a grid without a sign|E|M code, or wider than 8 bits, is not packed
+    for atom in (I.fp_atom("HIF7"), I.fp_atom("E3M6")):
+        arr = B.make_atoms([atom])
+        rc = lib.sop_pack(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, arr, 1, None, C.c_uint(0), 0, B.NO_ATOM, 0, None, 0, 12, 0,
+                          C.c_void_p(0x1000), FAKE, None, None, 0, None)
+        assert rc == -4
