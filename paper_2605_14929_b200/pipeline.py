@@ -154,3 +154,68 @@ class LayerSweep:
             dd_lut=self.dd_lut.cpu().numpy(), distortion=self.distortion.cpu().numpy(),
             pool_count=int(self.pool_count.item()), codes=self.codes.cpu(), words=self.words.cpu(),
             counts=self.counts.cpu().numpy(), atoms=self.full_atoms)
+
+
+class LayerStream:
+    """Streams host-resident layers of one shape through a ``LayerSweep``.  While layer i is swept, the
+    weights and activations of layer i + 1 travel host -> device and the results of layer i - 1 travel
+    device -> host: two input slots, two output slots, three CUDA streams ordered by events.  The host
+    tensors must be pinned for the copies to overlap.
+
+        stream = LayerStream(sweep)
+        for i, (W_host, X_host) in enumerate(layers):
+            stream.submit(i, W_host, X_host)
+            if i:
+                consume(stream.collect(i - 1))
+        consume(stream.collect(len(layers) - 1))
+
+    ``collect(i)`` waits for layer i and returns pinned host tensors (pair_table, signed_table, result,
+    codes, words) that stay valid until ``submit(i + 2)``."""
+
+    OUT = ("pair_table", "signed_table", "result", "codes", "words")
+
+    def __init__(self, sweep: LayerSweep):
+        self.sw = sweep
+        d = sweep.dev
+        self.s_in, self.s_run, self.s_out = torch.cuda.Stream(d), torch.cuda.Stream(d), torch.cuda.Stream(d)
+        self.W = [torch.empty((sweep.M, sweep.K), dtype=torch.bfloat16, device=d) for _ in range(2)]
+        self.X = [torch.empty((sweep.T, sweep.K), dtype=torch.float32, device=d) for _ in range(2)]
+        self.dev_out = [{k: torch.empty_like(getattr(sweep, k)) for k in self.OUT} for _ in range(2)]
+        self.host_out = [{k: torch.empty(getattr(sweep, k).shape, dtype=getattr(sweep, k).dtype).pin_memory() for k in self.OUT}
+                         for _ in range(2)]
+        ev = lambda: [torch.cuda.Event() for _ in range(2)]
+        self.in_ready, self.in_free, self.out_ready, self.out_done = ev(), ev(), ev(), ev()
+        self.h2d_bytes = self.W[0].numel() * 2 + self.X[0].numel() * 4
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.dev_out[0].values())
+        self.before_run = None       # optional callable run on the compute stream before every sweep
+
+    def submit(self, i: int, W_host: torch.Tensor, X_host: torch.Tensor) -> None:
+        slot = i & 1
+        sw = self.sw
+        with torch.cuda.stream(self.s_in):
+            if i >= 2:
+                self.s_in.wait_event(self.in_free[slot])      # the sweep of layer i - 2 has read this slot
+            self.W[slot].copy_(W_host, non_blocking=True)
+            self.X[slot].copy_(X_host, non_blocking=True)
+            self.in_ready[slot].record(self.s_in)
+        with torch.cuda.stream(self.s_run):
+            self.s_run.wait_event(self.in_ready[slot])
+            if i >= 2:
+                self.s_run.wait_event(self.out_done[slot])    # the results of layer i - 2 have left this slot
+            if self.before_run is not None:
+                self.before_run()
+            sw.run(self.W[slot], self.X[slot], self.s_run)
+            self.in_free[slot].record(self.s_run)
+            for k in self.OUT:
+                self.dev_out[slot][k].copy_(getattr(sw, k), non_blocking=True)
+            self.out_ready[slot].record(self.s_run)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.out_ready[slot])
+            for k in self.OUT:
+                self.host_out[slot][k].copy_(self.dev_out[slot][k], non_blocking=True)
+            self.out_done[slot].record(self.s_out)
+
+    def collect(self, i: int) -> dict:
+        slot = i & 1
+        self.out_done[slot].synchronize()
+        return self.host_out[slot]

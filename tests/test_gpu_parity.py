@@ -357,3 +357,31 @@ def test_pipeline_matches_oracle(B, fmt_name, rom, fp, iters, shape):
     assert np.array_equal(got.codes.numpy().reshape(pk["codes"].shape), pk["codes"])
     assert np.array_equal(got.words.numpy()[:pk["words"].size], pk["words"])
     assert (int(got.counts[0]), int(got.counts[1])) == (pk["n_sel1"], pk["n_neg"])
+
+
+def test_layer_stream_returns_each_layers_own_results(B):
+    # three different layers through the overlapped host -> device -> host stream: every layer's results
+    # equal those of a plain run on that layer
+    from paper_2605_14929_b200.pipeline import LayerStream, LayerSweep
+    fmt = I.scale_format("S1E4M4")
+    M, K, T = 48, 512, 64
+    layers = [I.outlier_channel_layer(40 + i, M, K, T) for i in range(3)]
+    sw = LayerSweep(M, K, T, fmt, ["NF4", "SH4"], [], 4, device=dev())
+    want = []
+    for L in layers:
+        sw.run(L.W.to(dev()), L.X.to(dev()))
+        torch.cuda.synchronize()
+        want.append({k: getattr(sw, k).cpu().clone() for k in LayerStream.OUT})
+    ls = LayerStream(sw)
+    host = [(L.W.pin_memory(), L.X.pin_memory()) for L in layers]
+    got = []
+    for i, (Wh, Xh) in enumerate(host):
+        ls.submit(i, Wh, Xh)
+        if i:
+            got.append({k: v.clone() for k, v in ls.collect(i - 1).items()})
+    got.append({k: v.clone() for k, v in ls.collect(len(host) - 1).items()})
+    assert ls.h2d_bytes == M * K * 2 + T * K * 4
+    for i in range(3):
+        for k in LayerStream.OUT:
+            assert torch.equal(got[i][k], want[i][k]), (i, k)
+    assert not torch.equal(want[0]["codes"], want[1]["codes"])
