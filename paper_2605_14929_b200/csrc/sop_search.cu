@@ -655,60 +655,69 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
   }
 }
 
-// Block-wide argmax of (value, index) with ties to the smaller index; index -1 = nothing.  `red` holds
-// blockDim.x / 32 entries.  Every thread returns the winner's index.
-__device__ int block_argmax(double v, int idx, double* red_v, int* red_i) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+// One warp.  The defined entry of `tab` ([A x A]) with the largest acos, ties to the smallest index: among the
+// entries above the diagonal (diag = 0) or among the diagonal entries of the candidates in lut_mask (diag = 1).  -1: none.
+__device__ __noinline__ int warp_best(const sop_pair_stat* tab, int A, int diag, unsigned lut_mask) {
+  const int lane = threadIdx.x & 31;
+  int best = -1;
+  double bv = 0.0;
+#pragma unroll 1
+  for (int i = lane; i < A * A; i += 32) {
+    const int a = i / A, b = i - a * A;
+    const bool in = diag ? (b == a && ((lut_mask >> a) & 1u)) : b > a;
+    if (in && tab[i].n_sel1 >= 0 && (best < 0 || tab[i].acos > bv)) { best = i; bv = tab[i].acos; }
+  }
+#pragma unroll 1
   for (int o = 16; o; o >>= 1) {
-    const double ov = __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    const int oi = __shfl_xor_sync(0xFFFFFFFFu, idx, o);
-    if (oi >= 0 && (idx < 0 || ov > v || (ov == v && oi < idx))) { v = ov; idx = oi; }
+    const double ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+    const int oi = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+    if (oi >= 0 && (best < 0 || ov > bv || (ov == bv && oi < best))) { bv = ov; best = oi; }
   }
-  __syncthreads();
-  if (lane == 0) { red_v[warp] = v; red_i[warp] = idx; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < n_warps; ++w) {
-      const double ov = red_v[w];
-      const int oi = red_i[w];
-      if (oi >= 0 && (idx < 0 || ov > v || (ov == v && oi < idx))) { v = ov; idx = oi; }
-    }
-    red_i[0] = idx;
-  }
-  __syncthreads();
-  return red_i[0];
+  return best;
 }
 
 // Run by one whole CTA of TB threads.  Thread (slot, chunk) adds the partials of CTAs chunk, chunk + C,
-// ... in that order (C = TB / n_slots chunks, loads coalesced over the slots), the chunks are then added
-// in chunk order: the result depends only on the grid size, not on scheduling.  s_pair / s_sig
-// (n_atoms^2 entries each) and s_red (TB entries) are shared-memory staging.
+// ... in that order (C = min(TB / n_slots, ceil(grid / 4)) chunks, loads coalesced over the slots and issued four at a
+// time), the chunks are then added in chunk order: the result depends only on the grid size, not on
+// scheduling.  s_pair / s_sig (n_atoms^2 entries each) and s_red (TB entries) are shared-memory staging.
 __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const Partial* partials, sop_pair_stat* s_pair, sop_pair_stat* s_sig,
                               Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
                               const int* cls_k, float wmax) {
-  __shared__ double red_v[TB / 32];
-  __shared__ int red_i[TB / 32];
   const int A = P.n_atoms, tid = threadIdx.x, n_slots = P.n_slots;
   for (int i = tid; i < A * A; i += blockDim.x) {
     sop_pair_stat u; u.acos = 0.0; u.mse = 0.0; u.n_sel1 = -1; u.n_neg = -1;
     s_pair[i] = u;
     s_sig[i] = u;
   }
-  const int n_chunks = (int)blockDim.x / n_slots;
+  const int n_chunks = min((int)blockDim.x / n_slots, (grid + 3) / 4);   // at best one round of four loads per thread
   const int slot = tid % n_slots, chunk = tid / n_slots;
   if (chunk < n_chunks) {
     Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
-    for (int g = chunk; g < grid; g += n_chunks) {
-      const double2* q = reinterpret_cast<const double2*>(partials + (size_t)g * MAX_SLOTS + slot);
-      const double2 a = __ldcg(q);
-      const longlong2 b = __ldcg(reinterpret_cast<const longlong2*>(q + 1));
-      t.gap += a.x; t.sse += a.y; t.n1 += b.x; t.nneg += b.y;
+#pragma unroll 1
+    for (int g0 = chunk; g0 < grid; g0 += 4 * n_chunks) {
+      double2 a[4];
+      longlong2 b[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int g = g0 + u * n_chunks;
+        a[u] = make_double2(0.0, 0.0);
+        b[u] = make_longlong2(0, 0);
+        if (g < grid) {
+          const double2* q = reinterpret_cast<const double2*>(partials + (size_t)g * MAX_SLOTS + slot);
+          a[u] = __ldcg(q);
+          b[u] = __ldcg(reinterpret_cast<const longlong2*>(q + 1));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (g0 + u * n_chunks < grid) { t.gap += a[u].x; t.sse += a[u].y; t.n1 += b[u].x; t.nneg += b[u].y; }
     }
     s_red[tid] = t;
   }
   __syncthreads();
   if (tid < n_slots) {
     Partial t = s_red[tid];
+#pragma unroll 1
     for (int c = 1; c < n_chunks; ++c) {
       const Partial q = s_red[c * n_slots + tid];
       t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
@@ -730,23 +739,22 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
     const bool present = tid < A && (((P.eval_mask | P.load_mask) >> tid) & 1u);
     res->k[tid] = present ? cls_k[P.cand[tid].cls] : 0;
   }
-  // best two-codebook pair, best single LUT candidate, best signed pair: largest ACos, ties to the smallest (a, b)
-  const int a = tid / A, b = tid - a * A;
-  const bool in = tid < A * A;
-  int ip = -1, is = -1, isg = -1;
-  double vp = 0.0, vs = 0.0, vsg = 0.0;
-  if (in && b > a && s_pair[tid].n_sel1 >= 0) { ip = tid; vp = s_pair[tid].acos; }
-  if (in && b == a && P.cand[a].kind == SOP_KIND_LUT && s_pair[tid].n_sel1 >= 0) { is = tid; vs = s_pair[tid].acos; }
-  if (in && b > a && signed_table && s_sig[tid].n_sel1 >= 0) { isg = tid; vsg = s_sig[tid].acos; }
-  ip = block_argmax(vp, ip, red_v, red_i);
-  is = block_argmax(vs, is, red_v, red_i);
-  isg = block_argmax(vsg, isg, red_v, red_i);
-  if (tid == 0) {
-    res->layer_absmax = wmax;
-    res->reserved[0] = res->reserved[1] = 0;
-    res->best_a = ip >= 0 ? ip / A : -1; res->best_b = ip >= 0 ? ip % A : -1;
-    res->best_single = is >= 0 ? is / A : -1;
-    res->best_sa = isg >= 0 ? isg / A : -1; res->best_sb = isg >= 0 ? isg % A : -1;
+  // best two-codebook pair, best single LUT candidate, best signed pair: largest ACos, ties to the smallest
+  // (a, b).  One warp, one small routine called three times: this code runs once per launch, so its size
+  // (instruction fetches that miss) costs more than its arithmetic.
+  if (tid < 32) {
+    unsigned lut_mask = 0;
+    for (int a = 0; a < A; ++a) lut_mask |= P.cand[a].kind == SOP_KIND_LUT ? 1u << a : 0u;
+    const int ip = warp_best(s_pair, A, 0, lut_mask);
+    const int is = warp_best(s_pair, A, 1, lut_mask);
+    const int isg = signed_table ? warp_best(s_sig, A, 0, lut_mask) : -1;
+    if (tid == 0) {
+      res->layer_absmax = wmax;
+      res->reserved[0] = res->reserved[1] = 0;
+      res->best_a = ip >= 0 ? ip / A : -1; res->best_b = ip >= 0 ? ip % A : -1;
+      res->best_single = is >= 0 ? is / A : -1;
+      res->best_sa = isg >= 0 ? isg / A : -1; res->best_sb = isg >= 0 ? isg % A : -1;
+    }
   }
 }
 
