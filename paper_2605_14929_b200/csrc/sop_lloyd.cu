@@ -35,6 +35,7 @@ namespace sop {
 
 constexpr int LTB = 256;
 constexpr int SETUP_TB = 1024;
+constexpr int SOP_MAX_LLOYD_ITERS = 64;
 constexpr int SORT_CHALF = 320;                 // lookup grid on u: cell width 2^-8, rows cover |u| <= 1.25,
 constexpr int SORT_ROWS = 2 * SORT_CHALF + 1;   // the first and last row take everything beyond
 constexpr float SORT_INVH = 256.0f;
@@ -64,7 +65,12 @@ struct LloydWs {
   float cmax;
   int k;
   int fmta;
-  unsigned done;         // CTAs of the running iteration that have added their sums
+  unsigned done;         // CTAs of the running iteration that have added their sums (one launch per iteration)
+  // one launch for all iterations: CTAs that have added their sums in iteration i, and the flag that the
+  // table of iteration i + 1 is published; never reset (the header is cleared before every call)
+  unsigned arrive[SOP_MAX_LLOYD_ITERS + 1];
+  unsigned ready[SOP_MAX_LLOYD_ITERS + 1];
+  unsigned error;        // a CTA gave up waiting for a flag
   unsigned list_count;   // blocks appended to the pool list
   int pad;
   // the current codebook, rewritten by whoever changes it (set-up, then each update)
@@ -491,8 +497,12 @@ __device__ __forceinline__ void flush_limbs(unsigned* n0, unsigned* n1, unsigned
   atomicAdd(&s2[code], (int)((long long)sv >> 24));
 }
 
-__global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                          int it, int last, float* __restrict__ out_lut) {
+// One iteration, by a whole CTA.  `counter` counts the CTAs that have added their sums; the CTA that arrives
+// last updates the table and returns true.  FRESH: the descriptor was written during this launch by another
+// CTA, so it is read past the L1.
+template <bool FRESH>
+__device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                int it, int last, float* __restrict__ out_lut, unsigned* counter, bool reset_counter) {
   __shared__ __align__(16) IterDesc d;
   __shared__ unsigned long long sN[SOP_MAX_ENTRIES], sS[SOP_MAX_ENTRIES];
   // flushes of the element walk: native 32-bit atomics on limbs, combined into sN / sS afterwards
@@ -510,7 +520,10 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
   {
     constexpr int DW = (int)(sizeof(IterDesc) / sizeof(unsigned));
     static_assert(DW <= LTB, "one descriptor word per thread");
-    if (tid < DW) reinterpret_cast<unsigned*>(&d)[tid] = reinterpret_cast<const unsigned*>(&ws->desc)[tid];
+    if (tid < DW) {
+      const unsigned* src = reinterpret_cast<const unsigned*>(&ws->desc) + tid;
+      reinterpret_cast<unsigned*>(&d)[tid] = FRESH ? __ldcg(src) : *src;
+    }
     if (tid == LTB - 1) s_list_count = ws->list_count;
     if (tid < 32) { sN[tid] = 0; sS[tid] = 0; lN[0][tid] = lN[1][tid] = lS0[tid] = lS1[tid] = 0; lS2[tid] = 0; }
     if (tid == 0) sD = 0.0;
@@ -636,9 +649,10 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
   // the CTA that arrives last owns the update; no CTA waits for another
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_is_last = atomicAdd(&ws->done, 1u) == gridDim.x - 1 ? 1 : 0;
+  if (tid == 0) s_is_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1 : 0;
   __syncthreads();
-  if (s_is_last && tid < 32) {
+  const bool is_last = s_is_last != 0;
+  if (is_last && tid < 32) {
     // one warp: every CTA has added its share (cells with a threshold element by element, the others by
     // their sums).  Centroids one lane per entry, a rank sort, and the next iteration's descriptor.
     __threadfence();
@@ -646,7 +660,7 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
     const long long sv = __ldcg(&ws->accS[tid]);
     if (tid == 0) distortion[it] = __ldcg(&ws->accD);
     ws->accN[tid] = 0; ws->accS[tid] = 0;
-    if (tid == 0) { ws->accD = 0.0; ws->done = 0; }
+    if (tid == 0) { ws->accD = 0.0; if (reset_counter) *counter = 0; }
     if (last) {
       out_lut[tid] = tid < ne ? lutv[tid] : 0.0f;
     } else {
@@ -673,6 +687,50 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
       if (tid >= ne) s_new[tid] = top;           // padded with the last entry
       __syncwarp();
       lloyd_publish_desc(ws, s_new, ne);
+    }
+  }
+  return is_last;
+}
+
+// One launch per iteration (the stream orders the iterations).
+__global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                          int it, int last, float* __restrict__ out_lut) {
+  lloyd_iteration<false>(a, ws, distortion, it, last, out_lut, &ws->done, true);
+}
+
+// All iterations in one launch (launched cooperatively: every CTA is resident).  Between two iterations the
+// CTAs wait for the flag that the CTA which arrived last sets after it has published the next table.  The
+// wait is bounded: a CTA that gives up raises ws->error, every CTA then leaves, and the last distortion entry
+// is set to -1 (a distortion is never negative) so that the caller can tell.
+constexpr unsigned WAIT_POLLS = 1u << 22;     // times ~100 ns: about half a second
+
+__global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
+                                                               int iters, float* __restrict__ out_lut) {
+  __shared__ int s_stop;
+  for (int it = 0; it <= iters; ++it) {
+    const int last = it == iters;
+    const bool updater = lloyd_iteration<true>(a, ws, distortion, it, last, out_lut, &ws->arrive[it], false);
+    if (last) break;
+    __syncthreads();                       // the updater's first warp has written the descriptor
+    if (threadIdx.x == 0) {
+      int stop = 0;
+      if (updater) {
+        __threadfence();
+        atomicExch(&ws->ready[it], 1u);
+      } else {
+        unsigned polls = 0;
+        while (*(volatile unsigned*)&ws->ready[it] == 0u) {
+          if (*(volatile unsigned*)&ws->error != 0u || ++polls > WAIT_POLLS) { atomicExch(&ws->error, 1u); stop = 1; break; }
+          __nanosleep(100);
+        }
+        __threadfence();
+      }
+      s_stop = stop;
+    }
+    __syncthreads();
+    if (s_stop) {
+      if (blockIdx.x == 0 && threadIdx.x == 0) distortion[iters] = -1.0;
+      return;
     }
   }
 }
@@ -769,9 +827,26 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   }
   if (grid < 1) grid = 1;
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
-  for (int it = 0; it <= iters; ++it) {
-    const int last = it == iters;
-    lloyd_split_kernel<<<(int)grid, LTB, 0, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
+  // All iterations in one cooperative launch when every CTA of the grid can be resident at once (the CTAs wait
+  // for one another between iterations); otherwise one launch per iteration.
+  static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
+  if (coop_blocks_per_sm < 0) {
+    int dev = 0, coop = 0, nb = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, lloyd_persistent_kernel, LTB, 0) == cudaSuccess)
+      coop_blocks_per_sm = nb;
+    else
+      coop_blocks_per_sm = 0;
+    cudaGetLastError();
+  }
+  if (iters >= 1 && coop_blocks_per_sm > 0 && grid <= (long long)coop_blocks_per_sm * sms) {
+    void* kargs[] = {(void*)&a, (void*)&ws, (void*)&distortion_dev, (void*)&iters, (void*)&out_lut_dev};
+    SOP_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)lloyd_persistent_kernel, dim3((unsigned)grid), dim3(LTB), kargs, 0, st));
+  } else {
+    for (int it = 0; it <= iters; ++it) {
+      const int last = it == iters;
+      lloyd_split_kernel<<<(int)grid, LTB, 0, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
+    }
   }
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;
   SOP_CUDA_TRY(cudaGetLastError());
