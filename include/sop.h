@@ -222,16 +222,26 @@ int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE
  *     SOP_LLOYD_POOL_THRESHOLD   axis (iv): the pool is every block whose metric is at least as bad as
  *       pool_threshold (cosine <= threshold, or error >= threshold); pool_rank is ignored.  An empty pool
  *       leaves the table as it is.
+ *     SOP_LLOYD_LAUNCH_PER_ITERATION  (no counterpart in the paper) one kernel launch per iteration even
+ *       where all iterations could run in one cooperative launch; the results are the same.
  *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
  *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
  *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
+ *     When the iterations run in one launch, its CTAs wait for one another between iterations; every
+ *     wait is bounded (about half a second).  A CTA that gives up makes all of them leave and the last
+ *     entry is set to -1 (a distortion is never negative): the table is then not valid.
  *   pool_count_dev: one long long, number of blocks in the pool.
  * Workspace: 8 bytes per weight element (u and omega of every pool element are kept across the
  *   iterations), 4 bytes per block (the pool list) and 4 bytes per channel, plus a fixed header. */
 #define SOP_LLOYD_POOL_BY_ERROR 1
 #define SOP_LLOYD_UNIFORM_WEIGHTS 2
 #define SOP_LLOYD_POOL_THRESHOLD 4
+#define SOP_LLOYD_LAUNCH_PER_ITERATION 8
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
+/* Number of kernel launches one sop_dd4_lloyd call with these sizes and flags makes on the current device
+ * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch when
+ * every CTA of the iteration grid can be resident at once; otherwise there is one launch per iteration. */
+int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches);
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
                   const float* block_metric_dev, long long pool_rank, float pool_threshold, int flags,

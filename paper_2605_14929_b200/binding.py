@@ -22,7 +22,7 @@ MAX_ATOMS = 16
 ALL_ATOMS = 0xFFFFFFFF
 SEARCH_SINGLES_ONLY = 1
 SEARCH_SELECT_MSE = 2
-LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD = 1, 2, 4
+LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD, LLOYD_LAUNCH_PER_ITERATION = 1, 2, 4, 8
 PACK_SELECT_MSE = 1
 MAX_ENTRIES = 32
 
@@ -82,7 +82,7 @@ def lib():
 def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
             "sop_channel_norms_static",
-            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd", "sop_pack",
+            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd", "sop_pack",
             "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
 
 
@@ -149,6 +149,13 @@ def dd4_lloyd_workspace(M: int, K: int) -> int:
     return n.value
 
 
+def dd4_lloyd_launches(M: int, K: int, iters: int, flags: int = 0) -> int:
+    """Kernel launches of one ``sop_dd4_lloyd`` call on the current device."""
+    n = C.c_int()
+    _check(lib().sop_dd4_lloyd_launches(_ll(M), _ll(K), iters, flags, C.byref(n)), "sop_dd4_lloyd_launches")
+    return n.value
+
+
 def alloc_workspace(nbytes: int, device) -> torch.Tensor:
     """A 256-byte aligned device buffer (torch's caching allocator aligns to 512 bytes)."""
     return torch.empty(max(256, nbytes), dtype=torch.uint8, device=device)
@@ -199,7 +206,8 @@ def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_
                   iters: int, out_lut: torch.Tensor, distortion: torch.Tensor, pool_count: torch.Tensor,
                   workspace: torch.Tensor, k_mode: int = K_FROM_RESULT, search_result: Optional[torch.Tensor] = None,
                   fmta_index: int = FMTA_FROM_RESULT, stream=None, g: int = 16, pool_by_error: bool = False,
-                  uniform_weights: bool = False, pool_threshold: Optional[float] = None) -> None:
+                  uniform_weights: bool = False, pool_threshold: Optional[float] = None,
+                  launch_per_iteration: bool = False) -> None:
     """``block_cos`` is the per-block metric that ranks the blocks: cosines, or errors with ``pool_by_error``.
     A ``pool_threshold`` replaces the rank."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
@@ -208,7 +216,8 @@ def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_
                                _ptr(search_result), _ptr(block_cos), _ll(pool_rank),
                                C.c_float(0.0 if pool_threshold is None else pool_threshold),
                                (LLOYD_POOL_BY_ERROR if pool_by_error else 0) | (LLOYD_UNIFORM_WEIGHTS if uniform_weights else 0)
-                               | (LLOYD_POOL_THRESHOLD if pool_threshold is not None else 0),
+                               | (LLOYD_POOL_THRESHOLD if pool_threshold is not None else 0)
+                               | (LLOYD_LAUNCH_PER_ITERATION if launch_per_iteration else 0),
                                make_atoms(atoms), len(atoms),
                                fmta_index, iters, _ptr(out_lut), _ptr(distortion), _ptr(pool_count), _ptr(workspace),
                                C.c_size_t(workspace.numel()), _stream(stream)), "sop_dd4_lloyd")

@@ -606,8 +606,11 @@ __device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __r
         if (item < i_hi) {
           int l = 0;                       // the split cell whose item range holds `item`: binary search over <= 32 offsets
 #pragma unroll
-          for (int step = 16; step >= 1; step >>= 1)
-            if (l + step < n_split && s_off[warp][l + step] <= item) l += step;
+          for (int step = 16; step >= 1; step >>= 1) {     // branch-free: s_off has MAX_SPLIT + 1 entries
+            const int t = l + step;
+            const bool ok = (t < n_split) & (s_off[warp][min(t, MAX_SPLIT)] <= item);
+            l = ok ? t : l;
+          }
           cell_l[k] = l;
           const unsigned pp = s_p0[warp][l] + (item - s_off[warp][l]);
           v[k] = __ldg(src + (pp & 15u) * LTB + (pp >> 4));
@@ -737,9 +740,51 @@ __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, Lloy
 
 int num_sms();
 
+// Grid of the iteration kernels and whether all iterations run in one cooperative launch: they do when every
+// CTA of a grid that keeps to four tiles per warp can be resident at once (the CTAs wait for one another
+// between iterations); otherwise there is one launch per iteration.
+static bool lloyd_iteration_plan(long long NB, int iters, int flags, long long* grid_out) {
+  const int sms = num_sms();
+  const long long tiles = (NB + LTB - 1) / LTB;
+  long long grid = (tiles + LTB / 32 - 1) / (LTB / 32);             // one warp per cache tile
+  if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+  // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
+  const long long need = (tiles + 4 * (LTB / 32) - 1) / (4 * (LTB / 32));
+  if (grid < need) grid = need;
+  if (grid < 1) grid = 1;
+  static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
+  if (coop_blocks_per_sm < 0) {
+    int dev = 0, coop = 0, nb = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, lloyd_persistent_kernel, LTB, 0) == cudaSuccess)
+      coop_blocks_per_sm = nb;
+    else
+      coop_blocks_per_sm = 0;
+    cudaGetLastError();
+  }
+  const long long resident = (long long)coop_blocks_per_sm * sms;
+  bool persistent = false;
+  if (iters >= 1 && resident >= need && resident >= 1 && !(flags & SOP_LLOYD_LAUNCH_PER_ITERATION)) {
+    persistent = true;
+    if (grid > resident) grid = resident;
+  }
+  *grid_out = grid;
+  return persistent;
+}
+
 }  // namespace sop
 
 extern "C" {
+
+int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches) {
+  if (!launches) return SOP_ERR_NULL;
+  if (M < 1 || K < 1 || (K % SOP_G) != 0 || iters < 0 || iters > sop::SOP_MAX_LLOYD_ITERS) return SOP_ERR_RANGE;
+  long long grid = 1;
+  const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), iters, flags, &grid);
+  // radix select (three passes, unless the pool is cut by a threshold), set-up, pool list, pool cache, iterations
+  *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + (persistent ? 1 : iters + 1);
+  return SOP_OK;
+}
 
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
@@ -759,7 +804,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
   if (rc) return rc;
   if (!block_metric_dev || !out_lut_dev || !distortion_dev || !pool_count_dev) return SOP_ERR_NULL;
-  if (flags & ~(SOP_LLOYD_POOL_BY_ERROR | SOP_LLOYD_UNIFORM_WEIGHTS | SOP_LLOYD_POOL_THRESHOLD)) return SOP_ERR_RANGE;
+  if (flags & ~(SOP_LLOYD_POOL_BY_ERROR | SOP_LLOYD_UNIFORM_WEIGHTS | SOP_LLOYD_POOL_THRESHOLD | SOP_LLOYD_LAUNCH_PER_ITERATION)) return SOP_ERR_RANGE;
   const bool by_threshold = (flags & SOP_LLOYD_POOL_THRESHOLD) != 0;
   if (by_threshold && !(pool_threshold == pool_threshold)) return SOP_ERR_RANGE;   // NaN orders nothing
   FmtDev F;
@@ -818,28 +863,10 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev);
     SOP_CUDA_TRY(cudaGetLastError());
   }
-  long long grid = ((NB + LTB - 1) / LTB + LTB / 32 - 1) / (LTB / 32);   // one warp per cache tile
-  if (grid > (long long)sms * 8) grid = (long long)sms * 8;
-  {
-    // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
-    const long long tiles = (NB + LTB - 1) / LTB, need = (tiles + 4 * (LTB / 32) - 1) / (4 * (LTB / 32));
-    if (grid < need) grid = need;
-  }
-  if (grid < 1) grid = 1;
+  long long grid = 1;
+  const bool persistent = lloyd_iteration_plan(NB, iters, flags, &grid);
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
-  // All iterations in one cooperative launch when every CTA of the grid can be resident at once (the CTAs wait
-  // for one another between iterations); otherwise one launch per iteration.
-  static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
-  if (coop_blocks_per_sm < 0) {
-    int dev = 0, coop = 0, nb = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, lloyd_persistent_kernel, LTB, 0) == cudaSuccess)
-      coop_blocks_per_sm = nb;
-    else
-      coop_blocks_per_sm = 0;
-    cudaGetLastError();
-  }
-  if (iters >= 1 && coop_blocks_per_sm > 0 && grid <= (long long)coop_blocks_per_sm * sms) {
+  if (persistent) {
     void* kargs[] = {(void*)&a, (void*)&ws, (void*)&distortion_dev, (void*)&iters, (void*)&out_lut_dev};
     SOP_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)lloyd_persistent_kernel, dim3((unsigned)grid), dim3(LTB), kargs, 0, st));
   } else {

@@ -114,6 +114,7 @@ class LayerSweep:
         self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
         self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
         self.kernel_launches_per_step = 0
+        self.lloyd_launches = B.dd4_lloyd_launches(M, K, lloyd_iters) if lloyd_iters > 0 else 0
 
     def run(self, W: torch.Tensor, X: torch.Tensor, stream=None) -> None:
         """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32."""
@@ -127,7 +128,7 @@ class LayerSweep:
             n += 2
             B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
-            n += 6 + (self.iters + 1)
+            n += self.lloyd_launches
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
                               block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask,

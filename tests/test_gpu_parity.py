@@ -218,14 +218,14 @@ def test_negation_symmetry_on_gpu(B):
 
 
 # ------------------------------------------------------------------ Lloyd
-def gpu_lloyd(B, W, c, fmt, atoms, bc, rank, iters, k, fmta):
+def gpu_lloyd(B, W, c, fmt, atoms, bc, rank, iters, k, fmta, **kw):
     M, K = W.shape
     out = torch.zeros(32, dtype=torch.float32, device=dev())
     dist = torch.zeros(iters + 1, dtype=torch.float64, device=dev())
     cnt = torch.zeros(1, dtype=torch.int64, device=dev())
     ws = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), dev())
     B.sop_dd4_lloyd(W.to(dev()), torch.as_tensor(c).to(dev()), fmt, atoms, bc, rank, iters, out, dist, cnt, ws,
-                    k_mode=k, fmta_index=fmta)
+                    k_mode=k, fmta_index=fmta, **kw)
     torch.cuda.synchronize()
     return out.cpu().numpy(), dist.cpu().numpy(), int(cnt.item())
 
@@ -244,11 +244,16 @@ def test_lloyd_matches_oracle(B, fmt_name, names, iters):
             init = np.sort(-a.lut) if a.negated else a.lut
             want = oracle.dd_lloyd(L.W, c, fmt, int(r["k"][fmta]), r["block_cos"][fmta], rank, init, iters)
             bc = torch.from_numpy(r["block_cos"]).to(dev())
-            got = gpu_lloyd(B, L.W, c, fmt, atoms, bc, rank, iters, int(r["k"][fmta]), fmta)
             ne = len(a.lut)
-            assert np.array_equal(got[0][:ne].view(np.uint32), want[0].view(np.uint32))
-            assert got[2] == want[2]
-            assert np.allclose(got[1], want[1], rtol=REL, atol=0)
+            # all iterations in one cooperative launch (the default where the grid fits), and one launch per iteration
+            for per_iteration in (False, True):
+                got = gpu_lloyd(B, L.W, c, fmt, atoms, bc, rank, iters, int(r["k"][fmta]), fmta, launch_per_iteration=per_iteration)
+                assert np.array_equal(got[0][:ne].view(np.uint32), want[0].view(np.uint32))
+                assert got[2] == want[2]
+                assert np.allclose(got[1], want[1], rtol=REL, atol=0)
+    M, K = L.W.shape
+    assert B.dd4_lloyd_launches(M, K, iters, B.LLOYD_LAUNCH_PER_ITERATION) == 6 + iters + 1
+    assert B.dd4_lloyd_launches(M, K, iters) in (7, 6 + iters + 1)
 
 
 def test_lloyd_with_entries_closer_than_the_lookup_grid(B):
