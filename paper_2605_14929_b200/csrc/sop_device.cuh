@@ -192,11 +192,13 @@ __device__ __forceinline__ void build_thresholds(const float* lut, int ne, float
   }
 }
 
-// number of thresholds strictly below u: branch-free binary search over 31 sorted entries (+inf padded)
+// number of thresholds strictly below u: branch-free binary search over 2^STEPS - 1 sorted entries (+inf
+// padded to 31).  Five steps cover any table; four are enough for a table of at most 16 entries.
+template <int STEPS = 5>
 __device__ __forceinline__ int count_below(const float* tau, float u) {
   int pos = 0;
 #pragma unroll
-  for (int step = 16; step >= 1; step >>= 1)
+  for (int step = 1 << (STEPS - 1); step >= 1; step >>= 1)
     if (tau[pos + step - 1] < u) pos += step;
   return pos;
 }

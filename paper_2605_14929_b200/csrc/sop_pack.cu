@@ -24,6 +24,8 @@ struct PackArgs {
   int cos_neg_a, cos_neg_b; // rows of the negated variants of index_a / index_b (-1: unknown, evaluate instead)
 };
 
+constexpr int KIND_LUT16 = 100;   // inside this file: a LUT of at most 16 entries (a four-step search is enough)
+
 struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; GridDev grid; int sign_pos; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
@@ -44,8 +46,8 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
       const float u = __fmul_rn(w[i], rcp);
       float q;
       uint32_t code;
-      if (KIND == SOP_KIND_LUT) {
-        code = (uint32_t)count_below(tau, neg ? -u : u);
+      if (KIND == SOP_KIND_LUT || KIND == KIND_LUT16) {
+        code = (uint32_t)(KIND == KIND_LUT16 ? count_below<4>(tau, neg ? -u : u) : count_below<5>(tau, neg ? -u : u));
         q = neg ? -lutv[code] : lutv[code];
       } else if (KIND == SOP_KIND_FP_E2M3) {
         q = fp_quantize<SOP_KIND_FP_E2M3>(u);
@@ -81,7 +83,8 @@ template <int METRIC>
 __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int kind, int neg, float rcp, float s_hat,
                                                 float& cos_out, uint32_t (&code4)[4], const GridDev grid, int sign_pos) {
-  if (kind == SOP_KIND_LUT) eval_block_kind<METRIC, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+  if (kind == KIND_LUT16) eval_block_kind<METRIC, KIND_LUT16>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+  else if (kind == SOP_KIND_LUT) eval_block_kind<METRIC, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
   else if (kind == SOP_KIND_FP_GRID) eval_block_kind<METRIC, SOP_KIND_FP_GRID>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4, grid, sign_pos);
   else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<METRIC, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
   else eval_block_kind<METRIC, SOP_KIND_FP_E4M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
@@ -114,7 +117,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
     for (int t = 0; t < nb; ++t) {
       const int idx = t ? ib : ia;
       const sop_atom& at = A.atoms[idx];
-      base[t].table = t; base[t].kind = at.kind; base[t].neg = at.negated; base[t].scope = at.scope; base[t].tmax = at.tmax;
+      base[t].table = t; base[t].kind = (at.kind == SOP_KIND_LUT && at.n_entries <= 16) ? KIND_LUT16 : at.kind; base[t].neg = at.negated; base[t].scope = at.scope; base[t].tmax = at.tmax;
       base[t].k = a.k_mode == SOP_K_FROM_RESULT ? res->k[idx] : a.k_mode;
       base[t].grid.min_eb = 128 - at.grid_bias; base[t].grid.sh = 23 - at.grid_man_bits;
       base[t].grid.vpos = at.tmax; base[t].grid.vneg = at.grid_neg_max;
