@@ -508,9 +508,10 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
           }
           moff = 2u * (unsigned)C.c_half * pitch + 2u * (unsigned)copy_off;
           // tables of this class with a usable cell grid: the table slot is a compile-time displacement
+          const unsigned cls_fast = P.cls_tables[cl] & fast_mask;
 #pragma unroll
           for (int T = 0; T < SOP_MAX_TABLES; ++T) {
-            if (T < P.n_tables && P.table_cls[T] == cl && ((fast_mask >> T) & 1u)) {
+            if ((cls_fast >> T) & 1u) {
               const unsigned char* tp = cell_bytes + T * 128;
               const int ap = P.table_pos[T], an = P.table_neg[T];
               if (ap != 255) {
