@@ -743,10 +743,11 @@ int num_sms();
 // Grid of the iteration kernels and whether all iterations run in one cooperative launch: they do when every
 // CTA of a grid that keeps to four tiles per warp can be resident at once (the CTAs wait for one another
 // between iterations); otherwise there is one launch per iteration.
-static bool lloyd_iteration_plan(long long NB, int iters, int flags, long long* grid_out) {
+static bool lloyd_iteration_plan(long long NB, long long pool_blocks, int iters, int flags, long long* grid_out) {
   const int sms = num_sms();
-  const long long tiles = (NB + LTB - 1) / LTB;
-  long long grid = (tiles + LTB / 32 - 1) / (LTB / 32);             // one warp per cache tile
+  const long long tiles = (NB + LTB - 1) / LTB;                     // all blocks in the pool: the most there can be
+  const long long likely = (pool_blocks + LTB - 1) / LTB;           // the pool without ties at its threshold
+  long long grid = (likely + LTB / 32 - 1) / (LTB / 32);            // one warp per cache tile
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
   // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
   const long long need = (tiles + 4 * (LTB / 32) - 1) / (4 * (LTB / 32));
@@ -780,7 +781,7 @@ int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* 
   if (!launches) return SOP_ERR_NULL;
   if (M < 1 || K < 1 || (K % SOP_G) != 0 || iters < 0 || iters > sop::SOP_MAX_LLOYD_ITERS) return SOP_ERR_RANGE;
   long long grid = 1;
-  const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), iters, flags, &grid);
+  const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), M * (K / SOP_G), iters, flags, &grid);
   // radix select (three passes, unless the pool is cut by a threshold), set-up, pool list, pool cache, iterations
   *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + (persistent ? 1 : iters + 1);
   return SOP_OK;
@@ -864,7 +865,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     SOP_CUDA_TRY(cudaGetLastError());
   }
   long long grid = 1;
-  const bool persistent = lloyd_iteration_plan(NB, iters, flags, &grid);
+  const bool persistent = lloyd_iteration_plan(NB, by_threshold ? NB : pool_rank, iters, flags, &grid);
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
   if (persistent) {
     void* kargs[] = {(void*)&a, (void*)&ws, (void*)&distortion_dev, (void*)&iters, (void*)&out_lut_dev};
