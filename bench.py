@@ -274,7 +274,9 @@ def run_gpu(args) -> None:
                                                        parallelism=f"layer-parallel x{world}, no collective"),
             kernels_ms=dict(kavg, note="per step, CUDA events recorded by the library around its main kernels; "
                                        "sweep1 = fixed candidates (singles), sweep2 = DD columns (all pairs), "
-                                       "lloyd = all iteration launches"),
+                                       "lloyd = all Lloyd iterations (one cooperative launch where the grid fits)"),
+            sweep_only=dict(value=world * E / sweep_t / 1e9, unit=UNIT,
+                            note="elements / time of the two sweep launches of a step (every candidate, every pair)"),
             roofline=dominant,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
                               sample=f"first {cpu_rows} of {M} rows, whole pipeline, {cpu_dt:.1f} s"),
