@@ -390,3 +390,18 @@ def test_layer_stream_returns_each_layers_own_results(B):
         for k in LayerStream.OUT:
             assert torch.equal(got[i][k], want[i][k]), (i, k)
     assert not torch.equal(want[0]["codes"], want[1]["codes"])
+
+
+def test_lloyd_without_iterations_reports_the_initial_table(B):
+    # iters = 0: the table stays the primary codebook's, the one distortion entry is that of this table
+    L = I.tiny_layer(17, 24, 256)
+    fmt = I.scale_format("UE4M4")
+    atoms = I.alphabet(["NF4"])
+    c = oracle.channel_norms(L.X.numpy())
+    r = oracle.pair_search(L.W, c, fmt, atoms, want_blocks=True)
+    NB = r["block_cos"].shape[1]
+    want = oracle.dd_lloyd(L.W, c, fmt, int(r["k"][0]), r["block_cos"][0], NB // 2, atoms[0].lut, 0)
+    got = gpu_lloyd(B, L.W, c, fmt, atoms, torch.from_numpy(r["block_cos"]).to(dev()), NB // 2, 0, int(r["k"][0]), 0)
+    assert np.array_equal(got[0][:16], atoms[0].lut) and np.array_equal(want[0], atoms[0].lut)
+    assert got[2] == want[2] and np.allclose(got[1], want[1], rtol=REL, atol=0)
+    assert B.dd4_lloyd_launches(24, 256, 0) == 7
