@@ -145,6 +145,24 @@ class LayerSweep:
         n += 1
         self.kernel_launches_per_step = n
 
+    def capture(self, W: torch.Tensor, X: torch.Tensor) -> None:
+        """Record the calls of ``run(W, X)`` into a CUDA graph bound to these two tensors (refill them in place
+        for the next layer); ``replay()`` then launches the whole pass at once, without the gaps between a
+        dozen launches.  Profiling (``binding.profile_enable``) must be off: events recorded inside a graph
+        cannot be read back."""
+        self.run(W, X)                       # the library's one-time set-ups happen outside the capture
+        torch.cuda.synchronize(self.dev)
+        side = torch.cuda.Stream(self.dev)
+        side.wait_stream(torch.cuda.current_stream(self.dev))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            self.run(W, X, side)
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        self._graph, self._graph_inputs = graph, (W, X)
+
+    def replay(self) -> None:
+        self._graph.replay()
+
     def outputs(self) -> SweepOutputs:
         torch.cuda.synchronize(self.dev)
         nF, nR = len(self.full_atoms), len(self.rom_atoms)

@@ -405,3 +405,24 @@ def test_lloyd_without_iterations_reports_the_initial_table(B):
     assert np.array_equal(got[0][:16], atoms[0].lut) and np.array_equal(want[0], atoms[0].lut)
     assert got[2] == want[2] and np.allclose(got[1], want[1], rtol=REL, atol=0)
     assert B.dd4_lloyd_launches(24, 256, 0) == 7
+
+
+def test_graph_replay_equals_the_calls(B):
+    # the layer's calls captured into one CUDA graph: refilling the bound input tensors and replaying gives the
+    # results of a plain run on the new layer
+    from paper_2605_14929_b200.pipeline import LayerStream, LayerSweep
+    fmt = I.scale_format("S1E4M4")
+    M, K, T = 40, 512, 64
+    a, b = I.outlier_channel_layer(50, M, K, T), I.outlier_channel_layer(51, M, K, T)
+    sw = LayerSweep(M, K, T, fmt, ["NF4", "SH4"], [], 4, device=dev())
+    sw.run(b.W.to(dev()), b.X.to(dev()))
+    torch.cuda.synchronize()
+    want = {k: getattr(sw, k).cpu().clone() for k in LayerStream.OUT}
+    Wd, Xd = a.W.to(dev()), a.X.to(dev())
+    sw.capture(Wd, Xd)
+    Wd.copy_(b.W)
+    Xd.copy_(b.X)
+    sw.replay()
+    torch.cuda.synchronize()
+    for k in LayerStream.OUT:
+        assert torch.equal(getattr(sw, k).cpu(), want[k]), k
