@@ -1,31 +1,35 @@
 // sop_dd4_lloyd: per-layer data-derived codebook (DD-n) by Lloyd iteration on the pool of blocks
 // that the primary codebook reconstructs worst.
 //
-//   select_kernel<PASS>   three-pass radix select (11 + 11 + 10 bits) of the pool_rank-th smallest
-//                         block cosine; each pass re-derives the prefix from the previous histograms
-//                         with a CTA-wide scan.
-//   lloyd_setup_kernel    threshold tau and pool count from the last histogram, max(c), the shift k,
-//                         the initial table (FMTa, reversed and negated if FMTa is a negated atom),
-//                         and the per-channel weight table omega = c / max(c).
-//   pool_list_kernel      compacts the indices of the pool blocks (cos <= tau) into a dense list, so
-//                         that every lane of the iteration kernel has work.
+//   select_kernel<PASS>   three-pass radix select (11 + 11 + 10 bits) of the pool_rank-th worst block by
+//                         its ranking key (cosine ascending, or error descending); each pass re-derives
+//                         the prefix from the previous histograms with a CTA-wide scan.  Not run when the
+//                         caller fixes the pool threshold.
+//   lloyd_setup_kernel    threshold key from the last histogram (or from the given threshold), max(c),
+//                         the shift k, the initial table (FMTa, reversed and negated if FMTa is a negated
+//                         atom), the per-channel weight table omega = c / max(c) (or 1), and the first
+//                         iteration descriptor.
+//   pool_list_kernel      compacts the indices of the pool blocks into a dense list.
 //   pool_cache_kernel     the pool elements never change between iterations, only the table does:
 //                         (u, omega) of every pool element is computed once (u = w / scale) and kept
 //                         in tiles of 4096 elements, each counting-sorted by the cell of u on a
 //                         uniform grid (641 cells of width 2^-8); the start of every cell inside
 //                         every tile is kept too, and per cell, over the whole pool, the int64
-//                         fixed-point sums of omega and omega u and the FP64 moments
+//                         fixed-point sums of omega and omega u and the moments
 //                         sum omega, sum omega u, sum omega u^2.
-//   lloyd_split_kernel    one iteration.  A cell that holds no decision threshold of the current
-//                         table lies inside one entry's interval: its elements are accounted for
-//                         by the cell's sums and moments, without touching them.  Only the cells
-//                         that hold a threshold (at most one per threshold) are walked element by
-//                         element, exactly: one warp per tile, one lane per such cell.  Per-entry
-//                         sums are int64 fixed point (exactly associative: the table is the same
-//                         bit for bit as a sequential sum over all elements gives), distortion
-//                         FP64.  The CTA that finishes last adds the untouched cells, turns the
-//                         sums into centroids, snaps them to bf16, sorts, prepares the next
-//                         iteration's tables and clears the accumulators.
+//   lloyd_iteration       one iteration (device function).  A cell that holds no decision threshold of
+//                         the current table lies inside one entry's interval: its elements are
+//                         accounted for by the cell's sums and moments, without touching them.  Only
+//                         the cells that hold a threshold are walked element by element, exactly: one
+//                         warp per tile, the lanes taking contiguous shares of those cells' elements.
+//                         Per-entry sums are int64 fixed point (exactly associative: the table is the
+//                         same bit for bit as a sequential sum over all elements gives), distortion
+//                         FP64.  The CTA that finishes last turns the sums into centroids, snaps them to
+//                         bf16, sorts, publishes the next iteration's descriptor and clears the
+//                         accumulators.
+//   lloyd_persistent_kernel  all iterations in one cooperative launch; between iterations the CTAs wait,
+//                         bounded, for the flag of the CTA that finished last.
+//   lloyd_split_kernel    one iteration per launch: used where the grid cannot be resident at once.
 #include <math.h>
 #include <string.h>
 
