@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
   __shared__ float s_pot[2];
   __shared__ unsigned s_cnt[2];
   __shared__ int s_row[4];   // rows of block_cos for the candidates a, -a, b, -b (-1: none)
+  __shared__ int s_idx[2];   // the two atoms
   const int tid = threadIdx.x;
   if (tid == 0) {
     int ia = a.index_a, ib = a.index_b;
@@ -123,10 +124,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
       base[t].grid.vpos = at.tmax; base[t].grid.vneg = at.grid_neg_max;
       base[t].sign_pos = at.grid_exp_bits + at.grid_man_bits;
       s_pot[t] = at.scope == 0 ? layer_pot_scale(wmax, at.tmax) : 0.0f;
-      const bool dd = (A.dd_mask >> idx) & 1u;
-      const int ne = at.kind == SOP_KIND_LUT ? at.n_entries : 2;
-      for (int j = 0; j < 32; ++j) lutv[t][j] = at.kind == SOP_KIND_LUT ? (dd ? A.dd_lut[min(j, ne - 1)] : at.lut[min(j, ne - 1)]) : 0.0f;
-      build_thresholds(lutv[t], ne, tau[t]);
+      s_idx[t] = idx;
     }
     // from a search result with signs, a and b are base atoms and each is followed by its negation
     s_row[0] = ia;
@@ -137,6 +135,20 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
   }
   __syncthreads();
   const int nb = s_nb, n = s_nbits, b = a.container_bits;
+  // table values and decision thresholds of the (up to two) tables: one thread per entry (the same rule as
+  // build_thresholds: the largest fp32 <= the midpoint, a repeated entry takes the threshold above it)
+  if (tid < 32 * nb) {
+    const int t = tid >> 5, j = tid & 31, idx = s_idx[t];
+    const sop_atom& at = A.atoms[idx];
+    const bool dd = (A.dd_mask >> idx) & 1u;
+    const int ne = at.kind == SOP_KIND_LUT ? at.n_entries : 2;
+    lutv[t][j] = at.kind == SOP_KIND_LUT ? (dd ? A.dd_lut[min(j, ne - 1)] : at.lut[min(j, ne - 1)]) : 0.0f;
+    __syncwarp();
+    int jj = j;
+    while (jj < ne - 1 && lutv[t][jj] == lutv[t][jj + 1]) ++jj;
+    tau[t][j] = jj < ne - 1 ? __double2float_rd(0.5 * ((double)lutv[t][jj] + (double)lutv[t][jj + 1])) : __int_as_float(0x7F800000);
+  }
+  __syncthreads();
 
   const int n_sign = a.use_sign ? 2 : 1;
   unsigned my_sel = 0, my_neg = 0;
@@ -358,7 +370,7 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
   if (counts_dev) SOP_CUDA_TRY(cudaMemsetAsync(counts_dev, 0, 2 * sizeof(long long), st));
   long long grid = (a.NB + PTB - 1) / PTB;
   const int sms = num_sms();
-  if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+  if (grid > (long long)sms * 4) grid = (long long)sms * 4;      // one wave of resident CTAs: the table set-up runs once per CTA
   if ((rc = profile_mark(SOP_PROFILE_PACK, 0, st))) return rc;
   const bool negs_known = !use_sign || from_result || (a.cos_neg_a >= 0 && (!pair || a.cos_neg_b >= 0));
   if (block_cos_dev && negs_known) pack_kernel<true><<<(int)grid, PTB, 0, st>>>(a, A, F, search_dev);
