@@ -310,7 +310,16 @@ __device__ void build_tables(const Plan& P, const AtomsDev& A, uint2* cell, floa
   }
   if (tid < SOP_MAX_TABLES) fast[tid] = 1;
   __syncthreads();
-  if (tid < P.n_tables) build_thresholds(lutv + tid * 32, A.atoms[P.table_atom[tid]].n_entries, tau + tid * 32);
+  // decision thresholds, one thread per entry (the rule of build_thresholds: the largest fp32 <= the midpoint,
+  // a repeated entry takes the threshold above it, +inf from the last entry on)
+  for (int i = tid; i < P.n_tables * 32; i += blockDim.x) {
+    const int t = i >> 5, j = i & 31;
+    const int ne = A.atoms[P.table_atom[t]].n_entries;
+    const float* lv = lutv + t * 32;
+    int jj = j;
+    while (jj < ne - 1 && lv[jj] == lv[jj + 1]) ++jj;
+    tau[i] = jj < ne - 1 ? __double2float_rd(0.5 * ((double)lv[jj] + (double)lv[jj + 1])) : __int_as_float(0x7F800000);
+  }
   __syncthreads();
   const int rows = P.rows;
   for (int i = tid; i < P.n_tables * rows; i += blockDim.x) {
