@@ -152,10 +152,20 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
 
   const int n_sign = a.use_sign ? 2 : 1;
   unsigned my_sel = 0, my_neg = 0;
-  for (long long blk = (long long)blockIdx.x * PTB + tid; blk < a.NB; blk += (long long)gridDim.x * PTB) {
-    const long long m = blk / a.nbk, j = blk - m * a.nbk;
-    const uint4* p = reinterpret_cast<const uint4*>(a.W + m * a.ldw + j * SOP_G);
+  const unsigned nbk32 = (unsigned)a.nbk, NB32 = (unsigned)a.NB;       // the block count fits 31 bits
+  const int n_cand = nb * n_sign;
+  for (unsigned blk = blockIdx.x * PTB + tid; blk < NB32; blk += gridDim.x * PTB) {
+    const unsigned m = blk / nbk32, j = blk - m * nbk32;
+    const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
     const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
+    float cs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};      // the candidates' per-block values, loaded together with W
+    if (USE_COS) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int slot = n_sign == 2 ? q : 2 * q;          // candidate q of the order a, (-a), b, (-b)
+        if (q < n_cand) cs4[q] = __ldg(a.block_cos + (size_t)s_row[slot] * a.NB + blk);
+      }
+    }
     const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     float w[16], c[16];
 #pragma unroll
@@ -180,11 +190,13 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
     int pick = -1;
     if (USE_COS) {
       // the winner follows from the cosines of the sweep (same arithmetic, bit for bit): only it is encoded
-      for (int t = 0; t < nb; ++t)
-        for (int sg = 0; sg < n_sign; ++sg) {
-          const float cs = __ldg(a.block_cos + (size_t)s_row[2 * t + sg] * a.NB + blk);
-          if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) { best_cos = cs; pick = 2 * t + sg; }
-        }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q >= n_cand) break;
+        const float cs = cs4[q];
+        const int slot = n_sign == 2 ? q : 2 * q;
+        if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) { best_cos = cs; pick = slot; }
+      }
       const int t = pick >> 1, sg = pick & 1;
       const PackCand cd = base[t];
       float s_hat;
@@ -250,7 +262,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
         hi |= v << (pos - 64);
       }
     }
-    unsigned short* dst = reinterpret_cast<unsigned short*>(a.codes + blk * 2 * n);
+    unsigned short* dst = reinterpret_cast<unsigned short*>(a.codes + (size_t)blk * 2 * n);
     if (n == 4) {
       *reinterpret_cast<uint2*>(dst) = make_uint2((unsigned)lo, (unsigned)(lo >> 32));
     } else if (n == 8) {
@@ -263,7 +275,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
     if (a.word_sign_bits) word = (sgn << (b - 1)) | (best_scode << a.meta_bits) | (a.meta_bits >= 1 ? sel : 0u);
     else if (a.meta_bits >= 1) word = (sel << (b - 1)) | (best_scode << (a.meta_bits - 1));
     else word = best_scode;
-    const long long bit = blk * b;
+    const long long bit = (long long)blk * b;
     const long long wi = bit >> 5;
     const int sh = (int)(bit & 31);
     if (b == 16) {
