@@ -103,10 +103,11 @@ __global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, FmtDe
   for (int i = threadIdx.x; i < P.n_classes * SOP_HIST_BINS; i += blockDim.x) sh[i] = 0;
   __syncthreads();
   uint32_t wmax = 0;
-  for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < L.NB; b += (long long)gridDim.x * blockDim.x) {
-    const long long m = b / L.nbk, j = b - m * L.nbk;
+  const unsigned nbk32 = (unsigned)L.nbk, NB32 = (unsigned)L.NB;         // the block count fits 31 bits
+  for (unsigned b = blockIdx.x * blockDim.x + threadIdx.x; b < NB32; b += gridDim.x * blockDim.x) {
+    const unsigned m = b / nbk32, j = b - m * nbk32;
     uint32_t v[8];
-    load_block_bits(L.W + m * L.ldw + j * SOP_G, v);
+    load_block_bits(L.W + (long long)m * L.ldw + (long long)j * SOP_G, v);
     const float a = absmax_bits(v);
     wmax = max(wmax, __float_as_uint(a));
     if (a > 0.0f) {
