@@ -154,18 +154,29 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
   unsigned my_sel = 0, my_neg = 0;
   const unsigned nbk32 = (unsigned)a.nbk, NB32 = (unsigned)a.NB;       // the block count fits 31 bits
   const int n_cand = nb * n_sign;
-  for (unsigned blk = blockIdx.x * PTB + tid; blk < NB32; blk += gridDim.x * PTB) {
+  // the loads of a block (its weights and, when the winner is read off a sweep, the candidates' values) are
+  // issued one iteration ahead
+  auto fetch = [&](unsigned blk, uint4& v0, uint4& v1, float (&cs4)[4]) {
     const unsigned m = blk / nbk32, j = blk - m * nbk32;
     const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
-    const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
-    float cs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};      // the candidates' per-block values, loaded together with W
+    v0 = __ldg(p); v1 = __ldg(p + 1);
     if (USE_COS) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int slot = n_sign == 2 ? q : 2 * q;          // candidate q of the order a, (-a), b, (-b)
-        if (q < n_cand) cs4[q] = __ldg(a.block_cos + (size_t)s_row[slot] * a.NB + blk);
+        cs4[q] = q < n_cand ? __ldg(a.block_cos + (size_t)s_row[slot] * a.NB + blk) : 0.0f;
       }
     }
+  };
+  const unsigned stride = gridDim.x * PTB;
+  uint4 nv0 = make_uint4(0u, 0u, 0u, 0u), nv1 = nv0;
+  float ncs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  if (blockIdx.x * PTB + tid < NB32) fetch(blockIdx.x * PTB + tid, nv0, nv1, ncs4);
+  for (unsigned blk = blockIdx.x * PTB + tid; blk < NB32; blk += stride) {
+    const unsigned j = blk % nbk32;
+    const uint4 v0 = nv0, v1 = nv1;
+    float cs4[4] = {ncs4[0], ncs4[1], ncs4[2], ncs4[3]};
+    if (blk + stride < NB32) fetch(blk + stride, nv0, nv1, ncs4);
     const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
     float w[16], c[16];
 #pragma unroll
