@@ -84,6 +84,20 @@ __device__ __forceinline__ QScale scale_quantize(float sigma, int k, const FmtDe
   if (!(sigma > 0.0f)) return r;
   const uint32_t b = __float_as_uint(sigma);
   int e = (int)(b >> 23);
+  {
+    // The usual case: the shifted value lies in the format's normal range below its top binade (so that a
+    // carry out of the mantissa cannot pass the largest code) and the format keeps at least one mantissa
+    // bit.  Rounding to nearest even on y bits is then one integer addition on the fp32 pattern; the shift
+    // k moves only the exponent, so the decoded scale is the rounded value itself.
+    const int ev0 = e - 127 + k;
+    if (e != 0 && f.y >= 1 && ev0 >= f.emin && ev0 < f.emax) {
+      const int sh0 = 23 - f.y;
+      const uint32_t rb = (b + ((1u << (sh0 - 1)) - 1u) + ((b >> sh0) & 1u)) & ~((1u << sh0) - 1u);
+      r.s_hat = __uint_as_float(rb);
+      r.code = (uint32_t)(((int)(rb >> 23) - 127 + k + f.bias) << f.y) | ((rb >> sh0) & ((1u << f.y) - 1u));
+      return r;
+    }
+  }
   uint32_t m = b & 0x7FFFFFu;
   if (e == 0) {
     const int sh = __clz((int)m) - 8;
