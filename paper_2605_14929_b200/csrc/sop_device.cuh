@@ -146,8 +146,9 @@ __device__ __forceinline__ float fp_quantize(float u) {
   constexpr int min_eb = KIND == SOP_KIND_FP_E2M3 ? 127 : 121;
   constexpr float vmax = KIND == SOP_KIND_FP_E2M3 ? 7.5f : 448.0f;
   const float au = fminf(fabsf(u), vmax);
-  const int eb = (int)(__float_as_uint(au) >> 23);
-  const float magic = __uint_as_float((uint32_t)(max(eb, min_eb) + 20) << 23);
+  // 2^(exponent of au, at least the smallest normal one) * 2^20: adding and subtracting it rounds au to a
+  // multiple of the binade's step (3 mantissa bits), ties to even
+  const float magic = __uint_as_float(max(__float_as_uint(au) & 0x7F800000u, (uint32_t)min_eb << 23) + (20u << 23));
   const float q = __fsub_rn(__fadd_rn(au, magic), magic);
   return __uint_as_float(__float_as_uint(q) | (__float_as_uint(u) & 0x80000000u));
 }
@@ -158,8 +159,7 @@ struct GridDev { int min_eb, sh; float vpos, vneg; };
 
 __device__ __forceinline__ float grid_quantize(float u, const GridDev g) {
   const float au = fminf(fabsf(u), u < 0.0f ? g.vneg : g.vpos);
-  const int eb = (int)(__float_as_uint(au) >> 23);
-  const float magic = __uint_as_float((uint32_t)(max(eb, g.min_eb) + g.sh) << 23);
+  const float magic = __uint_as_float(max(__float_as_uint(au) & 0x7F800000u, (uint32_t)g.min_eb << 23) + ((uint32_t)g.sh << 23));
   const float q = __fsub_rn(__fadd_rn(au, magic), magic);     // nearest multiple of the binade's step, ties to even
   return __uint_as_float(__float_as_uint(q) | (__float_as_uint(u) & 0x80000000u));
 }
