@@ -19,8 +19,9 @@
  *     the device per process (kernel attributes set once, the number of SMs, whether all Lloyd iterations
  *     fit one cooperative launch): one process drives one device, and calls are made from one host thread
  *     at a time.
- *   - Every entry point can be recorded into a CUDA graph by stream capture once it has been called
- *     normally on the device (the first call does the one-time set-ups), with profiling off.
+ *   - sop_channel_norms, sop_pair_search, sop_dd4_lloyd and sop_pack can be recorded into a CUDA graph by
+ *     stream capture once each has been called normally on the device (the first call does the one-time
+ *     set-ups), with profiling off.
  */
 #ifndef SOP_H_
 #define SOP_H_
