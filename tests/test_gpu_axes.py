@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2605_14929_b200 import inputs as I
 
-from .test_gpu_parity import B, REL, assert_tables, dev, gpu_pack  # noqa: F401  (B is a fixture)
+from .test_gpu_parity import B, REL, assert_tables, dev  # noqa: F401  (B is a fixture)
 
 pytestmark = pytest.mark.gpu
 

@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2605_14929_b200 import inputs as I
 
-from .test_gpu_parity import B, REL, assert_tables, dev, gpu_search, gpu_pack  # noqa: F401  (B is a fixture)
+from .test_gpu_parity import B, assert_tables, gpu_search, gpu_pack  # noqa: F401  (B is a fixture)
 
 pytestmark = pytest.mark.gpu
 

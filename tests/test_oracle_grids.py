@@ -2,7 +2,6 @@
 is pinned to the numbers the paper prints (80 / 96 values, ratios 120 / 240, E2M5 tops out at 3.94),
 to the two element formats that already have their own pinned quantiser (E2M3, E4M3), and to an
 exact-rational nearest-value search over the enumerated grid."""
-import dataclasses
 import os
 from fractions import Fraction
 
