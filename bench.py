@@ -1,12 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the SOP per-layer candidate sweep on B200.
 
-One step = one pass of the whole hot path over one synthetic layer: channel norms, sweep of every fixed
-candidate (single-candidate reduction: finds FMTa), DD4 Lloyd refinement, sweep of the two DD4 columns
-with the fixed candidates' per-block values loaded (all pairs), pack of the chosen pair.
-Workload at every N: the attention-projection configuration (W 4096 x 4096 bf16 with 1 % outlier
-channels, X 512 x 4096, E5M6 scale, NF4/SH4/BOF4/Split87/DD4 and negations plus E2M3/E4M3 singles).
-With N > 1 every rank sweeps its own layer (layers are independent: no data-path collective).
+Workload at every N: the 70B-shaped layer set (the largest single-GPU configuration): the five layers of one
+transformer block (8192 x 8192, 1024 x 8192 twice, 28672 x 8192, 8192 x 28672, bf16, Student-t(5) * 0.02 with
+lognormal(0, 1.2) input-channel scales, X 1024 x K), generated on the device from the seed, each swept at the
+eight scale formats of the paper's scale-format table with the full n = 4 alphabet (NF4, SH4, BOF4, Split87,
+DD4 by 8 Lloyd iterations, and their negations; every pair).  The model has 80 such blocks with layers that are
+independent and identically distributed by seed; one block is the streamed unit and the timed subset.
+
+One step = one pass of the whole hot path over that block: per layer the channel norms, then per scale format
+the sweep of every fixed candidate (finds FMTa), the DD4 Lloyd refinement, the sweep of the two DD4 columns
+(every pair), and the pack of the chosen pair.  The metric counts a weight element once per scale format.
+With N > 1 every rank sweeps its own transformer block (layers are independent: no data-path collective).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -29,25 +34,54 @@ if ROOT not in sys.path:
 
 METRIC = "G weight-elems/s through full alphabet pair sweep"
 UNIT = "G weight-elems/s"
-WORKLOAD = dict(workload="config2: attention projection 4096x4096 bf16, 1% outlier channels x20, X 512x4096, "
-                         "E5M6 scale, NF4/SH4/BOF4/Split87/DD4(8 Lloyd iters) + negations + E2M3/E4M3, all pairs",
-                M=4096, K=4096, T=512, scale_format="E5M6", rom=["NF4", "SH4", "BOF4", "Split87"], fp=["E2M3", "E4M3"],
-                lloyd_iters=8, g=16)
+ROM4 = ["NF4", "SH4", "BOF4", "Split87"]
+SCALE_FORMATS = ["UE4M4", "E4M3", "UE4M6", "E4M5", "UE5M7", "E5M6", "E4M7", "E8M7"]
+WORKLOAD = dict(
+    workload="config5: 70B-shaped layer set, transformer block b of 80 (layers are iid by seed: one block is the timed subset): "
+             "8192x8192, 1024x8192 x2, 28672x8192, 8192x28672 bf16, Student-t(5)*0.02, lognormal(0,1.2) channel scales, "
+             "X 1024xK, generated on device; NF4/SH4/BOF4/Split87/DD4(8 Lloyd iters) + negations, all pairs, at the "
+             "eight scale formats UE4M4 E4M3 UE4M6 E4M5 UE5M7 E5M6 E4M7 E8M7",
+    layers=["8192x8192", "1024x8192", "1024x8192", "28672x8192", "8192x28672"], T=1024, scale_formats=SCALE_FORMATS,
+    rom=ROM4, fp=[], lloyd_iters=8, g=16)
+# config 2 (the attention projection), kept for the per-config table and the full-size parity test
+CONFIG2 = dict(M=4096, K=4096, T=512, scale_format="E5M6", rom=ROM4, fp=["E2M3", "E4M3"], lloyd_iters=8)
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 
-
-def sweep_ops_per_element(n_lut: int, n_bits: int, n_fp: int, n_loaded: int, n_slots2: int, n_slots4: int) -> float:
-    """Algorithmic thread-level operations per weight element of one sweep launch: 6 shared (unpack,
-    absmax, c w, norm, u), 2n + 5 per evaluated LUT candidate (n-step search + reconstruct + 4 fused
-    multiply-adds), 12 per evaluated FP candidate, and per block: 6 per evaluated candidate (sqrt,
-    divide, products), 2 per loaded candidate, 2 per two-way table entry and 6 per four-way entry."""
-    n_eval = n_lut + n_fp
-    return 6 + n_lut * (2 * n_bits + 5) + n_fp * 12 + (6 * n_eval + 2 * n_loaded + 2 * n_slots2 + 6 * n_slots4) / 16.0
+# DRAM traffic of the sweep kernel per weight element and launch, from the ncu capture summarised in the named
+# file (dram__bytes_read.sum + dram__bytes_write.sum of one launch on a reduced-row layer divided by its
+# elements; traffic grows in proportion to the rows).  None: no capture of the kernel as it is now.
+NCU_SWEEP_TRAFFIC = dict(source=None, bytes_per_element_fixed_candidates=None, bytes_per_element_dd_columns=None)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of the sweep kernel on this
-# workload (cold cache; see the summary under profiles/); average over the two launches of one step
-NCU_TRAFFIC_BYTES = dict(sweep_kernel=93.1e6)
+# ---------------------------------------------------------------------------------------------------------
+# operation and byte models of the search (both sweep launches together), per weight element
+# ---------------------------------------------------------------------------------------------------------
+def search_ops_n_step(n_lut: int, n_bits: int, n_fp: int) -> float:
+    """The operation count of an n-step nearest-entry search: 6 shared (unpack, absmax, c w, norm, u), 2n + 5 per
+    LUT candidate (n compare-select steps, fetch, four multiply-adds), 12 per FP candidate; per block 2 per pair of
+    LUT candidates (diagonal included) and 6 per candidate."""
+    pairs = n_lut * (n_lut + 1) // 2
+    return 6 + n_lut * (2 * n_bits + 5) + n_fp * 12 + (2 * pairs + 6 * (n_lut + n_fp)) / 16.0
+
+
+def search_ops_cell_lookup(n_lut: int, n_bits: int, n_fp: int, n_dd: int, signed: bool) -> float:
+    """The operation count of the search as this library does it: W is unpacked in both launches (6 each); a LUT
+    candidate costs 4 for the cell lookup (fetch, compare, select, unpack) and 5 packed multiply-adds on element
+    pairs (2.5 per element) whatever n is; an FP candidate 12; per block 6 per evaluated candidate, 2 per
+    candidate loaded by the second launch, 2 per pair entry (diagonal included), and with a signed scale 4 per
+    base atom (the better of the atom and its negation) plus 2 per four-way entry."""
+    pairs = n_lut * (n_lut + 1) // 2
+    n_base = n_lut // 2 if signed else 0
+    four = n_base * (n_base + 1) // 2
+    per_block = 6 * (n_lut + n_fp) + 2 * (n_lut + n_fp - n_dd) + 2 * (pairs + n_fp) + 4 * n_base + 2 * four
+    return 12 + n_lut * 6.5 + n_fp * 12 + per_block / 16.0
+
+
+def search_bytes(n_cand: int, n_dd: int) -> float:
+    """Algorithmic DRAM bytes per element of the two launches as the call plan has them: W (2 bytes) read by each,
+    8 bytes per block for every candidate written (per-block cosine and error: the Lloyd pool and the pack read
+    them) and 8 per block for every fixed candidate the second launch loads."""
+    return 2 * 2.0 + (8.0 * n_cand + 8.0 * (n_cand - n_dd)) / 16.0
 
 
 class ClockSampler:
@@ -78,52 +112,61 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                pw.append(float(r[2]))
             except (ValueError, IndexError):
                 continue
             for nm, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
-        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+        # "under load": the samples taken while the GPU drew more than half of the largest power seen
+        load = [s for s, p in zip(sm, pw) if pw and p >= 0.5 * max(pw)]
+        return dict(sm_mhz=statistics.median(load or sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm), samples_under_load=len(load),
+                    power_w_max=max(pw) if pw else None)
 
 
 def make_layer(seed: int):
+    """The attention-projection layer of configuration 2 (host tensors)."""
     from paper_2605_14929_b200 import inputs as I
-    return I.config2(seed, WORKLOAD["M"], WORKLOAD["K"], WORKLOAD["T"])
+    return I.config2(seed, CONFIG2["M"], CONFIG2["K"], CONFIG2["T"])
 
 
-def cpu_oracle_time(rows: int, seed: int = 0):
-    """Times the oracle pipeline, as it stands, on the first ``rows`` rows of the workload's layer."""
+# ---------------------------------------------------------------------------------------------------------
+# the CPU oracle as a baseline: a bounded sample of the same workload
+# ---------------------------------------------------------------------------------------------------------
+def cpu_oracle_time(rows: int, fmt_name: str = "E5M6"):
+    """Times the oracle pipeline, as it stands, on the first ``rows`` rows of the workload's 8192 x 8192 layer at one
+    scale format (channel norms over the whole X, both searches, Lloyd, pack), single thread."""
     from paper_2605_14929_b200 import inputs as I
     from tests import oracle_pipeline
-    L = make_layer(seed)
-    sub = I.Layer(L.W[:rows].contiguous(), L.X)
+    L = I.config5_layer(0, 0, 0, rows=rows)
     t0 = time.perf_counter()
-    oracle_pipeline.run(sub, I.scale_format(WORKLOAD["scale_format"]), WORKLOAD["rom"], WORKLOAD["fp"], WORKLOAD["lloyd_iters"])
+    oracle_pipeline.run(L, I.scale_format(fmt_name), WORKLOAD["rom"], WORKLOAD["fp"], WORKLOAD["lloyd_iters"])
     dt = time.perf_counter() - t0
-    return rows * WORKLOAD["K"] / dt / 1e9, dt
+    return rows * 8192 / dt / 1e9, dt
 
 
 def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    rows = 128
-    for _ in range(args.warmup):
-        cpu_oracle_time(64)
+    rows = 64
+    for _ in range(min(args.warmup, 2)):
+        cpu_oracle_time(16)
     times = []
     for _ in range(args.steps):
         _, dt = cpu_oracle_time(rows)
         times.append(dt)
     ms = 1e3 * sum(times) / len(times)
-    value = rows * WORKLOAD["K"] / (ms * 1e-3) / 1e9
-    sample = f"first {rows} of {WORKLOAD['M']} rows per step, full alphabet and pipeline, single thread"
+    value = rows * 8192 / (ms * 1e-3) / 1e9
+    sample = (f"per step the first {rows} of 8192 rows of the 8192x8192 layer at E5M6 (1 of 5 layers, 1 of 8 scale formats), "
+              "full alphabet and pipeline, single thread")
     print(json.dumps(dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                           warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
                           dtype="f32", data="synthetic", config=WORKLOAD,
@@ -131,11 +174,123 @@ def run_reference(args) -> None:
                           e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
 
 
+# ---------------------------------------------------------------------------------------------------------
+# the other configurations: short timings for the per-config table (rank 0, N = 1)
+# ---------------------------------------------------------------------------------------------------------
+def time_sweeps(sweeps, reps, flush):
+    """Whole-path and sweep-only time (ms, medians) of a list of (sweep, W, X, norms) passes launched call by call;
+    ``flush`` is a buffer larger than L2 that is rewritten before every pass, or None."""
+    import torch
+    from paper_2605_14929_b200 import binding as B
+    st = torch.cuda.current_stream()
+
+    def one():
+        for sw, W, X, norms in sweeps:
+            sw.run(W, X, st, norms=norms)
+    for _ in range(3):
+        one()
+    torch.cuda.synchronize()
+    whole, sweep = [], []
+    B.profile_enable(True)
+    for _ in range(reps):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        t_sw = 0.0
+        for sw, W, X, norms in sweeps:
+            sw.run(W, X, st, norms=norms)
+            t_sw += B.profile_ms(B.PROFILE_SWEEP, 0) + (B.profile_ms(B.PROFILE_SWEEP, 1) if sw.iters > 0 else 0.0)
+        e1.record(st)
+        torch.cuda.synchronize()
+        whole.append(e0.elapsed_time(e1))
+        sweep.append(t_sw)
+    B.profile_enable(False)
+    return statistics.median(whole), statistics.median(sweep)
+
+
+def per_config_table(dev, alu_peak, flush):
+    """Configurations 1 to 4 at full size: G elements/s through the whole hot path and through the sweep launches
+    alone, with the operation count per element and the fraction of the issue peak it amounts to."""
+    import torch
+    from paper_2605_14929_b200 import binding as B, inputs as I
+    from paper_2605_14929_b200.pipeline import LayerSweep
+    out = {}
+
+    def entry(name, sweeps, elements, ops, note, fl):
+        whole, sweep = time_sweeps(sweeps, 5, fl)
+        out[name] = dict(elements_times_formats=elements, whole_path=dict(value=elements / whole / 1e6, unit=UNIT, ms=whole),
+                         sweep_only=dict(value=elements / sweep / 1e6, unit=UNIT, ms=sweep), ops_per_element_n_step=ops,
+                         frac_of_alu_peak=ops * elements / (sweep * 1e-3) / 1e12 / alu_peak, note=note)
+
+    # 1: single small layer, signed UE4M4, three ROM atoms
+    L = I.config1(0)
+    sw = LayerSweep(256, 1024, 128, I.scale_format("S1E4M4"), ["NF4", "SH4", "BOF4"], [], 0, device=dev)
+    entry("config1", [(sw, L.W.to(dev), L.X.to(dev), True)], 256 * 1024, search_ops_n_step(6, 4, 0),
+          "256x1024, S1E4M4, NF4/SH4/BOF4 + negations, no DD atom; launch-latency sized (one wave of 32 CTAs)", flush)
+    # 2: attention projection
+    L = make_layer(0)
+    sw = LayerSweep(CONFIG2["M"], CONFIG2["K"], CONFIG2["T"], I.scale_format("E5M6"), CONFIG2["rom"], CONFIG2["fp"], 8, device=dev)
+    entry("config2", [(sw, L.W.to(dev), L.X.to(dev), True)], CONFIG2["M"] * CONFIG2["K"], search_ops_n_step(10, 4, 2),
+          "4096x4096, E5M6, 10 LUT candidates + E2M3/E4M3, all pairs; L2 flushed between passes", flush)
+    del sw
+    # 3: the seven layers of one 7B-shaped transformer block, FP6 per block against FP8 per layer (singles only)
+    fmt = I.scale_format("UE4M4")
+    fp = ["E2M3", "E4M3^0"]
+    sweeps, elements, own = [], 0, {}
+    for which, (_, M, K) in enumerate(I.SHAPES_7B):
+        Lw = I.config3_layer(0, 0, which, device=str(dev))
+        sw = own.get((M, K))
+        if sw is None:
+            sw = own[(M, K)] = LayerSweep(M, K, 512, fmt, [], fp, 0, device=dev)
+        sweeps.append((sw, Lw.W, Lw.X, True))
+        elements += M * K
+    entry("config3", sweeps, elements, search_ops_n_step(0, 4, 2),
+          "block 0 of 32 (seven layers, 218 M elements > L2), E2M3sUE4M4 vs E4M3^0: two FP singles, no pairs, no DD atom, pack of the FP6 single", None)
+    del sweeps, own
+    torch.cuda.empty_cache()
+    # 4: the n = 5 MLP pair at both scale formats
+    sweeps, elements = [], 0
+    for which in (0, 1):
+        Lw = I.config4_layer(0, which, device=str(dev))
+        M, K = Lw.W.shape
+        first = None
+        for f in ("UE4M4", "E5M6"):
+            sw = LayerSweep(M, K, 2048, I.scale_format(f), ["NF5", "SH5", "BOF5", "E2M2"], [], 16, device=dev, share=first)
+            first = first or sw
+            sweeps.append((sw, Lw.W, Lw.X, f == "UE4M4"))
+            elements += M * K
+    entry("config4", sweeps, elements, search_ops_n_step(10, 5, 0),
+          "14336x4096 and 4096x14336 at UE4M4 and E5M6, 32-entry atoms, DD5 by 16 Lloyd iterations, all pairs", None)
+    del sweeps
+    torch.cuda.empty_cache()
+    return out
+
+
+# ---------------------------------------------------------------------------------------------------------
+# N > 1 bookkeeping (no data-path collective: the ranks only agree on the slowest time)
+# ---------------------------------------------------------------------------------------------------------
+def block_for_rank(rank: int) -> int:
+    """Layer-parallel sharding of the model sweep: rank r takes transformer block r (all blocks come from seed 0)."""
+    return rank
+
+
+def reduce_times(named: dict, device, world: int) -> dict:
+    """The largest value of every named time over the ranks (every rank gets the result)."""
+    import torch
+    import torch.distributed as dist
+    keys = sorted(named)
+    t = torch.tensor([float(named[k]) for k in keys], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return dict(zip(keys, (float(x) for x in t.cpu())))
+
+
 def run_gpu(args) -> None:
     import torch
     import torch.distributed as dist
-    from paper_2605_14929_b200 import binding as B, inputs as I
-    from paper_2605_14929_b200.pipeline import LayerSweep
+    from paper_2605_14929_b200 import binding as B, inputs as I, pipeline
+    from paper_2605_14929_b200.pipeline import LayerSetSweep, LayerStream
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -149,13 +304,15 @@ def run_gpu(args) -> None:
         dist.init_process_group("nccl", device_id=dev)
     B.lib()
 
-    M, K, T = WORKLOAD["M"], WORKLOAD["K"], WORKLOAD["T"]
-    fmt = I.scale_format(WORKLOAD["scale_format"])
-    L = make_layer(rank)                                  # every rank sweeps its own layer
-    Wh, Xh = L.W.pin_memory(), L.X.pin_memory()
-    Wd, Xd = Wh.to(dev), Xh.to(dev)
-    sw = LayerSweep(M, K, T, fmt, WORKLOAD["rom"], WORKLOAD["fp"], WORKLOAD["lloyd_iters"], device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
+    fmts = [I.scale_format(f) for f in WORKLOAD["scale_formats"]]
+    S = len(fmts)
+    block = block_for_rank(rank)                                  # every rank sweeps its own transformer block
+    layers = [I.config5_layer(0, block, which, device=str(dev)) for which in range(len(I.SHAPES_70B))]
+    dev_layers = [(L.W, L.X) for L in layers]
+    shapes = [(L.W.shape[0], L.W.shape[1], L.X.shape[0]) for L in layers]
+    sset = LayerSetSweep(shapes, fmts, WORKLOAD["rom"], WORKLOAD["fp"], WORKLOAD["lloyd_iters"], device=dev)
+    E = sset.elements                                             # weight elements of the block
+    units = float(E * S)                                          # the metric counts an element once per scale format
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -164,28 +321,28 @@ def run_gpu(args) -> None:
         torch.cuda.synchronize()
 
     def one_step(launch):
-        flush.fill_(1)                                    # evict W / X from L2 between timed steps
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         launch()
         e1.record(stream)
         return e0, e1
 
-    # The timed steps replay the layer's calls as one CUDA graph (what a job that sweeps many layers of one shape
-    # does).  A replayed graph gives no per-kernel events, so the same number of steps is then run call by call
-    # with the library's events around its main kernels: those times feed the roofline object.
+    # The timed steps replay the block's calls as one CUDA graph (what a job that sweeps 80 such blocks does).  A
+    # replayed graph gives no per-kernel events, so one more pass is run call by call with the library's events
+    # around its main kernels: those times feed the roofline object.
     launch_kind = "one CUDA graph replay per step"
-    step_launch = sw.replay
+    step_launch = sset.replay
     try:
-        sw.capture(Wd, Xd)
+        sset.capture(dev_layers)
     except RuntimeError as exc:                           # no graph capture here: time the calls themselves
         sys.stderr.write(f"graph capture failed ({exc}); timing call by call\n")
         torch.cuda.synchronize()
         launch_kind = "call by call (graph capture failed)"
-        step_launch = lambda: sw.run(Wd, Xd, stream)
+        step_launch = lambda: sset.run(dev_layers, stream)
     for _ in range(max(3, args.warmup)):
         one_step(step_launch)
     barrier()
+    sset.check()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -196,112 +353,147 @@ def run_gpu(args) -> None:
     barrier()
     t_wall = time.perf_counter() - t_wall
     step_ms = [a.elapsed_time(b) for a, b in evs]
-
-    B.profile_enable(True)
-    kern = dict(sweep1=[], sweep2=[], lloyd=[], pack=[], norms=[])
-    evs2 = []
-    for _ in range(args.steps):
-        evs2.append(one_step(lambda: sw.run(Wd, Xd, stream)))
-        # the library's own events around its main kernels, on the launching stream (waits for this step)
-        kern["sweep2"].append(B.profile_ms(B.PROFILE_SWEEP, 0))
-        kern["sweep1"].append(B.profile_ms(B.PROFILE_SWEEP, 1))
-        kern["lloyd"].append(B.profile_ms(B.PROFILE_LLOYD, 0))
-        kern["pack"].append(B.profile_ms(B.PROFILE_PACK, 0))
-        kern["norms"].append(B.profile_ms(B.PROFILE_NORMS, 0))
-    barrier()
-    call_ms = sum(a.elapsed_time(b) for a, b in evs2) / len(evs2)
     clocks = sampler.stop() if rank == 0 else {}
+
+    # ---- one pass call by call: per (layer, format) the library's events around its main kernels ----
+    B.profile_enable(True)
+    kern = dict(sweep1=0.0, sweep2=0.0, lloyd=0.0, pack=0.0, norms=0.0)
+    per_layer_sweep_ms = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for row, (W, X) in zip(sset.sweeps, dev_layers):
+        t_layer = 0.0
+        for f, sw in enumerate(row):
+            sw.run(W, X, stream, norms=(f == 0))
+            s2, s1 = B.profile_ms(B.PROFILE_SWEEP, 0), B.profile_ms(B.PROFILE_SWEEP, 1)
+            kern["sweep2"] += s2
+            kern["sweep1"] += s1
+            kern["lloyd"] += B.profile_ms(B.PROFILE_LLOYD, 0)
+            kern["pack"] += B.profile_ms(B.PROFILE_PACK, 0)
+            if f == 0:
+                kern["norms"] += B.profile_ms(B.PROFILE_NORMS, 0)
+            t_layer += s1 + s2
+        per_layer_sweep_ms.append(t_layer)
+    e1.record(stream)
+    barrier()
+    call_ms = e0.elapsed_time(e1)
     B.profile_enable(False)
 
-    # ---- end to end through the public API with host buffers: H2D of W and X, the path, D2H of the results ----
-    # end to end through the streaming API: every step copies its W and X from pinned host memory and reads its
-    # results (tables, result block, codes, scale words) back; copies of neighbouring steps overlap the sweep
-    from paper_2605_14929_b200.pipeline import LayerStream
-    ls = LayerStream(sw)
-    ls.before_run = lambda: flush.fill_(1)          # same L2 eviction as the device-resident timing
-    h2d, d2h = ls.h2d_bytes, ls.d2h_bytes
-    for i in range(3):
-        ls.submit(i, Wh, Xh)
-    ls.collect(2)
+    # ---- end to end through the streaming API with host buffers: every step copies the block's W and X from
+    #      pinned host memory and reads every (layer, format)'s results (tables, result block, codes, scale
+    #      words, distortion trace) back; the copies overlap the sweeps of the neighbouring layers ----
+    host_layers = [(L.W.cpu().pin_memory(), L.X.cpu().pin_memory()) for L in layers]
+    streams = (torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev))
+    ls_of, order = {}, []
+    for row, shape in zip(sset.sweeps, shapes):
+        if shape not in ls_of:
+            ls_of[shape] = LayerStream(row, streams)
+        order.append(ls_of[shape])
+    h2d = sum(ls.h2d_bytes for ls in order)
+    d2h = sum(ls.d2h_bytes for ls in order)
+    count = {id(ls): 0 for ls in order}
+
+    def e2e_step():
+        for ls, (Wh, Xh) in zip(order, host_layers):
+            i = count[id(ls)]
+            ls.submit(i, Wh, Xh)
+            if i:
+                ls.collect(i - 1)
+            count[id(ls)] = i + 1
+    for _ in range(2):
+        e2e_step()
+    for ls in set(order):
+        ls.collect(count[id(ls)] - 1)
     barrier()
+    e2e_steps = max(2, min(args.steps, 10))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(ls.s_in)
-    for i in range(args.steps):
-        ls.submit(i, Wh, Xh)
-        if i:
-            ls.collect(i - 1)
-    ls.collect(args.steps - 1)
-    e1.record(ls.s_out)
+    e0.record(streams[0])
+    for _ in range(e2e_steps):
+        e2e_step()
+    for ls in set(order):
+        ls.collect(count[id(ls)] - 1)
+    e1.record(streams[2])
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / args.steps
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    del order, ls_of, host_layers
 
     ms = sum(step_ms) / len(step_ms)
-    from paper_2605_14929_b200 import pipeline
-    job_value = pipeline.job_throughput(float(M * K), ms * 1e-3) / 1e9   # all ranks' elements / slowest rank's time
-    kavg = {k: sum(v) / len(v) for k, v in kern.items()}
-    knames = sorted(kavg)
-    t = torch.tensor([ms, e2e_ms] + [kavg[k] for k in knames], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    vals = [float(x) for x in t.cpu()]
-    ms, e2e_ms = vals[0], vals[1]
-    kavg = dict(zip(knames, vals[2:]))
-    E = M * K
+    job_value = pipeline.job_throughput(units, ms * 1e-3) / 1e9   # all ranks' element-formats / slowest rank's time
+    red = reduce_times(dict(kern, _ms=ms, _e2e_ms=e2e_ms, _call_ms=call_ms), dev, world)      # the slowest rank's, each
+    ms, e2e_ms, call_ms = red.pop("_ms"), red.pop("_e2e_ms"), red.pop("_call_ms")
+    kern = red
     if rank == 0:
         peaks = {}
         try:
             peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
         except OSError:
             pass
-        full = sw.full_atoms
-        nb = full[0].n_bits
-        n_lut = sum(a.kind == I.KIND_LUT for a in full)
-        n_fp = len(full) - n_lut
-        n_dd = bin(sw.dd_mask).count("1")
-        n_base = (n_lut // 2) if fmt.sign_bits else 0
-        slots2 = len(full) + n_lut * (n_lut - 1) // 2
-        slots4 = n_base * (n_base + 1) // 2
-        ops1 = sweep_ops_per_element(n_lut - n_dd, nb, n_fp, 0, len(full) - n_dd, 0)      # fixed candidates, singles only
-        ops2 = sweep_ops_per_element(n_dd, nb, 0, len(full) - n_dd, slots2, slots4)       # DD columns, every pair
         sm_max = peaks.get("sm_max_mhz", 1965.0)
         alu_peak = SM_COUNT * SCHEDULERS * LANES * sm_max * 1e6 / 1e12          # T thread-instructions/s
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
         of = "measured" if peaks else "fallback"
-        # sweep kernel: two launches per step; achieved = algorithmic ops of both / time of both
-        sweep_t = (kavg["sweep1"] + kavg["sweep2"]) * 1e-3
-        sweep_ach = (ops1 + ops2) * E / sweep_t / 1e12
-        sweep_roof = dict(kernel="sweep_kernel", launches_per_step=2, bound="alu", achieved=sweep_ach, peak=alu_peak,
-                          unit="T thread-instr/s", frac=sweep_ach / alu_peak,
-                          traffic=NCU_TRAFFIC_BYTES["sweep_kernel"] if (M, K) == (4096, 4096) else None,
-                          peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz (clocks.max.sm, {of})",
-                          ops_per_element=dict(fixed_candidates_singles=ops1, dd_columns_all_pairs=ops2),
-                          avg_launch_ms=sweep_t * 1e3 / 2,
-                          hbm=dict(achieved=2 * 2.0 * E / sweep_t / 1e9, peak=hbm_peak, unit="GB/s",
-                                   frac=2 * 2.0 * E / sweep_t / 1e9 / hbm_peak, of=of,
-                                   note="W read once per launch; the kernel is far from the HBM roofline"))
-        # the Lloyd iterations walk only the pool elements in cells that hold a decision threshold (a few per
-        # cent of the pool), so their launches are bound by launch and dependency latency, not by a roofline
-        dominant = sweep_roof
-        cpu_rows = 1024
+        n_lut, nb = len(sset.sweeps[0][0].full_atoms), 4
+        signed = [bool(f.sign_bits) for f in fmts]
+        ops_n_step = search_ops_n_step(n_lut, nb, 0)
+        ops_cell = sum(search_ops_cell_lookup(n_lut, nb, 0, 2, s) for s in signed) / S
+        sweep_t = (kern["sweep1"] + kern["sweep2"]) * 1e-3              # all 2 * 5 * 8 sweep launches of a step
+        n_launch = 2 * len(shapes) * S
+        ach = ops_n_step * units / sweep_t / 1e12
+        ach_cell = ops_cell * units / sweep_t / 1e12
+        alg_bytes = search_bytes(n_lut, 2)
+        bpe = [NCU_SWEEP_TRAFFIC["bytes_per_element_fixed_candidates"], NCU_SWEEP_TRAFFIC["bytes_per_element_dd_columns"]]
+        traffic = None if None in bpe else (bpe[0] + bpe[1]) / 2.0 * units / (n_launch / 2)
+        roofline = dict(
+            kernel="sweep_kernel", launches_per_step=n_launch, bound="alu", achieved=ach, peak=alu_peak, unit="T thread-instr/s",
+            frac=ach / alu_peak, traffic=traffic, traffic_source=NCU_SWEEP_TRAFFIC["source"],
+            peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz (clocks.max.sm, {of})",
+            avg_launch_ms=sweep_t * 1e3 / n_launch,
+            models=dict(
+                n_step_search=dict(ops_per_element=ops_n_step, achieved=ach, frac=ach / alu_peak,
+                                   note="operation count of an n-step nearest-entry search (2n + 5 per LUT candidate and element); "
+                                        "roofline.frac is this one"),
+                cell_lookup=dict(ops_per_element=ops_cell, achieved=ach_cell, frac=ach_cell / alu_peak,
+                                 note="operation count of the kernel's own scheme: one-step cell lookup (4) and packed multiply-adds "
+                                      "(2.5) per LUT candidate and element, W unpacked in both launches, loaded columns, signed entries")),
+            algorithmic_bytes_per_launch=alg_bytes / 2.0 * units / (n_launch / 2),
+            bytes_per_element=dict(algorithmic=alg_bytes, w_twice=4.0, over_w_twice=alg_bytes / 4.0),
+            hbm=dict(achieved=alg_bytes * units / sweep_t / 1e9, peak=hbm_peak, unit="GB/s",
+                     frac=alg_bytes * units / sweep_t / 1e9 / hbm_peak, of=of,
+                     note="algorithmic bytes of both launches (W twice, per-block values written and loaded) over their time: "
+                          "the sweep is far from the HBM roofline"))
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        try:
+            per_config = per_config_table(dev, alu_peak, flush) if world == 1 else None
+        except Exception as exc:                               # the headline line does not depend on the side table
+            per_config = dict(error=repr(exc))
+        if per_config is not None and "error" not in per_config:
+            per_config["config5"] = dict(elements_times_formats=units, whole_path=dict(value=units / ms / 1e6, unit=UNIT, ms=ms),
+                                         sweep_only=dict(value=units / (sweep_t * 1e3) / 1e6, unit=UNIT, ms=sweep_t * 1e3),
+                                         ops_per_element_n_step=ops_n_step, frac_of_alu_peak=ach / alu_peak,
+                                         note="the headline workload: block 0, five layers, eight scale formats")
+        cpu_rows = 384
         cpu_val, cpu_dt = cpu_oracle_time(cpu_rows)
         line = dict(
             metric=METRIC, value=job_value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=max(3, args.warmup), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
-            dtype="f32", data="synthetic", config=dict(WORKLOAD, l2="flushed between timed steps (256 MB write)", launch=launch_kind,
-                                                       parallelism=f"layer-parallel x{world}, no collective"),
-            kernels_ms=dict(kavg, ms_per_step_call_by_call=call_ms,
-                            note="per step of a second pass of the same number of steps launched call by call (a replayed graph "
-                                 "gives no per-kernel events), CUDA events recorded by the library around its main kernels; "
-                                       "sweep1 = fixed candidates (singles), sweep2 = DD columns (all pairs), "
-                                       "lloyd = all Lloyd iterations (one cooperative launch where the grid fits)"),
-            sweep_only=dict(value=world * E / sweep_t / 1e9, unit=UNIT,
-                            note="elements / time of the two sweep launches of a step (every candidate, every pair)"),
-            roofline=dominant,
+            dtype="f32", data="synthetic",
+            config=dict(WORKLOAD, block=f"rank r sweeps block r (seed 0)", elements_per_step=E, element_formats_per_step=units,
+                        l2="inputs larger than L2: 1.1 GB of W per step, every layer above 126 MB except the two 1024x8192 ones; "
+                           "a layer's eight formats run back to back, as in a real sweep, so its W may be served from L2 there",
+                        launch=launch_kind, parallelism=f"layer-parallel x{world}, no collective"),
+            kernels_ms=dict(kern, ms_per_step_call_by_call=call_ms, sweep_ms_per_layer=dict(zip(WORKLOAD["layers"], per_layer_sweep_ms)),
+                            note="sums over the 40 (layer, format) passes of one step launched call by call, CUDA events recorded "
+                                 "by the library around its main kernels; sweep1 = fixed candidates (finds FMTa), sweep2 = DD "
+                                 "columns (all pairs), lloyd = the iteration launches only, norms once per layer"),
+            sweep_only=dict(value=world * units / sweep_t / 1e9, unit=UNIT,
+                            note="element-formats / time of the sweep launches of a step (every candidate, every pair)"),
+            roofline=roofline, per_config=per_config,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
-                              sample=f"first {cpu_rows} of {M} rows, whole pipeline, {cpu_dt:.1f} s"),
-            e2e=dict(value=world * E / (e2e_ms * 1e-3) / 1e9, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-                     ms_per_step=e2e_ms),
-            gpu_launches=sw.kernel_launches_per_step * args.steps, clocks=clocks, wall_s=t_wall)
+                              sample=f"first {cpu_rows} of 8192 rows of the 8192x8192 layer at E5M6 (one layer, one format), whole "
+                                     f"pipeline, {cpu_dt:.1f} s"),
+            e2e=dict(value=world * units / (e2e_ms * 1e-3) / 1e9, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                     ms_per_step=e2e_ms, steps=e2e_steps),
+            gpu_launches=sset.kernel_launches_per_step * args.steps, clocks=clocks, wall_s=t_wall)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -310,7 +502,7 @@ def run_gpu(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

@@ -177,7 +177,10 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *   the same layer, alphabet, format and shift wrote them (both arrays are then required).  A
  *   candidate in neither mask is absent: every table entry that involves it is marked undefined and
  *   its shift is reported as 0.  The masks must be disjoint and not both empty.  At most 8 distinct
- *   tables may be evaluated per call (an atom and its negation share one).
+ *   tables may be evaluated per call (an atom and its negation share one).  The lookup tables of the
+ *   evaluated candidates live in shared memory; when a fine-grained alphabet would not fit beside the
+ *   staging tile, the lookup grid is coarsened and the tables that then share a cell between thresholds are
+ *   searched exactly instead (slower, same results): no alphabet within the limits above is refused for size.
  * flags: SOP_SEARCH_SINGLES_ONLY fills only the diagonal (and best_single): enough to choose the
  *   primary codebook FMTa before the Lloyd refinement.  SOP_SEARCH_SELECT_MSE (paragraph "Pair-search
  *   design axes", axis ii): in every two-way and signed entry the block goes to the candidate with the
@@ -234,9 +237,11 @@ int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE
  *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
  *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
  *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
- *     When the iterations run in one launch, its CTAs wait for one another between iterations; every
- *     wait is bounded (about half a second).  A CTA that gives up makes all of them leave and the last
- *     entry is set to -1 (a distortion is never negative): the table is then not valid.
+ *     The last entry doubles as the status of the call: it is set to -1 when the call starts and to the final
+ *     distortion (never negative) by the closing iteration.  When the iterations run in one launch, its CTAs
+ *     wait for one another between iterations; every wait is bounded (about half a second).  A CTA that gives
+ *     up makes all of them leave and the last entry stays (or is set back to) -1: the table is then not valid.
+ *     A caller reads distortion_dev[iters] after synchronising and treats a negative value as a failed call.
  *   pool_count_dev: one long long, number of blocks in the pool.
  * Workspace: 8 bytes per weight element (u and omega of every pool element are kept across the
  *   iterations), 4 bytes per block (the pool list) and 4 bytes per channel, plus a fixed header. */
@@ -249,6 +254,13 @@ int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
  * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch when
  * every CTA of the iteration grid can be resident at once; otherwise there is one launch per iteration. */
 int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches);
+/* Launch-shape parameters of sop_dd4_lloyd for this process (test aid, no counterpart in the paper; results do
+ * not depend on them).  cell_spill_tiles in [1, 128]: cache tiles a CTA sorts between two transfers of its
+ * per-cell partial sums to the global sums (default 128, the most the 32-bit limbs allow);
+ * cache_ctas >= 0: largest grid of the cache kernel (0 = default, three CTAs per SM);
+ * tiles_per_warp in [1, 4]: most cache tiles one warp of an iteration CTA may walk (default 4).
+ * SOP_ERR_RANGE outside these ranges. */
+int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp);
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
                   const float* block_metric_dev, long long pool_rank, float pool_threshold, int flags,
@@ -275,7 +287,10 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
  *     word_sign_bits = 1: sign at bit b-1, selector at bit 0, magnitude E:M above the
  *     m = b-1-x-y metabits; word_sign_bits = 0: selector at bit b-1 (if m >= 1), magnitude above
  *     the remaining m-1 metabits.  Unused metabits are zero.
- *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten.
+ *   counts_dev (may be NULL): two long long {n_sel1, n_neg}, overwritten.  With index_a = SOP_PAIR_FROM_RESULT
+ *     the search result may hold no pair (a singles-only search, a search without a signed table while
+ *     use_sign = 1, an alphabet with one base atom): nothing is packed then, codes_dev is left as it was and
+ *     counts_dev receives {-1, -1}; pass counts_dev whenever the pair comes from a result block.
  *   flags: SOP_PACK_SELECT_MSE (paragraph "Pair-search design axes", axis ii): the smallest block squared
  *     error wins instead of the largest block cosine, ties keep the earlier candidate.
  *   block_metric_dev (may be NULL): [n_atoms x N_b] per-block cosines (with SOP_PACK_SELECT_MSE: per-block

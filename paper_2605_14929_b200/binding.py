@@ -82,7 +82,8 @@ def lib():
 def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
             "sop_channel_norms_static",
-            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd", "sop_pack",
+            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd_tuning",
+            "sop_dd4_lloyd", "sop_pack",
             "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
 
 
@@ -154,6 +155,23 @@ def dd4_lloyd_launches(M: int, K: int, iters: int, flags: int = 0) -> int:
     n = C.c_int()
     _check(lib().sop_dd4_lloyd_launches(_ll(M), _ll(K), iters, flags, C.byref(n)), "sop_dd4_lloyd_launches")
     return n.value
+
+
+def dd4_lloyd_tuning(cell_spill_tiles: int = 128, cache_ctas: int = 0, tiles_per_warp: int = 4) -> None:
+    """Launch-shape parameters of ``sop_dd4_lloyd`` (test aid; the defaults restore the library's own)."""
+    _check(lib().sop_dd4_lloyd_tuning(cell_spill_tiles, cache_ctas, tiles_per_warp), "sop_dd4_lloyd_tuning")
+
+
+class LloydNotFinished(RuntimeError):
+    """``sop_dd4_lloyd`` left its status entry negative: a bounded wait between iterations gave up (or the call
+    never ran to its end), so the codebook it wrote must not be used."""
+
+
+def check_lloyd_status(distortion: torch.Tensor, iters: int) -> None:
+    """Reads the status entry ``distortion[iters]`` of a finished (synchronised) ``sop_dd4_lloyd`` call and
+    raises ``LloydNotFinished`` when it is negative."""
+    if float(distortion[iters].item()) < 0.0:
+        raise LloydNotFinished(f"sop_dd4_lloyd did not finish: distortion[{iters}] = {float(distortion[iters].item())}")
 
 
 def alloc_workspace(nbytes: int, device) -> torch.Tensor:

@@ -226,7 +226,7 @@ __device__ void lloyd_publish_desc(LloydWs* ws, const float* s_lut, int ne) {
 }
 
 __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, AtomsDev A, const sop_search_result* __restrict__ res,
-                                                               LloydWs* __restrict__ ws) {
+                                                               LloydWs* __restrict__ ws, double* __restrict__ distortion, int iters) {
   unsigned prefix = 0, cnt = 0;
   long long rank = 0, below = 0;
   if (a.flags & SOP_LLOYD_POOL_THRESHOLD) prefix = pool_key(a.pool_threshold, a.flags);   // the caller fixes the threshold
@@ -271,6 +271,8 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
     ws->accD = 0.0;
     ws->done = 0;
     ws->list_count = 0;
+    // "not finished": the closing iteration overwrites it with the final distortion (never negative)
+    distortion[iters] = -1.0;
   }
   for (int r = threadIdx.x; r < SORT_ROWS; r += SETUP_TB) {
     ws->cellN[r] = 0; ws->cellS[r] = 0; ws->cellA[0][r] = 0.0; ws->cellA[1][r] = 0.0; ws->cellA[2][r] = 0.0;
@@ -336,7 +338,14 @@ __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exa
 }
 
 constexpr int CELL_LIMBS = 14;
-constexpr unsigned CELL_SPILL_TILES = 128;
+constexpr int CELL_SPILL_TILES_MAX = 128;     // a low limb takes at most 258 * (2^16 - 1) per tile: 128 tiles stay below 2^32
+constexpr int TILES_PER_WARP_MAX = 4;         // bound of the limb sums of an iteration CTA (see flush_limbs)
+
+// Launch-shape parameters of the pool cache and of the iteration grid.  The defaults are the largest values the
+// limb arithmetic allows; sop_dd4_lloyd_tuning lowers them (tests reach the mid-loop spill and a multi-tile warp
+// share on small layers that way).  Results do not depend on them.
+struct LloydTune { int spill_tiles, cache_ctas, tiles_per_warp; };
+static LloydTune g_tune = {CELL_SPILL_TILES_MAX, 0, TILES_PER_WARP_MAX};
 constexpr double MOMENT_UNIT = 1099511627776.0;   // 2^40
 
 __device__ __forceinline__ void add_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell, long long v) {
@@ -377,7 +386,8 @@ __device__ void spill_cells(unsigned (*cL)[SORT_ROWS], LloydWs* ws) {
   }
 }
 
-__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out) {
+__global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out,
+                                                         unsigned spill_tiles) {
   __shared__ unsigned hist[SORT_ROWS + 3];
   __shared__ unsigned warp_tot[LTB / 32];
   extern __shared__ __align__(16) uint2 stage[];                  // TILE_ELEMS pairs (dynamic: the kernel needs 60 KB in all)
@@ -474,7 +484,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
     __syncthreads();
     // a cell takes at most 258 flushes per tile and a low limb 2^16 - 1 per flush: the limbs go to the
     // global sums before they can wrap
-    if (++tiles_since_spill == CELL_SPILL_TILES) {
+    if (++tiles_since_spill == spill_tiles) {
       spill_cells(cL, ws);
       tiles_since_spill = 0;
       __syncthreads();
@@ -735,11 +745,12 @@ __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, Lloy
       s_stop = stop;
     }
     __syncthreads();
-    if (s_stop) {
-      if (blockIdx.x == 0 && threadIdx.x == 0) distortion[iters] = -1.0;
-      return;
-    }
+    if (s_stop) break;
   }
+  // Whoever leaves with the error flag up marks the result as invalid, whichever CTA gave up and whenever: a CTA
+  // that arrived late can still run the remaining iterations alone (nobody else arrives, so it never closes
+  // the last one), and it must not leave a valid-looking trace behind.
+  if (threadIdx.x == 0 && *(volatile unsigned*)&ws->error != 0u) distortion[iters] = -1.0;
 }
 
 int num_sms();
@@ -754,7 +765,8 @@ static bool lloyd_iteration_plan(long long NB, long long pool_blocks, int iters,
   long long grid = (likely + LTB / 32 - 1) / (LTB / 32);            // one warp per cache tile
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
   // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
-  const long long need = (tiles + 4 * (LTB / 32) - 1) / (4 * (LTB / 32));
+  const long long per_cta = (long long)g_tune.tiles_per_warp * (LTB / 32);
+  const long long need = (tiles + per_cta - 1) / per_cta;
   if (grid < need) grid = need;
   if (grid < 1) grid = 1;
   static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
@@ -788,6 +800,16 @@ int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* 
   const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), M * (K / SOP_G), iters, flags, &grid);
   // radix select (three passes, unless the pool is cut by a threshold), set-up, pool list, pool cache, iterations
   *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + (persistent ? 1 : iters + 1);
+  return SOP_OK;
+}
+
+int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp) {
+  using namespace sop;
+  if (cell_spill_tiles < 1 || cell_spill_tiles > CELL_SPILL_TILES_MAX || cache_ctas < 0 || tiles_per_warp < 1 ||
+      tiles_per_warp > TILES_PER_WARP_MAX) return SOP_ERR_RANGE;
+  g_tune.spill_tiles = cell_spill_tiles;
+  g_tune.cache_ctas = cache_ctas;
+  g_tune.tiles_per_warp = tiles_per_warp;
   return SOP_OK;
 }
 
@@ -850,7 +872,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     select_kernel<2><<<(int)sg, LTB, 0, st>>>(a, search_dev, ws);
     SOP_CUDA_TRY(cudaGetLastError());
   }
-  lloyd_setup_kernel<<<1, SETUP_TB, 0, st>>>(a, A, search_dev, ws);
+  lloyd_setup_kernel<<<1, SETUP_TB, 0, st>>>(a, A, search_dev, ws, distortion_dev, iters);
   SOP_CUDA_TRY(cudaGetLastError());
   pool_list_kernel<<<(int)sg, LTB, 0, st>>>(a, ws);
   SOP_CUDA_TRY(cudaGetLastError());
@@ -858,14 +880,15 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   // (u, omega) of every pool element, once: sorted tiles, cell starts, per-cell sums and moments
   {
     long long cg = (NB + LTB - 1) / LTB;      // one tile per CTA pass
-    if (cg > (long long)sms * 3) cg = (long long)sms * 3;
+    const long long cg_max = g_tune.cache_ctas > 0 ? g_tune.cache_ctas : (long long)sms * 3;
+    if (cg > cg_max) cg = cg_max;
     const size_t stage_bytes = (size_t)TILE_ELEMS * sizeof(uint2);
     static bool attr_set = false;
     if (!attr_set) {
       SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
       attr_set = true;
     }
-    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev);
+    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
     SOP_CUDA_TRY(cudaGetLastError());
   }
   long long grid = 1;

@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
   __shared__ unsigned s_cnt[2];
   __shared__ int s_row[4];   // rows of block_cos for the candidates a, -a, b, -b (-1: none)
   __shared__ int s_idx[2];   // the two atoms
+  __shared__ int s_no_pair;  // the search result holds no pair to pack
   const int tid = threadIdx.x;
   if (tid == 0) {
     int ia = a.index_a, ib = a.index_b;
@@ -109,6 +110,10 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
       ia = a.use_sign ? res->best_sa : res->best_a;
       ib = a.use_sign ? res->best_sb : res->best_b;
     }
+    // a result without a pair (singles-only search, no signed table, one base atom): nothing is packed and the
+    // counts say so; with use_sign the second atom of each must exist too (the negation follows its atom)
+    s_no_pair = from_result && (ia < 0 || ib < 0 || ia >= A.n_atoms || ib >= A.n_atoms ||
+                                (a.use_sign && (ia + 1 >= A.n_atoms || ib + 1 >= A.n_atoms))) ? 1 : 0;
     ia = max(0, min(A.n_atoms - 1, ia));
     int nb = 1;
     if (ib != SOP_NO_ATOM) { ib = max(0, min(A.n_atoms - 1, ib)); nb = 2; }
@@ -134,6 +139,10 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
     s_cnt[0] = s_cnt[1] = 0;
   }
   __syncthreads();
+  if (s_no_pair) {
+    if (a.counts && blockIdx.x == 0 && tid < 2) a.counts[tid] = ~0ull;     // {-1, -1}
+    return;
+  }
   const int nb = s_nb, n = s_nbits, b = a.container_bits;
   // table values and decision thresholds of the (up to two) tables: one thread per entry (the same rule as
   // build_thresholds: the largest fp32 <= the midpoint, a repeated entry takes the threshold above it)

@@ -921,6 +921,24 @@ size_t sweep_smem_bytes(const Plan& P) {
   return (b + 15) & ~(size_t)15;
 }
 
+// Doubles the cell width of the LUT class with the most rows (its tables then hold several thresholds per cell
+// where they are dense, and such tables take the exact binary search).  False when no class can shrink further.
+static bool coarsen_cells(Plan* P) {
+  int pick = -1;
+  for (int c = 0; c < P->n_classes; ++c)
+    if (P->cls[c].kind == SOP_KIND_LUT && P->cls[c].c_half > 1 && (pick < 0 || P->cls[c].c_half > P->cls[pick].c_half)) pick = c;
+  if (pick < 0) return false;
+  ClassDev& C = P->cls[pick];
+  C.invh *= 0.5f;
+  C.c_half = (int)ceil(1.25 * (double)C.tmax * (double)C.invh);
+  if (C.c_half < 1) C.c_half = 1;
+  int rows = 1;
+  for (int c = 0; c < P->n_classes; ++c)
+    if (P->cls[c].kind == SOP_KIND_LUT) rows = rows > 2 * P->cls[c].c_half + 1 ? rows : 2 * P->cls[c].c_half + 1;
+  P->rows = rows;
+  return true;
+}
+
 static int g_num_sms = 0;
 int num_sms() {
   if (!g_num_sms) {
@@ -986,31 +1004,33 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   unsigned* hist = (unsigned*)(ws + ws_hist_off());
   Partial* partials = (Partial*)(ws + ws_part_off());
 
-  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
-  const int sms = num_sms();
-  if (!k_from_result) {
-    // one read of W: block scales' exponent histogram, max|W|, then the shifts (last CTA)
-    long long want = (L.NB + 255) / 256;
-    const int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
-    prepass_kernel<<<grid, 256, 0, st>>>(L, P, F, hist, hdr);
-    SOP_CUDA_TRY(cudaGetLastError());
-  }
-
-  const size_t smem = sweep_smem_bytes(P);
+  // everything that can refuse the call is decided before the first enqueue
   constexpr size_t SMEM_MAX = 226 * 1024;   // 227 KB per CTA minus the kernel's few static bytes
+  size_t smem = sweep_smem_bytes(P);
+  while (smem > SMEM_MAX && coarsen_cells(&P)) smem = sweep_smem_bytes(P);   // cell tables too large: coarser cells, exact search where needed
   if (smem > SMEM_MAX) return SOP_ERR_ALPHABET;
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
-    smem_set = SMEM_MAX;
-  }
+  const int sms = num_sms();
   // persistent grid: one CTA per SM, fewer when the layer is small; at least enough threads for one row
   long long grid = (L.NB + TB - 1) / TB;
   if (grid > sms) grid = sms;
   const long long min_grid = (L.nbk + TB - 1) / TB;
   if (grid < min_grid) grid = min_grid;
   if (grid > MAX_GRID) return SOP_ERR_SHAPE;
+
+  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
+  if (!k_from_result) {
+    // one read of W: block scales' exponent histogram, max|W|, then the shifts (last CTA)
+    long long want = (L.NB + 255) / 256;
+    const int pgrid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
+    prepass_kernel<<<pgrid, 256, 0, st>>>(L, P, F, hist, hdr);
+    SOP_CUDA_TRY(cudaGetLastError());
+  }
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+    smem_set = SMEM_MAX;
+  }
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
   if (flags & SOP_SEARCH_SELECT_MSE)
     sweep_kernel<true><<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev,

@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import dataclasses
 import math
-from typing import List, Sequence
+from typing import List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -67,15 +67,27 @@ class SweepOutputs:
 
 class LayerSweep:
     """Buffers and call order for one layer shape.  ``rom`` are base ROM atom names; every ROM atom
-    is followed by its negation; ``fp`` are FP singles; ``lloyd_iters`` = 0 disables the DD atom."""
+    is followed by its negation; ``fp`` are FP singles; ``lloyd_iters`` = 0 disables the DD atom.
+    ``share`` names another sweep of the same shape and alphabet (typically the same layer at another scale
+    format): the large scratch buffers -- workspaces, the per-block arrays, the channel norms, the packed
+    codes and scale words -- are then that sweep's, and only the small results (tables, result blocks, the DD
+    table, counts) are this sweep's own.  Sweeps that share buffers must run one after the other on one stream,
+    and the packed output of one is overwritten by the next."""
 
     def __init__(self, M: int, K: int, T: int, fmt: I.ScaleFormat, rom: Sequence[str], fp: Sequence[str] = (),
-                 lloyd_iters: int = 8, pool_percent: float = 50.0, device="cuda", want_blocks: bool = False):
+                 lloyd_iters: int = 8, pool_percent: float = 50.0, device="cuda", want_blocks: bool = False,
+                 share: Optional["LayerSweep"] = None):
         self.M, self.K, self.T, self.fmt = M, K, T, fmt
         self.dev = torch.device(device)
         self.iters = lloyd_iters
         self.rom_atoms = I.alphabet(rom, with_negations=True)
-        n_bits = self.rom_atoms[0].n_bits
+        if not self.rom_atoms:
+            # element formats only (a promotion-profile comparison): singles, no pair, no DD atom; the first one is packed
+            if lloyd_iters > 0 or not fp:
+                raise ValueError("without ROM atoms there is no DD atom to refine: need fp candidates and lloyd_iters = 0")
+            n_bits = I.fp_atom(fp[0]).n_bits
+        else:
+            n_bits = self.rom_atoms[0].n_bits
         self.full_atoms = list(self.rom_atoms)
         self.dd_mask = 0
         if lloyd_iters > 0:
@@ -91,10 +103,15 @@ class LayerSweep:
         self.pool_rank = max(1, min(self.NB, self.pool_rank))
         nR, nF = len(self.rom_atoms), len(self.full_atoms)
         d = self.dev
-        self.c = torch.empty(K, dtype=torch.float32, device=d)
-        self.ws_norm = B.alloc_workspace(B.channel_norms_workspace(T, K), d)
-        self.ws_search = B.alloc_workspace(B.pair_search_workspace(M, K, nF), d)
-        self.ws_lloyd = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), d)
+        if share is not None:
+            if (share.M, share.K, share.T, len(share.full_atoms), share.full_atoms[0].n_bits) != (M, K, T, nF, n_bits):
+                raise ValueError("a sweep shares buffers only with a sweep of the same shape and alphabet size")
+            self.c, self.ws_norm, self.ws_search, self.ws_lloyd = share.c, share.ws_norm, share.ws_search, share.ws_lloyd
+        else:
+            self.c = torch.empty(K, dtype=torch.float32, device=d)
+            self.ws_norm = B.alloc_workspace(B.channel_norms_workspace(T, K), d)
+            self.ws_search = B.alloc_workspace(B.pair_search_workspace(M, K, nF), d)
+            self.ws_lloyd = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), d)
         self.rom_table = B.new_pair_table(nF, d)
         self.rom_result = B.new_result(d)
         self.fixed_mask = ((1 << nF) - 1) & ~self.dd_mask
@@ -107,20 +124,31 @@ class LayerSweep:
         # the packed word carries sign + selector when both fit 16 bits; a 16-bit signed format (E8M7) has no
         # metabit left, so its pair is packed without the sign (the selector takes the sign's bit)
         self.use_sign = 1 if fmt.sign_bits and fmt.exp_bits + fmt.man_bits + 2 <= 16 else 0
-        self.container = scale_word_container(fmt, bool(self.use_sign), True)
-        self.codes = torch.empty(self.NB * 2 * n_bits, dtype=torch.uint8, device=d)
-        self.words = torch.empty(B.words_nbytes(self.NB, self.container), dtype=torch.uint8, device=d)
+        self.single = not self.rom_atoms                      # one element format packed alone: no sign choice, no selector
+        if self.single:
+            self.use_sign = 0
+        self.container = scale_word_container(fmt, bool(self.use_sign), not self.single)
         self.counts = torch.zeros(2, dtype=torch.int64, device=d)
-        self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
-        self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
+        if share is not None:
+            self.codes, self.full_cos, self.full_sse = share.codes, share.full_cos, share.full_sse
+            self.words = share._words_store[:B.words_nbytes(self.NB, self.container)]
+        else:
+            self.codes = torch.empty(self.NB * 2 * n_bits, dtype=torch.uint8, device=d)
+            self._words_store = torch.empty(B.words_nbytes(self.NB, 16), dtype=torch.uint8, device=d)   # room for any container
+            self.words = self._words_store[:B.words_nbytes(self.NB, self.container)]
+            self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
+            self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
         self.kernel_launches_per_step = 0
         self.lloyd_launches = B.dd4_lloyd_launches(M, K, lloyd_iters) if lloyd_iters > 0 else 0
 
-    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None) -> None:
-        """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32."""
+    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True) -> None:
+        """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32.  ``norms`` =
+        False skips the channel norms: they do not depend on the scale format, so a sweep that shares the
+        buffers of another one (same layer, other format) uses the norms that one has just computed."""
         n = 0
-        B.sop_channel_norms(X, self.c, self.ws_norm, stream)
-        n += 2
+        if norms:
+            B.sop_channel_norms(X, self.c, self.ws_norm, stream)
+            n += 2
         if self.iters > 0:
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.rom_table, None, self.rom_result, self.ws_search,
                               block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
@@ -139,6 +167,7 @@ class LayerSweep:
             n += 1
         n += 1
         B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, search_result=self.result,
+                   index_a=0 if self.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if self.single else B.PAIR_FROM_RESULT,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
                    counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
                    block_cos=self.full_cos, stream=stream)
@@ -165,6 +194,8 @@ class LayerSweep:
 
     def outputs(self) -> SweepOutputs:
         torch.cuda.synchronize(self.dev)
+        if self.iters > 0:
+            B.check_lloyd_status(self.distortion, self.iters)     # a codebook from an unfinished call is not handed out
         nF, nR = len(self.full_atoms), len(self.rom_atoms)
         return SweepOutputs(
             c=self.c.cpu(), pair_table=B.read_pair_table(self.pair_table, nF),
@@ -176,10 +207,11 @@ class LayerSweep:
 
 
 class LayerStream:
-    """Streams host-resident layers of one shape through a ``LayerSweep``.  While layer i is swept, the
-    weights and activations of layer i + 1 travel host -> device and the results of layer i - 1 travel
-    device -> host: two input slots, two output slots, three CUDA streams ordered by events.  The host
-    tensors must be pinned for the copies to overlap.
+    """Streams host-resident layers of one shape through a ``LayerSweep`` -- or through several sweeps that
+    share their buffers (the same layer at several scale formats).  While layer i is swept, the weights and
+    activations of layer i + 1 travel host -> device and the results of layer i - 1 travel device -> host: two
+    input slots, two output slots per sweep, three CUDA streams ordered by events.  The host tensors must be
+    pinned for the copies to overlap.
 
         stream = LayerStream(sweep)
         for i, (W_host, X_host) in enumerate(layers):
@@ -189,31 +221,37 @@ class LayerStream:
         consume(stream.collect(len(layers) - 1))
 
     ``collect(i)`` waits for layer i and returns pinned host tensors (pair_table, signed_table, result,
-    codes, words) that stay valid until ``submit(i + 2)``."""
+    codes, words, distortion) that stay valid until ``submit(i + 2)`` -- one dict for a single sweep, a list
+    of dicts (one per sweep) otherwise; it raises ``binding.LloydNotFinished`` when a Lloyd call of the layer
+    reports that it did not run to its end.  ``streams`` hands in the three CUDA streams (copy in, compute,
+    copy out) so that several LayerStream objects, one per layer shape, work as one ordered pipeline."""
 
-    OUT = ("pair_table", "signed_table", "result", "codes", "words")
+    OUT = ("pair_table", "signed_table", "result", "codes", "words", "distortion")
 
-    def __init__(self, sweep: LayerSweep):
-        self.sw = sweep
-        d = sweep.dev
-        self.s_in, self.s_run, self.s_out = torch.cuda.Stream(d), torch.cuda.Stream(d), torch.cuda.Stream(d)
-        self.W = [torch.empty((sweep.M, sweep.K), dtype=torch.bfloat16, device=d) for _ in range(2)]
-        self.X = [torch.empty((sweep.T, sweep.K), dtype=torch.float32, device=d) for _ in range(2)]
-        self.dev_out = [{k: torch.empty_like(getattr(sweep, k)) for k in self.OUT} for _ in range(2)]
-        self.host_out = [{k: torch.empty(getattr(sweep, k).shape, dtype=getattr(sweep, k).dtype).pin_memory() for k in self.OUT}
-                         for _ in range(2)]
+    def __init__(self, sweep, streams=None):
+        self.single = isinstance(sweep, LayerSweep)
+        self.sweeps = [sweep] if self.single else list(sweep)
+        sw = self.sw = self.sweeps[0]
+        d = sw.dev
+        self.s_in, self.s_run, self.s_out = streams if streams is not None else (torch.cuda.Stream(d), torch.cuda.Stream(d), torch.cuda.Stream(d))
+        self.W = [torch.empty((sw.M, sw.K), dtype=torch.bfloat16, device=d) for _ in range(2)]
+        self.X = [torch.empty((sw.T, sw.K), dtype=torch.float32, device=d) for _ in range(2)]
+        self.dev_out = [[{k: torch.empty_like(getattr(q, k)) for k in self.OUT} for q in self.sweeps] for _ in range(2)]
+        self.host_out = [[{k: torch.empty(getattr(q, k).shape, dtype=getattr(q, k).dtype).pin_memory() for k in self.OUT}
+                          for q in self.sweeps] for _ in range(2)]
         ev = lambda: [torch.cuda.Event() for _ in range(2)]
-        self.in_ready, self.in_free, self.out_ready, self.out_done = ev(), ev(), ev(), ev()
+        self.in_ready, self.in_free, self.out_done = ev(), ev(), ev()
+        self.out_ready = [[torch.cuda.Event() for _ in self.sweeps] for _ in range(2)]
         self.h2d_bytes = self.W[0].numel() * 2 + self.X[0].numel() * 4
-        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.dev_out[0].values())
-        self.before_run = None       # optional callable run on the compute stream before every sweep
+        self.d2h_bytes = sum(t.numel() * t.element_size() for o in self.dev_out[0] for t in o.values())
+        self.before_run = None       # optional callable run on the compute stream before every layer
+        self.n_submitted = 0
 
     def submit(self, i: int, W_host: torch.Tensor, X_host: torch.Tensor) -> None:
         slot = i & 1
-        sw = self.sw
         with torch.cuda.stream(self.s_in):
             if i >= 2:
-                self.s_in.wait_event(self.in_free[slot])      # the sweep of layer i - 2 has read this slot
+                self.s_in.wait_event(self.in_free[slot])      # the sweeps of layer i - 2 have read this slot
             self.W[slot].copy_(W_host, non_blocking=True)
             self.X[slot].copy_(X_host, non_blocking=True)
             self.in_ready[slot].record(self.s_in)
@@ -223,18 +261,81 @@ class LayerStream:
                 self.s_run.wait_event(self.out_done[slot])    # the results of layer i - 2 have left this slot
             if self.before_run is not None:
                 self.before_run()
-            sw.run(self.W[slot], self.X[slot], self.s_run)
+            for f, q in enumerate(self.sweeps):
+                q.run(self.W[slot], self.X[slot], self.s_run, norms=(f == 0))
+                # the sweeps share their packed output: it is set aside before the next format overwrites it
+                for k in self.OUT:
+                    self.dev_out[slot][f][k].copy_(getattr(q, k), non_blocking=True)
+                self.out_ready[slot][f].record(self.s_run)
             self.in_free[slot].record(self.s_run)
-            for k in self.OUT:
-                self.dev_out[slot][k].copy_(getattr(sw, k), non_blocking=True)
-            self.out_ready[slot].record(self.s_run)
         with torch.cuda.stream(self.s_out):
-            self.s_out.wait_event(self.out_ready[slot])
-            for k in self.OUT:
-                self.host_out[slot][k].copy_(self.dev_out[slot][k], non_blocking=True)
+            for f in range(len(self.sweeps)):
+                self.s_out.wait_event(self.out_ready[slot][f])     # a format's results leave while the next one is swept
+                for k in self.OUT:
+                    self.host_out[slot][f][k].copy_(self.dev_out[slot][f][k], non_blocking=True)
             self.out_done[slot].record(self.s_out)
+        self.n_submitted = max(self.n_submitted, i + 1)
 
-    def collect(self, i: int) -> dict:
+    def collect(self, i: int):
         slot = i & 1
         self.out_done[slot].synchronize()
-        return self.host_out[slot]
+        for f, q in enumerate(self.sweeps):
+            if q.iters > 0:
+                B.check_lloyd_status(self.host_out[slot][f]["distortion"], q.iters)
+        return self.host_out[slot][0] if self.single else self.host_out[slot]
+
+
+class LayerSetSweep:
+    """A set of layers (one transformer block, say), each swept at several scale formats: the unit of a model
+    sweep that is streamed layer by layer.  Layers of one shape share their large buffers, and so do the formats
+    of one layer; every (layer, format) keeps its own tables, result blocks and DD table.  ``run`` makes one
+    pass: per layer the channel norms once, then per format the candidate sweep, the Lloyd refinement, the sweep
+    of the new columns and the pack."""
+
+    def __init__(self, shapes: Sequence[tuple], fmts: Sequence[I.ScaleFormat], rom: Sequence[str], fp: Sequence[str] = (),
+                 lloyd_iters: int = 8, device="cuda"):
+        self.shapes, self.fmts = [tuple(s) for s in shapes], list(fmts)
+        self.dev = torch.device(device)
+        owner = {}
+        self.sweeps: List[List[LayerSweep]] = []
+        for shape in self.shapes:
+            row = []
+            for fmt in self.fmts:
+                sw = LayerSweep(*shape, fmt, rom, fp, lloyd_iters, device=device, share=owner.get(shape))
+                owner.setdefault(shape, sw)
+                row.append(sw)
+            self.sweeps.append(row)
+        self.elements = sum(M * K for M, K, _ in self.shapes)
+        self._graph = None
+
+    def run(self, layers: Sequence[tuple], stream=None) -> None:
+        """``layers``: one (W, X) pair of device tensors per shape given to the constructor, in that order."""
+        for row, (W, X) in zip(self.sweeps, layers):
+            for f, sw in enumerate(row):
+                sw.run(W, X, stream, norms=(f == 0))
+
+    @property
+    def kernel_launches_per_step(self) -> int:
+        return sum(sw.kernel_launches_per_step for row in self.sweeps for sw in row)
+
+    def capture(self, layers: Sequence[tuple]) -> None:
+        """Record one pass over these device tensors into a CUDA graph (see ``LayerSweep.capture``)."""
+        self.run(layers)
+        torch.cuda.synchronize(self.dev)
+        side = torch.cuda.Stream(self.dev)
+        side.wait_stream(torch.cuda.current_stream(self.dev))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            self.run(layers, side)
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        self._graph, self._graph_inputs = graph, list(layers)
+
+    def replay(self) -> None:
+        self._graph.replay()
+
+    def check(self) -> None:
+        """After a synchronise: raises when a Lloyd call of the pass did not run to its end."""
+        for row in self.sweeps:
+            for sw in row:
+                if sw.iters > 0:
+                    B.check_lloyd_status(sw.distortion, sw.iters)

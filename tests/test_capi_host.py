@@ -148,3 +148,22 @@ def test_grid_arguments_are_checked_on_the_host(lib):
         rc = lib.sop_pack(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, arr, 1, None, C.c_uint(0), 0, B.NO_ATOM, 0, None, 0, 12, 0,
                           C.c_void_p(0x1000), FAKE, None, None, 0, None)
         assert rc == -4
+
+
+def test_lloyd_status_entry_is_read_on_the_host(lib):
+    # distortion[iters] < 0 marks a call that did not run to its end: the binding turns it into an exception
+    import torch
+    d = torch.tensor([3.0, 2.0, 1.5], dtype=torch.float64)
+    B.check_lloyd_status(d, 2)
+    d[2] = -1.0
+    with pytest.raises(B.LloydNotFinished):
+        B.check_lloyd_status(d, 2)
+    B.check_lloyd_status(d, 1)
+
+
+def test_lloyd_tuning_ranges(lib):
+    assert lib.sop_dd4_lloyd_tuning(0, 0, 4) == -7 and lib.sop_dd4_lloyd_tuning(129, 0, 4) == -7
+    assert lib.sop_dd4_lloyd_tuning(128, -1, 4) == -7
+    assert lib.sop_dd4_lloyd_tuning(128, 0, 0) == -7 and lib.sop_dd4_lloyd_tuning(128, 0, 5) == -7
+    assert lib.sop_dd4_lloyd_tuning(1, 2, 1) == 0
+    assert lib.sop_dd4_lloyd_tuning(128, 0, 4) == 0      # the defaults again

@@ -1,7 +1,8 @@
 """GPU parity on the benchmark configurations: the attention-projection layer at its full size in
 the launch configuration that bench.py times (sampled blocks and rows against the oracle, the Lloyd
 table and the ROM part of the pair tables in full), and reduced-row cases of the 7B-shaped
-FP6-vs-FP8 comparison and of the 70B-shaped layer set at every scale format."""
+FP6-vs-FP8 comparison and of the 70B-shaped layer set at every scale format (the full-size cases of
+those configurations are in test_gpu_fullsize.py)."""
 import math
 
 import numpy as np
@@ -20,7 +21,7 @@ pytestmark = pytest.mark.gpu
 def test_config2_full_size_in_the_bench_configuration(B):
     import bench
     from paper_2605_14929_b200.pipeline import LayerSweep
-    Wl = bench.WORKLOAD
+    Wl = bench.CONFIG2
     M, K, T = Wl["M"], Wl["K"], Wl["T"]
     fmt = I.scale_format(Wl["scale_format"])
     L = bench.make_layer(0)
