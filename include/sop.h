@@ -41,6 +41,7 @@ extern "C" {
 #define SOP_ALL_ATOMS 0xFFFFFFFFu /* eval_mask of sop_pair_search: evaluate every candidate */
 #define SOP_SEARCH_SINGLES_ONLY 1 /* flags of sop_pair_search: reduce single candidates only, no pair / signed entries */
 #define SOP_SEARCH_SELECT_MSE 2   /* flags of sop_pair_search: the per-block reassignment takes the smaller block error */
+#define SOP_SEARCH_KEEP_LOADED_ENTRIES 4 /* flags of sop_pair_search: table entries among loaded candidates are kept, not formed again */
 
 enum {
   SOP_OK = 0,

@@ -22,6 +22,7 @@ MAX_ATOMS = 16
 ALL_ATOMS = 0xFFFFFFFF
 SEARCH_SINGLES_ONLY = 1
 SEARCH_SELECT_MSE = 2
+SEARCH_KEEP_LOADED_ENTRIES = 4
 LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD, LLOYD_LAUNCH_PER_ITERATION = 1, 2, 4, 8
 PACK_SELECT_MSE = 1
 MAX_ENTRIES = 32
@@ -208,13 +209,16 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
                     block_cos: Optional[torch.Tensor] = None, block_sse: Optional[torch.Tensor] = None,
                     stream=None, g: int = 16, eval_mask: int = ALL_ATOMS, load_mask: int = 0,
                     singles_only: bool = False, prev_result: Optional[torch.Tensor] = None,
-                    select_mse: bool = False) -> None:
+                    select_mse: bool = False, keep_loaded: bool = False) -> None:
+    """``keep_loaded``: the table entries among the candidates of ``load_mask`` stay as an earlier call wrote them
+    into ``pair_table`` / ``signed_table``; only the entries with a newly evaluated candidate are formed."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_pair_search(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
                                  make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), C.c_uint(eval_mask),
                                  C.c_uint(load_mask),
-                                 (SEARCH_SINGLES_ONLY if singles_only else 0) | (SEARCH_SELECT_MSE if select_mse else 0), _ptr(prev_result),
+                                 (SEARCH_SINGLES_ONLY if singles_only else 0) | (SEARCH_SELECT_MSE if select_mse else 0)
+                                 | (SEARCH_KEEP_LOADED_ENTRIES if keep_loaded else 0), _ptr(prev_result),
                                  _ptr(pair_table),
                                  _ptr(signed_table), _ptr(result), _ptr(block_cos), _ptr(block_sse), _ptr(workspace),
                                  C.c_size_t(workspace.numel()), _stream(stream)), "sop_pair_search")

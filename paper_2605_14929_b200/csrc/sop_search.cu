@@ -4,11 +4,16 @@
 //                    for every scale class that needs an F_layer search, and max|W|   (HBM-bound);
 //                    the CTA that finishes last derives the F_layer shift k* per class from the
 //                    histogram and the layer power-of-two scale for "^0" candidates.
-//   sweep_kernel     persistent, one thread per 16-element block: phase 1 evaluates every candidate
+//   sweep_kernel     persistent, one thread per 16-element block: evaluates every candidate of the call
 //                    in registers (cell-table lookup of the reconstruction value, packed f32x2
-//                    fused multiply-adds for the block metric, fixed quad-tree order); phase 2
-//                    reduces the per-block (cos, sse) of the CTA's tile into per-pair sums, one
-//                    pair per thread, FP64 accumulators.                                    (ALU-bound)
+//                    fused multiply-adds for the block metric, fixed quad-tree order) and writes
+//                    the per-block cosine and squared error of each as one column.          (ALU-bound)
+//   reduce_kernel    reads the columns of every candidate present in the call (those just written
+//                    and those an earlier call wrote) tile by tile into shared memory and forms
+//                    the table entries: a warp owns a few "tasks" (one anchor column against up to
+//                    four partner columns, so five columns are fetched for up to five entries), a
+//                    lane owns eight blocks of every tile, the sums of those eight are fp32 and go
+//                    to FP64 accumulators after every tile.
 //                    The CTA that finishes last adds the per-CTA partials in a fixed order
 //                    (deterministic), writes the tables and picks the best pair / best single.
 #include <math.h>
@@ -39,6 +44,28 @@ struct ClassDev {
 };
 struct SlotDev { unsigned char type, i0, i1, pad; };  // type 0: pair (i0, i1) (i0 == i1: single); 1: signed (i0, i0+1, i1, i1+1)
 
+// One unit of work of the reduction: an anchor candidate against up to four partners.  Entry q is the table slot
+// slot[q] of the pair {anchor, part[q]}; rev = 0: the anchor is the first candidate of all its entries (it keeps a
+// tie), rev = 1: it is the second one.  self_slot is the slot of the anchor alone (255: none).  sgn = 1: anchor and
+// partners are base atoms and stand for the better of the atom and its negation (a signed four-way entry).
+constexpr int TASK_PART = 4;
+constexpr int MAX_TASKS = 96;
+constexpr int MAX_TPW = 3;             // tasks per warp and launch
+struct TaskDev {
+  unsigned char anchor, n_part, self_slot, sgn, rev, pad[3];
+  unsigned char part[TASK_PART], slot[TASK_PART];
+};
+// One launch of the reduction: per warp its tasks (255: empty seat) and the first accumulator seat of each; the
+// candidates whose columns the launch fetches (col_slot: candidate -> column of the tile buffers, 255: not fetched)
+// and the base atoms whose signed-best column it forms (sb_slot likewise).
+struct SeatsDev {
+  unsigned char task[8][MAX_TPW];
+  unsigned short acc0[8][MAX_TPW];
+  unsigned char col_slot[SOP_MAX_ATOMS], sb_slot[SOP_MAX_ATOMS];
+  unsigned char cols[SOP_MAX_ATOMS], bases[SOP_MAX_ATOMS];      // the inverse lists
+  int n_cols, n_bases, n_seats;
+};
+
 struct Plan {
   int n_atoms, n_classes, n_tables, n_slots, n_pair_slots;
   int k_mode, rows, a_pad;
@@ -54,13 +81,16 @@ struct Plan {
   unsigned char table_neg[SOP_MAX_TABLES];    // candidate that uses the negated table (255: none)
   unsigned char cls_tables[SOP_MAX_CLASSES];  // bit t: table t belongs to the class
   SlotDev slots[MAX_SLOTS];
+  int keep_loaded;                            // entries among loaded candidates stay as the tables hold them
+  int n_tasks;
+  TaskDev tasks[MAX_TASKS];
 };
 
 struct WsHeader {
   unsigned wmax_bits;
   int cls_k[SOP_MAX_CLASSES];
   float cls_pot[SOP_MAX_CLASSES];
-  unsigned done_prepass, done_sweep;   // CTAs that have finished (the last one does the serial tail)
+  unsigned done_prepass, done_reduce;  // CTAs that have finished (the last one does the serial tail)
   int pad[5];
 };
 struct Partial { double gap, sse; long long n1, nneg; };
@@ -360,50 +390,41 @@ __device__ void build_tables(const Plan& P, const AtomsDev& A, uint2* cell, floa
   __syncthreads();
 }
 
-__device__ __forceinline__ void half_barrier(int half) {
-  asm volatile("bar.sync %0, %1;" ::"r"(half + 1), "n"(TB / 2) : "memory");
+// One evaluated candidate of one block: the cosine, then both per-block values into their columns.
+__device__ __forceinline__ void emit(float* __restrict__ block_cos, float* __restrict__ block_sse, size_t col_off, bool on, float nw,
+                                     const Metric& mt) {
+  const float cosv = block_cosine(nw, mt.nq, mt.dot);
+  if (on) {
+    block_cos[col_off] = cosv;
+    block_sse[col_off] = mt.sse;
+  }
 }
 
-// The CTA works as two halves of 256 threads with a barrier each, so that one half reduces its tile
-// (phase 2) while the other still evaluates candidates (phase 1).
-__device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const Partial* partials, sop_pair_stat* s_pair, sop_pair_stat* s_sig,
-                              Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
-                              const int* cls_k, float wmax);
-
-// SEL_ERR: the per-block reassignment takes the smaller block error instead of the larger block cosine
-// (paragraph "Pair-search design axes", axis ii); ties keep the earlier candidate either way.
-template <bool SEL_ERR>
-__global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, WsHeader* __restrict__ hdr,
-                                                      Partial* __restrict__ partials, float* __restrict__ block_cos,
-                                                      float* __restrict__ block_sse, sop_pair_stat* __restrict__ pair_table,
-                                                      sop_pair_stat* __restrict__ signed_table, sop_search_result* __restrict__ res,
+// Evaluates the candidates of eval_mask on every block and writes their columns of block_cos / block_sse.
+__global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, AtomsDev A, FmtDev F, const WsHeader* __restrict__ hdr,
+                                                      float* __restrict__ block_cos, float* __restrict__ block_sse,
                                                       const sop_search_result* __restrict__ prev) {
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
   uint2* cell = reinterpret_cast<uint2*>(smem);
   float* tau = reinterpret_cast<float*>(cell + (size_t)P.n_tables * P.rows * 16);
   float* lutv = tau + SOP_MAX_TABLES * 32;
   int* fast = reinterpret_cast<int*>(lutv + SOP_MAX_TABLES * 32);
   int* cls_k = fast + SOP_MAX_TABLES;
   float* cls_pot = reinterpret_cast<float*>(cls_k + SOP_MAX_CLASSES);
-  float2* cs_all = reinterpret_cast<float2*>(cls_pot + SOP_MAX_CLASSES);   // [2][n_atoms][HBP] (cos, sse), candidate-major
 
-  constexpr int HB = TB / 2;
-  const int tid = threadIdx.x, lane = tid & 31, half = tid / HB, htid = tid - half * HB;
+  const int tid = threadIdx.x, lane = tid & 31;
   build_tables(P, A, cell, tau, lutv, fast);
-  const float layer_wmax = P.k_from_result ? prev->layer_absmax : __uint_as_float(hdr->wmax_bits);
   if (tid < SOP_MAX_CLASSES) {
     if (P.k_from_result) {
       const bool live = tid < P.n_classes;
       cls_k[tid] = live && P.cls[tid].k_src >= 0 ? prev->k[P.cls[tid].k_src] : 0;
-      cls_pot[tid] = live && P.cls[tid].scope == 0 ? layer_pot_scale(layer_wmax, P.cls[tid].tmax) : 0.0f;
+      cls_pot[tid] = live && P.cls[tid].scope == 0 ? layer_pot_scale(prev->layer_absmax, P.cls[tid].tmax) : 0.0f;
     } else {
       cls_k[tid] = hdr->cls_k[tid];
       cls_pot[tid] = hdr->cls_pot[tid];
     }
   }
   __syncthreads();
-  constexpr int HBP = HB + 1;   // row pitch: candidates land in different banks
-  float2* cs = cs_all + (size_t)half * (P.n_atoms + P.n_bases) * HBP;
 
   // thread -> fixed column block j, rows m = r0, r0 + R, ...
   const long long GT = (long long)gridDim.x * TB;
@@ -428,241 +449,377 @@ __global__ void __launch_bounds__(TB, 1) sweep_kernel(LayerArgs L, Plan P, Atoms
 #pragma unroll
       for (int p = 0; p < 2; ++p) B.c[2 * i + p] = make_float2(cc[8 * p + i], cc[8 * p + 4 + i]);
   }
-
-  // phase-2 role of this thread inside its half: slot = table entry, group = range of the tile's blocks
-  const int n_slots = P.n_slots;
-  const int n_groups = HB / n_slots;
-  const int grp = htid / n_slots, slot = htid - grp * n_slots;
-  const bool red_on = grp < n_groups;
-  const SlotDev sd = P.slots[slot];
-  float2* my = cs + htid;                      // this thread's block in the staging buffer: my[a * HBP]
-  double acc_gap = 0.0, acc_sse = 0.0;
-  int acc_n1 = 0, acc_nneg = 0;
   const int copy_off = (lane & 15) * 8;
   const unsigned char* cell_bytes = reinterpret_cast<const unsigned char*>(cell);
 
   // Warp-uniform control flow: every thread evaluates a block in every iteration (a thread without
-  // work re-evaluates a valid block whose results nothing reads), so the class / candidate loops
-  // below are uniform branches.
+  // work re-evaluates a valid block and stores nothing), so the class / candidate loops below are
+  // uniform branches.
   const unsigned fast_mask = __ballot_sync(0xFFFFFFFFu, fast[lane & (SOP_MAX_TABLES - 1)] != 0);
   const uint16_t* wcol = L.W + j * SOP_G;
   uint32_t wb[8];
   load_block_bits(wcol + min(r0, L.M - 1) * L.ldw, wb);
+  const size_t NBs = (size_t)L.NB;
 
   for (long long it = 0; it < n_iter; ++it) {
     const long long m = r0 + it * R;
     const bool on = lane_on && m < L.M;
-    // number of valid threads of this half in this iteration (the valid threads of a CTA form a prefix)
-    long long nv = min(L.M - it * R, R) * L.nbk - (long long)blockIdx.x * TB - (long long)half * HB;
-    nv = max(0ll, min((long long)HB, nv));
-    {
-      // ---- unpack, block statistics ----
-      float wf[16];
+    // ---- unpack, block statistics ----
+    float wf[16];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) { wf[2 * q] = bf16lo(wb[q]); wf[2 * q + 1] = bf16hi(wb[q]); }
-      const float amax = absmax_bits(wb);
-      load_block_bits(wcol + min(m + R, L.M - 1) * L.ldw, wb);   // prefetch the next row's block
+    for (int q = 0; q < 8; ++q) { wf[2 * q] = bf16lo(wb[q]); wf[2 * q + 1] = bf16hi(wb[q]); }
+    const float amax = absmax_bits(wb);
+    load_block_bits(wcol + min(m + R, L.M - 1) * L.ldw, wb);   // prefetch the next row's block
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int p = 0; p < 2; ++p) B.w[2 * i + p] = make_float2(wf[8 * p + i], wf[8 * p + 4 + i]);
-      float2 nw2[2];
-      nw2[0] = nw2[1] = make_float2(0.0f, 0.0f);
+      for (int p = 0; p < 2; ++p) B.w[2 * i + p] = make_float2(wf[8 * p + i], wf[8 * p + 4 + i]);
+    float2 nw2[2];
+    nw2[0] = nw2[1] = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int p = 0; p < 2; ++p) {
-          const float2 cw = __fmul2_rn(B.c[2 * i + p], B.w[2 * i + p]);
-          nw2[p] = __ffma2_rn(cw, B.w[2 * i + p], nw2[p]);
-        }
-      const float nw = fold(nw2[0], nw2[1]);
-      const long long blk = m * L.nbk + j;
+      for (int p = 0; p < 2; ++p) {
+        const float2 cw = __fmul2_rn(B.c[2 * i + p], B.w[2 * i + p]);
+        nw2[p] = __ffma2_rn(cw, B.w[2 * i + p], nw2[p]);
+      }
+    const float nw = fold(nw2[0], nw2[1]);
+    const size_t blk = (size_t)(m * L.nbk + j);
 
-      // candidates evaluated by an earlier call: their per-block values go from the arrays straight into
-      // the staging buffer (asynchronous 4-byte copies, no registers held) while this call's candidates
-      // are evaluated; the copies are awaited before the half's barrier
-      if (on) {
-        for (unsigned lm = P.load_mask; lm; lm &= lm - 1u) {
-          const int a = __ffs((int)lm) - 1;
-          const unsigned dst = (unsigned)__cvta_generic_to_shared(my + a * HBP);
-          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(block_cos + (size_t)a * L.NB + blk) : "memory");
-          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + 4u), "l"(block_sse + (size_t)a * L.NB + blk) : "memory");
-        }
+    for (int cl = 0; cl < P.n_classes; ++cl) {
+      const ClassDev& C = P.cls[cl];
+      if (C.n_cand == 0) continue;
+      float s_hat;
+      if (C.scope == 0) {
+        s_hat = amax > 0.0f ? cls_pot[cl] : 0.0f;
+      } else {
+        const float sigma = C.tmax == 1.0f ? amax : __fdiv_rn(amax, C.tmax);
+        s_hat = scale_quantize(sigma, cls_k[cl], F).s_hat;
       }
-      for (int cl = 0; cl < P.n_classes; ++cl) {
-        const ClassDev& C = P.cls[cl];
-        if (C.n_cand == 0) continue;
-        float s_hat;
-        if (C.scope == 0) {
-          s_hat = amax > 0.0f ? cls_pot[cl] : 0.0f;
+      const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
+      const float2 r2 = make_float2(rcp, rcp);
+#pragma unroll
+      for (int idx = 0; idx < 8; ++idx) B.u[idx] = __fmul2_rn(B.w[idx], r2);
+      if (C.kind == SOP_KIND_LUT) {
+        const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
+        const float invh = C.invh;
+        const unsigned pitch = (unsigned)P.n_tables * 128u;
+        const unsigned cbias = (unsigned)copy_off - __float_as_uint(MAGIC) * pitch;   // modulo 2^32
+#pragma unroll
+        for (int idx = 0; idx < 8; ++idx) {
+          const float tx = fminf(fmaxf(__fmaf_rn(B.u[idx].x, invh, toff), tlo), thi);
+          const float ty = fminf(fmaxf(__fmaf_rn(B.u[idx].y, invh, toff), tlo), thi);
+          B.off[2 * idx] = __float_as_uint(tx) * pitch + cbias;
+          B.off[2 * idx + 1] = __float_as_uint(ty) * pitch + cbias;
+        }
+        const unsigned moff = 2u * (unsigned)C.c_half * pitch + 2u * (unsigned)copy_off;
+        // tables of this class with a usable cell grid: the table slot is a compile-time displacement
+        const unsigned cls_fast = P.cls_tables[cl] & fast_mask;
+#pragma unroll
+        for (int T = 0; T < SOP_MAX_TABLES; ++T) {
+          if ((cls_fast >> T) & 1u) {
+            const unsigned char* tp = cell_bytes + T * 128;
+            const int ap = P.table_pos[T], an = P.table_neg[T];
+            if (ap != 255) emit(block_cos, block_sse, (size_t)ap * NBs + blk, on, nw, eval_lut_cells<false>(tp, moff, B, s_hat));
+            if (an != 255) emit(block_cos, block_sse, (size_t)an * NBs + blk, on, nw, eval_lut_cells<true>(tp, moff, B, s_hat));
+          }
+        }
+        // tables without a usable cell grid: binary search over the thresholds
+        if (P.cls_tables[cl] & ~fast_mask) {
+          for (int ci = 0; ci < C.n_cand; ++ci) {
+            const int a = C.cand[ci];
+            const int t = P.cand[a].table;
+            if ((fast_mask >> t) & 1u) continue;
+            const Metric mt = P.cand[a].neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
+                                            : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
+            emit(block_cos, block_sse, (size_t)a * NBs + blk, on, nw, mt);
+          }
+        }
+      } else if (C.kind == SOP_KIND_FP_E2M3) {
+        for (int ci = 0; ci < C.n_cand; ++ci)
+          emit(block_cos, block_sse, (size_t)C.cand[ci] * NBs + blk, on, nw, eval_generic<SOP_KIND_FP_E2M3, false>(nullptr, nullptr, B, s_hat));
+      } else if (C.kind == SOP_KIND_FP_GRID) {
+        for (int ci = 0; ci < C.n_cand; ++ci)
+          emit(block_cos, block_sse, (size_t)C.cand[ci] * NBs + blk, on, nw,
+               eval_generic<SOP_KIND_FP_GRID, false>(nullptr, nullptr, B, s_hat, C.grid));
+      } else {
+        for (int ci = 0; ci < C.n_cand; ++ci)
+          emit(block_cos, block_sse, (size_t)C.cand[ci] * NBs + blk, on, nw, eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat));
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The reduction of the per-block columns into table entries.
+//   A CTA takes tiles of RTILE blocks.  The columns (cosines and errors of every candidate that a task of the
+//   launch touches) of a tile are brought into a ring of shared-memory buffers by 16-byte asynchronous copies
+//   (cp.async, every thread a few), up to three tiles ahead of the arithmetic; a thread waits for its own copy
+//   groups and the one barrier per tile makes everybody's visible.  (One-dimensional bulk copies with an
+//   mbarrier, one kilobyte per column, were measured first: the per-request cost of twenty small requests per
+//   tile bound the kernel.)  16-byte copies need aligned addresses, which holds when the number of blocks is a
+//   multiple of four and the arrays are 16-byte aligned; otherwise (odd small layers) the tile is fetched with
+//   plain loads.  Nothing in this kernel spins on a flag.
+//   A warp owns up to three tasks.  A lane owns eight blocks of the tile (two runs of four): per
+//   entry it sums eight gaps 1 - cos (exact in fp32 for cos in [0.5, 1]) and eight errors in fp32, then adds
+//   both to the lane's FP64 accumulators of that entry, which live in shared memory.  At the end the 32 lanes'
+//   accumulators of an entry are added in lane order: the result depends on the grid size only.
+//   A signed four-way entry {i, -i, j, -j} is the two-way entry of "the better of i and -i" and "the better of
+//   j and -j" (ties to the atom; the sign of the error marks a negated winner), formed on the fly from the two
+//   columns of each base atom.  A block beyond the end of the layer reads as (cos 1, error 0): it adds nothing.
+// ---------------------------------------------------------------------------------------------
+constexpr int RTB = 256;              // threads per CTA of the reduction: eight warps
+constexpr int RTILE = 256;            // blocks per tile: eight per lane
+constexpr int ENT = TASK_PART + 1;    // entries of a task: the anchor alone, then its partners
+constexpr int MAX_STAGE = 4;           // tile buffers of the ring
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const Partial* partials, sop_pair_stat* s_pair, sop_pair_stat* s_sig,
+                              Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
+                              const int* cls_k, float wmax);
+
+constexpr int ACC_BYTES = 32 * 24;     // accumulators of one entry: 32 lanes x (two FP64 sums, two counts)
+
+__device__ __forceinline__ void lds128(unsigned addr, float (&v)[4]) {
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "r"(addr));
+}
+
+// The accumulators of one entry and lane, in shared memory: FP64 sums (gap, error) at sums + seat * 512 + lane * 16 and
+// counts (second candidate chosen, negated winner) at counts + seat * 256 + lane * 8.
+__device__ __forceinline__ void acc_add(unsigned sums, unsigned counts, float cg, float ce, int n1, int nn) {
+  double g, e;
+  asm volatile("ld.shared.v2.f64 {%0, %1}, [%2];" : "=d"(g), "=d"(e) : "r"(sums));
+  g += (double)cg; e += (double)ce;
+  asm volatile("st.shared.v2.f64 [%0], {%1, %2};" ::"r"(sums), "d"(g), "d"(e) : "memory");
+  int a, b;
+  asm volatile("ld.shared.v2.s32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(counts));
+  a += n1; b += nn;
+  asm volatile("st.shared.v2.s32 [%0], {%1, %2};" ::"r"(counts), "r"(a), "r"(b) : "memory");
+}
+
+// One task on the lane's eight blocks of one tile (blocks 4 lane .. 4 lane + 3 and the same 128 further on: two 128-bit
+// loads per column and array).  The code is the same for every warp and task -- tasks differ in data only -- and small:
+// a loop over the task's partners whose body handles the eight blocks.  Per entry the eight gaps and errors are summed
+// in fp32 and added to the lane's FP64 accumulators.
+//   cos_base / sse_base: shared-memory addresses of the tile's columns (for a signed task the signed-best columns);
+//   tk: the task (in shared memory); sums / counts: shared-memory addresses of this lane's accumulators of the task's
+//   first seat (the anchor alone), the partners' seats follow.
+template <bool SEL_ERR, bool SGN, bool REV>
+__device__ __forceinline__ void run_task(const TaskDev* __restrict__ tk, unsigned cos_base, unsigned sse_base, int lane, unsigned sums, unsigned counts) {
+  constexpr unsigned COL = RTILE * 4u;          // bytes of one column
+  const unsigned lane_off = (unsigned)lane * 16u;
+  float ac0[4], ac1[4], ae0[4], ae1[4];
+  {
+    const unsigned a = (unsigned)tk->anchor * COL + lane_off;
+    lds128(cos_base + a, ac0); lds128(cos_base + a + 512u, ac1);
+    lds128(sse_base + a, ae0); lds128(sse_base + a + 512u, ae1);
+  }
+  float ga0[4], ga1[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) { ga0[r] = __fsub_rn(1.0f, ac0[r]); ga1[r] = __fsub_rn(1.0f, ac1[r]); }
+  if (tk->self_slot != 255) {
+    float cg = 0.0f, ce = 0.0f;
+    int nn = 0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      cg = __fadd_rn(cg, ga0[r]); ce = __fadd_rn(ce, fabsf(ae0[r]));
+      cg = __fadd_rn(cg, ga1[r]); ce = __fadd_rn(ce, fabsf(ae1[r]));
+      if (SGN) nn += (int)(__float_as_uint(ae0[r]) >> 31) + (int)(__float_as_uint(ae1[r]) >> 31);
+    }
+    acc_add(sums, counts, cg, ce, 0, nn);
+  }
+  const int np = tk->n_part;
+#pragma unroll 1
+  for (int q = 0; q < np; ++q) {
+    const unsigned b = (unsigned)tk->part[q] * COL + lane_off;
+    float bc0[4], bc1[4], be0[4], be1[4];
+    lds128(cos_base + b, bc0); lds128(cos_base + b + 512u, bc1);
+    lds128(sse_base + b, be0); lds128(sse_base + b + 512u, be1);
+    float cg = 0.0f, ce = 0.0f;
+    int n1 = 0, nn = 0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      // mu: the entry's second candidate is strictly better and takes the block.  REV = false: the anchor is the
+      // first candidate and the partner the second; REV = true: the other way round.
+      bool mu0, mu1;
+      float g0, g1, e0, e1;
+      if (!REV) {
+        mu0 = SEL_ERR ? fabsf(be0[r]) < fabsf(ae0[r]) : bc0[r] > ac0[r];
+        mu1 = SEL_ERR ? fabsf(be1[r]) < fabsf(ae1[r]) : bc1[r] > ac1[r];
+        g0 = mu0 ? __fsub_rn(1.0f, bc0[r]) : ga0[r]; e0 = mu0 ? be0[r] : ae0[r];
+        g1 = mu1 ? __fsub_rn(1.0f, bc1[r]) : ga1[r]; e1 = mu1 ? be1[r] : ae1[r];
+      } else {
+        mu0 = SEL_ERR ? fabsf(ae0[r]) < fabsf(be0[r]) : ac0[r] > bc0[r];
+        mu1 = SEL_ERR ? fabsf(ae1[r]) < fabsf(be1[r]) : ac1[r] > bc1[r];
+        g0 = mu0 ? ga0[r] : __fsub_rn(1.0f, bc0[r]); e0 = mu0 ? ae0[r] : be0[r];
+        g1 = mu1 ? ga1[r] : __fsub_rn(1.0f, bc1[r]); e1 = mu1 ? ae1[r] : be1[r];
+      }
+      cg = __fadd_rn(cg, g0); ce = __fadd_rn(ce, fabsf(e0));
+      cg = __fadd_rn(cg, g1); ce = __fadd_rn(ce, fabsf(e1));
+      n1 += (mu0 ? 1 : 0) + (mu1 ? 1 : 0);
+      if (SGN) nn += (int)(__float_as_uint(e0) >> 31) + (int)(__float_as_uint(e1) >> 31);
+    }
+    acc_add(sums + (unsigned)(q + 1) * 512u, counts + (unsigned)(q + 1) * 256u, cg, ce, n1, nn);
+  }
+}
+
+template <bool SEL_ERR, int TPW, bool VEC>
+__global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, SeatsDev seats, int n_stage, int do_final, WsHeader* __restrict__ hdr,
+                                                     Partial* __restrict__ partials, const float* __restrict__ block_cos,
+                                                     const float* __restrict__ block_sse, sop_pair_stat* pair_table,
+                                                     sop_pair_stat* signed_table, sop_search_result* __restrict__ res,
+                                                     const sop_search_result* __restrict__ prev) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int A = seats.n_cols;                                            // columns of a tile buffer
+  const int NBUF = VEC ? n_stage : 1;                                    // tile buffers: a ring, filled n_stage - 1 tiles ahead
+  float* cos0 = reinterpret_cast<float*>(smem);                          // [NBUF][A][RTILE]
+  float* sse0 = cos0 + (size_t)NBUF * A * RTILE;                         // [NBUF][A][RTILE]
+  // signed-best columns of the tile in work
+  float* scos = sse0 + (size_t)NBUF * A * RTILE;                         // [n_bases][RTILE]
+  float* ssse = scos + (size_t)seats.n_bases * RTILE;                    // [n_bases][RTILE]
+  double2* acc_sums = reinterpret_cast<double2*>(ssse + (size_t)seats.n_bases * RTILE);   // [n_seats][32]: seat-major, then lane
+  int2* acc_counts = reinterpret_cast<int2*>(acc_sums + (size_t)seats.n_seats * 32);      // [n_seats][32]
+  __shared__ unsigned long long s_coloff[SOP_MAX_ATOMS];   // first element of every fetched column in the arrays
+  __shared__ TaskDev s_task[RTB / 32][TPW];        // anchors and partners translated to columns of the buffers
+  __shared__ int s_acc0[RTB / 32][TPW];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (lane < TPW) {
+    const int ti = seats.task[warp][lane];
+    TaskDev t;
+    if (ti != 255) {
+      t = P.tasks[ti];
+      const unsigned char* map = t.sgn ? seats.sb_slot : seats.col_slot;
+      t.anchor = map[t.anchor];
+      for (int q = 0; q < t.n_part; ++q) t.part[q] = map[t.part[q]];
+    } else { t.anchor = 0; t.n_part = 0; t.self_slot = 255; t.sgn = 2; }   // sgn 2: an empty seat
+    s_task[warp][lane] = t;
+    s_acc0[warp][lane] = seats.acc0[warp][lane];
+  }
+  for (int i = tid; i < seats.n_seats * 32; i += RTB) { acc_sums[i] = make_double2(0.0, 0.0); acc_counts[i] = make_int2(0, 0); }
+  if (tid < seats.n_cols) s_coloff[tid] = (unsigned long long)seats.cols[tid] * (unsigned long long)L.NB;
+  __syncthreads();
+  const int ncols = seats.n_cols, nbases = seats.n_bases;
+  const long long n_tiles = (L.NB + RTILE - 1) / RTILE;
+
+  // Every thread's share of the 16-byte copies of one tile into buffer b.  Chunk c = (column, array, run of four blocks);
+  // thread t takes the chunks t, t + 256, ...: always the same array and run, every second column.  Runs beyond the
+  // end of the layer are filled with (cos 1, error 0) instead.  One commit group per tile.
+  const int f_arr = (tid >> 6) & 1, f_ch = tid & 63;
+  const float* f_src = (f_arr ? block_sse : block_cos) + 4 * f_ch;
+  const unsigned f_dst = smem_u32(f_arr ? sse0 : cos0) + (unsigned)(((tid >> 7) * RTILE + 4 * f_ch) * 4);
+  auto fetch = [&](long long tile, int b) {
+    if (tile < n_tiles) {
+      const long long blk0 = tile * RTILE;
+      const bool live = blk0 + 4 * f_ch < L.NB;
+      unsigned dst = f_dst + (unsigned)(b * A * RTILE * 4);
+      for (int i = tid >> 7; i < ncols; i += 2, dst += 2u * RTILE * 4u) {
+        if (live) {
+          const float* src = f_src + s_coloff[i] + blk0;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
         } else {
-          const float sigma = C.tmax == 1.0f ? amax : __fdiv_rn(amax, C.tmax);
-          s_hat = scale_quantize(sigma, cls_k[cl], F).s_hat;
-        }
-        const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
-        const float2 r2 = make_float2(rcp, rcp);
-#pragma unroll
-        for (int idx = 0; idx < 8; ++idx) B.u[idx] = __fmul2_rn(B.w[idx], r2);
-        unsigned moff = 0;
-        if (C.kind == SOP_KIND_LUT) {
-          const float tlo = MAGIC, thi = MAGIC + (float)(2 * C.c_half), toff = MAGIC + (float)C.c_half;
-          const float invh = C.invh;
-          const unsigned pitch = (unsigned)P.n_tables * 128u;
-          const unsigned cbias = (unsigned)copy_off - __float_as_uint(MAGIC) * pitch;   // modulo 2^32
-#pragma unroll
-          for (int idx = 0; idx < 8; ++idx) {
-            const float tx = fminf(fmaxf(__fmaf_rn(B.u[idx].x, invh, toff), tlo), thi);
-            const float ty = fminf(fmaxf(__fmaf_rn(B.u[idx].y, invh, toff), tlo), thi);
-            B.off[2 * idx] = __float_as_uint(tx) * pitch + cbias;
-            B.off[2 * idx + 1] = __float_as_uint(ty) * pitch + cbias;
-          }
-          moff = 2u * (unsigned)C.c_half * pitch + 2u * (unsigned)copy_off;
-          // tables of this class with a usable cell grid: the table slot is a compile-time displacement
-          const unsigned cls_fast = P.cls_tables[cl] & fast_mask;
-#pragma unroll
-          for (int T = 0; T < SOP_MAX_TABLES; ++T) {
-            if ((cls_fast >> T) & 1u) {
-              const unsigned char* tp = cell_bytes + T * 128;
-              const int ap = P.table_pos[T], an = P.table_neg[T];
-              if (ap != 255) {
-                const Metric mt = eval_lut_cells<false>(tp, moff, B, s_hat);
-                const float cosv = block_cosine(nw, mt.nq, mt.dot);
-                my[ap * HBP] = make_float2(cosv, mt.sse);
-                if (block_cos && on) block_cos[(size_t)ap * L.NB + blk] = cosv;
-                if (block_sse && on) block_sse[(size_t)ap * L.NB + blk] = mt.sse;
-              }
-              if (an != 255) {
-                const Metric mt = eval_lut_cells<true>(tp, moff, B, s_hat);
-                const float cosv = block_cosine(nw, mt.nq, mt.dot);
-                my[an * HBP] = make_float2(cosv, mt.sse);
-                if (block_cos && on) block_cos[(size_t)an * L.NB + blk] = cosv;
-                if (block_sse && on) block_sse[(size_t)an * L.NB + blk] = mt.sse;
-              }
-            }
-          }
-          // tables without a usable cell grid: binary search over the thresholds
-          if (P.cls_tables[cl] & ~fast_mask) {
-            for (int ci = 0; ci < C.n_cand; ++ci) {
-              const int a = C.cand[ci];
-              const int t = P.cand[a].table;
-              if ((fast_mask >> t) & 1u) continue;
-              const Metric mt = P.cand[a].neg ? eval_generic<0, true>(tau + t * 32, lutv + t * 32, B, s_hat)
-                                              : eval_generic<0, false>(tau + t * 32, lutv + t * 32, B, s_hat);
-              const float cosv = block_cosine(nw, mt.nq, mt.dot);
-              my[a * HBP] = make_float2(cosv, mt.sse);
-              if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
-              if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
-            }
-          }
-        } else if (C.kind == SOP_KIND_FP_E2M3) {
-          for (int ci = 0; ci < C.n_cand; ++ci) {
-            const int a = C.cand[ci];
-            const Metric mt = eval_generic<SOP_KIND_FP_E2M3, false>(nullptr, nullptr, B, s_hat);
-            const float cosv = block_cosine(nw, mt.nq, mt.dot);
-            my[a * HBP] = make_float2(cosv, mt.sse);
-            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
-            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
-          }
-        } else if (C.kind == SOP_KIND_FP_GRID) {
-          for (int ci = 0; ci < C.n_cand; ++ci) {
-            const int a = C.cand[ci];
-            const Metric mt = eval_generic<SOP_KIND_FP_GRID, false>(nullptr, nullptr, B, s_hat, C.grid);
-            const float cosv = block_cosine(nw, mt.nq, mt.dot);
-            my[a * HBP] = make_float2(cosv, mt.sse);
-            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
-            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
-          }
-        } else {
-          for (int ci = 0; ci < C.n_cand; ++ci) {
-            const int a = C.cand[ci];
-            const Metric mt = eval_generic<SOP_KIND_FP_E4M3, false>(nullptr, nullptr, B, s_hat);
-            const float cosv = block_cosine(nw, mt.nq, mt.dot);
-            my[a * HBP] = make_float2(cosv, mt.sse);
-            if (block_cos && on) block_cos[(size_t)a * L.NB + blk] = cosv;
-            if (block_sse && on) block_sse[(size_t)a * L.NB + blk] = mt.sse;
-          }
+          const float v = f_arr ? 0.0f : 1.0f;
+          asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "f"(v) : "memory");
         }
       }
     }
-    if (P.load_mask) asm volatile("cp.async.wait_all;" ::: "memory");
-    half_barrier(half);
-    // ---- signed bests: for every base atom the better of the atom and its negation (ties to the atom), as
-    //      one more column of the staging buffer; the sign of the stored error marks a negated winner.  The
-    //      four-way entry (i, -i, j, -j) is then the two-way entry of the columns of i and j, with the same
-    //      tie order ----
-    if (P.n_bases) {
-      for (int bi = 0; bi < P.n_bases; ++bi) {
-        const int a = P.base_atom[bi];
-        const float2 vp = my[a * HBP], vn = my[(a + 1) * HBP];
-        const bool neg = SEL_ERR ? vn.y < vp.y : vn.x > vp.x;
-        my[(P.n_atoms + bi) * HBP] = make_float2(neg ? vn.x : vp.x, neg ? -vn.y : vp.y);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  long long tile = blockIdx.x;
+  if (VEC)
+    for (int b = 0; b < n_stage - 1; ++b) fetch(tile + (long long)b * gridDim.x, b);
+  int cur = 0;                 // buffer of the tile in work
+  for (; tile < n_tiles; tile += gridDim.x) {
+    float* cosb = cos0 + (size_t)cur * A * RTILE;
+    float* sseb = sse0 + (size_t)cur * A * RTILE;
+    if (VEC) {
+      // this thread's copies of the tile in work are complete when at most n_stage - 2 newer groups are still pending
+      if (n_stage == 4) asm volatile("cp.async.wait_group 2;" ::: "memory");
+      else if (n_stage == 3) asm volatile("cp.async.wait_group 1;" ::: "memory");
+      else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else {
+      const long long blk0 = tile * RTILE;
+      const int nv = (int)min((long long)RTILE, L.NB - blk0);
+      __syncthreads();                                      // everybody has finished the previous tile
+      for (int i = 0; i < ncols; ++i) {
+        const size_t a = seats.cols[i];
+        cosb[i * RTILE + tid] = tid < nv ? __ldg(block_cos + a * L.NB + blk0 + tid) : 1.0f;
+        sseb[i * RTILE + tid] = tid < nv ? __ldg(block_sse + a * L.NB + blk0 + tid) : 0.0f;
       }
-      half_barrier(half);
     }
-    // ---- phase 2: one slot per thread, a contiguous range of the half's tile; fp32 sums of eight gaps
-    //      1 - cos (exact for cos in [0.5, 1]) and eight errors, then FP64 ----
-    if (red_on) {
-      const int nvi = (int)nv;
-      const int len = (nvi + n_groups - 1) / n_groups;     // group g takes blocks [g len, (g + 1) len) of the tile
-      const int lo = grp * len, hi = min(nvi, lo + len);
-      const float2* pa = cs + sd.i0 * HBP + lo;
-      const float2* pb = cs + sd.i1 * HBP + lo;
-      int b = lo;
-      for (; b + 8 <= hi; b += 8, pa += 8, pb += 8) {
-        float cg = 0.0f, ce = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const float2 va = pa[k], vb = pb[k];
-          const bool mu = SEL_ERR ? fabsf(vb.y) < fabsf(va.y) : vb.x > va.x;
-          const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
-          acc_n1 += mu ? 1 : 0;
-          acc_nneg += (int)(__float_as_uint(se_) >> 31);       // a negated winner of a signed column (error stored negative)
-          cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-          ce = __fadd_rn(ce, fabsf(se_));
-        }
-        acc_gap += (double)cg; acc_sse += (double)ce;
+    if (nbases) {
+      // Signed-best columns: this thread's block.  The values come from other threads' copies, and the previous tile's
+      // readers of these columns must be done first: hence the barrier.
+      __syncthreads();
+      for (int i = 0; i < nbases; ++i) {
+        const int a = seats.bases[i], cp = seats.col_slot[a], cn = seats.col_slot[a + 1];     // the atom and its negation
+        const float pc = cosb[cp * RTILE + tid], pe = sseb[cp * RTILE + tid];
+        const float nc = cosb[cn * RTILE + tid], ne = sseb[cn * RTILE + tid];
+        const bool neg = SEL_ERR ? ne < pe : nc > pc;           // ties to the atom; a negative error marks a negated winner
+        scos[i * RTILE + tid] = neg ? nc : pc;
+        ssse[i * RTILE + tid] = neg ? -ne : pe;
       }
-      float cg = 0.0f, ce = 0.0f;
-      for (; b < hi; ++b, ++pa, ++pb) {
-        const float2 va = pa[0], vb = pb[0];
-        const bool mu = SEL_ERR ? fabsf(vb.y) < fabsf(va.y) : vb.x > va.x;
-        const float sc_ = mu ? vb.x : va.x, se_ = mu ? vb.y : va.y;
-        acc_n1 += mu ? 1 : 0;
-        acc_nneg += (int)(__float_as_uint(se_) >> 31);
-        cg = __fadd_rn(cg, __fsub_rn(1.0f, sc_));
-        ce = __fadd_rn(ce, fabsf(se_));
-      }
-      acc_gap += (double)cg; acc_sse += (double)ce;
     }
-    half_barrier(half);
+    // One barrier per tile: the tile is complete for everybody, and everybody has finished the previous tile, whose
+    // buffer (the one before this in the ring) the next copies refill.
+    __syncthreads();
+    if (VEC) fetch(tile + (long long)(n_stage - 1) * gridDim.x, cur == 0 ? n_stage - 1 : cur - 1);
+#pragma unroll 1
+    for (int k = 0; k < TPW; ++k) {
+      const TaskDev* tk = &s_task[warp][k];
+      const unsigned sums = smem_u32(acc_sums) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 16u;
+      const unsigned counts = smem_u32(acc_counts) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 8u;
+      const int sgn = tk->sgn;
+      const int rev = tk->rev;
+      if (sgn == 0) {
+        if (rev) run_task<SEL_ERR, false, true>(tk, smem_u32(cosb), smem_u32(sseb), lane, sums, counts);
+        else run_task<SEL_ERR, false, false>(tk, smem_u32(cosb), smem_u32(sseb), lane, sums, counts);
+      } else if (sgn == 1) {
+        if (rev) run_task<SEL_ERR, true, true>(tk, smem_u32(scos), smem_u32(ssse), lane, sums, counts);
+        else run_task<SEL_ERR, true, false>(tk, smem_u32(scos), smem_u32(ssse), lane, sums, counts);
+      }
+    }
+    if (VEC && ++cur == n_stage) cur = 0;
   }
 
-  // ---- per-CTA partials: every phase-2 thread parks its sums; one thread per slot adds them in a fixed order ----
-  __syncthreads();
-  Partial* sc = reinterpret_cast<Partial*>(cs_all);
-  { Partial p; p.gap = acc_gap; p.sse = acc_sse; p.n1 = acc_n1; p.nneg = acc_nneg; sc[tid] = p; }
-  __syncthreads();
-  if (tid < n_slots) {
-    Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
-    for (int h = 0; h < 2; ++h)
-      for (int g = 0; g < n_groups; ++g) {
-        const Partial q = sc[h * HB + g * n_slots + tid];
-        t.gap += q.gap; t.sse += q.sse; t.n1 += q.n1; t.nneg += q.nneg;
+  // ---- per-CTA partials: lane (k, q) of a warp adds the 32 lanes' sums of entry q of the warp's task k, in lane order ----
+  __syncwarp();
+  if (lane < TPW * ENT) {
+    const int k = lane / ENT, q = lane - k * ENT;
+    const TaskDev t = s_task[warp][k];
+    const int slot = t.sgn == 2 ? 255 : (q == 0 ? t.self_slot : (q - 1 < t.n_part ? t.slot[q - 1] : 255));
+    if (slot != 255) {
+      Partial p; p.gap = 0.0; p.sse = 0.0; p.n1 = 0; p.nneg = 0;
+      for (int l = 0; l < 32; ++l) {
+        const double2 a = acc_sums[(size_t)(s_acc0[warp][k] + q) * 32 + l];
+        const int2 c = acc_counts[(size_t)(s_acc0[warp][k] + q) * 32 + l];
+        p.gap += a.x; p.sse += a.y; p.n1 += c.x; p.nneg += c.y;
       }
-    partials[(size_t)blockIdx.x * MAX_SLOTS + tid] = t;
+      partials[(size_t)blockIdx.x * MAX_SLOTS + slot] = p;
+    }
   }
+  if (!do_final) return;
   // the CTA that arrives last adds everybody's partials and writes the tables; nobody waits for anybody
   __shared__ int s_last;
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = atomicAdd(&hdr->done_sweep, 1u) == gridDim.x - 1 ? 1 : 0;
+  if (tid == 0) s_last = atomicAdd(&hdr->done_reduce, 1u) == gridDim.x - 1 ? 1 : 0;
   __syncthreads();
   if (s_last) {
     __threadfence();
-    sop_pair_stat* s_pair = reinterpret_cast<sop_pair_stat*>(cs_all);
+    __shared__ int cls_k[SOP_MAX_CLASSES];
+    if (tid < SOP_MAX_CLASSES) {
+      const bool live = tid < P.n_classes;
+      cls_k[tid] = P.k_from_result ? (live && P.cls[tid].k_src >= 0 ? prev->k[P.cls[tid].k_src] : 0) : __ldcg(&hdr->cls_k[tid]);
+    }
+    const float wmax = P.k_from_result ? prev->layer_absmax : __uint_as_float(__ldcg(&hdr->wmax_bits));
+    __syncthreads();
+    sop_pair_stat* s_pair = reinterpret_cast<sop_pair_stat*>(smem);
     sop_pair_stat* s_sig = s_pair + SOP_MAX_ATOMS * SOP_MAX_ATOMS;
     finalize_body(L, P, (int)gridDim.x, partials, s_pair, s_sig, reinterpret_cast<Partial*>(s_sig + SOP_MAX_ATOMS * SOP_MAX_ATOMS), pair_table,
-                  signed_table, res, cls_k, layer_wmax);
+                  signed_table, res, cls_k, wmax);
   }
 }
 
@@ -697,12 +854,16 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
   const int A = P.n_atoms, tid = threadIdx.x, n_slots = P.n_slots;
   for (int i = tid; i < A * A; i += blockDim.x) {
     sop_pair_stat u; u.acos = 0.0; u.mse = 0.0; u.n_sel1 = -1; u.n_neg = -1;
-    s_pair[i] = u;
-    s_sig[i] = u;
+    // entries among candidates that an earlier call evaluated stay as that call left them in the tables
+    const int a = i / A, b = i - a * A;
+    const bool keep = P.keep_loaded && ((P.load_mask >> a) & 1u) && ((P.load_mask >> b) & 1u);
+    s_pair[i] = keep ? pair_table[i] : u;
+    s_sig[i] = keep && signed_table ? signed_table[i] : u;
   }
-  const int n_chunks = min((int)blockDim.x / n_slots, (grid + 3) / 4);   // at best one round of four loads per thread
-  const int slot = tid % n_slots, chunk = tid / n_slots;
-  if (chunk < n_chunks) {
+  __syncthreads();
+  const int n_chunks = max(1, min((int)blockDim.x / max(n_slots, 1), (grid + 3) / 4));   // at best one round of four loads per thread
+  const int slot = tid % max(n_slots, 1), chunk = tid / max(n_slots, 1);
+  if (chunk < n_chunks && n_slots > 0) {
     Partial t; t.gap = 0.0; t.sse = 0.0; t.n1 = 0; t.nneg = 0;
 #pragma unroll 1
     for (int g0 = chunk; g0 < grid; g0 += 4 * n_chunks) {
@@ -739,7 +900,7 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
     st.n_sel1 = t.n1;
     const SlotDev sd = P.slots[tid];
     if (sd.type == 0) { st.n_neg = 0; s_pair[sd.i0 * A + sd.i1] = st; }
-    else { st.n_neg = t.nneg; s_sig[P.base_atom[sd.i0 - A] * A + P.base_atom[sd.i1 - A]] = st; }
+    else { st.n_neg = t.nneg; s_sig[sd.i0 * A + sd.i1] = st; }
   }
   __syncthreads();
   for (int i = tid; i < A * A; i += blockDim.x) {
@@ -790,7 +951,7 @@ static double min_threshold_gap(const sop_atom& a) {
   return best;
 }
 
-int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mask, unsigned load_mask, int singles_only, Plan* P) {
+int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mask, unsigned load_mask, int singles_only, int keep_loaded, Plan* P) {
   memset(P, 0, sizeof(*P));
   const int n = A.n_atoms;
   P->n_atoms = n;
@@ -870,16 +1031,19 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mas
   }
   P->rows = rows;
   P->a_pad = n | 1;
-  // slots: pair-type first (singles as (a, a)), then signed
+  // slots: pair-type first (singles as (a, a)), then signed.  With keep_loaded an entry whose candidates were all
+  // evaluated by an earlier call is not formed again: the tables hold it.
+  P->keep_loaded = keep_loaded;
   int ns = 0;
   auto has = [present](int i) { return ((present >> i) & 1u) != 0; };
+  auto old = [keep_loaded, load_mask](int i) { return keep_loaded && ((load_mask >> i) & 1u) != 0; };
   for (int a = 0; a < n; ++a) {
-    if (!has(a)) continue;
+    if (!has(a) || old(a)) continue;
     P->slots[ns].type = 0; P->slots[ns].i0 = P->slots[ns].i1 = (unsigned char)a; ++ns;
   }
   for (int a = 0; a < n && !singles_only; ++a)
     for (int b = a + 1; b < n; ++b) {
-      if (!has(a) || !has(b)) continue;
+      if (!has(a) || !has(b) || (old(a) && old(b))) continue;
       if (A.atoms[a].kind != SOP_KIND_LUT || A.atoms[b].kind != SOP_KIND_LUT || A.atoms[a].n_bits != A.atoms[b].n_bits) continue;
       P->slots[ns].type = 0; P->slots[ns].i0 = (unsigned char)a; P->slots[ns].i1 = (unsigned char)b; ++ns;
     }
@@ -894,31 +1058,129 @@ int build_plan(const AtomsDev& A, const FmtDev& F, int k_mode, unsigned eval_mas
       const bool da = (A.dd_mask >> i) & 1u, db = (A.dd_mask >> (i + 1)) & 1u;
       base[i] = (da && db && a.n_entries == b.n_entries) || (!da && !db && same_table(a, b));
     }
-    int col[SOP_MAX_ATOMS];
-    for (int i = 0; i < n; ++i) {
-      col[i] = -1;
-      if (base[i]) { col[i] = n + P->n_bases; P->base_atom[P->n_bases++] = (unsigned char)i; }
-    }
+    for (int i = 0; i < n; ++i)
+      if (base[i]) P->base_atom[P->n_bases++] = (unsigned char)i;
     for (int i = 0; i < n; ++i)
       for (int j = i; j < n; ++j) {
         if (!base[i] || !base[j] || A.atoms[i].n_bits != A.atoms[j].n_bits) continue;
-        P->slots[ns].type = 1; P->slots[ns].i0 = (unsigned char)col[i]; P->slots[ns].i1 = (unsigned char)col[j]; ++ns;
+        if (old(i) && old(i + 1) && old(j) && old(j + 1)) continue;
+        P->slots[ns].type = 1; P->slots[ns].i0 = (unsigned char)i; P->slots[ns].i1 = (unsigned char)j; ++ns;   // base atoms
       }
   }
   if (ns > MAX_SLOTS) return SOP_ERR_ALPHABET;
   P->n_slots = ns;
-  if (ns > TB / 2) return SOP_ERR_ALPHABET;
+  // tasks of the reduction: repeatedly the candidate with the most entries still to form on one side of it (as their
+  // first candidate, the one that keeps a tie, or as their second) becomes an anchor and takes up to four of them as
+  // partners; its own (single) entry rides with its first task.  Signed entries (type 1) make tasks of their own.
+  {
+    bool done[MAX_SLOTS];
+    int self_of[2][SOP_MAX_ATOMS];
+    bool self_used[2][SOP_MAX_ATOMS];
+    for (int ty = 0; ty < 2; ++ty)
+      for (int c = 0; c < SOP_MAX_ATOMS; ++c) { self_of[ty][c] = -1; self_used[ty][c] = false; }
+    for (int i = 0; i < ns; ++i) {
+      done[i] = P->slots[i].i0 == P->slots[i].i1;
+      if (done[i]) self_of[P->slots[i].type][P->slots[i].i0] = i;
+    }
+    int nt = 0;
+    for (;;) {
+      int cnt[2][2][SOP_MAX_ATOMS] = {};          // [type][side][candidate]; side 0: the candidate is the entry's first
+      for (int i = 0; i < ns; ++i)
+        if (!done[i]) { ++cnt[P->slots[i].type][0][P->slots[i].i0]; ++cnt[P->slots[i].type][1][P->slots[i].i1]; }
+      int pt = -1, pside = 0, pc = 0;
+      for (int ty = 0; ty < 2; ++ty)
+        for (int side = 0; side < 2; ++side)
+          for (int c = 0; c < SOP_MAX_ATOMS; ++c) {
+            // at most four partners ride with one anchor, so more than four entries count like four
+            const int v = cnt[ty][side][c] < TASK_PART ? cnt[ty][side][c] : TASK_PART;
+            const int best = pt < 0 ? 0 : (cnt[pt][pside][pc] < TASK_PART ? cnt[pt][pside][pc] : TASK_PART);
+            if (v > best) { pt = ty; pside = side; pc = c; }
+          }
+      if (pt < 0) break;
+      if (nt == MAX_TASKS) return SOP_ERR_ALPHABET;
+      TaskDev& t = P->tasks[nt++];
+      memset(&t, 0, sizeof(t));
+      t.anchor = (unsigned char)pc;
+      t.sgn = (unsigned char)pt;
+      t.rev = (unsigned char)pside;
+      t.self_slot = 255;
+      if (self_of[pt][pc] >= 0 && !self_used[pt][pc]) { t.self_slot = (unsigned char)self_of[pt][pc]; self_used[pt][pc] = true; }
+      for (int i = 0; i < ns && t.n_part < TASK_PART; ++i) {
+        if (done[i] || P->slots[i].type != pt || (pside ? P->slots[i].i1 : P->slots[i].i0) != pc) continue;
+        const int q = t.n_part++;
+        t.part[q] = pside ? P->slots[i].i0 : P->slots[i].i1;
+        t.slot[q] = (unsigned char)i;
+        done[i] = true;
+      }
+    }
+    for (int ty = 0; ty < 2; ++ty)
+      for (int c = 0; c < SOP_MAX_ATOMS; ++c) {
+        if (self_of[ty][c] < 0 || self_used[ty][c]) continue;
+        if (nt == MAX_TASKS) return SOP_ERR_ALPHABET;
+        TaskDev& t = P->tasks[nt++];
+        memset(&t, 0, sizeof(t));
+        t.anchor = (unsigned char)c; t.sgn = (unsigned char)ty; t.self_slot = (unsigned char)self_of[ty][c];
+      }
+    // heaviest first (a signed task costs about twice as much per entry: two columns per candidate)
+    auto weight = [](const TaskDev& t) { return (2 + 3 * (int)t.n_part) * (t.sgn ? 2 : 1); };
+    for (int i = 1; i < nt; ++i)
+      for (int j = i; j > 0 && weight(P->tasks[j]) > weight(P->tasks[j - 1]); --j) { const TaskDev x = P->tasks[j]; P->tasks[j] = P->tasks[j - 1]; P->tasks[j - 1] = x; }
+    P->n_tasks = nt;
+  }
   return SOP_OK;
+}
+
+// Seats of one launch of the reduction: tasks [task0, task0 + n) dealt to the eight warps, always to the warp with the
+// least work so far that still has a free seat; the columns to fetch and their places in the tile buffers; one
+// accumulator seat per entry.  Returns the largest number of tasks on one warp.
+static int deal_tasks(const Plan& P, int task0, int n, SeatsDev* seats) {
+  int load[8] = {0}, used[8] = {0};
+  memset(seats, 0, sizeof(*seats));
+  memset(seats->task, 255, sizeof(seats->task));
+  memset(seats->col_slot, 255, sizeof(seats->col_slot));
+  memset(seats->sb_slot, 255, sizeof(seats->sb_slot));
+  int tpw = 0;
+  unsigned cand = 0, bases = 0;
+  for (int i = 0; i < n; ++i) {
+    const TaskDev& t = P.tasks[task0 + i];
+    int w = -1;
+    for (int x = 0; x < 8; ++x)
+      if (used[x] < MAX_TPW && (w < 0 || load[x] < load[w])) w = x;
+    seats->task[w][used[w]++] = (unsigned char)(task0 + i);
+    load[w] += 2 + 3 * (int)t.n_part;
+    tpw = tpw > used[w] ? tpw : used[w];
+    unsigned m = 1u << t.anchor;
+    for (int q = 0; q < t.n_part; ++q) m |= 1u << t.part[q];
+    if (t.sgn) { bases |= m; cand |= m | (m << 1); }     // a base atom stands for itself and its negation
+    else cand |= m;
+  }
+  for (int a = 0; a < P.n_atoms; ++a) {
+    if ((cand >> a) & 1u) { seats->col_slot[a] = (unsigned char)seats->n_cols; seats->cols[seats->n_cols++] = (unsigned char)a; }
+    if ((bases >> a) & 1u) { seats->sb_slot[a] = (unsigned char)seats->n_bases; seats->bases[seats->n_bases++] = (unsigned char)a; }
+  }
+  for (int w = 0; w < 8; ++w)
+    for (int k = 0; k < MAX_TPW; ++k) {
+      if (seats->task[w][k] == 255) continue;
+      seats->acc0[w][k] = (unsigned short)seats->n_seats;
+      seats->n_seats += 1 + P.tasks[seats->task[w][k]].n_part;
+    }
+  return tpw > 0 ? tpw : 1;
 }
 
 size_t sweep_smem_bytes(const Plan& P) {
   size_t b = (size_t)P.n_tables * P.rows * 16 * 8;
   b += SOP_MAX_TABLES * 32 * 4 * 2 + SOP_MAX_TABLES * 4 + SOP_MAX_CLASSES * 8;
-  size_t tile = (size_t)2 * (P.n_atoms + P.n_bases) * (TB / 2 + 1) * sizeof(float2);
-  // the closing reduction of the last CTA: two staged tables and one partial per thread
-  const size_t red = sizeof(Partial) * (size_t)TB + 2 * sizeof(sop_pair_stat) * SOP_MAX_ATOMS * SOP_MAX_ATOMS;
-  b += tile > red ? tile : red;
   return (b + 15) & ~(size_t)15;
+}
+
+// the ring of tile buffers, the signed-best columns, the lanes' accumulators; at least the room the closing
+// reduction of the last CTA needs
+static size_t reduce_smem_bytes(const SeatsDev& S, int n_stage) {
+  const size_t tiles = ((size_t)n_stage * S.n_cols + S.n_bases) * 2 * RTILE * sizeof(float);
+  const size_t acc = (size_t)S.n_seats * ACC_BYTES;
+  const size_t fin = sizeof(Partial) * (size_t)RTB + 2 * sizeof(sop_pair_stat) * SOP_MAX_ATOMS * SOP_MAX_ATOMS;
+  const size_t b = tiles + acc;
+  return ((b > fin ? b : fin) + 127) & ~(size_t)127;
 }
 
 // Doubles the cell width of the LUT class with the most rows (its tables then hold several thresholds per cell
@@ -979,14 +1241,20 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   const bool k_from_result = k_mode == SOP_K_FROM_RESULT;
   if (k_mode != SOP_K_AUTO && !k_from_result && (k_mode < -64 || k_mode > 64)) return SOP_ERR_RANGE;
   if (k_from_result && (!prev_result_dev || prev_result_dev == result_dev)) return SOP_ERR_NULL;
-  if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < ws_total()) return SOP_ERR_WORKSPACE;
+  const long long NB = M * (K / SOP_G);
+  // without the caller's per-block arrays the columns live behind the fixed part of the workspace
+  const bool own_columns = !block_cos_dev || !block_sse_dev;
+  const size_t col_bytes = (((size_t)n_atoms * (size_t)NB * sizeof(float)) + 255) & ~(size_t)255;
+  const size_t need = ws_total() + (own_columns ? 2 * col_bytes : 0);
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < need) return SOP_ERR_WORKSPACE;
   const unsigned all = n_atoms >= 32 ? 0xFFFFFFFFu : ((1u << n_atoms) - 1u);
   eval_mask &= all;
   if ((load_mask & ~all) || (load_mask & eval_mask) || !(eval_mask | load_mask)) return SOP_ERR_ALPHABET;
-  if (load_mask && (!block_cos_dev || !block_sse_dev)) return SOP_ERR_NULL;
-  if (flags & ~(SOP_SEARCH_SINGLES_ONLY | SOP_SEARCH_SELECT_MSE)) return SOP_ERR_RANGE;
+  if (load_mask && own_columns) return SOP_ERR_NULL;
+  if (flags & ~(SOP_SEARCH_SINGLES_ONLY | SOP_SEARCH_SELECT_MSE | SOP_SEARCH_KEEP_LOADED_ENTRIES)) return SOP_ERR_RANGE;
+  const int keep_loaded = (flags & SOP_SEARCH_KEEP_LOADED_ENTRIES) && load_mask ? 1 : 0;
   Plan P;
-  if ((rc = build_plan(A, F, k_from_result ? 0 : k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, &P))) return rc;
+  if ((rc = build_plan(A, F, k_from_result ? 0 : k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, keep_loaded, &P))) return rc;
   P.k_from_result = k_from_result ? 1 : 0;
   for (int c = 0; c < P.n_classes; ++c) {
     // the shift of a class is read from a candidate of that class that the earlier call had
@@ -997,15 +1265,17 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   }
 
   LayerArgs L;
-  L.W = (const uint16_t*)W_dev; L.c = c_dev; L.M = M; L.K = K; L.ldw = ldw; L.nbk = K / SOP_G; L.NB = M * L.nbk;
+  L.W = (const uint16_t*)W_dev; L.c = c_dev; L.M = M; L.K = K; L.ldw = ldw; L.nbk = K / SOP_G; L.NB = NB;
   cudaStream_t st = (cudaStream_t)stream;
   unsigned char* ws = (unsigned char*)workspace_dev;
   WsHeader* hdr = (WsHeader*)ws;
   unsigned* hist = (unsigned*)(ws + ws_hist_off());
   Partial* partials = (Partial*)(ws + ws_part_off());
+  float* cos_cols = own_columns ? (float*)(ws + ws_total()) : block_cos_dev;
+  float* sse_cols = own_columns ? (float*)(ws + ws_total() + col_bytes) : block_sse_dev;
 
   // everything that can refuse the call is decided before the first enqueue
-  constexpr size_t SMEM_MAX = 226 * 1024;   // 227 KB per CTA minus the kernel's few static bytes
+  constexpr size_t SMEM_MAX = 226 * 1024;   // 227 KB per CTA minus the kernels' few static bytes
   size_t smem = sweep_smem_bytes(P);
   while (smem > SMEM_MAX && coarsen_cells(&P)) smem = sweep_smem_bytes(P);   // cell tables too large: coarser cells, exact search where needed
   if (smem > SMEM_MAX) return SOP_ERR_ALPHABET;
@@ -1016,6 +1286,14 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   const long long min_grid = (L.nbk + TB - 1) / TB;
   if (grid < min_grid) grid = min_grid;
   if (grid > MAX_GRID) return SOP_ERR_SHAPE;
+  // the reduction: up to MAX_TPW tasks per warp and launch, more launches for more tasks; persistent grid over tiles.
+  // 16-byte copies need 16-byte aligned column starts and runs: a block count that is a multiple of four.
+  constexpr int PER_LAUNCH = (RTB / 32) * MAX_TPW;
+  const int n_launch = P.n_tasks ? (P.n_tasks + PER_LAUNCH - 1) / PER_LAUNCH : 1;
+  const bool vec = (L.NB % 4) == 0 && (((uintptr_t)cos_cols | (uintptr_t)sse_cols) & 15u) == 0;
+  const long long n_tiles = (L.NB + RTILE - 1) / RTILE;
+  long long rgrid = n_tiles < (long long)sms * 2 ? n_tiles : (long long)sms * 2;
+  if (rgrid < 1) rgrid = 1;
 
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
   if (!k_from_result) {
@@ -1025,20 +1303,46 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     prepass_kernel<<<pgrid, 256, 0, st>>>(L, P, F, hist, hdr);
     SOP_CUDA_TRY(cudaGetLastError());
   }
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
-    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
-    smem_set = SMEM_MAX;
+  static bool attr_set = false;
+  if (!attr_set) {
+    SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
+#define SOP_REDUCE_ATTR(SE, T, BK) \
+  SOP_CUDA_TRY(cudaFuncSetAttribute(reduce_kernel<SE, T, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX))
+    SOP_REDUCE_ATTR(false, 1, false); SOP_REDUCE_ATTR(false, 2, false); SOP_REDUCE_ATTR(false, 3, false);
+    SOP_REDUCE_ATTR(false, 1, true); SOP_REDUCE_ATTR(false, 2, true); SOP_REDUCE_ATTR(false, 3, true);
+    SOP_REDUCE_ATTR(true, 1, false); SOP_REDUCE_ATTR(true, 2, false); SOP_REDUCE_ATTR(true, 3, false);
+    SOP_REDUCE_ATTR(true, 1, true); SOP_REDUCE_ATTR(true, 2, true); SOP_REDUCE_ATTR(true, 3, true);
+#undef SOP_REDUCE_ATTR
+    attr_set = true;
   }
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
-  if (flags & SOP_SEARCH_SELECT_MSE)
-    sweep_kernel<true><<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev,
-                                                    signed_table_dev, result_dev, prev_result_dev);
-  else
-    sweep_kernel<false><<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, partials, block_cos_dev, block_sse_dev, pair_table_dev,
-                                                     signed_table_dev, result_dev, prev_result_dev);
-  SOP_CUDA_TRY(cudaGetLastError());
+  if (eval_mask) {
+    sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, cos_cols, sse_cols, prev_result_dev);
+    SOP_CUDA_TRY(cudaGetLastError());
+  }
+  const bool sel_err = (flags & SOP_SEARCH_SELECT_MSE) != 0;
+  for (int l = 0; l < n_launch; ++l) {
+    const int task0 = l * PER_LAUNCH;
+    const int nt = P.n_tasks - task0 < PER_LAUNCH ? P.n_tasks - task0 : PER_LAUNCH;
+    SeatsDev seats;
+    const int tpw = deal_tasks(P, task0, nt, &seats);
+    // as many tile buffers as still let two CTAs share an SM (at most 16 columns, 8 signed-best ones and 120 seats: two
+    // buffers always fit one CTA)
+    int n_stage = vec ? MAX_STAGE : 1;
+    while (n_stage > 2 && reduce_smem_bytes(seats, n_stage) > SMEM_MAX / 2) --n_stage;
+    const size_t rs = reduce_smem_bytes(seats, n_stage);
+    const int fin = l == n_launch - 1 ? 1 : 0;
+#define SOP_LAUNCH_REDUCE(SE, T, BK)                                                                                          \
+  reduce_kernel<SE, T, BK><<<(int)rgrid, RTB, rs, st>>>(L, P, seats, n_stage, fin, hdr, partials, cos_cols, sse_cols, pair_table_dev, \
+                                                        signed_table_dev, result_dev, prev_result_dev)
+#define SOP_LAUNCH_REDUCE_T(SE, BK) \
+  do { if (tpw == 1) SOP_LAUNCH_REDUCE(SE, 1, BK); else if (tpw == 2) SOP_LAUNCH_REDUCE(SE, 2, BK); else SOP_LAUNCH_REDUCE(SE, 3, BK); } while (0)
+    if (sel_err) { if (vec) SOP_LAUNCH_REDUCE_T(true, true); else SOP_LAUNCH_REDUCE_T(true, false); }
+    else { if (vec) SOP_LAUNCH_REDUCE_T(false, true); else SOP_LAUNCH_REDUCE_T(false, false); }
+#undef SOP_LAUNCH_REDUCE_T
+#undef SOP_LAUNCH_REDUCE
+    SOP_CUDA_TRY(cudaGetLastError());
+  }
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
   return SOP_OK;
 }

@@ -112,7 +112,6 @@ class LayerSweep:
             self.ws_norm = B.alloc_workspace(B.channel_norms_workspace(T, K), d)
             self.ws_search = B.alloc_workspace(B.pair_search_workspace(M, K, nF), d)
             self.ws_lloyd = B.alloc_workspace(B.dd4_lloyd_workspace(M, K), d)
-        self.rom_table = B.new_pair_table(nF, d)
         self.rom_result = B.new_result(d)
         self.fixed_mask = ((1 << nF) - 1) & ~self.dd_mask
         self.dd_lut = torch.zeros(B.MAX_ENTRIES, dtype=torch.float32, device=d)
@@ -150,22 +149,23 @@ class LayerSweep:
             B.sop_channel_norms(X, self.c, self.ws_norm, stream)
             n += 2
         if self.iters > 0:
-            B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.rom_table, None, self.rom_result, self.ws_search,
-                              block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
-                              singles_only=True, stream=stream)
-            n += 2
+            # every fixed candidate and every table entry among them; the best single of the result is FMTa
+            B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.rom_result,
+                              self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
+                              stream=stream)
+            n += 3
             B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
             n += self.lloyd_launches
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
                               block_sse=self.full_sse, eval_mask=self.dd_mask, load_mask=self.fixed_mask,
-                              k_mode=B.K_FROM_RESULT, prev_result=self.rom_result, stream=stream)
+                              k_mode=B.K_FROM_RESULT, prev_result=self.rom_result, keep_loaded=True, stream=stream)
         else:
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
             n += 1
-        n += 1
+        n += 2
         B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, search_result=self.result,
                    index_a=0 if self.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if self.single else B.PAIR_FROM_RESULT,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,

@@ -38,7 +38,7 @@ def gpu_norms(B, X):
     return c
 
 
-def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0, two_calls_split=None):
+def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0, two_calls_split=None, keep=False):
     M, K = W.shape
     A = len(atoms)
     NB = M * K // 16
@@ -56,13 +56,14 @@ def gpu_search(B, W, c, fmt, atoms, k_mode=None, dd_lut=None, dd_mask=0, two_cal
         first = two_calls_split
         rest = ((1 << A) - 1) & ~first
         res1 = B.new_result(dev())
+        # (keep: the first call forms every entry among its candidates and the second one keeps them)
         B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res1, ws, k_mode=km, dd_lut=dd_lut, dd_mask=dd_mask, block_cos=bc,
-                          block_sse=bs, eval_mask=first, singles_only=True)
+                          block_sse=bs, eval_mask=first, singles_only=not keep)
         torch.cuda.synchronize()
         first_pass = dict(pair=B.read_pair_table(pt, A).copy(), **B.read_result(res1))
         # the second call takes the shifts and max|W| from the first call's result instead of reading W again
         B.sop_pair_search(Wd, cd, fmt, atoms, pt, st, res, ws, k_mode=B.K_FROM_RESULT, prev_result=res1, dd_lut=dd_lut,
-                          dd_mask=dd_mask, block_cos=bc, block_sse=bs, eval_mask=rest, load_mask=first)
+                          dd_mask=dd_mask, block_cos=bc, block_sse=bs, eval_mask=rest, load_mask=first, keep_loaded=keep)
     torch.cuda.synchronize()
     out = dict(pair=B.read_pair_table(pt, A), signed=B.read_pair_table(st, A), block_cos=bc.cpu().numpy(),
                block_sse=bs.cpu().numpy(), res_t=res, Wd=Wd, cd=cd, bc_t=bc, **B.read_result(res))
@@ -207,6 +208,16 @@ def test_sweep_in_two_calls_equals_one_call(B, fmt_name):
     lut_first = [a for a in range(A) if present[a] and atoms[a].kind == I.KIND_LUT]
     assert fp["best"][2] == max(lut_first, key=lambda a: (want["pair"]["acos"][a, a], -a))
     assert fp["best"][0] == -1 and fp["best"][3] == -1
+    # the first call forms every entry among its candidates, the second keeps those and adds the entries of the new ones
+    kept = gpu_search(B, L.W, c, fmt, atoms, two_calls_split=first, keep=True)
+    assert_tables(kept, want, len(atoms))
+    fp = kept["first_pass"]
+    for a in range(A):
+        for b in range(a, A):
+            both = (first >> a) & 1 and (first >> b) & 1
+            assert (fp["pair"]["n_sel1"][a, b] >= 0) == bool(both and want["pair"]["n_sel1"][a, b] >= 0)
+            if fp["pair"]["n_sel1"][a, b] >= 0:
+                assert fp["pair"]["n_sel1"][a, b] == want["pair"]["n_sel1"][a, b]
 
 
 def test_negation_symmetry_on_gpu(B):
