@@ -252,16 +252,20 @@ int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE
 #define SOP_LLOYD_LAUNCH_PER_ITERATION 8
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
 /* Number of kernel launches one sop_dd4_lloyd call with these sizes and flags makes on the current device
- * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch when
- * every CTA of the iteration grid can be resident at once; otherwise there is one launch per iteration. */
+ * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch where the
+ * device supports such launches (the grid is cut to what is resident at once); otherwise, or with
+ * SOP_LLOYD_LAUNCH_PER_ITERATION, there is one launch per iteration. */
 int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches);
 /* Launch-shape parameters of sop_dd4_lloyd for this process (test aid, no counterpart in the paper; results do
  * not depend on them).  cell_spill_tiles in [1, 128]: cache tiles a CTA sorts between two transfers of its
  * per-cell partial sums to the global sums (default 128, the most the 32-bit limbs allow);
  * cache_ctas >= 0: largest grid of the cache kernel (0 = default, three CTAs per SM);
- * tiles_per_warp in [1, 4]: most cache tiles one warp of an iteration CTA may walk (default 4).
+ * tiles_per_warp in [1, 4]: cache tiles one warp of an iteration CTA walks between two folds of its 32-bit partial
+ *   sums into 64-bit ones (default 4, the most the partial sums hold).
+ * iter_ctas >= 0: largest grid of the iteration kernels (0 = default: one warp per cache tile of the expected pool,
+ *   at most eight CTAs per SM and, in one cooperative launch, what is resident at once).
  * SOP_ERR_RANGE outside these ranges. */
-int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp);
+int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp, int iter_ctas);
 int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                   const sop_scale_fmt* fmt, int k_mode, const sop_search_result* search_dev,
                   const float* block_metric_dev, long long pool_rank, float pool_threshold, int flags,

@@ -158,9 +158,9 @@ def dd4_lloyd_launches(M: int, K: int, iters: int, flags: int = 0) -> int:
     return n.value
 
 
-def dd4_lloyd_tuning(cell_spill_tiles: int = 128, cache_ctas: int = 0, tiles_per_warp: int = 4) -> None:
+def dd4_lloyd_tuning(cell_spill_tiles: int = 128, cache_ctas: int = 0, tiles_per_warp: int = 4, iter_ctas: int = 0) -> None:
     """Launch-shape parameters of ``sop_dd4_lloyd`` (test aid; the defaults restore the library's own)."""
-    _check(lib().sop_dd4_lloyd_tuning(cell_spill_tiles, cache_ctas, tiles_per_warp), "sop_dd4_lloyd_tuning")
+    _check(lib().sop_dd4_lloyd_tuning(cell_spill_tiles, cache_ctas, tiles_per_warp, iter_ctas), "sop_dd4_lloyd_tuning")
 
 
 class LloydNotFinished(RuntimeError):

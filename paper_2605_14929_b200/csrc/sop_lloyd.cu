@@ -339,13 +339,13 @@ __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exa
 
 constexpr int CELL_LIMBS = 14;
 constexpr int CELL_SPILL_TILES_MAX = 128;     // a low limb takes at most 258 * (2^16 - 1) per tile: 128 tiles stay below 2^32
-constexpr int TILES_PER_WARP_MAX = 4;         // bound of the limb sums of an iteration CTA (see flush_limbs)
+constexpr int TILES_PER_WARP_MAX = 4;         // tiles a warp of an iteration CTA walks between two folds of its limb sums (see flush_limbs)
 
 // Launch-shape parameters of the pool cache and of the iteration grid.  The defaults are the largest values the
 // limb arithmetic allows; sop_dd4_lloyd_tuning lowers them (tests reach the mid-loop spill and a multi-tile warp
 // share on small layers that way).  Results do not depend on them.
-struct LloydTune { int spill_tiles, cache_ctas, tiles_per_warp; };
-static LloydTune g_tune = {CELL_SPILL_TILES_MAX, 0, TILES_PER_WARP_MAX};
+struct LloydTune { int spill_tiles, cache_ctas, tiles_per_warp, iter_ctas; };
+static LloydTune g_tune = {CELL_SPILL_TILES_MAX, 0, TILES_PER_WARP_MAX, 0};
 constexpr double MOMENT_UNIT = 1099511627776.0;   // 2^40
 
 __device__ __forceinline__ void add_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell, long long v) {
@@ -499,7 +499,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
 // accumulators with shared-memory atomics (a few hundred elements per tile).
 constexpr int MAX_SPLIT = 32;   // a table has at most 31 thresholds, so at most 31 cells hold one
 
-// A CTA walks at most 2^17 elements per launch (8 warps, a few tiles each), every element adds at most
+// Between two folds a CTA walks at most 2^17 elements (8 warps, at most four tiles each), every element adds at most
 // 2^24 to n and 2^32 in magnitude to sv, and there is at most one flush per element.  With 12-bit low
 // limbs every limb sum stays below 2^31: n = 12 bits + the rest, sv = 12 + 12 bits + the signed rest.
 __device__ __forceinline__ void flush_limbs(unsigned* n0, unsigned* n1, unsigned* s0, unsigned* s1, int* s2, int code,
@@ -516,7 +516,8 @@ __device__ __forceinline__ void flush_limbs(unsigned* n0, unsigned* n1, unsigned
 // CTA, so it is read past the L1.
 template <bool FRESH>
 __device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                int it, int last, float* __restrict__ out_lut, unsigned* counter, bool reset_counter) {
+                                                int it, int last, float* __restrict__ out_lut, unsigned* counter, bool reset_counter,
+                                                unsigned fold_period) {
   __shared__ __align__(16) IterDesc d;
   __shared__ unsigned long long sN[SOP_MAX_ENTRIES], sS[SOP_MAX_ENTRIES];
   // flushes of the element walk: native 32-bit atomics on limbs, combined into sN / sS afterwards
@@ -587,7 +588,23 @@ __device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __r
       }
     }
   }
-  for (unsigned tile = blockIdx.x * (LTB / 32) + warp; tile < n_tiles; tile += gridDim.x * (LTB / 32)) {
+  // Round k of the CTA covers tiles (k gridDim + blockIdx) 8 .. + 7, one per warp.  The limb accumulators hold what a
+  // warp adds in at most four rounds (flush_limbs), so every fold_period <= 4 rounds the CTA folds them into its
+  // 64-bit sums: a CTA may then walk any number of tiles, and a grid that is resident at once serves any pool.
+  for (unsigned k = 0;; ++k) {
+    const unsigned tile0 = (k * gridDim.x + blockIdx.x) * (LTB / 32);
+    if (tile0 >= n_tiles) break;                       // the same for every warp of the CTA
+    if (k != 0 && k % fold_period == 0) {
+      __syncthreads();
+      if (tid < 32 && !last) {
+        sN[tid] += (unsigned long long)lN[0][tid] + ((unsigned long long)lN[1][tid] << 12);
+        sS[tid] += (unsigned long long)lS0[tid] + ((unsigned long long)lS1[tid] << 12) + ((unsigned long long)(long long)lS2[tid] << 24);
+        lN[0][tid] = lN[1][tid] = lS0[tid] = lS1[tid] = 0; lS2[tid] = 0;
+      }
+      __syncthreads();
+    }
+    const unsigned tile = tile0 + warp;
+    if (tile >= n_tiles) continue;
     const unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
     const uint2* src = a.cache + (size_t)tile * TILE_ELEMS;
     // segment lengths -> exclusive offsets (one cell per lane)
@@ -711,8 +728,8 @@ __device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __r
 
 // One launch per iteration (the stream orders the iterations).
 __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                          int it, int last, float* __restrict__ out_lut) {
-  lloyd_iteration<false>(a, ws, distortion, it, last, out_lut, &ws->done, true);
+                                                          int it, int last, float* __restrict__ out_lut, unsigned fold_period) {
+  lloyd_iteration<false>(a, ws, distortion, it, last, out_lut, &ws->done, true, fold_period);
 }
 
 // All iterations in one launch (launched cooperatively: every CTA is resident).  Between two iterations the
@@ -722,11 +739,11 @@ __global__ void __launch_bounds__(LTB) lloyd_split_kernel(LloydArgs a, LloydWs* 
 constexpr unsigned WAIT_POLLS = 1u << 22;     // times ~100 ns: about half a second
 
 __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, LloydWs* __restrict__ ws, double* __restrict__ distortion,
-                                                               int iters, float* __restrict__ out_lut) {
+                                                               int iters, float* __restrict__ out_lut, unsigned fold_period) {
   __shared__ int s_stop;
   for (int it = 0; it <= iters; ++it) {
     const int last = it == iters;
-    const bool updater = lloyd_iteration<true>(a, ws, distortion, it, last, out_lut, &ws->arrive[it], false);
+    const bool updater = lloyd_iteration<true>(a, ws, distortion, it, last, out_lut, &ws->arrive[it], false, fold_period);
     if (last) break;
     __syncthreads();                       // the updater's first warp has written the descriptor
     if (threadIdx.x == 0) {
@@ -755,20 +772,17 @@ __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, Lloy
 
 int num_sms();
 
-// Grid of the iteration kernels and whether all iterations run in one cooperative launch: they do when every
-// CTA of a grid that keeps to four tiles per warp can be resident at once (the CTAs wait for one another
-// between iterations); otherwise there is one launch per iteration.
+// Grid of the iteration kernels and whether all iterations run in one cooperative launch: they do wherever the device
+// launches cooperatively (the CTAs wait for one another between iterations, so the whole grid has to be resident:
+// the grid is cut to what is, and a CTA walks as many tiles as that takes); otherwise there is one launch per iteration.
 static bool lloyd_iteration_plan(long long NB, long long pool_blocks, int iters, int flags, long long* grid_out) {
   const int sms = num_sms();
-  const long long tiles = (NB + LTB - 1) / LTB;                     // all blocks in the pool: the most there can be
-  const long long likely = (pool_blocks + LTB - 1) / LTB;           // the pool without ties at its threshold
+  const long long likely = (pool_blocks + LTB - 1) / LTB;           // cache tiles of the pool without ties at its threshold
   long long grid = (likely + LTB / 32 - 1) / (LTB / 32);            // one warp per cache tile
   if (grid > (long long)sms * 8) grid = (long long)sms * 8;
-  // at most four tiles per warp: bounds the limb sums of a CTA's shared-memory accumulators
-  const long long per_cta = (long long)g_tune.tiles_per_warp * (LTB / 32);
-  const long long need = (tiles + per_cta - 1) / per_cta;
-  if (grid < need) grid = need;
+  if (g_tune.iter_ctas > 0 && grid > g_tune.iter_ctas) grid = g_tune.iter_ctas;
   if (grid < 1) grid = 1;
+  (void)NB;
   static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
   if (coop_blocks_per_sm < 0) {
     int dev = 0, coop = 0, nb = 0;
@@ -781,7 +795,7 @@ static bool lloyd_iteration_plan(long long NB, long long pool_blocks, int iters,
   }
   const long long resident = (long long)coop_blocks_per_sm * sms;
   bool persistent = false;
-  if (iters >= 1 && resident >= need && resident >= 1 && !(flags & SOP_LLOYD_LAUNCH_PER_ITERATION)) {
+  if (iters >= 1 && resident >= 1 && !(flags & SOP_LLOYD_LAUNCH_PER_ITERATION)) {
     persistent = true;
     if (grid > resident) grid = resident;
   }
@@ -803,13 +817,14 @@ int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* 
   return SOP_OK;
 }
 
-int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp) {
+int sop_dd4_lloyd_tuning(int cell_spill_tiles, int cache_ctas, int tiles_per_warp, int iter_ctas) {
   using namespace sop;
   if (cell_spill_tiles < 1 || cell_spill_tiles > CELL_SPILL_TILES_MAX || cache_ctas < 0 || tiles_per_warp < 1 ||
-      tiles_per_warp > TILES_PER_WARP_MAX) return SOP_ERR_RANGE;
+      tiles_per_warp > TILES_PER_WARP_MAX || iter_ctas < 0) return SOP_ERR_RANGE;
   g_tune.spill_tiles = cell_spill_tiles;
   g_tune.cache_ctas = cache_ctas;
   g_tune.tiles_per_warp = tiles_per_warp;
+  g_tune.iter_ctas = iter_ctas;
   return SOP_OK;
 }
 
@@ -893,14 +908,15 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   }
   long long grid = 1;
   const bool persistent = lloyd_iteration_plan(NB, by_threshold ? NB : pool_rank, iters, flags, &grid);
+  unsigned fold_period = (unsigned)g_tune.tiles_per_warp;
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
   if (persistent) {
-    void* kargs[] = {(void*)&a, (void*)&ws, (void*)&distortion_dev, (void*)&iters, (void*)&out_lut_dev};
+    void* kargs[] = {(void*)&a, (void*)&ws, (void*)&distortion_dev, (void*)&iters, (void*)&out_lut_dev, (void*)&fold_period};
     SOP_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)lloyd_persistent_kernel, dim3((unsigned)grid), dim3(LTB), kargs, 0, st));
   } else {
     for (int it = 0; it <= iters; ++it) {
       const int last = it == iters;
-      lloyd_split_kernel<<<(int)grid, LTB, 0, st>>>(a, ws, distortion_dev, it, last, out_lut_dev);
+      lloyd_split_kernel<<<(int)grid, LTB, 0, st>>>(a, ws, distortion_dev, it, last, out_lut_dev, fold_period);
     }
   }
   if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;

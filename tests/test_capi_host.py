@@ -162,8 +162,8 @@ def test_lloyd_status_entry_is_read_on_the_host(lib):
 
 
 def test_lloyd_tuning_ranges(lib):
-    assert lib.sop_dd4_lloyd_tuning(0, 0, 4) == -7 and lib.sop_dd4_lloyd_tuning(129, 0, 4) == -7
-    assert lib.sop_dd4_lloyd_tuning(128, -1, 4) == -7
-    assert lib.sop_dd4_lloyd_tuning(128, 0, 0) == -7 and lib.sop_dd4_lloyd_tuning(128, 0, 5) == -7
-    assert lib.sop_dd4_lloyd_tuning(1, 2, 1) == 0
-    assert lib.sop_dd4_lloyd_tuning(128, 0, 4) == 0      # the defaults again
+    assert lib.sop_dd4_lloyd_tuning(0, 0, 4, 0) == -7 and lib.sop_dd4_lloyd_tuning(129, 0, 4, 0) == -7
+    assert lib.sop_dd4_lloyd_tuning(128, -1, 4, 0) == -7 and lib.sop_dd4_lloyd_tuning(128, 0, 4, -1) == -7
+    assert lib.sop_dd4_lloyd_tuning(128, 0, 0, 0) == -7 and lib.sop_dd4_lloyd_tuning(128, 0, 5, 0) == -7
+    assert lib.sop_dd4_lloyd_tuning(1, 2, 1, 3) == 0
+    assert lib.sop_dd4_lloyd_tuning(128, 0, 4, 0) == 0      # the defaults again

@@ -223,7 +223,7 @@ def _both_formats(B, make_layer, fmts, rom, iters):
 @pytest.mark.parametrize("which", [3, 4])
 def test_config5_largest_layers_at_an_e4_and_an_e5_scale_format(B, which):
     # 28672 x 8192 and 8192 x 28672 (235 M elements, 14.7 M blocks): K / 16 = 512 and 1792 column blocks with many
-    # row iterations of the sweep, a Lloyd pool of 7.3 M blocks that needs one launch per iteration, 12- and
+    # row iterations of the sweep, a Lloyd pool of 7.3 M blocks whose 28 672 cache tiles take several rounds per CTA, 12- and
     # 16-bit scale-word streams of 14.7 M words
     got = _both_formats(B, lambda: I.config5_layer(0, 0, which, device="cuda"), ["UE4M4", "E5M6"],
                         ["NF4", "SH4", "BOF4", "Split87"], 8)

@@ -14,11 +14,13 @@ from .test_gpu_parity import B, REL, check_search, dev, gpu_lloyd  # noqa: F401 
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("spill,ctas,per_warp", [(1, 2, 1), (3, 1, 4), (5, 7, 2)])
-def test_lloyd_partial_sum_transfers_inside_the_tile_loop(B, spill, ctas, per_warp):
-    # 128 cache tiles over one, two or seven CTAs with a transfer every 1, 3 or 5 tiles: every CTA spills in the
-    # middle of its loop and (3, 5) once more for the remainder; the table, the pool count and the trace stay
-    # those of the oracle.  All blocks are in the pool (rank = N_b) and half of them.
+@pytest.mark.parametrize("spill,ctas,per_warp,iter_ctas", [(1, 2, 1, 2), (3, 1, 4, 1), (5, 7, 2, 3)])
+def test_lloyd_partial_sum_transfers_inside_the_tile_loop(B, spill, ctas, per_warp, iter_ctas):
+    # 128 cache tiles over one, two or seven CTAs of the cache kernel with a transfer every 1, 3 or 5 tiles: every CTA
+    # spills in the middle of its loop and (3, 5) once more for the remainder.  The iteration kernels run on one,
+    # two or three CTAs, so a warp walks up to sixteen tiles and the CTA folds its 32-bit partial sums every
+    # 1, 4 or 2 rounds.  The table, the pool count and the trace stay those of the oracle.  All blocks are in
+    # the pool (rank = N_b) and half of them.
     L = I.outlier_channel_layer(31, 512, 1024, 64)
     fmt = I.scale_format("E5M6")
     atoms = I.alphabet(["NF4", "SH4"])
@@ -27,7 +29,7 @@ def test_lloyd_partial_sum_transfers_inside_the_tile_loop(B, spill, ctas, per_wa
     NB = r["block_cos"].shape[1]
     assert NB == 128 * 256
     bc = torch.from_numpy(r["block_cos"]).to(dev())
-    B.dd4_lloyd_tuning(spill, ctas, per_warp)
+    B.dd4_lloyd_tuning(spill, ctas, per_warp, iter_ctas)
     try:
         for rank in (NB, NB // 2):
             want = oracle.dd_lloyd(L.W, c, fmt, int(r["k"][0]), r["block_cos"][0], rank, atoms[0].lut, 8)
@@ -39,9 +41,9 @@ def test_lloyd_partial_sum_transfers_inside_the_tile_loop(B, spill, ctas, per_wa
     finally:
         B.dd4_lloyd_tuning()
     with pytest.raises(B.SopError):
-        B.dd4_lloyd_tuning(0, 0, 4)
+        B.dd4_lloyd_tuning(0, 0, 4, 0)
     with pytest.raises(B.SopError):
-        B.dd4_lloyd_tuning(128, 0, 5)
+        B.dd4_lloyd_tuning(128, 0, 5, 0)
 
 
 def test_outputs_refuse_a_codebook_from_an_unfinished_lloyd_call(B):
