@@ -200,6 +200,24 @@ def dd_lloyd(W, c, fmt, k: int, block_cos, pool_rank: int, init_lut, iters: int,
     return out, dist, cnt.value
 
 
+def dd_grid_dp(W, c, fmt, k: int, block_metric, pool_rank: int, n_entries: int, pool_by_error: bool = False,
+               pool_threshold: float = 0.0, uniform_weights: bool = False):
+    """Grid-constrained DD-n by dynamic programming over the cell histogram of the pool.
+    Returns (lut[n_entries], cost, pool_count); the pool arguments are those of ``dd_lloyd``."""
+    w16 = _w16(W)
+    M, K = w16.shape
+    c = np.ascontiguousarray(np.asarray(c, dtype=np.float32))
+    bm = np.ascontiguousarray(np.asarray(block_metric, dtype=np.float32))
+    out = np.zeros(n_entries, dtype=np.float32)
+    cost = C.c_double()
+    cnt = C.c_longlong()
+    lib().osop_dd_grid_dp(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
+                          C.byref(_fmt(fmt)), k, _p(bm, C.c_float), int(bool(pool_by_error)), C.c_longlong(pool_rank),
+                          C.c_float(pool_threshold), int(bool(uniform_weights)), n_entries, _p(out, C.c_float),
+                          C.byref(cost), C.byref(cnt))
+    return out, cost.value, cnt.value
+
+
 def pack(W, c, fmt, a, k_a: int, b=None, k_b: int = 0, use_sign: int = 0, container_bits: int = 8,
          word_sign_bits: int = 0, select_metric: int = 0):
     """Returns dict(rc, codes [N_b, 2n] uint8, words uint8 stream, n_sel1, n_neg)."""

@@ -548,6 +548,113 @@ void osop_dd_lloyd_axes(const uint16_t* W, long long M, long long K, long long l
   *pool_count = cnt;
 }
 
+// Grid-constrained DD-n (Section "Per-Layer Pair Search", steps 1 and 3: "histogram-DP cluster selection on the
+// deployed LUT value format's grid points", the construction that has no snap-displacement cost).  The paper names
+// the construction and prints no recurrence; the reading taken here, step by step:
+//   pool, scale, u = w / s_hat and weights omega: exactly those of the Lloyd construction above (same axes);
+//   histogram: element u falls into cell t = rint(256 u) (ties to even), clamped to [-320, 320]: cells of width 2^-8
+//     over [-1.25, 1.25].  Per cell the fixed-point sums H = sum fix(omega), S = sum fix(omega u) (the product
+//     clamped to +-256 as in the Lloyd sums) and Q = sum fix((omega u) u), with fix(v) = llrint(v 2^24) on the fp32
+//     products: integer sums, so the histogram does not depend on the order of the elements;
+//   clusters: the cells with H > 0, in ascending order, are cut into runs of neighbours; the code point of a run is
+//     the grid point of the LUT value format (bf16) nearest to the run's weighted mean S / H -- the quotient in
+//     double, rounded to fp32, then to bf16 (nearest even), clamped to [-1.25, 1.25] -- and the run costs
+//     Q - 2 q S + q^2 H in double, every product and sum rounded once, in that order;
+//   dynamic programme: best[r][j] = the least total cost of cutting cells 0..j into r + 1 runs, a tie between cuts
+//     goes to the earliest cut; exactly min(n_entries, cells) runs are used; the table is the runs' code points in
+//     ascending order, padded with its last entry when there are fewer cells than entries.
+// Returns the table, the least total cost (in units of 2^-24, divided out) and the pool size.
+void osop_dd_grid_dp(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f, int k,
+                     const float* block_metric, int pool_by_error, long long pool_rank, float pool_threshold,
+                     int uniform_weights, int n_entries, float* out_lut, double* cost_out, long long* pool_count) {
+  const long long nbk = K / G, NB = M * nbk;
+  float tau = pool_threshold;
+  if (pool_rank >= 1) {
+    std::vector<float> sorted(block_metric, block_metric + NB);
+    if (pool_by_error) std::nth_element(sorted.begin(), sorted.begin() + (pool_rank - 1), sorted.end(), [](float x, float y) { return x > y; });
+    else std::nth_element(sorted.begin(), sorted.begin() + (pool_rank - 1), sorted.end());
+    tau = sorted[pool_rank - 1];
+  }
+  float cmax = 0.0f;
+  for (long long i = 0; i < K; ++i) cmax = std::max(cmax, c[i]);
+  std::vector<float> omega(K);
+  for (long long i = 0; i < K; ++i) omega[i] = uniform_weights ? 1.0f : (cmax > 0.0f ? c[i] / cmax : 0.0f);
+  const int HALF = 320, CELLS = 2 * HALF + 1;
+  std::vector<long long> H(CELLS, 0), S(CELLS, 0), Q(CELLS, 0);
+  long long cnt = 0;
+  for (long long m = 0; m < M; ++m)
+    for (long long j = 0; j < nbk; ++j) {
+      const float metric = block_metric[m * nbk + j];
+      if (!(pool_by_error ? metric >= tau : metric <= tau)) continue;
+      ++cnt;
+      float w[G], absmax = 0.0f;
+      load_block(W, ldw, m, j, w);
+      for (int i = 0; i < G; ++i) absmax = std::max(absmax, std::fabs(w[i]));
+      const QScale qs = scale_quantize(*f, absmax, k);
+      const float rcp = qs.s_hat > 0.0f ? 1.0f / qs.s_hat : 0.0f;
+      for (int i = 0; i < G; ++i) {
+        const float u = w[i] * rcp;
+        const float om = omega[j * G + i];
+        const double t = std::nearbyint((double)u * 256.0);          // default rounding mode: ties to even
+        const int cell = (int)std::min((double)HALF, std::max((double)-HALF, t)) + HALF;
+        const float ou = std::min(256.0f, std::max(-256.0f, om * u));
+        const float ouu = ou * u;
+        H[cell] += std::llrint((double)om * 16777216.0);
+        S[cell] += std::llrint((double)ou * 16777216.0);
+        Q[cell] += std::llrint((double)ouu * 16777216.0);
+      }
+    }
+  *pool_count = cnt;
+  // the non-empty cells and their prefix sums
+  std::vector<long long> pH(1, 0), pS(1, 0), pQ(1, 0);
+  for (int t = 0; t < CELLS; ++t)
+    if (H[t] > 0) { pH.push_back(pH.back() + H[t]); pS.push_back(pS.back() + S[t]); pQ.push_back(pQ.back() + Q[t]); }
+  const int B = (int)pH.size() - 1;
+  if (B == 0) {                                   // an empty pool (or all weights zero): nothing to place
+    for (int e = 0; e < n_entries; ++e) out_lut[e] = 0.0f;
+    *cost_out = 0.0;
+    return;
+  }
+  auto run = [&](int i, int j, float* q_out) {     // cells i..j (inclusive) as one run: its code point and cost
+    const double h = (double)(pH[j + 1] - pH[i]), sm = (double)(pS[j + 1] - pS[i]), qq = (double)(pQ[j + 1] - pQ[i]);
+    float q = snap_bf16((float)(sm / h));
+    q = std::min(1.25f, std::max(-1.25f, q));
+    if (q_out) *q_out = q;
+    const double qd = (double)q;
+    const double a = (2.0 * qd) * sm;
+    const double b = (qd * qd) * h;
+    return (qq - a) + b;
+  };
+  const int R = std::min(n_entries, B);
+  std::vector<std::vector<double>> best(R, std::vector<double>(B, 0.0));
+  std::vector<std::vector<int>> cut(R, std::vector<int>(B, 0));     // first cell of the last run
+  for (int j = 0; j < B; ++j) best[0][j] = run(0, j, nullptr);
+  for (int r = 1; r < R; ++r)
+    for (int j = r; j < B; ++j) {
+      double bv = 0.0;
+      int bi = -1;
+      for (int i = r; i <= j; ++i) {               // the last run is cells i..j, the r runs before it cover 0..i-1
+        const double v = best[r - 1][i - 1] + run(i, j, nullptr);
+        if (bi < 0 || v < bv) { bv = v; bi = i; }
+      }
+      best[r][j] = bv;
+      cut[r][j] = bi;
+    }
+  std::vector<float> lut;
+  int j = B - 1;
+  for (int r = R - 1; r >= 0; --r) {
+    const int i = r == 0 ? 0 : cut[r][j];
+    float q;
+    run(i, j, &q);
+    lut.push_back(q);
+    j = i - 1;
+  }
+  std::sort(lut.begin(), lut.end());
+  while ((int)lut.size() < n_entries) lut.push_back(lut.back());
+  for (int e = 0; e < n_entries; ++e) out_lut[e] = lut[e];
+  *cost_out = best[R - 1][B - 1] / 16777216.0;
+}
+
 void osop_dd_lloyd(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f, int k,
                    const float* block_cos, long long pool_rank, const float* init_lut, int n_entries, int iters,
                    float* out_lut, double* distortion, long long* pool_count) {
