@@ -235,6 +235,15 @@ int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE
  *       leaves the table as it is.
  *     SOP_LLOYD_LAUNCH_PER_ITERATION  (no counterpart in the paper) one kernel launch per iteration even
  *       where all iterations could run in one cooperative launch; the results are the same.
+ *     SOP_LLOYD_GRID_DP  the grid-constrained construction of pair-search steps 1 and 3 ("histogram-DP cluster
+ *       selection on the deployed LUT value format's grid points") instead of Lloyd iterations with a snap: the pool
+ *       elements u are binned into cells of width 2^-8 over [-1.25, 1.25] (cell = rint(256 u), clamped) with the
+ *       integer sums H = sum fix(omega), S = sum fix(omega u), Q = sum fix((omega u) u) per cell; the cells with
+ *       H > 0 are cut, in ascending order, into min(n_entries, cells) runs; a run's code point is the bf16 value
+ *       nearest to S / H (clamped to +-1.25) and its cost Q - 2 q S + q^2 H in FP64; a dynamic programme finds the
+ *       cut of least total cost (ties to the earliest cut).  iters must be 0; out_lut_dev receives the code points in
+ *       ascending order (padded with the last one when there are fewer cells than entries) and distortion_dev[0]
+ *       the least total cost.  With fmta_index = SOP_FMTA_FROM_RESULT every table atom must have the same n_entries.
  *   k_mode: a shift in [-64, 64], or SOP_K_FROM_RESULT to use search_dev->k[fmta].
  *   out_lut_dev: SOP_MAX_ENTRIES floats (first n_entries valid, ascending).
  *   distortion_dev: iters + 1 doubles, sum omega (u - q)^2 before each update and after the last.
@@ -250,6 +259,7 @@ int sop_profile_last_sweep_ms(float* ms);   /* = sop_profile_last_ms(SOP_PROFILE
 #define SOP_LLOYD_UNIFORM_WEIGHTS 2
 #define SOP_LLOYD_POOL_THRESHOLD 4
 #define SOP_LLOYD_LAUNCH_PER_ITERATION 8
+#define SOP_LLOYD_GRID_DP 16
 int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
 /* Number of kernel launches one sop_dd4_lloyd call with these sizes and flags makes on the current device
  * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch where the

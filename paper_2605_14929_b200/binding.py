@@ -23,7 +23,7 @@ ALL_ATOMS = 0xFFFFFFFF
 SEARCH_SINGLES_ONLY = 1
 SEARCH_SELECT_MSE = 2
 SEARCH_KEEP_LOADED_ENTRIES = 4
-LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD, LLOYD_LAUNCH_PER_ITERATION = 1, 2, 4, 8
+LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD, LLOYD_LAUNCH_PER_ITERATION, LLOYD_GRID_DP = 1, 2, 4, 8, 16
 PACK_SELECT_MSE = 1
 MAX_ENTRIES = 32
 
@@ -229,9 +229,10 @@ def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_
                   workspace: torch.Tensor, k_mode: int = K_FROM_RESULT, search_result: Optional[torch.Tensor] = None,
                   fmta_index: int = FMTA_FROM_RESULT, stream=None, g: int = 16, pool_by_error: bool = False,
                   uniform_weights: bool = False, pool_threshold: Optional[float] = None,
-                  launch_per_iteration: bool = False) -> None:
+                  launch_per_iteration: bool = False, grid_dp: bool = False) -> None:
     """``block_cos`` is the per-block metric that ranks the blocks: cosines, or errors with ``pool_by_error``.
-    A ``pool_threshold`` replaces the rank."""
+    A ``pool_threshold`` replaces the rank.  ``grid_dp`` (with ``iters`` = 0) takes the grid-constrained construction
+    by dynamic programming instead of Lloyd iterations; ``distortion[0]`` is then its least total cost."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
     M, K = W.shape
     _check(lib().sop_dd4_lloyd(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), k_mode,
@@ -239,7 +240,7 @@ def sop_dd4_lloyd(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, block_
                                C.c_float(0.0 if pool_threshold is None else pool_threshold),
                                (LLOYD_POOL_BY_ERROR if pool_by_error else 0) | (LLOYD_UNIFORM_WEIGHTS if uniform_weights else 0)
                                | (LLOYD_POOL_THRESHOLD if pool_threshold is not None else 0)
-                               | (LLOYD_LAUNCH_PER_ITERATION if launch_per_iteration else 0),
+                               | (LLOYD_LAUNCH_PER_ITERATION if launch_per_iteration else 0) | (LLOYD_GRID_DP if grid_dp else 0),
                                make_atoms(atoms), len(atoms),
                                fmta_index, iters, _ptr(out_lut), _ptr(distortion), _ptr(pool_count), _ptr(workspace),
                                C.c_size_t(workspace.numel()), _stream(stream)), "sop_dd4_lloyd")

@@ -31,6 +31,7 @@
 //                         bounded, for the flag of the CTA that finished last.
 //   lloyd_split_kernel    one iteration per launch: used where the grid cannot be resident at once.
 #include <math.h>
+#include <stddef.h>
 #include <string.h>
 
 #include "sop_device.cuh"
@@ -83,6 +84,9 @@ struct LloydWs {
   unsigned long long cellN[SORT_ROWS];     // sum fix(omega)
   long long cellS[SORT_ROWS];              // sum fix(omega u)
   double cellA[3][SORT_ROWS];              // sum omega, sum omega u, sum omega u^2
+  long long cellQ[SORT_ROWS];              // sum fix((omega u) u): the exact second moment the grid-constrained construction needs
+  // not cleared per call: where the last run starts, per (number of runs, last cell), for the backtrack of the dynamic programme
+  short dp_cut[SOP_MAX_ENTRIES][SORT_ROWS];
 };
 
 struct LloydArgs {
@@ -275,7 +279,7 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
     distortion[iters] = -1.0;
   }
   for (int r = threadIdx.x; r < SORT_ROWS; r += SETUP_TB) {
-    ws->cellN[r] = 0; ws->cellS[r] = 0; ws->cellA[0][r] = 0.0; ws->cellA[1][r] = 0.0; ws->cellA[2][r] = 0.0;
+    ws->cellN[r] = 0; ws->cellS[r] = 0; ws->cellQ[r] = 0; ws->cellA[0][r] = 0.0; ws->cellA[1][r] = 0.0; ws->cellA[2][r] = 0.0;
   }
   __syncthreads();
   lloyd_publish_desc(ws, s_lut, s_ne);
@@ -337,7 +341,7 @@ __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exa
   return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
 }
 
-constexpr int CELL_LIMBS = 14;
+constexpr int CELL_LIMBS = 17;
 constexpr int CELL_SPILL_TILES_MAX = 128;     // a low limb takes at most 258 * (2^16 - 1) per tile: 128 tiles stay below 2^32
 constexpr int TILES_PER_WARP_MAX = 4;         // tiles a warp of an iteration CTA walks between two folds of its limb sums (see flush_limbs)
 
@@ -354,16 +358,17 @@ __device__ __forceinline__ void add_limbs3(unsigned (*cL)[SORT_ROWS], int first,
   atomicAdd(&cL[first + 2][cell], (unsigned)(int)(v >> 32));
 }
 
-// One run of elements of one cell (at most 16): fix(omega) sums below 2^28, fix(omega u) sums below 2^37
-// in magnitude, moments below 2^6 in magnitude (so below 2^46 in units of 2^-40).
+// One run of elements of one cell (at most 16): fix(omega) sums below 2^28, fix(omega u) and fix(omega u u) sums below
+// 2^37 in magnitude, moments below 2^6 in magnitude (so below 2^46 in units of 2^-40).
 __device__ __forceinline__ void flush_cell(unsigned (*cL)[SORT_ROWS], int cell, unsigned long long n, unsigned long long sv,
-                                           double a0, double a1, double a2) {
+                                           unsigned long long sq, double a0, double a1, double a2) {
   atomicAdd(&cL[0][cell], (unsigned)(n & 0xFFFFull));
   atomicAdd(&cL[1][cell], (unsigned)(n >> 16));
   add_limbs3(cL, 2, cell, (long long)sv);
   add_limbs3(cL, 5, cell, __double2ll_rn(a0 * MOMENT_UNIT));
   add_limbs3(cL, 8, cell, __double2ll_rn(a1 * MOMENT_UNIT));
   add_limbs3(cL, 11, cell, __double2ll_rn(a2 * MOMENT_UNIT));
+  add_limbs3(cL, 14, cell, (long long)sq);
 }
 
 __device__ __forceinline__ long long join_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell) {
@@ -376,6 +381,8 @@ __device__ void spill_cells(unsigned (*cL)[SORT_ROWS], LloydWs* ws) {
     const unsigned long long n = (unsigned long long)cL[0][r] + ((unsigned long long)cL[1][r] << 16);
     const long long sv = join_limbs3(cL, 2, r);
     const long long m0 = join_limbs3(cL, 5, r), m1 = join_limbs3(cL, 8, r), m2 = join_limbs3(cL, 11, r);
+    const long long sq = join_limbs3(cL, 14, r);
+    if (sq) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellQ[r]), (unsigned long long)sq);
     if (n) atomicAdd(&ws->cellN[r], n);
     if (sv) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellS[r]), (unsigned long long)sv);
     if (m0) atomicAdd(&ws->cellA[0][r], (double)m0 * (1.0 / MOMENT_UNIT));
@@ -462,7 +469,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
     // current cell's sums in registers and adds them to the CTA's limbs when the cell changes
     {
       int cur = -1;
-      unsigned long long n = 0, sv = 0;
+      unsigned long long n = 0, sv = 0, sq = 0;
       double a0 = 0.0, a1 = 0.0, a2 = 0.0;
 #pragma unroll 4
       for (int i2 = 0; i2 < 16; ++i2) {
@@ -470,16 +477,17 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
         const float u = __uint_as_float(v.x), om = __uint_as_float(v.y);
         const int c = sort_cell(u);
         if (c != cur) {
-          if (cur >= 0) flush_cell(cL, cur, n, sv, a0, a1, a2);
-          cur = c; n = 0; sv = 0; a0 = a1 = a2 = 0.0;
+          if (cur >= 0) flush_cell(cL, cur, n, sv, sq, a0, a1, a2);
+          cur = c; n = 0; sv = 0; sq = 0; a0 = a1 = a2 = 0.0;
         }
         const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
         n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
         sv += (unsigned long long)fix24(ou);
+        sq += (unsigned long long)fix24(__fmul_rn(ou, u));
         const double dou = (double)om * (double)u;
         a0 += (double)om; a1 += dou; a2 += dou * (double)u;
       }
-      flush_cell(cL, cur, n, sv, a0, a1, a2);
+      flush_cell(cL, cur, n, sv, sq, a0, a1, a2);
     }
     __syncthreads();
     // a cell takes at most 258 flushes per tile and a low limb 2^16 - 1 per flush: the limbs go to the
@@ -770,6 +778,97 @@ __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, Lloy
   if (threadIdx.x == 0 && *(volatile unsigned*)&ws->error != 0u) distortion[iters] = -1.0;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Grid-constrained DD-n (pair-search steps 1 and 3: cluster selection by dynamic programming on the grid points of the
+// LUT value format).  The histogram is the per-cell sums that pool_cache_kernel has formed -- H = sum fix(omega),
+// S = sum fix(omega u), Q = sum fix((omega u) u), integers, so independent of any order.  The cells with H > 0, in
+// ascending order, are cut into min(n_entries, cells) runs; a run's code point is the bf16 value nearest to S / H
+// (clamped to +-1.25) and it costs Q - 2 q S + q^2 H; the least total cost wins, a tie between cuts goes to the earliest.
+// One CTA: thread j owns "cells 0..j" and scans the start of the last run; the FP64 operations are written one by one
+// (no contraction), so every comparison sees the same numbers as a sequential evaluation.
+// ---------------------------------------------------------------------------------------------
+constexpr int DP_TB = 1024;
+
+__device__ __forceinline__ double dp_run_cost(const long long* pH, const long long* pS, const long long* pQ, int i, int j, float* q_out) {
+  const double h = __ll2double_rn(pH[j + 1] - pH[i]), sm = __ll2double_rn(pS[j + 1] - pS[i]), qq = __ll2double_rn(pQ[j + 1] - pQ[i]);
+  const float mean = __double2float_rn(__ddiv_rn(sm, h));
+  uint32_t b = __float_as_uint(mean);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  b &= 0xFFFF0000u;                                   // nearest bf16, ties to even
+  float q = __uint_as_float(b);
+  q = fminf(1.25f, fmaxf(-1.25f, q));
+  if (q_out) *q_out = q;
+  const double qd = (double)q;
+  const double a = __dmul_rn(__dmul_rn(2.0, qd), sm);
+  const double c = __dmul_rn(__dmul_rn(qd, qd), h);
+  return __dadd_rn(__dsub_rn(qq, a), c);
+}
+
+__global__ void __launch_bounds__(DP_TB) grid_dp_kernel(const LloydWs* __restrict__ ws, int n_entries, float* __restrict__ out_lut,
+                                                        double* __restrict__ cost_out, short* __restrict__ cut /* [n_entries][SORT_ROWS] */) {
+  __shared__ long long pH[SORT_ROWS + 1], pS[SORT_ROWS + 1], pQ[SORT_ROWS + 1];
+  __shared__ double best[2][SORT_ROWS];
+  __shared__ int s_B;
+  __shared__ float s_lut[SOP_MAX_ENTRIES];
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    // the non-empty cells and their prefix sums (641 cells: a short serial pass)
+    int B = 0;
+    pH[0] = pS[0] = pQ[0] = 0;
+    for (int t = 0; t < SORT_ROWS; ++t) {
+      const long long h = (long long)ws->cellN[t];
+      if (h > 0) { pH[B + 1] = pH[B] + h; pS[B + 1] = pS[B] + ws->cellS[t]; pQ[B + 1] = pQ[B] + ws->cellQ[t]; ++B; }
+    }
+    s_B = B;
+  }
+  __syncthreads();
+  const int B = s_B;
+  if (B == 0) {
+    if (tid < SOP_MAX_ENTRIES) out_lut[tid] = 0.0f;
+    if (tid == 0) cost_out[0] = 0.0;
+    return;
+  }
+  const int R = min(n_entries, B);
+  for (int j = tid; j < B; j += DP_TB) best[0][j] = dp_run_cost(pH, pS, pQ, 0, j, nullptr);
+  __syncthreads();
+  for (int r = 1; r < R; ++r) {
+    const double* prev = best[(r - 1) & 1];
+    double* cur = best[r & 1];
+    for (int j = tid; j < B; j += DP_TB) {
+      if (j < r) continue;
+      double bv = 0.0;
+      int bi = -1;
+      for (int i = r; i <= j; ++i) {               // the last run is cells i..j
+        const double v = __dadd_rn(prev[i - 1], dp_run_cost(pH, pS, pQ, i, j, nullptr));
+        if (bi < 0 || v < bv) { bv = v; bi = i; }
+      }
+      cur[j] = bv;
+      cut[(size_t)r * SORT_ROWS + j] = (short)bi;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    int j = B - 1, n = 0;
+    for (int r = R - 1; r >= 0; --r) {
+      const int i = r == 0 ? 0 : (int)cut[(size_t)r * SORT_ROWS + j];
+      float q;
+      dp_run_cost(pH, pS, pQ, i, j, &q);
+      s_lut[n++] = q;
+      j = i - 1;
+    }
+    // ascending (insertion sort of at most 32 values), padded with the last entry
+    for (int a = 1; a < n; ++a) {
+      const float v = s_lut[a];
+      int b = a - 1;
+      while (b >= 0 && s_lut[b] > v) { s_lut[b + 1] = s_lut[b]; --b; }
+      s_lut[b + 1] = v;
+    }
+    for (int e = n; e < SOP_MAX_ENTRIES; ++e) s_lut[e] = s_lut[n - 1];
+    for (int e = 0; e < SOP_MAX_ENTRIES; ++e) out_lut[e] = e < n_entries ? s_lut[e] : 0.0f;
+    cost_out[0] = __ddiv_rn(best[(R - 1) & 1][B - 1], 16777216.0);
+  }
+}
+
 int num_sms();
 
 // Grid of the iteration kernels and whether all iterations run in one cooperative launch: they do wherever the device
@@ -813,7 +912,7 @@ int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* 
   long long grid = 1;
   const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), M * (K / SOP_G), iters, flags, &grid);
   // radix select (three passes, unless the pool is cut by a threshold), set-up, pool list, pool cache, iterations
-  *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + (persistent ? 1 : iters + 1);
+  *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + ((flags & SOP_LLOYD_GRID_DP) ? 1 : (persistent ? 1 : iters + 1));
   return SOP_OK;
 }
 
@@ -846,7 +945,9 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   int rc = validate_layer(W_dev, M, K, ldw, c_dev, g);
   if (rc) return rc;
   if (!block_metric_dev || !out_lut_dev || !distortion_dev || !pool_count_dev) return SOP_ERR_NULL;
-  if (flags & ~(SOP_LLOYD_POOL_BY_ERROR | SOP_LLOYD_UNIFORM_WEIGHTS | SOP_LLOYD_POOL_THRESHOLD | SOP_LLOYD_LAUNCH_PER_ITERATION)) return SOP_ERR_RANGE;
+  if (flags & ~(SOP_LLOYD_POOL_BY_ERROR | SOP_LLOYD_UNIFORM_WEIGHTS | SOP_LLOYD_POOL_THRESHOLD | SOP_LLOYD_LAUNCH_PER_ITERATION | SOP_LLOYD_GRID_DP)) return SOP_ERR_RANGE;
+  const bool grid_dp = (flags & SOP_LLOYD_GRID_DP) != 0;
+  if (grid_dp && iters != 0) return SOP_ERR_RANGE;        // the dynamic programme replaces the iterations
   const bool by_threshold = (flags & SOP_LLOYD_POOL_THRESHOLD) != 0;
   if (by_threshold && !(pool_threshold == pool_threshold)) return SOP_ERR_RANGE;   // NaN orders nothing
   FmtDev F;
@@ -876,7 +977,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   a.tile_start = (unsigned short*)(wsb + lloyd_off_tiles(M, K));
   LloydWs* ws = (LloydWs*)workspace_dev;
   cudaStream_t st = (cudaStream_t)stream;
-  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(LloydWs), st));
+  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, offsetof(LloydWs, dp_cut), st));
   const int sms = num_sms();
   long long sg = (NB + LTB * 8 - 1) / (LTB * 8);
   if (sg > sms * 4) sg = sms * 4;
@@ -905,6 +1006,21 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     }
     pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
     SOP_CUDA_TRY(cudaGetLastError());
+  }
+  if (grid_dp) {
+    // entries of the new table: FMTa's; when FMTa is chosen on the device every table atom must agree on the number
+    int ne = fmta_index >= 0 ? atoms[fmta_index].n_entries : 0;
+    for (int i = 0; i < n_atoms && fmta_index < 0; ++i) {
+      if (atoms[i].kind != SOP_KIND_LUT) continue;
+      if (ne == 0) ne = atoms[i].n_entries;
+      else if (atoms[i].n_entries != ne) return SOP_ERR_ALPHABET;
+    }
+    if (ne < 2) return SOP_ERR_ALPHABET;
+    if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
+    grid_dp_kernel<<<1, DP_TB, 0, st>>>(ws, ne, out_lut_dev, distortion_dev, &ws->dp_cut[0][0]);
+    SOP_CUDA_TRY(cudaGetLastError());
+    if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;
+    return SOP_OK;
   }
   long long grid = 1;
   const bool persistent = lloyd_iteration_plan(NB, by_threshold ? NB : pool_rank, iters, flags, &grid);

@@ -108,7 +108,8 @@ def test_other_entry_points_reject_bad_arguments(lib):
         return lib.sop_dd4_lloyd(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, k, res, FAKE, ll(rank), C.c_float(thr), flags, arr,
                                  len(atoms), fmta, iters, FAKE, FAKE, FAKE, FAKE, C.c_size_t(1 << 20), None)
     assert lloyd(rank=0) == -7 and lloyd(rank=17) == -7 and lloyd(iters=65) == -7 and lloyd(k=99) == -7
-    assert lloyd(flags=16) == -7                                          # unknown flag
+    assert lloyd(flags=32) == -7                                          # unknown flag
+    assert lloyd(flags=B.LLOYD_GRID_DP, iters=8) == -7                    # the dynamic programme replaces the iterations
     assert lloyd(flags=B.LLOYD_POOL_THRESHOLD, thr=float("nan")) == -7    # a NaN threshold orders nothing
     assert lloyd(rank=0, flags=B.LLOYD_POOL_THRESHOLD, iters=65) == -7    # the rank is ignored, the rest is still checked
     assert lloyd(fmta=9) == -7

@@ -100,3 +100,33 @@ def test_eight_fine_tables_beyond_the_shared_memory_are_swept_exactly(B):
     L = I.tiny_layer(9, 96, 512)
     check_search(B, L, "UE4M4", atoms)
     check_search(B, L, "E5M6", atoms + [atoms[0].negation(), atoms[3].negation()])
+
+
+@pytest.mark.parametrize("fmt_name,names,layer", [("UE4M4", ["NF4", "SH4"], "config1"), ("E5M6", ["NF5", "SH5"], "config1"),
+                                                  ("E5M6", ["NF4", "BOF4"], "outlier")])
+def test_grid_constrained_dd_by_dynamic_programming(B, fmt_name, names, layer):
+    # pair-search steps 1 and 3: cluster selection on the LUT value format's grid points; the table bit for bit, the
+    # least total cost and the pool count, for a plain and a negated primary codebook and three pool sizes
+    L = I.config1() if layer == "config1" else I.outlier_channel_layer(8, 320, 1024, 64)
+    fmt = I.scale_format(fmt_name)
+    atoms = I.alphabet(names)
+    c = oracle.channel_norms(L.X.numpy())
+    r = oracle.pair_search(L.W, c, fmt, atoms, want_blocks=True)
+    NB = r["block_cos"].shape[1]
+    bc = torch.from_numpy(r["block_cos"]).to(dev())
+    ne = len(atoms[0].lut)
+    for fmta in (0, 1):
+        for rank in (NB // 2, 7, NB):
+            want = oracle.dd_grid_dp(L.W, c, fmt, int(r["k"][fmta]), r["block_cos"][fmta], rank, ne)
+            got = gpu_lloyd(B, L.W, c, fmt, atoms, bc, rank, 0, int(r["k"][fmta]), fmta, grid_dp=True)
+            assert np.array_equal(got[0][:ne].view(np.uint32), want[0].view(np.uint32))
+            assert got[2] == want[2]
+            assert got[1][0] == pytest.approx(want[1], rel=REL, abs=1e-12)
+    # the dynamic programme replaces the iterations: asking for both is refused
+    with pytest.raises(B.SopError):
+        gpu_lloyd(B, L.W, c, fmt, atoms, bc, NB // 2, 3, 0, 0, grid_dp=True)
+    # axes (i), (iii), (iv) reach the construction like they reach the Lloyd one
+    bs = torch.from_numpy(r["block_sse"]).to(dev())
+    want = oracle.dd_grid_dp(L.W, c, fmt, int(r["k"][0]), r["block_sse"][0], NB // 3, ne, pool_by_error=True, uniform_weights=True)
+    got = gpu_lloyd(B, L.W, c, fmt, atoms, bs, NB // 3, 0, int(r["k"][0]), 0, grid_dp=True, pool_by_error=True, uniform_weights=True)
+    assert np.array_equal(got[0][:ne].view(np.uint32), want[0].view(np.uint32)) and got[2] == want[2]
