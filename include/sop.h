@@ -264,7 +264,8 @@ int sop_dd4_lloyd_workspace(long long M, long long K, size_t* bytes);
 /* Number of kernel launches one sop_dd4_lloyd call with these sizes and flags makes on the current device
  * (measurement aid, no counterpart in the paper).  All iterations run in one cooperative launch where the
  * device supports such launches (the grid is cut to what is resident at once); otherwise, or with
- * SOP_LLOYD_LAUNCH_PER_ITERATION, there is one launch per iteration. */
+ * SOP_LLOYD_LAUNCH_PER_ITERATION, there is one launch per iteration.  With SOP_LLOYD_GRID_DP pass the number of
+ * table entries as `iters`: the dynamic programme takes one launch per row plus two. */
 int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches);
 /* Launch-shape parameters of sop_dd4_lloyd for this process (test aid, no counterpart in the paper; results do
  * not depend on them).  cell_spill_tiles in [1, 128]: cache tiles a CTA sorts between two transfers of its

@@ -85,8 +85,9 @@ struct LloydWs {
   long long cellS[SORT_ROWS];              // sum fix(omega u)
   double cellA[3][SORT_ROWS];              // sum omega, sum omega u, sum omega u^2
   long long cellQ[SORT_ROWS];              // sum fix((omega u) u): the exact second moment the grid-constrained construction needs
-  // not cleared per call: where the last run starts, per (number of runs, last cell), for the backtrack of the dynamic programme
+  // not cleared per call: scratch of the dynamic programme, and where the last run starts per (number of runs, last cell)
   short dp_cut[SOP_MAX_ENTRIES][SORT_ROWS];
+  long long dp_scratch[4 * (SORT_ROWS + 1) + 2 * SORT_ROWS];
 };
 
 struct LloydArgs {
@@ -341,7 +342,8 @@ __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exa
   return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
 }
 
-constexpr int CELL_LIMBS = 17;
+constexpr int CELL_LIMBS = 14;            // Lloyd: counts (2), sum omega u (3), three moments (3 each)
+constexpr int CELL_LIMBS_DP = 8;          // dynamic programme: counts (2), sum omega u (3), sum omega u u (3)
 constexpr int CELL_SPILL_TILES_MAX = 128;     // a low limb takes at most 258 * (2^16 - 1) per tile: 128 tiles stay below 2^32
 constexpr int TILES_PER_WARP_MAX = 4;         // tiles a warp of an iteration CTA walks between two folds of its limb sums (see flush_limbs)
 
@@ -360,15 +362,21 @@ __device__ __forceinline__ void add_limbs3(unsigned (*cL)[SORT_ROWS], int first,
 
 // One run of elements of one cell (at most 16): fix(omega) sums below 2^28, fix(omega u) and fix(omega u u) sums below
 // 2^37 in magnitude, moments below 2^6 in magnitude (so below 2^46 in units of 2^-40).
+// DP: the sums that the grid-constrained construction reads (fix(omega), fix(omega u), fix(omega u u)); otherwise those of
+// the Lloyd iterations (fix(omega), fix(omega u) and the three moments).
+template <bool DP>
 __device__ __forceinline__ void flush_cell(unsigned (*cL)[SORT_ROWS], int cell, unsigned long long n, unsigned long long sv,
                                            unsigned long long sq, double a0, double a1, double a2) {
   atomicAdd(&cL[0][cell], (unsigned)(n & 0xFFFFull));
   atomicAdd(&cL[1][cell], (unsigned)(n >> 16));
   add_limbs3(cL, 2, cell, (long long)sv);
-  add_limbs3(cL, 5, cell, __double2ll_rn(a0 * MOMENT_UNIT));
-  add_limbs3(cL, 8, cell, __double2ll_rn(a1 * MOMENT_UNIT));
-  add_limbs3(cL, 11, cell, __double2ll_rn(a2 * MOMENT_UNIT));
-  add_limbs3(cL, 14, cell, (long long)sq);
+  if (DP) {
+    add_limbs3(cL, 5, cell, (long long)sq);
+  } else {
+    add_limbs3(cL, 5, cell, __double2ll_rn(a0 * MOMENT_UNIT));
+    add_limbs3(cL, 8, cell, __double2ll_rn(a1 * MOMENT_UNIT));
+    add_limbs3(cL, 11, cell, __double2ll_rn(a2 * MOMENT_UNIT));
+  }
 }
 
 __device__ __forceinline__ long long join_limbs3(unsigned (*cL)[SORT_ROWS], int first, int cell) {
@@ -376,34 +384,40 @@ __device__ __forceinline__ long long join_limbs3(unsigned (*cL)[SORT_ROWS], int 
 }
 
 // Whole CTA, after a barrier: the CTA's limbs are added to the per-cell sums of the pool and cleared.
+template <bool DP>
 __device__ void spill_cells(unsigned (*cL)[SORT_ROWS], LloydWs* ws) {
   for (int r = threadIdx.x; r < SORT_ROWS; r += blockDim.x) {
     const unsigned long long n = (unsigned long long)cL[0][r] + ((unsigned long long)cL[1][r] << 16);
     const long long sv = join_limbs3(cL, 2, r);
-    const long long m0 = join_limbs3(cL, 5, r), m1 = join_limbs3(cL, 8, r), m2 = join_limbs3(cL, 11, r);
-    const long long sq = join_limbs3(cL, 14, r);
-    if (sq) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellQ[r]), (unsigned long long)sq);
     if (n) atomicAdd(&ws->cellN[r], n);
     if (sv) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellS[r]), (unsigned long long)sv);
-    if (m0) atomicAdd(&ws->cellA[0][r], (double)m0 * (1.0 / MOMENT_UNIT));
-    if (m1) atomicAdd(&ws->cellA[1][r], (double)m1 * (1.0 / MOMENT_UNIT));
-    if (m2) atomicAdd(&ws->cellA[2][r], (double)m2 * (1.0 / MOMENT_UNIT));
+    if (DP) {
+      const long long sq = join_limbs3(cL, 5, r);
+      if (sq) atomicAdd(reinterpret_cast<unsigned long long*>(&ws->cellQ[r]), (unsigned long long)sq);
+    } else {
+      const long long m0 = join_limbs3(cL, 5, r), m1 = join_limbs3(cL, 8, r), m2 = join_limbs3(cL, 11, r);
+      if (m0) atomicAdd(&ws->cellA[0][r], (double)m0 * (1.0 / MOMENT_UNIT));
+      if (m1) atomicAdd(&ws->cellA[1][r], (double)m1 * (1.0 / MOMENT_UNIT));
+      if (m2) atomicAdd(&ws->cellA[2][r], (double)m2 * (1.0 / MOMENT_UNIT));
+    }
 #pragma unroll
-    for (int l = 0; l < CELL_LIMBS; ++l) cL[l][r] = 0;
+    for (int l = 0; l < (DP ? CELL_LIMBS_DP : CELL_LIMBS); ++l) cL[l][r] = 0;
   }
 }
 
+template <bool DP>
 __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, LloydWs* __restrict__ ws, long long* __restrict__ pool_count_out,
                                                          unsigned spill_tiles) {
   __shared__ unsigned hist[SORT_ROWS + 3];
   __shared__ unsigned warp_tot[LTB / 32];
   extern __shared__ __align__(16) uint2 stage[];                  // TILE_ELEMS pairs (dynamic: the kernel needs 60 KB in all)
   // this CTA's share of the per-cell sums, as 32-bit limbs that native shared-memory atomics add:
-  // [0..1] sum fix(omega), [2..4] sum fix(omega u), [5..7], [8..10], [11..13] the three moments in units
-  // of 2^-40.  Low limbs hold 16 bits, the top limb the signed rest.
-  __shared__ unsigned cL[CELL_LIMBS][SORT_ROWS];
+  // [0..1] sum fix(omega), [2..4] sum fix(omega u), then either [5..7], [8..10], [11..13] the three moments in units
+  // of 2^-40 or (DP) [5..7] sum fix(omega u u).  Low limbs hold 16 bits, the top limb the signed rest.
+  constexpr int NL = DP ? CELL_LIMBS_DP : CELL_LIMBS;
+  __shared__ unsigned cL[NL][SORT_ROWS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = tid; i < CELL_LIMBS * SORT_ROWS; i += LTB) (&cL[0][0])[i] = 0;
+  for (int i = tid; i < NL * SORT_ROWS; i += LTB) (&cL[0][0])[i] = 0;
   unsigned tiles_since_spill = 0;
   const unsigned count = ws->list_count;
   const unsigned n_tiles = (count + LTB - 1) / LTB;
@@ -459,12 +473,14 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
       stage[(p & 15u) * LTB + (p >> 4)] = make_uint2(__float_as_uint(u[e]), __float_as_uint(om[e]));
     }
     __syncthreads();
-    uint4* dst = reinterpret_cast<uint4*>(a.cache + (size_t)tile * TILE_ELEMS);
-    const uint4* src = reinterpret_cast<const uint4*>(stage);
+    if (!DP) {      // the dynamic programme reads the per-cell sums only: no iteration walks the elements again
+      uint4* dst = reinterpret_cast<uint4*>(a.cache + (size_t)tile * TILE_ELEMS);
+      const uint4* src = reinterpret_cast<const uint4*>(stage);
 #pragma unroll
-    for (int q = 0; q < TILE_ELEMS / 2 / LTB; ++q) dst[q * LTB + tid] = src[q * LTB + tid];
-    unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
-    for (int r = tid; r <= SORT_ROWS; r += LTB) ts[r] = (unsigned short)hist[r];      // hist[SORT_ROWS] = 4096: the end of the last cell
+      for (int q = 0; q < TILE_ELEMS / 2 / LTB; ++q) dst[q * LTB + tid] = src[q * LTB + tid];
+      unsigned short* ts = a.tile_start + (size_t)tile * (SORT_ROWS + 1);
+      for (int r = tid; r <= SORT_ROWS; r += LTB) ts[r] = (unsigned short)hist[r];      // hist[SORT_ROWS] = 4096: the end of the last cell
+    }
     // per-cell sums: thread t owns the sorted positions 16 t .. 16 t + 15 (ascending cells), keeps the
     // current cell's sums in registers and adds them to the CTA's limbs when the cell changes
     {
@@ -477,28 +493,31 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
         const float u = __uint_as_float(v.x), om = __uint_as_float(v.y);
         const int c = sort_cell(u);
         if (c != cur) {
-          if (cur >= 0) flush_cell(cL, cur, n, sv, sq, a0, a1, a2);
+          if (cur >= 0) flush_cell<DP>(cL, cur, n, sv, sq, a0, a1, a2);
           cur = c; n = 0; sv = 0; sq = 0; a0 = a1 = a2 = 0.0;
         }
         const float ou = fminf(fmaxf(__fmul_rn(om, u), -256.0f), 256.0f);
         n += (unsigned long long)__float2uint_rn(__fmul_rn(om, 16777216.0f));   // omega in [0, 1]
         sv += (unsigned long long)fix24(ou);
-        sq += (unsigned long long)fix24(__fmul_rn(ou, u));
-        const double dou = (double)om * (double)u;
-        a0 += (double)om; a1 += dou; a2 += dou * (double)u;
+        if (DP) {
+          sq += (unsigned long long)fix24(__fmul_rn(ou, u));
+        } else {
+          const double dou = (double)om * (double)u;
+          a0 += (double)om; a1 += dou; a2 += dou * (double)u;
+        }
       }
-      flush_cell(cL, cur, n, sv, sq, a0, a1, a2);
+      flush_cell<DP>(cL, cur, n, sv, sq, a0, a1, a2);
     }
     __syncthreads();
     // a cell takes at most 258 flushes per tile and a low limb 2^16 - 1 per flush: the limbs go to the
     // global sums before they can wrap
     if (++tiles_since_spill == spill_tiles) {
-      spill_cells(cL, ws);
+      spill_cells<DP>(cL, ws);
       tiles_since_spill = 0;
       __syncthreads();
     }
   }
-  if (tiles_since_spill) spill_cells(cL, ws);
+  if (tiles_since_spill) spill_cells<DP>(cL, ws);
 }
 
 // One warp per tile.  The elements of the tile that lie in cells holding a threshold (sorted positions
@@ -784,10 +803,10 @@ __global__ void __launch_bounds__(LTB) lloyd_persistent_kernel(LloydArgs a, Lloy
 // S = sum fix(omega u), Q = sum fix((omega u) u), integers, so independent of any order.  The cells with H > 0, in
 // ascending order, are cut into min(n_entries, cells) runs; a run's code point is the bf16 value nearest to S / H
 // (clamped to +-1.25) and it costs Q - 2 q S + q^2 H; the least total cost wins, a tie between cuts goes to the earliest.
-// One CTA: thread j owns "cells 0..j" and scans the start of the last run; the FP64 operations are written one by one
-// (no contraction), so every comparison sees the same numbers as a sequential evaluation.
+// One launch per row of the programme (number of runs), one warp per last cell; the FP64 operations are written one by
+// one (no contraction), so every comparison sees the same numbers as a sequential evaluation.
 // ---------------------------------------------------------------------------------------------
-constexpr int DP_TB = 1024;
+constexpr int DP_TB = 256;
 
 __device__ __forceinline__ double dp_run_cost(const long long* pH, const long long* pS, const long long* pQ, int i, int j, float* q_out) {
   const double h = __ll2double_rn(pH[j + 1] - pH[i]), sm = __ll2double_rn(pS[j + 1] - pS[i]), qq = __ll2double_rn(pQ[j + 1] - pQ[i]);
@@ -804,69 +823,85 @@ __device__ __forceinline__ double dp_run_cost(const long long* pH, const long lo
   return __dadd_rn(__dsub_rn(qq, a), c);
 }
 
-__global__ void __launch_bounds__(DP_TB) grid_dp_kernel(const LloydWs* __restrict__ ws, int n_entries, float* __restrict__ out_lut,
-                                                        double* __restrict__ cost_out, short* __restrict__ cut /* [n_entries][SORT_ROWS] */) {
-  __shared__ long long pH[SORT_ROWS + 1], pS[SORT_ROWS + 1], pQ[SORT_ROWS + 1];
-  __shared__ double best[2][SORT_ROWS];
+// Scratch of the dynamic programme in the workspace: prefix sums of the non-empty cells, two rows of least costs.
+struct DpScratch {
+  int B;
+  int pad;
+  long long pH[SORT_ROWS + 1], pS[SORT_ROWS + 1], pQ[SORT_ROWS + 1];
+  double best[2][SORT_ROWS];
+};
+
+// One CTA: the non-empty cells, their prefix sums, and row 0 (cells 0..j as one run).
+__global__ void __launch_bounds__(DP_TB) grid_dp_first_kernel(const LloydWs* __restrict__ ws, DpScratch* __restrict__ dp) {
   __shared__ int s_B;
-  __shared__ float s_lut[SOP_MAX_ENTRIES];
-  const int tid = threadIdx.x;
-  if (tid == 0) {
-    // the non-empty cells and their prefix sums (641 cells: a short serial pass)
+  if (threadIdx.x == 0) {
     int B = 0;
-    pH[0] = pS[0] = pQ[0] = 0;
+    dp->pH[0] = dp->pS[0] = dp->pQ[0] = 0;
     for (int t = 0; t < SORT_ROWS; ++t) {
       const long long h = (long long)ws->cellN[t];
-      if (h > 0) { pH[B + 1] = pH[B] + h; pS[B + 1] = pS[B] + ws->cellS[t]; pQ[B + 1] = pQ[B] + ws->cellQ[t]; ++B; }
+      if (h > 0) { dp->pH[B + 1] = dp->pH[B] + h; dp->pS[B + 1] = dp->pS[B] + ws->cellS[t]; dp->pQ[B + 1] = dp->pQ[B] + ws->cellQ[t]; ++B; }
     }
+    dp->B = B;
     s_B = B;
   }
   __syncthreads();
-  const int B = s_B;
+  for (int j = threadIdx.x; j < s_B; j += DP_TB) dp->best[0][j] = dp_run_cost(dp->pH, dp->pS, dp->pQ, 0, j, nullptr);
+}
+
+// Row r of the programme: one warp per last cell j, the lanes share the starts i of the last run; the least value wins,
+// a tie goes to the smallest i (what a sequential scan from the first start on keeps).
+__global__ void __launch_bounds__(DP_TB) grid_dp_row_kernel(DpScratch* __restrict__ dp, int r, short* __restrict__ cut) {
+  const int B = dp->B;
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * (DP_TB / 32) + (threadIdx.x >> 5);
+  if (j >= B || j < r) return;
+  const double* prev = dp->best[(r - 1) & 1];
+  double bv = 0.0;
+  int bi = -1;
+  for (int i = r + lane; i <= j; i += 32) {
+    const double v = __dadd_rn(prev[i - 1], dp_run_cost(dp->pH, dp->pS, dp->pQ, i, j, nullptr));
+    if (bi < 0 || v < bv) { bv = v; bi = i; }
+  }
+  for (int o = 16; o; o >>= 1) {
+    const double ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+    const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+    if (oi >= 0 && (bi < 0 || ov < bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+  }
+  if (lane == 0) {
+    dp->best[r & 1][j] = bv;
+    cut[(size_t)r * SORT_ROWS + j] = (short)bi;
+  }
+}
+
+// One thread: the backtrack, the code points in ascending order, the least total cost.  rows = rows the host launched
+// (n_entries - 1 at most); with fewer cells than entries the programme stops at the last row that has a cell.
+__global__ void grid_dp_last_kernel(const DpScratch* __restrict__ dp, int n_entries, const short* __restrict__ cut, float* __restrict__ out_lut,
+                                    double* __restrict__ cost_out) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const int B = dp->B;
   if (B == 0) {
-    if (tid < SOP_MAX_ENTRIES) out_lut[tid] = 0.0f;
-    if (tid == 0) cost_out[0] = 0.0;
+    for (int e = 0; e < SOP_MAX_ENTRIES; ++e) out_lut[e] = 0.0f;
+    cost_out[0] = 0.0;
     return;
   }
   const int R = min(n_entries, B);
-  for (int j = tid; j < B; j += DP_TB) best[0][j] = dp_run_cost(pH, pS, pQ, 0, j, nullptr);
-  __syncthreads();
-  for (int r = 1; r < R; ++r) {
-    const double* prev = best[(r - 1) & 1];
-    double* cur = best[r & 1];
-    for (int j = tid; j < B; j += DP_TB) {
-      if (j < r) continue;
-      double bv = 0.0;
-      int bi = -1;
-      for (int i = r; i <= j; ++i) {               // the last run is cells i..j
-        const double v = __dadd_rn(prev[i - 1], dp_run_cost(pH, pS, pQ, i, j, nullptr));
-        if (bi < 0 || v < bv) { bv = v; bi = i; }
-      }
-      cur[j] = bv;
-      cut[(size_t)r * SORT_ROWS + j] = (short)bi;
-    }
-    __syncthreads();
+  float lut[SOP_MAX_ENTRIES];
+  int j = B - 1, n = 0;
+  for (int r = R - 1; r >= 0; --r) {
+    const int i = r == 0 ? 0 : (int)cut[(size_t)r * SORT_ROWS + j];
+    float q;
+    dp_run_cost(dp->pH, dp->pS, dp->pQ, i, j, &q);
+    lut[n++] = q;
+    j = i - 1;
   }
-  if (tid == 0) {
-    int j = B - 1, n = 0;
-    for (int r = R - 1; r >= 0; --r) {
-      const int i = r == 0 ? 0 : (int)cut[(size_t)r * SORT_ROWS + j];
-      float q;
-      dp_run_cost(pH, pS, pQ, i, j, &q);
-      s_lut[n++] = q;
-      j = i - 1;
-    }
-    // ascending (insertion sort of at most 32 values), padded with the last entry
-    for (int a = 1; a < n; ++a) {
-      const float v = s_lut[a];
-      int b = a - 1;
-      while (b >= 0 && s_lut[b] > v) { s_lut[b + 1] = s_lut[b]; --b; }
-      s_lut[b + 1] = v;
-    }
-    for (int e = n; e < SOP_MAX_ENTRIES; ++e) s_lut[e] = s_lut[n - 1];
-    for (int e = 0; e < SOP_MAX_ENTRIES; ++e) out_lut[e] = e < n_entries ? s_lut[e] : 0.0f;
-    cost_out[0] = __ddiv_rn(best[(R - 1) & 1][B - 1], 16777216.0);
+  for (int a = 1; a < n; ++a) {                   // ascending: insertion sort of at most 32 values
+    const float v = lut[a];
+    int b = a - 1;
+    while (b >= 0 && lut[b] > v) { lut[b + 1] = lut[b]; --b; }
+    lut[b + 1] = v;
   }
+  for (int e = 0; e < SOP_MAX_ENTRIES; ++e) out_lut[e] = e < n ? lut[e] : (e < n_entries ? lut[n - 1] : 0.0f);
+  cost_out[0] = __ddiv_rn(dp->best[(R - 1) & 1][B - 1], 16777216.0);
 }
 
 int num_sms();
@@ -908,11 +943,13 @@ extern "C" {
 
 int sop_dd4_lloyd_launches(long long M, long long K, int iters, int flags, int* launches) {
   if (!launches) return SOP_ERR_NULL;
+  const int dp_entries = iters > 1 ? iters : 2;      // with SOP_LLOYD_GRID_DP the caller passes the number of table entries here
   if (M < 1 || K < 1 || (K % SOP_G) != 0 || iters < 0 || iters > sop::SOP_MAX_LLOYD_ITERS) return SOP_ERR_RANGE;
   long long grid = 1;
   const bool persistent = sop::lloyd_iteration_plan(M * (K / SOP_G), M * (K / SOP_G), iters, flags, &grid);
   // radix select (three passes, unless the pool is cut by a threshold), set-up, pool list, pool cache, iterations
-  *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + ((flags & SOP_LLOYD_GRID_DP) ? 1 : (persistent ? 1 : iters + 1));
+  // the dynamic programme: first row, one launch per further row (callers with a 16-entry table: 15), the backtrack
+  *launches = ((flags & SOP_LLOYD_POOL_THRESHOLD) ? 0 : 3) + 3 + ((flags & SOP_LLOYD_GRID_DP) ? 2 + (dp_entries - 1) : (persistent ? 1 : iters + 1));
   return SOP_OK;
 }
 
@@ -1001,10 +1038,12 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     const size_t stage_bytes = (size_t)TILE_ELEMS * sizeof(uint2);
     static bool attr_set = false;
     if (!attr_set) {
-      SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
+      SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
+      SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
       attr_set = true;
     }
-    pool_cache_kernel<<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
+    if (grid_dp) pool_cache_kernel<true><<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
+    else pool_cache_kernel<false><<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
     SOP_CUDA_TRY(cudaGetLastError());
   }
   if (grid_dp) {
@@ -1017,7 +1056,12 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     }
     if (ne < 2) return SOP_ERR_ALPHABET;
     if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
-    grid_dp_kernel<<<1, DP_TB, 0, st>>>(ws, ne, out_lut_dev, distortion_dev, &ws->dp_cut[0][0]);
+    static_assert(sizeof(DpScratch) <= sizeof(((LloydWs*)nullptr)->dp_scratch), "scratch of the dynamic programme");
+    DpScratch* dp = reinterpret_cast<DpScratch*>(ws->dp_scratch);
+    grid_dp_first_kernel<<<1, DP_TB, 0, st>>>(ws, dp);
+    for (int r = 1; r < ne; ++r)      // a row without a cell (fewer cells than entries) returns at once
+      grid_dp_row_kernel<<<(SORT_ROWS + DP_TB / 32 - 1) / (DP_TB / 32), DP_TB, 0, st>>>(dp, r, &ws->dp_cut[0][0]);
+    grid_dp_last_kernel<<<1, 32, 0, st>>>(dp, ne, &ws->dp_cut[0][0], out_lut_dev, distortion_dev);
     SOP_CUDA_TRY(cudaGetLastError());
     if ((rc = profile_mark(SOP_PROFILE_LLOYD, 1, st))) return rc;
     return SOP_OK;

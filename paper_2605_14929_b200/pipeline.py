@@ -72,14 +72,18 @@ class LayerSweep:
     format): the large scratch buffers -- workspaces, the per-block arrays, the channel norms, the packed
     codes and scale words -- are then that sweep's, and only the small results (tables, result blocks, the DD
     table, counts) are this sweep's own.  Sweeps that share buffers must run one after the other on one stream,
-    and the packed output of one is overwritten by the next."""
+    and the packed output of one is overwritten by the next.  ``grid_dp`` builds the DD atom by the grid-constrained
+    dynamic programme instead of Lloyd iterations with a snap (``lloyd_iters`` > 0 then only says that there is a DD
+    atom)."""
 
     def __init__(self, M: int, K: int, T: int, fmt: I.ScaleFormat, rom: Sequence[str], fp: Sequence[str] = (),
                  lloyd_iters: int = 8, pool_percent: float = 50.0, device="cuda", want_blocks: bool = False,
-                 share: Optional["LayerSweep"] = None):
+                 share: Optional["LayerSweep"] = None, grid_dp: bool = False):
         self.M, self.K, self.T, self.fmt = M, K, T, fmt
         self.dev = torch.device(device)
         self.iters = lloyd_iters
+        self.grid_dp = bool(grid_dp) and lloyd_iters > 0
+        self.dd_iters = 0 if self.grid_dp else lloyd_iters        # iterations handed to sop_dd4_lloyd; its status entry
         self.rom_atoms = I.alphabet(rom, with_negations=True)
         if not self.rom_atoms:
             # element formats only (a promotion-profile comparison): singles, no pair, no DD atom; the first one is packed
@@ -138,7 +142,10 @@ class LayerSweep:
             self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
             self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
         self.kernel_launches_per_step = 0
-        self.lloyd_launches = B.dd4_lloyd_launches(M, K, lloyd_iters) if lloyd_iters > 0 else 0
+        self.lloyd_launches = 0
+        if lloyd_iters > 0:      # (the query takes the table size in place of the iterations for the dynamic programme)
+            self.lloyd_launches = (B.dd4_lloyd_launches(M, K, 1 << n_bits, B.LLOYD_GRID_DP) if self.grid_dp
+                                   else B.dd4_lloyd_launches(M, K, lloyd_iters))
 
     def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True) -> None:
         """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32.  ``norms`` =
@@ -154,8 +161,9 @@ class LayerSweep:
                               self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
                               stream=stream)
             n += 3
-            B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.iters, self.dd_lut,
-                            self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream)
+            B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.dd_iters, self.dd_lut,
+                            self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream,
+                            grid_dp=self.grid_dp)
             n += self.lloyd_launches
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
                               self.ws_search, dd_lut=self.dd_lut, dd_mask=self.dd_mask, block_cos=self.full_cos,
@@ -195,7 +203,7 @@ class LayerSweep:
     def outputs(self) -> SweepOutputs:
         torch.cuda.synchronize(self.dev)
         if self.iters > 0:
-            B.check_lloyd_status(self.distortion, self.iters)     # a codebook from an unfinished call is not handed out
+            B.check_lloyd_status(self.distortion, self.dd_iters)  # a codebook from an unfinished call is not handed out
         nF, nR = len(self.full_atoms), len(self.rom_atoms)
         return SweepOutputs(
             c=self.c.cpu(), pair_table=B.read_pair_table(self.pair_table, nF),
@@ -281,7 +289,7 @@ class LayerStream:
         self.out_done[slot].synchronize()
         for f, q in enumerate(self.sweeps):
             if q.iters > 0:
-                B.check_lloyd_status(self.host_out[slot][f]["distortion"], q.iters)
+                B.check_lloyd_status(self.host_out[slot][f]["distortion"], q.dd_iters)
         return self.host_out[slot][0] if self.single else self.host_out[slot]
 
 
@@ -338,4 +346,4 @@ class LayerSetSweep:
         for row in self.sweeps:
             for sw in row:
                 if sw.iters > 0:
-                    B.check_lloyd_status(sw.distortion, sw.iters)
+                    B.check_lloyd_status(sw.distortion, sw.dd_iters)
