@@ -196,11 +196,20 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
   if (PASS > 0) derive_prefix(ws, a.pool_rank, PASS, &prefix, &rank, &below, &cnt);
   __syncthreads();
   const float* row = a.cosrow_base + (size_t)resolve_fmta(a, res) * a.NB;
-  for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += (long long)gridDim.x * LTB) {
-    const unsigned key = pool_key(__ldg(row + i), a.flags);
-    if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
-    else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&sh[(key >> 10) & 2047u], 1u); }
-    else { if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u); }
+  // four keys per thread and round, their loads in flight together (the pass is bound by memory latency otherwise)
+  const long long stride = (long long)gridDim.x * LTB;
+  for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += 4 * stride) {
+    float v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) v[q] = i + q * stride < a.NB ? __ldg(row + i + q * stride) : 0.0f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (i + q * stride >= a.NB) break;
+      const unsigned key = pool_key(v[q], a.flags);
+      if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
+      else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&sh[(key >> 10) & 2047u], 1u); }
+      else { if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u); }
+    }
   }
   __syncthreads();
   for (int i = threadIdx.x; i < 2048; i += LTB)
@@ -286,22 +295,31 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   lloyd_publish_desc(ws, s_lut, s_ne);
 }
 
-// Dense list of the pool blocks.  One counter update per CTA and round: the warps' counts are scanned
-// in shared memory.  The order of the list depends on the scheduling of the CTAs; nothing downstream
-// depends on it (integer sums, and an FP64 sum compared with a tolerance).
+// Dense list of the pool blocks.  A thread takes four consecutive blocks per round; the CTA's count goes to the list's
+// counter once per round (a warp scan of the threads' counts, then a scan of the eight warp totals).  The order of the
+// list depends on the scheduling of the CTAs; nothing downstream depends on it (integer sums, and an FP64 sum compared
+// with a tolerance).
 __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __restrict__ ws) {
   __shared__ unsigned s_cnt[LTB / 32];
   __shared__ unsigned s_base;
   const unsigned tau_key = ws->tau_key;
   const float* row = a.cosrow_base + (size_t)ws->fmta * a.NB;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long stride = (long long)gridDim.x * LTB;
+  const long long stride = (long long)gridDim.x * LTB * 4;
   const long long n_round = (a.NB + stride - 1) / stride;
-  long long i = (long long)blockIdx.x * LTB + threadIdx.x;
+  long long i = ((long long)blockIdx.x * LTB + threadIdx.x) * 4;
   for (long long r = 0; r < n_round; ++r, i += stride) {
-    const bool in = i < a.NB && pool_key(__ldg(row + i), a.flags) <= tau_key;
-    const unsigned bal = __ballot_sync(0xFFFFFFFFu, in);
-    if (lane == 0) s_cnt[warp] = (unsigned)__popc(bal);
+    unsigned in = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (i + q < a.NB && pool_key(__ldg(row + i + q), a.flags) <= tau_key) in |= 1u << q;
+    const unsigned mine = (unsigned)__popc(in);
+    unsigned incl = mine;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_cnt[warp] = incl;
     __syncthreads();
     if (threadIdx.x == 0) {
       unsigned tot = 0;
@@ -309,8 +327,11 @@ __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __
       s_base = tot ? atomicAdd(&ws->list_count, tot) : 0u;
     }
     __syncthreads();
-    if (in) a.pool_idx[s_base + s_cnt[warp] + __popc(bal & ((1u << lane) - 1u))] = (unsigned)i;
-    __syncthreads();
+    unsigned at = s_base + s_cnt[warp] + incl - mine;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if ((in >> q) & 1u) a.pool_idx[at++] = (unsigned)(i + q);
+    __syncthreads();             // s_cnt and s_base are rewritten in the next round
   }
 }
 

@@ -116,13 +116,11 @@ __device__ __forceinline__ void load_block_bits(const uint16_t* p, uint32_t (&v)
 }
 
 __device__ __forceinline__ float absmax_bits(const uint32_t (&v)[8]) {
-  // bf16 magnitudes order like their bit patterns
+  // bf16 magnitudes order like their bit patterns: the maximum of the sixteen 15-bit patterns, two per word at a time
   uint32_t m = 0;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    m = max(m, v[i] & 0x7FFFu);
-    m = max(m, (v[i] >> 16) & 0x7FFFu);
-  }
+  for (int i = 0; i < 8; ++i) m = __vmaxu2(m, v[i] & 0x7FFF7FFFu);
+  m = max(m & 0xFFFFu, m >> 16);
   return __uint_as_float(m << 16);
 }
 
