@@ -13,9 +13,11 @@ the sweep of every fixed candidate (finds FMTa), the DD4 Lloyd refinement, the s
 (every pair), and the pack of the chosen pair.  The metric counts a weight element once per scale format.
 With N > 1 every rank sweeps its own transformer block (layers are independent: no data-path collective).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload block|layer]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on a bounded sample.
+``--workload layer`` runs a smaller case of the same kernels -- the block's first layer (8192 x 8192) at one scale
+format (E5M6) -- sized for profiler captures (1.5 GB on the device, W larger than L2); its line says so in ``config``.
 """
 from __future__ import annotations
 
@@ -51,6 +53,8 @@ SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # file (dram__bytes_read.sum + dram__bytes_write.sum of one launch on a reduced-row layer divided by its
 # elements; traffic grows in proportion to the rows).  None: no capture of the kernel as it is now.
 NCU_SWEEP_TRAFFIC = dict(source=None, bytes_per_element_fixed_candidates=None, bytes_per_element_dd_columns=None)
+# the same for the reduction kernel (first call: the fixed candidates' entries; second call: the DD columns' entries)
+NCU_REDUCE_TRAFFIC = dict(source=None, bytes_per_element_fixed_candidates=None, bytes_per_element_dd_columns=None)
 
 
 # ---------------------------------------------------------------------------------------------------------
@@ -77,11 +81,18 @@ def search_ops_cell_lookup(n_lut: int, n_bits: int, n_fp: int, n_dd: int, signed
     return 12 + n_lut * 6.5 + n_fp * 12 + per_block / 16.0
 
 
+def sweep_kernel_ops_n_step(n_eval_lut: int, n_bits: int, n_eval_fp: int) -> float:
+    """The part of ``search_ops_n_step`` that one launch of the evaluation kernel does: the shared 6, 2n + 5 per LUT
+    candidate it evaluates, 12 per FP candidate, and per block 6 per evaluated candidate (its cosine)."""
+    return 6 + n_eval_lut * (2 * n_bits + 5) + n_eval_fp * 12 + 6 * (n_eval_lut + n_eval_fp) / 16.0
+
+
 def search_bytes(n_cand: int, n_dd: int) -> float:
-    """Algorithmic DRAM bytes per element of the two launches as the call plan has them: W (2 bytes) read by each,
-    8 bytes per block for every candidate written (per-block cosine and error: the Lloyd pool and the pack read
-    them) and 8 per block for every fixed candidate the second launch loads."""
-    return 2 * 2.0 + (8.0 * n_cand + 8.0 * (n_cand - n_dd)) / 16.0
+    """Algorithmic DRAM bytes per element of the search as the call plan has it: W (2 bytes) read by each of the two
+    evaluation launches, 8 bytes per block for every candidate's column written (per-block cosine and error: the
+    reduction, the Lloyd pool and the pack read them), the fixed candidates' columns read by the first reduction and
+    every column by the second."""
+    return 2 * 2.0 + (8.0 * n_cand + 8.0 * (n_cand - n_dd) + 8.0 * n_cand) / 16.0
 
 
 class ClockSampler:
@@ -200,7 +211,8 @@ def time_sweeps(sweeps, reps, flush):
         t_sw = 0.0
         for sw, W, X, norms in sweeps:
             sw.run(W, X, st, norms=norms)
-            t_sw += B.profile_ms(B.PROFILE_SWEEP, 0) + (B.profile_ms(B.PROFILE_SWEEP, 1) if sw.iters > 0 else 0.0)
+            for back in range(2 if sw.iters > 0 else 1):           # with a DD atom the search is two calls
+                t_sw += B.profile_ms(B.PROFILE_SWEEP, back) + B.profile_ms(B.PROFILE_REDUCE, back)
         e1.record(st)
         torch.cuda.synchronize()
         whole.append(e0.elapsed_time(e1))
@@ -304,10 +316,13 @@ def run_gpu(args) -> None:
         dist.init_process_group("nccl", device_id=dev)
     B.lib()
 
-    fmts = [I.scale_format(f) for f in WORKLOAD["scale_formats"]]
+    small = args.workload == "layer"                              # the profiling case: one layer, one format
+    fmt_names = ["E5M6"] if small else WORKLOAD["scale_formats"]
+    fmts = [I.scale_format(f) for f in fmt_names]
     S = len(fmts)
     block = block_for_rank(rank)                                  # every rank sweeps its own transformer block
-    layers = [I.config5_layer(0, block, which, device=str(dev)) for which in range(len(I.SHAPES_70B))]
+    layers = [I.config5_layer(0, block, which, device=str(dev)) for which in range(1 if small else len(I.SHAPES_70B))]
+    layer_names = WORKLOAD["layers"][:len(layers)]
     dev_layers = [(L.W, L.X) for L in layers]
     shapes = [(L.W.shape[0], L.W.shape[1], L.X.shape[0]) for L in layers]
     sset = LayerSetSweep(shapes, fmts, WORKLOAD["rom"], WORKLOAD["fp"], WORKLOAD["lloyd_iters"], device=dev)
@@ -357,7 +372,7 @@ def run_gpu(args) -> None:
 
     # ---- one pass call by call: per (layer, format) the library's events around its main kernels ----
     B.profile_enable(True)
-    kern = dict(sweep1=0.0, sweep2=0.0, lloyd=0.0, pack=0.0, norms=0.0)
+    kern = dict(sweep1=0.0, sweep2=0.0, reduce1=0.0, reduce2=0.0, lloyd=0.0, pack=0.0, norms=0.0)
     per_layer_sweep_ms = []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -366,13 +381,16 @@ def run_gpu(args) -> None:
         for f, sw in enumerate(row):
             sw.run(W, X, stream, norms=(f == 0))
             s2, s1 = B.profile_ms(B.PROFILE_SWEEP, 0), B.profile_ms(B.PROFILE_SWEEP, 1)
+            r2, r1 = B.profile_ms(B.PROFILE_REDUCE, 0), B.profile_ms(B.PROFILE_REDUCE, 1)
             kern["sweep2"] += s2
             kern["sweep1"] += s1
+            kern["reduce2"] += r2
+            kern["reduce1"] += r1
             kern["lloyd"] += B.profile_ms(B.PROFILE_LLOYD, 0)
             kern["pack"] += B.profile_ms(B.PROFILE_PACK, 0)
             if f == 0:
                 kern["norms"] += B.profile_ms(B.PROFILE_NORMS, 0)
-            t_layer += s1 + s2
+            t_layer += s1 + s2 + r1 + r2
         per_layer_sweep_ms.append(t_layer)
     e1.record(stream)
     barrier()
@@ -433,42 +451,61 @@ def run_gpu(args) -> None:
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
         of = "measured" if peaks else "fallback"
         n_lut, nb = len(sset.sweeps[0][0].full_atoms), 4
+        n_dd = 2
         signed = [bool(f.sign_bits) for f in fmts]
         ops_n_step = search_ops_n_step(n_lut, nb, 0)
-        ops_cell = sum(search_ops_cell_lookup(n_lut, nb, 0, 2, s) for s in signed) / S
-        sweep_t = (kern["sweep1"] + kern["sweep2"]) * 1e-3              # all 2 * 5 * 8 sweep launches of a step
-        n_launch = 2 * len(shapes) * S
-        ach = ops_n_step * units / sweep_t / 1e12
-        ach_cell = ops_cell * units / sweep_t / 1e12
-        alg_bytes = search_bytes(n_lut, 2)
+        ops_cell = sum(search_ops_cell_lookup(n_lut, nb, 0, n_dd, s) for s in signed) / S
+        n_pass = len(shapes) * S                                        # (layer, format) passes of a step
+        sweep_t = (kern["sweep1"] + kern["sweep2"]) * 1e-3              # the 2 n_pass launches of the evaluation kernel
+        reduce_t = (kern["reduce1"] + kern["reduce2"]) * 1e-3           # the 2 n_pass launches of the reduction kernel
+        search_t = sweep_t + reduce_t
+        # the evaluation kernel by itself: its own share of the operation count
+        ops_sweep = sweep_kernel_ops_n_step(n_lut - n_dd, nb, 0) + sweep_kernel_ops_n_step(n_dd, nb, 0)
+        ach_sweep = ops_sweep * units / sweep_t / 1e12
+        ach = ops_n_step * units / search_t / 1e12
+        ach_cell = ops_cell * units / search_t / 1e12
+        alg_bytes = search_bytes(n_lut, n_dd)
+        sweep_bytes = 2 * 2.0 + 8.0 * n_lut / 16.0                       # W by each launch, every column written once
         bpe = [NCU_SWEEP_TRAFFIC["bytes_per_element_fixed_candidates"], NCU_SWEEP_TRAFFIC["bytes_per_element_dd_columns"]]
-        traffic = None if None in bpe else (bpe[0] + bpe[1]) / 2.0 * units / (n_launch / 2)
+        traffic = None if None in bpe else (bpe[0] + bpe[1]) / 2.0 * units / n_pass
+        rbpe = [NCU_REDUCE_TRAFFIC["bytes_per_element_fixed_candidates"], NCU_REDUCE_TRAFFIC["bytes_per_element_dd_columns"]]
         roofline = dict(
-            kernel="sweep_kernel", launches_per_step=n_launch, bound="alu", achieved=ach, peak=alu_peak, unit="T thread-instr/s",
-            frac=ach / alu_peak, traffic=traffic, traffic_source=NCU_SWEEP_TRAFFIC["source"],
+            kernel="sweep_kernel", launches_per_step=2 * n_pass, bound="alu", achieved=ach_sweep, peak=alu_peak, unit="T thread-instr/s",
+            frac=ach_sweep / alu_peak, traffic=traffic, traffic_source=NCU_SWEEP_TRAFFIC["source"],
             peak_source=f"{SM_COUNT} SMs x {SCHEDULERS} schedulers x {LANES} lanes x {sm_max:.0f} MHz (clocks.max.sm, {of})",
-            avg_launch_ms=sweep_t * 1e3 / n_launch,
-            models=dict(
+            avg_launch_ms=sweep_t * 1e3 / (2 * n_pass),
+            ops_per_element=dict(fixed_candidates=sweep_kernel_ops_n_step(n_lut - n_dd, nb, 0), dd_columns=sweep_kernel_ops_n_step(n_dd, nb, 0)),
+            algorithmic_bytes_per_launch=sweep_bytes / 2.0 * units / n_pass,
+            note="the dominant kernel of the step: the evaluation of every candidate on every block (two launches per layer and "
+                 "format: the fixed candidates, then the DD columns), against its own share of the n-step operation count; "
+                 "`search` below is the whole search (evaluation + reduction of the table entries) against the whole count",
+            search=dict(
+                kernels=["sweep_kernel", "reduce_kernel"], launches_per_step=4 * n_pass, ms_per_step=search_t * 1e3,
                 n_step_search=dict(ops_per_element=ops_n_step, achieved=ach, frac=ach / alu_peak,
-                                   note="operation count of an n-step nearest-entry search (2n + 5 per LUT candidate and element); "
-                                        "roofline.frac is this one"),
+                                   note="operation count of an n-step nearest-entry search: 6 shared, 2n + 5 per LUT candidate and "
+                                        "element, per block 6 per candidate and 2 per pair of candidates (diagonal included)"),
                 cell_lookup=dict(ops_per_element=ops_cell, achieved=ach_cell, frac=ach_cell / alu_peak,
-                                 note="operation count of the kernel's own scheme: one-step cell lookup (4) and packed multiply-adds "
-                                      "(2.5) per LUT candidate and element, W unpacked in both launches, loaded columns, signed entries")),
-            algorithmic_bytes_per_launch=alg_bytes / 2.0 * units / (n_launch / 2),
-            bytes_per_element=dict(algorithmic=alg_bytes, w_twice=4.0, over_w_twice=alg_bytes / 4.0),
-            hbm=dict(achieved=alg_bytes * units / sweep_t / 1e9, peak=hbm_peak, unit="GB/s",
-                     frac=alg_bytes * units / sweep_t / 1e9 / hbm_peak, of=of,
-                     note="algorithmic bytes of both launches (W twice, per-block values written and loaded) over their time: "
-                          "the sweep is far from the HBM roofline"))
+                                 note="operation count of this library's own scheme: one-step cell lookup (4) and packed multiply-adds "
+                                      "(2.5) per LUT candidate and element, W unpacked in both launches, loaded columns, signed entries"),
+                reduce_kernel=dict(ms_per_step=reduce_t * 1e3, avg_launch_ms=reduce_t * 1e3 / (2 * n_pass),
+                                   traffic=None if None in rbpe else (rbpe[0] + rbpe[1]) / 2.0 * units / n_pass,
+                                   traffic_source=NCU_REDUCE_TRAFFIC["source"],
+                                   algorithmic_bytes_per_launch=(8.0 * (n_lut - n_dd) + 8.0 * n_lut) / 16.0 / 2.0 * units / n_pass,
+                                   hbm=dict(achieved=(8.0 * (n_lut - n_dd) + 8.0 * n_lut) / 16.0 * units / reduce_t / 1e9, peak=hbm_peak,
+                                            unit="GB/s", frac=(8.0 * (n_lut - n_dd) + 8.0 * n_lut) / 16.0 * units / reduce_t / 1e9 / hbm_peak, of=of)),
+                bytes_per_element=dict(algorithmic=alg_bytes, w_twice=4.0, over_w_twice=alg_bytes / 4.0),
+                hbm=dict(achieved=alg_bytes * units / search_t / 1e9, peak=hbm_peak, unit="GB/s",
+                         frac=alg_bytes * units / search_t / 1e9 / hbm_peak, of=of,
+                         note="algorithmic bytes of the search (W twice, every column written once and read by the reductions) over "
+                              "its time: the search is far from the HBM roofline")))
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
         try:
-            per_config = per_config_table(dev, alu_peak, flush) if world == 1 else None
+            per_config = per_config_table(dev, alu_peak, flush) if world == 1 and not small else None
         except Exception as exc:                               # the headline line does not depend on the side table
             per_config = dict(error=repr(exc))
         if per_config is not None and "error" not in per_config:
             per_config["config5"] = dict(elements_times_formats=units, whole_path=dict(value=units / ms / 1e6, unit=UNIT, ms=ms),
-                                         sweep_only=dict(value=units / (sweep_t * 1e3) / 1e6, unit=UNIT, ms=sweep_t * 1e3),
+                                         sweep_only=dict(value=units / (search_t * 1e3) / 1e6, unit=UNIT, ms=search_t * 1e3),
                                          ops_per_element_n_step=ops_n_step, frac_of_alu_peak=ach / alu_peak,
                                          note="the headline workload: block 0, five layers, eight scale formats")
         cpu_rows = 384
@@ -477,16 +514,21 @@ def run_gpu(args) -> None:
             metric=METRIC, value=job_value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=max(3, args.warmup), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
             dtype="f32", data="synthetic",
-            config=dict(WORKLOAD, block=f"rank r sweeps block r (seed 0)", elements_per_step=E, element_formats_per_step=units,
-                        l2="inputs larger than L2: 1.1 GB of W per step, every layer above 126 MB except the two 1024x8192 ones; "
-                           "a layer's eight formats run back to back, as in a real sweep, so its W may be served from L2 there",
+            config=dict(WORKLOAD if not small else dict(WORKLOAD, workload="profiling case of config5: its first layer (8192x8192) at E5M6 only",
+                                                        layers=layer_names, scale_formats=fmt_names),
+                        block=f"rank r sweeps block r (seed 0)", elements_per_step=E, element_formats_per_step=units,
+                        l2=("inputs larger than L2: 1.1 GB of W per step, every layer above 126 MB except the two 1024x8192 ones; "
+                            "a layer's eight formats run back to back, as in a real sweep, so its W may be served from L2 there")
+                        if not small else "W (134 MB) and the per-block columns (335 MB) are larger than L2",
                         launch=launch_kind, parallelism=f"layer-parallel x{world}, no collective"),
-            kernels_ms=dict(kern, ms_per_step_call_by_call=call_ms, sweep_ms_per_layer=dict(zip(WORKLOAD["layers"], per_layer_sweep_ms)),
-                            note="sums over the 40 (layer, format) passes of one step launched call by call, CUDA events recorded "
-                                 "by the library around its main kernels; sweep1 = fixed candidates (finds FMTa), sweep2 = DD "
-                                 "columns (all pairs), lloyd = the iteration launches only, norms once per layer"),
-            sweep_only=dict(value=world * units / sweep_t / 1e9, unit=UNIT,
-                            note="element-formats / time of the sweep launches of a step (every candidate, every pair)"),
+            kernels_ms=dict(kern, ms_per_step_call_by_call=call_ms, search_ms_per_layer=dict(zip(layer_names, per_layer_sweep_ms)),
+                            note="sums over the (layer, format) passes of one step launched call by call, CUDA events recorded by the "
+                                 "library around its main kernels; sweep1 / reduce1 = the fixed candidates' columns and the table "
+                                 "entries among them (finds FMTa), sweep2 / reduce2 = the DD columns and their entries, lloyd = the "
+                                 "iteration launches only, norms once per layer"),
+            sweep_only=dict(value=world * units / search_t / 1e9, unit=UNIT,
+                            note="element-formats / time of the search launches of a step (every candidate, every pair: evaluation "
+                                 "and reduction kernels)"),
             roofline=roofline, per_config=per_config,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
                               sample=f"first {cpu_rows} of 8192 rows of the 8192x8192 layer at E5M6 (one layer, one format), whole "
@@ -505,6 +547,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="block", choices=["block", "layer"],
+                    help="block: the benchmark (one transformer block, eight scale formats); layer: its first layer at one format, for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -1318,6 +1318,8 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     sweep_kernel<<<(int)grid, TB, smem, st>>>(L, P, A, F, hdr, cos_cols, sse_cols, prev_result_dev);
     SOP_CUDA_TRY(cudaGetLastError());
   }
+  if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
+  if ((rc = profile_mark(SOP_PROFILE_REDUCE, 0, st))) return rc;
   const bool sel_err = (flags & SOP_SEARCH_SELECT_MSE) != 0;
   for (int l = 0; l < n_launch; ++l) {
     const int task0 = l * PER_LAUNCH;
@@ -1341,7 +1343,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
 #undef SOP_LAUNCH_REDUCE
     SOP_CUDA_TRY(cudaGetLastError());
   }
-  if ((rc = profile_mark(SOP_PROFILE_SWEEP, 1, st))) return rc;
+  if ((rc = profile_mark(SOP_PROFILE_REDUCE, 1, st))) return rc;
   return SOP_OK;
 }
 
