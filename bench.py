@@ -372,7 +372,7 @@ def run_gpu(args) -> None:
 
     # ---- one pass call by call: per (layer, format) the library's events around its main kernels ----
     B.profile_enable(True)
-    kern = dict(sweep1=0.0, sweep2=0.0, reduce1=0.0, reduce2=0.0, lloyd=0.0, pack=0.0, norms=0.0)
+    kern = dict(prepass=0.0, sweep1=0.0, sweep2=0.0, reduce1=0.0, reduce2=0.0, pool=0.0, lloyd=0.0, pack=0.0, norms=0.0)
     per_layer_sweep_ms = []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -386,6 +386,8 @@ def run_gpu(args) -> None:
             kern["sweep1"] += s1
             kern["reduce2"] += r2
             kern["reduce1"] += r1
+            kern["prepass"] += B.profile_ms(B.PROFILE_PREPASS, 1)
+            kern["pool"] += B.profile_ms(B.PROFILE_POOL, 0)
             kern["lloyd"] += B.profile_ms(B.PROFILE_LLOYD, 0)
             kern["pack"] += B.profile_ms(B.PROFILE_PACK, 0)
             if f == 0:

@@ -205,12 +205,15 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
  *   SOP_PROFILE_SWEEP   the sweep kernel of sop_pair_search (one launch; the events coincide when the call evaluates nothing)
  *   SOP_PROFILE_REDUCE  the reduction kernel(s) of sop_pair_search
  *   SOP_PROFILE_LLOYD   the iteration kernel(s) of sop_dd4_lloyd, or the launches of its dynamic programme
+ *   SOP_PROFILE_POOL    what sop_dd4_lloyd launches before them: radix select, set-up, pool list, pool cache
+ *   SOP_PROFILE_PREPASS the shift prepass of sop_pair_search (the events coincide when the call takes its shifts from a result)
  *   SOP_PROFILE_PACK    the kernel of sop_pack
  *   SOP_PROFILE_NORMS   both kernels of sop_channel_norms
  * sop_profile_ms waits for the second event of a call of that kind (back = 0: the last call, 1: the one
  * before, ... up to 7) and returns the time between its two events in milliseconds (SOP_ERR_RANGE if
  * no such call has run since profiling was enabled).  Not thread-safe. */
-enum { SOP_PROFILE_SWEEP = 0, SOP_PROFILE_LLOYD = 1, SOP_PROFILE_PACK = 2, SOP_PROFILE_NORMS = 3, SOP_PROFILE_REDUCE = 4, SOP_PROFILE_KINDS = 5 };
+enum { SOP_PROFILE_SWEEP = 0, SOP_PROFILE_LLOYD = 1, SOP_PROFILE_PACK = 2, SOP_PROFILE_NORMS = 3, SOP_PROFILE_REDUCE = 4, SOP_PROFILE_POOL = 5,
+       SOP_PROFILE_PREPASS = 6, SOP_PROFILE_KINDS = 7 };
 int sop_profile_enable(int on);
 int sop_profile_ms(int which, int back, float* ms);
 int sop_profile_last_ms(int which, float* ms);    /* = sop_profile_ms(which, 0, ms) */

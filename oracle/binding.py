@@ -45,6 +45,9 @@ def lib():
         _lib.osop_layer_pot_scale.restype = C.c_float
         _lib.osop_grid_quantize.restype = C.c_float
         _lib.osop_grid_value.restype = C.c_double
+        _lib.osop_opq_threshold.restype = C.c_double
+        _lib.osop_opq_extract.restype = C.c_longlong
+        _lib.osop_wr_extract.restype = C.c_longlong
     return _lib
 
 
@@ -233,3 +236,42 @@ def pack(W, c, fmt, a, k_a: int, b=None, k_b: int = 0, use_sign: int = 0, contai
                          use_sign, container_bits, word_sign_bits, int(select_metric), _p(codes, C.c_ubyte), _p(words, C.c_ubyte),
                          C.byref(n1), C.byref(nn))
     return dict(rc=rc, codes=codes, words=words, n_sel1=n1.value, n_neg=nn.value)
+
+
+def opq_threshold(q: float, max_order: int = 16) -> float:
+    """m with (2 Phi(m) - 1)^M = q (Section "Outlier Per-Quantum Extraction (OPQ)")."""
+    return float(lib().osop_opq_threshold(C.c_double(q), int(max_order)))
+
+
+def opq_extract(W, m: float, capacity: int = None):
+    """Returns dict(W_out [M, K] uint16 bf16 bits, row_start [M + 1] uint32, records uint32 (k | bf16 << 16), count)."""
+    w16 = _w16(W)
+    M, K = w16.shape
+    cap = M * K if capacity is None else int(capacity)
+    out = np.zeros_like(w16)
+    row_start = np.zeros(M + 1, dtype=np.uint32)
+    records = np.zeros(max(cap, 1), dtype=np.uint32)
+    n = lib().osop_opq_extract(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), C.c_double(m),
+                               _p(out, C.c_uint16), C.c_longlong(K), _p(row_start, C.c_uint), _p(records, C.c_uint), C.c_longlong(cap))
+    return dict(W_out=out, row_start=row_start, records=records[:min(n, cap)].copy(), count=int(n))
+
+
+def wr_extract(W, c, fmt, a, k_a: int, b=None, k_b: int = 0, use_sign: int = 0, n_keep: int = 1, select_metric: int = 0,
+               capacity: int = None, want_resid: bool = False):
+    """Returns dict(row_start, records uint32 (k | E3M4 code << 16), count, scale_exp, tau[, resid [M, K] float32])."""
+    w16 = _w16(W)
+    M, K = w16.shape
+    c = np.ascontiguousarray(np.asarray(c, dtype=np.float32))
+    cap = M * K if capacity is None else int(capacity)
+    row_start = np.zeros(M + 1, dtype=np.uint32)
+    records = np.zeros(max(cap, 1), dtype=np.uint32)
+    resid = np.zeros((M, K), dtype=np.float32) if want_resid else None
+    e, tau = C.c_int(), C.c_float()
+    n = lib().osop_wr_extract(_p(w16, C.c_uint16), C.c_longlong(M), C.c_longlong(K), C.c_longlong(K), _p(c, C.c_float),
+                              C.byref(_fmt(fmt)), C.byref(_atom(a)), k_a, C.byref(_atom(b)) if b is not None else None, k_b,
+                              use_sign, int(select_metric), C.c_longlong(int(n_keep)), _p(row_start, C.c_uint), _p(records, C.c_uint),
+                              C.c_longlong(cap), C.byref(e), C.byref(tau), _p(resid, C.c_float) if want_resid else None)
+    out = dict(row_start=row_start, records=records[:min(n, cap)].copy(), count=int(n), scale_exp=e.value, tau=float(tau.value))
+    if want_resid:
+        out["resid"] = resid
+    return out

@@ -24,6 +24,8 @@
 //                                                       paragraph "HIF7/HIF8 hardware rationale"
 //   design axes (i)-(iv): partition metric, reassignment metric, Lloyd weighting, pool definition
 //                                                       paragraph "Pair-search design axes"
+//   outlier extraction before the search (OPQ) ........ Section "Outlier Per-Quantum Extraction (OPQ)"
+//   sparse correction of the residual (Wr) ............ Section "Sparse Residual Correction (Wr)"
 //
 // Where the paper is silent the reading taken is stated at the function that needs it.
 //
@@ -723,6 +725,130 @@ int osop_pack(const uint16_t* W, long long M, long long K, long long ldw, const 
               const Atom* a, int k_a, const Atom* b, int k_b, int use_sign, int container_bits, int word_sign_bits,
               unsigned char* codes, unsigned char* words, long long* n_sel1, long long* n_neg) {
   return osop_pack_axes(W, M, K, ldw, c, f, a, k_a, b, k_b, use_sign, container_bits, word_sign_bits, 0, codes, words, n_sel1, n_neg);
+}
+
+// ---------------------------------------------------------------------------------------------
+// OPQ (Section "Outlier Per-Quantum Extraction (OPQ)").
+// Threshold: the m with F_M(m) = (2 Phi(m) - 1)^M = q.  2 Phi(m) - 1 = erf(m / sqrt 2), so m solves
+// erf(m / sqrt 2) = q^(1/M); erf is increasing, bisection on [0, 16].
+// ---------------------------------------------------------------------------------------------
+double osop_opq_threshold(double q, int max_order) {
+  const double target = std::pow(q, 1.0 / (double)max_order);
+  double lo = 0.0, hi = 16.0;
+  for (int it = 0; it < 200; ++it) {
+    const double mid = 0.5 * (lo + hi);
+    if (std::erf(mid / std::sqrt(2.0)) < target) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+// Extraction.  Element i of block b is an outlier when |w_i| / sigma_b > m.  Readings (the paper does not
+// define sigma_b or the record layout beyond "16-bit element index + BF16 value"):
+//   sigma_b = sqrt(mean_j w_j^2) over the block's g = 16 elements (root mean square: weights are centred), so the
+//   test is w_i^2 g > m^2 sum_j w_j^2, taken in binary64: the squares of bf16 values are exact, the sum runs over
+//   j = 0..15 in order, one product m^2 * sum on the right.  A zero block has no outlier.
+//   W_out = W with the outliers set to +0 (the codebook input); an outlier keeps its exact bf16 value in the stream.
+//   Stream: records ascending by (row m, column k); record = k | bf16 bits << 16 (the 16-bit index is the column:
+//   K <= 65536); row_start[m] = first record of row m, row_start[M] = number of records.
+//   Records beyond `capacity` are counted, not written.  Returns the number of records.
+long long osop_opq_extract(const uint16_t* W, long long M, long long K, long long ldw, double m_thr,
+                           uint16_t* W_out, long long ldo, unsigned* row_start, unsigned* records, long long capacity) {
+  const long long nbk = K / G;
+  const double m2 = m_thr * m_thr;
+  long long n = 0;
+  for (long long m = 0; m < M; ++m) {
+    row_start[m] = (unsigned)n;
+    for (long long j = 0; j < nbk; ++j) {
+      double w[G], s2 = 0.0;
+      for (int i = 0; i < G; ++i) { w[i] = (double)bf16_to_float(W[m * ldw + j * G + i]); s2 = s2 + w[i] * w[i]; }
+      const double rhs = m2 * s2;
+      for (int i = 0; i < G; ++i) {
+        const long long k = j * G + i;
+        const uint16_t bits = W[m * ldw + k];
+        const bool out = w[i] * w[i] * (double)G > rhs;
+        W_out[m * ldo + k] = out ? (uint16_t)0 : bits;
+        if (out) {
+          if (n < capacity) records[n] = (unsigned)k | ((unsigned)bits << 16);
+          ++n;
+        }
+      }
+    }
+  }
+  row_start[M] = (unsigned)n;
+  return n;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Wr (Section "Sparse Residual Correction (Wr)").  E = W - W_hat for the reconstruction of the chosen codebook(s)
+// (per block the winner among a, (-a), b, (-b) exactly as the packer chooses it; W_hat = s_hat q, E_i = w_i - s_hat q_i
+// with one rounding, as the block error forms it).  The entries with the largest |E_mk| c_k are kept.  Readings:
+//   metric = |E| c_k as one binary32 product; "top sigma" is a rank n_keep given by the caller: tau = the n_keep-th
+//   largest metric of the layer, an entry is kept when metric >= tau (ties all in) and metric > 0 (a zero residual
+//   corrects nothing);
+//   values are E3M4 (sign, 3 exponent bits with bias 3 and the all-ones exponent left out, 4 mantissa bits: largest
+//   15.5) of E / 2^e with one exponent e per layer (the "header"): 2^e = the smallest power of two with
+//   max|E_kept| / 2^e <= 15.5; nearest, ties to the even magnitude number;
+//   stream as for OPQ: record = k | code << 16, ascending by (m, k), row_start[M + 1].
+// Returns the number of records; *scale_exp = e (0 when nothing is kept), *tau_out = tau.
+// ---------------------------------------------------------------------------------------------
+long long osop_wr_extract(const uint16_t* W, long long M, long long K, long long ldw, const float* c, const ScaleFmt* f,
+                          const Atom* a, int k_a, const Atom* b, int k_b, int use_sign, int select_metric, long long n_keep,
+                          unsigned* row_start, unsigned* records, long long capacity, int* scale_exp, float* tau_out,
+                          float* resid_out) {
+  const long long nbk = K / G;
+  float wmax = 0.0f;
+  for (long long m = 0; m < M; ++m)
+    for (long long i = 0; i < K; ++i) wmax = std::max(wmax, std::fabs(bf16_to_float(W[m * ldw + i])));
+  std::vector<float> E((size_t)(M * K)), metric((size_t)(M * K));
+  for (long long m = 0; m < M; ++m)
+    for (long long j = 0; j < nbk; ++j) {
+      float w[G];
+      load_block(W, ldw, m, j, w);
+      BlockEval bestr{};
+      int pick = -1;
+      for (int which = 0; which < (b ? 2 : 1); ++which) {
+        const Atom& base = which ? *b : *a;
+        for (int sg = 0; sg < (use_sign ? 2 : 1); ++sg) {
+          Atom cand = base;
+          if (sg) cand.negated = 1 - cand.negated;
+          const BlockEval r = eval_block(w, c + j * G, cand, *f, which ? k_b : k_a, layer_pot_scale(wmax, cand.tmax));
+          if (pick < 0 || (select_metric ? r.sse < bestr.sse : r.cos > bestr.cos)) { bestr = r; pick = which * 2 + sg; }
+        }
+      }
+      for (int i = 0; i < G; ++i) {
+        const long long at = m * K + j * G + i;
+        E[(size_t)at] = std::fmaf(-bestr.s_hat, bestr.q[i], w[i]);
+        metric[(size_t)at] = std::fabs(E[(size_t)at]) * c[j * G + i];
+        if (resid_out) resid_out[at] = E[(size_t)at];
+      }
+    }
+  std::vector<float> sorted(metric);
+  std::sort(sorted.begin(), sorted.end(), [](float x, float y) { return x > y; });
+  const float tau = sorted[(size_t)(n_keep - 1)];
+  float emax = 0.0f;
+  for (size_t i = 0; i < E.size(); ++i)
+    if (metric[i] >= tau && metric[i] > 0.0f) emax = std::max(emax, std::fabs(E[i]));
+  Atom e3m4{};
+  e3m4.n_bits = 8; e3m4.kind = KIND_FP_GRID; e3m4.scope = 0; e3m4.tmax = 15.5f; e3m4.grid_neg_max = 15.5f;
+  e3m4.grid_exp_bits = 3; e3m4.grid_man_bits = 4; e3m4.grid_bias = 3;
+  int e = 0;
+  if (emax > 0.0f) e = std::ilogb(layer_pot_scale(emax, 15.5f));
+  long long n = 0;
+  for (long long m = 0; m < M; ++m) {
+    row_start[m] = (unsigned)n;
+    for (long long k = 0; k < K; ++k) {
+      const size_t at = (size_t)(m * K + k);
+      if (!(metric[at] >= tau && metric[at] > 0.0f)) continue;
+      int code = 0;
+      grid_quantize(e3m4, std::ldexp(E[at], -e), &code);
+      if (n < capacity) records[n] = (unsigned)k | ((unsigned)code << 16);
+      ++n;
+    }
+  }
+  row_start[M] = (unsigned)n;
+  *scale_exp = e;
+  *tau_out = tau;
+  return n;
 }
 
 }  // extern "C"

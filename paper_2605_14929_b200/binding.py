@@ -265,7 +265,7 @@ def profile_enable(on: bool) -> None:
     _check(lib().sop_profile_enable(1 if on else 0), "sop_profile_enable")
 
 
-PROFILE_SWEEP, PROFILE_LLOYD, PROFILE_PACK, PROFILE_NORMS, PROFILE_REDUCE = 0, 1, 2, 3, 4
+PROFILE_SWEEP, PROFILE_LLOYD, PROFILE_PACK, PROFILE_NORMS, PROFILE_REDUCE, PROFILE_POOL, PROFILE_PREPASS = 0, 1, 2, 3, 4, 5, 6
 
 
 def profile_ms(which: int, back: int = 0) -> float:

@@ -1023,6 +1023,19 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   sop_dd4_lloyd_workspace(M, K, &need);
   if (!workspace_dev || ((uintptr_t)workspace_dev & 255u) || workspace_bytes < need) return SOP_ERR_WORKSPACE;
 
+  // entries of the table the dynamic programme builds: FMTa's; when FMTa is chosen on the device every table atom must
+  // agree on the number (decided here, before the first enqueue)
+  int ne = 0;
+  if (grid_dp) {
+    ne = fmta_index >= 0 ? atoms[fmta_index].n_entries : 0;
+    for (int i = 0; i < n_atoms && fmta_index < 0; ++i) {
+      if (atoms[i].kind != SOP_KIND_LUT) continue;
+      if (ne == 0) ne = atoms[i].n_entries;
+      else if (atoms[i].n_entries != ne) return SOP_ERR_ALPHABET;
+    }
+    if (ne < 2) return SOP_ERR_ALPHABET;
+  }
+
   unsigned char* wsb = (unsigned char*)workspace_dev;
   LloydArgs a;
   a.W = (const uint16_t*)W_dev; a.c = c_dev; a.cosrow_base = block_metric_dev;
@@ -1036,6 +1049,7 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
   LloydWs* ws = (LloydWs*)workspace_dev;
   cudaStream_t st = (cudaStream_t)stream;
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, offsetof(LloydWs, dp_cut), st));
+  if ((rc = profile_mark(SOP_PROFILE_POOL, 0, st))) return rc;
   const int sms = num_sms();
   long long sg = (NB + LTB * 8 - 1) / (LTB * 8);
   if (sg > sms * 4) sg = sms * 4;
@@ -1067,15 +1081,8 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     else pool_cache_kernel<false><<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
     SOP_CUDA_TRY(cudaGetLastError());
   }
+  if ((rc = profile_mark(SOP_PROFILE_POOL, 1, st))) return rc;
   if (grid_dp) {
-    // entries of the new table: FMTa's; when FMTa is chosen on the device every table atom must agree on the number
-    int ne = fmta_index >= 0 ? atoms[fmta_index].n_entries : 0;
-    for (int i = 0; i < n_atoms && fmta_index < 0; ++i) {
-      if (atoms[i].kind != SOP_KIND_LUT) continue;
-      if (ne == 0) ne = atoms[i].n_entries;
-      else if (atoms[i].n_entries != ne) return SOP_ERR_ALPHABET;
-    }
-    if (ne < 2) return SOP_ERR_ALPHABET;
     if ((rc = profile_mark(SOP_PROFILE_LLOYD, 0, st))) return rc;
     static_assert(sizeof(DpScratch) <= sizeof(((LloydWs*)nullptr)->dp_scratch), "scratch of the dynamic programme");
     DpScratch* dp = reinterpret_cast<DpScratch*>(ws->dp_scratch);

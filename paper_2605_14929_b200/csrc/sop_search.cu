@@ -1294,6 +1294,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   if (rgrid < 1) rgrid = 1;
 
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
+  if ((rc = profile_mark(SOP_PROFILE_PREPASS, 0, st))) return rc;
   if (!k_from_result) {
     // one read of W: block scales' exponent histogram, max|W|, then the shifts (last CTA)
     long long want = (L.NB + 255) / 256;
@@ -1301,6 +1302,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     prepass_kernel<<<pgrid, 256, 0, st>>>(L, P, F, hist, hdr);
     SOP_CUDA_TRY(cudaGetLastError());
   }
+  if ((rc = profile_mark(SOP_PROFILE_PREPASS, 1, st))) return rc;
   static bool attr_set = false;
   if (!attr_set) {
     SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
