@@ -207,13 +207,15 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
  *   SOP_PROFILE_LLOYD   the iteration kernel(s) of sop_dd4_lloyd, or the launches of its dynamic programme
  *   SOP_PROFILE_POOL    what sop_dd4_lloyd launches before them: radix select, set-up, pool list, pool cache
  *   SOP_PROFILE_PREPASS the shift prepass of sop_pair_search (the events coincide when the call takes its shifts from a result)
+ *   SOP_PROFILE_OPQ     the three kernels of sop_opq_extract
+ *   SOP_PROFILE_WR      the kernels of sop_wr_extract
  *   SOP_PROFILE_PACK    the kernel of sop_pack
  *   SOP_PROFILE_NORMS   both kernels of sop_channel_norms
  * sop_profile_ms waits for the second event of a call of that kind (back = 0: the last call, 1: the one
  * before, ... up to 7) and returns the time between its two events in milliseconds (SOP_ERR_RANGE if
  * no such call has run since profiling was enabled).  Not thread-safe. */
 enum { SOP_PROFILE_SWEEP = 0, SOP_PROFILE_LLOYD = 1, SOP_PROFILE_PACK = 2, SOP_PROFILE_NORMS = 3, SOP_PROFILE_REDUCE = 4, SOP_PROFILE_POOL = 5,
-       SOP_PROFILE_PREPASS = 6, SOP_PROFILE_KINDS = 7 };
+       SOP_PROFILE_PREPASS = 6, SOP_PROFILE_OPQ = 7, SOP_PROFILE_WR = 8, SOP_PROFILE_KINDS = 9 };
 int sop_profile_enable(int on);
 int sop_profile_ms(int which, int back, float* ms);
 int sop_profile_last_ms(int which, float* ms);    /* = sop_profile_ms(which, 0, ms) */
@@ -327,6 +329,63 @@ int sop_pack(const void* W_dev, long long M, long long K, long long ldw, const f
              unsigned dd_mask, int index_a, int index_b, int k_mode, const sop_search_result* search_dev,
              int use_sign, int container_bits, int word_sign_bits, unsigned char* codes_dev,
              unsigned char* words_dev, long long* counts_dev, const float* block_metric_dev, int flags, void* stream);
+
+/* ---- OPQ: outlier extraction before the search (Section "Outlier Per-Quantum Extraction (OPQ)") ----
+ * Positions with |w_i| / sigma_b > m are taken out of the codebook input and kept as exact bf16 values in a
+ * sparse stream.  sigma_b = sqrt(mean_j w_j^2) over the block's g = 16 elements (the paper names sigma_b
+ * without defining it), so the test is w_i^2 g > m^2 sum_j w_j^2; it is taken in binary64 (squares of bf16
+ * values are exact, the sum runs in element order, one product on the right), so the decision does not
+ * depend on the device.  A zero block has no outlier.
+ *
+ * sop_opq_threshold (host only): the m with F_M(m) = (2 Phi(m) - 1)^M = q, Phi the standard normal CDF,
+ * M = max_order (the paper's default: M = g = 16, q = 0.92).  q in (0, 1), max_order >= 1, else SOP_ERR_RANGE.
+ *
+ * sop_opq_extract:
+ *   W_dev [M x K] bf16, ldw as for sop_pair_search; m: the threshold, in (0, 1e6).
+ *   W_out_dev [M x K] bf16 with row stride ldo (16-byte aligned, ldo % 8 == 0, ldo >= K), overwritten: W with
+ *     every outlier replaced by +0; it is the input of the search that follows.  Must not be W_dev
+ *     (SOP_ERR_RANGE): the stream is read from the untouched input.
+ *   Stream: records ascend by (row, column); a record is the column k in bits 0-15 and the bf16 pattern of
+ *     the weight in bits 16-31 (32 bits per outlier, as the paper counts them), so K <= 65536 (SOP_ERR_SHAPE
+ *     beyond).  row_start_dev [M + 1] unsigned, overwritten: first record of every row, [M] = the number of
+ *     records.  records_dev [capacity] unsigned: records beyond `capacity` are counted but not written (compare
+ *     *count_dev with the capacity; M * K always suffices).  count_dev: one long long, overwritten.
+ *   workspace_dev: sop_opq_workspace bytes, 256-byte aligned.
+ * Inference applies the stream as Y[t, m] += sum over the row's records of value * X[t, k]; that step is
+ * outside this library. */
+int sop_opq_threshold(double q, int max_order, double* m_out);
+int sop_opq_workspace(long long M, long long K, size_t* bytes);
+int sop_opq_extract(const void* W_dev, long long M, long long K, long long ldw, int g, double m,
+                    void* W_out_dev, long long ldo, unsigned* row_start_dev, unsigned* records_dev, long long capacity,
+                    long long* count_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---- Wr: sparse correction of the codebook residual (Section "Sparse Residual Correction (Wr)") ----
+ * E = W - W_hat for the packed layer, the entries with the largest activation-weighted magnitude |E_mk| c_k
+ * are stored as a sparse stream with E3M4 values.  W_hat is decoded from the stream sop_pack wrote (scale
+ * word -> sign, selector, scale; codes -> table values), E_i = w_i - s_hat q_i with one rounding, the metric
+ * is the binary32 product |E_i| c_k.  The paper fixes neither ties nor the value scaling; here:
+ *   n_keep (in [1, M K], the "top sigma" as a rank, e.g. ceil(0.001 M K)): tau = the n_keep-th largest metric
+ *     of the layer; an entry is kept when its metric >= tau (ties all in) and > 0;
+ *   values: E3M4 = sign, 3 exponent bits (bias 3, the all-ones exponent left out), 4 mantissa bits, largest
+ *     15.5; the code is the nearest grid point (ties to the even magnitude number) of E / 2^e with one
+ *     exponent e per layer, the smallest e with max |E_kept| / 2^e <= 15.5 (the stream's header).
+ *   Arguments W_dev .. words_dev: exactly those given to sop_pack for this layer (codes_dev and words_dev now
+ *     inputs); with index_a = SOP_PAIR_FROM_RESULT and a result without a pair nothing was packed: no record
+ *     is written and *count_dev = -1.
+ *   Stream: as for sop_opq_extract, a record is the column k in bits 0-15 and the E3M4 code in bits 16-23;
+ *     row_start_dev [M + 1], records_dev [capacity], count_dev as there.  scale_exp_dev: one int, e (0 when
+ *     nothing is kept).  tau_dev (may be NULL): one float, tau.
+ *   workspace_dev: sop_wr_workspace bytes, 256-byte aligned.
+ * The residual is recomputed in each of the five passes (three selection passes, count, write) rather than
+ * stored: W, codes and scale words are 2.6 bytes per element, a stored residual 4. */
+int sop_wr_workspace(long long M, long long K, size_t* bytes);
+int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
+                   const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev, unsigned dd_mask,
+                   int index_a, int index_b, int k_mode, const sop_search_result* search_dev, int use_sign,
+                   int container_bits, int word_sign_bits, const unsigned char* codes_dev, const unsigned char* words_dev,
+                   long long n_keep, unsigned* row_start_dev, unsigned* records_dev, long long capacity,
+                   long long* count_dev, int* scale_exp_dev, float* tau_dev, void* workspace_dev, size_t workspace_bytes,
+                   void* stream);
 
 #ifdef __cplusplus
 }

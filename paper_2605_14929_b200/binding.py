@@ -84,7 +84,8 @@ def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
             "sop_channel_norms_static",
             "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd_tuning",
-            "sop_dd4_lloyd", "sop_pack",
+            "sop_dd4_lloyd", "sop_pack", "sop_opq_threshold", "sop_opq_workspace", "sop_opq_extract", "sop_wr_workspace",
+            "sop_wr_extract",
             "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
 
 
@@ -261,11 +262,58 @@ def sop_pack(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes: torc
                           _ptr(counts), _ptr(block_cos), PACK_SELECT_MSE if select_mse else 0, _stream(stream)), "sop_pack")
 
 
+def opq_threshold(q: float = 0.92, max_order: int = 16) -> float:
+    """The m with (2 Phi(m) - 1)^max_order = q."""
+    m = C.c_double()
+    _check(lib().sop_opq_threshold(C.c_double(q), int(max_order), C.byref(m)), "sop_opq_threshold")
+    return m.value
+
+
+def opq_workspace(M: int, K: int, device) -> torch.Tensor:
+    n = C.c_size_t()
+    _check(lib().sop_opq_workspace(_ll(M), _ll(K), C.byref(n)), "sop_opq_workspace")
+    return torch.empty(n.value, dtype=torch.uint8, device=device)
+
+
+def sop_opq_extract(W: torch.Tensor, m: float, W_out: torch.Tensor, row_start: torch.Tensor, records: Optional[torch.Tensor],
+                    count: torch.Tensor, workspace: torch.Tensor, stream=None, g: int = 16) -> None:
+    """``row_start``: M + 1 int32/uint32 words, ``records``: the capacity in 32-bit words (None: count only),
+    ``count``: one int64."""
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1 and W_out.stride(1) == 1
+    M, K = W.shape
+    _check(lib().sop_opq_extract(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), g, C.c_double(m), _ptr(W_out), _ll(W_out.stride(0)),
+                                 _ptr(row_start), _ptr(records), _ll(0 if records is None else records.numel()), _ptr(count),
+                                 _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)), "sop_opq_extract")
+
+
+def wr_workspace(M: int, K: int, device) -> torch.Tensor:
+    n = C.c_size_t()
+    _check(lib().sop_wr_workspace(_ll(M), _ll(K), C.byref(n)), "sop_wr_workspace")
+    return torch.empty(n.value, dtype=torch.uint8, device=device)
+
+
+def sop_wr_extract(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes: torch.Tensor, words: torch.Tensor, n_keep: int,
+                   row_start: torch.Tensor, records: Optional[torch.Tensor], count: torch.Tensor, scale_exp: torch.Tensor,
+                   workspace: torch.Tensor, tau: Optional[torch.Tensor] = None,
+                   index_a: int = PAIR_FROM_RESULT, index_b: int = PAIR_FROM_RESULT, k_mode: int = K_FROM_RESULT,
+                   search_result: Optional[torch.Tensor] = None, use_sign: int = 0, container_bits: int = 8,
+                   word_sign_bits: int = 0, dd_lut: Optional[torch.Tensor] = None, dd_mask: int = 0, stream=None, g: int = 16) -> None:
+    """The arguments from ``fmt`` to ``word_sign_bits`` are those given to ``sop_pack`` for this layer."""
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
+    M, K = W.shape
+    _check(lib().sop_wr_extract(_ptr(W), _ll(M), _ll(K), _ll(W.stride(0)), _ptr(c), g, C.byref(make_fmt(fmt)), make_atoms(atoms),
+                                len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), index_a, index_b, k_mode, _ptr(search_result), use_sign,
+                                container_bits, word_sign_bits, _ptr(codes), _ptr(words), _ll(n_keep), _ptr(row_start),
+                                _ptr(records), _ll(0 if records is None else records.numel()), _ptr(count), _ptr(scale_exp),
+                                _ptr(tau), _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)), "sop_wr_extract")
+
+
 def profile_enable(on: bool) -> None:
     _check(lib().sop_profile_enable(1 if on else 0), "sop_profile_enable")
 
 
 PROFILE_SWEEP, PROFILE_LLOYD, PROFILE_PACK, PROFILE_NORMS, PROFILE_REDUCE, PROFILE_POOL, PROFILE_PREPASS = 0, 1, 2, 3, 4, 5, 6
+PROFILE_OPQ, PROFILE_WR = 7, 8
 
 
 def profile_ms(which: int, back: int = 0) -> float:

@@ -168,3 +168,37 @@ def test_lloyd_tuning_ranges(lib):
     assert lib.sop_dd4_lloyd_tuning(128, 0, 0, 0) == -7 and lib.sop_dd4_lloyd_tuning(128, 0, 5, 0) == -7
     assert lib.sop_dd4_lloyd_tuning(1, 2, 1, 3) == 0
     assert lib.sop_dd4_lloyd_tuning(128, 0, 4, 0) == 0      # the defaults again
+
+
+def test_sparse_stream_entry_points_reject_bad_arguments(lib):
+    ll = C.c_longlong
+    m = C.c_double()
+    assert lib.sop_opq_threshold(C.c_double(0.92), 16, C.byref(m)) == 0 and 2.79 < m.value < 2.80
+    assert lib.sop_opq_threshold(C.c_double(0.92), 16, None) == -1
+    assert lib.sop_opq_threshold(C.c_double(1.0), 16, C.byref(m)) == -7 and lib.sop_opq_threshold(C.c_double(0.5), 0, C.byref(m)) == -7
+    n = C.c_size_t()
+    assert lib.sop_opq_workspace(ll(4), ll(60), C.byref(n)) == -2 and lib.sop_wr_workspace(ll(0), ll(64), C.byref(n)) == -2
+    assert lib.sop_opq_workspace(ll(4), ll(64), C.byref(n)) == 0 and n.value >= 4 * 4 * 2
+    OUT = C.c_void_p(0x20000)
+
+    def opq(W=FAKE, out=OUT, K=64, ldo=64, thr=2.8, cap=16, rec=FAKE, ws=FAKE, wsb=1 << 20, cnt=FAKE):
+        return lib.sop_opq_extract(W, ll(4), ll(K), ll(K), 16, C.c_double(thr), out, ll(ldo), FAKE, rec, ll(cap), cnt, ws, C.c_size_t(wsb), None)
+    assert opq(W=None) == -1 and opq(cnt=None) == -1 and opq(rec=None) == -1
+    assert opq(out=FAKE) == -7                       # in place: the stream is read from the untouched input
+    assert opq(thr=0.0) == -7 and opq(thr=float("nan")) == -7
+    assert opq(ldo=60) == -2 and opq(K=65552) == -2  # the record holds the column in 16 bits
+    assert opq(wsb=64) == -5 and opq(ws=None) == -5
+    assert opq(cap=-1) == -1
+
+    fmt = C.byref(B.make_fmt(I.scale_format("UE4M4")))
+    atoms = I.alphabet(["NF4", "SH4"])
+    arr = B.make_atoms(atoms)
+
+    def wr(ia=0, ib=2, k=0, sign=0, b=12, wsb=0, res=None, keep=3, cap=8, rec=FAKE, exp=FAKE, ws=FAKE, wbytes=1 << 20):
+        return lib.sop_wr_extract(FAKE, ll(4), ll(64), ll(64), FAKE, 16, fmt, arr, len(atoms), None, C.c_uint(0), ia, ib, k, res, sign, b, wsb,
+                                  FAKE, FAKE, ll(keep), FAKE, rec, ll(cap), FAKE, exp, None, ws, C.c_size_t(wbytes), None)
+    assert wr(keep=0) == -7 and wr(keep=4 * 64 + 1) == -7
+    assert wr(b=8) == -3 and wr(sign=1, wsb=0) == -3
+    assert wr(ia=5) == -7 and wr(ia=B.PAIR_FROM_RESULT) == -1 and wr(k=B.K_FROM_RESULT) == -1
+    assert wr(exp=None) == -1 and wr(rec=None) == -1
+    assert wr(wbytes=16) == -5

@@ -1,0 +1,171 @@
+"""GPU parity of the two sparse side streams against the oracle: outlier extraction before the search (Section
+"Outlier Per-Quantum Extraction (OPQ)") and the sparse correction of the codebook residual (Section "Sparse
+Residual Correction (Wr)").  Everything is integer or bit work: W_out, row starts, records, counts, the layer
+exponent and the threshold are compared exactly."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_14929_b200 import binding as B
+from paper_2605_14929_b200 import inputs as I
+from paper_2605_14929_b200.pipeline import LayerSweep
+
+from . import oracle_pipeline
+from .test_gpu_parity import dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_opq(W: torch.Tensor, m: float, capacity=None, ldw=None):
+    M, K = W.shape
+    d = dev()
+    if ldw:
+        buf = torch.zeros(M, ldw, dtype=torch.bfloat16, device=d)
+        buf[:, :K] = W.to(d)
+        Wd = buf[:, :K]
+        out = torch.full((M, ldw), 7.0, dtype=torch.bfloat16, device=d)[:, :K]
+    else:
+        Wd = W.to(d)
+        out = torch.full((M, K), 7.0, dtype=torch.bfloat16, device=d)
+    cap = M * K if capacity is None else capacity
+    row_start = torch.zeros(M + 1, dtype=torch.int32, device=d)
+    records = torch.zeros(max(cap, 1), dtype=torch.int32, device=d) if cap else None
+    count = torch.zeros(1, dtype=torch.int64, device=d)
+    ws = B.opq_workspace(M, K, d)
+    B.sop_opq_extract(Wd, m, out, row_start, records, count, ws)
+    torch.cuda.synchronize()
+    n = int(count.item())
+    rec = records.cpu().numpy().view(np.uint32)[:min(n, cap)] if cap else np.zeros(0, np.uint32)
+    return dict(W_out=out.contiguous().cpu().view(torch.int16).numpy().view(np.uint16), row_start=row_start.cpu().numpy().view(np.uint32),
+                records=rec, count=n)
+
+
+def assert_opq(got, want):
+    assert got["count"] == want["count"]
+    assert np.array_equal(got["row_start"], want["row_start"])
+    assert np.array_equal(got["records"], want["records"])
+    assert np.array_equal(got["W_out"], want["W_out"])
+
+
+@pytest.mark.parametrize("M,K,ldw", [(8, 64, None), (37, 1040, None), (300, 4096, None), (19, 208, 256), (1, 16, None)])
+@pytest.mark.parametrize("q", [0.92, 0.5])
+def test_opq_matches_oracle(M, K, ldw, q):
+    L = I.laplace_outlier_layer(7, 1, M, K, 8)
+    m = B.opq_threshold(q, 16)
+    assert m == pytest.approx(oracle.opq_threshold(q, 16), rel=1e-12)
+    got = run_opq(L.W, m, ldw=ldw)
+    want = oracle.opq_extract(L.W, m)
+    assert q > 0.9 or want["count"] > M * K // 100          # the lower quantile takes a real share
+    assert_opq(got, want)
+
+
+def test_opq_edge_cases():
+    m = B.opq_threshold(0.92, 16)
+    # zero layer, constant-magnitude layer: no outliers, W_out = W
+    for W in (torch.zeros(5, 48, dtype=torch.bfloat16), torch.full((5, 48), -0.5, dtype=torch.bfloat16)):
+        got = run_opq(W, m)
+        assert got["count"] == 0 and not got["row_start"].any()
+        assert np.array_equal(got["W_out"], W.view(torch.int16).numpy().view(np.uint16))
+    # a capacity below the count: the count is reported, the records that fit are written, W_out is complete
+    L = I.laplace_outlier_layer(3, 0, 64, 512, 8)
+    want = oracle.opq_extract(L.W, 2.0)
+    assert want["count"] > 40
+    got = run_opq(L.W, 2.0, capacity=40)
+    assert got["count"] == want["count"] and np.array_equal(got["records"], want["records"][:40]) and np.array_equal(got["W_out"], want["W_out"])
+    got = run_opq(L.W, 2.0, capacity=0)
+    assert got["count"] == want["count"] and np.array_equal(got["row_start"], want["row_start"])
+    # an outlier in every block of a row, in the last column of the last row
+    W = torch.ones(3, 64, dtype=torch.float32) * 0.01
+    W[1, 5::16] = 3.0
+    W[2, 63] = -2.0
+    Wb = W.to(torch.bfloat16)
+    assert_opq(run_opq(Wb, m), oracle.opq_extract(Wb, m))
+
+
+def run_wr(L, fmt, rom, n_keep, use_sign, lloyd_iters=0, capacity=None, single=False):
+    """The layer through the pipeline (search, pack), then the correction of what was packed."""
+    d = dev()
+    M, K = L.W.shape
+    sw = LayerSweep(M, K, L.X.shape[0], fmt, rom, [], lloyd_iters, device=d)
+    Wd, Xd = L.W.to(d), L.X.to(d)
+    sw.run(Wd, Xd)
+    out = sw.outputs()
+    cap = M * K if capacity is None else capacity
+    row_start = torch.zeros(M + 1, dtype=torch.int32, device=d)
+    records = torch.zeros(max(cap, 1), dtype=torch.int32, device=d)
+    count = torch.zeros(1, dtype=torch.int64, device=d)
+    e = torch.zeros(1, dtype=torch.int32, device=d)
+    tau = torch.zeros(1, dtype=torch.float32, device=d)
+    ws = B.wr_workspace(M, K, d)
+    B.sop_wr_extract(Wd, sw.c, sw.fmt_c, sw.atoms_c, sw.codes, sw._words_store, n_keep, row_start, records, count, e, ws, tau=tau,
+                     search_result=sw.result, use_sign=sw.use_sign, container_bits=sw.container, word_sign_bits=sw.use_sign,
+                     dd_lut=sw.dd_lut if sw.dd_mask else None, dd_mask=sw.dd_mask)
+    torch.cuda.synchronize()
+    n = int(count.item())
+    got = dict(count=n, row_start=row_start.cpu().numpy().view(np.uint32), records=records.cpu().numpy().view(np.uint32)[:min(n, cap)],
+               scale_exp=int(e.item()), tau=float(tau.item()))
+    return sw, out, got
+
+
+def oracle_wr(L, fmt, out, sw, n_keep):
+    best = out.result["best"]
+    ia, ib = (int(best[3]), int(best[4])) if sw.use_sign else (int(best[0]), int(best[1]))
+    atoms = list(out.atoms)
+    dd = out.dd_lut[:16]
+
+    def atom(i):
+        a = atoms[i]
+        if (sw.dd_mask >> i) & 1:
+            a = I.Atom(a.name, a.n_bits, I.KIND_LUT, a.negated, I.SCOPE_BLOCK, 1.0, dd)
+        return a
+    c = out.c.numpy()
+    return oracle.wr_extract(L.W, c, fmt, atom(ia), int(out.result["k"][ia]), atom(ib), int(out.result["k"][ib]),
+                             use_sign=sw.use_sign, n_keep=n_keep)
+
+
+@pytest.mark.parametrize("fmt_name,rows,K,iters", [("E5M6", 24, 512, 4), ("UE4M4", 40, 256, 0), ("S1E5M5", 9, 1024, 2), ("E4M3", 64, 128, 0)])
+def test_wr_matches_oracle_on_the_packed_layer(fmt_name, rows, K, iters):
+    L = I.student_layer(11, 2, rows, K, 64, 4.0)
+    fmt = I.scale_format(fmt_name)
+    for n_keep in (1, max(1, math.ceil(0.001 * rows * K)), rows * K // 50):
+        sw, out, got = run_wr(L, fmt, ["NF4", "SH4", "BOF4"], n_keep, None, lloyd_iters=iters)
+        want = oracle_wr(L, fmt, out, sw, n_keep)
+        assert want["count"] >= n_keep
+        assert got["count"] == want["count"] and got["scale_exp"] == want["scale_exp"]
+        assert np.float32(got["tau"]).view(np.uint32) == np.float32(want["tau"]).view(np.uint32)
+        assert np.array_equal(got["row_start"], want["row_start"])
+        assert np.array_equal(got["records"], want["records"])
+
+
+def test_wr_edge_cases():
+    fmt = I.scale_format("E5M6")
+    L = I.student_layer(5, 0, 16, 256, 64, 5.0)
+    # every element asked for: everything with a residual is kept
+    sw, out, got = run_wr(L, fmt, ["NF4", "SH4"], 16 * 256, None)
+    want = oracle_wr(L, fmt, out, sw, 16 * 256)
+    assert got["count"] == want["count"] <= 16 * 256 and np.array_equal(got["records"], want["records"])
+    # a capacity below the count
+    sw, out, got = run_wr(L, fmt, ["NF4", "SH4"], 100, None, capacity=10)
+    want = oracle_wr(L, fmt, out, sw, 100)
+    assert got["count"] == want["count"] >= 100 and np.array_equal(got["records"], want["records"][:10])
+    assert np.array_equal(got["row_start"], want["row_start"])
+
+
+def test_opq_then_search_then_wr_chain():
+    """The three steps as the paper orders them: outliers out, the search on the rest, the correction of its residual."""
+    L = I.laplace_outlier_layer(9, 0, 48, 512, 64)
+    m = B.opq_threshold(0.92, 16)
+    o = run_opq(L.W, m)
+    assert o["count"] > 0
+    W2 = torch.from_numpy(o["W_out"].view(np.int16).copy()).view(torch.bfloat16)
+    L2 = I.Layer(W2, L.X)
+    fmt = I.scale_format("E5M6")
+    n_keep = math.ceil(0.001 * 48 * 512)
+    sw, out, got = run_wr(L2, fmt, ["NF4", "SH4", "BOF4", "Split87"], n_keep, None, lloyd_iters=4)
+    want = oracle_wr(L2, fmt, out, sw, n_keep)
+    assert got["count"] == want["count"] and np.array_equal(got["records"], want["records"]) and got["scale_exp"] == want["scale_exp"]
+    # an outlier position holds +0 in the search input: its residual is minus the table value nearest to zero, times the scale
+    assert np.array_equal(o["W_out"], oracle.opq_extract(L.W, m)["W_out"])
