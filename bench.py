@@ -279,6 +279,50 @@ def per_config_table(dev, alu_peak, flush):
     return out
 
 
+def sparse_streams_table(dev, hbm_peak, of, flush):
+    """The two sparse side streams (outlier extraction before the search, correction of the packed residual after it)
+    on the 8192x8192 layer at E5M6: time of each by the library's events, record counts, algorithmic bytes and the
+    fraction of the HBM peak they amount to.  They are off in the headline workload."""
+    import torch
+    from paper_2605_14929_b200 import binding as B, inputs as I
+    from paper_2605_14929_b200.pipeline import LayerSweep
+    L = I.config5_layer(0, 0, 0, device=str(dev))
+    M, K = L.W.shape
+    sw = LayerSweep(M, K, L.X.shape[0], I.scale_format("E5M6"), ROM4, [], 8, device=dev, opq_q=0.92, wr_sigma=0.001)
+    for _ in range(2):
+        sw.run(L.W, L.X)
+    torch.cuda.synchronize(dev)
+    B.profile_enable(True)
+    t_opq, t_wr, t_all = [], [], []
+    for _ in range(5):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sw.run(L.W, L.X)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        t_opq.append(B.profile_ms(B.PROFILE_OPQ, 0)); t_wr.append(B.profile_ms(B.PROFILE_WR, 0)); t_all.append(e0.elapsed_time(e1))
+    B.profile_enable(False)
+    sp = sw.sparse_outputs()
+    sw.outputs()                                   # raises if the Lloyd call of the pass did not finish
+    E = M * K
+    opq_ms, wr_ms, all_ms = sorted(t_opq)[2], sorted(t_wr)[2], sorted(t_all)[2]
+    opq_bytes = (2.0 + 2.0 + 2 * 2.0 / 16.0) * E + 4.0 * sp["opq"]["count"]
+    wr_bytes = 6 * (2.0 + 0.5 + sw.container / 8.0 / 16.0) * E + 4.0 * sp["wr"]["count"]
+
+    def hbm(b, ms):
+        return dict(achieved=b / (ms * 1e-3) / 1e9, peak=hbm_peak, unit="GB/s", frac=b / (ms * 1e-3) / 1e9 / hbm_peak, of=of)
+    return dict(workload="8192x8192 at E5M6, ROM4 + DD4, outlier quantile 0.92, correction sparsity 0.001", elements=E,
+                opq=dict(ms=opq_ms, records=sp["opq"]["count"], rate=sp["opq"]["count"] / E, threshold_m=sp["opq"]["m"],
+                         bpw=32.0 * sp["opq"]["count"] / E, algorithmic_bytes=opq_bytes, hbm=hbm(opq_bytes, opq_ms),
+                         note="three launches: mask + zeroed copy (W read once, written once), scan of the tile counts, records"),
+                wr=dict(ms=wr_ms, records=sp["wr"]["count"], n_keep=sp["wr"]["n_keep"], scale_exp=sp["wr"]["scale_exp"],
+                        bpw=32.0 * sp["wr"]["count"] / E, algorithmic_bytes=wr_bytes, hbm=hbm(wr_bytes, wr_ms),
+                        note="eleven launches: block-maximum pass, three selection passes, count, scan, write; every pass decodes W, codes and scale "
+                             "words (2.6 bytes per element) instead of reading a stored residual"),
+                whole_path_ms=all_ms, whole_path_value=E / all_ms / 1e6)
+
+
 # ---------------------------------------------------------------------------------------------------------
 # N > 1 bookkeeping (no data-path collective: the ranks only agree on the slowest time)
 # ---------------------------------------------------------------------------------------------------------
@@ -510,7 +554,11 @@ def run_gpu(args) -> None:
                                          sweep_only=dict(value=units / (search_t * 1e3) / 1e6, unit=UNIT, ms=search_t * 1e3),
                                          ops_per_element_n_step=ops_n_step, frac_of_alu_peak=ach / alu_peak,
                                          note="the headline workload: block 0, five layers, eight scale formats")
-        cpu_rows = 384
+        try:
+            sparse = sparse_streams_table(dev, hbm_peak, of, flush) if world == 1 else None
+        except Exception as exc:
+            sparse = dict(error=repr(exc))
+        cpu_rows = 1536
         cpu_val, cpu_dt = cpu_oracle_time(cpu_rows)
         line = dict(
             metric=METRIC, value=job_value, unit=UNIT, n_gpus=world, steps=args.steps,
@@ -531,7 +579,7 @@ def run_gpu(args) -> None:
             sweep_only=dict(value=world * units / search_t / 1e9, unit=UNIT,
                             note="element-formats / time of the search launches of a step (every candidate, every pair: evaluation "
                                  "and reduction kernels)"),
-            roofline=roofline, per_config=per_config,
+            roofline=roofline, per_config=per_config, sparse_streams=sparse,
             cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=1, kind="oracle",
                               sample=f"first {cpu_rows} of 8192 rows of the 8192x8192 layer at E5M6 (one layer, one format), whole "
                                      f"pipeline, {cpu_dt:.1f} s"),

@@ -14,7 +14,11 @@
 //   opq_write_kernel    reads the masks, and W only where a mask is set: records (column | bf16 bits << 16)
 //   wr_hist_kernel<P>   decodes the packed stream (scale word -> s_hat, codes -> table values), forms the residual
 //                       E = w - s_hat q (one rounding) and the metric |E| c_k, histograms 11 / 11 / 10 bits of the
-//                       inverted metric bits (three-pass radix select of the n_keep-th largest metric)
+//                       inverted metric bits (three-pass radix select of the n_keep-th largest metric).  Pass -1 goes
+//                       first and histograms one value per block, the block's largest metric: at least n_keep
+//                       elements are as large as the n_keep-th largest block maximum, so the threshold lies in that
+//                       value's bin or an earlier one and pass 0 skips every element of a later bin (all but a few
+//                       per cent: shared-memory atomics on a handful of hot bins would otherwise dominate)
 //   wr_pick_kernel      after each pass: the bin that holds the rank, the prefix for the next pass
 //   wr_count_kernel     per-tile counts of kept entries (metric >= tau, metric > 0), max |E| over them
 //   wr_write_kernel     E3M4 codes of E / 2^e, records (column | code << 16)
@@ -32,6 +36,8 @@ int num_sms();
 
 struct SparseWs {
   unsigned hist[3][2048];
+  unsigned hist_bm[2048];         // histogram of the per-block maxima of the metric (top 11 bits of the inverted key)
+  unsigned bm_bin;                // bin of the n_keep-th largest block maximum: the threshold cannot lie in a later bin
   unsigned prefix;                // inverted-key prefix fixed by the selection passes so far
   unsigned tau_bits;              // the threshold metric as fp32 bits (a NaN pattern: nothing is kept)
   unsigned long long rank;        // rank still to find among the keys with that prefix
@@ -131,7 +137,7 @@ __global__ void __launch_bounds__(STB) opq_mask_kernel(OpqArgs a) {
     const long long blk = tile * STB + tid;
     unsigned mask = 0;
     if (blk < a.NB) {
-      const long long m = blk / a.nbk, j = blk - m * a.nbk;
+      const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
       const uint4* p = reinterpret_cast<const uint4*>(a.W + m * a.ldw + j * SOP_G);
       const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
       uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -175,7 +181,7 @@ __global__ void __launch_bounds__(STB) opq_write_kernel(OpqArgs a) {
     const unsigned excl = cta_excl_scan((unsigned)__popc(mask), s_warp, &tot);
     if (blk >= a.NB) continue;
     unsigned pos = a.tile_sums[tile] + excl;
-    const long long m = blk / a.nbk, j = blk - m * a.nbk;
+    const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
     if (j == 0) a.row_start[m] = pos;
     if (mask) {
       const uint16_t* p = a.W + m * a.ldw + j * SOP_G;
@@ -327,13 +333,19 @@ __device__ __forceinline__ void wr_block(const WrArgs& a, const FmtDev& F, const
     const float4 v = __ldg(cq + q);
     c[4 * q] = v.x; c[4 * q + 1] = v.y; c[4 * q + 2] = v.z; c[4 * q + 3] = v.w;
   }
+  const uint32_t lo32[2] = {(uint32_t)lo, (uint32_t)(lo >> 32)};
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const int pos = i * n;
-    unsigned long long v;
-    if (pos < 64) { v = lo >> pos; if (pos + n > 64) v |= hi << (64 - pos); }
-    else v = hi >> (pos - 64);
-    const uint32_t code = (uint32_t)v & emask;
+    uint32_t code;
+    if (n == 4) {                     // the common width: 32-bit shifts by constants
+      code = (lo32[i >> 3] >> (4 * (i & 7))) & 15u;
+    } else {
+      const int pos = i * n;
+      unsigned long long v;
+      if (pos < 64) { v = lo >> pos; if (pos + n > 64) v |= hi << (64 - pos); }
+      else v = hi >> (pos - 64);
+      code = (uint32_t)v & emask;
+    }
     float q;
     if (cd.kind == SOP_KIND_LUT) { q = sh.lutv[sel][code & 31u]; q = neg ? -q : q; }
     else q = fp_grid_decode(code, cd.sign_pos, cd.y, cd.bias);
@@ -359,47 +371,58 @@ __global__ void __launch_bounds__(STB) wr_hist_kernel(WrArgs a, AtomsDev A, FmtD
   if (tid == 0) wr_setup(a, A, res, sh);
   __syncthreads();
   if (sh.no_pair) return;
-  const unsigned prefix = PASS ? ws->prefix : 0u;
+  const unsigned prefix = PASS > 0 ? ws->prefix : 0u;
+  const unsigned bm_bin = PASS == 0 ? ws->bm_bin : 2047u;
   const long long n_tiles = (a.NB + STB - 1) / STB;
   for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const long long blk = tile * STB + tid;
     if (blk >= a.NB) continue;
-    const long long m = blk / a.nbk, j = blk - m * a.nbk;
+    const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
     float E[16], met[16];
     wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+    if constexpr (PASS < 0) {
+      float bm = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const unsigned key = wr_key(met[i]);
-      if (PASS == 0) {
-        // most elements share a handful of bins: one addition per distinct bin of the warp
-        const unsigned bin = key >> 21;
-        const unsigned same = __match_any_sync(__activemask(), bin);
-        if ((__ffs((int)same) - 1) == (tid & 31)) atomicAdd(&hist[bin], (unsigned)__popc(same));
-      } else if (PASS == 1) {
-        if ((key >> 21) == prefix) atomicAdd(&hist[(key >> 10) & 2047u], 1u);
-      } else {
-        if ((key >> 10) == prefix) atomicAdd(&hist[key & 1023u], 1u);
+      for (int i = 0; i < 16; ++i) bm = fmaxf(bm, met[i]);             // fmaxf drops a NaN
+      // most blocks share a handful of bins: one addition per distinct bin of the warp
+      const unsigned bin = wr_key(bm) >> 21;
+      const unsigned same = __match_any_sync(__activemask(), bin);
+      if ((__ffs((int)same) - 1) == (tid & 31)) atomicAdd(&hist[bin], (unsigned)__popc(same));
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const unsigned key = wr_key(met[i]);
+        if (PASS == 0) {
+          if ((key >> 21) <= bm_bin) atomicAdd(&hist[key >> 21], 1u);
+        } else if (PASS == 1) {
+          if ((key >> 21) == prefix) atomicAdd(&hist[(key >> 10) & 2047u], 1u);
+        } else {
+          if ((key >> 10) == prefix) atomicAdd(&hist[key & 1023u], 1u);
+        }
       }
     }
   }
   __syncthreads();
+  unsigned* out = PASS < 0 ? ws->hist_bm : ws->hist[PASS < 0 ? 0 : PASS];
   for (int i = tid; i < 2048; i += STB)
-    if (hist[i]) atomicAdd(&ws->hist[PASS][i], hist[i]);
+    if (hist[i]) atomicAdd(&out[i], hist[i]);
 }
 
 // One CTA after each histogram pass: the bin that holds the rank, the prefix and the rank inside it for the next
-// pass; after the last pass the threshold itself.  A rank beyond the histogram's total (no pair to correct, so the
-// histogram is empty) leaves a NaN threshold: nothing compares >= to it.
+// pass; after the last pass the threshold itself.  Pass -1: the bin of the n_keep-th largest block maximum.  A rank
+// beyond the histogram's total (no pair to correct, so the histogram is empty) leaves a NaN threshold: nothing
+// compares >= to it.
 __global__ void __launch_bounds__(1024) wr_pick_kernel(SparseWs* __restrict__ ws, int pass, long long n_keep) {
   __shared__ unsigned long long s_warp[32];
   __shared__ int s_bin;
   __shared__ unsigned long long s_before;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nb = pass < 2 ? 2048 : 1024;
-  const unsigned long long rank = pass == 0 ? (unsigned long long)n_keep : ws->rank;
+  const unsigned long long rank = pass <= 0 ? (unsigned long long)n_keep : ws->rank;
   if (tid == 0) { s_bin = -1; s_before = 0; }
   const int b0 = 2 * tid;
-  const unsigned long long c0 = b0 < nb ? ws->hist[pass][b0] : 0ull, c1 = b0 + 1 < nb ? ws->hist[pass][b0 + 1] : 0ull;
+  const unsigned* h = pass < 0 ? ws->hist_bm : ws->hist[pass];
+  const unsigned long long c0 = b0 < nb ? h[b0] : 0ull, c1 = b0 + 1 < nb ? h[b0 + 1] : 0ull;
   const unsigned long long local = c0 + c1;
   unsigned long long incl = local;
 #pragma unroll
@@ -417,7 +440,10 @@ __global__ void __launch_bounds__(1024) wr_pick_kernel(SparseWs* __restrict__ ws
     else { s_bin = b0 + 1; s_before = excl + c0; }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && pass < 0) {
+    // fewer blocks than entries to keep: no bound, every bin counts
+    ws->bm_bin = s_bin < 0 ? 2047u : (unsigned)s_bin;
+  } else if (tid == 0) {
     const unsigned prev = pass ? ws->prefix : 0u;
     if (s_bin < 0) {
       ws->prefix = 0xFFFFFFFFu; ws->rank = 0; ws->tau_bits = 0x7FC00000u;
@@ -449,7 +475,7 @@ __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, Fmt
     const long long blk = tile * STB + tid;
     unsigned cnt = 0;
     if (blk < a.NB && !sh.no_pair) {
-      const long long m = blk / a.nbk, j = blk - m * a.nbk;
+      const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
       float E[16], met[16];
       wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
 #pragma unroll
@@ -490,13 +516,13 @@ __global__ void __launch_bounds__(STB) wr_write_kernel(WrArgs a, AtomsDev A, Fmt
     unsigned keep = 0;
     long long m = 0, j = 0;
     if (blk < a.NB && !sh.no_pair) {
-      m = blk / a.nbk; j = blk - m * a.nbk;
+      m = (long long)((unsigned)blk / (unsigned)a.nbk); j = blk - m * a.nbk;
       wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
 #pragma unroll
       for (int i = 0; i < 16; ++i)
         if (wr_kept(met[i], tau)) keep |= 1u << i;
     } else if (blk < a.NB) {
-      m = blk / a.nbk; j = blk - m * a.nbk;
+      m = (long long)((unsigned)blk / (unsigned)a.nbk); j = blk - m * a.nbk;
     }
     unsigned tot;
     const unsigned excl = cta_excl_scan((unsigned)__popc(keep), s_warp, &tot);
@@ -649,6 +675,8 @@ int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, c
   const int grid = (int)(n_tiles < cap ? n_tiles : cap);
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(SparseWs), st));
   if ((rc = profile_mark(SOP_PROFILE_WR, 0, st))) return rc;
+  wr_hist_kernel<-1><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
+  wr_pick_kernel<<<1, 1024, 0, st>>>(ws, -1, n_keep);
   wr_hist_kernel<0><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
   wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 0, n_keep);
   wr_hist_kernel<1><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);

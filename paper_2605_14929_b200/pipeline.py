@@ -74,11 +74,15 @@ class LayerSweep:
     table, counts) are this sweep's own.  Sweeps that share buffers must run one after the other on one stream,
     and the packed output of one is overwritten by the next.  ``grid_dp`` builds the DD atom by the grid-constrained
     dynamic programme instead of Lloyd iterations with a snap (``lloyd_iters`` > 0 then only says that there is a DD
-    atom)."""
+    atom).  ``opq_q`` (a quantile in (0, 1), the paper's default 0.92) takes the outliers out of the weights before
+    anything else and keeps them as a sparse stream; the search, the DD atom and the packer then work on the weights
+    with the outliers zeroed.  ``wr_sigma`` (a fraction of the layer's elements, the paper's default 0.001) adds the
+    sparse correction of the packed layer's residual after the packer."""
 
     def __init__(self, M: int, K: int, T: int, fmt: I.ScaleFormat, rom: Sequence[str], fp: Sequence[str] = (),
                  lloyd_iters: int = 8, pool_percent: float = 50.0, device="cuda", want_blocks: bool = False,
-                 share: Optional["LayerSweep"] = None, grid_dp: bool = False):
+                 share: Optional["LayerSweep"] = None, grid_dp: bool = False, opq_q: Optional[float] = None,
+                 wr_sigma: Optional[float] = None, opq_capacity: Optional[int] = None):
         self.M, self.K, self.T, self.fmt = M, K, T, fmt
         self.dev = torch.device(device)
         self.iters = lloyd_iters
@@ -141,6 +145,23 @@ class LayerSweep:
             self.words = self._words_store[:B.words_nbytes(self.NB, self.container)]
             self.full_cos = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
             self.full_sse = torch.empty((nF, self.NB), dtype=torch.float32, device=d)
+        # the two sparse side streams (both off unless asked for)
+        self.opq_m = B.opq_threshold(opq_q, 16) if opq_q is not None else None
+        self.wr_keep = int(math.ceil(wr_sigma * M * K)) if wr_sigma is not None else 0
+        if self.opq_m is not None:
+            cap = opq_capacity if opq_capacity is not None else max(1024, M * K // 32)    # 3 % of the elements: six times the Gaussian rate at q = 0.92
+            self.W_opq = torch.empty((M, K), dtype=torch.bfloat16, device=d)
+            self.opq_row_start = torch.zeros(M + 1, dtype=torch.int32, device=d)
+            self.opq_records = torch.zeros(cap, dtype=torch.int32, device=d)
+            self.opq_count = torch.zeros(1, dtype=torch.int64, device=d)
+            self.ws_opq = B.opq_workspace(M, K, d)
+        if self.wr_keep:
+            self.wr_row_start = torch.zeros(M + 1, dtype=torch.int32, device=d)
+            self.wr_records = torch.zeros(2 * self.wr_keep + 1024, dtype=torch.int32, device=d)     # ties at the threshold all enter
+            self.wr_count = torch.zeros(1, dtype=torch.int64, device=d)
+            self.wr_exp = torch.zeros(1, dtype=torch.int32, device=d)
+            self.wr_tau = torch.zeros(1, dtype=torch.float32, device=d)
+            self.ws_wr = B.wr_workspace(M, K, d)
         self.kernel_launches_per_step = 0
         self.lloyd_launches = 0
         if lloyd_iters > 0:      # (the query takes the table size in place of the iterations for the dynamic programme)
@@ -155,6 +176,10 @@ class LayerSweep:
         if norms:
             B.sop_channel_norms(X, self.c, self.ws_norm, stream)
             n += 2
+        if self.opq_m is not None:
+            B.sop_opq_extract(W, self.opq_m, self.W_opq, self.opq_row_start, self.opq_records, self.opq_count, self.ws_opq, stream)
+            W = self.W_opq
+            n += 3
         if self.iters > 0:
             # every fixed candidate and every table entry among them; the best single of the result is FMTa
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.rom_result,
@@ -180,6 +205,14 @@ class LayerSweep:
                    counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
                    block_cos=self.full_cos, stream=stream)
         n += 1
+        if self.wr_keep:
+            B.sop_wr_extract(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, self.wr_keep, self.wr_row_start,
+                             self.wr_records, self.wr_count, self.wr_exp, self.ws_wr, tau=self.wr_tau,
+                             index_a=0 if self.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if self.single else B.PAIR_FROM_RESULT,
+                             search_result=self.result, use_sign=self.use_sign, container_bits=self.container,
+                             word_sign_bits=self.use_sign, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
+                             stream=stream)
+            n += 11
         self.kernel_launches_per_step = n
 
     def capture(self, W: torch.Tensor, X: torch.Tensor) -> None:
@@ -199,6 +232,23 @@ class LayerSweep:
 
     def replay(self) -> None:
         self._graph.replay()
+
+    def sparse_outputs(self) -> dict:
+        """The two sparse streams of the last pass: per stream the row starts, the records that fit the buffer and
+        the count; for Wr also the layer exponent and the threshold."""
+        torch.cuda.synchronize(self.dev)
+        out = {}
+        if self.opq_m is not None:
+            n = int(self.opq_count.item())
+            out["opq"] = dict(count=n, row_start=self.opq_row_start.cpu().numpy().view(np.uint32),
+                              records=self.opq_records[:min(n, self.opq_records.numel())].cpu().numpy().view(np.uint32),
+                              W_out=self.W_opq.cpu(), m=self.opq_m)
+        if self.wr_keep:
+            n = int(self.wr_count.item())
+            out["wr"] = dict(count=n, row_start=self.wr_row_start.cpu().numpy().view(np.uint32),
+                             records=self.wr_records[:max(0, min(n, self.wr_records.numel()))].cpu().numpy().view(np.uint32),
+                             scale_exp=int(self.wr_exp.item()), tau=float(self.wr_tau.item()), n_keep=self.wr_keep)
+        return out
 
     def outputs(self) -> SweepOutputs:
         torch.cuda.synchronize(self.dev)

@@ -169,3 +169,36 @@ def test_opq_then_search_then_wr_chain():
     assert got["count"] == want["count"] and np.array_equal(got["records"], want["records"]) and got["scale_exp"] == want["scale_exp"]
     # an outlier position holds +0 in the search input: its residual is minus the table value nearest to zero, times the scale
     assert np.array_equal(o["W_out"], oracle.opq_extract(L.W, m)["W_out"])
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_layer_sweep_with_both_streams(graph):
+    """LayerSweep with opq_q and wr_sigma: the outlier stream, the search on the zeroed weights and the correction of
+    the packed layer, call by call and replayed as one CUDA graph."""
+    d = dev()
+    L = I.laplace_outlier_layer(13, 2, 96, 1024, 64)
+    fmt = I.scale_format("E5M6")
+    rom = ["NF4", "SH4", "BOF4", "Split87"]
+    sw = LayerSweep(96, 1024, 64, fmt, rom, [], 4, device=d, opq_q=0.92, wr_sigma=0.001)
+    Wd, Xd = L.W.to(d), L.X.to(d)
+    if graph:
+        sw.capture(Wd, Xd)
+        sw.replay()
+    else:
+        sw.run(Wd, Xd)
+    out = sw.outputs()
+    sp = sw.sparse_outputs()
+    o = oracle.opq_extract(L.W, oracle.opq_threshold(0.92, 16))
+    assert sp["opq"]["count"] == o["count"] > 0
+    assert np.array_equal(sp["opq"]["records"], o["records"]) and np.array_equal(sp["opq"]["row_start"], o["row_start"])
+    assert np.array_equal(sp["opq"]["W_out"].view(torch.int16).numpy().view(np.uint16), o["W_out"])
+    W2 = torch.from_numpy(o["W_out"].view(np.int16).copy()).view(torch.bfloat16)
+    L2 = I.Layer(W2, L.X)
+    want = oracle_pipeline.run(L2, fmt, rom, [], lloyd_iters=4)
+    assert np.array_equal(out.dd_lut[:16].view(np.uint32), want["dd_lut"].view(np.uint32))
+    pk = want["pack"]
+    assert np.array_equal(out.codes.numpy().reshape(pk["codes"].shape), pk["codes"])
+    w = oracle_wr(L2, fmt, out, sw, sw.wr_keep)
+    assert sp["wr"]["count"] == w["count"] >= sw.wr_keep == math.ceil(0.001 * 96 * 1024)
+    assert np.array_equal(sp["wr"]["records"], w["records"]) and np.array_equal(sp["wr"]["row_start"], w["row_start"])
+    assert sp["wr"]["scale_exp"] == w["scale_exp"]
