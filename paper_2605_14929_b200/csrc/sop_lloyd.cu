@@ -355,9 +355,13 @@ __device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F
 }
 
 // One tile = the 256 pool blocks (4096 elements) of one CTA pass.  The tile is counting-sorted by
-// cell in shared memory; sorted position p is stored at (p % 16) * 256 + p / 16, so that thread t of
-// the iteration kernel reads positions 16 t .. 16 t + 15 as loads number 0 .. 15 at index i * 256 + t.
+// cell in shared memory.  Sorted position p is stored at slot (p & ~15) | ((p ^ (p >> 4)) & 15): the elements of a
+// cell stay next to each other in memory (an iteration reads the split cells' runs, a few 32-byte sectors each,
+// instead of one sector per element), and the thread that sums positions 16 t .. 16 t + 15 of the tile in shared
+// memory meets no bank conflict (the slots of one step differ in their low four bits over a half-warp).  The
+// exclusive-or keeps a group of four consecutive positions inside one 32-byte sector.
 // A tile that the pool does not fill is padded with (u, omega) = (0, 0): such elements add nothing.
+__device__ __forceinline__ unsigned tile_slot(unsigned p) { return (p & ~15u) | ((p ^ (p >> 4)) & 15u); }
 __device__ __forceinline__ long long fix24(float v) {   // llrint(v * 2^24): exact scaling, one rounding to an integer
   const float s = __fmul_rn(v, 16777216.0f);
   return fabsf(s) < 2147483648.0f ? (long long)__float2int_rn(s) : __float2ll_rn(s);
@@ -491,7 +495,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
       const unsigned p = hist[where[e] >> 16] + (where[e] & 0xFFFFu);
-      stage[(p & 15u) * LTB + (p >> 4)] = make_uint2(__float_as_uint(u[e]), __float_as_uint(om[e]));
+      stage[tile_slot(p)] = make_uint2(__float_as_uint(u[e]), __float_as_uint(om[e]));
     }
     __syncthreads();
     if (!DP) {      // the dynamic programme reads the per-cell sums only: no iteration walks the elements again
@@ -510,7 +514,7 @@ __global__ void __launch_bounds__(LTB) pool_cache_kernel(LloydArgs a, FmtDev F, 
       double a0 = 0.0, a1 = 0.0, a2 = 0.0;
 #pragma unroll 4
       for (int i2 = 0; i2 < 16; ++i2) {
-        const uint2 v = stage[i2 * LTB + tid];
+        const uint2 v = stage[tile_slot(16u * (unsigned)tid + (unsigned)i2)];
         const float u = __uint_as_float(v.x), om = __uint_as_float(v.y);
         const int c = sort_cell(u);
         if (c != cur) {
@@ -692,7 +696,7 @@ __device__ __forceinline__ bool lloyd_iteration(const LloydArgs& a, LloydWs* __r
           }
           cell_l[k] = l;
           const unsigned pp = s_p0[warp][l] + (item - s_off[warp][l]);
-          v[k] = __ldg(src + (pp & 15u) * LTB + (pp >> 4));
+          v[k] = __ldg(src + tile_slot(pp));
         }
       }
 #pragma unroll
