@@ -15,11 +15,11 @@
  *   - Return value: SOP_OK (0) or a negative SOP_ERR_* code; nothing throws, aborts or traps.
  *     Argument errors are detected on the host before anything is launched.
  *   - Required: K % 16 == 0, M, K, T >= 1, ldw >= K, ldx >= K, M*K < 2^31 blocks*16, finite inputs.
- *   - A call works on the CUDA device that is current when it is made.  The library keeps a few facts about
- *     the device per process (kernel attributes set once, the number of SMs, whether all Lloyd iterations
- *     fit one cooperative launch): one process drives one device, and calls are made from one host thread
+ *   - A call works on the CUDA device that is current when it is made.  The library keeps a few facts per
+ *     device ordinal (kernel attributes set once, the number of SMs, whether all Lloyd iterations fit one
+ *     cooperative launch), so one process may drive several devices; calls are made from one host thread
  *     at a time.
- *   - sop_channel_norms, sop_pair_search, sop_dd4_lloyd and sop_pack can be recorded into a CUDA graph by
+ *   - sop_channel_norms, sop_opq_extract, sop_pair_search, sop_dd4_lloyd, sop_pack and sop_wr_extract can be recorded into a CUDA graph by
  *     stream capture once each has been called normally on the device (the first call does the one-time
  *     set-ups), with profiling off.
  */

@@ -19,6 +19,35 @@ static cudaEvent_t g_ev[SOP_PROFILE_KINDS][PROFILE_RING][2];
 static bool g_ev_made = false;
 static long long g_ev_count[SOP_PROFILE_KINDS];
 
+constexpr int FACTS_DEVICES = 64;
+static DeviceFacts g_facts[FACTS_DEVICES + 1];
+static bool g_facts_init = false;
+
+DeviceFacts* device_facts() {
+  if (!g_facts_init) {
+    for (int i = 0; i <= FACTS_DEVICES; ++i) { g_facts[i].sms = 0; g_facts[i].coop_blocks_per_sm = -1; g_facts[i].search_attr_set = g_facts[i].lloyd_attr_set = false; }
+    g_facts_init = true;
+  }
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= FACTS_DEVICES) {
+    cudaGetLastError();
+    DeviceFacts* f = &g_facts[FACTS_DEVICES];      // beyond the table: nothing is remembered
+    f->sms = 0; f->coop_blocks_per_sm = -1; f->search_attr_set = f->lloyd_attr_set = false;
+    return f;
+  }
+  return &g_facts[dev];
+}
+
+int num_sms() {
+  DeviceFacts* f = device_facts();
+  if (!f->sms) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    f->sms = n;
+  }
+  return f->sms;
+}
+
 int profile_mark(int which, int edge, cudaStream_t st) {
   if (!g_profile) return SOP_OK;
   if (!g_ev_made) {

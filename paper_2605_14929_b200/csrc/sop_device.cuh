@@ -26,6 +26,18 @@ void set_cuda_error(cudaError_t e, const char* where);
     }                                                      \
   } while (0)
 
+// What the library remembers about a device, per device ordinal (a process may drive several devices; a call works
+// on the device that is current when it is made).  device_facts() returns the entry of the current device, or a
+// scratch entry that is never marked as known when the ordinal is beyond the table.
+struct DeviceFacts {
+  int sms;                    // 0: not asked yet
+  int coop_blocks_per_sm;     // resident CTAs of the persistent Lloyd kernel per SM; -1: not asked yet, 0: no cooperative launch
+  bool search_attr_set;       // the dynamic shared-memory limits of the search kernels have been raised on this device
+  bool lloyd_attr_set;        // the same for the pool cache kernels
+};
+DeviceFacts* device_facts();
+int num_sms();
+
 // Optional timing of one kernel family of a call (CUDA events on the launching stream): edge 0 before
 // the first launch, edge 1 after the last.  No-op unless profiling is enabled.
 int profile_mark(int which, int edge, cudaStream_t st);

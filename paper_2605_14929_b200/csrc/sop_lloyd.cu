@@ -942,17 +942,17 @@ static bool lloyd_iteration_plan(long long NB, long long pool_blocks, int iters,
   if (g_tune.iter_ctas > 0 && grid > g_tune.iter_ctas) grid = g_tune.iter_ctas;
   if (grid < 1) grid = 1;
   (void)NB;
-  static int coop_blocks_per_sm = -1;     // -1: not asked yet, 0: no cooperative launch on this device
-  if (coop_blocks_per_sm < 0) {
+  DeviceFacts* facts = device_facts();
+  if (facts->coop_blocks_per_sm < 0) {
     int dev = 0, coop = 0, nb = 0;
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, lloyd_persistent_kernel, LTB, 0) == cudaSuccess)
-      coop_blocks_per_sm = nb;
+      facts->coop_blocks_per_sm = nb;
     else
-      coop_blocks_per_sm = 0;
+      facts->coop_blocks_per_sm = 0;
     cudaGetLastError();
   }
-  const long long resident = (long long)coop_blocks_per_sm * sms;
+  const long long resident = (long long)facts->coop_blocks_per_sm * sms;
   bool persistent = false;
   if (iters >= 1 && resident >= 1 && !(flags & SOP_LLOYD_LAUNCH_PER_ITERATION)) {
     persistent = true;
@@ -1075,11 +1075,11 @@ int sop_dd4_lloyd(const void* W_dev, long long M, long long K, long long ldw, co
     const long long cg_max = g_tune.cache_ctas > 0 ? g_tune.cache_ctas : (long long)sms * 3;
     if (cg > cg_max) cg = cg_max;
     const size_t stage_bytes = (size_t)TILE_ELEMS * sizeof(uint2);
-    static bool attr_set = false;
-    if (!attr_set) {
+    DeviceFacts* facts = device_facts();
+    if (!facts->lloyd_attr_set) {
       SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
       SOP_CUDA_TRY(cudaFuncSetAttribute(pool_cache_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
-      attr_set = true;
+      facts->lloyd_attr_set = true;
     }
     if (grid_dp) pool_cache_kernel<true><<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);
     else pool_cache_kernel<false><<<(int)cg, LTB, stage_bytes, st>>>(a, F, ws, pool_count_dev, (unsigned)g_tune.spill_tiles);

@@ -1199,16 +1199,6 @@ static bool coarsen_cells(Plan* P) {
   return true;
 }
 
-static int g_num_sms = 0;
-int num_sms() {
-  if (!g_num_sms) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
-    g_num_sms = n;
-  }
-  return g_num_sms;
-}
-
 }  // namespace sop
 
 extern "C" {
@@ -1303,8 +1293,8 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     SOP_CUDA_TRY(cudaGetLastError());
   }
   if ((rc = profile_mark(SOP_PROFILE_PREPASS, 1, st))) return rc;
-  static bool attr_set = false;
-  if (!attr_set) {
+  DeviceFacts* facts = device_facts();
+  if (!facts->search_attr_set) {
     SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
 #define SOP_REDUCE_ATTR(SE, T, BK) \
   SOP_CUDA_TRY(cudaFuncSetAttribute(reduce_kernel<SE, T, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX))
@@ -1313,7 +1303,7 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     SOP_REDUCE_ATTR(true, 1, false); SOP_REDUCE_ATTR(true, 2, false); SOP_REDUCE_ATTR(true, 3, false);
     SOP_REDUCE_ATTR(true, 1, true); SOP_REDUCE_ATTR(true, 2, true); SOP_REDUCE_ATTR(true, 3, true);
 #undef SOP_REDUCE_ATTR
-    attr_set = true;
+    facts->search_attr_set = true;
   }
   if ((rc = profile_mark(SOP_PROFILE_SWEEP, 0, st))) return rc;
   if (eval_mask) {

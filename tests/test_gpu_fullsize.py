@@ -293,3 +293,39 @@ def test_config3_mlp_layers_fp6_against_fp8_in_full(B, which):
         assert pk["rc"] == 0
         assert np.array_equal(codes[m0 * nbk:(m0 + 8) * nbk], pk["codes"])
         assert np.array_equal(words[m0 * nbk:(m0 + 8) * nbk], pk["words"])
+
+
+def test_config5_attention_layer_with_both_sparse_streams_in_full(B):
+    """The 8192x8192 layer at E5M6 with the outlier stream in front and the residual correction behind: 16384 tiles
+    of 256 blocks per stream pass.  The outlier stream and the zeroed weights are compared in full; the correction is
+    computed by the oracle in full from the pair, shifts and DD table that the device pipeline chose."""
+    from paper_2605_14929_b200.pipeline import LayerSweep
+    L = I.config5_layer(0, 0, 0, device=str(dev()))
+    M, K = L.W.shape
+    fmt = I.scale_format("E5M6")
+    sw = LayerSweep(M, K, L.X.shape[0], fmt, ["NF4", "SH4", "BOF4", "Split87"], [], 8, device=dev(), opq_q=0.92, wr_sigma=0.001,
+                    opq_capacity=M * K // 8)
+    sw.run(L.W, L.X)
+    out = sw.outputs()
+    sp = sw.sparse_outputs()
+    w16, _ = _host_w(L.W)
+    W_host = torch.from_numpy(w16.view(np.int16).copy()).view(torch.bfloat16)
+    o = oracle.opq_extract(W_host, oracle.opq_threshold(0.92, 16), capacity=M * K // 8)
+    assert sp["opq"]["count"] == o["count"] <= M * K // 8
+    assert np.array_equal(sp["opq"]["row_start"], o["row_start"]) and np.array_equal(sp["opq"]["records"], o["records"])
+    assert np.array_equal(sp["opq"]["W_out"].view(torch.int16).numpy().view(np.uint16), o["W_out"])
+    # the correction of the packed layer: the oracle re-evaluates the chosen pair on every block of the zeroed weights
+    W2 = torch.from_numpy(o["W_out"].view(np.int16).copy()).view(torch.bfloat16)
+    best = out.result["best"]
+    assert sw.use_sign == 1
+    ia, ib = int(best[3]), int(best[4])
+    atoms = list(out.atoms)
+
+    def atom(i):
+        a = atoms[i]
+        return I.Atom(a.name, a.n_bits, I.KIND_LUT, a.negated, I.SCOPE_BLOCK, 1.0, out.dd_lut[:16]) if (sw.dd_mask >> i) & 1 else a
+    w = oracle.wr_extract(W2, out.c.numpy(), fmt, atom(ia), int(out.result["k"][ia]), atom(ib), int(out.result["k"][ib]), use_sign=1,
+                          n_keep=sw.wr_keep, capacity=2 * sw.wr_keep + 1024)
+    assert sp["wr"]["count"] == w["count"] >= sw.wr_keep and sp["wr"]["scale_exp"] == w["scale_exp"]
+    assert np.float32(sp["wr"]["tau"]).view(np.uint32) == np.float32(w["tau"]).view(np.uint32)
+    assert np.array_equal(sp["wr"]["row_start"], w["row_start"]) and np.array_equal(sp["wr"]["records"], w["records"])

@@ -202,3 +202,17 @@ def test_layer_sweep_with_both_streams(graph):
     assert sp["wr"]["count"] == w["count"] >= sw.wr_keep == math.ceil(0.001 * 96 * 1024)
     assert np.array_equal(sp["wr"]["records"], w["records"]) and np.array_equal(sp["wr"]["row_start"], w["row_start"])
     assert sp["wr"]["scale_exp"] == w["scale_exp"]
+
+
+def test_streams_beyond_one_round_of_the_tile_scan():
+    """More than 1024 tiles of 256 blocks: the one-CTA scan carries its running sum from round to round."""
+    M, K = 2304, 2048                                  # 294912 blocks = 1152 tiles
+    L = I.laplace_outlier_layer(21, 3, M, K, 64)
+    m = B.opq_threshold(0.92, 16)
+    assert_opq(run_opq(L.W, m), oracle.opq_extract(L.W, m))
+    fmt = I.scale_format("UE4M4")
+    n_keep = math.ceil(0.001 * M * K)
+    sw, out, got = run_wr(L, fmt, ["NF4", "SH4"], n_keep, None)
+    want = oracle_wr(L, fmt, out, sw, n_keep)
+    assert got["count"] == want["count"] >= n_keep and got["scale_exp"] == want["scale_exp"]
+    assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
