@@ -70,36 +70,39 @@ __device__ __forceinline__ unsigned cta_excl_scan(unsigned v, unsigned* s_warp, 
   return base + incl - v;
 }
 
-// In place: tile_sums[t] becomes the number of records before tile t.  One CTA; the total goes to row_start[M]
-// and *count.  With `wr` the kernel also turns the largest kept |E| into the layer exponent of the Wr values.
+// In place: tile_sums[t] becomes the number of records before tile t.  One CTA of 32 warps: a warp takes a contiguous
+// share of the tiles and sums it with coalesced loads, the 32 sums are scanned, the warp then walks its share again
+// 32 tiles at a time (a warp scan plus the running sum).  The total goes to row_start[M] and *count.  With `wr` the
+// kernel also turns the largest kept |E| into the layer exponent of the Wr values.
 __global__ void __launch_bounds__(1024) tile_scan_kernel(unsigned* __restrict__ tile_sums, long long n_tiles, unsigned* __restrict__ row_start,
                                                          long long M, long long* __restrict__ count, SparseWs* __restrict__ ws, int wr,
                                                          int* __restrict__ scale_exp_out, float* __restrict__ tau_out) {
   __shared__ unsigned s_warp[32];
-  __shared__ unsigned s_carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_carry = 0;
+  const long long per = ((n_tiles + 31) / 32 + 31) / 32 * 32;            // tiles per warp, a multiple of 32
+  const long long t0 = (long long)warp * per, t1 = t0 + per < n_tiles ? t0 + per : n_tiles;
+  unsigned local = 0;
+  for (long long i = t0 + lane; i < t1; i += 32) local += tile_sums[i];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
+  if (lane == 0) s_warp[warp] = local;
   __syncthreads();
-  for (long long base = 0; base < n_tiles; base += 1024) {
-    const long long i = base + tid;
-    const unsigned v = i < n_tiles ? tile_sums[i] : 0u;
+  unsigned run = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < 32; ++w) { const unsigned c = s_warp[w]; total += c; if (w < warp) run += c; }
+  for (long long i0 = t0; i0 < t1; i0 += 32) {
+    const long long i = i0 + lane;
+    const unsigned v = i < t1 ? tile_sums[i] : 0u;
     unsigned incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
       if (lane >= o) incl += t;
     }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    unsigned before = s_carry;
-    for (int w = 0; w < warp; ++w) before += s_warp[w];
-    if (i < n_tiles) tile_sums[i] = before + incl - v;
-    __syncthreads();
-    if (tid == 1023) s_carry = before + incl;
-    __syncthreads();
+    if (i < t1) tile_sums[i] = run + incl - v;
+    run += __shfl_sync(0xFFFFFFFFu, incl, 31);
   }
   if (tid == 0) {
-    const unsigned total = s_carry;
     row_start[M] = total;
     if (count) *count = wr && ws->no_pair ? -1ll : (long long)total;
     if (wr) {
@@ -273,12 +276,14 @@ __device__ void wr_setup(const WrArgs& a, const AtomsDev& A, const sop_search_re
 }
 
 // One block of the packed layer: the residual E_i = w_i - s_hat q_i (one rounding) and the metric |E_i| c_k.
+// LUT4: both codebooks are tables of at most 16 entries (the common case): constant shifts, no kind test per element.
+template <bool LUT4>
 __device__ __forceinline__ void wr_block(const WrArgs& a, const FmtDev& F, const WrShared& sh, long long blk, long long j,
                                          const uint16_t* __restrict__ wrow, float (&E)[16], float (&met)[16]) {
   const uint4* p = reinterpret_cast<const uint4*>(wrow);
   const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
   const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-  const int n = sh.n_bits, b = a.container_bits;
+  const int n = LUT4 ? 4 : sh.n_bits, b = a.container_bits;
   // the 16n-bit payload as one little-endian integer
   unsigned long long lo = 0, hi = 0;
   const unsigned char* cp = a.codes + (size_t)blk * 2 * n;
@@ -337,7 +342,7 @@ __device__ __forceinline__ void wr_block(const WrArgs& a, const FmtDev& F, const
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     uint32_t code;
-    if (n == 4) {                     // the common width: 32-bit shifts by constants
+    if (LUT4 || n == 4) {             // the common width: 32-bit shifts by constants
       code = (lo32[i >> 3] >> (4 * (i & 7))) & 15u;
     } else {
       const int pos = i * n;
@@ -347,7 +352,7 @@ __device__ __forceinline__ void wr_block(const WrArgs& a, const FmtDev& F, const
       code = (uint32_t)v & emask;
     }
     float q;
-    if (cd.kind == SOP_KIND_LUT) { q = sh.lutv[sel][code & 31u]; q = neg ? -q : q; }
+    if (LUT4 || cd.kind == SOP_KIND_LUT) { q = sh.lutv[sel][code & 31u]; q = neg ? -q : q; }
     else q = fp_grid_decode(code, cd.sign_pos, cd.y, cd.bias);
     const float w = (i & 1) ? bf16hi(wb[i >> 1]) : bf16lo(wb[i >> 1]);
     E[i] = __fmaf_rn(-s_hat, q, w);
@@ -361,7 +366,7 @@ __device__ __forceinline__ unsigned wr_key(float met) {
   return ~(met > 0.0f ? __float_as_uint(met) : 0u);
 }
 
-template <int PASS>
+template <int PASS, bool LUT4>
 __global__ void __launch_bounds__(STB) wr_hist_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
                                                       SparseWs* __restrict__ ws) {
   __shared__ WrShared sh;
@@ -379,7 +384,7 @@ __global__ void __launch_bounds__(STB) wr_hist_kernel(WrArgs a, AtomsDev A, FmtD
     if (blk >= a.NB) continue;
     const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
     float E[16], met[16];
-    wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+    wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
     if constexpr (PASS < 0) {
       float bm = 0.0f;
 #pragma unroll
@@ -458,6 +463,7 @@ __global__ void __launch_bounds__(1024) wr_pick_kernel(SparseWs* __restrict__ ws
 
 __device__ __forceinline__ bool wr_kept(float met, float tau) { return met >= tau && met > 0.0f; }
 
+template <bool LUT4>
 __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
                                                        SparseWs* __restrict__ ws) {
   __shared__ WrShared sh;
@@ -477,7 +483,7 @@ __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, Fmt
     if (blk < a.NB && !sh.no_pair) {
       const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;   // the block count fits 31 bits
       float E[16], met[16];
-      wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+      wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
 #pragma unroll
       for (int i = 0; i < 16; ++i)
         if (wr_kept(met[i], tau)) { ++cnt; emax = max(emax, __float_as_uint(fabsf(E[i]))); }
@@ -494,6 +500,7 @@ __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, Fmt
   if ((tid & 31) == 0 && emax) atomicMax(&ws->emax_bits, emax);
 }
 
+template <bool LUT4>
 __global__ void __launch_bounds__(STB) wr_write_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
                                                        const SparseWs* __restrict__ ws) {
   __shared__ WrShared sh;
@@ -517,7 +524,7 @@ __global__ void __launch_bounds__(STB) wr_write_kernel(WrArgs a, AtomsDev A, Fmt
     long long m = 0, j = 0;
     if (blk < a.NB && !sh.no_pair) {
       m = (long long)((unsigned)blk / (unsigned)a.nbk); j = blk - m * a.nbk;
-      wr_block(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+      wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
 #pragma unroll
       for (int i = 0; i < 16; ++i)
         if (wr_kept(met[i], tau)) keep |= 1u << i;
@@ -675,17 +682,32 @@ int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, c
   const int grid = (int)(n_tiles < cap ? n_tiles : cap);
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(SparseWs), st));
   if ((rc = profile_mark(SOP_PROFILE_WR, 0, st))) return rc;
-  wr_hist_kernel<-1><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
-  wr_pick_kernel<<<1, 1024, 0, st>>>(ws, -1, n_keep);
-  wr_hist_kernel<0><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
-  wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 0, n_keep);
-  wr_hist_kernel<1><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
-  wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 1, n_keep);
-  wr_hist_kernel<2><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
-  wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 2, n_keep);
-  wr_count_kernel<<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
-  tile_scan_kernel<<<1, 1024, 0, st>>>(a.tile_sums, n_tiles, row_start_dev, M, count_dev, ws, 1, scale_exp_dev, tau_dev);
-  wr_write_kernel<<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);
+  // both codebooks tables of at most 16 entries: the decode with constant shifts (a pair taken from a search result is
+  // always a pair of tables, and n_bits is then the alphabet's)
+  bool lut4 = true;
+  if (from_result) {
+    for (int i = 0; i < n_atoms; ++i)
+      if (atoms[i].kind == SOP_KIND_LUT && atoms[i].n_bits != 4) lut4 = false;
+  } else {
+    lut4 = atoms[index_a].kind == SOP_KIND_LUT && atoms[index_a].n_bits == 4 &&
+           (index_b == SOP_NO_ATOM || (atoms[index_b].kind == SOP_KIND_LUT && atoms[index_b].n_bits == 4));
+  }
+#define SOP_WR_LAUNCHES(L4)                                                          \
+  do {                                                                               \
+    wr_hist_kernel<-1, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);           \
+    wr_pick_kernel<<<1, 1024, 0, st>>>(ws, -1, n_keep);                              \
+    wr_hist_kernel<0, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
+    wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 0, n_keep);                               \
+    wr_hist_kernel<1, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
+    wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 1, n_keep);                               \
+    wr_hist_kernel<2, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
+    wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 2, n_keep);                               \
+    wr_count_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);              \
+    tile_scan_kernel<<<1, 1024, 0, st>>>(a.tile_sums, n_tiles, row_start_dev, M, count_dev, ws, 1, scale_exp_dev, tau_dev); \
+    wr_write_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);              \
+  } while (0)
+  if (lut4) SOP_WR_LAUNCHES(true); else SOP_WR_LAUNCHES(false);
+#undef SOP_WR_LAUNCHES
   SOP_CUDA_TRY(cudaGetLastError());
   if ((rc = profile_mark(SOP_PROFILE_WR, 1, st))) return rc;
   return SOP_OK;

@@ -85,11 +85,11 @@ def test_opq_edge_cases():
     assert_opq(run_opq(Wb, m), oracle.opq_extract(Wb, m))
 
 
-def run_wr(L, fmt, rom, n_keep, use_sign, lloyd_iters=0, capacity=None, single=False):
+def run_wr(L, fmt, rom, n_keep, use_sign, lloyd_iters=0, capacity=None, fp=()):
     """The layer through the pipeline (search, pack), then the correction of what was packed."""
     d = dev()
     M, K = L.W.shape
-    sw = LayerSweep(M, K, L.X.shape[0], fmt, rom, [], lloyd_iters, device=d)
+    sw = LayerSweep(M, K, L.X.shape[0], fmt, rom, list(fp), lloyd_iters, device=d)
     Wd, Xd = L.W.to(d), L.X.to(d)
     sw.run(Wd, Xd)
     out = sw.outputs()
@@ -101,6 +101,7 @@ def run_wr(L, fmt, rom, n_keep, use_sign, lloyd_iters=0, capacity=None, single=F
     tau = torch.zeros(1, dtype=torch.float32, device=d)
     ws = B.wr_workspace(M, K, d)
     B.sop_wr_extract(Wd, sw.c, sw.fmt_c, sw.atoms_c, sw.codes, sw._words_store, n_keep, row_start, records, count, e, ws, tau=tau,
+                     index_a=0 if sw.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if sw.single else B.PAIR_FROM_RESULT,
                      search_result=sw.result, use_sign=sw.use_sign, container_bits=sw.container, word_sign_bits=sw.use_sign,
                      dd_lut=sw.dd_lut if sw.dd_mask else None, dd_mask=sw.dd_mask)
     torch.cuda.synchronize()
@@ -111,10 +112,12 @@ def run_wr(L, fmt, rom, n_keep, use_sign, lloyd_iters=0, capacity=None, single=F
 
 
 def oracle_wr(L, fmt, out, sw, n_keep):
+    if sw.single:           # one element format packed alone
+        return oracle.wr_extract(L.W, out.c.numpy(), fmt, out.atoms[0], int(out.result["k"][0]), None, 0, use_sign=0, n_keep=n_keep)
     best = out.result["best"]
     ia, ib = (int(best[3]), int(best[4])) if sw.use_sign else (int(best[0]), int(best[1]))
     atoms = list(out.atoms)
-    dd = out.dd_lut[:16]
+    dd = out.dd_lut[:1 << atoms[0].n_bits]
 
     def atom(i):
         a = atoms[i]
@@ -213,6 +216,20 @@ def test_streams_beyond_one_round_of_the_tile_scan():
     fmt = I.scale_format("UE4M4")
     n_keep = math.ceil(0.001 * M * K)
     sw, out, got = run_wr(L, fmt, ["NF4", "SH4"], n_keep, None)
+    want = oracle_wr(L, fmt, out, sw, n_keep)
+    assert got["count"] == want["count"] >= n_keep and got["scale_exp"] == want["scale_exp"]
+    assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
+
+
+@pytest.mark.parametrize("rom,fp,fmt_name,iters", [(["NF5", "SH5", "BOF5"], (), "UE4M4", 0), (["NF5", "E2M2"], (), "E5M6", 3),
+                                                  ([], ("E2M3",), "UE4M4", 0), ([], ("E4M3",), "E5M6", 0), ([], ("E3M4",), "UE4M4", 0)])
+def test_wr_on_wider_codes_and_element_formats(rom, fp, fmt_name, iters):
+    """The general decode: 5-bit table codes (ten bytes per block), and single element formats whose codes are the
+    format's own bit pattern (6 and 8 bits)."""
+    L = I.student_layer(17, 1, 20, 320, 64, 4.0)
+    fmt = I.scale_format(fmt_name)
+    n_keep = 40
+    sw, out, got = run_wr(L, fmt, rom, n_keep, None, lloyd_iters=iters, fp=fp)
     want = oracle_wr(L, fmt, out, sw, n_keep)
     assert got["count"] == want["count"] >= n_keep and got["scale_exp"] == want["scale_exp"]
     assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
