@@ -42,6 +42,7 @@ extern "C" {
 #define SOP_SEARCH_SINGLES_ONLY 1 /* flags of sop_pair_search: reduce single candidates only, no pair / signed entries */
 #define SOP_SEARCH_SELECT_MSE 2   /* flags of sop_pair_search: the per-block reassignment takes the smaller block error */
 #define SOP_SEARCH_KEEP_LOADED_ENTRIES 4 /* flags of sop_pair_search: table entries among loaded candidates are kept, not formed again */
+#define SOP_SEARCH_REUSE_PREPASS 8 /* flags of sop_pair_search: the shifts come from the exponent histograms an earlier call left in the workspace */
 
 enum {
   SOP_OK = 0,
@@ -187,6 +188,11 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *   design axes", axis ii): in every two-way and signed entry the block goes to the candidate with the
  *   smaller block squared error instead of the larger block cosine (ties keep the earlier candidate);
  *   acos, mse and the counts are those of that assignment, the best pair is still ranked by acos.
+ *   SOP_SEARCH_REUSE_PREPASS: the exponent histogram of the block scales and max|W| do not depend on the scale
+ *   format, so a layer that is swept at several scale formats needs them once.  With this flag the call takes them
+ *   from workspace_dev as the last call without the flag (and without SOP_K_FROM_RESULT) left them, and only derives
+ *   this format's shifts: the caller guarantees that W, M, K, the alphabet and eval_mask are those of that call
+ *   (calls with SOP_K_FROM_RESULT in between leave the histograms alone).  Ignored with SOP_K_FROM_RESULT.
  * prev_result_dev (may be NULL): with k_mode = SOP_K_FROM_RESULT, the result block of the earlier call on
  *   this layer (not result_dev itself).  The shift of every scale class and max|W| are taken from it
  *   instead of reading W once more; every per-block-scaled class of this call must then contain a

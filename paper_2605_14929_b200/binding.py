@@ -23,6 +23,7 @@ ALL_ATOMS = 0xFFFFFFFF
 SEARCH_SINGLES_ONLY = 1
 SEARCH_SELECT_MSE = 2
 SEARCH_KEEP_LOADED_ENTRIES = 4
+SEARCH_REUSE_PREPASS = 8
 LLOYD_POOL_BY_ERROR, LLOYD_UNIFORM_WEIGHTS, LLOYD_POOL_THRESHOLD, LLOYD_LAUNCH_PER_ITERATION, LLOYD_GRID_DP = 1, 2, 4, 8, 16
 PACK_SELECT_MSE = 1
 MAX_ENTRIES = 32
@@ -210,7 +211,7 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
                     block_cos: Optional[torch.Tensor] = None, block_sse: Optional[torch.Tensor] = None,
                     stream=None, g: int = 16, eval_mask: int = ALL_ATOMS, load_mask: int = 0,
                     singles_only: bool = False, prev_result: Optional[torch.Tensor] = None,
-                    select_mse: bool = False, keep_loaded: bool = False) -> None:
+                    select_mse: bool = False, keep_loaded: bool = False, reuse_prepass: bool = False) -> None:
     """``keep_loaded``: the table entries among the candidates of ``load_mask`` stay as an earlier call wrote them
     into ``pair_table`` / ``signed_table``; only the entries with a newly evaluated candidate are formed."""
     assert W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.stride(1) == 1
@@ -219,7 +220,8 @@ def sop_pair_search(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, pair
                                  make_atoms(atoms), len(atoms), _ptr(dd_lut), C.c_uint(dd_mask), C.c_uint(eval_mask),
                                  C.c_uint(load_mask),
                                  (SEARCH_SINGLES_ONLY if singles_only else 0) | (SEARCH_SELECT_MSE if select_mse else 0)
-                                 | (SEARCH_KEEP_LOADED_ENTRIES if keep_loaded else 0), _ptr(prev_result),
+                                 | (SEARCH_KEEP_LOADED_ENTRIES if keep_loaded else 0) | (SEARCH_REUSE_PREPASS if reuse_prepass else 0),
+                                 _ptr(prev_result),
                                  _ptr(pair_table),
                                  _ptr(signed_table), _ptr(result), _ptr(block_cos), _ptr(block_sse), _ptr(workspace),
                                  C.c_size_t(workspace.numel()), _stream(stream)), "sop_pair_search")

@@ -96,7 +96,10 @@ struct WsHeader {
 struct Partial { double gap, sse; long long n1, nneg; };
 
 static size_t ws_hist_off() { return 256; }
-static size_t ws_part_off() { return 256 + sizeof(unsigned) * SOP_MAX_CLASSES * SOP_HIST_BINS; }
+// after the histograms: max|W| as the prepass found it (the header is cleared by every call, the histograms and this
+// word stay until the next prepass)
+static size_t ws_wmax_off() { return 256 + sizeof(unsigned) * SOP_MAX_CLASSES * SOP_HIST_BINS; }
+static size_t ws_part_off() { return ws_wmax_off() + 256; }
 static size_t ws_total() { return ((ws_part_off() + sizeof(Partial) * (size_t)MAX_GRID * MAX_SLOTS) + 255) & ~(size_t)255; }
 
 struct LayerArgs {
@@ -159,8 +162,17 @@ __global__ void __launch_bounds__(256) prepass_kernel(LayerArgs L, Plan P, FmtDe
   __syncthreads();
   if (s_last) {
     __threadfence();
+    if (threadIdx.x == 0) hist[SOP_MAX_CLASSES * SOP_HIST_BINS] = __ldcg(&hdr->wmax_bits);    // kept for later calls on this layer
     kselect_body(P, F, hist, hdr);
   }
+}
+
+// The shifts of another scale format from the histograms that an earlier prepass of the same layer left in the workspace.
+__global__ void __launch_bounds__(256) kselect_kernel(Plan P, FmtDev F, const unsigned* __restrict__ hist, WsHeader* __restrict__ hdr) {
+  if (threadIdx.x == 0) hdr->wmax_bits = hist[SOP_MAX_CLASSES * SOP_HIST_BINS];
+  __threadfence();
+  __syncthreads();
+  kselect_body(P, F, hist, hdr);
 }
 
 // One CTA of 256 threads.  Reads the global histogram and max|W| through the L2 (they were written by
@@ -1239,7 +1251,8 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   eval_mask &= all;
   if ((load_mask & ~all) || (load_mask & eval_mask) || !(eval_mask | load_mask)) return SOP_ERR_ALPHABET;
   if (load_mask && own_columns) return SOP_ERR_NULL;
-  if (flags & ~(SOP_SEARCH_SINGLES_ONLY | SOP_SEARCH_SELECT_MSE | SOP_SEARCH_KEEP_LOADED_ENTRIES)) return SOP_ERR_RANGE;
+  if (flags & ~(SOP_SEARCH_SINGLES_ONLY | SOP_SEARCH_SELECT_MSE | SOP_SEARCH_KEEP_LOADED_ENTRIES | SOP_SEARCH_REUSE_PREPASS)) return SOP_ERR_RANGE;
+  const bool reuse_prepass = (flags & SOP_SEARCH_REUSE_PREPASS) && !k_from_result;
   const int keep_loaded = (flags & SOP_SEARCH_KEEP_LOADED_ENTRIES) && load_mask ? 1 : 0;
   Plan P;
   if ((rc = build_plan(A, F, k_from_result ? 0 : k_mode, eval_mask, load_mask, flags & SOP_SEARCH_SINGLES_ONLY, keep_loaded, &P))) return rc;
@@ -1283,9 +1296,13 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   long long rgrid = n_tiles < (long long)sms * 2 ? n_tiles : (long long)sms * 2;
   if (rgrid < 1) rgrid = 1;
 
-  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, ws_part_off(), st));
+  // the header always starts from zero; the histograms (and max|W| behind them) only when this call fills them
+  SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, (k_from_result || reuse_prepass) ? ws_hist_off() : ws_part_off(), st));
   if ((rc = profile_mark(SOP_PROFILE_PREPASS, 0, st))) return rc;
-  if (!k_from_result) {
+  if (reuse_prepass) {
+    kselect_kernel<<<1, 256, 0, st>>>(P, F, hist, hdr);
+    SOP_CUDA_TRY(cudaGetLastError());
+  } else if (!k_from_result) {
     // one read of W: block scales' exponent histogram, max|W|, then the shifts (last CTA)
     long long want = (L.NB + 255) / 256;
     const int pgrid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);

@@ -168,10 +168,13 @@ class LayerSweep:
             self.lloyd_launches = (B.dd4_lloyd_launches(M, K, 1 << n_bits, B.LLOYD_GRID_DP) if self.grid_dp
                                    else B.dd4_lloyd_launches(M, K, lloyd_iters))
 
-    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True) -> None:
+    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True, reuse_prepass: bool = False) -> None:
         """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32.  ``norms`` =
         False skips the channel norms: they do not depend on the scale format, so a sweep that shares the
-        buffers of another one (same layer, other format) uses the norms that one has just computed."""
+        buffers of another one (same layer, other format) uses the norms that one has just computed.
+        ``reuse_prepass``: the same holds for the exponent histogram of the block scales behind the per-layer
+        shift: the search takes it from the shared workspace as the sweep of this layer at the previous format
+        left it, and only derives this format's shifts."""
         n = 0
         if norms:
             B.sop_channel_norms(X, self.c, self.ws_norm, stream)
@@ -184,7 +187,7 @@ class LayerSweep:
             # every fixed candidate and every table entry among them; the best single of the result is FMTa
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.rom_result,
                               self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, eval_mask=self.fixed_mask,
-                              stream=stream)
+                              stream=stream, reuse_prepass=reuse_prepass)
             n += 3
             B.sop_dd4_lloyd(W, self.c, self.fmt_c, self.atoms_c, self.full_cos, self.pool_rank, self.dd_iters, self.dd_lut,
                             self.distortion, self.pool_count, self.ws_lloyd, search_result=self.rom_result, stream=stream,
@@ -196,7 +199,8 @@ class LayerSweep:
                               k_mode=B.K_FROM_RESULT, prev_result=self.rom_result, keep_loaded=True, stream=stream)
         else:
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.result,
-                              self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream)
+                              self.ws_search, block_cos=self.full_cos, block_sse=self.full_sse, stream=stream,
+                              reuse_prepass=reuse_prepass)
             n += 1
         n += 2
         B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, search_result=self.result,
@@ -320,7 +324,7 @@ class LayerStream:
             if self.before_run is not None:
                 self.before_run()
             for f, q in enumerate(self.sweeps):
-                q.run(self.W[slot], self.X[slot], self.s_run, norms=(f == 0))
+                q.run(self.W[slot], self.X[slot], self.s_run, norms=(f == 0), reuse_prepass=(f > 0))
                 # the sweeps share their packed output: it is set aside before the next format overwrites it
                 for k in self.OUT:
                     self.dev_out[slot][f][k].copy_(getattr(q, k), non_blocking=True)
@@ -370,7 +374,7 @@ class LayerSetSweep:
         """``layers``: one (W, X) pair of device tensors per shape given to the constructor, in that order."""
         for row, (W, X) in zip(self.sweeps, layers):
             for f, sw in enumerate(row):
-                sw.run(W, X, stream, norms=(f == 0))
+                sw.run(W, X, stream, norms=(f == 0), reuse_prepass=(f > 0))
 
     @property
     def kernel_launches_per_step(self) -> int:

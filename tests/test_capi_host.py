@@ -87,7 +87,7 @@ def test_pair_search_rejects_bad_arguments(lib):
     assert _search(lib, emask=0, lmask=4, bc=FAKE) == -4   # load bit beyond the alphabet
     atoms2 = I.alphabet(["NF4"])
     assert _search(lib, atoms=atoms2, emask=1, lmask=2) == -1   # loading needs the per-block arrays
-    assert _search(lib, flags=8) == -7                 # unknown flag
+    assert _search(lib, flags=16) == -7                # unknown flag
     assert _search(lib, k=B.K_FROM_RESULT) == -1       # shifts from an earlier result need that result
     assert _search(lib, k=B.K_FROM_RESULT, prev=C.c_void_p(0x20000)) == -7   # ... and a loaded candidate in every class
 

@@ -130,3 +130,37 @@ def test_grid_constrained_dd_by_dynamic_programming(B, fmt_name, names, layer):
     want = oracle.dd_grid_dp(L.W, c, fmt, int(r["k"][0]), r["block_sse"][0], NB // 3, ne, pool_by_error=True, uniform_weights=True)
     got = gpu_lloyd(B, L.W, c, fmt, atoms, bs, NB // 3, 0, int(r["k"][0]), 0, grid_dp=True, pool_by_error=True, uniform_weights=True)
     assert np.array_equal(got[0][:ne].view(np.uint32), want[0].view(np.uint32)) and got[2] == want[2]
+
+
+def test_shifts_from_the_histogram_of_an_earlier_format():
+    """A layer swept at several scale formats builds the exponent histogram of its block scales once: the sweeps of
+    the later formats derive their shifts from the workspace (flag SOP_SEARCH_REUSE_PREPASS) and give what a sweep
+    of their own gives, the layer-wide power-of-two scale of a ^0 candidate included."""
+    from paper_2605_14929_b200.pipeline import LayerSweep
+    d = torch.device("cuda:0")
+    L = I.config5_layer(0, 1, 1, rows=48)
+    L = I.Layer(L.W, L.X[:128].contiguous())
+    M, K = L.W.shape
+    Wd, Xd = L.W.to(d), L.X.to(d)
+    rom, fp = ["NF4", "SH4", "BOF4"], ["E4M3^0", "E2M3"]
+    fmts = [I.scale_format(f) for f in ("E5M6", "UE4M4", "E4M3", "UE8M0")]
+    first = None
+    shared = []
+    for f, fmt in enumerate(fmts):
+        sw = LayerSweep(M, K, 128, fmt, rom, fp, 3, device=d, share=first)
+        first = first or sw
+        sw.run(Wd, Xd, norms=(f == 0), reuse_prepass=(f > 0))
+        shared.append(sw.outputs())
+    ks = set()
+    for fmt, got in zip(fmts, shared):
+        own = LayerSweep(M, K, 128, fmt, rom, fp, 3, device=d)
+        own.run(Wd, Xd)
+        want = own.outputs()
+        assert np.array_equal(got.result["k"], want.result["k"]) and np.array_equal(got.result["best"], want.result["best"])
+        assert got.result["layer_absmax"] == want.result["layer_absmax"] > 0
+        assert np.array_equal(got.pair_table["n_sel1"], want.pair_table["n_sel1"])
+        assert np.array_equal(got.pair_table["acos"], want.pair_table["acos"], equal_nan=True)
+        assert np.array_equal(got.dd_lut.view(np.uint32), want.dd_lut.view(np.uint32))
+        assert torch.equal(got.codes, want.codes) and torch.equal(got.words, want.words)
+        ks.add(int(want.result["k"][0]))
+    assert len(ks) > 1          # the formats really need different shifts
