@@ -454,7 +454,7 @@ def run_gpu(args) -> None:
     ls_of, order = {}, []
     for row, shape in zip(sset.sweeps, shapes):
         if shape not in ls_of:
-            ls_of[shape] = LayerStream(row, streams)
+            ls_of[shape] = LayerStream(row, streams, graphs=True)
         order.append(ls_of[shape])
     h2d = sum(ls.h2d_bytes for ls in order)
     d2h = sum(ls.d2h_bytes for ls in order)

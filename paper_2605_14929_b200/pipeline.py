@@ -168,13 +168,17 @@ class LayerSweep:
             self.lloyd_launches = (B.dd4_lloyd_launches(M, K, 1 << n_bits, B.LLOYD_GRID_DP) if self.grid_dp
                                    else B.dd4_lloyd_launches(M, K, lloyd_iters))
 
-    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True, reuse_prepass: bool = False) -> None:
+    def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True, reuse_prepass: bool = False,
+            codes: Optional[torch.Tensor] = None, words: Optional[torch.Tensor] = None) -> None:
         """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32.  ``norms`` =
         False skips the channel norms: they do not depend on the scale format, so a sweep that shares the
         buffers of another one (same layer, other format) uses the norms that one has just computed.
         ``reuse_prepass``: the same holds for the exponent histogram of the block scales behind the per-layer
         shift: the search takes it from the shared workspace as the sweep of this layer at the previous format
-        left it, and only derives this format's shifts."""
+        left it, and only derives this format's shifts.  ``codes`` / ``words``: buffers of the sizes of ``self.codes`` /
+        ``self.words`` that receive the packed layer instead of them (a stream hands in the slot the result leaves from)."""
+        codes = self.codes if codes is None else codes
+        words = self.words if words is None else words
         n = 0
         if norms:
             B.sop_channel_norms(X, self.c, self.ws_norm, stream)
@@ -203,14 +207,14 @@ class LayerSweep:
                               reuse_prepass=reuse_prepass)
             n += 1
         n += 2
-        B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, search_result=self.result,
+        B.sop_pack(W, self.c, self.fmt_c, self.atoms_c, codes, words, search_result=self.result,
                    index_a=0 if self.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if self.single else B.PAIR_FROM_RESULT,
                    use_sign=self.use_sign, container_bits=self.container, word_sign_bits=self.use_sign,
                    counts=self.counts, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
                    block_cos=self.full_cos, stream=stream)
         n += 1
         if self.wr_keep:
-            B.sop_wr_extract(W, self.c, self.fmt_c, self.atoms_c, self.codes, self.words, self.wr_keep, self.wr_row_start,
+            B.sop_wr_extract(W, self.c, self.fmt_c, self.atoms_c, codes, words, self.wr_keep, self.wr_row_start,
                              self.wr_records, self.wr_count, self.wr_exp, self.ws_wr, tau=self.wr_tau,
                              index_a=0 if self.single else B.PAIR_FROM_RESULT, index_b=B.NO_ATOM if self.single else B.PAIR_FROM_RESULT,
                              search_result=self.result, use_sign=self.use_sign, container_bits=self.container,
@@ -286,18 +290,23 @@ class LayerStream:
     codes, words, distortion) that stay valid until ``submit(i + 2)`` -- one dict for a single sweep, a list
     of dicts (one per sweep) otherwise; it raises ``binding.LloydNotFinished`` when a Lloyd call of the layer
     reports that it did not run to its end.  ``streams`` hands in the three CUDA streams (copy in, compute,
-    copy out) so that several LayerStream objects, one per layer shape, work as one ordered pipeline."""
+    copy out) so that several LayerStream objects, one per layer shape, work as one ordered pipeline.  The packer
+    writes codes and scale words straight into the slot they leave the device from.  ``graphs`` = True records
+    the calls of every (slot, format) into a CUDA graph once (on zero-filled slots) and replays it per layer: no
+    gaps between the dozen launches of a pass."""
 
     OUT = ("pair_table", "signed_table", "result", "codes", "words", "distortion")
 
-    def __init__(self, sweep, streams=None):
+    SMALL = ("pair_table", "signed_table", "result", "distortion")      # copied aside; codes and words are packed in place
+
+    def __init__(self, sweep, streams=None, graphs: bool = False):
         self.single = isinstance(sweep, LayerSweep)
         self.sweeps = [sweep] if self.single else list(sweep)
         sw = self.sw = self.sweeps[0]
         d = sw.dev
         self.s_in, self.s_run, self.s_out = streams if streams is not None else (torch.cuda.Stream(d), torch.cuda.Stream(d), torch.cuda.Stream(d))
-        self.W = [torch.empty((sw.M, sw.K), dtype=torch.bfloat16, device=d) for _ in range(2)]
-        self.X = [torch.empty((sw.T, sw.K), dtype=torch.float32, device=d) for _ in range(2)]
+        self.W = [torch.zeros((sw.M, sw.K), dtype=torch.bfloat16, device=d) for _ in range(2)]
+        self.X = [torch.zeros((sw.T, sw.K), dtype=torch.float32, device=d) for _ in range(2)]
         self.dev_out = [[{k: torch.empty_like(getattr(q, k)) for k in self.OUT} for q in self.sweeps] for _ in range(2)]
         self.host_out = [[{k: torch.empty(getattr(q, k).shape, dtype=getattr(q, k).dtype).pin_memory() for k in self.OUT}
                           for q in self.sweeps] for _ in range(2)]
@@ -308,6 +317,35 @@ class LayerStream:
         self.d2h_bytes = sum(t.numel() * t.element_size() for o in self.dev_out[0] for t in o.values())
         self.before_run = None       # optional callable run on the compute stream before every layer
         self.n_submitted = 0
+        self.graphs = None
+        if graphs:
+            torch.cuda.synchronize(d)
+            for slot in range(2):                 # the library's one-time set-ups happen outside the captures
+                self._run_slot(slot, self.s_run)
+            torch.cuda.synchronize(d)
+            self.graphs = [[None] * len(self.sweeps) for _ in range(2)]
+            side = torch.cuda.Stream(d)
+            for slot in range(2):
+                for f in range(len(self.sweeps)):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        self._run_format(slot, f, side)
+                    self.graphs[slot][f] = g
+            torch.cuda.synchronize(d)
+
+    def _run_format(self, slot: int, f: int, stream) -> None:
+        """The calls of one format on the layer in ``slot``, on ``stream``: the pass (packed output straight into the
+        slot's buffers), then the small results set aside before the next format overwrites them."""
+        q = self.sweeps[f]
+        out = self.dev_out[slot][f]
+        q.run(self.W[slot], self.X[slot], stream, norms=(f == 0), reuse_prepass=(f > 0), codes=out["codes"], words=out["words"])
+        with torch.cuda.stream(stream):
+            for k in self.SMALL:
+                out[k].copy_(getattr(q, k), non_blocking=True)
+
+    def _run_slot(self, slot: int, stream) -> None:
+        for f in range(len(self.sweeps)):
+            self._run_format(slot, f, stream)
 
     def submit(self, i: int, W_host: torch.Tensor, X_host: torch.Tensor) -> None:
         slot = i & 1
@@ -323,11 +361,11 @@ class LayerStream:
                 self.s_run.wait_event(self.out_done[slot])    # the results of layer i - 2 have left this slot
             if self.before_run is not None:
                 self.before_run()
-            for f, q in enumerate(self.sweeps):
-                q.run(self.W[slot], self.X[slot], self.s_run, norms=(f == 0), reuse_prepass=(f > 0))
-                # the sweeps share their packed output: it is set aside before the next format overwrites it
-                for k in self.OUT:
-                    self.dev_out[slot][f][k].copy_(getattr(q, k), non_blocking=True)
+            for f in range(len(self.sweeps)):
+                if self.graphs is not None:
+                    self.graphs[slot][f].replay()
+                else:
+                    self._run_format(slot, f, self.s_run)
                 self.out_ready[slot][f].record(self.s_run)
             self.in_free[slot].record(self.s_run)
         with torch.cuda.stream(self.s_out):

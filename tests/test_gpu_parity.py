@@ -380,20 +380,21 @@ def test_pipeline_matches_oracle(B, fmt_name, rom, fp, iters, shape):
     assert (int(got.counts[0]), int(got.counts[1])) == (pk["n_sel1"], pk["n_neg"])
 
 
-def test_layer_stream_returns_each_layers_own_results(B):
-    # three different layers through the overlapped host -> device -> host stream: every layer's results
-    # equal those of a plain run on that layer
+@pytest.mark.parametrize("graphs", [False, True])
+def test_layer_stream_returns_each_layers_own_results(B, graphs):
+    # five different layers through the overlapped host -> device -> host stream (every slot is used again): every
+    # layer's results equal those of a plain run on that layer, launched call by call or as recorded CUDA graphs
     from paper_2605_14929_b200.pipeline import LayerStream, LayerSweep
     fmt = I.scale_format("S1E4M4")
     M, K, T = 48, 512, 64
-    layers = [I.outlier_channel_layer(40 + i, M, K, T) for i in range(3)]
+    layers = [I.outlier_channel_layer(40 + i, M, K, T) for i in range(5)]
     sw = LayerSweep(M, K, T, fmt, ["NF4", "SH4"], [], 4, device=dev())
     want = []
     for L in layers:
         sw.run(L.W.to(dev()), L.X.to(dev()))
         torch.cuda.synchronize()
         want.append({k: getattr(sw, k).cpu().clone() for k in LayerStream.OUT})
-    ls = LayerStream(sw)
+    ls = LayerStream(sw, graphs=graphs)
     host = [(L.W.pin_memory(), L.X.pin_memory()) for L in layers]
     got = []
     for i, (Wh, Xh) in enumerate(host):
@@ -402,7 +403,7 @@ def test_layer_stream_returns_each_layers_own_results(B):
             got.append({k: v.clone() for k, v in ls.collect(i - 1).items()})
     got.append({k: v.clone() for k, v in ls.collect(len(host) - 1).items()})
     assert ls.h2d_bytes == M * K * 2 + T * K * 4
-    for i in range(3):
+    for i in range(5):
         for k in LayerStream.OUT:
             if k == "distortion":       # an FP64 sum in scheduling order: equal to rounding, not bit for bit
                 assert torch.allclose(got[i][k], want[i][k], rtol=1e-9, atol=0), (i, k)
@@ -448,3 +449,37 @@ def test_graph_replay_equals_the_calls(B):
             assert torch.allclose(sw.distortion.cpu(), want[k], rtol=1e-9, atol=0)
         else:
             assert torch.equal(getattr(sw, k).cpu(), want[k]), k
+
+
+@pytest.mark.parametrize("graphs", [False, True])
+def test_layer_stream_over_several_scale_formats(B, graphs):
+    # one layer shape at three scale formats whose sweeps share the large buffers, the channel norms and the exponent
+    # histogram: every (layer, format) result equals that of a sweep of its own
+    from paper_2605_14929_b200.pipeline import LayerStream, LayerSweep
+    M, K, T = 40, 768, 64
+    fmts = [I.scale_format(f) for f in ("UE4M4", "E5M6", "E4M3")]
+    layers = [I.student_layer(60 + i, 0, M, K, T, 4.0, channel_sigma=0.8) for i in range(3)]
+    row, first = [], None
+    for fmt in fmts:
+        sw = LayerSweep(M, K, T, fmt, ["NF4", "SH4", "BOF4"], [], 3, device=dev(), share=first)
+        first = first or sw
+        row.append(sw)
+    ls = LayerStream(row, graphs=graphs)
+    host = [(L.W.pin_memory(), L.X.pin_memory()) for L in layers]
+    got = []
+    for i, (Wh, Xh) in enumerate(host):
+        ls.submit(i, Wh, Xh)
+        if i:
+            got.append([{k: v.clone() for k, v in o.items()} for o in ls.collect(i - 1)])
+    got.append([{k: v.clone() for k, v in o.items()} for o in ls.collect(len(host) - 1)])
+    for i, L in enumerate(layers):
+        for f, fmt in enumerate(fmts):
+            own = LayerSweep(M, K, T, fmt, ["NF4", "SH4", "BOF4"], [], 3, device=dev())
+            own.run(L.W.to(dev()), L.X.to(dev()))
+            torch.cuda.synchronize()
+            for k in LayerStream.OUT:
+                w = getattr(own, k).cpu()
+                if k == "distortion":
+                    assert torch.allclose(got[i][f][k], w, rtol=1e-9, atol=0), (i, f, k)
+                else:
+                    assert torch.equal(got[i][f][k], w), (i, f, k)
