@@ -311,7 +311,7 @@ def sparse_streams_table(dev, hbm_peak, of, flush):
     E = M * K
     opq_ms, wr_ms, all_ms = sorted(t_opq)[2], sorted(t_wr)[2], sorted(t_all)[2]
     opq_bytes = (2.0 + 2.0 + 2 * 2.0 / 16.0) * E + 4.0 * sp["opq"]["count"]
-    wr_bytes = 6 * (2.0 + 0.5 + sw.container / 8.0 / 16.0) * E + 4.0 * sp["wr"]["count"]
+    wr_bytes = 2 * (2.0 + 0.5 + sw.container / 8.0 / 16.0) * E + 4.0 * sp["wr"]["count"]
 
     def hbm(b, ms):
         return dict(achieved=b / (ms * 1e-3) / 1e9, peak=hbm_peak, unit="GB/s", frac=b / (ms * 1e-3) / 1e9 / hbm_peak, of=of)
@@ -321,8 +321,10 @@ def sparse_streams_table(dev, hbm_peak, of, flush):
                          note="three launches: mask + zeroed copy (W read once, written once), scan of the tile counts, records"),
                 wr=dict(ms=wr_ms, records=sp["wr"]["count"], n_keep=sp["wr"]["n_keep"], scale_exp=sp["wr"]["scale_exp"],
                         bpw=32.0 * sp["wr"]["count"] / E, algorithmic_bytes=wr_bytes, hbm=hbm(wr_bytes, wr_ms),
-                        note="eleven launches: block-maximum pass, three selection passes, count, scan, write; every pass decodes W, codes and scale "
-                             "words (2.6 bytes per element) instead of reading a stored residual"),
+                        note="two passes decode W, codes and scale words (2.6 bytes per element) into the residual: block maxima, then the "
+                             "candidates above the bound they give; threshold, kept set and counts come from the candidate list, the "
+                             "write pass decodes only blocks with a kept entry (eighteen launches, seven of them the unused "
+                             "full-decode path that returns at once)"),
                 whole_path_ms=all_ms, whole_path_value=E / all_ms / 1e6)
 
 

@@ -382,8 +382,12 @@ int sop_opq_extract(const void* W_dev, long long M, long long K, long long ldw, 
  *     row_start_dev [M + 1], records_dev [capacity], count_dev as there.  scale_exp_dev: one int, e (0 when
  *     nothing is kept).  tau_dev (may be NULL): one float, tau.
  *   workspace_dev: sop_wr_workspace bytes, 256-byte aligned.
- * The residual is recomputed in each of the six passes (block maxima, three selection passes, count, write)
- * rather than stored: W, codes and scale words are 2.6 bytes per element, a stored residual 4. */
+ * The residual is never stored (W, codes and scale words are 2.6 bytes per element, a stored residual 4): one
+ * decode pass histograms the block maxima of the metric, which bounds the threshold from below; a second one
+ * collects the elements above that bound (typically a fraction of a per cent) into a candidate list in the
+ * workspace, from which the threshold, the kept set and the stream follow.  A layer whose candidates do not fit
+ * the list (more than max(65536, M K / 64): metrics nearly all alike) is handled by full decode passes instead;
+ * the results are the same. */
 int sop_wr_workspace(long long M, long long K, size_t* bytes);
 int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                    const sop_scale_fmt* fmt, const sop_atom* atoms, int n_atoms, const float* dd_lut_dev, unsigned dd_mask,

@@ -20,8 +20,15 @@
 //                       value's bin or an earlier one and pass 0 skips every element of a later bin (all but a few
 //                       per cent: shared-memory atomics on a handful of hot bins would otherwise dominate)
 //   wr_pick_kernel      after each pass: the bin that holds the rank, the prefix for the next pass
-//   wr_count_kernel     per-tile counts of kept entries (metric >= tau, metric > 0), max |E| over them
-//   wr_write_kernel     E3M4 codes of E / 2^e, records (column | code << 16)
+//   wr_collect_kernel   second decode pass: every element whose bin is not later than that of the n_keep-th largest
+//                       block maximum goes to a candidate list (position, residual, metric): a fraction of a per cent
+//                       of the layer.  The threshold, the kept set (a bitmap), the largest kept |E| and the per-tile
+//                       counts then come from the list (wr_cand_hist_kernel, wr_mark_kernel);
+//                       the write pass decodes only the blocks that hold a kept entry.
+//   wr_hist_kernel<0,1,2>, wr_count_kernel, wr_write_kernel<.., false>
+//                       the same steps as full decode passes: taken when the candidates do not fit their list (a
+//                       layer whose metrics are nearly all alike).  Both sets of launches are enqueued; the set
+//                       that is not needed returns at once (flag in the workspace, set on the device).
 // The residual is never stored: decoding a block (2.6 bytes per element read) is cheaper than reading 4 bytes.
 #include <math.h>
 #include <string.h>
@@ -44,12 +51,17 @@ struct SparseWs {
   unsigned emax_bits;             // max |E| over the kept entries, fp32 bits
   int scale_exp;
   int no_pair;                    // the search result holds no pair: nothing was packed, nothing is corrected
-  unsigned pad;
+  unsigned n_cand;                // candidates found (may exceed the list's capacity: then the list is not used)
+  unsigned overflow;              // 1: the candidates did not fit, the full decode passes do the work
+  unsigned pad[3];
 };
 
 static size_t sparse_tiles_off() { return (sizeof(SparseWs) + 255) & ~(size_t)255; }
 static long long sparse_tiles(long long NB) { return (NB + STB - 1) / STB; }
 static size_t sparse_masks_off(long long NB) { return sparse_tiles_off() + (((size_t)sparse_tiles(NB) * 4 + 255) & ~(size_t)255); }
+// Wr: behind the per-block masks the candidate list, three 32-bit arrays of wr_cand_cap entries
+static size_t wr_cand_off(long long NB) { return sparse_masks_off(NB) + (((size_t)NB * 2 + 255) & ~(size_t)255); }
+static unsigned wr_cand_cap(long long NB) { const long long c = NB / 4; return (unsigned)(c > 65536 ? c : 65536); }   // 1/64 of the elements
 
 // exclusive prefix sum of one value per thread over the CTA (STB threads); *total = the CTA's sum
 __device__ __forceinline__ unsigned cta_excl_scan(unsigned v, unsigned* s_warp, unsigned* total) {
@@ -213,6 +225,11 @@ struct WrArgs {
   unsigned* row_start;
   unsigned* records;
   long long capacity;
+  unsigned short* kept;           // workspace: per block the 16-bit mask of kept entries (candidate path)
+  unsigned* cand_pos;             // workspace: candidate list: element position blk * 16 + i,
+  unsigned* cand_e;               //   residual bits,
+  unsigned* cand_m;               //   metric bits
+  unsigned cand_cap;
 };
 
 struct WrCand { int kind, neg, scope, k, sign_pos, y, bias; float tmax; };
@@ -372,6 +389,7 @@ __global__ void __launch_bounds__(STB) wr_hist_kernel(WrArgs a, AtomsDev A, FmtD
   __shared__ WrShared sh;
   __shared__ unsigned hist[2048];
   const int tid = threadIdx.x;
+  if (PASS >= 0 && !ws->overflow) return;          // the candidate list serves the selection
   for (int i = tid; i < 2048; i += STB) hist[i] = 0;
   if (tid == 0) wr_setup(a, A, res, sh);
   __syncthreads();
@@ -463,15 +481,131 @@ __global__ void __launch_bounds__(1024) wr_pick_kernel(SparseWs* __restrict__ ws
 
 __device__ __forceinline__ bool wr_kept(float met, float tau) { return met >= tau && met > 0.0f; }
 
+// The stored value of a residual: the E3M4 code (bias 3, 4 mantissa bits, largest 15.5) of E / 2^e.  The quotient is
+// formed by two exact multiplications by powers of two (|E| / 2^e <= 15.5; a quotient below the fp32 normal range is
+// far below half the smallest E3M4 step and rounds to zero either way).
+struct WrValue {
+  float f1, f2;
+  GridDev g;
+  __device__ explicit WrValue(int e) {
+    const int e1 = max(-100, min(100, -e));
+    f1 = pow2f_int(e1); f2 = pow2f_int(max(-120, min(120, -e - e1)));
+    g.min_eb = 125; g.sh = 19; g.vpos = 15.5f; g.vneg = 15.5f;
+  }
+  __device__ __forceinline__ uint32_t code(float E) const {
+    return grid_code(grid_quantize(__fmul_rn(__fmul_rn(E, f1), f2), g), g, 7);
+  }
+};
+
+// Second decode pass: the candidates.  A thread counts its block's candidates, the warp reserves room for all of them
+// with one addition to the list's counter, every thread writes its own.  Beyond the capacity nothing is written; the
+// counter keeps counting, which is how the overflow is seen.
+template <bool LUT4>
+__global__ void __launch_bounds__(STB) wr_collect_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
+                                                         SparseWs* __restrict__ ws) {
+  __shared__ WrShared sh;
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid == 0) wr_setup(a, A, res, sh);
+  __syncthreads();
+  if (blockIdx.x == 0 && tid == 0) ws->no_pair = sh.no_pair;
+  if (sh.no_pair) return;
+  const unsigned bm_bin = ws->bm_bin;
+  const long long n_tiles = (a.NB + STB - 1) / STB;
+  for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const long long blk = tile * STB + tid;
+    float E[16], met[16];
+    unsigned in = 0;
+    if (blk < a.NB) {
+      const long long m = (long long)((unsigned)blk / (unsigned)a.nbk), j = blk - m * a.nbk;
+      wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+      float bm = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) bm = fmaxf(bm, met[i]);
+      if ((wr_key(bm) >> 21) <= bm_bin) {            // few blocks reach the bound at all
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if ((wr_key(met[i]) >> 21) <= bm_bin) in |= 1u << i;
+      }
+    }
+    if (!__any_sync(0xFFFFFFFFu, in != 0u)) continue;
+    const unsigned mine = (unsigned)__popc(in);
+    unsigned incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    const unsigned total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    unsigned base = 0;
+    if (lane == 31 && total) base = atomicAdd(&ws->n_cand, total);
+    base = __shfl_sync(0xFFFFFFFFu, base, 31);
+    unsigned at = base + incl - mine;
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if ((in >> i) & 1u) {
+        if (at < a.cand_cap) {
+          a.cand_pos[at] = (unsigned)blk * 16u + (unsigned)i;
+          a.cand_e[at] = __float_as_uint(E[i]);
+          a.cand_m[at] = __float_as_uint(met[i]);
+        }
+        ++at;
+      }
+  }
+}
+
+__global__ void wr_mode_kernel(SparseWs* __restrict__ ws, unsigned cand_cap) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) ws->overflow = ws->n_cand > cand_cap ? 1u : 0u;
+}
+
+// The selection passes over the candidate list instead of the layer.
+template <int PASS>
+__global__ void __launch_bounds__(STB) wr_cand_hist_kernel(WrArgs a, SparseWs* __restrict__ ws) {
+  __shared__ unsigned hist[2048];
+  if (ws->overflow) return;
+  const int tid = threadIdx.x;
+  for (int i = tid; i < 2048; i += STB) hist[i] = 0;
+  __syncthreads();
+  const unsigned n = ws->n_cand, prefix = PASS > 0 ? ws->prefix : 0u;
+  for (unsigned i = blockIdx.x * STB + tid; i < n; i += gridDim.x * STB) {
+    const unsigned key = wr_key(__uint_as_float(a.cand_m[i]));
+    if (PASS == 0) atomicAdd(&hist[key >> 21], 1u);
+    else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&hist[(key >> 10) & 2047u], 1u); }
+    else { if ((key >> 10) == prefix) atomicAdd(&hist[key & 1023u], 1u); }
+  }
+  __syncthreads();
+  for (int i = tid; i < 2048; i += STB)
+    if (hist[i]) atomicAdd(&ws->hist[PASS][i], hist[i]);
+}
+
+// The kept candidates: their bit in the per-block masks (two blocks per 32-bit word), their tile's record count (cleared
+// by the host call), the largest |E| among them.
+__global__ void __launch_bounds__(STB) wr_mark_kernel(WrArgs a, SparseWs* __restrict__ ws) {
+  if (ws->overflow) return;
+  const float tau = __uint_as_float(ws->tau_bits);
+  const unsigned n = ws->n_cand;
+  unsigned emax = 0;
+  unsigned* map = reinterpret_cast<unsigned*>(a.kept);
+  for (unsigned i = blockIdx.x * STB + threadIdx.x; i < n; i += gridDim.x * STB) {
+    if (!wr_kept(__uint_as_float(a.cand_m[i]), tau)) continue;
+    const unsigned pos = a.cand_pos[i];
+    atomicOr(&map[pos >> 5], 1u << (pos & 31u));
+    atomicAdd(&a.tile_sums[pos >> 12], 1u);          // a tile is 256 blocks of 16 elements
+    emax = max(emax, a.cand_e[i] & 0x7FFFFFFFu);
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, o));
+  if ((threadIdx.x & 31) == 0 && emax) atomicMax(&ws->emax_bits, emax);
+}
+
 template <bool LUT4>
 __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
                                                        SparseWs* __restrict__ ws) {
   __shared__ WrShared sh;
   __shared__ unsigned s_cnt;
   const int tid = threadIdx.x;
+  if (!ws->overflow) return;
   if (tid == 0) wr_setup(a, A, res, sh);
   __syncthreads();
-  if (blockIdx.x == 0 && tid == 0) ws->no_pair = sh.no_pair;
   const float tau = __uint_as_float(ws->tau_bits);
   const long long n_tiles = (a.NB + STB - 1) / STB;
   unsigned emax = 0;
@@ -500,36 +634,32 @@ __global__ void __launch_bounds__(STB) wr_count_kernel(WrArgs a, AtomsDev A, Fmt
   if ((tid & 31) == 0 && emax) atomicMax(&ws->emax_bits, emax);
 }
 
+// The full-decode write pass: every block is decoded and its entries are compared with the threshold.
 template <bool LUT4>
 __global__ void __launch_bounds__(STB) wr_write_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
                                                        const SparseWs* __restrict__ ws) {
   __shared__ WrShared sh;
   __shared__ unsigned s_warp[STB / 32];
   const int tid = threadIdx.x;
+  if (!ws->overflow) return;
   if (tid == 0) wr_setup(a, A, res, sh);
   __syncthreads();
   const float tau = __uint_as_float(ws->tau_bits);
-  const int e = ws->scale_exp;
-  // E / 2^e as two exact multiplications by powers of two (|E| / 2^e <= 15.5; a quotient below the fp32 normal
-  // range is far below half the smallest E3M4 step and rounds to zero either way)
-  const int e1 = max(-100, min(100, -e));
-  const float f1 = pow2f_int(e1), f2 = pow2f_int(max(-120, min(120, -e - e1)));
-  GridDev G3;
-  G3.min_eb = 125; G3.sh = 19; G3.vpos = 15.5f; G3.vneg = 15.5f;      // E3M4: bias 3, 4 mantissa bits, largest 15.5
+  const WrValue V(ws->scale_exp);
   const long long n_tiles = (a.NB + STB - 1) / STB;
   for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const long long blk = tile * STB + tid;
     float E[16], met[16];
     unsigned keep = 0;
     long long m = 0, j = 0;
-    if (blk < a.NB && !sh.no_pair) {
+    if (blk < a.NB) {
       m = (long long)((unsigned)blk / (unsigned)a.nbk); j = blk - m * a.nbk;
-      wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
+      if (!sh.no_pair) {
+        wr_block<LUT4>(a, F, sh, blk, j, a.W + m * a.ldw + j * SOP_G, E, met);
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
-        if (wr_kept(met[i], tau)) keep |= 1u << i;
-    } else if (blk < a.NB) {
-      m = (long long)((unsigned)blk / (unsigned)a.nbk); j = blk - m * a.nbk;
+        for (int i = 0; i < 16; ++i)
+          if (wr_kept(met[i], tau)) keep |= 1u << i;
+      }
     }
     unsigned tot;
     const unsigned excl = cta_excl_scan((unsigned)__popc(keep), s_warp, &tot);
@@ -539,11 +669,61 @@ __global__ void __launch_bounds__(STB) wr_write_kernel(WrArgs a, AtomsDev A, Fmt
 #pragma unroll
     for (int i = 0; i < 16; ++i)
       if ((keep >> i) & 1u) {
-        const float x = __fmul_rn(__fmul_rn(E[i], f1), f2);
-        const uint32_t code = grid_code(grid_quantize(x, G3), G3, 7);
-        if ((long long)pos < a.capacity) a.records[pos] = (unsigned)(j * SOP_G + i) | (code << 16);
+        if ((long long)pos < a.capacity) a.records[pos] = (unsigned)(j * SOP_G + i) | (V.code(E[i]) << 16);
         ++pos;
       }
+  }
+}
+
+// The write pass of the candidate path: the kept entries come from the per-block masks.  Every thread scans its
+// block's count; the few blocks of a tile that hold a kept entry are put on a list in shared memory and decoded by the
+// first threads of the CTA, so that a warp does not run a decode for one lane.
+template <bool LUT4>
+__global__ void __launch_bounds__(STB) wr_map_write_kernel(WrArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res,
+                                                           const SparseWs* __restrict__ ws) {
+  __shared__ WrShared sh;
+  __shared__ unsigned s_warp[STB / 32];
+  __shared__ unsigned s_n;
+  __shared__ unsigned s_pos[STB];          // per listed block: its first record
+  __shared__ unsigned short s_blk[STB], s_keep[STB];
+  const int tid = threadIdx.x;
+  if (ws->overflow) return;
+  if (tid == 0) { wr_setup(a, A, res, sh); s_n = 0; }
+  __syncthreads();
+  const WrValue V(ws->scale_exp);
+  const long long n_tiles = (a.NB + STB - 1) / STB;
+  for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const long long blk = tile * STB + tid;
+    const unsigned keep = blk < a.NB && !sh.no_pair ? (unsigned)a.kept[blk] : 0u;
+    unsigned tot;
+    const unsigned excl = cta_excl_scan((unsigned)__popc(keep), s_warp, &tot);        // (two barriers)
+    if (blk < a.NB) {
+      const unsigned pos = a.tile_sums[tile] + excl;
+      const long long m = (long long)((unsigned)blk / (unsigned)a.nbk);
+      if (blk - m * a.nbk == 0) a.row_start[m] = pos;
+      if (keep) {
+        const unsigned at = atomicAdd(&s_n, 1u);
+        s_pos[at] = pos; s_blk[at] = (unsigned short)tid; s_keep[at] = (unsigned short)keep;
+      }
+    }
+    __syncthreads();
+    const unsigned n = s_n;
+    for (unsigned q = tid; q < n; q += STB) {
+      const long long b = tile * STB + s_blk[q];
+      const long long m = (long long)((unsigned)b / (unsigned)a.nbk), j = b - m * a.nbk;
+      float E[16], met[16];
+      wr_block<LUT4>(a, F, sh, b, j, a.W + m * a.ldw + j * SOP_G, E, met);
+      unsigned pos = s_pos[q];
+      const unsigned k = s_keep[q];
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        if ((k >> i) & 1u) {
+          if ((long long)pos < a.capacity) a.records[pos] = (unsigned)(j * SOP_G + i) | (V.code(E[i]) << 16);
+          ++pos;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) s_n = 0;                  // read again only after the next tile's scan barriers
   }
 }
 
@@ -611,7 +791,8 @@ int sop_opq_extract(const void* W_dev, long long M, long long K, long long ldw, 
 int sop_wr_workspace(long long M, long long K, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
   if (M < 1 || K < 1 || (K % SOP_G) != 0 || M > (1ll << 31) / (K / SOP_G)) return SOP_ERR_SHAPE;
-  *bytes = sop::sparse_masks_off(M * (K / SOP_G));
+  const long long NB = M * (K / SOP_G);
+  *bytes = sop::wr_cand_off(NB) + 3 * (((size_t)sop::wr_cand_cap(NB) * 4 + 255) & ~(size_t)255);
   return SOP_OK;
 }
 
@@ -676,9 +857,20 @@ int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, c
   SparseWs* ws = (SparseWs*)workspace_dev;
   a.tile_sums = (unsigned*)(wsb + sparse_tiles_off());
   a.row_start = row_start_dev; a.records = records_dev; a.capacity = capacity;
+  a.kept = (unsigned short*)(wsb + sparse_masks_off(a.NB));
+  a.cand_cap = wr_cand_cap(a.NB);
+  {
+    const size_t one = ((size_t)a.cand_cap * 4 + 255) & ~(size_t)255;
+    a.cand_pos = (unsigned*)(wsb + wr_cand_off(a.NB));
+    a.cand_e = (unsigned*)(wsb + wr_cand_off(a.NB) + one);
+    a.cand_m = (unsigned*)(wsb + wr_cand_off(a.NB) + 2 * one);
+  }
   cudaStream_t st = (cudaStream_t)stream;
   const long long n_tiles = sparse_tiles(a.NB);
   const long long cap = (long long)num_sms() * 6;
+  const int lgrid = num_sms() * 2;                       // the kernels over the candidate list
+  SOP_CUDA_TRY(cudaMemsetAsync(a.kept, 0, ((size_t)a.NB * 2 + 3) & ~(size_t)3, st));
+  SOP_CUDA_TRY(cudaMemsetAsync(a.tile_sums, 0, (size_t)n_tiles * 4, st));
   const int grid = (int)(n_tiles < cap ? n_tiles : cap);
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(SparseWs), st));
   if ((rc = profile_mark(SOP_PROFILE_WR, 0, st))) return rc;
@@ -696,14 +888,21 @@ int sop_wr_extract(const void* W_dev, long long M, long long K, long long ldw, c
   do {                                                                               \
     wr_hist_kernel<-1, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);           \
     wr_pick_kernel<<<1, 1024, 0, st>>>(ws, -1, n_keep);                              \
+    wr_collect_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
+    wr_mode_kernel<<<1, 32, 0, st>>>(ws, a.cand_cap);                                \
+    wr_cand_hist_kernel<0><<<lgrid, STB, 0, st>>>(a, ws);                            \
     wr_hist_kernel<0, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
     wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 0, n_keep);                               \
+    wr_cand_hist_kernel<1><<<lgrid, STB, 0, st>>>(a, ws);                            \
     wr_hist_kernel<1, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
     wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 1, n_keep);                               \
+    wr_cand_hist_kernel<2><<<lgrid, STB, 0, st>>>(a, ws);                            \
     wr_hist_kernel<2, L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);            \
     wr_pick_kernel<<<1, 1024, 0, st>>>(ws, 2, n_keep);                               \
+    wr_mark_kernel<<<lgrid, STB, 0, st>>>(a, ws);                                    \
     wr_count_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);              \
     tile_scan_kernel<<<1, 1024, 0, st>>>(a.tile_sums, n_tiles, row_start_dev, M, count_dev, ws, 1, scale_exp_dev, tau_dev); \
+    wr_map_write_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);          \
     wr_write_kernel<L4><<<grid, STB, 0, st>>>(a, A, F, search_dev, ws);              \
   } while (0)
   if (lut4) SOP_WR_LAUNCHES(true); else SOP_WR_LAUNCHES(false);

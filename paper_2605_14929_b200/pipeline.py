@@ -220,7 +220,7 @@ class LayerSweep:
                              search_result=self.result, use_sign=self.use_sign, container_bits=self.container,
                              word_sign_bits=self.use_sign, dd_lut=self.dd_lut if self.dd_mask else None, dd_mask=self.dd_mask,
                              stream=stream)
-            n += 11
+            n += 18
         self.kernel_launches_per_step = n
 
     def capture(self, W: torch.Tensor, X: torch.Tensor) -> None:

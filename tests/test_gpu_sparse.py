@@ -233,3 +233,26 @@ def test_wr_on_wider_codes_and_element_formats(rom, fp, fmt_name, iters):
     want = oracle_wr(L, fmt, out, sw, n_keep)
     assert got["count"] == want["count"] >= n_keep and got["scale_exp"] == want["scale_exp"]
     assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
+
+
+def test_wr_when_the_candidates_do_not_fit_their_list():
+    """A layer whose residuals are all alike: every element lies in the bin of the block maxima, the candidate list
+    (65536 entries here) overflows and the full decode passes take over.  The metrics differ through the channel
+    norms only, so the threshold cuts between columns."""
+    d = dev()
+    M, K, T = 128, 2048, 16
+    W = torch.full((M, K), 1.0078125, dtype=torch.bfloat16)            # 1 + 2^-7: the 6-bit scale mantissa rounds it to 1
+    X = (1.0 + 0.2 * torch.arange(K, dtype=torch.float32) / K).repeat(T, 1).contiguous()
+    L = I.Layer(W, X)
+    fmt = I.scale_format("E5M6")
+    n_keep = 5000
+    sw, out, got = run_wr(L, fmt, ["NF4", "SH4"], n_keep, None)
+    want = oracle_wr(L, fmt, out, sw, n_keep)
+    assert want["count"] >= n_keep and want["count"] % M == 0 and want["count"] < M * K // 8        # whole columns, a small share
+    assert got["count"] == want["count"] and got["scale_exp"] == want["scale_exp"]
+    assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
+    # the same layer with equal channel norms: every metric ties, everything is kept
+    L1 = I.Layer(W, torch.ones(T, K))
+    sw, out, got = run_wr(L1, fmt, ["NF4", "SH4"], 100, None)
+    want = oracle_wr(L1, fmt, out, sw, 100)
+    assert got["count"] == want["count"] == M * K and np.array_equal(got["records"], want["records"])
