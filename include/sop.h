@@ -198,6 +198,10 @@ int sop_channel_norms_static(const float* X_dev, long long T, long long K, long 
  *   instead of reading W once more; every per-block-scaled class of this call must then contain a
  *   candidate of load_mask (SOP_ERR_RANGE otherwise). */
 int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes);
+/* Launch shape of the reduction of the table entries (no counterpart in the paper): reduce_tile_pairs = 1 (the
+ * default) lets a CTA work on two tiles of 256 blocks at a time where its shared memory allows, 0 keeps it to one.
+ * The additions and their order are the same: results do not depend on it.  SOP_ERR_RANGE for other values. */
+int sop_pair_search_tuning(int reduce_tile_pairs);
 int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, const float* c_dev, int g,
                     const sop_scale_fmt* fmt, int k_mode, const sop_atom* atoms, int n_atoms,
                     const float* dd_lut_dev, unsigned dd_mask, unsigned eval_mask, unsigned load_mask, int flags,

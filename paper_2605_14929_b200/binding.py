@@ -84,7 +84,7 @@ def lib():
 def exported_symbols():
     return ["sop_strerror", "sop_last_cuda_error", "sop_version", "sop_channel_norms_workspace", "sop_channel_norms",
             "sop_channel_norms_static",
-            "sop_pair_search_workspace", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd_tuning",
+            "sop_pair_search_workspace", "sop_pair_search_tuning", "sop_pair_search", "sop_dd4_lloyd_workspace", "sop_dd4_lloyd_launches", "sop_dd4_lloyd_tuning",
             "sop_dd4_lloyd", "sop_pack", "sop_opq_threshold", "sop_opq_workspace", "sop_opq_extract", "sop_wr_workspace",
             "sop_wr_extract",
             "sop_profile_enable", "sop_profile_ms", "sop_profile_last_ms", "sop_profile_last_sweep_ms"]
@@ -308,6 +308,11 @@ def sop_wr_extract(W: torch.Tensor, c: torch.Tensor, fmt, atoms: Sequence, codes
                                 container_bits, word_sign_bits, _ptr(codes), _ptr(words), _ll(n_keep), _ptr(row_start),
                                 _ptr(records), _ll(0 if records is None else records.numel()), _ptr(count), _ptr(scale_exp),
                                 _ptr(tau), _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)), "sop_wr_extract")
+
+
+def pair_search_tuning(reduce_tile_pairs: bool = True) -> None:
+    """Launch shape of the reduction kernel (results do not depend on it)."""
+    _check(lib().sop_pair_search_tuning(1 if reduce_tile_pairs else 0), "sop_pair_search_tuning")
 
 
 def profile_enable(on: bool) -> None:

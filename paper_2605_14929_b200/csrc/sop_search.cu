@@ -589,23 +589,30 @@ __device__ void finalize_body(const LayerArgs& L, const Plan& P, int grid, const
                               Partial* s_red, sop_pair_stat* pair_table, sop_pair_stat* signed_table, sop_search_result* res,
                               const int* cls_k, float wmax);
 
-constexpr int ACC_BYTES = 32 * 24;     // accumulators of one entry: 32 lanes x (two FP64 sums, two counts)
+constexpr int ACC_BYTES = 32 * 20;     // accumulators of one entry: 32 lanes x (two FP64 sums, two 16-bit counts)
 
 __device__ __forceinline__ void lds128(unsigned addr, float (&v)[4]) {
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "r"(addr));
 }
 
 // The accumulators of one entry and lane, in shared memory: FP64 sums (gap, error) at sums + seat * 512 + lane * 16 and
-// counts (second candidate chosen, negated winner) at counts + seat * 256 + lane * 8.
-__device__ __forceinline__ void acc_add(unsigned sums, unsigned counts, float cg, float ce, int n1, int nn) {
+// counts (second candidate chosen, negated winner; 16 bits each: a lane sees at most 8 blocks per tile and a CTA a few
+// thousand tiles) at counts + seat * 128 + lane * 4.
+// NT = 1: the sums of one tile; NT = 2: of two tiles, added one after the other (the same additions in the same order
+// as two calls, with one load and one store of the accumulators).
+template <int NT>
+__device__ __forceinline__ void acc_add(unsigned sums, unsigned counts, const float (&cg)[NT], const float (&ce)[NT], const int (&n1)[NT],
+                                        const int (&nn)[NT]) {
   double g, e;
   asm volatile("ld.shared.v2.f64 {%0, %1}, [%2];" : "=d"(g), "=d"(e) : "r"(sums));
-  g += (double)cg; e += (double)ce;
+#pragma unroll
+  for (int t = 0; t < NT; ++t) { g += (double)cg[t]; e += (double)ce[t]; }
   asm volatile("st.shared.v2.f64 [%0], {%1, %2};" ::"r"(sums), "d"(g), "d"(e) : "memory");
-  int a, b;
-  asm volatile("ld.shared.v2.s32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(counts));
-  a += n1; b += nn;
-  asm volatile("st.shared.v2.s32 [%0], {%1, %2};" ::"r"(counts), "r"(a), "r"(b) : "memory");
+  unsigned c;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(c) : "r"(counts));
+#pragma unroll
+  for (int t = 0; t < NT; ++t) c += (unsigned)n1[t] + ((unsigned)nn[t] << 16);       // neither half can carry: both stay below 2^16
+  asm volatile("st.shared.u32 [%0], %1;" ::"r"(counts), "r"(c) : "memory");
 }
 
 // One task on the lane's eight blocks of one tile (blocks 4 lane .. 4 lane + 3 and the same 128 further on: two 128-bit
@@ -614,67 +621,82 @@ __device__ __forceinline__ void acc_add(unsigned sums, unsigned counts, float cg
 // in fp32 and added to the lane's FP64 accumulators.
 //   cos_base / sse_base: shared-memory addresses of the tile's columns (for a signed task the signed-best columns);
 //   tk: the task (in shared memory); sums / counts: shared-memory addresses of this lane's accumulators of the task's
-//   first seat (the anchor alone), the partners' seats follow.
-template <bool SEL_ERR, bool SGN, bool REV>
-__device__ __forceinline__ void run_task(const TaskDev* __restrict__ tk, unsigned cos_base, unsigned sse_base, int lane, unsigned sums, unsigned counts) {
+//   first seat: the anchor alone if the task has that entry, then the partners.
+//   NT = 2: the same task on two tiles at once -- the tile in work and the one `pair_off` bytes further on in shared
+//   memory -- so that the accumulators are loaded and stored once for both.
+template <bool SEL_ERR, bool SGN, bool REV, int NT>
+__device__ __forceinline__ void run_task(const TaskDev* __restrict__ tk, unsigned cos_base, unsigned sse_base, unsigned pair_off, int lane,
+                                         unsigned sums, unsigned counts) {
   constexpr unsigned COL = RTILE * 4u;          // bytes of one column
   const unsigned lane_off = (unsigned)lane * 16u;
-  float ac0[4], ac1[4], ae0[4], ae1[4];
-  {
-    const unsigned a = (unsigned)tk->anchor * COL + lane_off;
-    lds128(cos_base + a, ac0); lds128(cos_base + a + 512u, ac1);
-    lds128(sse_base + a, ae0); lds128(sse_base + a + 512u, ae1);
+  float ac0[NT][4], ac1[NT][4], ae0[NT][4], ae1[NT][4], ga0[NT][4], ga1[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) {
+    const unsigned a = (unsigned)tk->anchor * COL + lane_off + (unsigned)t * pair_off;
+    lds128(cos_base + a, ac0[t]); lds128(cos_base + a + 512u, ac1[t]);
+    lds128(sse_base + a, ae0[t]); lds128(sse_base + a + 512u, ae1[t]);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) { ga0[t][r] = __fsub_rn(1.0f, ac0[t][r]); ga1[t][r] = __fsub_rn(1.0f, ac1[t][r]); }
   }
-  float ga0[4], ga1[4];
-#pragma unroll
-  for (int r = 0; r < 4; ++r) { ga0[r] = __fsub_rn(1.0f, ac0[r]); ga1[r] = __fsub_rn(1.0f, ac1[r]); }
   if (tk->self_slot != 255) {
-    float cg = 0.0f, ce = 0.0f;
-    int nn = 0;
+    float cg[NT], ce[NT];
+    int n1[NT], nn[NT];
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      cg = __fadd_rn(cg, ga0[r]); ce = __fadd_rn(ce, fabsf(ae0[r]));
-      cg = __fadd_rn(cg, ga1[r]); ce = __fadd_rn(ce, fabsf(ae1[r]));
-      if (SGN) nn += (int)(__float_as_uint(ae0[r]) >> 31) + (int)(__float_as_uint(ae1[r]) >> 31);
+    for (int t = 0; t < NT; ++t) {
+      cg[t] = 0.0f; ce[t] = 0.0f; n1[t] = 0; nn[t] = 0;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        cg[t] = __fadd_rn(cg[t], ga0[t][r]); ce[t] = __fadd_rn(ce[t], fabsf(ae0[t][r]));
+        cg[t] = __fadd_rn(cg[t], ga1[t][r]); ce[t] = __fadd_rn(ce[t], fabsf(ae1[t][r]));
+        if (SGN) nn[t] += (int)(__float_as_uint(ae0[t][r]) >> 31) + (int)(__float_as_uint(ae1[t][r]) >> 31);
+      }
     }
-    acc_add(sums, counts, cg, ce, 0, nn);
+    acc_add<NT>(sums, counts, cg, ce, n1, nn);
+    sums += 512u; counts += 128u;            // the partners' seats follow
   }
   const int np = tk->n_part;
 #pragma unroll 1
   for (int q = 0; q < np; ++q) {
-    const unsigned b = (unsigned)tk->part[q] * COL + lane_off;
-    float bc0[4], bc1[4], be0[4], be1[4];
-    lds128(cos_base + b, bc0); lds128(cos_base + b + 512u, bc1);
-    lds128(sse_base + b, be0); lds128(sse_base + b + 512u, be1);
-    float cg = 0.0f, ce = 0.0f;
-    int n1 = 0, nn = 0;
+    float cg[NT], ce[NT];
+    int n1[NT], nn[NT];
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      // mu: the entry's second candidate is strictly better and takes the block.  REV = false: the anchor is the
-      // first candidate and the partner the second; REV = true: the other way round.
-      bool mu0, mu1;
-      float g0, g1, e0, e1;
-      if (!REV) {
-        mu0 = SEL_ERR ? fabsf(be0[r]) < fabsf(ae0[r]) : bc0[r] > ac0[r];
-        mu1 = SEL_ERR ? fabsf(be1[r]) < fabsf(ae1[r]) : bc1[r] > ac1[r];
-        g0 = mu0 ? __fsub_rn(1.0f, bc0[r]) : ga0[r]; e0 = mu0 ? be0[r] : ae0[r];
-        g1 = mu1 ? __fsub_rn(1.0f, bc1[r]) : ga1[r]; e1 = mu1 ? be1[r] : ae1[r];
-      } else {
-        mu0 = SEL_ERR ? fabsf(ae0[r]) < fabsf(be0[r]) : ac0[r] > bc0[r];
-        mu1 = SEL_ERR ? fabsf(ae1[r]) < fabsf(be1[r]) : ac1[r] > bc1[r];
-        g0 = mu0 ? ga0[r] : __fsub_rn(1.0f, bc0[r]); e0 = mu0 ? ae0[r] : be0[r];
-        g1 = mu1 ? ga1[r] : __fsub_rn(1.0f, bc1[r]); e1 = mu1 ? ae1[r] : be1[r];
+    for (int t = 0; t < NT; ++t) {
+      const unsigned b = (unsigned)tk->part[q] * COL + lane_off + (unsigned)t * pair_off;
+      float bc0[4], bc1[4], be0[4], be1[4];
+      lds128(cos_base + b, bc0); lds128(cos_base + b + 512u, bc1);
+      lds128(sse_base + b, be0); lds128(sse_base + b + 512u, be1);
+      cg[t] = 0.0f; ce[t] = 0.0f; n1[t] = 0; nn[t] = 0;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        // mu: the entry's second candidate is strictly better and takes the block.  REV = false: the anchor is the
+        // first candidate and the partner the second; REV = true: the other way round.
+        bool mu0, mu1;
+        float g0, g1, e0, e1;
+        if (!REV) {
+          mu0 = SEL_ERR ? fabsf(be0[r]) < fabsf(ae0[t][r]) : bc0[r] > ac0[t][r];
+          mu1 = SEL_ERR ? fabsf(be1[r]) < fabsf(ae1[t][r]) : bc1[r] > ac1[t][r];
+          g0 = mu0 ? __fsub_rn(1.0f, bc0[r]) : ga0[t][r]; e0 = mu0 ? be0[r] : ae0[t][r];
+          g1 = mu1 ? __fsub_rn(1.0f, bc1[r]) : ga1[t][r]; e1 = mu1 ? be1[r] : ae1[t][r];
+        } else {
+          mu0 = SEL_ERR ? fabsf(ae0[t][r]) < fabsf(be0[r]) : ac0[t][r] > bc0[r];
+          mu1 = SEL_ERR ? fabsf(ae1[t][r]) < fabsf(be1[r]) : ac1[t][r] > bc1[r];
+          g0 = mu0 ? ga0[t][r] : __fsub_rn(1.0f, bc0[r]); e0 = mu0 ? ae0[t][r] : be0[r];
+          g1 = mu1 ? ga1[t][r] : __fsub_rn(1.0f, bc1[r]); e1 = mu1 ? ae1[t][r] : be1[r];
+        }
+        cg[t] = __fadd_rn(cg[t], g0); ce[t] = __fadd_rn(ce[t], fabsf(e0));
+        cg[t] = __fadd_rn(cg[t], g1); ce[t] = __fadd_rn(ce[t], fabsf(e1));
+        n1[t] += (mu0 ? 1 : 0) + (mu1 ? 1 : 0);
+        if (SGN) nn[t] += (int)(__float_as_uint(e0) >> 31) + (int)(__float_as_uint(e1) >> 31);
       }
-      cg = __fadd_rn(cg, g0); ce = __fadd_rn(ce, fabsf(e0));
-      cg = __fadd_rn(cg, g1); ce = __fadd_rn(ce, fabsf(e1));
-      n1 += (mu0 ? 1 : 0) + (mu1 ? 1 : 0);
-      if (SGN) nn += (int)(__float_as_uint(e0) >> 31) + (int)(__float_as_uint(e1) >> 31);
     }
-    acc_add(sums + (unsigned)(q + 1) * 512u, counts + (unsigned)(q + 1) * 256u, cg, ce, n1, nn);
+    acc_add<NT>(sums + (unsigned)q * 512u, counts + (unsigned)q * 128u, cg, ce, n1, nn);
   }
 }
 
-template <bool SEL_ERR, int TPW, bool VEC>
+// PAIR (with VEC and a ring of four buffers): the CTA works on two tiles at a time -- buffers (0, 1), then (2, 3) while
+// (0, 1) are refilled -- so that a lane owns sixteen blocks per step and touches its accumulators half as often.  The
+// additions and their order are those of the one-tile path: the results are the same bit for bit.
+template <bool SEL_ERR, int TPW, bool VEC, bool PAIR>
 __global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, SeatsDev seats, int n_stage, int do_final, WsHeader* __restrict__ hdr,
                                                      Partial* __restrict__ partials, const float* __restrict__ block_cos,
                                                      const float* __restrict__ block_sse, sop_pair_stat* pair_table,
@@ -686,10 +708,11 @@ __global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, Sea
   float* cos0 = reinterpret_cast<float*>(smem);                          // [NBUF][A][RTILE]
   float* sse0 = cos0 + (size_t)NBUF * A * RTILE;                         // [NBUF][A][RTILE]
   // signed-best columns of the tile in work
-  float* scos = sse0 + (size_t)NBUF * A * RTILE;                         // [n_bases][RTILE]
-  float* ssse = scos + (size_t)seats.n_bases * RTILE;                    // [n_bases][RTILE]
-  double2* acc_sums = reinterpret_cast<double2*>(ssse + (size_t)seats.n_bases * RTILE);   // [n_seats][32]: seat-major, then lane
-  int2* acc_counts = reinterpret_cast<int2*>(acc_sums + (size_t)seats.n_seats * 32);      // [n_seats][32]
+  constexpr int NSB = PAIR ? 2 : 1;                                      // tiles in work at a time
+  float* scos = sse0 + (size_t)NBUF * A * RTILE;                         // [NSB][n_bases][RTILE]
+  float* ssse = scos + (size_t)NSB * seats.n_bases * RTILE;              // [NSB][n_bases][RTILE]
+  double2* acc_sums = reinterpret_cast<double2*>(ssse + (size_t)NSB * seats.n_bases * RTILE);   // [n_seats][32]: seat-major, then lane
+  unsigned* acc_counts = reinterpret_cast<unsigned*>(acc_sums + (size_t)seats.n_seats * 32);   // [n_seats][32]: two 16-bit counts
   __shared__ unsigned long long s_coloff[SOP_MAX_ATOMS];   // first element of every fetched column in the arrays
   __shared__ TaskDev s_task[RTB / 32][TPW];        // anchors and partners translated to columns of the buffers
   __shared__ int s_acc0[RTB / 32][TPW];
@@ -707,7 +730,7 @@ __global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, Sea
     s_task[warp][lane] = t;
     s_acc0[warp][lane] = seats.acc0[warp][lane];
   }
-  for (int i = tid; i < seats.n_seats * 32; i += RTB) { acc_sums[i] = make_double2(0.0, 0.0); acc_counts[i] = make_int2(0, 0); }
+  for (int i = tid; i < seats.n_seats * 32; i += RTB) { acc_sums[i] = make_double2(0.0, 0.0); acc_counts[i] = 0u; }
   if (tid < seats.n_cols) s_coloff[tid] = (unsigned long long)seats.cols[tid] * (unsigned long long)L.NB;
   __syncthreads();
   const int ncols = seats.n_cols, nbases = seats.n_bases;
@@ -733,65 +756,120 @@ __global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, Sea
           asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "f"(v) : "memory");
         }
       }
+    } else if (PAIR) {
+      // the second tile of the last pair does not exist: it reads as (cos 1, error 0) and adds nothing
+      unsigned dst = f_dst + (unsigned)(b * A * RTILE * 4);
+      const float v = f_arr ? 0.0f : 1.0f;
+      for (int i = tid >> 7; i < ncols; i += 2, dst += 2u * RTILE * 4u)
+        asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "f"(v) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
 
-  long long tile = blockIdx.x;
-  if (VEC)
-    for (int b = 0; b < n_stage - 1; ++b) fetch(tile + (long long)b * gridDim.x, b);
-  int cur = 0;                 // buffer of the tile in work
-  for (; tile < n_tiles; tile += gridDim.x) {
-    float* cosb = cos0 + (size_t)cur * A * RTILE;
-    float* sseb = sse0 + (size_t)cur * A * RTILE;
-    if (VEC) {
-      // this thread's copies of the tile in work are complete when at most n_stage - 2 newer groups are still pending
-      if (n_stage == 4) asm volatile("cp.async.wait_group 2;" ::: "memory");
-      else if (n_stage == 3) asm volatile("cp.async.wait_group 1;" ::: "memory");
-      else asm volatile("cp.async.wait_group 0;" ::: "memory");
-    } else {
-      const long long blk0 = tile * RTILE;
-      const int nv = (int)min((long long)RTILE, L.NB - blk0);
-      __syncthreads();                                      // everybody has finished the previous tile
-      for (int i = 0; i < ncols; ++i) {
-        const size_t a = seats.cols[i];
-        cosb[i * RTILE + tid] = tid < nv ? __ldg(block_cos + a * L.NB + blk0 + tid) : 1.0f;
-        sseb[i * RTILE + tid] = tid < nv ? __ldg(block_sse + a * L.NB + blk0 + tid) : 0.0f;
+  if constexpr (PAIR) {
+    const long long step = gridDim.x;
+    long long tile = blockIdx.x;
+    fetch(tile, 0);
+    fetch(tile + step, 1);
+    int ps = 0;                  // the pair of buffers in work: (0, 1) or (2, 3)
+    for (; tile < n_tiles; tile += 2 * step) {
+      float* cosb = cos0 + (size_t)(2 * ps) * A * RTILE;
+      float* sseb = sse0 + (size_t)(2 * ps) * A * RTILE;
+      asm volatile("cp.async.wait_group 0;" ::: "memory");       // this thread's copies of both tiles have landed
+      if (nbases) {
+        __syncthreads();                                          // ... and everybody's; the previous pair's readers are done
+        for (int t = 0; t < 2; ++t)
+          for (int i = 0; i < nbases; ++i) {
+            const int a = seats.bases[i], cp = seats.col_slot[a], cn = seats.col_slot[a + 1];
+            const float* cb = cosb + (size_t)t * A * RTILE;
+            const float* sb = sseb + (size_t)t * A * RTILE;
+            const float pc = cb[cp * RTILE + tid], pe = sb[cp * RTILE + tid];
+            const float nc = cb[cn * RTILE + tid], ne = sb[cn * RTILE + tid];
+            const bool neg = SEL_ERR ? ne < pe : nc > pc;
+            scos[((size_t)t * nbases + i) * RTILE + tid] = neg ? nc : pc;
+            ssse[((size_t)t * nbases + i) * RTILE + tid] = neg ? -ne : pe;
+          }
       }
-    }
-    if (nbases) {
-      // Signed-best columns: this thread's block.  The values come from other threads' copies, and the previous tile's
-      // readers of these columns must be done first: hence the barrier.
       __syncthreads();
-      for (int i = 0; i < nbases; ++i) {
-        const int a = seats.bases[i], cp = seats.col_slot[a], cn = seats.col_slot[a + 1];     // the atom and its negation
-        const float pc = cosb[cp * RTILE + tid], pe = sseb[cp * RTILE + tid];
-        const float nc = cosb[cn * RTILE + tid], ne = sseb[cn * RTILE + tid];
-        const bool neg = SEL_ERR ? ne < pe : nc > pc;           // ties to the atom; a negative error marks a negated winner
-        scos[i * RTILE + tid] = neg ? nc : pc;
-        ssse[i * RTILE + tid] = neg ? -ne : pe;
-      }
-    }
-    // One barrier per tile: the tile is complete for everybody, and everybody has finished the previous tile, whose
-    // buffer (the one before this in the ring) the next copies refill.
-    __syncthreads();
-    if (VEC) fetch(tile + (long long)(n_stage - 1) * gridDim.x, cur == 0 ? n_stage - 1 : cur - 1);
+      // the other pair of buffers is free (everybody has passed the barrier, so nobody reads the previous pair any more)
+      fetch(tile + 2 * step, 2 * (ps ^ 1));
+      fetch(tile + 3 * step, 2 * (ps ^ 1) + 1);
 #pragma unroll 1
-    for (int k = 0; k < TPW; ++k) {
-      const TaskDev* tk = &s_task[warp][k];
-      const unsigned sums = smem_u32(acc_sums) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 16u;
-      const unsigned counts = smem_u32(acc_counts) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 8u;
-      const int sgn = tk->sgn;
-      const int rev = tk->rev;
-      if (sgn == 0) {
-        if (rev) run_task<SEL_ERR, false, true>(tk, smem_u32(cosb), smem_u32(sseb), lane, sums, counts);
-        else run_task<SEL_ERR, false, false>(tk, smem_u32(cosb), smem_u32(sseb), lane, sums, counts);
-      } else if (sgn == 1) {
-        if (rev) run_task<SEL_ERR, true, true>(tk, smem_u32(scos), smem_u32(ssse), lane, sums, counts);
-        else run_task<SEL_ERR, true, false>(tk, smem_u32(scos), smem_u32(ssse), lane, sums, counts);
+      for (int k = 0; k < TPW; ++k) {
+        const TaskDev* tk = &s_task[warp][k];
+        const unsigned sums = smem_u32(acc_sums) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 16u;
+        const unsigned counts = smem_u32(acc_counts) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 4u;
+        const int sgn = tk->sgn;
+        const int rev = tk->rev;
+        const unsigned poff = (unsigned)(A * RTILE * 4), soff = (unsigned)(nbases * RTILE * 4);
+        if (sgn == 0) {
+          if (rev) run_task<SEL_ERR, false, true, 2>(tk, smem_u32(cosb), smem_u32(sseb), poff, lane, sums, counts);
+          else run_task<SEL_ERR, false, false, 2>(tk, smem_u32(cosb), smem_u32(sseb), poff, lane, sums, counts);
+        } else if (sgn == 1) {
+          if (rev) run_task<SEL_ERR, true, true, 2>(tk, smem_u32(scos), smem_u32(ssse), soff, lane, sums, counts);
+          else run_task<SEL_ERR, true, false, 2>(tk, smem_u32(scos), smem_u32(ssse), soff, lane, sums, counts);
+        }
       }
+      ps ^= 1;
     }
-    if (VEC && ++cur == n_stage) cur = 0;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");         // nothing of this CTA's is in flight when it leaves
+  } else {
+    long long tile = blockIdx.x;
+    if (VEC)
+      for (int b = 0; b < n_stage - 1; ++b) fetch(tile + (long long)b * gridDim.x, b);
+    int cur = 0;                 // buffer of the tile in work
+    for (; tile < n_tiles; tile += gridDim.x) {
+      float* cosb = cos0 + (size_t)cur * A * RTILE;
+      float* sseb = sse0 + (size_t)cur * A * RTILE;
+      if (VEC) {
+        // this thread's copies of the tile in work are complete when at most n_stage - 2 newer groups are still pending
+        if (n_stage == 4) asm volatile("cp.async.wait_group 2;" ::: "memory");
+        else if (n_stage == 3) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      } else {
+        const long long blk0 = tile * RTILE;
+        const int nv = (int)min((long long)RTILE, L.NB - blk0);
+        __syncthreads();                                      // everybody has finished the previous tile
+        for (int i = 0; i < ncols; ++i) {
+          const size_t a = seats.cols[i];
+          cosb[i * RTILE + tid] = tid < nv ? __ldg(block_cos + a * L.NB + blk0 + tid) : 1.0f;
+          sseb[i * RTILE + tid] = tid < nv ? __ldg(block_sse + a * L.NB + blk0 + tid) : 0.0f;
+        }
+      }
+      if (nbases) {
+        // Signed-best columns: this thread's block.  The values come from other threads' copies, and the previous tile's
+        // readers of these columns must be done first: hence the barrier.
+        __syncthreads();
+        for (int i = 0; i < nbases; ++i) {
+          const int a = seats.bases[i], cp = seats.col_slot[a], cn = seats.col_slot[a + 1];     // the atom and its negation
+          const float pc = cosb[cp * RTILE + tid], pe = sseb[cp * RTILE + tid];
+          const float nc = cosb[cn * RTILE + tid], ne = sseb[cn * RTILE + tid];
+          const bool neg = SEL_ERR ? ne < pe : nc > pc;           // ties to the atom; a negative error marks a negated winner
+          scos[i * RTILE + tid] = neg ? nc : pc;
+          ssse[i * RTILE + tid] = neg ? -ne : pe;
+        }
+      }
+      // One barrier per tile: the tile is complete for everybody, and everybody has finished the previous tile, whose
+      // buffer (the one before this in the ring) the next copies refill.
+      __syncthreads();
+      if (VEC) fetch(tile + (long long)(n_stage - 1) * gridDim.x, cur == 0 ? n_stage - 1 : cur - 1);
+  #pragma unroll 1
+      for (int k = 0; k < TPW; ++k) {
+        const TaskDev* tk = &s_task[warp][k];
+        const unsigned sums = smem_u32(acc_sums) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 16u;
+        const unsigned counts = smem_u32(acc_counts) + (unsigned)(s_acc0[warp][k] * 32 + lane) * 4u;
+        const int sgn = tk->sgn;
+        const int rev = tk->rev;
+        if (sgn == 0) {
+          if (rev) run_task<SEL_ERR, false, true, 1>(tk, smem_u32(cosb), smem_u32(sseb), 0u, lane, sums, counts);
+          else run_task<SEL_ERR, false, false, 1>(tk, smem_u32(cosb), smem_u32(sseb), 0u, lane, sums, counts);
+        } else if (sgn == 1) {
+          if (rev) run_task<SEL_ERR, true, true, 1>(tk, smem_u32(scos), smem_u32(ssse), 0u, lane, sums, counts);
+          else run_task<SEL_ERR, true, false, 1>(tk, smem_u32(scos), smem_u32(ssse), 0u, lane, sums, counts);
+        }
+      }
+      if (VEC && ++cur == n_stage) cur = 0;
+    }
   }
 
   // ---- per-CTA partials: lane (k, q) of a warp adds the 32 lanes' sums of entry q of the warp's task k, in lane order ----
@@ -802,10 +880,11 @@ __global__ void __launch_bounds__(RTB, 2) reduce_kernel(LayerArgs L, Plan P, Sea
     const int slot = t.sgn == 2 ? 255 : (q == 0 ? t.self_slot : (q - 1 < t.n_part ? t.slot[q - 1] : 255));
     if (slot != 255) {
       Partial p; p.gap = 0.0; p.sse = 0.0; p.n1 = 0; p.nneg = 0;
+      const int seat = s_acc0[warp][k] + (q == 0 ? 0 : q - 1 + (t.self_slot != 255 ? 1 : 0));
       for (int l = 0; l < 32; ++l) {
-        const double2 a = acc_sums[(size_t)(s_acc0[warp][k] + q) * 32 + l];
-        const int2 c = acc_counts[(size_t)(s_acc0[warp][k] + q) * 32 + l];
-        p.gap += a.x; p.sse += a.y; p.n1 += c.x; p.nneg += c.y;
+        const double2 a = acc_sums[(size_t)seat * 32 + l];
+        const unsigned c = acc_counts[(size_t)seat * 32 + l];
+        p.gap += a.x; p.sse += a.y; p.n1 += (long long)(c & 0xFFFFu); p.nneg += (long long)(c >> 16);
       }
       partials[(size_t)blockIdx.x * MAX_SLOTS + slot] = p;
     }
@@ -1172,7 +1251,8 @@ static int deal_tasks(const Plan& P, int task0, int n, SeatsDev* seats) {
     for (int k = 0; k < MAX_TPW; ++k) {
       if (seats->task[w][k] == 255) continue;
       seats->acc0[w][k] = (unsigned short)seats->n_seats;
-      seats->n_seats += 1 + P.tasks[seats->task[w][k]].n_part;
+      const TaskDev& t = P.tasks[seats->task[w][k]];
+      seats->n_seats += (t.self_slot != 255 ? 1 : 0) + t.n_part;
     }
   return tpw > 0 ? tpw : 1;
 }
@@ -1185,8 +1265,8 @@ size_t sweep_smem_bytes(const Plan& P) {
 
 // the ring of tile buffers, the signed-best columns, the lanes' accumulators; at least the room the closing
 // reduction of the last CTA needs
-static size_t reduce_smem_bytes(const SeatsDev& S, int n_stage) {
-  const size_t tiles = ((size_t)n_stage * S.n_cols + S.n_bases) * 2 * RTILE * sizeof(float);
+static size_t reduce_smem_bytes(const SeatsDev& S, int n_stage, bool pair = false) {
+  const size_t tiles = ((size_t)n_stage * S.n_cols + (pair ? 2 : 1) * (size_t)S.n_bases) * 2 * RTILE * sizeof(float);
   const size_t acc = (size_t)S.n_seats * ACC_BYTES;
   const size_t fin = sizeof(Partial) * (size_t)RTB + 2 * sizeof(sop_pair_stat) * SOP_MAX_ATOMS * SOP_MAX_ATOMS;
   const size_t b = tiles + acc;
@@ -1195,6 +1275,10 @@ static size_t reduce_smem_bytes(const SeatsDev& S, int n_stage) {
 
 // Doubles the cell width of the LUT class with the most rows (its tables then hold several thresholds per cell
 // where they are dense, and such tables take the exact binary search).  False when no class can shrink further.
+// Two tiles per step in the reduction (see reduce_kernel) wherever the shared memory allows; sop_pair_search_tuning
+// turns it off (tests compare both paths: the results are the same bit for bit).
+static bool g_reduce_pairs = true;
+
 static bool coarsen_cells(Plan* P) {
   int pick = -1;
   for (int c = 0; c < P->n_classes; ++c)
@@ -1214,6 +1298,12 @@ static bool coarsen_cells(Plan* P) {
 }  // namespace sop
 
 extern "C" {
+
+int sop_pair_search_tuning(int reduce_tile_pairs) {
+  if (reduce_tile_pairs != 0 && reduce_tile_pairs != 1) return SOP_ERR_RANGE;
+  sop::g_reduce_pairs = reduce_tile_pairs != 0;
+  return SOP_OK;
+}
 
 int sop_pair_search_workspace(long long M, long long K, int n_atoms, size_t* bytes) {
   if (!bytes) return SOP_ERR_NULL;
@@ -1295,6 +1385,9 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   const long long n_tiles = (L.NB + RTILE - 1) / RTILE;
   long long rgrid = n_tiles < (long long)sms * 2 ? n_tiles : (long long)sms * 2;
   if (rgrid < 1) rgrid = 1;
+  // a lane counts at most 8 blocks per tile in 16 bits: a CTA takes fewer than 8000 tiles (never near it on a GPU with
+  // a hundred SMs: 2^19 tiles at most)
+  if (n_tiles / rgrid >= 8000) rgrid = (n_tiles + 7999) / 8000;
 
   // the header always starts from zero; the histograms (and max|W| behind them) only when this call fills them
   SOP_CUDA_TRY(cudaMemsetAsync(ws, 0, (k_from_result || reuse_prepass) ? ws_hist_off() : ws_part_off(), st));
@@ -1313,12 +1406,14 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
   DeviceFacts* facts = device_facts();
   if (!facts->search_attr_set) {
     SOP_CUDA_TRY(cudaFuncSetAttribute(sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX));
-#define SOP_REDUCE_ATTR(SE, T, BK) \
-  SOP_CUDA_TRY(cudaFuncSetAttribute(reduce_kernel<SE, T, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX))
-    SOP_REDUCE_ATTR(false, 1, false); SOP_REDUCE_ATTR(false, 2, false); SOP_REDUCE_ATTR(false, 3, false);
-    SOP_REDUCE_ATTR(false, 1, true); SOP_REDUCE_ATTR(false, 2, true); SOP_REDUCE_ATTR(false, 3, true);
-    SOP_REDUCE_ATTR(true, 1, false); SOP_REDUCE_ATTR(true, 2, false); SOP_REDUCE_ATTR(true, 3, false);
-    SOP_REDUCE_ATTR(true, 1, true); SOP_REDUCE_ATTR(true, 2, true); SOP_REDUCE_ATTR(true, 3, true);
+#define SOP_REDUCE_ATTR(SE, T, BK, PR) \
+  SOP_CUDA_TRY(cudaFuncSetAttribute(reduce_kernel<SE, T, BK, PR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_MAX))
+    SOP_REDUCE_ATTR(false, 1, false, false); SOP_REDUCE_ATTR(false, 2, false, false); SOP_REDUCE_ATTR(false, 3, false, false);
+    SOP_REDUCE_ATTR(false, 1, true, false); SOP_REDUCE_ATTR(false, 2, true, false); SOP_REDUCE_ATTR(false, 3, true, false);
+    SOP_REDUCE_ATTR(true, 1, false, false); SOP_REDUCE_ATTR(true, 2, false, false); SOP_REDUCE_ATTR(true, 3, false, false);
+    SOP_REDUCE_ATTR(true, 1, true, false); SOP_REDUCE_ATTR(true, 2, true, false); SOP_REDUCE_ATTR(true, 3, true, false);
+    SOP_REDUCE_ATTR(false, 1, true, true); SOP_REDUCE_ATTR(false, 2, true, true); SOP_REDUCE_ATTR(false, 3, true, true);
+    SOP_REDUCE_ATTR(true, 1, true, true); SOP_REDUCE_ATTR(true, 2, true, true); SOP_REDUCE_ATTR(true, 3, true, true);
 #undef SOP_REDUCE_ATTR
     facts->search_attr_set = true;
   }
@@ -1339,15 +1434,17 @@ int sop_pair_search(const void* W_dev, long long M, long long K, long long ldw, 
     // buffers always fit one CTA)
     int n_stage = vec ? MAX_STAGE : 1;
     while (n_stage > 2 && reduce_smem_bytes(seats, n_stage) > SMEM_MAX / 2) --n_stage;
-    const size_t rs = reduce_smem_bytes(seats, n_stage);
+    // two tiles at a time when the ring has its four buffers and the second set of signed-best columns still fits
+    const bool pair = vec && n_stage == MAX_STAGE && reduce_smem_bytes(seats, n_stage, true) <= SMEM_MAX / 2 && g_reduce_pairs;
+    const size_t rs = reduce_smem_bytes(seats, n_stage, pair);
     const int fin = l == n_launch - 1 ? 1 : 0;
-#define SOP_LAUNCH_REDUCE(SE, T, BK)                                                                                          \
-  reduce_kernel<SE, T, BK><<<(int)rgrid, RTB, rs, st>>>(L, P, seats, n_stage, fin, hdr, partials, cos_cols, sse_cols, pair_table_dev, \
-                                                        signed_table_dev, result_dev, prev_result_dev)
-#define SOP_LAUNCH_REDUCE_T(SE, BK) \
-  do { if (tpw == 1) SOP_LAUNCH_REDUCE(SE, 1, BK); else if (tpw == 2) SOP_LAUNCH_REDUCE(SE, 2, BK); else SOP_LAUNCH_REDUCE(SE, 3, BK); } while (0)
-    if (sel_err) { if (vec) SOP_LAUNCH_REDUCE_T(true, true); else SOP_LAUNCH_REDUCE_T(true, false); }
-    else { if (vec) SOP_LAUNCH_REDUCE_T(false, true); else SOP_LAUNCH_REDUCE_T(false, false); }
+#define SOP_LAUNCH_REDUCE(SE, T, BK, PR)                                                                                      \
+  reduce_kernel<SE, T, BK, PR><<<(int)rgrid, RTB, rs, st>>>(L, P, seats, n_stage, fin, hdr, partials, cos_cols, sse_cols, pair_table_dev, \
+                                                            signed_table_dev, result_dev, prev_result_dev)
+#define SOP_LAUNCH_REDUCE_T(SE, BK, PR) \
+  do { if (tpw == 1) SOP_LAUNCH_REDUCE(SE, 1, BK, PR); else if (tpw == 2) SOP_LAUNCH_REDUCE(SE, 2, BK, PR); else SOP_LAUNCH_REDUCE(SE, 3, BK, PR); } while (0)
+    if (sel_err) { if (pair) SOP_LAUNCH_REDUCE_T(true, true, true); else if (vec) SOP_LAUNCH_REDUCE_T(true, true, false); else SOP_LAUNCH_REDUCE_T(true, false, false); }
+    else { if (pair) SOP_LAUNCH_REDUCE_T(false, true, true); else if (vec) SOP_LAUNCH_REDUCE_T(false, true, false); else SOP_LAUNCH_REDUCE_T(false, false, false); }
 #undef SOP_LAUNCH_REDUCE_T
 #undef SOP_LAUNCH_REDUCE
     SOP_CUDA_TRY(cudaGetLastError());

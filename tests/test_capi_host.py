@@ -173,6 +173,7 @@ def test_lloyd_tuning_ranges(lib):
 def test_sparse_stream_entry_points_reject_bad_arguments(lib):
     ll = C.c_longlong
     m = C.c_double()
+    assert lib.sop_pair_search_tuning(2) == -7 and lib.sop_pair_search_tuning(1) == 0
     assert lib.sop_opq_threshold(C.c_double(0.92), 16, C.byref(m)) == 0 and 2.79 < m.value < 2.80
     assert lib.sop_opq_threshold(C.c_double(0.92), 16, None) == -1
     assert lib.sop_opq_threshold(C.c_double(1.0), 16, C.byref(m)) == -7 and lib.sop_opq_threshold(C.c_double(0.5), 0, C.byref(m)) == -7

@@ -164,3 +164,30 @@ def test_shifts_from_the_histogram_of_an_earlier_format():
         assert torch.equal(got.codes, want.codes) and torch.equal(got.words, want.words)
         ks.add(int(want.result["k"][0]))
     assert len(ks) > 1          # the formats really need different shifts
+
+
+def test_reduction_on_one_tile_and_on_two_tiles_at_a_time():
+    """The reduction kernel's two launch shapes (two tiles of 256 blocks per step where the shared memory allows, one
+    otherwise) make the same additions in the same order: every table entry is the same bit for bit, at a signed and
+    an unsigned scale format, with a ragged last tile and an odd number of tiles per CTA."""
+    from paper_2605_14929_b200 import binding as Bd
+    from paper_2605_14929_b200.pipeline import LayerSweep
+    d = torch.device("cuda:0")
+    L = I.student_layer(71, 0, 1345, 1024, 64, 4.0, channel_sigma=0.6)      # 86080 blocks: 337 tiles, the last one ragged
+    Wd, Xd = L.W.to(d), L.X.to(d)
+    for fmt_name in ("E5M6", "UE4M4"):
+        fmt = I.scale_format(fmt_name)
+        got = []
+        try:
+            for pairs in (True, False):
+                Bd.pair_search_tuning(pairs)
+                sw = LayerSweep(1345, 1024, 64, fmt, ["NF4", "SH4", "BOF4", "Split87"], [], 3, device=d)
+                sw.run(Wd, Xd)
+                got.append(sw.outputs())
+        finally:
+            Bd.pair_search_tuning(True)
+        a, b = got
+        for name in ("pair_table", "signed_table"):
+            for field in ("acos", "mse", "n_sel1", "n_neg"):
+                assert np.array_equal(getattr(a, name)[field], getattr(b, name)[field], equal_nan=(field in ("acos", "mse"))), (fmt_name, name, field)
+        assert np.array_equal(a.result["best"], b.result["best"])
