@@ -25,8 +25,12 @@ struct PackArgs {
 };
 
 constexpr int KIND_LUT16 = 100;   // inside this file: a LUT of at most 16 entries (a four-step search is enough)
+constexpr int KIND_LUT_CELL = 101; // inside this file: a LUT whose codes come from a uniform cell grid on u (one look-up, one compare)
+constexpr int CELL_ROWS_MAX = 1025;
+constexpr float CELL_MAGIC = 12582912.0f;   // 1.5 * 2^23: adding it leaves rint(x) in the low mantissa bits
 
-struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; GridDev grid; int sign_pos; };
+// cell grid of a table: cell = rint(u * invh) + c_half, clamped to [0, 2 c_half]
+struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; GridDev grid; int sign_pos; float invh; int c_half; };
 
 // One candidate on one block, everything in registers; same operation order as the sweep kernel.
 // The 16 codes come back as bytes, four per word (element i in byte i % 4 of word i / 4).
@@ -34,7 +38,8 @@ struct PackCand { int table; int kind; int neg; int scope; int k; float tmax; Gr
 template <int METRIC, int KIND>
 __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int neg, float rcp, float s_hat,
-                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid = GridDev(), int sign_pos = 0) {
+                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid = GridDev(), int sign_pos = 0,
+                                                const uint2* __restrict__ cells = nullptr, float invh = 0.0f, int c_half = 0) {
   float qn[4], qd[4], qw[4];
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
@@ -46,7 +51,15 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
       const float u = __fmul_rn(w[i], rcp);
       float q;
       uint32_t code;
-      if (KIND == SOP_KIND_LUT || KIND == KIND_LUT16) {
+      if (KIND == KIND_LUT_CELL) {
+        // the cell holds at most one decision threshold: the code is the number of thresholds below the cell, plus one
+        // when u lies above the cell's own threshold (+inf when it has none)
+        const float uu = neg ? -u : u;
+        const float t = fminf(fmaxf(__fmaf_rn(uu, invh, CELL_MAGIC + (float)c_half), CELL_MAGIC), CELL_MAGIC + (float)(2 * c_half));
+        const uint2 e = cells[__float_as_uint(t) - __float_as_uint(CELL_MAGIC)];
+        code = e.y + (uu > __uint_as_float(e.x) ? 1u : 0u);
+        q = neg ? -lutv[code] : lutv[code];
+      } else if (KIND == SOP_KIND_LUT || KIND == KIND_LUT16) {
         code = (uint32_t)(KIND == KIND_LUT16 ? count_below<4>(tau, neg ? -u : u) : count_below<5>(tau, neg ? -u : u));
         q = neg ? -lutv[code] : lutv[code];
       } else if (KIND == SOP_KIND_FP_E2M3) {
@@ -82,8 +95,10 @@ __device__ __forceinline__ void eval_block_kind(const float (&w)[16], const floa
 template <int METRIC>
 __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const float (&c)[16], const float* __restrict__ tau,
                                                 const float* __restrict__ lutv, int kind, int neg, float rcp, float s_hat,
-                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid, int sign_pos) {
-  if (kind == KIND_LUT16) eval_block_kind<METRIC, KIND_LUT16>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
+                                                float& cos_out, uint32_t (&code4)[4], const GridDev grid, int sign_pos,
+                                                const uint2* __restrict__ cells, float invh, int c_half) {
+  if (kind == KIND_LUT_CELL) eval_block_kind<METRIC, KIND_LUT_CELL>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4, grid, sign_pos, cells, invh, c_half);
+  else if (kind == KIND_LUT16) eval_block_kind<METRIC, KIND_LUT16>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
   else if (kind == SOP_KIND_LUT) eval_block_kind<METRIC, SOP_KIND_LUT>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
   else if (kind == SOP_KIND_FP_GRID) eval_block_kind<METRIC, SOP_KIND_FP_GRID>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4, grid, sign_pos);
   else if (kind == SOP_KIND_FP_E2M3) eval_block_kind<METRIC, SOP_KIND_FP_E2M3>(w, c, tau, lutv, neg, rcp, s_hat, cos_out, code4);
@@ -95,6 +110,7 @@ __device__ __forceinline__ void eval_block_regs(const float (&w)[16], const floa
 template <bool USE_COS>
 __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, AtomsDev A, FmtDev F, const sop_search_result* __restrict__ res) {
   __shared__ float lutv[2][32], tau[2][32];
+  __shared__ uint2 cells[2][CELL_ROWS_MAX];       // per table and cell: {the cell's threshold (+inf: none), thresholds below the cell}
   __shared__ PackCand base[2];
   __shared__ int s_nb, s_nbits;
   __shared__ float s_pot[2];
@@ -128,6 +144,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
       base[t].grid.min_eb = 128 - at.grid_bias; base[t].grid.sh = 23 - at.grid_man_bits;
       base[t].grid.vpos = at.tmax; base[t].grid.vneg = at.grid_neg_max;
       base[t].sign_pos = at.grid_exp_bits + at.grid_man_bits;
+      base[t].invh = 0.0f; base[t].c_half = 0;
       s_pot[t] = at.scope == 0 ? layer_pot_scale(wmax, at.tmax) : 0.0f;
       s_idx[t] = idx;
     }
@@ -156,6 +173,58 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
     int jj = j;
     while (jj < ne - 1 && lutv[t][jj] == lutv[t][jj + 1]) ++jj;
     tau[t][j] = jj < ne - 1 ? __double2float_rd(0.5 * ((double)lutv[t][jj] + (double)lutv[t][jj + 1])) : __int_as_float(0x7F800000);
+  }
+  __syncthreads();
+  // Cell grids of the tables.  A grid of width h <= (smallest gap between two thresholds) / 2 puts at most one threshold
+  // into a cell's closed interval [(k - 1/2) h, (k + 1/2) h]; the first and last cells lie beyond every threshold.  A
+  // table with repeated thresholds, or one that would need more than CELL_ROWS_MAX cells, keeps the binary search.
+  if (tid < nb) {
+    const int t = tid;
+    PackCand cd = base[t];
+    const int ne = A.atoms[s_idx[t]].kind == SOP_KIND_LUT ? A.atoms[s_idx[t]].n_entries : 0;
+    if (ne >= 2) {
+      float gap = __int_as_float(0x7F800000), reach = 0.0f;
+      bool ok = true;
+      for (int j = 0; j < ne - 1; ++j) {
+        reach = fmaxf(reach, fabsf(tau[t][j]));
+        if (j + 1 < ne - 1) {
+          const float g = __fsub_rn(tau[t][j + 1], tau[t][j]);
+          if (!(g > 0.0f)) ok = false;
+          gap = fminf(gap, g);
+        }
+      }
+      if (ne == 2) gap = 1.0f;
+      if (ok && gap > 0.0f && reach < 1.0e6f) {
+        const int eh = ilogb_pos(gap) - 1;                       // h = 2^eh <= gap / 2
+        if (eh >= -20 && eh <= 20) {
+          const float h = pow2f_int(eh);
+          const float rows_half = ceilf(__fdiv_rn(reach, h)) + 1.0f;
+          if (2.0f * rows_half + 1.0f <= (float)CELL_ROWS_MAX) {
+            cd.invh = pow2f_int(-eh);
+            cd.c_half = (int)rows_half;
+            cd.kind = KIND_LUT_CELL;
+          }
+        }
+      }
+    }
+    base[t] = cd;
+  }
+  __syncthreads();
+  for (int t = 0; t < nb; ++t) {
+    if (base[t].kind != KIND_LUT_CELL) continue;
+    const int ch = base[t].c_half, ne = A.atoms[s_idx[t]].n_entries;
+    const float h = __fdiv_rn(1.0f, base[t].invh);
+    for (int r = tid; r <= 2 * ch; r += PTB) {
+      const float lo = __fmul_rn((float)(r - ch) - 0.5f, h), hi = __fmul_rn((float)(r - ch) + 0.5f, h);   // exact: small integers and halves times a power of two
+      unsigned below = 0;
+      float thr = __int_as_float(0x7F800000);
+      for (int j = 0; j < ne - 1; ++j) {
+        const float tj = tau[t][j];
+        if (r > 0 && tj < lo) ++below;
+        else if (r == 2 * ch || tj <= hi) thr = fminf(thr, tj);
+      }
+      cells[t][r] = make_uint2(__float_as_uint(thr), below);
+    }
   }
   __syncthreads();
 
@@ -230,7 +299,7 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
       }
       const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;
       float unused;
-      eval_block_regs<0>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, unused, best4, cd.grid, cd.sign_pos);
+      eval_block_regs<0>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, unused, best4, cd.grid, cd.sign_pos, cells[t], cd.invh, cd.c_half);
     } else {
       for (int t = 0; t < nb; ++t) {
         const PackCand cd = base[t];
@@ -248,8 +317,8 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
         for (int sg = 0; sg < n_sign; ++sg) {
           float cs;
           uint32_t c4[4];
-          if (a.select_err) eval_block_regs<2>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos);
-          else eval_block_regs<1>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos);
+          if (a.select_err) eval_block_regs<2>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos, cells[t], cd.invh, cd.c_half);
+          else eval_block_regs<1>(w, c, tau[t], lutv[t], cd.kind, sg ? 1 - cd.neg : cd.neg, rcp, s_hat, cs, c4, cd.grid, cd.sign_pos, cells[t], cd.invh, cd.c_half);
           if (pick < 0 || (a.select_err ? cs < best_cos : cs > best_cos)) {
             best_cos = cs; best_scode = sc; pick = 2 * t + sg;
 #pragma unroll
