@@ -344,9 +344,10 @@ __device__ __forceinline__ void pool_block_u(const LloydArgs& a, const FmtDev& F
   const uint4* p = reinterpret_cast<const uint4*>(a.W + (long long)m * a.ldw + (long long)j * SOP_G);
   const uint4 v0 = __ldg(p), v1 = __ldg(p + 1);
   const uint32_t wb[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-  uint32_t mb = 0;
+  uint32_t mb = 0;       // the maximum of the sixteen 15-bit magnitude patterns, two per word at a time
 #pragma unroll
-  for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
+  for (int q = 0; q < 8; ++q) mb = __vmaxu2(mb, wb[q] & 0x7FFF7FFFu);
+  mb = max(mb & 0xFFFFu, mb >> 16);
   const float amax = __uint_as_float(mb << 16);
   const float s_hat = scale_quantize(amax, k, F).s_hat;    // a DD table declares tmax = 1
   const float rcp = s_hat > 0.0f ? __frcp_rn(s_hat) : 0.0f;

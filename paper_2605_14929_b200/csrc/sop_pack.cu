@@ -270,9 +270,11 @@ __global__ void __launch_bounds__(PTB, USE_COS ? 4 : 1) pack_kernel(PackArgs a, 
         c[4 * q] = v.x; c[4 * q + 1] = v.y; c[4 * q + 2] = v.z; c[4 * q + 3] = v.w;
       }
     }
+    // bf16 magnitudes order like their bit patterns: the maximum of the sixteen 15-bit patterns, two per word at a time
     uint32_t mb = 0;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) { mb = max(mb, wb[q] & 0x7FFFu); mb = max(mb, (wb[q] >> 16) & 0x7FFFu); }
+    for (int q = 0; q < 8; ++q) mb = __vmaxu2(mb, wb[q] & 0x7FFF7FFFu);
+    mb = max(mb & 0xFFFFu, mb >> 16);
     const float amax = __uint_as_float(mb << 16);
     float best_cos = 0.0f;
     uint32_t best_scode = 0, best4[4] = {0u, 0u, 0u, 0u};
