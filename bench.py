@@ -53,11 +53,11 @@ SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # file (dram__bytes_read.sum + dram__bytes_write.sum of one launch on the 8192x8192 layer at E5M6 divided by its
 # elements; traffic grows in proportion to the elements, so a launch of the block is scaled by its elements).
 # None: no capture of the kernel as it is now.
-NCU_SWEEP_TRAFFIC = dict(source="profiles/kernels_config5_layer_8192x8192_E5M6.md", bytes_per_element_fixed_candidates=5.1737,
-                         bytes_per_element_dd_columns=2.5774)
+NCU_SWEEP_TRAFFIC = dict(source="profiles/kernels_config5_layer_8192x8192_E5M6.md", bytes_per_element_fixed_candidates=5.1796,
+                         bytes_per_element_dd_columns=2.5803)
 # the same for the reduction kernel (first call: the fixed candidates' entries; second call: the DD columns' entries)
-NCU_REDUCE_TRAFFIC = dict(source="profiles/kernels_config5_layer_8192x8192_E5M6.md", bytes_per_element_fixed_candidates=4.0832,
-                          bytes_per_element_dd_columns=5.0762)
+NCU_REDUCE_TRAFFIC = dict(source="profiles/kernels_config5_layer_8192x8192_E5M6.md", bytes_per_element_fixed_candidates=4.0759,
+                          bytes_per_element_dd_columns=5.0753)
 
 
 # ---------------------------------------------------------------------------------------------------------
