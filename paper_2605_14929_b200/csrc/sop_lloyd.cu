@@ -196,19 +196,34 @@ __global__ void __launch_bounds__(LTB) select_kernel(LloydArgs a, const sop_sear
   if (PASS > 0) derive_prefix(ws, a.pool_rank, PASS, &prefix, &rank, &below, &cnt);
   __syncthreads();
   const float* row = a.cosrow_base + (size_t)resolve_fmta(a, res) * a.NB;
-  // four keys per thread and round, their loads in flight together (the pass is bound by memory latency otherwise)
+  auto count = [&](float x) {
+    const unsigned key = pool_key(x, a.flags);
+    if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
+    else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&sh[(key >> 10) & 2047u], 1u); }
+    else { if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u); }
+  };
+  // sixteen keys per thread and round, their loads in flight together (the pass is bound by memory latency otherwise):
+  // four 128-bit loads where the row is 16-byte aligned, else four rounds of four single loads
   const long long stride = (long long)gridDim.x * LTB;
-  for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += 4 * stride) {
+  const long long nv = (reinterpret_cast<uintptr_t>(row) & 15u) == 0 ? a.NB / 4 : 0;      // whole float4 groups
+  for (long long i = (long long)blockIdx.x * LTB + threadIdx.x; i < nv; i += 4 * stride) {
+    float4 v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) v[q] = i + q * stride < nv ? __ldg(reinterpret_cast<const float4*>(row) + i + q * stride) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (i + q * stride >= nv) break;
+      count(v[q].x); count(v[q].y); count(v[q].z); count(v[q].w);
+    }
+  }
+  for (long long i = 4 * nv + (long long)blockIdx.x * LTB + threadIdx.x; i < a.NB; i += 4 * stride) {
     float v[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) v[q] = i + q * stride < a.NB ? __ldg(row + i + q * stride) : 0.0f;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       if (i + q * stride >= a.NB) break;
-      const unsigned key = pool_key(v[q], a.flags);
-      if (PASS == 0) atomicAdd(&sh[key >> 21], 1u);
-      else if (PASS == 1) { if ((key >> 21) == prefix) atomicAdd(&sh[(key >> 10) & 2047u], 1u); }
-      else { if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u); }
+      count(v[q]);
     }
   }
   __syncthreads();
@@ -295,24 +310,39 @@ __global__ void __launch_bounds__(SETUP_TB) lloyd_setup_kernel(LloydArgs a, Atom
   lloyd_publish_desc(ws, s_lut, s_ne);
 }
 
-// Dense list of the pool blocks.  A thread takes four consecutive blocks per round; the CTA's count goes to the list's
-// counter once per round (a warp scan of the threads' counts, then a scan of the eight warp totals).  The order of the
-// list depends on the scheduling of the CTAs; nothing downstream depends on it (integer sums, and an FP64 sum compared
-// with a tolerance).
+// Dense list of the pool blocks.  A thread takes sixteen consecutive blocks per round (four 128-bit loads in flight
+// where the row is 16-byte aligned); the CTA's count goes to the list's counter once per round (a warp scan of the
+// threads' counts, then a scan of the eight warp totals).  The order of the list depends on the scheduling of the
+// CTAs; nothing downstream depends on it (integer sums, and an FP64 sum compared with a tolerance).
+constexpr int LIST_PER_THREAD = 16;
 __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __restrict__ ws) {
   __shared__ unsigned s_cnt[LTB / 32];
   __shared__ unsigned s_base;
   const unsigned tau_key = ws->tau_key;
   const float* row = a.cosrow_base + (size_t)ws->fmta * a.NB;
+  const bool vec = (reinterpret_cast<uintptr_t>(row) & 15u) == 0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long stride = (long long)gridDim.x * LTB * 4;
+  const long long stride = (long long)gridDim.x * LTB * LIST_PER_THREAD;
   const long long n_round = (a.NB + stride - 1) / stride;
-  long long i = ((long long)blockIdx.x * LTB + threadIdx.x) * 4;
+  long long i = ((long long)blockIdx.x * LTB + threadIdx.x) * LIST_PER_THREAD;
   for (long long r = 0; r < n_round; ++r, i += stride) {
     unsigned in = 0;
+    if (vec && i + LIST_PER_THREAD <= a.NB) {
+      float4 v[LIST_PER_THREAD / 4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      if (i + q < a.NB && pool_key(__ldg(row + i + q), a.flags) <= tau_key) in |= 1u << q;
+      for (int q = 0; q < LIST_PER_THREAD / 4; ++q) v[q] = __ldg(reinterpret_cast<const float4*>(row + i) + q);
+#pragma unroll
+      for (int q = 0; q < LIST_PER_THREAD / 4; ++q) {
+        in |= (pool_key(v[q].x, a.flags) <= tau_key ? 1u : 0u) << (4 * q);
+        in |= (pool_key(v[q].y, a.flags) <= tau_key ? 1u : 0u) << (4 * q + 1);
+        in |= (pool_key(v[q].z, a.flags) <= tau_key ? 1u : 0u) << (4 * q + 2);
+        in |= (pool_key(v[q].w, a.flags) <= tau_key ? 1u : 0u) << (4 * q + 3);
+      }
+    } else {
+#pragma unroll 4
+      for (int q = 0; q < LIST_PER_THREAD; ++q)
+        if (i + q < a.NB && pool_key(__ldg(row + i + q), a.flags) <= tau_key) in |= 1u << q;
+    }
     const unsigned mine = (unsigned)__popc(in);
     unsigned incl = mine;
     for (int o = 1; o < 32; o <<= 1) {
@@ -328,9 +358,7 @@ __global__ void __launch_bounds__(LTB) pool_list_kernel(LloydArgs a, LloydWs* __
     }
     __syncthreads();
     unsigned at = s_base + s_cnt[warp] + incl - mine;
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      if ((in >> q) & 1u) a.pool_idx[at++] = (unsigned)(i + q);
+    for (unsigned rest = in; rest; rest &= rest - 1u) a.pool_idx[at++] = (unsigned)(i + (__ffs((int)rest) - 1));
     __syncthreads();             // s_cnt and s_base are rewritten in the next round
   }
 }
