@@ -232,22 +232,36 @@ def per_config_table(dev, alu_peak, flush):
     from paper_2605_14929_b200.pipeline import LayerSweep
     out = {}
 
-    def entry(name, sweeps, elements, ops, note, fl):
+    def entry(name, sweeps, elements, ops, note, fl, baseline=None):
         whole, sweep = time_sweeps(sweeps, 5, fl)
         out[name] = dict(elements_times_formats=elements, whole_path=dict(value=elements / whole / 1e6, unit=UNIT, ms=whole),
                          sweep_only=dict(value=elements / sweep / 1e6, unit=UNIT, ms=sweep), ops_per_element_n_step=ops,
                          frac_of_alu_peak=ops * elements / (sweep * 1e-3) / 1e12 / alu_peak, note=note)
+        if baseline is not None:          # the oracle, as it stands, on a small sample of this configuration (one host core)
+            n_el, sample, fn = baseline
+            t0 = time.perf_counter()
+            fn()
+            dt = time.perf_counter() - t0
+            out[name]["oracle_baseline"] = dict(value=n_el / dt / 1e9, unit=UNIT, cores=1, sample=sample, seconds=dt)
 
     # 1: single small layer, signed UE4M4, three ROM atoms
+    from tests import oracle_pipeline
+    import oracle
     L = I.config1(0)
     sw = LayerSweep(256, 1024, 128, I.scale_format("S1E4M4"), ["NF4", "SH4", "BOF4"], [], 0, device=dev)
+    L1 = L
     entry("config1", [(sw, L.W.to(dev), L.X.to(dev), True)], 256 * 1024, search_ops_n_step(6, 4, 0),
-          "256x1024, S1E4M4, NF4/SH4/BOF4 + negations, no DD atom; launch-latency sized (one wave of 32 CTAs)", flush)
+          "256x1024, S1E4M4, NF4/SH4/BOF4 + negations, no DD atom; launch-latency sized (one wave of 32 CTAs)", flush,
+          baseline=(256 * 1024, "the whole layer, whole pipeline",
+                    lambda: oracle_pipeline.run(L1, I.scale_format("S1E4M4"), ["NF4", "SH4", "BOF4"], [], 0)))
     # 2: attention projection
     L = make_layer(0)
     sw = LayerSweep(CONFIG2["M"], CONFIG2["K"], CONFIG2["T"], I.scale_format("E5M6"), CONFIG2["rom"], CONFIG2["fp"], 8, device=dev)
+    L2 = I.Layer(L.W[:128].contiguous(), L.X)
     entry("config2", [(sw, L.W.to(dev), L.X.to(dev), True)], CONFIG2["M"] * CONFIG2["K"], search_ops_n_step(10, 4, 2),
-          "4096x4096, E5M6, 10 LUT candidates + E2M3/E4M3, all pairs; L2 flushed between passes", flush)
+          "4096x4096, E5M6, 10 LUT candidates + E2M3/E4M3, all pairs; L2 flushed between passes", flush,
+          baseline=(128 * CONFIG2["K"], "the first 128 of 4096 rows, whole pipeline",
+                    lambda: oracle_pipeline.run(L2, I.scale_format("E5M6"), CONFIG2["rom"], CONFIG2["fp"], 8)))
     del sw
     # 3: the seven layers of one 7B-shaped transformer block, FP6 per block against FP8 per layer (singles only)
     fmt = I.scale_format("UE4M4")
@@ -260,8 +274,14 @@ def per_config_table(dev, alu_peak, flush):
             sw = own[(M, K)] = LayerSweep(M, K, 512, fmt, [], fp, 0, device=dev)
         sweeps.append((sw, Lw.W, Lw.X, True))
         elements += M * K
+    L3 = I.config3_layer(0, 0, 4, rows=128)
+
+    def oracle3():
+        c = oracle.channel_norms(L3.X.numpy())
+        oracle.pair_search(L3.W, c, fmt, [I.fp_atom(f) for f in fp])
     entry("config3", sweeps, elements, search_ops_n_step(0, 4, 2),
-          "block 0 of 32 (seven layers, 218 M elements > L2), E2M3sUE4M4 vs E4M3^0: two FP singles, no pairs, no DD atom, pack of the FP6 single", None)
+          "block 0 of 32 (seven layers, 218 M elements > L2), E2M3sUE4M4 vs E4M3^0: two FP singles, no pairs, no DD atom, pack of the FP6 single", None,
+          baseline=(128 * L3.W.shape[1], "the first 128 rows of the 14336x4096 layer, channel norms and the search of both candidates", oracle3))
     del sweeps, own
     torch.cuda.empty_cache()
     # 4: the n = 5 MLP pair at both scale formats
@@ -275,8 +295,11 @@ def per_config_table(dev, alu_peak, flush):
             first = first or sw
             sweeps.append((sw, Lw.W, Lw.X, f == "UE4M4"))
             elements += M * K
+    L4 = I.config4_layer(0, 0, rows=128)
     entry("config4", sweeps, elements, search_ops_n_step(10, 5, 0),
-          "14336x4096 and 4096x14336 at UE4M4 and E5M6, 32-entry atoms, DD5 by 16 Lloyd iterations, all pairs", None)
+          "14336x4096 and 4096x14336 at UE4M4 and E5M6, 32-entry atoms, DD5 by 16 Lloyd iterations, all pairs", None,
+          baseline=(128 * L4.W.shape[1], "the first 128 rows of the 14336x4096 layer at UE4M4, whole pipeline",
+                    lambda: oracle_pipeline.run(L4, I.scale_format("UE4M4"), ["NF5", "SH5", "BOF5", "E2M2"], [], 16)))
     del sweeps
     torch.cuda.empty_cache()
     return out
