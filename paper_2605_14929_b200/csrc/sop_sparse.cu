@@ -12,23 +12,22 @@
 //   opq_mask_kernel     reads W once: per block the outlier mask (binary64 test w_i^2 g > m^2 sum w^2), W_out with
 //                       the outliers zeroed, the 16-bit mask, the tile count
 //   opq_write_kernel    reads the masks, and W only where a mask is set: records (column | bf16 bits << 16)
-//   wr_hist_kernel<P>   decodes the packed stream (scale word -> s_hat, codes -> table values), forms the residual
-//                       E = w - s_hat q (one rounding) and the metric |E| c_k, histograms 11 / 11 / 10 bits of the
-//                       inverted metric bits (three-pass radix select of the n_keep-th largest metric).  Pass -1 goes
-//                       first and histograms one value per block, the block's largest metric: at least n_keep
-//                       elements are as large as the n_keep-th largest block maximum, so the threshold lies in that
-//                       value's bin or an earlier one and pass 0 skips every element of a later bin (all but a few
-//                       per cent: shared-memory atomics on a handful of hot bins would otherwise dominate)
-//   wr_pick_kernel      after each pass: the bin that holds the rank, the prefix for the next pass
-//   wr_collect_kernel   second decode pass: every element whose bin is not later than that of the n_keep-th largest
-//                       block maximum goes to a candidate list (position, residual, metric): a fraction of a per cent
-//                       of the layer.  The threshold, the kept set (a bitmap), the largest kept |E| and the per-tile
-//                       counts then come from the list (wr_cand_hist_kernel, wr_mark_kernel);
-//                       the write pass decodes only the blocks that hold a kept entry.
-//   wr_hist_kernel<0,1,2>, wr_count_kernel, wr_write_kernel<.., false>
+//   wr_hist_kernel<-1>  first decode pass of the packed stream (scale word -> s_hat, codes -> table values, residual
+//                       E = w - s_hat q with one rounding, metric |E| c_k): histogram of one value per block, the
+//                       block's largest metric (top 11 bits of the inverted metric bits).  At least n_keep elements
+//                       are as large as the n_keep-th largest block maximum, so the threshold lies in that value's
+//                       bin or an earlier one
+//   wr_pick_kernel      after each histogram: the bin that holds the rank, the prefix for the next pass
+//   wr_collect_kernel   second decode pass: every element whose bin is not later than that bound goes to a candidate
+//                       list (position, residual, metric): a fraction of a per cent of the layer
+//   wr_cand_hist_kernel<0,1,2>, wr_mark_kernel
+//                       over the list: three-pass radix select (11 / 11 / 10 bits) of the n_keep-th largest metric,
+//                       then the kept set as one 16-bit mask per block, the per-tile counts and the largest kept |E|
+//   wr_map_write_kernel E3M4 codes of E / 2^e, records (column | code << 16): decodes only the blocks with a kept entry
+//   wr_hist_kernel<0,1,2>, wr_count_kernel, wr_write_kernel
 //                       the same steps as full decode passes: taken when the candidates do not fit their list (a
 //                       layer whose metrics are nearly all alike).  Both sets of launches are enqueued; the set
-//                       that is not needed returns at once (flag in the workspace, set on the device).
+//                       that is not needed returns at once (wr_mode_kernel sets the flag on the device).
 // The residual is never stored: decoding a block (2.6 bytes per element read) is cheaper than reading 4 bytes.
 #include <math.h>
 #include <string.h>
