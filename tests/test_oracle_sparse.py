@@ -254,3 +254,61 @@ def test_ties_at_the_threshold_all_enter_and_zero_residuals_never_do():
     assert np.array_equal(Wg.to(torch.float32).numpy(), lut[idx] * np.float32(0.25))
     z = oracle.wr_extract(Wg, c, fmt, a, 0, None, 0, use_sign=0, n_keep=7, want_resid=True)
     assert not z["resid"].any() and z["count"] == 0 and z["scale_exp"] == 0
+
+
+# ---------------------------------------------------------------- soft checks against the paper's claims
+
+def block_acos(W, What, c):
+    """Mean over blocks of the c-weighted cosine between w and its reconstruction (float64)."""
+    M, K = W.shape
+    w = W.astype(np.float64).reshape(M, K // 16, 16)
+    q = What.astype(np.float64).reshape(M, K // 16, 16)
+    cb = np.asarray(c, dtype=np.float64).reshape(1, K // 16, 16)
+    dot = (cb * w * q).sum(axis=2)
+    nw = (cb * w * w).sum(axis=2)
+    nq = (cb * q * q).sum(axis=2)
+    cos = np.where((nw > 0) & (nq > 0), dot / np.sqrt(np.where(nw * nq > 0, nw * nq, 1.0)), np.where((nw == 0) & (nq == 0), 1.0, 0.0))
+    return float(cos.mean())
+
+
+def test_wr_gains_a_few_ppm_of_acos_at_four_bits():
+    # the paper: sparsity 0.001 costs about 0.032 bpw and typically gains 5-15 ppm of pair-mean ACos at 4-bit codebooks
+    L = I.student_layer(23, 0, 96, 1024, 256, 5.0, channel_sigma=0.5)
+    c = oracle.channel_norms(L.X.numpy())
+    fmt = I.scale_format("S1E5M5")
+    a, b = I.rom_atom("NF4"), I.rom_atom("SH4")
+    n_keep = int(np.ceil(0.001 * 96 * 1024))
+    wr = oracle.wr_extract(L.W, c, fmt, a, 0, b, 0, use_sign=1, n_keep=n_keep, want_resid=True)
+    Wf = L.W.to(torch.float32).numpy()
+    What = Wf.astype(np.float64) - wr["resid"].astype(np.float64)
+    before = block_acos(Wf, What, c)
+    corrected = What.copy()
+    rs = wr["row_start"]
+    for r in range(96):
+        for rec in wr["records"][rs[r]:rs[r + 1]]:
+            corrected[r, rec & 0xFFFF] += e3m4_value(int(rec >> 16)) * 2.0 ** wr["scale_exp"]
+    after = block_acos(Wf, corrected, c)
+    gain_ppm = (after - before) * 1e6
+    assert 0.997 < before < 0.9995                 # the paper's typical range of 4-bit pairs is [0.997, 0.999]
+    assert 1.0 < gain_ppm < 200.0                  # a few ppm to a few tens of ppm
+    assert 32.0 * wr["count"] / (96 * 1024) == pytest.approx(0.032, abs=0.002)
+
+
+def test_opq_makes_the_codebook_input_easier():
+    # with the outliers stored exactly, the rest of the block concentrates inside the table's range: the best pair's
+    # ACos on the zeroed weights is above that on the original ones, and the stream costs 32 bits per outlier
+    L = I.laplace_outlier_layer(29, 0, 64, 1024, 128, frac=0.003)
+    c = oracle.channel_norms(L.X.numpy())
+    fmt = I.scale_format("S1E5M5")
+    atoms = I.alphabet(["NF4", "SH4", "BOF4"])
+    m = oracle.opq_threshold(0.92, 16)
+    o = oracle.opq_extract(L.W, m)
+    W2 = torch.from_numpy(o["W_out"].view(np.int16).copy()).view(torch.bfloat16)
+    r0 = oracle.pair_search(L.W, c, fmt, atoms)
+    r1 = oracle.pair_search(W2, c, fmt, atoms)
+    best0 = r0["pair"]["acos"][r0["best"][0], r0["best"][1]]
+    best1 = r1["pair"]["acos"][r1["best"][0], r1["best"][1]]
+    assert best1 > best0
+    rate = o["count"] / (64 * 1024)
+    assert 0.003 <= rate < 0.05                    # at least the planted 8-sigma spikes
+    assert 32.0 * rate < 1.6
