@@ -148,7 +148,11 @@ class LayerSweep:
         # the two sparse side streams (both off unless asked for)
         self.opq_m = B.opq_threshold(opq_q, 16) if opq_q is not None else None
         self.wr_keep = int(math.ceil(wr_sigma * M * K)) if wr_sigma is not None else 0
-        if self.opq_m is not None:
+        if self.opq_m is not None and share is not None and getattr(share, "opq_m", None) == self.opq_m:
+            # the outlier stream does not depend on the scale format: the sharing sweep's is this sweep's too
+            self.W_opq, self.opq_row_start, self.opq_records = share.W_opq, share.opq_row_start, share.opq_records
+            self.opq_count, self.ws_opq = share.opq_count, share.ws_opq
+        elif self.opq_m is not None:
             cap = opq_capacity if opq_capacity is not None else max(1024, M * K // 32)    # 3 % of the elements: six times the Gaussian rate at q = 0.92
             self.W_opq = torch.empty((M, K), dtype=torch.bfloat16, device=d)
             self.opq_row_start = torch.zeros(M + 1, dtype=torch.int32, device=d)
@@ -171,8 +175,8 @@ class LayerSweep:
     def run(self, W: torch.Tensor, X: torch.Tensor, stream=None, norms: bool = True, reuse_prepass: bool = False,
             codes: Optional[torch.Tensor] = None, words: Optional[torch.Tensor] = None) -> None:
         """One pass of the whole hot path over device-resident W [M, K] bf16 and X [T, K] fp32.  ``norms`` =
-        False skips the channel norms: they do not depend on the scale format, so a sweep that shares the
-        buffers of another one (same layer, other format) uses the norms that one has just computed.
+        False skips the channel norms (and the outlier extraction, if any): they do not depend on the scale format, so
+        a sweep that shares the buffers of another one (same layer, other format) uses what that one has just computed.
         ``reuse_prepass``: the same holds for the exponent histogram of the block scales behind the per-layer
         shift: the search takes it from the shared workspace as the sweep of this layer at the previous format
         left it, and only derives this format's shifts.  ``codes`` / ``words``: buffers of the sizes of ``self.codes`` /
@@ -184,9 +188,10 @@ class LayerSweep:
             B.sop_channel_norms(X, self.c, self.ws_norm, stream)
             n += 2
         if self.opq_m is not None:
-            B.sop_opq_extract(W, self.opq_m, self.W_opq, self.opq_row_start, self.opq_records, self.opq_count, self.ws_opq, stream)
+            if norms:          # like the norms, the outlier stream of a layer is extracted once for all its scale formats
+                B.sop_opq_extract(W, self.opq_m, self.W_opq, self.opq_row_start, self.opq_records, self.opq_count, self.ws_opq, stream)
+                n += 3
             W = self.W_opq
-            n += 3
         if self.iters > 0:
             # every fixed candidate and every table entry among them; the best single of the result is FMTa
             B.sop_pair_search(W, self.c, self.fmt_c, self.atoms_c, self.pair_table, self.signed_table, self.rom_result,
@@ -393,7 +398,7 @@ class LayerSetSweep:
     of the new columns and the pack."""
 
     def __init__(self, shapes: Sequence[tuple], fmts: Sequence[I.ScaleFormat], rom: Sequence[str], fp: Sequence[str] = (),
-                 lloyd_iters: int = 8, device="cuda"):
+                 lloyd_iters: int = 8, device="cuda", opq_q: Optional[float] = None, wr_sigma: Optional[float] = None):
         self.shapes, self.fmts = [tuple(s) for s in shapes], list(fmts)
         self.dev = torch.device(device)
         owner = {}
@@ -401,7 +406,7 @@ class LayerSetSweep:
         for shape in self.shapes:
             row = []
             for fmt in self.fmts:
-                sw = LayerSweep(*shape, fmt, rom, fp, lloyd_iters, device=device, share=owner.get(shape))
+                sw = LayerSweep(*shape, fmt, rom, fp, lloyd_iters, device=device, share=owner.get(shape), opq_q=opq_q, wr_sigma=wr_sigma)
                 owner.setdefault(shape, sw)
                 row.append(sw)
             self.sweeps.append(row)

@@ -256,3 +256,35 @@ def test_wr_when_the_candidates_do_not_fit_their_list():
     sw, out, got = run_wr(L1, fmt, ["NF4", "SH4"], 100, None)
     want = oracle_wr(L1, fmt, out, sw, 100)
     assert got["count"] == want["count"] == M * K and np.array_equal(got["records"], want["records"])
+
+
+def test_layer_set_with_both_streams_shares_the_outlier_stream_between_formats():
+    """A layer set at two scale formats with both streams: the outlier stream of a layer is extracted once (it does not
+    depend on the scale format) and every (layer, format) correction equals that of a sweep of its own."""
+    from paper_2605_14929_b200.pipeline import LayerSetSweep
+    d = dev()
+    shapes = [(48, 512, 64), (32, 768, 64), (48, 512, 64)]
+    fmts = [I.scale_format("E5M6"), I.scale_format("UE4M4")]
+    rom = ["NF4", "SH4", "BOF4"]
+    layers = [I.laplace_outlier_layer(80 + i, i, M, K, T) for i, (M, K, T) in enumerate(shapes)]
+    sset = LayerSetSweep(shapes, fmts, rom, [], 3, device=d, opq_q=0.92, wr_sigma=0.002)
+    dev_layers = [(L.W.to(d), L.X.to(d)) for L in layers]
+    got = {}
+    for li, (row, (W, X)) in enumerate(zip(sset.sweeps, dev_layers)):       # layer by layer: the formats of a layer share its buffers
+        for f, sw in enumerate(row):
+            sw.run(W, X, norms=(f == 0), reuse_prepass=(f > 0))
+            got[(li, f)] = (sw.outputs(), sw.sparse_outputs())
+    for li, L in enumerate(layers):
+        M, K, T = shapes[li]
+        for f, fmt in enumerate(fmts):
+            own = LayerSweep(M, K, T, fmt, rom, [], 3, device=d, opq_q=0.92, wr_sigma=0.002)
+            own.run(*dev_layers[li])
+            wo, ws = own.outputs(), own.sparse_outputs()
+            go, gs = got[(li, f)]
+            assert np.array_equal(gs["opq"]["records"], ws["opq"]["records"]) and gs["opq"]["count"] == ws["opq"]["count"] > 0
+            assert torch.equal(go.codes, wo.codes) and torch.equal(go.words, wo.words)
+            assert gs["wr"]["count"] == ws["wr"]["count"] and gs["wr"]["scale_exp"] == ws["wr"]["scale_exp"]
+            assert np.array_equal(gs["wr"]["records"], ws["wr"]["records"]) and np.array_equal(gs["wr"]["row_start"], ws["wr"]["row_start"])
+    # the whole set in one pass gives the last layer's results in the shared buffers, and runs without error
+    sset.run(dev_layers)
+    sset.check()
