@@ -288,3 +288,26 @@ def test_layer_set_with_both_streams_shares_the_outlier_stream_between_formats()
     # the whole set in one pass gives the last layer's results in the shared buffers, and runs without error
     sset.run(dev_layers)
     sset.check()
+
+
+def test_wr_with_dead_channels_zero_blocks_and_large_rows():
+    """Channels that never fire (c_k = 0: their residuals have no salience and are never kept), all-zero blocks, and
+    rows scaled by 2^12 and 2^-12 (residuals far from 1: the layer exponent follows the largest kept residual)."""
+    L = I.student_layer(31, 0, 24, 512, 64, 4.0)
+    Wf = L.W.to(torch.float32).numpy().copy()
+    Wf[3] *= 4096.0
+    Wf[7] *= 1.0 / 4096.0
+    Wf[5, 64:128] = 0.0
+    X = L.X.clone()
+    X[:, 16:48] = 0.0
+    X[:, 300] = 0.0
+    L2 = I.Layer(torch.from_numpy(Wf).to(torch.bfloat16), X)
+    fmt = I.scale_format("E5M6")
+    for n_keep in (5, 200, 24 * 512):
+        sw, out, got = run_wr(L2, fmt, ["NF4", "SH4"], n_keep, None, lloyd_iters=2)
+        want = oracle_wr(L2, fmt, out, sw, n_keep)
+        assert got["count"] == want["count"] and got["scale_exp"] == want["scale_exp"] > 0
+        assert np.array_equal(got["row_start"], want["row_start"]) and np.array_equal(got["records"], want["records"])
+        cols = got["records"] & 0xFFFF
+        assert not np.isin(cols, np.r_[16:48, 300]).any()              # dead channels are never kept
+    assert got["count"] < 24 * 512                                       # ... even when everything is asked for
