@@ -1,7 +1,8 @@
-// sop_pack: materialise the chosen codebook(s): per block re-evaluate the (up to four) candidates
-// with the same arithmetic as the sweep, keep the best, and emit 2n bytes of codes plus one b-bit
-// scale word (sign, exponent, mantissa, selector).  HBM-bound: reads W once, writes ~n/8 + b/128
-// bytes per element.
+// sop_pack: materialise the chosen codebook(s): per block the best of the (up to four) candidates -- read off
+// the per-block cosines of the sweep where they are given, else re-evaluated with the same arithmetic -- is
+// encoded: 2n bytes of codes plus one b-bit scale word (sign, exponent, mantissa, selector).  Reads W once,
+// writes ~n/8 + b/128 bytes per element; bound by instruction issue (the encode), not by bytes.  Table codes
+// come from a uniform cell grid on u where the table allows it, else from a binary search over the thresholds.
 #include <string.h>
 
 #include "sop_device.cuh"

@@ -4,6 +4,8 @@
 //                    for every scale class that needs an F_layer search, and max|W|   (HBM-bound);
 //                    the CTA that finishes last derives the F_layer shift k* per class from the
 //                    histogram and the layer power-of-two scale for "^0" candidates.
+//   kselect_kernel   that last step alone: the shifts of another scale format from the histogram a prepass of the
+//                    same layer left in the workspace (SOP_SEARCH_REUSE_PREPASS).
 //   sweep_kernel     persistent, one thread per 16-element block: evaluates every candidate of the call
 //                    in registers (cell-table lookup of the reconstruction value, packed f32x2
 //                    fused multiply-adds for the block metric, fixed quad-tree order) and writes
@@ -13,7 +15,8 @@
 //                    the table entries: a warp owns a few "tasks" (one anchor column against up to
 //                    four partner columns, so five columns are fetched for up to five entries), a
 //                    lane owns eight blocks of every tile, the sums of those eight are fp32 and go
-//                    to FP64 accumulators after every tile.
+//                    to FP64 accumulators after every tile (two tiles per step where the shared
+//                    memory allows: the accumulators are then touched once per sixteen blocks).
 //                    The CTA that finishes last adds the per-CTA partials in a fixed order
 //                    (deterministic), writes the tables and picks the best pair / best single.
 #include <math.h>
