@@ -329,3 +329,11 @@ def test_config5_attention_layer_with_both_sparse_streams_in_full(B):
     assert sp["wr"]["count"] == w["count"] >= sw.wr_keep and sp["wr"]["scale_exp"] == w["scale_exp"]
     assert np.float32(sp["wr"]["tau"]).view(np.uint32) == np.float32(w["tau"]).view(np.uint32)
     assert np.array_equal(sp["wr"]["row_start"], w["row_start"]) and np.array_equal(sp["wr"]["records"], w["records"])
+
+
+def test_config5_attention_layer_at_the_other_six_scale_formats(B):
+    # the 8192 x 8192 layer in full at the six scale formats of the paper's table that the largest layers above do not
+    # take: the oracle's passes for the formats run side by side on the host
+    got = _both_formats(B, lambda: I.config5_layer(0, 0, 0, device="cuda"), ["E4M3", "UE4M6", "E4M5", "UE5M7", "E4M7", "E8M7"],
+                        ["NF4", "SH4", "BOF4", "Split87"], 8)
+    assert len(got) == 6
