@@ -386,6 +386,18 @@ def run_gpu(args) -> None:
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    # the library is built in-tree beforehand; where it is missing (a fresh checkout) local rank 0 builds it with nvcc and
+    # the other ranks wait for the file -- there is no other path: without it B.lib() raises
+    from paper_2605_14929_b200 import build as libbuild
+    if not os.path.exists(libbuild.LIB):
+        if local == 0:
+            libbuild.build()
+        else:
+            for _ in range(600):
+                if os.path.exists(libbuild.LIB):
+                    break
+                time.sleep(1.0)
+            time.sleep(2.0)
     B.lib()
 
     small = args.workload == "layer"                              # the profiling case: one layer, one format
